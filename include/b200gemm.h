@@ -1,0 +1,163 @@
+/*
+ * b200gemm -- dense GEMM  C = A * B^T  on one NVIDIA B200 (sm_100a) in the three
+ * precisions of the multi-precision tensor-core study this library follows.
+ *
+ * Operation (paper Sec. II-A: the tensor-core operation D = A*B + C, used with a
+ * zero initial accumulator; Listing 2(c): ".row.col" operands; Listing 1: row i
+ * of A starts i*K elements after the base, i*K/2 bytes for 4-bit data; Sec. VI:
+ * INT32 results, no dequantisation or scaling inside the kernel):
+ *
+ *     C[i][j] = sum_{k=0}^{K-1} a(i,k) * b(j,k)      0 <= i < M, 0 <= j < N
+ *
+ * Layouts, common to all entry points:
+ *     A : M rows, K elements each, row-major, leading dimension K  (device memory)
+ *     B : N rows, K elements each, K contiguous ("K-major"), leading dimension K
+ *     C : M x N row-major, leading dimension N, 32-bit elements, OVERWRITTEN
+ *         (no alpha/beta; previous contents are ignored)
+ *
+ * Every pointer is a DEVICE pointer owned by the caller; it must stay valid
+ * until `stream` has passed the call.  Calls are asynchronous on `stream` and
+ * never synchronise.  Argument errors are reported by the return value and
+ * enqueue nothing.  M and N are arbitrary; K carries an alignment rule because
+ * operand rows are fetched by TMA (row pitch must be a multiple of 16 bytes).
+ *
+ * All functions return GEMM_OK (0) or a negative GEMM_ERR_* code.
+ * A process may call from several host threads; calls that share a stream are
+ * ordered by it.
+ */
+#ifndef B200GEMM_H_
+#define B200GEMM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Opaque CUDA stream handle (a cudaStream_t); 0 / NULL is the default stream. */
+typedef struct CUstream_st* gemm_stream_t;
+
+enum {
+  GEMM_OK = 0,
+  GEMM_ERR_INVALID_ARG = -1,  /* null pointer, non-positive dimension, unknown enum value */
+  GEMM_ERR_MISALIGNED = -2,   /* base pointer or K violates the alignment rule */
+  GEMM_ERR_K_TOO_LARGE = -3,  /* integer paths: K > 131071, an INT32 result could overflow */
+  GEMM_ERR_UNSUPPORTED_DEVICE = -4, /* current device is not compute capability 10.x */
+  GEMM_ERR_CUDA = -5,         /* a CUDA runtime/driver call failed (see gemm_last_cuda_error) */
+  GEMM_ERR_WORKSPACE = -6,    /* caller-supplied workspace too small or misaligned */
+  GEMM_ERR_TOO_LARGE = -7     /* problem exceeds a fixed capacity of the entry point */
+};
+
+enum { GEMM_PREC_FP16 = 0, GEMM_PREC_S8 = 1, GEMM_PREC_S4 = 2 };
+
+/*
+ * FP16 inputs, FP32 accumulate, FP32 output (the study's FP16 family, Table VI:
+ * f16 operands with f32 accumulators; Sec. IV Run 1 counts a 4-byte C).
+ * A, B: IEEE binary16.  Accumulation order inside the tensor core is hardware
+ * defined; results satisfy |C - exact| <= 1e-4 * sum_k|a*b| + 1e-6.
+ * Alignment: A, B, C 16-byte aligned; K % 8 == 0.
+ */
+int gemm_fp16(int M, int N, int K, const void* A, const void* B, float* C, gemm_stream_t stream);
+
+/*
+ * Signed 8-bit inputs, INT32 accumulate and output, exact (the study's INT8
+ * family, Sec. IV Run 2).  Alignment: A, B, C 16-byte aligned; K % 16 == 0;
+ * K <= 131071 so that no INT32 sum can overflow.
+ */
+int gemm_s8(int M, int N, int K, const int8_t* A, const int8_t* B, int32_t* C,
+            gemm_stream_t stream);
+
+/*
+ * Signed 4-bit inputs, INT32 accumulate and output, exact (the study's INT4
+ * family, Sec. IV Runs 3-4; Listing 2(c) ".s4.s4 -> .s32").  A: M rows of K/2
+ * bytes, B: N rows of K/2 bytes; element k of a row is bits [4*(k&1), 4*(k&1)+4)
+ * of byte k>>1 (low nibble first), two's complement.
+ *
+ * Blackwell's tcgen05.mma has no 4-bit integer kind, so the operands are first
+ * sign-extended to int8 by a streaming pre-pass into a workspace of
+ * gemm_s4_workspace_bytes(M, N, K) bytes and then multiplied by the INT8
+ * kernel.  gemm_s4 keeps one grow-only workspace per device inside the library:
+ * the first call on a device (and any call that needs a larger one) allocates
+ * with cudaMalloc, which synchronises the device; the buffer is reused by later
+ * calls, so concurrent gemm_s4 calls on different streams of one device must be
+ * ordered by the caller.  Use gemm_s4_ws to supply the workspace yourself.
+ * Alignment: A, B, C 16-byte aligned; K % 32 == 0; K <= 131071.
+ */
+int gemm_s4(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t* C,
+            gemm_stream_t stream);
+
+/* Bytes of device scratch gemm_s4_ws needs for this problem (0 on bad sizes). */
+size_t gemm_s4_workspace_bytes(int M, int N, int K);
+
+/*
+ * gemm_s4 with caller-owned scratch: `workspace` is a device buffer of at least
+ * gemm_s4_workspace_bytes(M, N, K) bytes, 256-byte aligned, which the call
+ * overwrites; it must not be shared by calls that may overlap on the GPU.
+ * Allocates nothing.
+ */
+int gemm_s4_ws(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t* C,
+               void* workspace, size_t workspace_bytes, gemm_stream_t stream);
+
+/*
+ * Frees the per-device workspaces held for gemm_s4 (synchronises).  Optional;
+ * they are otherwise released when the process exits.
+ */
+int gemm_release_workspaces(void);
+
+/*
+ * The INT4 pre-pass on its own (Sec. IV Run 3 discusses why the 4-bit path's
+ * cost is the cost of getting nibbles into the MMA's operand format): expands
+ * `rows` rows of K packed signed 4-bit values (K/2 bytes per row, pitch K/2)
+ * into int8, one value per byte, row pitch `out_pitch` bytes (>= K, multiple of
+ * 16; bytes K..out_pitch-1 of each row are set to zero).  K % 32 == 0,
+ * `packed` and `out` 16-byte aligned.
+ */
+int gemm_unpack_s4(int rows, int K, const uint8_t* packed, int8_t* out, size_t out_pitch,
+                   gemm_stream_t stream);
+
+/*
+ * Measurement aid (Sec. III-B profiles every kernel against the hardware's
+ * limits): runs `iters` back-to-back tcgen05.mma instructions of the production
+ * tile shape per SM on shared-memory operands that are never reloaded, on
+ * every SM, and adds the operation count it performed to *ops_out (host
+ * pointer).  Time it with events on `stream` to get the MMA-issue-only peak of
+ * the given precision (GEMM_PREC_FP16 or GEMM_PREC_S8).
+ */
+int gemm_mma_peak_probe(int precision, int iters, double* ops_out, gemm_stream_t stream);
+
+/*
+ * Writes a human-readable description of the tile configuration the selector
+ * picks for this problem ("BM=128 BN=256 stages=4 ...") into buf (NUL
+ * terminated, truncated to len).  Host only, no GPU work.
+ */
+int gemm_query_config(int precision, int M, int N, int K, char* buf, int len);
+
+/*
+ * Overrides the selector for later calls from this process: tile width BN
+ * (0 = automatic) and raster band height in tiles (0 = automatic).  For
+ * ablation sweeps.  Returns GEMM_ERR_INVALID_ARG for a width that is not built.
+ */
+int gemm_set_config_override(int bn, int group_m);
+
+/*
+ * Kernels never spin forever: a barrier wait that exceeds its limit makes the
+ * kernel record a non-zero code and drain.  This reads that code for the
+ * current device (synchronises the device) and clears it.  0 = no event;
+ * 1/2/3 = producer / MMA / epilogue wait expired.
+ */
+int gemm_last_device_status(void);
+
+/* cudaError_t value of the last failed CUDA call made by this library, or 0. */
+int gemm_last_cuda_error(void);
+
+/* Text for a GEMM_* return code. */
+const char* gemm_status_string(int status);
+
+/* Library version: major * 1000 + minor. */
+int gemm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* B200GEMM_H_ */

@@ -77,6 +77,8 @@ def _check(rc):
         raise ValueError("oracle: bad argument (shape, index or odd K for int4)")
     if rc == -2:
         raise ValueError("oracle: non-finite fp16 input")
+    if rc == -3:
+        raise MemoryError("oracle: out of memory")
     if rc != 0:
         raise RuntimeError("oracle: error %d" % rc)
 

@@ -29,10 +29,12 @@
 #include <stdint.h>
 #include <stddef.h>
 #include <math.h>
+#include <stdlib.h>
 
 #define ORACLE_OK 0
 #define ORACLE_BAD_ARG -1
 #define ORACLE_NONFINITE -2
+#define ORACLE_NO_MEMORY -3
 
 /* IEEE binary16 -> double by bit fields.  Returns 0 and sets *ok = 0 for
  * infinities and NaNs: the GEMM inputs are finite by construction. */
@@ -79,6 +81,25 @@ static int bad_args(int M, int N, int K, const void *A, const void *B,
     return 0;
 }
 
+/* Step 1 of the FP16 path: decode a whole operand once.  Every binary16 value
+ * is exactly representable in binary32, so the decoded copy loses nothing and
+ * halves the scratch memory; products and sums are formed in fp64 below. */
+static float *decode_half_matrix(const uint16_t *X, size_t count, int *ok_out)
+{
+    float *out = (float *)malloc(count * sizeof(float));
+    int bad = 0;
+    if (!out)
+        return NULL;
+#pragma omp parallel for schedule(static) reduction(|:bad)
+    for (long long t = 0; t < (long long)count; ++t) {
+        int ok = 1;
+        out[t] = (float)half_bits_to_double(X[t], &ok);
+        if (!ok) bad |= 1;
+    }
+    if (bad) *ok_out = 0;
+    return out;
+}
+
 /* FP16 inputs, fp64 accumulation.  C gets the sums, S (may be NULL) gets
  * sum_k |a*b|, the quantity the FP16 error bound is stated in.  Every
  * fp16 x fp16 product has at most 22 significant bits and is exact in fp64. */
@@ -86,31 +107,37 @@ int oracle_gemm_fp16(int M, int N, int K, const uint16_t *A, const uint16_t *B,
                      const int32_t *rows, int nr, const int32_t *cols, int nc,
                      double *C, double *S)
 {
-    int bad = 0;
+    int ok = 1;
+    float *a32, *b32;
     if (bad_args(M, N, K, A, B, rows, nr, cols, nc, C))
         return ORACLE_BAD_ARG;
     if (!rows) nr = M;
     if (!cols) nc = N;
-#pragma omp parallel for schedule(static) reduction(|:bad)
+    a32 = decode_half_matrix(A, (size_t)M * K, &ok);
+    b32 = decode_half_matrix(B, (size_t)N * K, &ok);
+    if (!a32 || !b32) {
+        free(a32);
+        free(b32);
+        return ORACLE_NO_MEMORY;
+    }
+#pragma omp parallel for schedule(static)
     for (int r = 0; r < nr; ++r) {
         int i = rows ? rows[r] : r;
         for (int c = 0; c < nc; ++c) {
             int j = cols ? cols[c] : c;
             double acc = 0.0, mag = 0.0;
-            int ok = 1;
             for (int k = 0; k < K; ++k) {
-                double a = half_bits_to_double(A[(size_t)i * K + k], &ok);
-                double b = half_bits_to_double(B[(size_t)j * K + k], &ok);
-                double p = a * b;
+                double p = (double)a32[(size_t)i * K + k] * (double)b32[(size_t)j * K + k];
                 acc += p;
                 mag += fabs(p);
             }
-            if (!ok) bad |= 1;
             C[(size_t)r * nc + c] = acc;
             if (S) S[(size_t)r * nc + c] = mag;
         }
     }
-    return bad ? ORACLE_NONFINITE : ORACLE_OK;
+    free(a32);
+    free(b32);
+    return ok ? ORACLE_OK : ORACLE_NONFINITE;
 }
 
 /* Signed 8-bit inputs, exact int64 sums (the caller checks the int32 range). */

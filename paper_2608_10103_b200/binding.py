@@ -1,0 +1,205 @@
+"""ctypes binding of libb200gemm.so: argument marshalling only.
+
+Every function here has the name and meaning of the C entry point it calls
+(see include/b200gemm.h); tensors are torch CUDA tensors used purely as device
+memory, `stream` is a torch.cuda.Stream (default: the current stream).  There
+is no fallback: if the shared library is missing or an entry point fails, an
+exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+GEMM_OK = 0
+PREC_FP16, PREC_S8, PREC_S4 = 0, 1, 2
+PRECISION_ID = {"fp16": PREC_FP16, "s8": PREC_S8, "s4": PREC_S4}
+
+EXPORTS = (
+    "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
+    "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
+    "gemm_set_config_override", "gemm_last_device_status", "gemm_last_cuda_error",
+    "gemm_status_string", "gemm_version",
+)
+
+_lib = None
+
+
+class GemmError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        text = lib().gemm_status_string(code).decode()
+        extra = ""
+        if code == -5:
+            extra = " (cudaError %d)" % lib().gemm_last_cuda_error()
+        super().__init__("%s failed: %s [%d]%s" % (where, text, code, extra))
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the shared library (never builds it implicitly)."""
+    global _lib
+    if _lib is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise ImportError(
+                "%s not found: build it with `python -m paper_2608_10103_b200.build`" % path)
+        L = ctypes.CDLL(path)
+        vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.gemm_fp16.argtypes = [i, i, i, vp, vp, vp, vp]
+        L.gemm_s8.argtypes = [i, i, i, vp, vp, vp, vp]
+        L.gemm_s4.argtypes = [i, i, i, vp, vp, vp, vp]
+        L.gemm_s4_ws.argtypes = [i, i, i, vp, vp, vp, vp, sz, vp]
+        L.gemm_s4_workspace_bytes.argtypes = [i, i, i]
+        L.gemm_s4_workspace_bytes.restype = sz
+        L.gemm_unpack_s4.argtypes = [i, i, vp, vp, sz, vp]
+        L.gemm_mma_peak_probe.argtypes = [i, i, ctypes.POINTER(ctypes.c_double), vp]
+        L.gemm_query_config.argtypes = [i, i, i, i, ctypes.c_char_p, i]
+        L.gemm_set_config_override.argtypes = [i, i]
+        L.gemm_status_string.argtypes = [i]
+        L.gemm_status_string.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            fn = getattr(L, name)
+            if name not in ("gemm_s4_workspace_bytes", "gemm_status_string"):
+                fn.restype = i
+        _lib = L
+    return _lib
+
+
+def _stream_handle(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _check(rc: int, where: str):
+    if rc != GEMM_OK:
+        raise GemmError(rc, where)
+
+
+def _dev_ptr(t: torch.Tensor, dtype, what: str) -> int:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError("%s must be a CUDA tensor" % what)
+    if t.dtype != dtype:
+        raise TypeError("%s must have dtype %s, got %s" % (what, dtype, t.dtype))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % what)
+    return t.data_ptr()
+
+
+def _out(C, M, N, dtype, device):
+    if C is None:
+        C = torch.empty((M, N), dtype=dtype, device=device)
+    elif tuple(C.shape) != (M, N):
+        raise ValueError("C must have shape (%d, %d)" % (M, N))
+    return C
+
+
+def gemm_fp16(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor | None = None, stream=None):
+    """C[M,N] (float32) = A[M,K] (float16) @ B[N,K]^T (float16)."""
+    M, K = A.shape
+    N, Kb = B.shape
+    if K != Kb:
+        raise ValueError("A and B disagree on K")
+    C = _out(C, M, N, torch.float32, A.device)
+    _check(lib().gemm_fp16(M, N, K, _dev_ptr(A, torch.float16, "A"), _dev_ptr(B, torch.float16, "B"),
+                           _dev_ptr(C, torch.float32, "C"), _stream_handle(stream)), "gemm_fp16")
+    return C
+
+
+def gemm_s8(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor | None = None, stream=None):
+    """C[M,N] (int32) = A[M,K] (int8) @ B[N,K]^T (int8), exact."""
+    M, K = A.shape
+    N, Kb = B.shape
+    if K != Kb:
+        raise ValueError("A and B disagree on K")
+    C = _out(C, M, N, torch.int32, A.device)
+    _check(lib().gemm_s8(M, N, K, _dev_ptr(A, torch.int8, "A"), _dev_ptr(B, torch.int8, "B"),
+                         _dev_ptr(C, torch.int32, "C"), _stream_handle(stream)), "gemm_s8")
+    return C
+
+
+def gemm_s4(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor | None = None, stream=None):
+    """C[M,N] (int32) = A @ B^T for packed signed 4-bit operands: A is (M, K/2)
+    uint8, B is (N, K/2) uint8, low nibble first."""
+    M, Kh = A.shape
+    N, Khb = B.shape
+    if Kh != Khb:
+        raise ValueError("A and B disagree on K")
+    C = _out(C, M, N, torch.int32, A.device)
+    _check(lib().gemm_s4(M, N, 2 * Kh, _dev_ptr(A, torch.uint8, "A"), _dev_ptr(B, torch.uint8, "B"),
+                         _dev_ptr(C, torch.int32, "C"), _stream_handle(stream)), "gemm_s4")
+    return C
+
+
+def gemm_s4_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(lib().gemm_s4_workspace_bytes(M, N, K))
+
+
+def gemm_s4_ws(A: torch.Tensor, B: torch.Tensor, workspace: torch.Tensor,
+               C: torch.Tensor | None = None, stream=None):
+    """gemm_s4 with caller-owned scratch (a uint8 CUDA tensor)."""
+    M, Kh = A.shape
+    N, Khb = B.shape
+    if Kh != Khb:
+        raise ValueError("A and B disagree on K")
+    C = _out(C, M, N, torch.int32, A.device)
+    _check(lib().gemm_s4_ws(M, N, 2 * Kh, _dev_ptr(A, torch.uint8, "A"),
+                            _dev_ptr(B, torch.uint8, "B"), _dev_ptr(C, torch.int32, "C"),
+                            _dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel(),
+                            _stream_handle(stream)), "gemm_s4_ws")
+    return C
+
+
+def gemm_unpack_s4(packed: torch.Tensor, out: torch.Tensor | None = None, stream=None):
+    """(rows, K/2) uint8 packed nibbles -> (rows, K) int8."""
+    rows, Kh = packed.shape
+    K = 2 * Kh
+    if out is None:
+        out = torch.empty((rows, K), dtype=torch.int8, device=packed.device)
+    _check(lib().gemm_unpack_s4(rows, K, _dev_ptr(packed, torch.uint8, "packed"),
+                                _dev_ptr(out, torch.int8, "out"), out.stride(0),
+                                _stream_handle(stream)), "gemm_unpack_s4")
+    return out
+
+
+def gemm_release_workspaces():
+    _check(lib().gemm_release_workspaces(), "gemm_release_workspaces")
+
+
+def gemm_mma_peak_probe(precision: str, iters: int, stream=None) -> float:
+    """Launches the MMA-only probe; returns the operation count it performs."""
+    ops = ctypes.c_double(0.0)
+    _check(lib().gemm_mma_peak_probe(PRECISION_ID[precision], iters, ctypes.byref(ops),
+                                     _stream_handle(stream)), "gemm_mma_peak_probe")
+    return ops.value
+
+
+def gemm_query_config(precision: str, M: int, N: int, K: int) -> str:
+    buf = ctypes.create_string_buffer(256)
+    _check(lib().gemm_query_config(PRECISION_ID[precision], M, N, K, buf, 256), "gemm_query_config")
+    return buf.value.decode()
+
+
+def gemm_set_config_override(bn: int = 0, group_m: int = 0):
+    _check(lib().gemm_set_config_override(bn, group_m), "gemm_set_config_override")
+
+
+def gemm_last_device_status() -> int:
+    return int(lib().gemm_last_device_status())
+
+
+def gemm_version() -> int:
+    return int(lib().gemm_version())
+
+
+def gemm(precision: str, A, B, C=None, stream=None):
+    """Dispatch by precision name ("fp16", "s8", "s4")."""
+    return {"fp16": gemm_fp16, "s8": gemm_s8, "s4": gemm_s4}[precision](A, B, C, stream)

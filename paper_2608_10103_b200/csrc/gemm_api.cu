@@ -1,0 +1,451 @@
+// C-ABI of the library: argument validation, tile selection, tensor-map
+// encoding and kernel launch.  See include/b200gemm.h for the contract.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "../../include/b200gemm.h"
+#include "gemm_kernel.cuh"
+#include "peak_probe.cuh"
+#include "unpack_s4.cuh"
+
+namespace b200gemm {
+namespace {
+
+constexpr int MAX_DEVICES = 64;
+constexpr int K_LIMIT_INT = 131071;  // 128*128*K and 16384*K stay below 2^31
+
+__device__ int g_device_status = 0;
+
+struct DeviceState {
+  bool ready = false;
+  int num_sms = 0;
+  int* status_ptr = nullptr;
+  void* s4_workspace = nullptr;
+  size_t s4_workspace_bytes = 0;
+  uint64_t attr_set = 0;  // bit i: dynamic-smem attribute set for kernel variant i
+};
+
+std::mutex g_mutex;
+DeviceState g_dev[MAX_DEVICES];
+int g_last_cuda_error = 0;
+int g_override_bn = 0;
+int g_override_group_m = 0;
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = static_cast<int>(e);
+  return GEMM_ERR_CUDA;
+}
+
+// Looks up (once per device) what every launch needs.  Call with the mutex held.
+int device_state(DeviceState** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= MAX_DEVICES) return GEMM_ERR_UNSUPPORTED_DEVICE;
+  DeviceState& s = g_dev[dev];
+  if (!s.ready) {
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (major != 10) return GEMM_ERR_UNSUPPORTED_DEVICE;
+    e = cudaDeviceGetAttribute(&s.num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&s.status_ptr), g_device_status);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (!g_encode) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult q;
+      e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+      if (e != cudaSuccess) return cuda_fail(e);
+      if (!fn || q != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported);
+      g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    s.ready = true;
+  }
+  *out = &s;
+  return GEMM_OK;
+}
+
+// Row-major 2-D tensor of `rows` x `cols` elements, pitch in bytes; the box is
+// box_rows rows of 128 bytes, written to shared memory with the 128-byte swizzle.
+int encode_operand_map(CUtensorMap* map, CUtensorMapDataType type, int elem_bytes, const void* ptr,
+                       uint64_t rows, uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {pitch_bytes};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(BK_BYTES / elem_bytes), box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(map, type, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda_error = static_cast<int>(cudaErrorInvalidValue);
+    return GEMM_ERR_CUDA;
+  }
+  return GEMM_OK;
+}
+
+// ------------------------------------------------------------------ selector
+struct TileConfig {
+  int bn;
+  int stages;
+  int group_m;
+};
+
+constexpr int kWidths[] = {256, 128, 64, 32};
+
+int stages_for(int bn) {
+  switch (bn) {
+    case 256: return 4;
+    case 128: return 6;
+    case 64: return 8;
+    default: return 8;
+  }
+}
+
+int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b); }
+
+// Picks the C-tile width.  The paper fixes one tiling for all sizes (Sec.
+// III-A); on 148 SMs small problems need narrower tiles to fill the machine.
+// Cost model: waves of CTAs x (tile width + a fixed per-tile overhead).
+TileConfig select_config(int M, int N, int num_sms) {
+  TileConfig best{256, 4, 16};
+  if (g_override_bn) {
+    best.bn = g_override_bn;
+  } else {
+    long long best_cost = -1;
+    for (int bn : kWidths) {
+      long long tiles = static_cast<long long>(ceil_div(M, BM)) * ceil_div(N, bn);
+      long long waves = (tiles + num_sms - 1) / num_sms;
+      long long cost = waves * (bn + 16);
+      if (best_cost < 0 || cost < best_cost) {
+        best_cost = cost;
+        best.bn = bn;
+      }
+    }
+  }
+  best.stages = stages_for(best.bn);
+  // Band height: make one wave of tiles roughly square in operand bytes.
+  int g = 16;
+  if (best.bn == 128) g = 12;
+  if (best.bn <= 64) g = 8;
+  if (g_override_group_m) g = g_override_group_m;
+  int tiles_m = ceil_div(M, BM);
+  if (g > tiles_m) g = tiles_m;
+  best.group_m = g;
+  return best;
+}
+
+template <int KIND, int BN, int STAGES>
+int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUtensorMap& tb,
+                   const GemmParams& p, int grid, cudaStream_t stream) {
+  using L = SmemLayout<BN, STAGES>;
+  auto kernel = gemm_kernel<KIND, BN, STAGES>;
+  if (!(s->attr_set & (1ull << variant))) {
+    cudaError_t e =
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
+    if (e != cudaSuccess) return cuda_fail(e);
+    s->attr_set |= 1ull << variant;
+  }
+  kernel<<<grid, NUM_THREADS, L::DYN_BYTES, stream>>>(ta, tb, p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return GEMM_OK;
+}
+
+// A, B already in the element type of KIND (fp16 or int8), pitches in bytes.
+template <int KIND>
+int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* B, size_t b_pitch,
+                void* C, cudaStream_t stream) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceState* s = nullptr;
+  int rc = device_state(&s);
+  if (rc != GEMM_OK) return rc;
+  constexpr int ELEM = (KIND == ptx::KIND_F16) ? 2 : 1;
+  const CUtensorMapDataType type =
+      (KIND == ptx::KIND_F16) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+  const TileConfig cfg = select_config(M, N, s->num_sms);
+
+  CUtensorMap ta, tb;
+  rc = encode_operand_map(&ta, type, ELEM, A, M, K, a_pitch, BM);
+  if (rc != GEMM_OK) return rc;
+  rc = encode_operand_map(&tb, type, ELEM, B, N, K, b_pitch, cfg.bn);
+  if (rc != GEMM_OK) return rc;
+
+  GemmParams p;
+  p.M = M;
+  p.N = N;
+  p.K = K;
+  p.tiles_m = ceil_div(M, BM);
+  p.tiles_n = ceil_div(N, cfg.bn);
+  p.group_m = cfg.group_m;
+  p.k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
+  p.c_vec_ok = (N % 4 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+  p.C = static_cast<uint32_t*>(C);
+  p.status = s->status_ptr;
+  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
+  const int grid = static_cast<int>(tiles < s->num_sms ? tiles : s->num_sms);
+
+  const int kbase = (KIND == ptx::KIND_F16) ? 0 : 8;
+  switch (cfg.bn) {
+    case 256: return launch_variant<KIND, 256, 4>(s, kbase + 0, ta, tb, p, grid, stream);
+    case 128: return launch_variant<KIND, 128, 6>(s, kbase + 1, ta, tb, p, grid, stream);
+    case 64: return launch_variant<KIND, 64, 8>(s, kbase + 2, ta, tb, p, grid, stream);
+    case 32: return launch_variant<KIND, 32, 8>(s, kbase + 3, ta, tb, p, grid, stream);
+    default: return GEMM_ERR_INVALID_ARG;
+  }
+}
+
+int check_common(int M, int N, int K, const void* A, const void* B, const void* C) {
+  if (M <= 0 || N <= 0 || K <= 0 || !A || !B || !C) return GEMM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) |
+       reinterpret_cast<uintptr_t>(C)) & 15)
+    return GEMM_ERR_MISALIGNED;
+  return GEMM_OK;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int launch_unpack(long long rows, int K, const uint8_t* packed, int8_t* out, size_t out_pitch,
+                  cudaStream_t stream) {
+  const long long chunks = rows * (K / 32);
+  long long blocks = (chunks + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  unpack_s4_kernel<<<static_cast<int>(blocks), 256, 0, stream>>>(
+      reinterpret_cast<const uint4*>(packed), out, rows, K / 32, static_cast<long long>(out_pitch));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return GEMM_OK;
+}
+
+int check_s4(int M, int N, int K, const void* A, const void* B, const void* C) {
+  int rc = check_common(M, N, K, A, B, C);
+  if (rc != GEMM_OK) return rc;
+  if (K % 32) return GEMM_ERR_MISALIGNED;
+  if (K > K_LIMIT_INT) return GEMM_ERR_K_TOO_LARGE;
+  return GEMM_OK;
+}
+
+}  // namespace
+}  // namespace b200gemm
+
+using namespace b200gemm;
+
+extern "C" {
+
+int gemm_fp16(int M, int N, int K, const void* A, const void* B, float* C, gemm_stream_t stream) {
+  int rc = check_common(M, N, K, A, B, C);
+  if (rc != GEMM_OK) return rc;
+  if (K % 8) return GEMM_ERR_MISALIGNED;
+  return launch_gemm<ptx::KIND_F16>(M, N, K, A, static_cast<size_t>(K) * 2, B,
+                                    static_cast<size_t>(K) * 2, C,
+                                    reinterpret_cast<cudaStream_t>(stream));
+}
+
+int gemm_s8(int M, int N, int K, const int8_t* A, const int8_t* B, int32_t* C,
+            gemm_stream_t stream) {
+  int rc = check_common(M, N, K, A, B, C);
+  if (rc != GEMM_OK) return rc;
+  if (K % 16) return GEMM_ERR_MISALIGNED;
+  if (K > K_LIMIT_INT) return GEMM_ERR_K_TOO_LARGE;
+  return launch_gemm<ptx::KIND_I8>(M, N, K, A, static_cast<size_t>(K), B, static_cast<size_t>(K), C,
+                                   reinterpret_cast<cudaStream_t>(stream));
+}
+
+size_t gemm_s4_workspace_bytes(int M, int N, int K) {
+  if (M <= 0 || N <= 0 || K <= 0) return 0;
+  return align_up(static_cast<size_t>(M) * K, 256) + align_up(static_cast<size_t>(N) * K, 256);
+}
+
+int gemm_s4_ws(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t* C,
+               void* workspace, size_t workspace_bytes, gemm_stream_t stream) {
+  int rc = check_s4(M, N, K, A, B, C);
+  if (rc != GEMM_OK) return rc;
+  if (!workspace) return GEMM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255) ||
+      workspace_bytes < gemm_s4_workspace_bytes(M, N, K))
+    return GEMM_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int8_t* a8 = static_cast<int8_t*>(workspace);
+  int8_t* b8 = a8 + align_up(static_cast<size_t>(M) * K, 256);
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState* s = nullptr;
+    rc = device_state(&s);
+    if (rc != GEMM_OK) return rc;
+  }
+  rc = launch_unpack(M, K, A, a8, static_cast<size_t>(K), st);
+  if (rc != GEMM_OK) return rc;
+  rc = launch_unpack(N, K, B, b8, static_cast<size_t>(K), st);
+  if (rc != GEMM_OK) return rc;
+  return launch_gemm<ptx::KIND_I8>(M, N, K, a8, static_cast<size_t>(K), b8, static_cast<size_t>(K),
+                                   C, st);
+}
+
+int gemm_s4(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t* C,
+            gemm_stream_t stream) {
+  int rc = check_s4(M, N, K, A, B, C);
+  if (rc != GEMM_OK) return rc;
+  const size_t need = gemm_s4_workspace_bytes(M, N, K);
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState* s = nullptr;
+    rc = device_state(&s);
+    if (rc != GEMM_OK) return rc;
+    if (s->s4_workspace_bytes < need) {
+      // Grow: earlier launches may still read the old buffer.
+      cudaError_t e = cudaDeviceSynchronize();
+      if (e != cudaSuccess) return cuda_fail(e);
+      if (s->s4_workspace) cudaFree(s->s4_workspace);
+      s->s4_workspace = nullptr;
+      s->s4_workspace_bytes = 0;
+      e = cudaMalloc(&s->s4_workspace, need);
+      if (e != cudaSuccess) return cuda_fail(e);
+      s->s4_workspace_bytes = need;
+    }
+    ws = s->s4_workspace;
+    ws_bytes = s->s4_workspace_bytes;
+  }
+  return gemm_s4_ws(M, N, K, A, B, C, ws, ws_bytes, stream);
+}
+
+int gemm_release_workspaces(void) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  int cur = 0;
+  if (cudaGetDevice(&cur) != cudaSuccess) cur = -1;
+  int rc = GEMM_OK;
+  for (int d = 0; d < MAX_DEVICES; ++d) {
+    if (!g_dev[d].s4_workspace) continue;
+    cudaError_t e = cudaSetDevice(d);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaFree(g_dev[d].s4_workspace);
+    if (e != cudaSuccess) rc = cuda_fail(e);
+    g_dev[d].s4_workspace = nullptr;
+    g_dev[d].s4_workspace_bytes = 0;
+  }
+  if (cur >= 0) cudaSetDevice(cur);
+  return rc;
+}
+
+int gemm_unpack_s4(int rows, int K, const uint8_t* packed, int8_t* out, size_t out_pitch,
+                   gemm_stream_t stream) {
+  if (rows <= 0 || K <= 0 || !packed || !out) return GEMM_ERR_INVALID_ARG;
+  if (K % 32 || out_pitch % 16 || out_pitch < static_cast<size_t>(K) ||
+      ((reinterpret_cast<uintptr_t>(packed) | reinterpret_cast<uintptr_t>(out)) & 15))
+    return GEMM_ERR_MISALIGNED;
+  return launch_unpack(rows, K, packed, out, out_pitch, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int gemm_mma_peak_probe(int precision, int iters, double* ops_out, gemm_stream_t stream) {
+  if (iters <= 0 || !ops_out || (precision != GEMM_PREC_FP16 && precision != GEMM_PREC_S8))
+    return GEMM_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceState* s = nullptr;
+  int rc = device_state(&s);
+  if (rc != GEMM_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  cudaError_t e;
+  int k_per_mma;
+  if (precision == GEMM_PREC_FP16) {
+    auto kernel = mma_peak_probe_kernel<ptx::KIND_F16>;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PROBE_SMEM);
+    if (e != cudaSuccess) return cuda_fail(e);
+    kernel<<<s->num_sms, 128, PROBE_SMEM, st>>>(iters, s->status_ptr);
+    k_per_mma = MMA_K_BYTES / 2;
+  } else {
+    auto kernel = mma_peak_probe_kernel<ptx::KIND_I8>;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PROBE_SMEM);
+    if (e != cudaSuccess) return cuda_fail(e);
+    kernel<<<s->num_sms, 128, PROBE_SMEM, st>>>(iters, s->status_ptr);
+    k_per_mma = MMA_K_BYTES;
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  *ops_out += 2.0 * BM * PROBE_BN * k_per_mma * static_cast<double>(iters) * s->num_sms;
+  return GEMM_OK;
+}
+
+int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
+  if (!buf || len <= 0 || M <= 0 || N <= 0 || K <= 0 || precision < GEMM_PREC_FP16 ||
+      precision > GEMM_PREC_S4)
+    return GEMM_ERR_INVALID_ARG;
+  int num_sms = 148;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < MAX_DEVICES && g_dev[dev].ready)
+      num_sms = g_dev[dev].num_sms;
+  }
+  const TileConfig c = select_config(M, N, num_sms);
+  const int elem = precision == GEMM_PREC_FP16 ? 2 : 1;
+  const long long tiles = static_cast<long long>(ceil_div(M, BM)) * ceil_div(N, c.bn);
+  snprintf(buf, static_cast<size_t>(len),
+           "BM=%d BN=%d BK=%d stages=%d group_m=%d tiles=%lld ctas=%lld kind=%s%s", BM, c.bn,
+           BK_BYTES / elem, c.stages, c.group_m, tiles, tiles < num_sms ? tiles : num_sms,
+           precision == GEMM_PREC_FP16 ? "f16" : "i8",
+           precision == GEMM_PREC_S4 ? " prepass=unpack_s4" : "");
+  return GEMM_OK;
+}
+
+int gemm_set_config_override(int bn, int group_m) {
+  if (group_m < 0) return GEMM_ERR_INVALID_ARG;
+  if (bn != 0) {
+    bool ok = false;
+    for (int w : kWidths) ok = ok || (w == bn);
+    if (!ok) return GEMM_ERR_INVALID_ARG;
+  }
+  std::lock_guard<std::mutex> lock(g_mutex);
+  g_override_bn = bn;
+  g_override_group_m = group_m;
+  return GEMM_OK;
+}
+
+int gemm_last_device_status(void) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceState* s = nullptr;
+  int rc = device_state(&s);
+  if (rc != GEMM_OK) return rc;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e);
+  int v = 0;
+  e = cudaMemcpy(&v, s->status_ptr, sizeof(int), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (v != 0) {
+    e = cudaMemset(s->status_ptr, 0, sizeof(int));
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  return v;
+}
+
+int gemm_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* gemm_status_string(int status) {
+  switch (status) {
+    case GEMM_OK: return "ok";
+    case GEMM_ERR_INVALID_ARG: return "invalid argument";
+    case GEMM_ERR_MISALIGNED: return "misaligned pointer or K";
+    case GEMM_ERR_K_TOO_LARGE: return "K too large: INT32 result could overflow";
+    case GEMM_ERR_UNSUPPORTED_DEVICE: return "unsupported device (needs compute capability 10.x)";
+    case GEMM_ERR_CUDA: return "CUDA call failed";
+    case GEMM_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case GEMM_ERR_TOO_LARGE: return "problem exceeds the capacity of this entry point";
+    default: return "unknown status";
+  }
+}
+
+int gemm_version(void) { return 1000; }
+
+}  // extern "C"

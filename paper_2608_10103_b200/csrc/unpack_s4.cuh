@@ -1,0 +1,57 @@
+// INT4 pre-pass: packed signed 4-bit values -> int8, one value per byte.
+//
+// The paper's INT4 kernels feed nibbles straight to mma.sync.m16n8k64.s4
+// (Listing 2c).  tcgen05.mma has no 4-bit integer kind, so here every operand
+// element is sign-extended once, in a streaming pass bound by HBM bandwidth
+// (reads 1/2 byte, writes 1 byte per element), and the INT8 tensor-core kernel
+// then consumes the result.  Doing it once per operand costs O(N^2) bytes;
+// doing it inside the GEMM pipeline would repeat it for every tile that
+// re-reads the operand (N/BN resp. M/BM times).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace b200gemm {
+
+// Eight nibbles of `w` (byte b holds element 2b in bits 0-3 and element 2b+1 in
+// bits 4-7) -> eight sign-extended bytes in element order: lo = elements 0-3,
+// hi = elements 4-7.
+__device__ __forceinline__ void unpack8_s4(uint32_t w, uint32_t& lo, uint32_t& hi) {
+  uint32_t even = w & 0x0F0F0F0Fu;         // elements 0,2,4,6 (one per byte)
+  uint32_t odd = (w >> 4) & 0x0F0F0F0Fu;   // elements 1,3,5,7
+  even |= (even & 0x08080808u) * 0x1Eu;    // bit 3 set -> fill bits 4-7 (0x08 * 0x1E = 0xF0)
+  odd |= (odd & 0x08080808u) * 0x1Eu;
+  lo = __byte_perm(even, odd, 0x5140);     // e0 o0 e1 o1
+  hi = __byte_perm(even, odd, 0x7362);     // e2 o2 e3 o3
+}
+
+// One thread expands 16 packed bytes (32 elements) into 32 output bytes.
+// chunks_per_row = K / 32.  Bytes K .. out_pitch-1 of each output row are zeroed.
+__global__ void __launch_bounds__(256)
+unpack_s4_kernel(const uint4* __restrict__ packed, int8_t* __restrict__ out, long long rows,
+                 int chunks_per_row, long long out_pitch) {
+  const long long total = rows * chunks_per_row;
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total;
+       idx += stride) {
+    const long long row = idx / chunks_per_row;
+    const int chunk = static_cast<int>(idx - row * chunks_per_row);
+    const uint4 w = __ldg(packed + idx);
+    uint4 o0, o1;
+    unpack8_s4(w.x, o0.x, o0.y);
+    unpack8_s4(w.y, o0.z, o0.w);
+    unpack8_s4(w.z, o1.x, o1.y);
+    unpack8_s4(w.w, o1.z, o1.w);
+    uint4* dst = reinterpret_cast<uint4*>(out + row * out_pitch + static_cast<long long>(chunk) * 32);
+    dst[0] = o0;
+    dst[1] = o1;
+    if (chunk == chunks_per_row - 1) {
+      const long long k_end = static_cast<long long>(chunks_per_row) * 32;
+      for (long long b = k_end; b < out_pitch; b += 16)
+        *reinterpret_cast<uint4*>(out + row * out_pitch + b) = make_uint4(0, 0, 0, 0);
+    }
+  }
+}
+
+}  // namespace b200gemm

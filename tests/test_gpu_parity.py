@@ -1,0 +1,256 @@
+"""GPU parity: the CUDA library, called through its C-ABI, against the CPU
+oracle on the same seeded inputs.  Integer paths must match bit for bit; FP16
+must satisfy |C_gpu - C_ref| <= 1e-4 * sum_k|a*b| + 1e-6 element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_10103_b200 import binding, synth
+from gpu_util import (assert_block, check_against_oracle, decode_s4, freivalds, oracle_block,
+                      run_gpu, to_dev)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def _clean_state():
+    binding.gemm_set_config_override(0, 0)
+    yield
+    binding.gemm_set_config_override(0, 0)
+    assert binding.gemm_last_device_status() == 0
+
+
+# ------------------------------------------------------------ the named configs
+def test_config_fp16_512_seed0():
+    A, B = synth.fp16_uniform(512, 512, 512, seed=0)
+    C = run_gpu("fp16", A, B, fill=float("nan"))
+    assert check_against_oracle("fp16", A, B, C) == 512 * 512
+
+
+def test_config_s8_2048_seed1():
+    A, B = synth.s8_uniform(2048, 2048, 2048, seed=1)
+    C = run_gpu("s8", A, B, fill=-1)
+    assert check_against_oracle("s8", A, B, C) == 2048 * 2048
+
+
+def test_config_s4_4096_seed2():
+    A, B = synth.s4_uniform(4096, 4096, 4096, seed=2)
+    C = run_gpu("s4", A, B, fill=-1)
+    check_against_oracle("s4", A, B, C, seed=2)
+    freivalds("s4", A, B, C, seed=2)
+
+
+def test_config_fp16_8192_seed3_normal():
+    A, B = synth.fp16_normal_clipped(8192, 8192, 8192, seed=3)
+    C = run_gpu("fp16", A, B, fill=float("nan"))
+    assert np.isfinite(C).all()
+    check_against_oracle("fp16", A, B, C, seed=3)
+    freivalds("fp16", A, B, C, seed=3)
+
+
+@pytest.mark.parametrize("N", synth.SWEEP_SIZES)
+@pytest.mark.parametrize("prec", synth.PRECISIONS)
+def test_sweep(prec, N):
+    seed = synth.sweep_seed(prec, N)
+    A, B = synth.make(prec, N, N, N, seed)
+    C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
+    check_against_oracle(prec, A, B, C, seed=seed)
+    if N > 2048:
+        freivalds(prec, A, B, C, seed=seed)
+
+
+# --------------------------------------------------- ragged and degenerate shapes
+RAGGED = [
+    # (M, N, K): K obeys the alignment rule of each precision (multiple of 32 works for all)
+    (1, 1, 32), (1, 300, 64), (300, 1, 96), (127, 129, 160), (130, 70, 224),
+    (257, 513, 288), (300, 520, 320), (640, 33, 1056), (129, 1030, 4128),
+]
+
+
+@pytest.mark.parametrize("prec", synth.PRECISIONS)
+@pytest.mark.parametrize("M,N,K", RAGGED)
+def test_ragged_shapes(prec, M, N, K):
+    A, B = synth.make(prec, M, N, K, seed=1000 + M + N + K)
+    C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
+    check_against_oracle(prec, A, B, C, force_full=True)
+
+
+@pytest.mark.parametrize("N", [1, 2, 3, 5, 30, 66, 131])
+def test_n_not_multiple_of_four(N):
+    """Rows of C that are not 16-byte multiples take the scalar store path."""
+    M, K = 200, 128
+    for prec in synth.PRECISIONS:
+        A, B = synth.make(prec, M, N, K, seed=N)
+        C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
+        check_against_oracle(prec, A, B, C, force_full=True)
+
+
+def test_minimal_k():
+    A, B = synth.fp16_uniform(140, 260, 8, seed=5)
+    check_against_oracle("fp16", A, B, run_gpu("fp16", A, B, fill=float("nan")), force_full=True)
+    A, B = synth.s8_uniform(140, 260, 16, seed=6)
+    check_against_oracle("s8", A, B, run_gpu("s8", A, B, fill=-7), force_full=True)
+    A, B = synth.s4_uniform(140, 260, 32, seed=7)
+    check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), force_full=True)
+
+
+# ------------------------------------------------ every tile width the selector has
+@pytest.mark.parametrize("bn", [32, 64, 128, 256])
+@pytest.mark.parametrize("prec", synth.PRECISIONS)
+def test_every_tile_width(prec, bn):
+    M, N, K = 520, 1100, 1184           # several tiles in both directions + ragged tails
+    A, B = synth.make(prec, M, N, K, seed=bn)
+    binding.gemm_set_config_override(bn, 0)
+    assert ("BN=%d " % bn) in binding.gemm_query_config(prec, M, N, K)
+    C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
+    check_against_oracle(prec, A, B, C, force_full=True)
+
+
+@pytest.mark.parametrize("group_m", [1, 2, 3, 7, 64])
+def test_raster_band_heights(group_m):
+    M, N, K = 1300, 1500, 256
+    A, B = synth.s8_uniform(M, N, K, seed=group_m)
+    binding.gemm_set_config_override(64, group_m)
+    check_against_oracle("s8", A, B, run_gpu("s8", A, B, fill=-7), force_full=True)
+
+
+# --------------------------------------------------------------- structured cases
+def test_index_mapping_product_table():
+    """a(i,0) = i mod 97 - 48, b(j,0) = j mod 89 - 44, rest 0: any row, column,
+    lane-quarter or tile mix-up shows as a structured difference."""
+    M, N, K = 1024, 1024, 128
+    a = np.zeros((M, K), np.int8)
+    b = np.zeros((N, K), np.int8)
+    a[:, 0] = (np.arange(M) % 97) - 48
+    b[:, 0] = (np.arange(N) % 89) - 44
+    want = np.outer(a[:, 0].astype(np.int32), b[:, 0].astype(np.int32))
+    for bn in (0, 32, 64, 128, 256):
+        binding.gemm_set_config_override(bn, 0)
+        assert np.array_equal(run_gpu("s8", a, b, fill=-7), want)
+        got = run_gpu("fp16", a.astype(np.float16), b.astype(np.float16), fill=float("nan"))
+        assert np.array_equal(got, want.astype(np.float32))
+        a4, b4 = np.clip(a, -8, 7), np.clip(b, -8, 7)
+        want4 = np.outer(a4[:, 0].astype(np.int32), b4[:, 0].astype(np.int32))
+        assert np.array_equal(run_gpu("s4", synth.pack_s4(a4), synth.pack_s4(b4), fill=-7), want4)
+
+
+def test_one_hot_k_positions():
+    """C = [k0 == k1] for one-hot rows: pins the K order through swizzle, the
+    32-byte MMA steps, the k-block ring and (int4) the nibble order."""
+    K = 512
+    ks = [0, 1, 2, 15, 16, 31, 32, 63, 64, 65, 127, 128, 129, 255, 256, 383, 384, K - 1]
+    a = np.zeros((len(ks), K), np.int8)
+    for r, k in enumerate(ks):
+        a[r, k] = 1
+    eye = np.eye(len(ks), dtype=np.int32)
+    assert np.array_equal(run_gpu("s8", a, a, fill=-7), eye)
+    assert np.array_equal(run_gpu("s4", synth.pack_s4(a), synth.pack_s4(a), fill=-7), eye)
+    assert np.array_equal(run_gpu("fp16", a.astype(np.float16), a.astype(np.float16)),
+                          eye.astype(np.float32))
+
+
+def test_all_ones_and_identity():
+    K = 2048
+    ones8 = np.ones((256, K), np.int8)
+    assert np.all(run_gpu("s8", ones8, ones8) == K)
+    assert np.all(run_gpu("fp16", ones8.astype(np.float16), ones8.astype(np.float16)) == K)
+    assert np.all(run_gpu("s4", synth.pack_s4(ones8), synth.pack_s4(ones8)) == K)
+    A, _ = synth.s8_uniform(300, 8, 256, seed=3)
+    eye = np.eye(256, dtype=np.int8)
+    assert np.array_equal(run_gpu("s8", A, eye), A.astype(np.int32))          # B = I -> C = A
+    assert np.array_equal(run_gpu("s8", eye, A), A.T.astype(np.int32))        # A = I -> C = B^T
+
+
+def test_int32_extremes():
+    K = 8192
+    lo8 = np.full((130, K), -128, np.int8)
+    hi8 = np.full((70, K), 127, np.int8)
+    assert np.all(run_gpu("s8", lo8, lo8) == 2 ** 27)
+    assert np.all(run_gpu("s8", lo8, hi8) == -133169152)
+    lo4 = synth.pack_s4(np.full((130, K), -8))
+    hi4 = synth.pack_s4(np.full((70, K), 7))
+    assert np.all(run_gpu("s4", lo4, lo4) == 524288)
+    assert np.all(run_gpu("s4", lo4, hi4) == -458752)
+
+
+def test_largest_k_for_int8():
+    """K = 131056 (largest multiple of 16 <= 131071): 16384*K < 2^31 holds exactly."""
+    K = 131056
+    lo8 = np.full((3, K), -128, np.int8)
+    assert np.all(run_gpu("s8", lo8, lo8) == 16384 * K)
+    A, B = synth.s8_uniform(5, 7, K, seed=8)
+    check_against_oracle("s8", A, B, run_gpu("s8", A, B), force_full=True)
+
+
+def test_fp16_subnormals_and_large_values():
+    g = np.random.Generator(np.random.PCG64(9))
+    M, N, K = 150, 140, 256
+    A = (g.integers(0, 0x0400, size=(M, K)).astype(np.uint16)
+         | (g.integers(0, 2, size=(M, K)).astype(np.uint16) << 15)).view(np.float16)  # subnormals
+    B = g.uniform(-60000, 60000, size=(N, K)).astype(np.float16)
+    C = run_gpu("fp16", A, B, fill=float("nan"))
+    check_against_oracle("fp16", A, B, C, force_full=True)
+
+
+# ------------------------------------------------------------------ the pre-pass
+def test_unpack_s4_matches_decoder():
+    g = np.random.Generator(np.random.PCG64(10))
+    P = g.integers(0, 256, size=(333, 480), dtype=np.uint8)
+    out = binding.gemm_unpack_s4(to_dev(P))
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().astype(np.int16), decode_s4(P))
+    # every byte value, in every position of a 16-byte group
+    P = np.tile(np.arange(256, dtype=np.uint8), (16, 1))
+    P = np.stack([np.roll(P[i], i) for i in range(16)])
+    out = binding.gemm_unpack_s4(to_dev(P)).cpu().numpy()
+    assert np.array_equal(out.astype(np.int16), decode_s4(P))
+
+
+def test_s4_with_caller_workspace():
+    M, N, K = 300, 200, 512
+    A, B = synth.s4_uniform(M, N, K, seed=11)
+    need = binding.gemm_s4_workspace_bytes(M, N, K)
+    assert need >= (M + N) * K
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    C = binding.gemm_s4_ws(to_dev(A), to_dev(B), ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(C.cpu().numpy(), oracle.gemm_s4(A, B, K))
+    with pytest.raises(binding.GemmError) as e:
+        binding.gemm_s4_ws(to_dev(A), to_dev(B), ws[: need - 256])
+    assert e.value.code == -6
+
+
+# ------------------------------------------------------------- API behaviour
+def test_non_default_stream_and_repeat_calls():
+    A, B = synth.s8_uniform(512, 384, 1024, seed=12)
+    dA, dB = to_dev(A), to_dev(B)
+    ref = oracle.gemm_s8(A, B)
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(st):
+        outs = [binding.gemm_s8(dA, dB) for _ in range(5)]
+    st.synchronize()
+    for C in outs:
+        assert np.array_equal(C.cpu().numpy(), ref)
+
+
+def test_argument_errors_enqueue_nothing():
+    L = binding.lib()
+    A = torch.zeros(64, 64, dtype=torch.int8, device="cuda")
+    C = torch.full((64, 64), 5, dtype=torch.int32, device="cuda")
+    p, c = A.data_ptr(), C.data_ptr()
+    assert L.gemm_s8(64, 64, 64, None, p, c, None) == -1
+    assert L.gemm_s8(0, 64, 64, p, p, c, None) == -1
+    assert L.gemm_s8(64, -1, 64, p, p, c, None) == -1
+    assert L.gemm_s8(64, 64, 24, p, p, c, None) == -2          # K % 16
+    assert L.gemm_s8(64, 64, 64, p + 1, p, c, None) == -2      # pointer alignment
+    assert L.gemm_s8(2, 2, 131072, p, p, c, None) == -3
+    assert L.gemm_fp16(64, 64, 12, p, p, c, None) == -2        # K % 8
+    assert L.gemm_s4(64, 64, 48, p, p, c, None) == -2          # K % 32
+    assert L.gemm_s4(2, 2, 131072, p, p, c, None) == -3
+    assert L.gemm_unpack_s4(4, 32, p, None, 32, None) == -1
+    torch.cuda.synchronize()
+    assert int((C != 5).sum()) == 0
+    assert binding.gemm_status_string if True else None
+    assert L.gemm_status_string(-3).decode().startswith("K too large")
