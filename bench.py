@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of the GEMM hot path on B200:  C = A * B^T at N = 8192.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--size N] [--e2e-steps E] [--no-cpu-baseline]
+
+One step = one pass of the whole path over one batch of seeded synthetic
+operands: an FP16 GEMM, an INT8 GEMM and an INT4 GEMM (nibble unpack pre-pass
++ INT8 tensor-core kernel) of size N^3, each bracketed by CUDA events on the
+launching stream.  The headline `value` is the FP16 rate (TFLOP/s, 2 N^3 per
+GEMM); the INT8 / INT4 rates (TOP/s) and every fraction-of-peak are in
+`precisions`.  Operands stay resident in HBM for `value`; `e2e` repeats the
+FP16 GEMM with pinned host buffers and both copies inside the timed region.
+
+Prints ONE JSON line on rank 0.  Under torchrun each rank runs an independent
+replica of the same workload (no data-path collective; weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+SPEC_PEAK = {"fp16": 2250.0, "s8": 4500.0, "s4": 4500.0}   # vendor dense figures, T(FL)OP/s
+UNIT = {"fp16": "TFLOP/s", "s8": "TOP/s", "s4": "TOP/s"}
+KERNEL_LAUNCHES = {"fp16": 1, "s8": 1, "s4": 3}            # s4: two unpack launches + GEMM
+# DRAM bytes per launch of the FP16 GEMM kernel at N = 8192 (dram__bytes_read.sum +
+# dram__bytes_write.sum from one ncu capture; see profiles/).  None until captured.
+NCU_TRAFFIC_BYTES = {"fp16": {}}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_burst": float(d["bf16_tflops"]),
+                "bf16_sustained": float(d["bf16_tflops_sustained"]),
+                "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    except Exception:
+        return {"bf16_burst": 1590.0, "bf16_sustained": 1400.0, "hbm_gbs": 6650.0,
+                "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while a region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "20"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        if self.thread:
+            self.thread.join(timeout=2)
+        sm, mx, pw = [], [], []
+        reasons = set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                pw.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except (ValueError, IndexError):
+            return local
+    return local
+
+
+# --------------------------------------------------------------------- reference arm
+def run_reference(args, rank):
+    """Times the CPU oracle, as it stands, on a bounded sample of the same FP16
+    workload (a block of rows of C, all columns), on this machine's host cores."""
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    from paper_2608_10103_b200 import synth
+    N = args.size
+    A, B = synth.fp16_normal_clipped(N, N, N, seed=3)
+    rows = np.arange(args.ref_rows, dtype=np.int32)
+    ops = synth.gemm_ops(len(rows), N, N)
+    for _ in range(args.warmup):
+        oracle.gemm_fp16(A, B, rows=rows[:2])
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.gemm_fp16(A, B, rows=rows)
+    dt = time.perf_counter() - t0
+    value = ops * args.steps / dt / 1e12
+    sample = "%d rows x %d cols of C per step (K=%d)" % (len(rows), N, N)
+    line = {
+        "impl": "reference", "metric": "fp16_gemm_tflops_n%d" % N, "value": value,
+        "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "FP16 GEMM M=N=K=%d, N(0,1) clipped to [-4,4], seed 3" % N,
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": oracle.threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- our arm
+def cpu_baseline(N, A, B, target_seconds=12.0):
+    """The oracle, as it stands, on a block of rows of the FP16 problem sized to
+    take about `target_seconds` on this machine's cores."""
+    import numpy as np
+    import oracle
+    from paper_2608_10103_b200 import synth
+
+    def run(n):
+        t0 = time.perf_counter()
+        oracle.gemm_fp16(A, B, rows=np.arange(n, dtype=np.int32))
+        return time.perf_counter() - t0
+
+    th = oracle.threads()
+    n_a, n_b = 2 * th, 6 * th
+    t_a, t_b = run(n_a), run(n_b)
+    per_row = max((t_b - t_a) / (n_b - n_a), 1e-7)
+    fixed = max(t_a - n_a * per_row, 0.0)          # one-off operand decode
+    nrows = int((target_seconds - fixed) / per_row) // th * th
+    nrows = max(n_b, min(N, nrows))
+    dt = run(nrows)
+    return {"value": synth.gemm_ops(nrows, N, N) / dt / 1e12, "unit": "TFLOP/s",
+            "cores": th, "kind": "oracle",
+            "sample": "%d rows x %d cols of the FP16 C (K=%d), %.1f s" % (nrows, N, N, dt)}
+
+
+def run_ours(args, rank, world):
+    import numpy as np
+    import torch
+    from paper_2608_10103_b200 import binding, replicas, synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the GEMM path has no CPU fallback")
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    binding.lib()
+    N = args.size
+    ops = synth.gemm_ops(N, N, N)
+    stream = torch.cuda.current_stream()
+
+    # Operands: the named N = 8192 configurations (FP16: N(0,1) clipped, seed 3; INT8 / INT4:
+    # the sweep's uniform draws).  Each rank draws its own replica (seed + rank).
+    want = args.precisions.split(",")
+    host = {"fp16": synth.fp16_normal_clipped(N, N, N, seed=replicas.replica_seed(3, rank))}
+    if "s8" in want:
+        host["s8"] = synth.s8_uniform(
+            N, N, N, seed=replicas.replica_seed(synth.sweep_seed("s8", 8192), rank))
+    if "s4" in want:
+        host["s4"] = synth.s4_uniform(
+            N, N, N, seed=replicas.replica_seed(synth.sweep_seed("s4", 8192), rank))
+    dev = {p: (torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()) for p, (a, b) in host.items()}
+    out = {p: torch.empty((N, N), dtype=torch.float32 if p == "fp16" else torch.int32,
+                          device="cuda") for p in host}
+    precs = tuple(x for x in ("fp16", "s8", "s4") if x in args.precisions.split(","))
+    if "fp16" not in precs:
+        raise SystemExit("bench.py: --precisions must include fp16 (the headline)")
+
+    def step(events=None):
+        for p in precs:
+            if events is not None:
+                events[p][0].record(stream)
+            binding.gemm(p, dev[p][0], dev[p][1], out[p], stream)
+            if events is not None:
+                events[p][1].record(stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    evs = [{p: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+            for p in precs} for _ in range(args.steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record(stream)
+    for i in range(args.steps):
+        step(evs[i])
+    stop.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    total_ms = start.elapsed_time(stop)
+    per_prec_ms = {p: sum(e[p][0].elapsed_time(e[p][1]) for e in evs) / args.steps for p in precs}
+    best_ms = {p: min(e[p][0].elapsed_time(e[p][1]) for e in evs) for p in precs}
+    if binding.gemm_last_device_status() != 0:
+        raise SystemExit("bench.py: a kernel reported a barrier timeout")
+
+    # max over ranks (device time)
+    times = replicas.max_over_ranks([total_ms] + [per_prec_ms[p] for p in precs], dist, "cuda")
+    total_ms = times[0]
+    worst = dict(zip(precs, times[1:]))
+
+    # ---- MMA-issue-only peak of this machine, per kind (same run, same clocks regime)
+    mma_peak = {}
+    for kind in (() if args.no_peak_probe else ("fp16", "s8")):
+        binding.gemm_mma_peak_probe(kind, 2048)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        pops = binding.gemm_mma_peak_probe(kind, 200000)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        mma_peak[kind] = pops / (e0.elapsed_time(e1) * 1e-3) / 1e12
+    if mma_peak:
+        mma_peak["s4"] = mma_peak["s8"]
+
+    # ---- end to end: FP16 GEMM with pinned host buffers, both copies timed
+    e2e = None
+    if args.e2e_steps > 0:
+        hA = torch.from_numpy(host["fp16"][0]).pin_memory()
+        hB = torch.from_numpy(host["fp16"][1]).pin_memory()
+        hC = torch.empty((N, N), dtype=torch.float32).pin_memory()
+        dA, dB = torch.empty_like(dev["fp16"][0]), torch.empty_like(dev["fp16"][1])
+
+        def e2e_step():
+            dA.copy_(hA, non_blocking=True)
+            dB.copy_(hB, non_blocking=True)
+            binding.gemm_fp16(dA, dB, out["fp16"], stream)
+            hC.copy_(out["fp16"], non_blocking=True)
+
+        e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = replicas.max_over_ranks([e0.elapsed_time(e1)], dist, "cuda")[0] / args.e2e_steps
+        e2e = {"value": replicas.whole_job_rate(ops, world, e2e_ms), "unit": "TFLOP/s",
+               "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": hA.numel() * 2 + hB.numel() * 2,
+               "d2h_bytes_per_step": hC.numel() * 4,
+               "what": "FP16 GEMM via gemm_fp16 with pinned host A, B, C; H2D + kernel + D2H"}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    # the GEMMs are timed inside a long back-to-back loop -> sustained figure
+    ref_peak = {"fp16": peaks["bf16_sustained"], "s8": 2 * peaks["bf16_sustained"],
+                "s4": 2 * peaks["bf16_sustained"]}
+    precisions = {}
+    for p in precs:
+        rate = replicas.whole_job_rate(ops, world, worst[p])
+        precisions[p] = {
+            "value": rate, "unit": UNIT[p], "ms": worst[p], "best_ms_rank0": best_ms[p],
+            "frac_of_spec_peak": rate / world / SPEC_PEAK[p], "spec_peak": SPEC_PEAK[p],
+            "frac_of_mma_only_peak": rate / world / mma_peak[p] if mma_peak else None,
+            "mma_only_peak": mma_peak.get(p),
+            "config": binding.gemm_query_config(p, N, N, N),
+        }
+    if "s4" in worst and "s8" in worst:
+        precisions["s4"]["overhead_vs_s8"] = worst["s4"] / worst["s8"] - 1.0
+
+    fp16_rate_1gpu = ops / (worst["fp16"] * 1e-3) / 1e12
+    traffic = NCU_TRAFFIC_BYTES["fp16"].get(N)
+    line = {
+        "metric": "fp16_gemm_tflops_n%d" % N, "value": precisions["fp16"]["value"],
+        "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+        "config": {
+            "workload": "FP16 GEMM M=N=K=%d, N(0,1) clipped to [-4,4], seed 3, FP32 accumulate and C; "
+                        "one step runs the GEMMs of this size for: %s" % (N, ",".join(precs)),
+            "l2": "operands + C of every GEMM exceed the 126 MB L2; no flush",
+            "replicas": "one independent problem per GPU" if world > 1 else "single GPU",
+        },
+        "precisions": precisions,
+        "roofline": {
+            "bound": "tensor", "achieved": fp16_rate_1gpu, "peak": ref_peak["fp16"],
+            "unit": "TFLOP/s", "frac": fp16_rate_1gpu / ref_peak["fp16"], "traffic": traffic,
+            "peak_source": "%s cuBLAS bf16 sustained (kernel timed inside a long step)" % peaks["source"],
+            "kernel": "gemm_kernel<f16> N=%d, avg of %d launches" % (N, args.steps),
+        },
+        "clocks": clocks,
+        "e2e": e2e,
+        "gpu_launches": args.steps * sum(KERNEL_LAUNCHES[p] for p in precs),
+    }
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(N, host["fp16"][0], host["fp16"][1])
+    if dist is not None:
+        dist.destroy_process_group()
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--size", type=int, default=8192)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--ref-rows", type=int, default=32)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-peak-probe", action="store_true")
+    ap.add_argument("--precisions", default="fp16,s8,s4")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, world)
+
+
+if __name__ == "__main__":
+    main()

@@ -135,10 +135,12 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len);
 
 /*
  * Overrides the selector for later calls from this process: tile width BN
- * (0 = automatic) and raster band height in tiles (0 = automatic).  For
- * ablation sweeps.  Returns GEMM_ERR_INVALID_ARG for a width that is not built.
+ * (0 = automatic), raster band height in tiles (0 = automatic) and the number
+ * of CTAs that share one tile (0 = automatic, 1 = 128 x BN tile per CTA, 2 =
+ * 256 x BN tile per CTA pair).  For ablation sweeps in the spirit of the
+ * paper's Run 4.  Returns GEMM_ERR_INVALID_ARG for a shape that is not built.
  */
-int gemm_set_config_override(int bn, int group_m);
+int gemm_set_config_override(int bn, int group_m, int cta_group);
 
 /*
  * Kernels never spin forever: a barrier wait that exceeds its limit makes the

@@ -62,7 +62,7 @@ def lib() -> ctypes.CDLL:
         L.gemm_unpack_s4.argtypes = [i, i, vp, vp, sz, vp]
         L.gemm_mma_peak_probe.argtypes = [i, i, ctypes.POINTER(ctypes.c_double), vp]
         L.gemm_query_config.argtypes = [i, i, i, i, ctypes.c_char_p, i]
-        L.gemm_set_config_override.argtypes = [i, i]
+        L.gemm_set_config_override.argtypes = [i, i, i]
         L.gemm_status_string.argtypes = [i]
         L.gemm_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -188,12 +188,20 @@ def gemm_query_config(precision: str, M: int, N: int, K: int) -> str:
     return buf.value.decode()
 
 
-def gemm_set_config_override(bn: int = 0, group_m: int = 0):
-    _check(lib().gemm_set_config_override(bn, group_m), "gemm_set_config_override")
+def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0):
+    _check(lib().gemm_set_config_override(bn, group_m, cta_group), "gemm_set_config_override")
 
 
 def gemm_last_device_status() -> int:
     return int(lib().gemm_last_device_status())
+
+
+def gemm_status_string(code: int) -> str:
+    return lib().gemm_status_string(code).decode()
+
+
+def gemm_last_cuda_error() -> int:
+    return int(lib().gemm_last_cuda_error())
 
 
 def gemm_version() -> int:

@@ -35,6 +35,7 @@ DeviceState g_dev[MAX_DEVICES];
 int g_last_cuda_error = 0;
 int g_override_bn = 0;
 int g_override_group_m = 0;
+int g_override_cta_group = 0;
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                    const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -98,67 +99,95 @@ int encode_operand_map(CUtensorMap* map, CUtensorMapDataType type, int elem_byte
 // ------------------------------------------------------------------ selector
 struct TileConfig {
   int bn;
+  int cta_group;  // 1: one CTA per 128 x bn tile; 2: a CTA pair per 256 x bn tile
   int stages;
   int group_m;
 };
 
 constexpr int kWidths[] = {256, 128, 64, 32};
 
-int stages_for(int bn) {
+int stages_for(int bn, int cta_group) {
+  if (cta_group == 2) return bn == 256 ? 6 : 8;
   switch (bn) {
     case 256: return 4;
     case 128: return 6;
-    case 64: return 8;
     default: return 8;
   }
 }
 
+bool variant_exists(int bn, int cta_group) {
+  if (cta_group == 1) return bn == 256 || bn == 128 || bn == 64 || bn == 32;
+  if (cta_group == 2) return bn == 256 || bn == 128 || bn == 64;
+  return false;
+}
+
 int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b); }
 
-// Picks the C-tile width.  The paper fixes one tiling for all sizes (Sec.
-// III-A); on 148 SMs small problems need narrower tiles to fill the machine.
-// Cost model: waves of CTAs x (tile width + a fixed per-tile overhead).
+// Picks the C-tile shape.  The paper fixes one tiling for all sizes (Sec.
+// III-A); on 148 SMs small problems need smaller tiles to fill the machine and
+// large ones want the CTA-pair tile, which halves the B bytes each SM pulls
+// from L2.  Cost model: waves of tiles x (tile width + a fixed per-tile
+// overhead), with a discount for the pair shape.
 TileConfig select_config(int M, int N, int num_sms) {
-  TileConfig best{256, 4, 16};
-  if (g_override_bn) {
-    best.bn = g_override_bn;
-  } else {
-    long long best_cost = -1;
+  TileConfig best{256, 2, 6, 8};
+  long long best_cost = -1;
+  for (int cg = 2; cg >= 1; --cg) {
+    if (g_override_cta_group && cg != g_override_cta_group) continue;
     for (int bn : kWidths) {
-      long long tiles = static_cast<long long>(ceil_div(M, BM)) * ceil_div(N, bn);
-      long long waves = (tiles + num_sms - 1) / num_sms;
-      long long cost = waves * (bn + 16);
+      if (g_override_bn && bn != g_override_bn) continue;
+      if (!variant_exists(bn, cg)) continue;
+      long long tiles = static_cast<long long>(ceil_div(M, BM * cg)) * ceil_div(N, bn);
+      long long units = num_sms / cg;
+      long long waves = (tiles + units - 1) / units;
+      long long cost = waves * (bn + 160) * (cg == 2 ? 85 : 100);
       if (best_cost < 0 || cost < best_cost) {
         best_cost = cost;
         best.bn = bn;
+        best.cta_group = cg;
       }
     }
   }
-  best.stages = stages_for(best.bn);
+  best.stages = stages_for(best.bn, best.cta_group);
   // Band height: make one wave of tiles roughly square in operand bytes.
-  int g = 16;
-  if (best.bn == 128) g = 12;
-  if (best.bn <= 64) g = 8;
+  int rows_per_tile = BM * best.cta_group;
+  int units = num_sms / best.cta_group;
+  int g = 1;
+  while ((g + 1) * (g + 1) * rows_per_tile <= units * best.bn) ++g;
   if (g_override_group_m) g = g_override_group_m;
-  int tiles_m = ceil_div(M, BM);
+  int tiles_m = ceil_div(M, rows_per_tile);
   if (g > tiles_m) g = tiles_m;
+  if (g < 1) g = 1;
   best.group_m = g;
   return best;
 }
 
-template <int KIND, int BN, int STAGES>
+template <int KIND, int BN, int STAGES, int CTA_GROUP>
 int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUtensorMap& tb,
-                   const GemmParams& p, int grid, cudaStream_t stream) {
-  using L = SmemLayout<BN, STAGES>;
-  auto kernel = gemm_kernel<KIND, BN, STAGES>;
+                   const GemmParams& p, cudaStream_t stream) {
+  using L = SmemLayout<BN, STAGES, CTA_GROUP>;
+  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP>;
   if (!(s->attr_set & (1ull << variant))) {
     cudaError_t e =
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
     if (e != cudaSuccess) return cuda_fail(e);
     s->attr_set |= 1ull << variant;
   }
-  kernel<<<grid, NUM_THREADS, L::DYN_BYTES, stream>>>(ta, tb, p);
-  cudaError_t e = cudaGetLastError();
+  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
+  const long long units = s->num_sms / CTA_GROUP;
+  const int grid = static_cast<int>((tiles < units ? tiles : units) * CTA_GROUP);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = L::DYN_BYTES;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTA_GROUP;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, p);
   if (e != cudaSuccess) return cuda_fail(e);
   return GEMM_OK;
 }
@@ -179,29 +208,35 @@ int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* 
   CUtensorMap ta, tb;
   rc = encode_operand_map(&ta, type, ELEM, A, M, K, a_pitch, BM);
   if (rc != GEMM_OK) return rc;
-  rc = encode_operand_map(&tb, type, ELEM, B, N, K, b_pitch, cfg.bn);
+  rc = encode_operand_map(&tb, type, ELEM, B, N, K, b_pitch, cfg.bn / cfg.cta_group);
   if (rc != GEMM_OK) return rc;
 
   GemmParams p;
   p.M = M;
   p.N = N;
   p.K = K;
-  p.tiles_m = ceil_div(M, BM);
+  p.tiles_m = ceil_div(M, BM * cfg.cta_group);
   p.tiles_n = ceil_div(N, cfg.bn);
   p.group_m = cfg.group_m;
   p.k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
   p.c_vec_ok = (N % 4 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
   p.C = static_cast<uint32_t*>(C);
   p.status = s->status_ptr;
-  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
-  const int grid = static_cast<int>(tiles < s->num_sms ? tiles : s->num_sms);
 
-  const int kbase = (KIND == ptx::KIND_F16) ? 0 : 8;
+  const int kbase = (KIND == ptx::KIND_F16) ? 0 : 16;
+  if (cfg.cta_group == 2) {
+    switch (cfg.bn) {
+      case 256: return launch_variant<KIND, 256, 6, 2>(s, kbase + 8, ta, tb, p, stream);
+      case 128: return launch_variant<KIND, 128, 8, 2>(s, kbase + 9, ta, tb, p, stream);
+      case 64: return launch_variant<KIND, 64, 8, 2>(s, kbase + 10, ta, tb, p, stream);
+      default: return GEMM_ERR_INVALID_ARG;
+    }
+  }
   switch (cfg.bn) {
-    case 256: return launch_variant<KIND, 256, 4>(s, kbase + 0, ta, tb, p, grid, stream);
-    case 128: return launch_variant<KIND, 128, 6>(s, kbase + 1, ta, tb, p, grid, stream);
-    case 64: return launch_variant<KIND, 64, 8>(s, kbase + 2, ta, tb, p, grid, stream);
-    case 32: return launch_variant<KIND, 32, 8>(s, kbase + 3, ta, tb, p, grid, stream);
+    case 256: return launch_variant<KIND, 256, 4, 1>(s, kbase + 0, ta, tb, p, stream);
+    case 128: return launch_variant<KIND, 128, 6, 1>(s, kbase + 1, ta, tb, p, stream);
+    case 64: return launch_variant<KIND, 64, 8, 1>(s, kbase + 2, ta, tb, p, stream);
+    case 32: return launch_variant<KIND, 32, 8, 1>(s, kbase + 3, ta, tb, p, stream);
     default: return GEMM_ERR_INVALID_ARG;
   }
 }
@@ -391,25 +426,33 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
   }
   const TileConfig c = select_config(M, N, num_sms);
   const int elem = precision == GEMM_PREC_FP16 ? 2 : 1;
-  const long long tiles = static_cast<long long>(ceil_div(M, BM)) * ceil_div(N, c.bn);
+  const long long tiles =
+      static_cast<long long>(ceil_div(M, BM * c.cta_group)) * ceil_div(N, c.bn);
+  const long long units = num_sms / c.cta_group;
   snprintf(buf, static_cast<size_t>(len),
-           "BM=%d BN=%d BK=%d stages=%d group_m=%d tiles=%lld ctas=%lld kind=%s%s", BM, c.bn,
-           BK_BYTES / elem, c.stages, c.group_m, tiles, tiles < num_sms ? tiles : num_sms,
+           "BM=%d BN=%d BK=%d cta_group=%d stages=%d group_m=%d tiles=%lld ctas=%lld kind=%s%s",
+           BM * c.cta_group, c.bn, BK_BYTES / elem, c.cta_group, c.stages, c.group_m, tiles,
+           (tiles < units ? tiles : units) * c.cta_group,
            precision == GEMM_PREC_FP16 ? "f16" : "i8",
            precision == GEMM_PREC_S4 ? " prepass=unpack_s4" : "");
   return GEMM_OK;
 }
 
-int gemm_set_config_override(int bn, int group_m) {
-  if (group_m < 0) return GEMM_ERR_INVALID_ARG;
-  if (bn != 0) {
-    bool ok = false;
-    for (int w : kWidths) ok = ok || (w == bn);
-    if (!ok) return GEMM_ERR_INVALID_ARG;
+int gemm_set_config_override(int bn, int group_m, int cta_group) {
+  if (group_m < 0 || cta_group < 0 || cta_group > 2) return GEMM_ERR_INVALID_ARG;
+  bool ok = false;
+  for (int cg = 1; cg <= 2; ++cg) {
+    if (cta_group && cg != cta_group) continue;
+    for (int w : kWidths) {
+      if (bn && w != bn) continue;
+      ok = ok || variant_exists(w, cg);
+    }
   }
+  if (!ok) return GEMM_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
   g_override_bn = bn;
   g_override_group_m = group_m;
+  g_override_cta_group = cta_group;
   return GEMM_OK;
 }
 

@@ -15,9 +15,9 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(autouse=True)
 def _clean_state():
-    binding.gemm_set_config_override(0, 0)
+    binding.gemm_set_config_override(0, 0, 0)
     yield
-    binding.gemm_set_config_override(0, 0)
+    binding.gemm_set_config_override(0, 0, 0)
     assert binding.gemm_last_device_status() == 0
 
 
@@ -72,8 +72,11 @@ RAGGED = [
 @pytest.mark.parametrize("M,N,K", RAGGED)
 def test_ragged_shapes(prec, M, N, K):
     A, B = synth.make(prec, M, N, K, seed=1000 + M + N + K)
-    C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
-    check_against_oracle(prec, A, B, C, force_full=True)
+    ref, S = oracle_block(prec, A, B)
+    for cta_group in (0, 1, 2):
+        binding.gemm_set_config_override(0, 0, cta_group)
+        C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
+        assert_block(prec, C, ref, S, "cta_group=%d" % cta_group)
 
 
 @pytest.mark.parametrize("N", [1, 2, 3, 5, 30, 66, 131])
@@ -96,13 +99,17 @@ def test_minimal_k():
 
 
 # ------------------------------------------------ every tile width the selector has
-@pytest.mark.parametrize("bn", [32, 64, 128, 256])
+SHAPES = [(32, 1), (64, 1), (128, 1), (256, 1), (64, 2), (128, 2), (256, 2)]   # (BN, CTAs per tile)
+
+
+@pytest.mark.parametrize("bn,cta_group", SHAPES)
 @pytest.mark.parametrize("prec", synth.PRECISIONS)
-def test_every_tile_width(prec, bn):
-    M, N, K = 520, 1100, 1184           # several tiles in both directions + ragged tails
-    A, B = synth.make(prec, M, N, K, seed=bn)
-    binding.gemm_set_config_override(bn, 0)
-    assert ("BN=%d " % bn) in binding.gemm_query_config(prec, M, N, K)
+def test_every_tile_shape(prec, bn, cta_group):
+    M, N, K = 650, 1100, 1184           # several tiles in both directions + ragged tails
+    A, B = synth.make(prec, M, N, K, seed=bn + cta_group)
+    binding.gemm_set_config_override(bn, 0, cta_group)
+    cfg = binding.gemm_query_config(prec, M, N, K)
+    assert ("BN=%d " % bn) in cfg and ("cta_group=%d " % cta_group) in cfg
     C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
     check_against_oracle(prec, A, B, C, force_full=True)
 
@@ -111,8 +118,9 @@ def test_every_tile_width(prec, bn):
 def test_raster_band_heights(group_m):
     M, N, K = 1300, 1500, 256
     A, B = synth.s8_uniform(M, N, K, seed=group_m)
-    binding.gemm_set_config_override(64, group_m)
-    check_against_oracle("s8", A, B, run_gpu("s8", A, B, fill=-7), force_full=True)
+    for cta_group in (1, 2):
+        binding.gemm_set_config_override(64, group_m, cta_group)
+        check_against_oracle("s8", A, B, run_gpu("s8", A, B, fill=-7), force_full=True)
 
 
 # --------------------------------------------------------------- structured cases
@@ -125,8 +133,8 @@ def test_index_mapping_product_table():
     a[:, 0] = (np.arange(M) % 97) - 48
     b[:, 0] = (np.arange(N) % 89) - 44
     want = np.outer(a[:, 0].astype(np.int32), b[:, 0].astype(np.int32))
-    for bn in (0, 32, 64, 128, 256):
-        binding.gemm_set_config_override(bn, 0)
+    for bn, cta_group in [(0, 0)] + SHAPES:
+        binding.gemm_set_config_override(bn, 0, cta_group)
         assert np.array_equal(run_gpu("s8", a, b, fill=-7), want)
         got = run_gpu("fp16", a.astype(np.float16), b.astype(np.float16), fill=float("nan"))
         assert np.array_equal(got, want.astype(np.float32))
@@ -144,10 +152,12 @@ def test_one_hot_k_positions():
     for r, k in enumerate(ks):
         a[r, k] = 1
     eye = np.eye(len(ks), dtype=np.int32)
-    assert np.array_equal(run_gpu("s8", a, a, fill=-7), eye)
-    assert np.array_equal(run_gpu("s4", synth.pack_s4(a), synth.pack_s4(a), fill=-7), eye)
-    assert np.array_equal(run_gpu("fp16", a.astype(np.float16), a.astype(np.float16)),
-                          eye.astype(np.float32))
+    for cta_group in (1, 2):
+        binding.gemm_set_config_override(0, 0, cta_group)
+        assert np.array_equal(run_gpu("s8", a, a, fill=-7), eye)
+        assert np.array_equal(run_gpu("s4", synth.pack_s4(a), synth.pack_s4(a), fill=-7), eye)
+        assert np.array_equal(run_gpu("fp16", a.astype(np.float16), a.astype(np.float16)),
+                              eye.astype(np.float32))
 
 
 def test_all_ones_and_identity():
@@ -252,5 +262,4 @@ def test_argument_errors_enqueue_nothing():
     assert L.gemm_unpack_s4(4, 32, p, None, 32, None) == -1
     torch.cuda.synchronize()
     assert int((C != 5).sum()) == 0
-    assert binding.gemm_status_string if True else None
     assert L.gemm_status_string(-3).decode().startswith("K too large")

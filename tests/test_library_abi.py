@@ -1,0 +1,102 @@
+"""CPU-only checks of the boundary: the shared library loads, exports every
+symbol the header declares, and rejects bad arguments without a GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2608_10103_b200 import binding, build as lib_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "b200gemm.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    lib_build.build()
+    return binding.lib()
+
+
+def declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"\b(gemm_[a-z0-9_]+)\s*\(", text)
+    return sorted(set(names))
+
+
+def test_header_and_binding_agree():
+    assert declared_functions() == sorted(binding.EXPORTS)
+
+
+def test_every_declared_symbol_is_exported(lib):
+    for name in declared_functions():
+        assert getattr(lib, name) is not None
+
+
+def test_status_strings_and_version(lib):
+    assert binding.gemm_version() >= 1000
+    assert binding.gemm_status_string(0) == "ok"
+    for code in range(-7, 0):
+        assert binding.gemm_status_string(code) != "unknown status"
+    assert binding.gemm_status_string(-99) == "unknown status"
+
+
+def test_argument_validation_needs_no_gpu(lib):
+    # these are rejected before any CUDA call is made
+    assert lib.gemm_fp16(0, 8, 8, 16, 16, 16, None) == -1
+    assert lib.gemm_fp16(8, 8, 8, None, 16, 16, None) == -1
+    assert lib.gemm_fp16(8, 8, 12, 16, 16, 16, None) == -2
+    assert lib.gemm_fp16(8, 8, 8, 24, 16, 16, None) == -2
+    assert lib.gemm_s8(8, 8, 8, 16, 16, 16, None) == -2          # K % 16
+    assert lib.gemm_s8(8, 8, 131072, 16, 16, 16, None) == -3
+    assert lib.gemm_s4(8, 8, 16, 16, 16, 16, None) == -2         # K % 32
+    assert lib.gemm_s4(8, 8, 131104, 16, 16, 16, None) == -3
+    assert lib.gemm_s4_ws(8, 8, 32, 16, 16, 16, None, 0, None) == -1
+    assert lib.gemm_s4_ws(8, 8, 32, 16, 16, 16, 256, 16, None) == -6
+    assert lib.gemm_unpack_s4(4, 48, 16, 16, 48, None) == -2
+    assert lib.gemm_mma_peak_probe(2, 10, ctypes.pointer(ctypes.c_double(0)), None) == -1
+    assert lib.gemm_set_config_override(48, 0, 0) == -1
+    assert lib.gemm_set_config_override(32, 0, 2) == -1          # no 32-wide pair tile
+    assert lib.gemm_set_config_override(0, 0, 3) == -1
+    assert lib.gemm_set_config_override(0, 0, 0) == 0
+
+
+def test_workspace_size(lib):
+    assert binding.gemm_s4_workspace_bytes(0, 8, 32) == 0
+    assert binding.gemm_s4_workspace_bytes(8192, 8192, 8192) == 2 * 8192 * 8192
+    assert binding.gemm_s4_workspace_bytes(3, 5, 32) == 512      # each half rounded up to 256
+
+
+def test_selector_descriptions(lib):
+    cfg = binding.gemm_query_config("fp16", 8192, 8192, 8192)
+    assert "BN=256" in cfg and "cta_group=2" in cfg and "kind=f16" in cfg
+    assert "prepass=unpack_s4" in binding.gemm_query_config("s4", 4096, 4096, 4096)
+    binding.gemm_set_config_override(64, 3, 1)
+    try:
+        cfg = binding.gemm_query_config("s8", 1000, 1000, 1024)
+        assert "BM=128 BN=64 " in cfg and "group_m=3" in cfg and "tiles=%d" % (8 * 16) in cfg
+    finally:
+        binding.gemm_set_config_override(0, 0, 0)
+
+
+def test_binding_rejects_cpu_tensors(lib):
+    import torch
+    a = torch.zeros(8, 8, dtype=torch.float16)
+    with pytest.raises(TypeError):
+        binding.gemm_fp16(a, a, torch.zeros(8, 8))
+
+
+def test_product_path_never_touches_the_oracle():
+    """The library, its binding and its build script must not import or link the checker."""
+    pkg = os.path.join(ROOT, "paper_2608_10103_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in text and "from oracle" not in text, f
+                assert "gemm_oracle" not in text, f
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith((".py", ".c")):
+            text = open(os.path.join(ROOT, "oracle", f)).read()
+            assert "paper_2608_10103_b200" not in text and "b200gemm" not in text, f
