@@ -100,6 +100,41 @@ int gemm_s4_ws(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t*
                void* workspace, size_t workspace_bytes, gemm_stream_t stream);
 
 /*
+ * gemm_s4 for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: its INT4 kernels need no scratch.)
+ *
+ * Who needs it: a process that hands all device memory to its own pool at
+ * start-up (an inference server, a trainer running under a memory cap) cannot
+ * let a library call cudaMalloc behind its back -- it may fail, or break the
+ * budget -- and has no spare buffer to lend to gemm_s4_ws; and a latency-
+ * critical loop cannot afford the device-wide synchronisation that cudaMalloc
+ * and cudaFree imply, which gemm_s4 incurs whenever its workspace has to grow.
+ *
+ * This entry point computes exactly what gemm_s4 computes, but unpacks into a
+ * fixed 32 MiB array that is part of the library's device image.  It calls no
+ * cudaMalloc, cudaFree or other allocating routine.  Limits and rules:
+ *   - gemm_s4_workspace_bytes(M, N, K) must not exceed gemm_s4_static_capacity()
+ *     (32 MiB: M*K + N*K <= 2 * 4096 * 4096); larger problems are refused with
+ *     GEMM_ERR_TOO_LARGE and enqueue nothing.
+ *   - Every GPU on which the library is loaded holds the 32 MiB until the
+ *     process exits.
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress, with that device current).  Make that first call
+ *     before starting any stream capture.
+ *   - All calls on a device share the one array: calls that may overlap on the
+ *     GPU (different streams without an ordering between them) race on it and
+ *     give wrong results.  Calls on one stream are safe.  The array keeps the
+ *     previous call's bytes; each call rewrites every byte it later reads.
+ * Arguments, layouts, alignment (K % 32 == 0, 16-byte pointers, K <= 131071)
+ * and error codes are those of gemm_s4.
+ */
+int gemm_s4_static(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t* C,
+                   gemm_stream_t stream);
+
+/* Size in bytes of the fixed scratch behind gemm_s4_static. */
+size_t gemm_s4_static_capacity(void);
+
+/*
  * Frees the per-device workspaces held for gemm_s4 (synchronises).  Optional;
  * they are otherwise released when the process exits.
  */

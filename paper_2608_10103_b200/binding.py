@@ -21,7 +21,7 @@ PRECISION_ID = {"fp16": PREC_FP16, "s8": PREC_S8, "s4": PREC_S4}
 
 EXPORTS = (
     "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
-    "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
+    "gemm_s4_static", "gemm_s4_static_capacity", "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
     "gemm_set_config_override", "gemm_last_device_status", "gemm_last_cuda_error",
     "gemm_status_string", "gemm_version",
 )
@@ -59,6 +59,9 @@ def lib() -> ctypes.CDLL:
         L.gemm_s4_ws.argtypes = [i, i, i, vp, vp, vp, vp, sz, vp]
         L.gemm_s4_workspace_bytes.argtypes = [i, i, i]
         L.gemm_s4_workspace_bytes.restype = sz
+        L.gemm_s4_static.argtypes = [i, i, i, vp, vp, vp, vp]
+        L.gemm_s4_static_capacity.argtypes = []
+        L.gemm_s4_static_capacity.restype = sz
         L.gemm_unpack_s4.argtypes = [i, i, vp, vp, sz, vp]
         L.gemm_mma_peak_probe.argtypes = [i, i, ctypes.POINTER(ctypes.c_double), vp]
         L.gemm_query_config.argtypes = [i, i, i, i, ctypes.c_char_p, i]
@@ -67,7 +70,8 @@ def lib() -> ctypes.CDLL:
         L.gemm_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
             fn = getattr(L, name)
-            if name not in ("gemm_s4_workspace_bytes", "gemm_status_string"):
+            if name not in ("gemm_s4_workspace_bytes", "gemm_s4_static_capacity",
+                            "gemm_status_string"):
                 fn.restype = i
         _lib = L
     return _lib
@@ -156,6 +160,26 @@ def gemm_s4_ws(A: torch.Tensor, B: torch.Tensor, workspace: torch.Tensor,
                             _dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel(),
                             _stream_handle(stream)), "gemm_s4_ws")
     return C
+
+
+def gemm_s4_static(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor | None = None, stream=None):
+    """gemm_s4 without any device allocation inside the library: the unpacked
+    operands go to a fixed 32 MiB array in the library's device image.  Pass C
+    (preallocated) if the caller itself must not allocate either.  Problems
+    whose workspace exceeds gemm_s4_static_capacity() raise GemmError(-7)."""
+    M, Kh = A.shape
+    N, Khb = B.shape
+    if Kh != Khb:
+        raise ValueError("A and B disagree on K")
+    C = _out(C, M, N, torch.int32, A.device)
+    _check(lib().gemm_s4_static(M, N, 2 * Kh, _dev_ptr(A, torch.uint8, "A"),
+                                _dev_ptr(B, torch.uint8, "B"), _dev_ptr(C, torch.int32, "C"),
+                                _stream_handle(stream)), "gemm_s4_static")
+    return C
+
+
+def gemm_s4_static_capacity() -> int:
+    return int(lib().gemm_s4_static_capacity())
 
 
 def gemm_unpack_s4(packed: torch.Tensor, out: torch.Tensor | None = None, stream=None):

@@ -492,3 +492,63 @@ const char* gemm_status_string(int status) {
 int gemm_version(void) { return 1000; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// gemm_s4_static: the INT4 GEMM for callers that must not allocate.
+//
+// The int8 images of A and B that gemm_s4 keeps in a cudaMalloc'ed workspace
+// live here in a fixed array inside the library's device image, so the call
+// needs no allocator at all.  Cost: every GPU that loads the library carries
+// the array until the process exits.
+// ---------------------------------------------------------------------------
+namespace b200gemm {
+namespace {
+
+constexpr size_t kStaticScratchBytes = 32u << 20;  // 32 MiB: up to M*K + N*K = 2 * 4096 * 4096
+
+static __device__ __align__(256) unsigned char g_s4_static_scratch[kStaticScratchBytes];
+
+// In host code the array's name is only a handle for the runtime, not a device
+// address: the address a kernel can use is looked up once per device.
+void* g_s4_static_ptr[MAX_DEVICES] = {};
+std::mutex g_s4_static_mutex;
+
+int static_scratch_for_current_device(void** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= MAX_DEVICES) return GEMM_ERR_UNSUPPORTED_DEVICE;
+  std::lock_guard<std::mutex> lock(g_s4_static_mutex);
+  if (!g_s4_static_ptr[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_s4_static_scratch);  // resolves for the current device
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (!ptr || (reinterpret_cast<uintptr_t>(ptr) & 255)) return cuda_fail(cudaErrorInvalidSymbol);
+    g_s4_static_ptr[dev] = ptr;
+  }
+  *out = g_s4_static_ptr[dev];
+  return GEMM_OK;
+}
+
+}  // namespace
+}  // namespace b200gemm
+
+extern "C" {
+
+size_t gemm_s4_static_capacity(void) { return b200gemm::kStaticScratchBytes; }
+
+int gemm_s4_static(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t* C,
+                   gemm_stream_t stream) {
+  int rc = check_s4(M, N, K, A, B, C);
+  if (rc != GEMM_OK) return rc;
+  if (gemm_s4_workspace_bytes(M, N, K) > kStaticScratchBytes) return GEMM_ERR_TOO_LARGE;
+  void* scratch = nullptr;
+  rc = static_scratch_for_current_device(&scratch);
+  if (rc != GEMM_OK) return rc;
+  // Every byte of the scratch that the GEMM reads is rewritten by the unpack
+  // launches of this call, so nothing left over from an earlier call is used.
+  return gemm_s4_ws(M, N, K, A, B, C, scratch, kStaticScratchBytes, stream);
+}
+
+}  // extern "C"
+
