@@ -153,13 +153,20 @@ int gemm_unpack_s4(int rows, int K, const uint8_t* packed, int8_t* out, size_t o
 
 /*
  * Measurement aid (Sec. III-B profiles every kernel against the hardware's
- * limits): runs `iters` back-to-back tcgen05.mma instructions of the production
- * tile shape per SM on shared-memory operands that are never reloaded, on
- * every SM, and adds the operation count it performed to *ops_out (host
- * pointer).  Time it with events on `stream` to get the MMA-issue-only peak of
- * the given precision (GEMM_PREC_FP16 or GEMM_PREC_S8).
+ * limits): every SM issues `iters` back-to-back tcgen05.mma instructions of
+ * shape 128 x n_cols x (32 bytes of K) on shared-memory operands that are never
+ * reloaded, and the operation count performed is added to *ops_out (host
+ * pointer).  n_cols: multiple of 16 up to 256 (256 = the production tile).
+ * iters is rounded down to a multiple of 4 (MMAs are issued in groups of 4, one
+ * k-block of the GEMM kernels).  commit_every: 0 = none inside the loop; c > 0 =
+ * a tcgen05.commit after every c groups, as a pipelined GEMM does once per
+ * k-block (c = 1).
+ * Time it with events on `stream` for the MMA-issue-only rate of the given
+ * precision (GEMM_PREC_FP16 or GEMM_PREC_S8); with tracing on, words [0] and
+ * [1] of each CTA's trace record hold the cycles and nanoseconds of the loop.
  */
-int gemm_mma_peak_probe(int precision, int iters, double* ops_out, gemm_stream_t stream);
+int gemm_mma_peak_probe(int precision, int iters, int n_cols, int commit_every, double* ops_out,
+                        gemm_stream_t stream);
 
 /*
  * Writes a human-readable description of the tile configuration the selector
@@ -184,6 +191,28 @@ int gemm_set_config_override(int bn, int group_m, int cta_group);
  * 1/2/3 = producer / MMA / epilogue wait expired.
  */
 int gemm_last_device_status(void);
+
+/*
+ * Cycle accounting, in the spirit of the counter attribution the paper does
+ * with its profiler (Sec. III-B).  gemm_trace_enable(1) makes later GEMM
+ * launches record, per CTA, 12 unsigned 64-bit words: [0] SM cycles and [1]
+ * nanoseconds the CTA ran (their ratio is the SM clock during the kernel),
+ * cycles the producer waited for a free slot [2], the MMA issuer waited for
+ * operands [3] and for a free accumulator [4], one epilogue warp waited for a
+ * finished accumulator [5] and spent draining [6], the tile count [7], and the
+ * issuer's cycles inside tcgen05.mma [8], tcgen05.commit [9] and fence +
+ * descriptor set-up [10], and the producer's cycles issuing loads [11].
+ * gemm_trace_read synchronises the device, copies the words of the first
+ * min(max_ctas, 160) CTAs of the last traced launch to `out` (host memory,
+ * 12 * max_ctas words) and returns that CTA count.  Off by default; the cost
+ * when on is a few clock reads per k-block.
+ * `on` is a bit set: 1 = record; 2 = ablation, issue no MMAs (operand loads and
+ * barriers only); 4 = ablation, issue no operand loads (MMAs and barriers only,
+ * on whatever shared memory holds).  With an ablation bit set C is garbage; the
+ * bits exist to attribute cycles to the load path or the MMA path.
+ */
+int gemm_trace_enable(int on);
+int gemm_trace_read(unsigned long long* out, int max_ctas);
 
 /* cudaError_t value of the last failed CUDA call made by this library, or 0. */
 int gemm_last_cuda_error(void);

@@ -22,7 +22,7 @@ PRECISION_ID = {"fp16": PREC_FP16, "s8": PREC_S8, "s4": PREC_S4}
 EXPORTS = (
     "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
     "gemm_s4_static", "gemm_s4_static_capacity", "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
-    "gemm_set_config_override", "gemm_last_device_status", "gemm_last_cuda_error",
+    "gemm_set_config_override", "gemm_trace_enable", "gemm_trace_read", "gemm_last_device_status", "gemm_last_cuda_error",
     "gemm_status_string", "gemm_version",
 )
 
@@ -63,9 +63,11 @@ def lib() -> ctypes.CDLL:
         L.gemm_s4_static_capacity.argtypes = []
         L.gemm_s4_static_capacity.restype = sz
         L.gemm_unpack_s4.argtypes = [i, i, vp, vp, sz, vp]
-        L.gemm_mma_peak_probe.argtypes = [i, i, ctypes.POINTER(ctypes.c_double), vp]
+        L.gemm_mma_peak_probe.argtypes = [i, i, i, i, ctypes.POINTER(ctypes.c_double), vp]
         L.gemm_query_config.argtypes = [i, i, i, i, ctypes.c_char_p, i]
         L.gemm_set_config_override.argtypes = [i, i, i]
+        L.gemm_trace_enable.argtypes = [i]
+        L.gemm_trace_read.argtypes = [ctypes.POINTER(ctypes.c_ulonglong), i]
         L.gemm_status_string.argtypes = [i]
         L.gemm_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -198,11 +200,13 @@ def gemm_release_workspaces():
     _check(lib().gemm_release_workspaces(), "gemm_release_workspaces")
 
 
-def gemm_mma_peak_probe(precision: str, iters: int, stream=None) -> float:
+def gemm_mma_peak_probe(precision: str, iters: int, n_cols: int = 256, commit_every: int = 0,
+                        stream=None) -> float:
     """Launches the MMA-only probe; returns the operation count it performs."""
     ops = ctypes.c_double(0.0)
-    _check(lib().gemm_mma_peak_probe(PRECISION_ID[precision], iters, ctypes.byref(ops),
-                                     _stream_handle(stream)), "gemm_mma_peak_probe")
+    _check(lib().gemm_mma_peak_probe(PRECISION_ID[precision], iters, n_cols, commit_every,
+                                     ctypes.byref(ops), _stream_handle(stream)),
+           "gemm_mma_peak_probe")
     return ops.value
 
 
@@ -214,6 +218,26 @@ def gemm_query_config(precision: str, M: int, N: int, K: int) -> str:
 
 def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0):
     _check(lib().gemm_set_config_override(bn, group_m, cta_group), "gemm_set_config_override")
+
+
+TRACE_FIELDS = ("cycles", "nanos", "producer_wait", "mma_wait_operands", "mma_wait_accumulator",
+                "epilogue_wait", "epilogue_busy", "tiles", "mma_issue", "mma_commit", "mma_fence",
+                "producer_issue")
+TRACE_SLOTS = len(TRACE_FIELDS)
+
+
+def gemm_trace_enable(flags: int = 1):
+    """1 = record cycles; +2 = issue no MMAs; +4 = issue no operand loads; 0 = off."""
+    _check(lib().gemm_trace_enable(int(flags)), "gemm_trace_enable")
+
+
+def gemm_trace_read(max_ctas: int = 160):
+    """Per-CTA cycle accounting of the last traced launch: list of dicts."""
+    buf = (ctypes.c_ulonglong * (TRACE_SLOTS * max_ctas))()
+    n = lib().gemm_trace_read(buf, max_ctas)
+    if n < 0:
+        raise GemmError(n, "gemm_trace_read")
+    return [dict(zip(TRACE_FIELDS, buf[TRACE_SLOTS * c: TRACE_SLOTS * (c + 1)])) for c in range(n)]
 
 
 def gemm_last_device_status() -> int:

@@ -21,10 +21,14 @@ constexpr int K_LIMIT_INT = 131071;  // 128*128*K and 16384*K stay below 2^31
 
 __device__ int g_device_status = 0;
 
+constexpr int TRACE_MAX_CTAS = 160;
+__device__ unsigned long long g_trace[TRACE_MAX_CTAS * TRACE_SLOTS];
+
 struct DeviceState {
   bool ready = false;
   int num_sms = 0;
   int* status_ptr = nullptr;
+  unsigned long long* trace_ptr = nullptr;
   void* s4_workspace = nullptr;
   size_t s4_workspace_bytes = 0;
   uint64_t attr_set = 0;  // bit i: dynamic-smem attribute set for kernel variant i
@@ -36,6 +40,7 @@ int g_last_cuda_error = 0;
 int g_override_bn = 0;
 int g_override_group_m = 0;
 int g_override_cta_group = 0;
+int g_trace_on = 0;
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                    const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -63,6 +68,8 @@ int device_state(DeviceState** out) {
     e = cudaDeviceGetAttribute(&s.num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return cuda_fail(e);
     e = cudaGetSymbolAddress(reinterpret_cast<void**>(&s.status_ptr), g_device_status);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&s.trace_ptr), g_trace);
     if (e != cudaSuccess) return cuda_fail(e);
     if (!g_encode) {
       void* fn = nullptr;
@@ -96,6 +103,24 @@ int encode_operand_map(CUtensorMap* map, CUtensorMapDataType type, int elem_byte
   return GEMM_OK;
 }
 
+// C (or any row-major 32-bit matrix) for the epilogue's TMA stores: boxes of 32 rows x
+// 32 values (128 bytes), 128-byte swizzle.  Needs a 16-byte aligned base and pitch.
+int encode_c_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 4};
+  cuuint32_t box[2] = {32, 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(ptr), dims,
+                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda_error = static_cast<int>(cudaErrorInvalidValue);
+    return GEMM_ERR_CUDA;
+  }
+  return GEMM_OK;
+}
+
 // ------------------------------------------------------------------ selector
 struct TileConfig {
   int bn;
@@ -106,14 +131,17 @@ struct TileConfig {
 
 constexpr int kWidths[] = {256, 128, 64, 32};
 
+// Ring depth and 128-byte K atoms per slot of each built shape.
 int stages_for(int bn, int cta_group) {
-  if (cta_group == 2) return bn == 256 ? 6 : 8;
+  if (cta_group == 2) return bn == 256 ? 3 : 4;
   switch (bn) {
     case 256: return 4;
-    case 128: return 6;
-    default: return 8;
+    case 128: return 3;
+    default: return 4;
   }
 }
+
+int atoms_for(int bn, int cta_group) { return (cta_group == 1 && bn == 256) ? 1 : 2; }
 
 bool variant_exists(int bn, int cta_group) {
   if (cta_group == 1) return bn == 256 || bn == 128 || bn == 64 || bn == 32;
@@ -161,11 +189,11 @@ TileConfig select_config(int M, int N, int num_sms) {
   return best;
 }
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP>
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB>
 int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUtensorMap& tb,
-                   const GemmParams& p, cudaStream_t stream) {
-  using L = SmemLayout<BN, STAGES, CTA_GROUP>;
-  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP>;
+                   const CUtensorMap& tc, const GemmParams& p, cudaStream_t stream) {
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB>;
+  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB>;
   if (!(s->attr_set & (1ull << variant))) {
     cudaError_t e =
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
@@ -187,7 +215,7 @@ int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUt
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, p);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, tc, p);
   if (e != cudaSuccess) return cuda_fail(e);
   return GEMM_OK;
 }
@@ -220,23 +248,32 @@ int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* 
   p.group_m = cfg.group_m;
   p.k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
   p.c_vec_ok = (N % 4 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+  CUtensorMap tc;
+  if (p.c_vec_ok) {
+    rc = encode_c_map(&tc, C, M, N);
+    if (rc != GEMM_OK) return rc;
+  } else {
+    tc = ta;  // unused by the kernel on the plain-store path
+  }
   p.C = static_cast<uint32_t*>(C);
   p.status = s->status_ptr;
+  p.trace = (g_trace_on & 1) ? s->trace_ptr : nullptr;
+  p.ablate = (g_trace_on >> 1) & 3;
 
   const int kbase = (KIND == ptx::KIND_F16) ? 0 : 16;
   if (cfg.cta_group == 2) {
     switch (cfg.bn) {
-      case 256: return launch_variant<KIND, 256, 6, 2>(s, kbase + 8, ta, tb, p, stream);
-      case 128: return launch_variant<KIND, 128, 8, 2>(s, kbase + 9, ta, tb, p, stream);
-      case 64: return launch_variant<KIND, 64, 8, 2>(s, kbase + 10, ta, tb, p, stream);
+      case 256: return launch_variant<KIND, 256, 3, 2, 2>(s, kbase + 8, ta, tb, tc, p, stream);
+      case 128: return launch_variant<KIND, 128, 4, 2, 2>(s, kbase + 9, ta, tb, tc, p, stream);
+      case 64: return launch_variant<KIND, 64, 4, 2, 2>(s, kbase + 10, ta, tb, tc, p, stream);
       default: return GEMM_ERR_INVALID_ARG;
     }
   }
   switch (cfg.bn) {
-    case 256: return launch_variant<KIND, 256, 4, 1>(s, kbase + 0, ta, tb, p, stream);
-    case 128: return launch_variant<KIND, 128, 6, 1>(s, kbase + 1, ta, tb, p, stream);
-    case 64: return launch_variant<KIND, 64, 8, 1>(s, kbase + 2, ta, tb, p, stream);
-    case 32: return launch_variant<KIND, 32, 8, 1>(s, kbase + 3, ta, tb, p, stream);
+    case 256: return launch_variant<KIND, 256, 4, 1, 1>(s, kbase + 0, ta, tb, tc, p, stream);
+    case 128: return launch_variant<KIND, 128, 3, 1, 2>(s, kbase + 1, ta, tb, tc, p, stream);
+    case 64: return launch_variant<KIND, 64, 4, 1, 2>(s, kbase + 2, ta, tb, tc, p, stream);
+    case 32: return launch_variant<KIND, 32, 4, 1, 2>(s, kbase + 3, ta, tb, tc, p, stream);
     default: return GEMM_ERR_INVALID_ARG;
   }
 }
@@ -384,32 +421,35 @@ int gemm_unpack_s4(int rows, int K, const uint8_t* packed, int8_t* out, size_t o
   return launch_unpack(rows, K, packed, out, out_pitch, reinterpret_cast<cudaStream_t>(stream));
 }
 
-int gemm_mma_peak_probe(int precision, int iters, double* ops_out, gemm_stream_t stream) {
-  if (iters <= 0 || !ops_out || (precision != GEMM_PREC_FP16 && precision != GEMM_PREC_S8))
+int gemm_mma_peak_probe(int precision, int iters, int n_cols, int commit_every, double* ops_out,
+                        gemm_stream_t stream) {
+  if (iters <= 0 || !ops_out || (precision != GEMM_PREC_FP16 && precision != GEMM_PREC_S8) ||
+      n_cols < 16 || n_cols > PROBE_BN || n_cols % 16 || commit_every < 0)
     return GEMM_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
   DeviceState* s = nullptr;
   int rc = device_state(&s);
   if (rc != GEMM_OK) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  unsigned long long* trace = (g_trace_on & 1) ? s->trace_ptr : nullptr;
   cudaError_t e;
   int k_per_mma;
   if (precision == GEMM_PREC_FP16) {
     auto kernel = mma_peak_probe_kernel<ptx::KIND_F16>;
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PROBE_SMEM);
     if (e != cudaSuccess) return cuda_fail(e);
-    kernel<<<s->num_sms, 128, PROBE_SMEM, st>>>(iters, s->status_ptr);
+    kernel<<<s->num_sms, 128, PROBE_SMEM, st>>>(iters, n_cols, commit_every, s->status_ptr, trace);
     k_per_mma = MMA_K_BYTES / 2;
   } else {
     auto kernel = mma_peak_probe_kernel<ptx::KIND_I8>;
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PROBE_SMEM);
     if (e != cudaSuccess) return cuda_fail(e);
-    kernel<<<s->num_sms, 128, PROBE_SMEM, st>>>(iters, s->status_ptr);
+    kernel<<<s->num_sms, 128, PROBE_SMEM, st>>>(iters, n_cols, commit_every, s->status_ptr, trace);
     k_per_mma = MMA_K_BYTES;
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
-  *ops_out += 2.0 * BM * PROBE_BN * k_per_mma * static_cast<double>(iters) * s->num_sms;
+  *ops_out += 2.0 * BM * n_cols * k_per_mma * static_cast<double>(iters / 4 * 4) * s->num_sms;
   return GEMM_OK;
 }
 
@@ -431,7 +471,7 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
   const long long units = num_sms / c.cta_group;
   snprintf(buf, static_cast<size_t>(len),
            "BM=%d BN=%d BK=%d cta_group=%d stages=%d group_m=%d tiles=%lld ctas=%lld kind=%s%s",
-           BM * c.cta_group, c.bn, BK_BYTES / elem, c.cta_group, c.stages, c.group_m, tiles,
+           BM * c.cta_group, c.bn, atoms_for(c.bn, c.cta_group) * BK_BYTES / elem, c.cta_group, c.stages, c.group_m, tiles,
            (tiles < units ? tiles : units) * c.cta_group,
            precision == GEMM_PREC_FP16 ? "f16" : "i8",
            precision == GEMM_PREC_S4 ? " prepass=unpack_s4" : "");
@@ -471,6 +511,28 @@ int gemm_last_device_status(void) {
     if (e != cudaSuccess) return cuda_fail(e);
   }
   return v;
+}
+
+int gemm_trace_enable(int on) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  g_trace_on = on & 7;
+  return GEMM_OK;
+}
+
+int gemm_trace_read(unsigned long long* out, int max_ctas) {
+  static_assert(TRACE_SLOTS == 12, "header documents 12 words per CTA");
+  if (!out || max_ctas <= 0) return GEMM_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceState* s = nullptr;
+  int rc = device_state(&s);
+  if (rc != GEMM_OK) return rc;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e);
+  const int n = max_ctas < TRACE_MAX_CTAS ? max_ctas : TRACE_MAX_CTAS;
+  e = cudaMemcpy(out, s->trace_ptr, sizeof(unsigned long long) * TRACE_SLOTS * n,
+                 cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return n;
 }
 
 int gemm_last_cuda_error(void) { return g_last_cuda_error; }

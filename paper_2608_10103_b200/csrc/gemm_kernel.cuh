@@ -61,20 +61,51 @@ struct GemmParams {
   int M, N, K;
   int tiles_m, tiles_n;  // number of C tiles (128*CTA_GROUP x BN) along M and N
   int group_m;           // raster: tiles are walked in bands of `group_m` tile rows
-  int k_blocks;          // ceil(K bytes / BK_BYTES)
-  int c_vec_ok;          // 1 if C rows allow 16-byte vector stores (N % 4 == 0, base aligned)
+  int k_blocks;          // ceil(K bytes / BK_BYTES): 128-byte K atoms to cover K
+  int c_vec_ok;          // 1 if C rows allow 16-byte accesses (N % 4 == 0, base 16-byte aligned):
+                         // the epilogue then stages C in shared memory and stores it by TMA
   uint32_t* C;
   int* status;           // device status word (0 = ok)
+  // Optional per-CTA cycle accounting (TRACE_SLOTS 64-bit words per CTA), or null.
+  unsigned long long* trace;
+  // Ablation switches for cycle accounting runs (results are then meaningless):
+  // bit 0 = issue no MMAs (loads + barriers only), bit 1 = issue no loads (MMAs + barriers only).
+  int ablate;
 };
 
-template <int BN, int STAGES, int CTA_GROUP>
+// Trace slots written per CTA when GemmParams::trace is set.
+enum TraceSlot {
+  TRACE_CYCLES = 0,         // SM cycles from kernel start to teardown
+  TRACE_NANOS = 1,          // the same interval in ns of %globaltimer
+  TRACE_PROD_WAIT = 2,      // producer: cycles waiting for a free slot
+  TRACE_MMA_WAIT_FULL = 3,  // MMA issuer: cycles waiting for operands
+  TRACE_MMA_WAIT_ACC = 4,   // MMA issuer: cycles waiting for a free accumulator buffer
+  TRACE_EPI_WAIT = 5,       // epilogue warp 2: cycles waiting for a finished accumulator
+  TRACE_EPI_BUSY = 6,       // epilogue warp 2: cycles draining accumulators
+  TRACE_TILES = 7,          // tiles this CTA worked on
+  TRACE_MMA_ISSUE = 8,      // MMA issuer: cycles inside the tcgen05.mma issue instructions
+  TRACE_MMA_COMMIT = 9,     // MMA issuer: cycles inside tcgen05.commit
+  TRACE_MMA_FENCE = 10,     // MMA issuer: cycles in the fence + descriptor set-up
+  TRACE_PROD_ISSUE = 11,    // producer: cycles issuing expect_tx + TMA loads
+  TRACE_SLOTS = 12
+};
+
+// One ring slot holds KB "atoms" per operand; an atom is a tile of rows x 128
+// bytes of K in the 128-byte-swizzle layout (the widest a swizzled TMA box can
+// be).  KB = 2 halves the per-slot barrier work (one wait, one commit per 8 MMAs)
+// of the single issuing thread, whose instruction time is the scarce resource.
+template <int BN, int STAGES, int CTA_GROUP, int KB>
 struct SmemLayout {
   static constexpr int B_ROWS = BN / CTA_GROUP;  // B rows each CTA loads
-  static constexpr int A_BYTES = BM * BK_BYTES;
-  static constexpr int B_BYTES = B_ROWS * BK_BYTES;
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int A_BYTES = BM * BK_BYTES;       // one A atom
+  static constexpr int B_BYTES = B_ROWS * BK_BYTES;   // one B atom
+  static constexpr int STAGE_BYTES = KB * (A_BYTES + B_BYTES);
   static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
-  static constexpr int BAR_OFFSET = RING_BYTES;
+  // Epilogue staging: per epilogue warp two buffers of 32 rows x 128 bytes (32 x 32 C values).
+  static constexpr int EPI_BUF_BYTES = 32 * 128;
+  static constexpr int EPI_OFFSET = RING_BYTES;
+  static constexpr int EPI_BYTES = EPI_WARPS * 2 * EPI_BUF_BYTES;
+  static constexpr int BAR_OFFSET = EPI_OFFSET + EPI_BYTES;
   // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], drain
   static constexpr int NUM_BARS = 2 * STAGES + 5;
   static constexpr int MISC_OFFSET = BAR_OFFSET + NUM_BARS * 8;
@@ -120,11 +151,11 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int t, int& tm,
   tn = r / rows_in_band;
 }
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP>
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-            const GemmParams p) {
-  using L = SmemLayout<BN, STAGES, CTA_GROUP>;
+            const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB>;
   constexpr int ELEM_BYTES = (KIND == ptx::KIND_F16) ? 2 : 1;
   constexpr int BK_ELEMS = BK_BYTES / ELEM_BYTES;
   constexpr int TILE_M = BM * CTA_GROUP;
@@ -152,8 +183,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   const uint32_t cta_rank = (CTA_GROUP == 2) ? ptx::cluster_ctarank() : 0u;
   const bool leader = (cta_rank == 0);
   const int num_tiles = p.tiles_m * p.tiles_n;
+  const int k_slots = (p.k_blocks + KB - 1) / KB;  // ring slots per tile; a K tail is zero-filled
   const int first_tile = static_cast<int>(blockIdx.x) / CTA_GROUP;
   const int tile_stride = static_cast<int>(gridDim.x) / CTA_GROUP;
+  unsigned long long* const trace =
+      p.trace ? p.trace + static_cast<size_t>(blockIdx.x) * TRACE_SLOTS : nullptr;
+  const long long clk_start = trace ? clock64() : 0;
+  const uint64_t ns_start = trace ? ptx::globaltimer_ns() : 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -169,6 +205,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmap_a);
     ptx::prefetch_tensormap(&tmap_b);
+    ptx::prefetch_tensormap(&tmap_c);
   }
   if (warp == 1) {
     ptx::tmem_alloc<CTA_GROUP>(ptx::smem_addr(const_cast<uint32_t*>(tmem_holder)), TMEM_COLS);
@@ -190,31 +227,50 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       uint32_t phase = 0;
       int issued = 0;
       bool ok = true;
+      long long waited = 0, prod_issue = 0;
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
         int tm, tn;
         tile_coords(p, t, tm, tn);
         const int a_row = tm * TILE_M + static_cast<int>(cta_rank) * BM;
         const int b_row = tn * BN + static_cast<int>(cta_rank) * L::B_ROWS;
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int ks = 0; ks < k_slots; ++ks) {
+          const long long w0 = trace ? clock64() : 0;
           ok = wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status,
                             DEV_TIMEOUT_PRODUCER);
+          const long long w9 = trace ? clock64() : 0;
+          if (trace) waited += w9 - w0;
           if (!ok) break;
           const uint32_t a_dst = base + stage * L::STAGE_BYTES;
-          const uint32_t b_dst = a_dst + L::A_BYTES;
-          if constexpr (CTA_GROUP == 1) {
+          const uint32_t b_dst = a_dst + KB * L::A_BYTES;
+          if (p.ablate & 2) {
+            if (leader) ptx::mbar_arrive(full_bar(stage));
+          } else if constexpr (CTA_GROUP == 1) {
             ptx::mbar_arrive_expect_tx(full_bar(stage), L::STAGE_BYTES);
-            ptx::tma_load_2d(a_dst, &tmap_a, kb * BK_ELEMS, a_row, full_bar(stage));
-            ptx::tma_load_2d(b_dst, &tmap_b, kb * BK_ELEMS, b_row, full_bar(stage));
+#pragma unroll
+            for (int a = 0; a < KB; ++a) {
+              const int k0 = (ks * KB + a) * BK_ELEMS;
+              ptx::tma_load_2d(a_dst + a * L::A_BYTES, &tmap_a, k0, a_row, full_bar(stage));
+              ptx::tma_load_2d(b_dst + a * L::B_BYTES, &tmap_b, k0, b_row, full_bar(stage));
+            }
           } else {
             // Bytes of both CTAs are counted on the leader's barrier.
             if (leader) ptx::mbar_arrive_expect_tx(full_bar(stage), 2 * L::STAGE_BYTES);
             const uint32_t lead_full = ptx::map_to_cta(full_bar(stage), 0);
-            ptx::tma_load_2d_pair(a_dst, &tmap_a, kb * BK_ELEMS, a_row, lead_full);
-            ptx::tma_load_2d_pair(b_dst, &tmap_b, kb * BK_ELEMS, b_row, lead_full);
+#pragma unroll
+            for (int a = 0; a < KB; ++a) {
+              const int k0 = (ks * KB + a) * BK_ELEMS;
+              ptx::tma_load_2d_pair(a_dst + a * L::A_BYTES, &tmap_a, k0, a_row, lead_full);
+              ptx::tma_load_2d_pair(b_dst + a * L::B_BYTES, &tmap_b, k0, b_row, lead_full);
+            }
           }
           ++issued;
+          if (trace) prod_issue += clock64() - w9;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
+      }
+      if (trace) {
+        trace[TRACE_PROD_WAIT] = static_cast<unsigned long long>(waited);
+        trace[TRACE_PROD_ISSUE] = static_cast<unsigned long long>(prod_issue);
       }
       if (!ok && (CTA_GROUP == 1 || leader)) {
         // Gave up: let the copies already in flight land before the CTA exits.
@@ -238,29 +294,50 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
+      long long wait_full = 0, wait_acc = 0, t_fence = 0, t_issue = 0, t_commit = 0;
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
+        const long long w0 = trace ? clock64() : 0;
         ok = wait_bounded(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, p.status,
                           DEV_TIMEOUT_MMA);
+        if (trace) wait_acc += clock64() - w0;
         if (!ok) break;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int ks = 0; ks < k_slots; ++ks) {
+          const long long w1 = trace ? clock64() : 0;
           ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
+          const long long w2 = trace ? clock64() : 0;
+          if (trace) wait_full += w2 - w1;
           if (!ok) break;
           ptx::tc_fence_after_sync();
           const uint32_t a_src = base + stage * L::STAGE_BYTES;
           const uint64_t a_desc = ptx::smem_desc_sw128(a_src);
-          const uint64_t b_desc = ptx::smem_desc_sw128(a_src + L::A_BYTES);
+          const uint64_t b_desc = ptx::smem_desc_sw128(a_src + KB * L::A_BYTES);
+          const long long w3 = trace ? clock64() : 0;
+          if (!(p.ablate & 1)) {
 #pragma unroll
-          for (int kk = 0; kk < BK_BYTES / MMA_K_BYTES; ++kk) {
-            const uint64_t step = static_cast<uint64_t>((kk * MMA_K_BYTES) >> 4);
-            ptx::mma_ss<KIND, CTA_GROUP>(d_tmem, a_desc + step, b_desc + step, idesc,
-                                         (kb > 0 || kk > 0) ? 1u : 0u);
+            for (int a = 0; a < KB; ++a) {
+#pragma unroll
+              for (int kk = 0; kk < BK_BYTES / MMA_K_BYTES; ++kk) {
+                // descriptor addresses are in 16-byte units
+                const uint64_t a_step = static_cast<uint64_t>((a * L::A_BYTES + kk * MMA_K_BYTES) >> 4);
+                const uint64_t b_step = static_cast<uint64_t>((a * L::B_BYTES + kk * MMA_K_BYTES) >> 4);
+                ptx::mma_ss<KIND, CTA_GROUP>(d_tmem, a_desc + a_step, b_desc + b_step, idesc,
+                                             (ks > 0 || a > 0 || kk > 0) ? 1u : 0u);
+              }
+            }
           }
+          const long long w4 = trace ? clock64() : 0;
           if constexpr (CTA_GROUP == 1) {
             ptx::mma_commit<1>(empty_bar(stage));
           } else {
             ptx::mma_commit_pair(empty_bar(stage), 0x3);
+          }
+          if (trace) {
+            const long long w5 = clock64();
+            t_fence += w3 - w2;
+            t_issue += w4 - w3;
+            t_commit += w5 - w4;
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -272,6 +349,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         }
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
+      }
+      if (trace) {
+        trace[TRACE_MMA_WAIT_FULL] = static_cast<unsigned long long>(wait_full);
+        trace[TRACE_MMA_WAIT_ACC] = static_cast<unsigned long long>(wait_acc);
+        trace[TRACE_MMA_ISSUE] = static_cast<unsigned long long>(t_issue);
+        trace[TRACE_MMA_COMMIT] = static_cast<unsigned long long>(t_commit);
+        trace[TRACE_MMA_FENCE] = static_cast<unsigned long long>(t_fence);
       }
       if (!ok) {
         // Gave up: wait for the MMAs already issued before TMEM is released.
@@ -286,33 +370,67 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     // ---------------------------------------------------------------- epilogue
     const int quarter = warp & 3;  // TMEM lane quarter this warp may read
     const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
+    const uint32_t epi_base =
+        base + L::EPI_OFFSET + static_cast<uint32_t>((warp - 2) * 2 * L::EPI_BUF_BYTES);
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
+    long long epi_wait = 0, epi_busy = 0, tiles_done = 0;
     for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
       int tm, tn;
       tile_coords(p, t, tm, tn);
+      const long long w0 = trace ? clock64() : 0;
       ok = wait_bounded(acc_full_bar(acc), acc_phase, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
+      const long long w1 = trace ? clock64() : 0;
+      epi_wait += w1 - w0;
       if (!ok) break;
       ptx::tc_fence_after_sync();
-      const int row = tm * TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32 + lane;
+      const int row0 = tm * TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
+      const int row = row0 + lane;
       const int col0 = tn * BN;
-      uint32_t* crow = p.C + static_cast<size_t>(row) * p.N;
+      if (p.c_vec_ok) {
+        // TMEM -> registers -> swizzled shared memory -> one TMA store per 32 x 32 block.
+        // Thread `lane` owns row `lane` of the block; 16-byte chunk j of the row goes to
+        // chunk j ^ (lane & 7), the 128-byte swizzle the C tensor map expects, which also
+        // spreads the warp's 16-byte stores over all banks.
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t r[32];
-        ptx::tmem_ld_32x32b_x32(tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32),
-                                r);
-        ptx::tmem_wait_ld();
-        const int col = col0 + c * 32;
-        if (row < p.M) {
-          if (p.c_vec_ok && col + 32 <= p.N) {
-            uint4* dst = reinterpret_cast<uint4*>(crow + col);
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32b_x32(
+              tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), r);
+          const uint32_t buf = epi_base + static_cast<uint32_t>((c & 1) * L::EPI_BUF_BYTES);
+          // the store issued from this buffer two blocks ago must have read it
+          if (lane == 0) ptx::bulk_wait_group_read<1>();
+          __syncwarp();
+          ptx::tmem_wait_ld();
+          const uint32_t row_addr = buf + static_cast<uint32_t>(lane * 128);
 #pragma unroll
-            for (int v = 0; v < 8; ++v)
-              dst[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
-          } else {
+          for (int j = 0; j < 8; ++j)
+            ptx::st_shared_v4(row_addr + static_cast<uint32_t>(((j ^ (lane & 7)) * 16)), r[4 * j],
+                              r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          // Partly outside C: the hardware clips.  Wholly outside: issue no store, but still
+          // close a (then empty) group so that "one group per block" keeps the buffer
+          // reuse rule above exact.
+          if (lane == 0) {
+            if (row0 < p.M && col0 + c * 32 < p.N)
+              ptx::tma_store_2d(&tmap_c, col0 + c * 32, row0, buf);
+            ptx::bulk_commit_group();
+          }
+        }
+      } else {
+        // C rows are not 16-byte multiples: plain predicated stores.
+        uint32_t* crow = p.C + static_cast<size_t>(row) * p.N;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32b_x32(
+              tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), r);
+          ptx::tmem_wait_ld();
+          const int col = col0 + c * 32;
+          if (row < p.M) {
 #pragma unroll
             for (int v = 0; v < 32; ++v)
               if (col + v < p.N) crow[col + v] = r[v];
@@ -329,8 +447,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           ptx::mbar_arrive_cluster(ptx::map_to_cta(acc_empty_bar(acc), 0));
         }
       }
+      if (trace) epi_busy += clock64() - w1;
+      ++tiles_done;
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
+    }
+    // C stores still in flight read this CTA's shared memory: wait before leaving.
+    if (lane == 0) ptx::bulk_wait_group<0>();
+    __syncwarp();
+    if (trace && warp == 2 && lane == 0) {
+      trace[TRACE_EPI_WAIT] = static_cast<unsigned long long>(epi_wait);
+      trace[TRACE_EPI_BUSY] = static_cast<unsigned long long>(epi_busy);
+      trace[TRACE_TILES] = static_cast<unsigned long long>(tiles_done);
     }
   }
 
@@ -346,6 +474,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc<CTA_GROUP>(tmem_base, TMEM_COLS);
+  }
+  if (trace && threadIdx.x == 0) {
+    trace[TRACE_CYCLES] = static_cast<unsigned long long>(clock64() - clk_start);
+    trace[TRACE_NANOS] = ptx::globaltimer_ns() - ns_start;
   }
 }
 

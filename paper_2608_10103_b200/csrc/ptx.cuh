@@ -23,6 +23,23 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   return t;
 }
 
+// True in exactly one lane of a fully active, converged warp.  Code that issues
+// TMA / tcgen05 instructions should be reached by the whole warp and guarded
+// with this (not with `lane == 0` around the whole loop): the compiler then
+// knows the surrounding control flow is warp-uniform and keeps descriptors and
+// addresses in uniform registers, which makes issuing several times cheaper.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred = 0;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 // ------------------------------------------------------------------- cluster
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
