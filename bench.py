@@ -197,6 +197,10 @@ def run_ours(args, rank, world):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     binding.lib()
+    if args.override:
+        binding.gemm_set_config_override(*[int(x) for x in args.override.split(",")])
+    if args.l2_policy >= 0:
+        binding.gemm_set_l2_policy(args.l2_policy)
     N = args.size
     ops = synth.gemm_ops(N, N, N)
     stream = torch.cuda.current_stream()
@@ -365,6 +369,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-peak-probe", action="store_true")
     ap.add_argument("--precisions", default="fp16,s8,s4")
+    ap.add_argument("--l2-policy", type=int, default=-1, help="ablation: gemm_set_l2_policy")
+    ap.add_argument("--override", default="",
+                    help="ablation: BN,GROUP_M,CTA_GROUP passed to gemm_set_config_override")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -193,6 +193,15 @@ int gemm_set_config_override(int bn, int group_m, int cta_group);
 int gemm_last_device_status(void);
 
 /*
+ * L2 eviction priority given to the operand loads of later calls (the paper's
+ * Run 4 ablates the analogous .ca / .cg cache policy of cp.async): 0 = normal
+ * for A and B; 1 = A "evict last" (kept), B "evict first" (streamed), which
+ * suits the raster that walks a band of A rows across all of B; 2 = both
+ * "evict last".  Results never depend on it.
+ */
+int gemm_set_l2_policy(int policy);
+
+/*
  * Cycle accounting, in the spirit of the counter attribution the paper does
  * with its profiler (Sec. III-B).  gemm_trace_enable(1) makes later GEMM
  * launches record, per CTA, 12 unsigned 64-bit words: [0] SM cycles and [1]

@@ -22,7 +22,7 @@ PRECISION_ID = {"fp16": PREC_FP16, "s8": PREC_S8, "s4": PREC_S4}
 EXPORTS = (
     "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
     "gemm_s4_static", "gemm_s4_static_capacity", "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
-    "gemm_set_config_override", "gemm_trace_enable", "gemm_trace_read", "gemm_last_device_status", "gemm_last_cuda_error",
+    "gemm_set_config_override", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_last_device_status", "gemm_last_cuda_error",
     "gemm_status_string", "gemm_version",
 )
 
@@ -66,6 +66,7 @@ def lib() -> ctypes.CDLL:
         L.gemm_mma_peak_probe.argtypes = [i, i, i, i, ctypes.POINTER(ctypes.c_double), vp]
         L.gemm_query_config.argtypes = [i, i, i, i, ctypes.c_char_p, i]
         L.gemm_set_config_override.argtypes = [i, i, i]
+        L.gemm_set_l2_policy.argtypes = [i]
         L.gemm_trace_enable.argtypes = [i]
         L.gemm_trace_read.argtypes = [ctypes.POINTER(ctypes.c_ulonglong), i]
         L.gemm_status_string.argtypes = [i]
@@ -218,6 +219,11 @@ def gemm_query_config(precision: str, M: int, N: int, K: int) -> str:
 
 def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0):
     _check(lib().gemm_set_config_override(bn, group_m, cta_group), "gemm_set_config_override")
+
+
+def gemm_set_l2_policy(policy: int = 0):
+    """0 = normal; 1 = keep A / stream B; 2 = keep both (L2 eviction priority of operand loads)."""
+    _check(lib().gemm_set_l2_policy(int(policy)), "gemm_set_l2_policy")
 
 
 TRACE_FIELDS = ("cycles", "nanos", "producer_wait", "mma_wait_operands", "mma_wait_accumulator",

@@ -41,6 +41,7 @@ int g_override_bn = 0;
 int g_override_group_m = 0;
 int g_override_cta_group = 0;
 int g_trace_on = 0;
+int g_l2_policy = 0;
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                    const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -133,15 +134,15 @@ constexpr int kWidths[] = {256, 128, 64, 32};
 
 // Ring depth and 128-byte K atoms per slot of each built shape.
 int stages_for(int bn, int cta_group) {
-  if (cta_group == 2) return bn == 256 ? 3 : 4;
+  if (cta_group == 2) return bn == 256 ? 6 : 8;
   switch (bn) {
     case 256: return 4;
-    case 128: return 3;
-    default: return 4;
+    case 128: return 6;
+    default: return 8;
   }
 }
 
-int atoms_for(int bn, int cta_group) { return (cta_group == 1 && bn == 256) ? 1 : 2; }
+int atoms_for(int, int) { return 1; }
 
 bool variant_exists(int bn, int cta_group) {
   if (cta_group == 1) return bn == 256 || bn == 128 || bn == 64 || bn == 32;
@@ -259,21 +260,22 @@ int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* 
   p.status = s->status_ptr;
   p.trace = (g_trace_on & 1) ? s->trace_ptr : nullptr;
   p.ablate = (g_trace_on >> 1) & 3;
+  p.l2_policy = g_l2_policy;
 
   const int kbase = (KIND == ptx::KIND_F16) ? 0 : 16;
   if (cfg.cta_group == 2) {
     switch (cfg.bn) {
-      case 256: return launch_variant<KIND, 256, 3, 2, 2>(s, kbase + 8, ta, tb, tc, p, stream);
-      case 128: return launch_variant<KIND, 128, 4, 2, 2>(s, kbase + 9, ta, tb, tc, p, stream);
-      case 64: return launch_variant<KIND, 64, 4, 2, 2>(s, kbase + 10, ta, tb, tc, p, stream);
+      case 256: return launch_variant<KIND, 256, 6, 2, 1>(s, kbase + 8, ta, tb, tc, p, stream);
+      case 128: return launch_variant<KIND, 128, 8, 2, 1>(s, kbase + 9, ta, tb, tc, p, stream);
+      case 64: return launch_variant<KIND, 64, 8, 2, 1>(s, kbase + 10, ta, tb, tc, p, stream);
       default: return GEMM_ERR_INVALID_ARG;
     }
   }
   switch (cfg.bn) {
     case 256: return launch_variant<KIND, 256, 4, 1, 1>(s, kbase + 0, ta, tb, tc, p, stream);
-    case 128: return launch_variant<KIND, 128, 3, 1, 2>(s, kbase + 1, ta, tb, tc, p, stream);
-    case 64: return launch_variant<KIND, 64, 4, 1, 2>(s, kbase + 2, ta, tb, tc, p, stream);
-    case 32: return launch_variant<KIND, 32, 4, 1, 2>(s, kbase + 3, ta, tb, tc, p, stream);
+    case 128: return launch_variant<KIND, 128, 6, 1, 1>(s, kbase + 1, ta, tb, tc, p, stream);
+    case 64: return launch_variant<KIND, 64, 8, 1, 1>(s, kbase + 2, ta, tb, tc, p, stream);
+    case 32: return launch_variant<KIND, 32, 8, 1, 1>(s, kbase + 3, ta, tb, tc, p, stream);
     default: return GEMM_ERR_INVALID_ARG;
   }
 }
@@ -511,6 +513,13 @@ int gemm_last_device_status(void) {
     if (e != cudaSuccess) return cuda_fail(e);
   }
   return v;
+}
+
+int gemm_set_l2_policy(int policy) {
+  if (policy < 0 || policy > 2) return GEMM_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  g_l2_policy = policy;
+  return GEMM_OK;
 }
 
 int gemm_trace_enable(int on) {

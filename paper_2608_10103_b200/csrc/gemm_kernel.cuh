@@ -68,6 +68,9 @@ struct GemmParams {
   int* status;           // device status word (0 = ok)
   // Optional per-CTA cycle accounting (TRACE_SLOTS 64-bit words per CTA), or null.
   unsigned long long* trace;
+  // L2 eviction priority of the operand loads: 0 = normal for both; 1 = keep A (evict last),
+  // stream B (evict first); 2 = keep both.
+  int l2_policy;
   // Ablation switches for cycle accounting runs (results are then meaningless):
   // bit 0 = issue no MMAs (loads + barriers only), bit 1 = issue no loads (MMAs + barriers only).
   int ablate;
@@ -222,12 +225,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    {
+      // The whole warp walks the loops and polls the barriers (so loop state stays
+      // warp-uniform and cheap to turn into TMA operands); the lane elected here, once,
+      // issues the copies.  Nothing inside the loops is warp-collective, so a lane whose
+      // wait gives up can leave on its own.
+      const bool elected = ptx::elect_one();
       int stage = 0;
       uint32_t phase = 0;
       int issued = 0;
       bool ok = true;
       long long waited = 0, prod_issue = 0;
+      const uint64_t pol_a = p.l2_policy == 0 ? ptx::policy_evict_normal() : ptx::policy_evict_last();
+      const uint64_t pol_b = p.l2_policy == 0 ? ptx::policy_evict_normal()
+                             : p.l2_policy == 1 ? ptx::policy_evict_first()
+                                                : ptx::policy_evict_last();
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
         int tm, tn;
         tile_coords(p, t, tm, tn);
@@ -242,15 +254,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           if (!ok) break;
           const uint32_t a_dst = base + stage * L::STAGE_BYTES;
           const uint32_t b_dst = a_dst + KB * L::A_BYTES;
-          if (p.ablate & 2) {
+          if (!elected) {
+            // nothing to issue in this lane
+          } else if (p.ablate & 2) {
             if (leader) ptx::mbar_arrive(full_bar(stage));
           } else if constexpr (CTA_GROUP == 1) {
             ptx::mbar_arrive_expect_tx(full_bar(stage), L::STAGE_BYTES);
 #pragma unroll
             for (int a = 0; a < KB; ++a) {
               const int k0 = (ks * KB + a) * BK_ELEMS;
-              ptx::tma_load_2d(a_dst + a * L::A_BYTES, &tmap_a, k0, a_row, full_bar(stage));
-              ptx::tma_load_2d(b_dst + a * L::B_BYTES, &tmap_b, k0, b_row, full_bar(stage));
+              ptx::tma_load_2d(a_dst + a * L::A_BYTES, &tmap_a, k0, a_row, full_bar(stage), pol_a);
+              ptx::tma_load_2d(b_dst + a * L::B_BYTES, &tmap_b, k0, b_row, full_bar(stage), pol_b);
             }
           } else {
             // Bytes of both CTAs are counted on the leader's barrier.
@@ -259,8 +273,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 #pragma unroll
             for (int a = 0; a < KB; ++a) {
               const int k0 = (ks * KB + a) * BK_ELEMS;
-              ptx::tma_load_2d_pair(a_dst + a * L::A_BYTES, &tmap_a, k0, a_row, lead_full);
-              ptx::tma_load_2d_pair(b_dst + a * L::B_BYTES, &tmap_b, k0, b_row, lead_full);
+              ptx::tma_load_2d_pair(a_dst + a * L::A_BYTES, &tmap_a, k0, a_row, lead_full, pol_a);
+              ptx::tma_load_2d_pair(b_dst + a * L::B_BYTES, &tmap_b, k0, b_row, lead_full, pol_b);
             }
           }
           ++issued;
@@ -268,11 +282,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
-      if (trace) {
+      if (trace && elected) {
         trace[TRACE_PROD_WAIT] = static_cast<unsigned long long>(waited);
         trace[TRACE_PROD_ISSUE] = static_cast<unsigned long long>(prod_issue);
       }
-      if (!ok && (CTA_GROUP == 1 || leader)) {
+      if (!ok && elected && (CTA_GROUP == 1 || leader)) {
         // Gave up: let the copies already in flight land before the CTA exits.
         int n = issued < STAGES ? issued : STAGES;
         for (int i = 0; i < n; ++i) {
@@ -287,7 +301,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     __syncwarp();
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
-    if (lane == 0 && leader) {
+    if (leader) {  // whole warp walks the loops, the lane elected once issues (see producer)
+      const bool elected = ptx::elect_one();
       constexpr uint32_t idesc = ptx::make_idesc<KIND>(TILE_M, BN);
       int stage = 0;
       uint32_t phase = 0;
@@ -313,51 +328,52 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const uint32_t a_src = base + stage * L::STAGE_BYTES;
           const uint64_t a_desc = ptx::smem_desc_sw128(a_src);
           const uint64_t b_desc = ptx::smem_desc_sw128(a_src + KB * L::A_BYTES);
-          const long long w3 = trace ? clock64() : 0;
-          if (!(p.ablate & 1)) {
+          if (elected && !(p.ablate & 1)) {
 #pragma unroll
             for (int a = 0; a < KB; ++a) {
 #pragma unroll
               for (int kk = 0; kk < BK_BYTES / MMA_K_BYTES; ++kk) {
                 // descriptor addresses are in 16-byte units
-                const uint64_t a_step = static_cast<uint64_t>((a * L::A_BYTES + kk * MMA_K_BYTES) >> 4);
-                const uint64_t b_step = static_cast<uint64_t>((a * L::B_BYTES + kk * MMA_K_BYTES) >> 4);
+                const uint64_t a_step =
+                    static_cast<uint64_t>((a * L::A_BYTES + kk * MMA_K_BYTES) >> 4);
+                const uint64_t b_step =
+                    static_cast<uint64_t>((a * L::B_BYTES + kk * MMA_K_BYTES) >> 4);
                 ptx::mma_ss<KIND, CTA_GROUP>(d_tmem, a_desc + a_step, b_desc + b_step, idesc,
                                              (ks > 0 || a > 0 || kk > 0) ? 1u : 0u);
               }
             }
           }
+          if (trace) t_issue += clock64() - w2;
           const long long w4 = trace ? clock64() : 0;
-          if constexpr (CTA_GROUP == 1) {
-            ptx::mma_commit<1>(empty_bar(stage));
-          } else {
-            ptx::mma_commit_pair(empty_bar(stage), 0x3);
+          if (elected) {
+            if constexpr (CTA_GROUP == 1) {
+              ptx::mma_commit<1>(empty_bar(stage));
+            } else {
+              ptx::mma_commit_pair(empty_bar(stage), 0x3);
+            }
           }
-          if (trace) {
-            const long long w5 = clock64();
-            t_fence += w3 - w2;
-            t_issue += w4 - w3;
-            t_commit += w5 - w4;
-          }
+          if (trace) t_commit += clock64() - w4;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        if constexpr (CTA_GROUP == 1) {
-          ptx::mma_commit<1>(acc_full_bar(acc));
-        } else {
-          ptx::mma_commit_pair(acc_full_bar(acc), 0x3);
+        if (elected) {
+          if constexpr (CTA_GROUP == 1) {
+            ptx::mma_commit<1>(acc_full_bar(acc));
+          } else {
+            ptx::mma_commit_pair(acc_full_bar(acc), 0x3);
+          }
         }
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
-      if (trace) {
+      if (trace && elected) {
         trace[TRACE_MMA_WAIT_FULL] = static_cast<unsigned long long>(wait_full);
         trace[TRACE_MMA_WAIT_ACC] = static_cast<unsigned long long>(wait_acc);
         trace[TRACE_MMA_ISSUE] = static_cast<unsigned long long>(t_issue);
         trace[TRACE_MMA_COMMIT] = static_cast<unsigned long long>(t_commit);
         trace[TRACE_MMA_FENCE] = static_cast<unsigned long long>(t_fence);
       }
-      if (!ok) {
+      if (!ok && elected) {
         // Gave up: wait for the MMAs already issued before TMEM is released.
         ptx::mma_commit<CTA_GROUP>(drain_bar);
         uint64_t t0 = ptx::globaltimer_ns();
