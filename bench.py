@@ -32,7 +32,7 @@ if ROOT not in sys.path:
 
 SPEC_PEAK = {"fp16": 2250.0, "s8": 4500.0, "s4": 4500.0}   # vendor dense figures, T(FL)OP/s
 UNIT = {"fp16": "TFLOP/s", "s8": "TOP/s", "s4": "TOP/s"}
-KERNEL_LAUNCHES = {"fp16": 1, "s8": 1, "s4": 3}            # s4: two unpack launches + GEMM
+KERNEL_LAUNCHES = {"fp16": 1, "s8": 1, "s4": 2}            # s4: unpack launch + GEMM
 # DRAM bytes per launch of the FP16 GEMM kernel at N = 8192 (dram__bytes_read.sum +
 # dram__bytes_write.sum from one ncu capture; see profiles/).  None until captured.
 NCU_TRAFFIC_BYTES = {"fp16": {}}
@@ -357,6 +357,77 @@ def run_ours(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """Precision x size sweep (the paper's Sec. III-B sizes): one JSON line per cell.
+    Each cell: seeded operands resident in HBM; `reps` launches are captured once in a
+    CUDA graph and the graph is replayed between two CUDA events, so the number is device
+    time and not the host's cost of issuing a call (which exceeds the kernel at N <= 1024;
+    it is reported separately as `host_us_per_call`).  Median of 5 replays; an L2 flush
+    (256 MB write) precedes each, so the first launch starts cold and, at sizes whose
+    operands fit in L2, later ones run warm: the batch mean and a cold single launch are
+    both reported."""
+    import numpy as np
+    import torch
+    from paper_2608_10103_b200 import binding, synth
+    torch.cuda.set_device(0)
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    peaks = measured_peaks()
+
+    def timed(fn, reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        flush.fill_(1)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    def graph_of(call, reps):
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(reps):
+                    call(side)
+        torch.cuda.current_stream().wait_stream(side)
+        return g
+
+    for prec in synth.PRECISIONS:
+        for N in synth.SWEEP_SIZES:
+            A, B = synth.make(prec, N, N, N, synth.sweep_seed(prec, N))
+            dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+            C = torch.empty((N, N), dtype=torch.float32 if prec == "fp16" else torch.int32,
+                            device="cuda")
+            call = lambda st: binding.gemm(prec, dA, dB, C, st)
+            for _ in range(3):
+                call(stream)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(200):
+                call(stream)
+            host_us = (time.perf_counter() - t0) / 200 * 1e6
+            torch.cuda.synchronize()
+            reps = max(5, min(100, int(20.0 / max(timed(lambda: call(stream), 5), 1e-3))))
+            g_many, g_one = graph_of(call, reps), graph_of(call, 1)
+            warm = float(np.median([timed(g_many.replay, 1) for _ in range(5)])) / reps
+            cold = float(np.median([timed(g_one.replay, 1) for _ in range(5)]))
+            ops = synth.gemm_ops(N, N, N)
+            rate = ops / (warm * 1e-3) / 1e12
+            ref = peaks["bf16_burst"] * (1 if prec == "fp16" else 2)
+            print(json.dumps({
+                "sweep": True, "precision": prec, "N": N, "seed": synth.sweep_seed(prec, N),
+                "ms": warm, "reps": reps, "ms_cold_single_launch": cold,
+                "host_us_per_call": host_us,
+                "value": rate, "unit": UNIT[prec], "frac_of_spec_peak": rate / SPEC_PEAK[prec],
+                "frac_of_cublas_bf16_burst_scaled": rate / ref,
+                "config": binding.gemm_query_config(prec, N, N, N)}), flush=True)
+    if binding.gemm_last_device_status() != 0:
+        raise SystemExit("bench.py: a kernel reported a barrier timeout")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -368,6 +439,8 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-peak-probe", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="precision x size sweep N=512..8192, one JSON line per cell (1 GPU)")
     ap.add_argument("--precisions", default="fp16,s8,s4")
     ap.add_argument("--l2-policy", type=int, default=-1, help="ablation: gemm_set_l2_policy")
     ap.add_argument("--override", default="",
@@ -377,7 +450,10 @@ def main():
         args.warmup = 3
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.impl == "reference":
+    if args.sweep:
+        if rank == 0:
+            run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args, rank)
     else:
         run_ours(args, rank, world)

@@ -193,11 +193,18 @@ int gemm_set_config_override(int bn, int group_m, int cta_group);
 int gemm_last_device_status(void);
 
 /*
- * L2 eviction priority given to the operand loads of later calls (the paper's
- * Run 4 ablates the analogous .ca / .cg cache policy of cp.async): 0 = normal
- * for A and B; 1 = A "evict last" (kept), B "evict first" (streamed), which
- * suits the raster that walks a band of A rows across all of B; 2 = both
- * "evict last".  Results never depend on it.
+ * L2 behaviour of later calls, a bit set (the paper's Run 4 ablates the
+ * analogous .ca / .cg cache policy of cp.async).  Bits 0-1, eviction priority
+ * of the operand loads: 0 = normal for A and B; 1 = A "evict last" (kept), B
+ * "evict first" (streamed); 2 = both "evict last"; 3 = A "evict last", B
+ * normal.  Bit 2 (4): turn OFF the serpentine K order (by default successive
+ * tiles of a CTA walk K forward, backward, forward, ... so that a tile begins
+ * on the K range its predecessor, which shares its A rows, read last and still
+ * finds in L2).  Bit 3 (8): mark the C stores "evict first" (written once,
+ * never re-read).  Default 11 = 3 + 8 with the serpentine order on, which gave
+ * the lowest DRAM traffic at N = 8192.  Integer results never depend on any of
+ * this; FP16 results may differ in the last bits (summation order) within the
+ * bound.
  */
 int gemm_set_l2_policy(int policy);
 

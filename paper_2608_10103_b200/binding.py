@@ -221,8 +221,9 @@ def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0):
     _check(lib().gemm_set_config_override(bn, group_m, cta_group), "gemm_set_config_override")
 
 
-def gemm_set_l2_policy(policy: int = 0):
-    """0 = normal; 1 = keep A / stream B; 2 = keep both (L2 eviction priority of operand loads)."""
+def gemm_set_l2_policy(policy: int = 11):
+    """Bit set: bits 0-1 operand eviction priority (0 normal, 1 keep A / stream B, 2 keep
+    both, 3 keep A), +4 serpentine K order off, +8 C stores evict-first.  Default 11."""
     _check(lib().gemm_set_l2_policy(int(policy)), "gemm_set_l2_policy")
 
 

@@ -41,7 +41,7 @@ int g_override_bn = 0;
 int g_override_group_m = 0;
 int g_override_cta_group = 0;
 int g_trace_on = 0;
-int g_l2_policy = 0;
+int g_l2_policy = 11;  // keep A, B normal, serpentine K, C stores evict-first
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                    const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -177,11 +177,12 @@ TileConfig select_config(int M, int N, int num_sms) {
     }
   }
   best.stages = stages_for(best.bn, best.cta_group);
-  // Band height: make one wave of tiles roughly square in operand bytes.
+  // Band height: one wave of tiles about twice as tall as wide in operand bytes (measured
+  // DRAM traffic at N = 8192 is lowest there: the A band is what later waves re-read).
   int rows_per_tile = BM * best.cta_group;
   int units = num_sms / best.cta_group;
   int g = 1;
-  while ((g + 1) * (g + 1) * rows_per_tile <= units * best.bn) ++g;
+  while ((g + 1) * (g + 1) * rows_per_tile <= 2 * units * best.bn) ++g;
   if (g_override_group_m) g = g_override_group_m;
   int tiles_m = ceil_div(M, rows_per_tile);
   if (g > tiles_m) g = tiles_m;
@@ -260,7 +261,9 @@ int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* 
   p.status = s->status_ptr;
   p.trace = (g_trace_on & 1) ? s->trace_ptr : nullptr;
   p.ablate = (g_trace_on >> 1) & 3;
-  p.l2_policy = g_l2_policy;
+  p.l2_policy = g_l2_policy & 3;
+  p.serpentine_k = (g_l2_policy & 4) ? 0 : 1;
+  p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
 
   const int kbase = (KIND == ptx::KIND_F16) ? 0 : 16;
   if (cfg.cta_group == 2) {
@@ -290,14 +293,18 @@ int check_common(int M, int N, int K, const void* A, const void* B, const void* 
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-int launch_unpack(long long rows, int K, const uint8_t* packed, int8_t* out, size_t out_pitch,
+// Unpacks one or two packed matrices (rows_b may be 0) with the same K and output pitch.
+int launch_unpack(long long rows_a, const uint8_t* packed_a, int8_t* out_a, long long rows_b,
+                  const uint8_t* packed_b, int8_t* out_b, int K, size_t out_pitch,
                   cudaStream_t stream) {
-  const long long chunks = rows * (K / 32);
+  UnpackJob a{reinterpret_cast<const uint4*>(packed_a), out_a, rows_a * (K / 32)};
+  UnpackJob b{reinterpret_cast<const uint4*>(packed_b), out_b, rows_b * (K / 32)};
+  const long long chunks = a.chunks + b.chunks;
   long long blocks = (chunks + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > 148 * 32) blocks = 148 * 32;
   if (blocks < 1) blocks = 1;
   unpack_s4_kernel<<<static_cast<int>(blocks), 256, 0, stream>>>(
-      reinterpret_cast<const uint4*>(packed), out, rows, K / 32, static_cast<long long>(out_pitch));
+      a, b, K / 32, static_cast<long long>(out_pitch));
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   return GEMM_OK;
@@ -359,9 +366,7 @@ int gemm_s4_ws(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t*
     rc = device_state(&s);
     if (rc != GEMM_OK) return rc;
   }
-  rc = launch_unpack(M, K, A, a8, static_cast<size_t>(K), st);
-  if (rc != GEMM_OK) return rc;
-  rc = launch_unpack(N, K, B, b8, static_cast<size_t>(K), st);
+  rc = launch_unpack(M, A, a8, N, B, b8, K, static_cast<size_t>(K), st);
   if (rc != GEMM_OK) return rc;
   return launch_gemm<ptx::KIND_I8>(M, N, K, a8, static_cast<size_t>(K), b8, static_cast<size_t>(K),
                                    C, st);
@@ -420,7 +425,8 @@ int gemm_unpack_s4(int rows, int K, const uint8_t* packed, int8_t* out, size_t o
   if (K % 32 || out_pitch % 16 || out_pitch < static_cast<size_t>(K) ||
       ((reinterpret_cast<uintptr_t>(packed) | reinterpret_cast<uintptr_t>(out)) & 15))
     return GEMM_ERR_MISALIGNED;
-  return launch_unpack(rows, K, packed, out, out_pitch, reinterpret_cast<cudaStream_t>(stream));
+  return launch_unpack(rows, packed, out, 0, nullptr, nullptr, K, out_pitch,
+                       reinterpret_cast<cudaStream_t>(stream));
 }
 
 int gemm_mma_peak_probe(int precision, int iters, int n_cols, int commit_every, double* ops_out,
@@ -516,7 +522,7 @@ int gemm_last_device_status(void) {
 }
 
 int gemm_set_l2_policy(int policy) {
-  if (policy < 0 || policy > 2) return GEMM_ERR_INVALID_ARG;
+  if (policy < 0 || policy > 15) return GEMM_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
   g_l2_policy = policy;
   return GEMM_OK;

@@ -69,8 +69,12 @@ struct GemmParams {
   // Optional per-CTA cycle accounting (TRACE_SLOTS 64-bit words per CTA), or null.
   unsigned long long* trace;
   // L2 eviction priority of the operand loads: 0 = normal for both; 1 = keep A (evict last),
-  // stream B (evict first); 2 = keep both.
+  // stream B (evict first); 2 = keep both; 3 = keep A, B normal.
   int l2_policy;
+  int c_evict_first;     // 1: C stores are marked evict-first (written once, never re-read)
+  // 1: successive tiles of a CTA walk K in opposite directions, so a tile starts on the
+  // K range its predecessor (same A rows) touched last and finds it still in L2.
+  int serpentine_k;
   // Ablation switches for cycle accounting runs (results are then meaningless):
   // bit 0 = issue no MMAs (loads + barriers only), bit 1 = issue no loads (MMAs + barriers only).
   int ablate;
@@ -237,9 +241,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       bool ok = true;
       long long waited = 0, prod_issue = 0;
       const uint64_t pol_a = p.l2_policy == 0 ? ptx::policy_evict_normal() : ptx::policy_evict_last();
-      const uint64_t pol_b = p.l2_policy == 0 ? ptx::policy_evict_normal()
-                             : p.l2_policy == 1 ? ptx::policy_evict_first()
-                                                : ptx::policy_evict_last();
+      const uint64_t pol_b = (p.l2_policy == 0 || p.l2_policy == 3) ? ptx::policy_evict_normal()
+                             : p.l2_policy == 1                      ? ptx::policy_evict_first()
+                                                                     : ptx::policy_evict_last();
+      bool backward = false;
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
         int tm, tn;
         tile_coords(p, t, tm, tn);
@@ -262,7 +267,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             ptx::mbar_arrive_expect_tx(full_bar(stage), L::STAGE_BYTES);
 #pragma unroll
             for (int a = 0; a < KB; ++a) {
-              const int k0 = (ks * KB + a) * BK_ELEMS;
+              const int k0 = ((backward ? k_slots - 1 - ks : ks) * KB + a) * BK_ELEMS;
               ptx::tma_load_2d(a_dst + a * L::A_BYTES, &tmap_a, k0, a_row, full_bar(stage), pol_a);
               ptx::tma_load_2d(b_dst + a * L::B_BYTES, &tmap_b, k0, b_row, full_bar(stage), pol_b);
             }
@@ -272,7 +277,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             const uint32_t lead_full = ptx::map_to_cta(full_bar(stage), 0);
 #pragma unroll
             for (int a = 0; a < KB; ++a) {
-              const int k0 = (ks * KB + a) * BK_ELEMS;
+              const int k0 = ((backward ? k_slots - 1 - ks : ks) * KB + a) * BK_ELEMS;
               ptx::tma_load_2d_pair(a_dst + a * L::A_BYTES, &tmap_a, k0, a_row, lead_full, pol_a);
               ptx::tma_load_2d_pair(b_dst + a * L::B_BYTES, &tmap_b, k0, b_row, lead_full, pol_b);
             }
@@ -281,6 +286,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           if (trace) prod_issue += clock64() - w9;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
+        if (p.serpentine_k) backward = !backward;
       }
       if (trace && elected) {
         trace[TRACE_PROD_WAIT] = static_cast<unsigned long long>(waited);
@@ -388,6 +394,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
     const uint32_t epi_base =
         base + L::EPI_OFFSET + static_cast<uint32_t>((warp - 2) * 2 * L::EPI_BUF_BYTES);
+    const uint64_t pol_c = p.c_evict_first ? ptx::policy_evict_first() : ptx::policy_evict_normal();
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -432,7 +439,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           // reuse rule above exact.
           if (lane == 0) {
             if (row0 < p.M && col0 + c * 32 < p.N)
-              ptx::tma_store_2d(&tmap_c, col0 + c * 32, row0, buf);
+              ptx::tma_store_2d(&tmap_c, col0 + c * 32, row0, buf, pol_c);
             ptx::bulk_commit_group();
           }
         }

@@ -162,11 +162,13 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
 
 // 2-D tiled store shared -> global (bulk-group completion).  Rows/columns of
 // the box that fall outside the tensor are clipped by the hardware.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, int c0, int c1, uint32_t src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::
-                   "l"(reinterpret_cast<uint64_t>(m)),
-               "r"(c0), "r"(c1), "r"(src)
-               : "memory");
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, int c0, int c1, uint32_t src,
+                                             uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint "
+      "[%0, {%1, %2}], [%3], %4;" ::"l"(reinterpret_cast<uint64_t>(m)),
+      "r"(c0), "r"(c1), "r"(src), "l"(policy)
+      : "memory");
 }
 
 __device__ __forceinline__ void bulk_commit_group() {

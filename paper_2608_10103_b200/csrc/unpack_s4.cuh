@@ -28,16 +28,27 @@ __device__ __forceinline__ void unpack8_s4(uint32_t w, uint32_t& lo, uint32_t& h
 
 // One thread expands 16 packed bytes (32 elements) into 32 output bytes.
 // chunks_per_row = K / 32.  Bytes K .. out_pitch-1 of each output row are zeroed.
+// The kernel handles two matrices in one launch (A then B of a GEMM): chunk
+// indices [0, chunks_a) belong to the first, the rest to the second.
+struct UnpackJob {
+  const uint4* packed;
+  int8_t* out;
+  long long chunks;  // rows * chunks_per_row
+};
+
 __global__ void __launch_bounds__(256)
-unpack_s4_kernel(const uint4* __restrict__ packed, int8_t* __restrict__ out, long long rows,
-                 int chunks_per_row, long long out_pitch) {
-  const long long total = rows * chunks_per_row;
+unpack_s4_kernel(UnpackJob a, UnpackJob b, int chunks_per_row, long long out_pitch) {
+  const long long total = a.chunks + b.chunks;
   const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-  for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total;
-       idx += stride) {
+  for (long long g = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; g < total;
+       g += stride) {
+    const bool second = g >= a.chunks;
+    const long long idx = second ? g - a.chunks : g;
+    const uint4* src = second ? b.packed : a.packed;
+    int8_t* out = second ? b.out : a.out;
     const long long row = idx / chunks_per_row;
     const int chunk = static_cast<int>(idx - row * chunks_per_row);
-    const uint4 w = __ldg(packed + idx);
+    const uint4 w = __ldg(src + idx);
     uint4 o0, o1;
     unpack8_s4(w.x, o0.x, o0.y);
     unpack8_s4(w.y, o0.z, o0.w);
@@ -48,8 +59,8 @@ unpack_s4_kernel(const uint4* __restrict__ packed, int8_t* __restrict__ out, lon
     dst[1] = o1;
     if (chunk == chunks_per_row - 1) {
       const long long k_end = static_cast<long long>(chunks_per_row) * 32;
-      for (long long b = k_end; b < out_pitch; b += 16)
-        *reinterpret_cast<uint4*>(out + row * out_pitch + b) = make_uint4(0, 0, 0, 0);
+      for (long long t = k_end; t < out_pitch; t += 16)
+        *reinterpret_cast<uint4*>(out + row * out_pitch + t) = make_uint4(0, 0, 0, 0);
     }
   }
 }
