@@ -33,9 +33,10 @@ if ROOT not in sys.path:
 SPEC_PEAK = {"fp16": 2250.0, "s8": 4500.0, "s4": 4500.0}   # vendor dense figures, T(FL)OP/s
 UNIT = {"fp16": "TFLOP/s", "s8": "TOP/s", "s4": "TOP/s"}
 KERNEL_LAUNCHES = {"fp16": 1, "s8": 1, "s4": 2}            # s4: unpack launch + GEMM
-# DRAM bytes per launch of the FP16 GEMM kernel at N = 8192 (dram__bytes_read.sum +
-# dram__bytes_write.sum from one ncu capture; see profiles/).  None until captured.
-NCU_TRAFFIC_BYTES = {"fp16": {}}
+# DRAM bytes per launch of the FP16 GEMM kernel (dram__bytes_read.sum + dram__bytes_write.sum
+# from one ncu capture of this workload; profiles/gemm_kernels_n8192_ncu_metrics.md and
+# profiles/gemm_kernel_fp16_n4096_ncu_full.md).  Sizes that were not captured report null.
+NCU_TRAFFIC_BYTES = {"fp16": {8192: 845519872 + 254798848, 4096: 95784960 + 41198336}}
 
 
 def measured_peaks():
