@@ -429,6 +429,76 @@ def run_sweep(args):
         raise SystemExit("bench.py: a kernel reported a barrier timeout")
 
 
+def run_ablation(args):
+    """One-variable-at-a-time ablation at N = args.size (the analogue of the paper's Run 4):
+    tile shape, raster band height, L2 policy, and load-only / MMA-only runs, each with
+    the per-role cycle accounting of the kernel.  One JSON line per variant."""
+    import numpy as np
+    import torch
+    from paper_2608_10103_b200 import binding, synth
+    torch.cuda.set_device(0)
+    N = args.size
+    ops = synth.gemm_ops(N, N, N)
+    data = {"fp16": synth.fp16_normal_clipped(N, N, N, seed=3),
+            "s8": synth.s8_uniform(N, N, N, seed=synth.sweep_seed("s8", 8192))}
+    variants = [("baseline (selector default)", (0, 0, 0), 11, 1)]
+    variants += [("tile 128x%d, one CTA" % bn, (bn, 0, 1), 11, 1) for bn in (256, 128, 64, 32)]
+    variants += [("tile 256x%d, CTA pair" % bn, (bn, 0, 2), 11, 1) for bn in (256, 128, 64)]
+    variants += [("band height %d" % g, (256, g, 2), 11, 1) for g in (2, 4, 8, 16, 32)]
+    variants += [("L2: no hints, forward K only", (0, 0, 0), 4, 1),
+                 ("L2: no hints, serpentine K", (0, 0, 0), 0, 1),
+                 ("L2: keep A, stream B", (0, 0, 0), 1, 1),
+                 ("L2: keep A and B", (0, 0, 0), 2, 1),
+                 ("L2: default + 128-byte promotion", (0, 0, 0), 27, 1),
+                 ("ablate: no MMAs (loads + barriers only)", (0, 0, 0), 11, 3),
+                 ("ablate: no loads (MMAs + barriers only)", (0, 0, 0), 11, 5),
+                 ("epilogue waits with nanosleep back-off", (0, 0, 0), 11, 9)]
+    for prec in ("fp16", "s8"):
+        dA, dB = (torch.from_numpy(x).cuda() for x in data[prec])
+        C = torch.empty((N, N), dtype=torch.float32 if prec == "fp16" else torch.int32,
+                        device="cuda")
+        flop_per_clk = 8192 if prec == "fp16" else 16384
+        for name, override, policy, trace in variants:
+            binding.gemm_set_config_override(*override)
+            binding.gemm_set_l2_policy(policy)
+            binding.gemm_trace_enable(trace)
+            cfg = binding.gemm_query_config(prec, N, N, N)
+            for _ in range(3):
+                binding.gemm(prec, dA, dB, C)
+            torch.cuda.synchronize()
+            time.sleep(1.5)        # let the power state settle: every variant starts alike
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                binding.gemm(prec, dA, dB, C)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / args.steps
+            tr = binding.gemm_trace_read(148)
+            a = {k: np.array([t[k] for t in tr], dtype=np.float64) for k in binding.TRACE_FIELDS}
+            lead = a["mma_issue"] > 0
+            kb_total = a["tiles"].mean() * (N * (2 if prec == "fp16" else 1) // 128)
+            cyc = float(a["cycles"].max())
+            print(json.dumps({
+                "ablation": name, "precision": prec, "N": N, "config": cfg,
+                "ms": ms, "value": ops / (ms * 1e-3) / 1e12, "unit": UNIT[prec],
+                "sm_cycles": cyc, "pipe_utilisation": ops / (148 * flop_per_clk) / cyc,
+                "sm_mhz_during_kernel": float(np.median(a["cycles"] / a["nanos"] * 1e3)),
+                "cycles_per_kblock": {
+                    "mma_wait_operands": float(a["mma_wait_operands"][lead].mean() / kb_total),
+                    "mma_issue": float(a["mma_issue"][lead].mean() / kb_total),
+                    "mma_commit": float(a["mma_commit"][lead].mean() / kb_total),
+                    "producer_wait": float(a["producer_wait"].mean() / kb_total),
+                    "producer_issue": float(a["producer_issue"].mean() / kb_total)},
+                "epilogue_busy_frac": float(a["epilogue_busy"].mean() / a["cycles"].mean()),
+                "result_valid": trace in (1, 9)}), flush=True)
+    binding.gemm_set_config_override(0, 0, 0)
+    binding.gemm_set_l2_policy(11)
+    binding.gemm_trace_enable(0)
+    if binding.gemm_last_device_status() != 0:
+        raise SystemExit("bench.py: a kernel reported a barrier timeout")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -440,6 +510,8 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-peak-probe", action="store_true")
+    ap.add_argument("--ablation", action="store_true",
+                    help="tile / raster / L2 / load-vs-MMA ablation with cycle accounting (1 GPU)")
     ap.add_argument("--sweep", action="store_true",
                     help="precision x size sweep N=512..8192, one JSON line per cell (1 GPU)")
     ap.add_argument("--precisions", default="fp16,s8,s4")
@@ -451,7 +523,10 @@ def main():
         args.warmup = 3
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.sweep:
+    if args.ablation:
+        if rank == 0:
+            run_ablation(args)
+    elif args.sweep:
         if rank == 0:
             run_sweep(args)
     elif args.impl == "reference":

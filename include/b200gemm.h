@@ -201,7 +201,8 @@ int gemm_last_device_status(void);
  * tiles of a CTA walk K forward, backward, forward, ... so that a tile begins
  * on the K range its predecessor, which shares its A rows, read last and still
  * finds in L2).  Bit 3 (8): mark the C stores "evict first" (written once,
- * never re-read).  Default 11 = 3 + 8 with the serpentine order on, which gave
+ * never re-read).  Bit 4 (16): fetch operands with 128-byte instead of 256-byte
+ * L2 promotion.  Default 11 = 3 + 8 with the serpentine order on, which gave
  * the lowest DRAM traffic at N = 8192.  Integer results never depend on any of
  * this; FP16 results may differ in the last bits (summation order) within the
  * bound.
@@ -224,8 +225,9 @@ int gemm_set_l2_policy(int policy);
  * when on is a few clock reads per k-block.
  * `on` is a bit set: 1 = record; 2 = ablation, issue no MMAs (operand loads and
  * barriers only); 4 = ablation, issue no operand loads (MMAs and barriers only,
- * on whatever shared memory holds).  With an ablation bit set C is garbage; the
- * bits exist to attribute cycles to the load path or the MMA path.
+ * on whatever shared memory holds); 8 = the epilogue's waits back off with
+ * nanosleep instead of polling.  With bit 2 or 4 set C is garbage; the bits
+ * exist to attribute cycles to the load path or the MMA path.
  */
 int gemm_trace_enable(int on);
 int gemm_trace_read(unsigned long long* out, int max_ctas);

@@ -223,7 +223,8 @@ def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0):
 
 def gemm_set_l2_policy(policy: int = 11):
     """Bit set: bits 0-1 operand eviction priority (0 normal, 1 keep A / stream B, 2 keep
-    both, 3 keep A), +4 serpentine K order off, +8 C stores evict-first.  Default 11."""
+    both, 3 keep A), +4 serpentine K order off, +8 C stores evict-first, +16 128-byte L2
+    promotion.  Default 11."""
     _check(lib().gemm_set_l2_policy(int(policy)), "gemm_set_l2_policy")
 
 
@@ -234,7 +235,8 @@ TRACE_SLOTS = len(TRACE_FIELDS)
 
 
 def gemm_trace_enable(flags: int = 1):
-    """1 = record cycles; +2 = issue no MMAs; +4 = issue no operand loads; 0 = off."""
+    """1 = record cycles; +2 = issue no MMAs; +4 = issue no operand loads; +8 = epilogue
+    waits back off with nanosleep; 0 = off."""
     _check(lib().gemm_trace_enable(int(flags)), "gemm_trace_enable")
 
 

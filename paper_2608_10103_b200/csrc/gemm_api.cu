@@ -89,14 +89,17 @@ int device_state(DeviceState** out) {
 // Row-major 2-D tensor of `rows` x `cols` elements, pitch in bytes; the box is
 // box_rows rows of 128 bytes, written to shared memory with the 128-byte swizzle.
 int encode_operand_map(CUtensorMap* map, CUtensorMapDataType type, int elem_bytes, const void* ptr,
-                       uint64_t rows, uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows) {
+                       uint64_t rows, uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows,
+                       bool promote_256 = true) {
   cuuint64_t dims[2] = {cols, rows};
   cuuint64_t strides[1] = {pitch_bytes};
   cuuint32_t box[2] = {static_cast<cuuint32_t>(BK_BYTES / elem_bytes), box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = g_encode(map, type, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                        promote_256 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B
+                                    : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     g_last_cuda_error = static_cast<int>(cudaErrorInvalidValue);
     return GEMM_ERR_CUDA;
@@ -236,9 +239,10 @@ int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* 
   const TileConfig cfg = select_config(M, N, s->num_sms);
 
   CUtensorMap ta, tb;
-  rc = encode_operand_map(&ta, type, ELEM, A, M, K, a_pitch, BM);
+  const bool promote = !(g_l2_policy & 16);
+  rc = encode_operand_map(&ta, type, ELEM, A, M, K, a_pitch, BM, promote);
   if (rc != GEMM_OK) return rc;
-  rc = encode_operand_map(&tb, type, ELEM, B, N, K, b_pitch, cfg.bn / cfg.cta_group);
+  rc = encode_operand_map(&tb, type, ELEM, B, N, K, b_pitch, cfg.bn / cfg.cta_group, promote);
   if (rc != GEMM_OK) return rc;
 
   GemmParams p;
@@ -260,7 +264,7 @@ int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* 
   p.C = static_cast<uint32_t*>(C);
   p.status = s->status_ptr;
   p.trace = (g_trace_on & 1) ? s->trace_ptr : nullptr;
-  p.ablate = (g_trace_on >> 1) & 3;
+  p.ablate = (g_trace_on >> 1) & 7;
   p.l2_policy = g_l2_policy & 3;
   p.serpentine_k = (g_l2_policy & 4) ? 0 : 1;
   p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
@@ -522,7 +526,7 @@ int gemm_last_device_status(void) {
 }
 
 int gemm_set_l2_policy(int policy) {
-  if (policy < 0 || policy > 15) return GEMM_ERR_INVALID_ARG;
+  if (policy < 0 || policy > 31) return GEMM_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
   g_l2_policy = policy;
   return GEMM_OK;
@@ -530,7 +534,7 @@ int gemm_set_l2_policy(int policy) {
 
 int gemm_trace_enable(int on) {
   std::lock_guard<std::mutex> lock(g_mutex);
-  g_trace_on = on & 7;
+  g_trace_on = on & 15;
   return GEMM_OK;
 }
 

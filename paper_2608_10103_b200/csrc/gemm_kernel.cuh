@@ -124,13 +124,16 @@ struct SmemLayout {
 
 // Bounded wait: polls the barrier; after the limit (or once another role has
 // given up) records `code` and returns false.  The caller then leaves its loop.
+template <bool BACKOFF = false>
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity,
-                                             volatile uint32_t* abort_flag, int* status, int code) {
+                                             volatile uint32_t* abort_flag, int* status, int code,
+                                             uint32_t backoff_ns = 0) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
   uint64_t t0 = 0;
   uint32_t spins = 0;
   while (true) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
+    if (BACKOFF && backoff_ns) __nanosleep(backoff_ns);
     if ((++spins & 255u) == 0) {
       if (*abort_flag) return false;
       uint64_t now = ptx::globaltimer_ns();
@@ -195,6 +198,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   const int tile_stride = static_cast<int>(gridDim.x) / CTA_GROUP;
   unsigned long long* const trace =
       p.trace ? p.trace + static_cast<size_t>(blockIdx.x) * TRACE_SLOTS : nullptr;
+  if (trace && threadIdx.x < TRACE_SLOTS) trace[threadIdx.x] = 0;  // roles that do not run leave 0
   const long long clk_start = trace ? clock64() : 0;
   const uint64_t ns_start = trace ? ptx::globaltimer_ns() : 0;
 
@@ -403,7 +407,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       int tm, tn;
       tile_coords(p, t, tm, tn);
       const long long w0 = trace ? clock64() : 0;
-      ok = wait_bounded(acc_full_bar(acc), acc_phase, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+      ok = wait_bounded<true>(acc_full_bar(acc), acc_phase, abort_flag, p.status,
+                              DEV_TIMEOUT_EPILOGUE, (p.ablate & 4) ? 500u : 0u);
       ok = __all_sync(0xffffffffu, ok);
       const long long w1 = trace ? clock64() : 0;
       epi_wait += w1 - w0;
