@@ -100,6 +100,37 @@ int gemm_s4_ws(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t*
                void* workspace, size_t workspace_bytes, gemm_stream_t stream);
 
 /*
+ * FP16 inputs, FP32 accumulate, FP16 OUTPUT: each FP32 sum is rounded once to
+ * binary16 (round to nearest even) on the way out, halving the bytes of C.
+ * (The study's closest variant, fp16_ptx_fp16acc in Table VI, keeps FP16
+ * accumulators; here only the stored result is narrowed, so the error is the
+ * FP32 path's plus one half-precision rounding.)  C: M x N binary16, row-major.
+ * Alignment as gemm_fp16; rows of C that are not 16-byte multiples (N % 8 != 0)
+ * take a slower scalar store path.
+ */
+int gemm_fp16_f16out(int M, int N, int K, const void* A, const void* B, void* C,
+                     gemm_stream_t stream);
+
+/*
+ * INT8 / INT4 GEMM with the dequantisation fused into the epilogue -- the step
+ * the study leaves to the surrounding inference pipeline (Sec. VI: its kernels
+ * stop at INT32 "without in-kernel dequantization or scaling"):
+ *
+ *     C[i][j] = float(sum_k a(i,k) * b(j,k)) * row_scale[i] * col_scale[j]
+ *
+ * computed in FP32 from the exact INT32 sum (conversion and the two products
+ * each round once), stored as FP32 (c_is_fp16 = 0) or rounded once more to
+ * binary16 (c_is_fp16 = 1).  row_scale: M floats, col_scale: N floats, device
+ * memory, 4-byte aligned.  Operand layouts, K rules and (for INT4) the internal
+ * workspace are those of gemm_s8 / gemm_s4.
+ */
+int gemm_s8_dequant(int M, int N, int K, const int8_t* A, const int8_t* B, const float* row_scale,
+                    const float* col_scale, void* C, int c_is_fp16, gemm_stream_t stream);
+int gemm_s4_dequant(int M, int N, int K, const uint8_t* A, const uint8_t* B,
+                    const float* row_scale, const float* col_scale, void* C, int c_is_fp16,
+                    gemm_stream_t stream);
+
+/*
  * gemm_s4 for callers that cannot allocate device memory.  (The paper has no
  * counterpart: its INT4 kernels need no scratch.)
  *

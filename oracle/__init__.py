@@ -170,3 +170,60 @@ def fp16_check(C_got, C_ref, S):
     ratio = np.abs(got - C_ref) / fp16_bound(S)
     worst = float(ratio.max())
     return worst <= 1.0, worst
+
+
+# ---------------------------------------------------------------------------
+# Output variants: FP16-rounded C and dequantised integer GEMM.  The reference
+# values are the exact sums above pushed through the definition in fp64; the
+# bounds add the roundings the definition allows.
+# ---------------------------------------------------------------------------
+HALF_EPS = 2.0 ** -11          # half an ulp of binary16, relative (normal range)
+HALF_TINY = 2.0 ** -25         # half the smallest binary16 subnormal
+FLOAT_EPS = 2.0 ** -24         # half an ulp of binary32, relative
+
+
+def fp16_out_bound(C_ref, S):
+    """FP32-accumulate bound plus one rounding of the result to binary16."""
+    return fp16_bound(S) + HALF_EPS * np.abs(C_ref) + HALF_TINY
+
+
+def fp16_out_check(C_got, C_ref, S):
+    got = np.asarray(C_got)
+    if got.dtype != np.float16 or got.shape != C_ref.shape:
+        return False, float("inf")
+    got = got.astype(np.float64)
+    if got.size == 0:
+        return True, 0.0
+    if not np.isfinite(got).all():
+        return False, float("inf")
+    ratio = np.abs(got - C_ref) / fp16_out_bound(C_ref, S)
+    worst = float(ratio.max())
+    return worst <= 1.0, worst
+
+
+def dequant_ref(C64, row_scale, col_scale):
+    """C[i][j] = sum * row_scale[i] * col_scale[j], in fp64 from the exact integer sums."""
+    rs = np.asarray(row_scale, dtype=np.float32).astype(np.float64)
+    cs = np.asarray(col_scale, dtype=np.float32).astype(np.float64)
+    assert C64.shape == (rs.size, cs.size)
+    return C64.astype(np.float64) * rs[:, None] * cs[None, :]
+
+
+def dequant_check(C_got, ref, out_is_fp16):
+    """The definition allows three FP32 roundings (int -> float, two products) and, for
+    binary16 output, one more; the bound is their sum with a 2x margin on the FP32 part."""
+    got = np.asarray(C_got)
+    want_dtype = np.float16 if out_is_fp16 else np.float32
+    if got.dtype != want_dtype or got.shape != ref.shape:
+        return False, float("inf")
+    got = got.astype(np.float64)
+    if got.size == 0:
+        return True, 0.0
+    if not np.isfinite(got).all():
+        return False, float("inf")
+    bound = 6 * FLOAT_EPS * np.abs(ref) + 1e-37
+    if out_is_fp16:
+        bound = bound + HALF_EPS * np.abs(ref) + HALF_TINY
+    ratio = np.abs(got - ref) / bound
+    worst = float(ratio.max())
+    return worst <= 1.0, worst

@@ -21,6 +21,7 @@ PRECISION_ID = {"fp16": PREC_FP16, "s8": PREC_S8, "s4": PREC_S4}
 
 EXPORTS = (
     "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
+    "gemm_fp16_f16out", "gemm_s8_dequant", "gemm_s4_dequant",
     "gemm_s4_static", "gemm_s4_static_capacity", "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
     "gemm_set_config_override", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_last_device_status", "gemm_last_cuda_error",
     "gemm_status_string", "gemm_version",
@@ -57,6 +58,9 @@ def lib() -> ctypes.CDLL:
         L.gemm_s8.argtypes = [i, i, i, vp, vp, vp, vp]
         L.gemm_s4.argtypes = [i, i, i, vp, vp, vp, vp]
         L.gemm_s4_ws.argtypes = [i, i, i, vp, vp, vp, vp, sz, vp]
+        L.gemm_fp16_f16out.argtypes = [i, i, i, vp, vp, vp, vp]
+        L.gemm_s8_dequant.argtypes = [i, i, i, vp, vp, vp, vp, vp, i, vp]
+        L.gemm_s4_dequant.argtypes = [i, i, i, vp, vp, vp, vp, vp, i, vp]
         L.gemm_s4_workspace_bytes.argtypes = [i, i, i]
         L.gemm_s4_workspace_bytes.restype = sz
         L.gemm_s4_static.argtypes = [i, i, i, vp, vp, vp, vp]
@@ -144,6 +148,50 @@ def gemm_s4(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor | None = None, str
     _check(lib().gemm_s4(M, N, 2 * Kh, _dev_ptr(A, torch.uint8, "A"), _dev_ptr(B, torch.uint8, "B"),
                          _dev_ptr(C, torch.int32, "C"), _stream_handle(stream)), "gemm_s4")
     return C
+
+
+def gemm_fp16_f16out(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor | None = None, stream=None):
+    """C[M,N] (float16) = A[M,K] (float16) @ B[N,K]^T, FP32 accumulate, one rounding to half."""
+    M, K = A.shape
+    N, Kb = B.shape
+    if K != Kb:
+        raise ValueError("A and B disagree on K")
+    C = _out(C, M, N, torch.float16, A.device)
+    _check(lib().gemm_fp16_f16out(M, N, K, _dev_ptr(A, torch.float16, "A"),
+                                  _dev_ptr(B, torch.float16, "B"), _dev_ptr(C, torch.float16, "C"),
+                                  _stream_handle(stream)), "gemm_fp16_f16out")
+    return C
+
+
+def _dequant(fn_name, A, B, K, row_scale, col_scale, C, out_dtype, a_dtype, stream):
+    M, N = A.shape[0], B.shape[0]
+    if out_dtype not in (torch.float32, torch.float16):
+        raise TypeError("out_dtype must be float32 or float16")
+    C = _out(C, M, N, out_dtype, A.device)
+    if row_scale.numel() != M or col_scale.numel() != N:
+        raise ValueError("row_scale needs M entries, col_scale N")
+    _check(getattr(lib(), fn_name)(M, N, K, _dev_ptr(A, a_dtype, "A"), _dev_ptr(B, a_dtype, "B"),
+                                   _dev_ptr(row_scale, torch.float32, "row_scale"),
+                                   _dev_ptr(col_scale, torch.float32, "col_scale"),
+                                   _dev_ptr(C, out_dtype, "C"), 1 if out_dtype == torch.float16 else 0,
+                                   _stream_handle(stream)), fn_name)
+    return C
+
+
+def gemm_s8_dequant(A, B, row_scale, col_scale, C=None, out_dtype=torch.float32, stream=None):
+    """C[i,j] = float(int32 sum) * row_scale[i] * col_scale[j], as float32 or float16."""
+    if A.shape[1] != B.shape[1]:
+        raise ValueError("A and B disagree on K")
+    return _dequant("gemm_s8_dequant", A, B, A.shape[1], row_scale, col_scale, C, out_dtype,
+                    torch.int8, stream)
+
+
+def gemm_s4_dequant(A, B, row_scale, col_scale, C=None, out_dtype=torch.float32, stream=None):
+    """gemm_s8_dequant for packed signed 4-bit operands ((rows, K/2) uint8)."""
+    if A.shape[1] != B.shape[1]:
+        raise ValueError("A and B disagree on K")
+    return _dequant("gemm_s4_dequant", A, B, 2 * A.shape[1], row_scale, col_scale, C, out_dtype,
+                    torch.uint8, stream)
 
 
 def gemm_s4_workspace_bytes(M: int, N: int, K: int) -> int:

@@ -31,7 +31,7 @@ struct DeviceState {
   unsigned long long* trace_ptr = nullptr;
   void* s4_workspace = nullptr;
   size_t s4_workspace_bytes = 0;
-  uint64_t attr_set = 0;  // bit i: dynamic-smem attribute set for kernel variant i
+  uint64_t attr_set[2] = {0, 0};  // bit i: dynamic-smem attribute set for kernel variant i
 };
 
 std::mutex g_mutex;
@@ -107,14 +107,16 @@ int encode_operand_map(CUtensorMap* map, CUtensorMapDataType type, int elem_byte
   return GEMM_OK;
 }
 
-// C (or any row-major 32-bit matrix) for the epilogue's TMA stores: boxes of 32 rows x
-// 32 values (128 bytes), 128-byte swizzle.  Needs a 16-byte aligned base and pitch.
-int encode_c_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols) {
+// C (row-major, 32- or 16-bit elements) for the epilogue's TMA stores: boxes of 32 rows x
+// 128 bytes, 128-byte swizzle.  Needs a 16-byte aligned base and pitch.
+int encode_c_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, int elem_bytes) {
   cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 4};
-  cuuint32_t box[2] = {32, 32};
+  cuuint64_t strides[1] = {cols * static_cast<uint64_t>(elem_bytes)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elem_bytes), 32};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(ptr), dims,
+  CUresult r = g_encode(map, elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
+                                             : CU_TENSOR_MAP_DATA_TYPE_UINT16,
+                        2, const_cast<void*>(ptr), dims,
                         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -160,14 +162,14 @@ int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b
 // large ones want the CTA-pair tile, which halves the B bytes each SM pulls
 // from L2.  Cost model: waves of tiles x (tile width + a fixed per-tile
 // overhead), with a discount for the pair shape.
-TileConfig select_config(int M, int N, int num_sms) {
+TileConfig select_config(int M, int N, int num_sms, int min_bn = 32) {
   TileConfig best{256, 2, 6, 8};
   long long best_cost = -1;
   for (int cg = 2; cg >= 1; --cg) {
     if (g_override_cta_group && cg != g_override_cta_group) continue;
     for (int bn : kWidths) {
       if (g_override_bn && bn != g_override_bn) continue;
-      if (!variant_exists(bn, cg)) continue;
+      if (!variant_exists(bn, cg) || bn < min_bn) continue;
       long long tiles = static_cast<long long>(ceil_div(M, BM * cg)) * ceil_div(N, bn);
       long long units = num_sms / cg;
       long long waves = (tiles + units - 1) / units;
@@ -178,6 +180,10 @@ TileConfig select_config(int M, int N, int num_sms) {
         best.cta_group = cg;
       }
     }
+  }
+  if (best_cost < 0) {  // the override names a shape this output mode does not have
+    best.bn = 0;
+    return best;
   }
   best.stages = stages_for(best.bn, best.cta_group);
   // Band height: one wave of tiles about twice as tall as wide in operand bytes (measured
@@ -194,16 +200,16 @@ TileConfig select_config(int M, int N, int num_sms) {
   return best;
 }
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB>
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI>
 int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUtensorMap& tb,
                    const CUtensorMap& tc, const GemmParams& p, cudaStream_t stream) {
   using L = SmemLayout<BN, STAGES, CTA_GROUP, KB>;
-  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB>;
-  if (!(s->attr_set & (1ull << variant))) {
+  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI>;
+  if (!(s->attr_set[variant >> 6] & (1ull << (variant & 63)))) {
     cudaError_t e =
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
     if (e != cudaSuccess) return cuda_fail(e);
-    s->attr_set |= 1ull << variant;
+    s->attr_set[variant >> 6] |= 1ull << (variant & 63);
   }
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   const long long units = s->num_sms / CTA_GROUP;
@@ -225,18 +231,27 @@ int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUt
   return GEMM_OK;
 }
 
+// Output options of one GEMM call.
+struct OutputSpec {
+  int epi = EPI_RAW32;
+  const float* row_scale = nullptr;
+  const float* col_scale = nullptr;
+};
+
 // A, B already in the element type of KIND (fp16 or int8), pitches in bytes.
-template <int KIND>
-int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* B, size_t b_pitch,
-                void* C, cudaStream_t stream) {
+template <int KIND, int EPI>
+int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const void* B,
+                    size_t b_pitch, void* C, const OutputSpec& out, cudaStream_t stream) {
   std::lock_guard<std::mutex> lock(g_mutex);
   DeviceState* s = nullptr;
   int rc = device_state(&s);
   if (rc != GEMM_OK) return rc;
   constexpr int ELEM = (KIND == ptx::KIND_F16) ? 2 : 1;
+  constexpr int C_ELEM = (EPI == EPI_OUT16) ? 2 : 4;
   const CUtensorMapDataType type =
       (KIND == ptx::KIND_F16) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
-  const TileConfig cfg = select_config(M, N, s->num_sms);
+  const TileConfig cfg = select_config(M, N, s->num_sms, EPI == EPI_OUT16 ? 64 : 32);
+  if (cfg.bn == 0) return GEMM_ERR_INVALID_ARG;  // override asks for a shape this mode lacks
 
   CUtensorMap ta, tb;
   const bool promote = !(g_l2_policy & 16);
@@ -253,15 +268,17 @@ int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* 
   p.tiles_n = ceil_div(N, cfg.bn);
   p.group_m = cfg.group_m;
   p.k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
-  p.c_vec_ok = (N % 4 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+  p.c_vec_ok = (N % (16 / C_ELEM) == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
   CUtensorMap tc;
   if (p.c_vec_ok) {
-    rc = encode_c_map(&tc, C, M, N);
+    rc = encode_c_map(&tc, C, M, N, C_ELEM);
     if (rc != GEMM_OK) return rc;
   } else {
     tc = ta;  // unused by the kernel on the plain-store path
   }
   p.C = static_cast<uint32_t*>(C);
+  p.row_scale = out.row_scale;
+  p.col_scale = out.col_scale;
   p.status = s->status_ptr;
   p.trace = (g_trace_on & 1) ? s->trace_ptr : nullptr;
   p.ablate = (g_trace_on >> 1) & 7;
@@ -269,20 +286,40 @@ int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* 
   p.serpentine_k = (g_l2_policy & 4) ? 0 : 1;
   p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
 
-  const int kbase = (KIND == ptx::KIND_F16) ? 0 : 16;
+  const int vbase = ((KIND == ptx::KIND_F16) ? 0 : 32) + EPI * 8;  // bit index in attr_set
   if (cfg.cta_group == 2) {
     switch (cfg.bn) {
-      case 256: return launch_variant<KIND, 256, 6, 2, 1>(s, kbase + 8, ta, tb, tc, p, stream);
-      case 128: return launch_variant<KIND, 128, 8, 2, 1>(s, kbase + 9, ta, tb, tc, p, stream);
-      case 64: return launch_variant<KIND, 64, 8, 2, 1>(s, kbase + 10, ta, tb, tc, p, stream);
+      case 256: return launch_variant<KIND, 256, 6, 2, 1, EPI>(s, vbase + 4, ta, tb, tc, p, stream);
+      case 128: return launch_variant<KIND, 128, 8, 2, 1, EPI>(s, vbase + 5, ta, tb, tc, p, stream);
+      case 64: return launch_variant<KIND, 64, 8, 2, 1, EPI>(s, vbase + 6, ta, tb, tc, p, stream);
       default: return GEMM_ERR_INVALID_ARG;
     }
   }
   switch (cfg.bn) {
-    case 256: return launch_variant<KIND, 256, 4, 1, 1>(s, kbase + 0, ta, tb, tc, p, stream);
-    case 128: return launch_variant<KIND, 128, 6, 1, 1>(s, kbase + 1, ta, tb, tc, p, stream);
-    case 64: return launch_variant<KIND, 64, 8, 1, 1>(s, kbase + 2, ta, tb, tc, p, stream);
-    case 32: return launch_variant<KIND, 32, 8, 1, 1>(s, kbase + 3, ta, tb, tc, p, stream);
+    case 256: return launch_variant<KIND, 256, 4, 1, 1, EPI>(s, vbase + 0, ta, tb, tc, p, stream);
+    case 128: return launch_variant<KIND, 128, 6, 1, 1, EPI>(s, vbase + 1, ta, tb, tc, p, stream);
+    case 64: return launch_variant<KIND, 64, 8, 1, 1, EPI>(s, vbase + 2, ta, tb, tc, p, stream);
+    case 32:
+      if constexpr (EPI != EPI_OUT16)
+        return launch_variant<KIND, 32, 8, 1, 1, EPI>(s, vbase + 3, ta, tb, tc, p, stream);
+      return GEMM_ERR_INVALID_ARG;
+    default: return GEMM_ERR_INVALID_ARG;
+  }
+}
+
+template <int KIND>
+int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* B, size_t b_pitch,
+                void* C, cudaStream_t stream, const OutputSpec& out = OutputSpec()) {
+  switch (out.epi) {
+    case EPI_RAW32:
+      return launch_gemm_epi<KIND, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+    case EPI_OUT16:
+      return launch_gemm_epi<KIND, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+    case EPI_F32_SCALED:
+      if constexpr (KIND == ptx::KIND_I8)
+        return launch_gemm_epi<KIND, EPI_F32_SCALED>(M, N, K, A, a_pitch, B, b_pitch, C, out,
+                                                     stream);
+      return GEMM_ERR_INVALID_ARG;
     default: return GEMM_ERR_INVALID_ARG;
   }
 }
@@ -322,6 +359,66 @@ int check_s4(int M, int N, int K, const void* A, const void* B, const void* C) {
   return GEMM_OK;
 }
 
+size_t s4_workspace_need(int M, int N, int K) {
+  return align_up(static_cast<size_t>(M) * K, 256) + align_up(static_cast<size_t>(N) * K, 256);
+}
+
+// INT4 GEMM through caller-visible scratch: unpack A and B to int8, then the INT8 kernel.
+int s4_with_workspace(int M, int N, int K, const uint8_t* A, const uint8_t* B, void* C,
+                      void* workspace, size_t workspace_bytes, const OutputSpec& out,
+                      cudaStream_t st) {
+  if (!workspace) return GEMM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < s4_workspace_need(M, N, K))
+    return GEMM_ERR_WORKSPACE;
+  int8_t* a8 = static_cast<int8_t*>(workspace);
+  int8_t* b8 = a8 + align_up(static_cast<size_t>(M) * K, 256);
+  int rc;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState* s = nullptr;
+    rc = device_state(&s);
+    if (rc != GEMM_OK) return rc;
+  }
+  rc = launch_unpack(M, A, a8, N, B, b8, K, static_cast<size_t>(K), st);
+  if (rc != GEMM_OK) return rc;
+  return launch_gemm<ptx::KIND_I8>(M, N, K, a8, static_cast<size_t>(K), b8, static_cast<size_t>(K),
+                                   C, st, out);
+}
+
+// The library's own grow-only scratch for the current device (cudaMalloc on growth).
+int s4_internal_workspace(size_t need, void** ws, size_t* ws_bytes) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceState* s = nullptr;
+  int rc = device_state(&s);
+  if (rc != GEMM_OK) return rc;
+  if (s->s4_workspace_bytes < need) {
+    // Grow: earlier launches may still read the old buffer.
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (s->s4_workspace) cudaFree(s->s4_workspace);
+    s->s4_workspace = nullptr;
+    s->s4_workspace_bytes = 0;
+    e = cudaMalloc(&s->s4_workspace, need);
+    if (e != cudaSuccess) return cuda_fail(e);
+    s->s4_workspace_bytes = need;
+  }
+  *ws = s->s4_workspace;
+  *ws_bytes = s->s4_workspace_bytes;
+  return GEMM_OK;
+}
+
+int check_scales(const float* row_scale, const float* col_scale, const void* C, int c_is_fp16,
+                 OutputSpec* out) {
+  if (!row_scale || !col_scale || !C || (c_is_fp16 != 0 && c_is_fp16 != 1))
+    return GEMM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(row_scale) | reinterpret_cast<uintptr_t>(col_scale)) & 3)
+    return GEMM_ERR_MISALIGNED;
+  out->epi = c_is_fp16 ? EPI_OUT16 : EPI_F32_SCALED;
+  out->row_scale = row_scale;
+  out->col_scale = col_scale;
+  return GEMM_OK;
+}
+
 }  // namespace
 }  // namespace b200gemm
 
@@ -350,59 +447,68 @@ int gemm_s8(int M, int N, int K, const int8_t* A, const int8_t* B, int32_t* C,
 
 size_t gemm_s4_workspace_bytes(int M, int N, int K) {
   if (M <= 0 || N <= 0 || K <= 0) return 0;
-  return align_up(static_cast<size_t>(M) * K, 256) + align_up(static_cast<size_t>(N) * K, 256);
+  return s4_workspace_need(M, N, K);
 }
 
 int gemm_s4_ws(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t* C,
                void* workspace, size_t workspace_bytes, gemm_stream_t stream) {
   int rc = check_s4(M, N, K, A, B, C);
   if (rc != GEMM_OK) return rc;
-  if (!workspace) return GEMM_ERR_INVALID_ARG;
-  if ((reinterpret_cast<uintptr_t>(workspace) & 255) ||
-      workspace_bytes < gemm_s4_workspace_bytes(M, N, K))
-    return GEMM_ERR_WORKSPACE;
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  int8_t* a8 = static_cast<int8_t*>(workspace);
-  int8_t* b8 = a8 + align_up(static_cast<size_t>(M) * K, 256);
-  {
-    std::lock_guard<std::mutex> lock(g_mutex);
-    DeviceState* s = nullptr;
-    rc = device_state(&s);
-    if (rc != GEMM_OK) return rc;
-  }
-  rc = launch_unpack(M, A, a8, N, B, b8, K, static_cast<size_t>(K), st);
-  if (rc != GEMM_OK) return rc;
-  return launch_gemm<ptx::KIND_I8>(M, N, K, a8, static_cast<size_t>(K), b8, static_cast<size_t>(K),
-                                   C, st);
+  return s4_with_workspace(M, N, K, A, B, C, workspace, workspace_bytes, OutputSpec(),
+                           reinterpret_cast<cudaStream_t>(stream));
 }
 
 int gemm_s4(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t* C,
             gemm_stream_t stream) {
   int rc = check_s4(M, N, K, A, B, C);
   if (rc != GEMM_OK) return rc;
-  const size_t need = gemm_s4_workspace_bytes(M, N, K);
   void* ws = nullptr;
   size_t ws_bytes = 0;
-  {
-    std::lock_guard<std::mutex> lock(g_mutex);
-    DeviceState* s = nullptr;
-    rc = device_state(&s);
-    if (rc != GEMM_OK) return rc;
-    if (s->s4_workspace_bytes < need) {
-      // Grow: earlier launches may still read the old buffer.
-      cudaError_t e = cudaDeviceSynchronize();
-      if (e != cudaSuccess) return cuda_fail(e);
-      if (s->s4_workspace) cudaFree(s->s4_workspace);
-      s->s4_workspace = nullptr;
-      s->s4_workspace_bytes = 0;
-      e = cudaMalloc(&s->s4_workspace, need);
-      if (e != cudaSuccess) return cuda_fail(e);
-      s->s4_workspace_bytes = need;
-    }
-    ws = s->s4_workspace;
-    ws_bytes = s->s4_workspace_bytes;
-  }
-  return gemm_s4_ws(M, N, K, A, B, C, ws, ws_bytes, stream);
+  rc = s4_internal_workspace(s4_workspace_need(M, N, K), &ws, &ws_bytes);
+  if (rc != GEMM_OK) return rc;
+  return s4_with_workspace(M, N, K, A, B, C, ws, ws_bytes, OutputSpec(),
+                           reinterpret_cast<cudaStream_t>(stream));
+}
+
+int gemm_fp16_f16out(int M, int N, int K, const void* A, const void* B, void* C,
+                     gemm_stream_t stream) {
+  int rc = check_common(M, N, K, A, B, C);
+  if (rc != GEMM_OK) return rc;
+  if (K % 8) return GEMM_ERR_MISALIGNED;
+  OutputSpec out;
+  out.epi = EPI_OUT16;
+  return launch_gemm<ptx::KIND_F16>(M, N, K, A, static_cast<size_t>(K) * 2, B,
+                                    static_cast<size_t>(K) * 2, C,
+                                    reinterpret_cast<cudaStream_t>(stream), out);
+}
+
+int gemm_s8_dequant(int M, int N, int K, const int8_t* A, const int8_t* B, const float* row_scale,
+                    const float* col_scale, void* C, int c_is_fp16, gemm_stream_t stream) {
+  int rc = check_common(M, N, K, A, B, C);
+  if (rc != GEMM_OK) return rc;
+  if (K % 16) return GEMM_ERR_MISALIGNED;
+  if (K > K_LIMIT_INT) return GEMM_ERR_K_TOO_LARGE;
+  OutputSpec out;
+  rc = check_scales(row_scale, col_scale, C, c_is_fp16, &out);
+  if (rc != GEMM_OK) return rc;
+  return launch_gemm<ptx::KIND_I8>(M, N, K, A, static_cast<size_t>(K), B, static_cast<size_t>(K), C,
+                                   reinterpret_cast<cudaStream_t>(stream), out);
+}
+
+int gemm_s4_dequant(int M, int N, int K, const uint8_t* A, const uint8_t* B,
+                    const float* row_scale, const float* col_scale, void* C, int c_is_fp16,
+                    gemm_stream_t stream) {
+  int rc = check_s4(M, N, K, A, B, C);
+  if (rc != GEMM_OK) return rc;
+  OutputSpec out;
+  rc = check_scales(row_scale, col_scale, C, c_is_fp16, &out);
+  if (rc != GEMM_OK) return rc;
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  rc = s4_internal_workspace(s4_workspace_need(M, N, K), &ws, &ws_bytes);
+  if (rc != GEMM_OK) return rc;
+  return s4_with_workspace(M, N, K, A, B, C, ws, ws_bytes, out,
+                           reinterpret_cast<cudaStream_t>(stream));
 }
 
 int gemm_release_workspaces(void) {

@@ -34,6 +34,7 @@
 #pragma once
 
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -57,6 +58,14 @@ enum DeviceStatus {
   DEV_TIMEOUT_DRAIN = 4,
 };
 
+// What the epilogue writes.
+enum EpiMode {
+  EPI_RAW32 = 0,       // the 32-bit accumulators as they are (FP32 resp. INT32)
+  EPI_OUT16 = 1,       // binary16: FP32 accumulators rounded once (RNE); INT32 accumulators
+                       // converted to float and multiplied by row_scale[i] * col_scale[j] first
+  EPI_F32_SCALED = 2,  // float(INT32 accumulator) * row_scale[i] * col_scale[j]
+};
+
 struct GemmParams {
   int M, N, K;
   int tiles_m, tiles_n;  // number of C tiles (128*CTA_GROUP x BN) along M and N
@@ -64,7 +73,9 @@ struct GemmParams {
   int k_blocks;          // ceil(K bytes / BK_BYTES): 128-byte K atoms to cover K
   int c_vec_ok;          // 1 if C rows allow 16-byte accesses (N % 4 == 0, base 16-byte aligned):
                          // the epilogue then stages C in shared memory and stores it by TMA
-  uint32_t* C;
+  uint32_t* C;           // element size 4 bytes, or 2 with EPI_OUT16
+  const float* row_scale;  // EPI_OUT16 (integer kinds) / EPI_F32_SCALED: M per-row factors
+  const float* col_scale;  // and N per-column factors; both null = no scaling (FP16 kind)
   int* status;           // device status word (0 = ok)
   // Optional per-CTA cycle accounting (TRACE_SLOTS 64-bit words per CTA), or null.
   unsigned long long* trace;
@@ -161,7 +172,19 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int t, int& tm,
   tn = r / rows_in_band;
 }
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB>
+// Accumulator bits -> output value as float (identity for raw mode is handled by the caller).
+template <int KIND>
+__device__ __forceinline__ float acc_to_float(uint32_t bits) {
+  if constexpr (KIND == ptx::KIND_F16) return __uint_as_float(bits);
+  return static_cast<float>(static_cast<int32_t>(bits));
+}
+
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
@@ -417,51 +440,85 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       const int row0 = tm * TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
       const int row = row0 + lane;
       const int col0 = tn * BN;
-      if (p.c_vec_ok) {
-        // TMEM -> registers -> swizzled shared memory -> one TMA store per 32 x 32 block.
-        // Thread `lane` owns row `lane` of the block; 16-byte chunk j of the row goes to
-        // chunk j ^ (lane & 7), the 128-byte swizzle the C tensor map expects, which also
-        // spreads the warp's 16-byte stores over all banks.
+      float rs = 1.0f;
+      if constexpr (EPI != EPI_RAW32) {
+        if (p.row_scale && row < p.M) rs = __ldg(p.row_scale + row);
+      }
+      // One staging block = 32 rows x 128 bytes = 32 columns of 32-bit or 64 columns of
+      // 16-bit results.  Thread `lane` owns row `lane`; 16-byte chunk j of the row goes to
+      // chunk j ^ (lane & 7), the 128-byte swizzle the C tensor map expects, which also
+      // spreads the warp's 16-byte stores over all banks.
+      constexpr int BLOCK_COLS = (EPI == EPI_OUT16) ? 64 : 32;
+      static_assert(BN % BLOCK_COLS == 0, "tile width must be a multiple of the store block");
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t r[32];
+      for (int c = 0; c < BN / BLOCK_COLS; ++c) {
+        const int col = col0 + c * BLOCK_COLS;
+        uint32_t w[32];  // the thread's 128 bytes of output
+        if constexpr (EPI == EPI_RAW32) {
           ptx::tmem_ld_32x32b_x32(
-              tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), r);
+              tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), w);
+          ptx::tmem_wait_ld();
+        } else if constexpr (EPI == EPI_F32_SCALED) {
+          ptx::tmem_ld_32x32b_x32(
+              tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), w);
+          ptx::tmem_wait_ld();
+#pragma unroll
+          for (int v = 0; v < 32; ++v) {
+            const float cs = (col + v < p.N) ? __ldg(p.col_scale + col + v) : 0.0f;
+            w[v] = __float_as_uint(acc_to_float<KIND>(w[v]) * rs * cs);
+          }
+        } else {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint32_t r[32];
+            ptx::tmem_ld_32x32b_x32(
+                tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 64 + h * 32), r);
+            ptx::tmem_wait_ld();
+#pragma unroll
+            for (int v = 0; v < 32; v += 2) {
+              float x0 = acc_to_float<KIND>(r[v]), x1 = acc_to_float<KIND>(r[v + 1]);
+              if (p.col_scale) {
+                const int cc = col + h * 32 + v;
+                x0 *= rs * ((cc < p.N) ? __ldg(p.col_scale + cc) : 0.0f);
+                x1 *= rs * ((cc + 1 < p.N) ? __ldg(p.col_scale + cc + 1) : 0.0f);
+              }
+              w[h * 16 + v / 2] = pack_half2(x0, x1);
+            }
+          }
+        }
+        if (p.c_vec_ok) {
+          // registers -> swizzled shared memory -> one TMA store per block
           const uint32_t buf = epi_base + static_cast<uint32_t>((c & 1) * L::EPI_BUF_BYTES);
           // the store issued from this buffer two blocks ago must have read it
           if (lane == 0) ptx::bulk_wait_group_read<1>();
           __syncwarp();
-          ptx::tmem_wait_ld();
           const uint32_t row_addr = buf + static_cast<uint32_t>(lane * 128);
 #pragma unroll
           for (int j = 0; j < 8; ++j)
-            ptx::st_shared_v4(row_addr + static_cast<uint32_t>(((j ^ (lane & 7)) * 16)), r[4 * j],
-                              r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+            ptx::st_shared_v4(row_addr + static_cast<uint32_t>(((j ^ (lane & 7)) * 16)), w[4 * j],
+                              w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
           ptx::fence_proxy_async_smem();
           __syncwarp();
           // Partly outside C: the hardware clips.  Wholly outside: issue no store, but still
           // close a (then empty) group so that "one group per block" keeps the buffer
           // reuse rule above exact.
           if (lane == 0) {
-            if (row0 < p.M && col0 + c * 32 < p.N)
-              ptx::tma_store_2d(&tmap_c, col0 + c * 32, row0, buf, pol_c);
+            if (row0 < p.M && col < p.N) ptx::tma_store_2d(&tmap_c, col, row0, buf, pol_c);
             ptx::bulk_commit_group();
           }
-        }
-      } else {
-        // C rows are not 16-byte multiples: plain predicated stores.
-        uint32_t* crow = p.C + static_cast<size_t>(row) * p.N;
-#pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t r[32];
-          ptx::tmem_ld_32x32b_x32(
-              tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), r);
-          ptx::tmem_wait_ld();
-          const int col = col0 + c * 32;
-          if (row < p.M) {
+        } else if (row < p.M) {
+          // C rows are not 16-byte multiples: plain predicated stores.
+          if constexpr (EPI == EPI_OUT16) {
+            uint16_t* crow = reinterpret_cast<uint16_t*>(p.C) + static_cast<size_t>(row) * p.N;
+#pragma unroll
+            for (int v = 0; v < 64; ++v)
+              if (col + v < p.N)
+                crow[col + v] = static_cast<uint16_t>(w[v / 2] >> (16 * (v & 1)));
+          } else {
+            uint32_t* crow = p.C + static_cast<size_t>(row) * p.N;
 #pragma unroll
             for (int v = 0; v < 32; ++v)
-              if (col + v < p.N) crow[col + v] = r[v];
+              if (col + v < p.N) crow[col + v] = w[v];
           }
         }
       }

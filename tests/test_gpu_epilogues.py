@@ -1,0 +1,144 @@
+"""GPU parity of the output variants: FP16-rounded C and fused dequantisation.
+References come from the oracle's exact sums pushed through the definition in fp64."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_10103_b200 import binding, synth
+from gpu_util import to_dev
+
+pytestmark = pytest.mark.gpu
+
+SHAPES16 = [(64, 1), (128, 1), (256, 1), (64, 2), (128, 2), (256, 2)]
+
+
+@pytest.fixture(autouse=True)
+def _clean_state():
+    binding.gemm_set_config_override(0, 0, 0)
+    yield
+    binding.gemm_set_config_override(0, 0, 0)
+    assert binding.gemm_last_device_status() == 0
+
+
+def scales(M, N, seed):
+    g = np.random.Generator(np.random.PCG64(seed))
+    rs = (g.uniform(0.5, 2.0, M) * g.choice([-1.0, 1.0], M) * 1e-2).astype(np.float32)
+    cs = (g.uniform(0.5, 2.0, N) * g.choice([-1.0, 1.0], N) * 1e-1).astype(np.float32)
+    return rs, cs
+
+
+def run_f16out(A, B):
+    C = torch.full((A.shape[0], B.shape[0]), float("nan"), dtype=torch.float16, device="cuda")
+    binding.gemm_fp16_f16out(to_dev(A), to_dev(B), C)
+    torch.cuda.synchronize()
+    return C.cpu().numpy()
+
+
+@pytest.mark.parametrize("M,N,K", [(512, 512, 512), (300, 520, 320), (129, 1032, 4128),
+                                   (200, 100, 128), (77, 3, 64), (1, 8, 8)])
+def test_fp16_out_full(M, N, K):
+    A, B = synth.fp16_uniform(M, N, K, seed=M + N)
+    ref, S = oracle.gemm_fp16(A, B)
+    ok, worst = oracle.fp16_out_check(run_f16out(A, B), ref, S)
+    assert ok, "error %.3g x bound" % worst
+
+
+@pytest.mark.parametrize("bn,cta_group", SHAPES16)
+def test_fp16_out_every_tile_shape(bn, cta_group):
+    M, N, K = 650, 1096, 1184
+    A, B = synth.fp16_normal_clipped(M, N, K, seed=bn + cta_group)
+    ref, S = oracle.gemm_fp16(A, B)
+    binding.gemm_set_config_override(bn, 0, cta_group)
+    ok, worst = oracle.fp16_out_check(run_f16out(A, B), ref, S)
+    assert ok, "error %.3g x bound" % worst
+
+
+def test_fp16_out_rejects_the_32_wide_tile():
+    A, B = synth.fp16_uniform(64, 64, 64, seed=1)
+    binding.gemm_set_config_override(32, 0, 1)
+    with pytest.raises(binding.GemmError):
+        run_f16out(A, B)
+
+
+def test_fp16_out_sampled_4096_and_exact_small_integers():
+    N = 4096
+    A, B = synth.fp16_normal_clipped(N, N, N, seed=3)
+    got = run_f16out(A, B)
+    rows, cols = synth.sample_rows_cols(N, N, seed=3)
+    ref, S = oracle.gemm_fp16(A, B, rows=rows)
+    assert oracle.fp16_out_check(got[rows], ref, S)[0]
+    ref, S = oracle.gemm_fp16(A, B, cols=cols)
+    assert oracle.fp16_out_check(got[:, cols], ref, S)[0]
+    # sums that are small integers are exact in binary16
+    a = np.zeros((256, 64), np.float16)
+    a[:, 0] = (np.arange(256) % 31) - 15
+    b = np.zeros((256, 64), np.float16)
+    b[:, 0] = (np.arange(256) % 29) - 14
+    want = np.outer(a[:, 0].astype(np.float64), b[:, 0].astype(np.float64))
+    assert np.array_equal(run_f16out(a, b).astype(np.float64), want)
+
+
+def run_dequant(prec, A, B, rs, cs, out_dtype):
+    fn = binding.gemm_s8_dequant if prec == "s8" else binding.gemm_s4_dequant
+    C = torch.full((A.shape[0], B.shape[0]), float("nan"), dtype=out_dtype, device="cuda")
+    fn(to_dev(A), to_dev(B), to_dev(rs), to_dev(cs), C, out_dtype)
+    torch.cuda.synchronize()
+    return C.cpu().numpy()
+
+
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.float16])
+@pytest.mark.parametrize("prec", ["s8", "s4"])
+@pytest.mark.parametrize("M,N,K", [(512, 512, 512), (300, 520, 320), (129, 1030, 4128),
+                                   (200, 100, 128), (77, 3, 64)])
+def test_dequant_full(prec, M, N, K, out_dtype):
+    A, B = synth.make(prec, M, N, K, seed=M + K)
+    rs, cs = scales(M, N, seed=N)
+    exact = oracle.gemm_s8_i64(A, B) if prec == "s8" else oracle.gemm_s4_i64(A, B, K)
+    ref = oracle.dequant_ref(exact, rs, cs)
+    ok, worst = oracle.dequant_check(run_dequant(prec, A, B, rs, cs, out_dtype), ref,
+                                     out_dtype == torch.float16)
+    assert ok, "error %.3g x bound" % worst
+
+
+@pytest.mark.parametrize("bn,cta_group", [(32, 1)] + SHAPES16)
+def test_dequant_every_tile_shape(bn, cta_group):
+    M, N, K = 650, 1096, 1184
+    A, B = synth.s8_uniform(M, N, K, seed=bn)
+    rs, cs = scales(M, N, seed=bn)
+    ref = oracle.dequant_ref(oracle.gemm_s8_i64(A, B), rs, cs)
+    binding.gemm_set_config_override(bn, 0, cta_group)
+    assert oracle.dequant_check(run_dequant("s8", A, B, rs, cs, torch.float32), ref, False)[0]
+    if bn >= 64:
+        assert oracle.dequant_check(run_dequant("s8", A, B, rs, cs, torch.float16), ref, True)[0]
+
+
+def test_dequant_with_unit_scales_is_the_exact_integer():
+    M, N, K = 384, 640, 256                      # |sum| <= 128*128*256 = 2^22: exact in float32
+    A, B = synth.s8_uniform(M, N, K, seed=5)
+    ones_r, ones_c = np.ones(M, np.float32), np.ones(N, np.float32)
+    got = run_dequant("s8", A, B, ones_r, ones_c, torch.float32)
+    assert np.array_equal(got.astype(np.int64), oracle.gemm_s8_i64(A, B))
+    # row / column scale really index rows / columns
+    rs = np.arange(1, M + 1, dtype=np.float32)
+    cs = np.ones(N, np.float32)
+    a = np.ones((M, K), np.int8)
+    b = np.ones((N, K), np.int8)
+    got = run_dequant("s8", a, b, rs, cs, torch.float32)
+    assert np.array_equal(got, np.repeat((K * rs)[:, None], N, axis=1))
+    got = run_dequant("s8", b, a, cs, rs, torch.float32)
+    assert np.array_equal(got, np.repeat((K * rs)[None, :], N, axis=0))
+
+
+def test_dequant_argument_errors():
+    L = binding.lib()
+    A = torch.zeros(64, 64, dtype=torch.int8, device="cuda")
+    C = torch.zeros(64, 64, dtype=torch.float32, device="cuda")
+    sc = torch.ones(64, dtype=torch.float32, device="cuda")
+    p, c, s = A.data_ptr(), C.data_ptr(), sc.data_ptr()
+    assert L.gemm_s8_dequant(64, 64, 64, p, p, None, s, c, 0, None) == -1
+    assert L.gemm_s8_dequant(64, 64, 64, p, p, s, s, c, 2, None) == -1
+    assert L.gemm_s8_dequant(64, 64, 64, p, p, s + 2, s, c, 0, None) == -2
+    assert L.gemm_s8_dequant(64, 64, 24, p, p, s, s, c, 0, None) == -2
+    assert L.gemm_s4_dequant(64, 64, 48, p, p, s, s, c, 0, None) == -2
+    assert L.gemm_fp16_f16out(64, 64, 12, p, p, c, None) == -2

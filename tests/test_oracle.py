@@ -366,3 +366,31 @@ def test_ops_convention_matches_paper_table(golden_dir):
         n = int(n)
         derived = synth.gemm_ops(n, n, n) / (float(ms) * 1e-3) / 1e12
         assert abs(derived - float(tops)) <= 0.012 * float(tops) + 5e-4, name
+
+
+# ------------------------------------------------------- output-variant references
+def test_fp16_out_bound_by_hand():
+    ref = np.array([[1.0 + 2.0 ** -11, 1000.0, 2.0 ** -26]])
+    S = np.zeros_like(ref)
+    # nearest halfs: 1.0 (tie -> even) or 1+2^-10, 1000.0, 0.0 -- all inside the bound
+    assert oracle.fp16_out_check(np.array([[1.0, 1000.0, 0.0]], np.float16), ref, S)[0]
+    assert oracle.fp16_out_check(np.array([[1.0 + 2.0 ** -10, 1000.0, 0.0]], np.float16), ref, S)[0]
+    # one half-ulp further is outside: 1 + 2^-9, 1001
+    assert not oracle.fp16_out_check(np.array([[1.0 + 2.0 ** -9, 1000.0, 0.0]], np.float16), ref, S)[0]
+    assert not oracle.fp16_out_check(np.array([[1.0, 1001.0, 0.0]], np.float16), ref, S)[0]
+    assert not oracle.fp16_out_check(np.array([[1.0, 1000.0, 0.0]], np.float32), ref, S)[0]
+
+
+def test_dequant_reference_by_hand():
+    C = np.array([[4, -6], [10, 0]], dtype=np.int64)
+    ref = oracle.dequant_ref(C, np.array([0.5, 2.0], np.float32), np.array([3.0, -0.25], np.float32))
+    assert ref.tolist() == [[6.0, 0.75], [60.0, -0.0]]
+    assert oracle.dequant_check(ref.astype(np.float32), ref, False)[0]
+    assert oracle.dequant_check(ref.astype(np.float16), ref, True)[0]
+    bad = ref.astype(np.float32)
+    bad[0, 0] = np.nextafter(np.float32(6.0), np.float32(7.0), dtype=np.float32) * np.float32(1 + 1e-5)
+    assert not oracle.dequant_check(bad, ref, False)[0]
+    assert not oracle.dequant_check(ref.astype(np.float32), ref, True)[0]
+    # scales are taken at float32 precision: 0.1 means float32(0.1)
+    r = oracle.dequant_ref(np.array([[10]], np.int64), [0.1], [1.0])
+    assert r[0, 0] == 10 * float(np.float32(0.1))
