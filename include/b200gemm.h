@@ -257,8 +257,12 @@ int gemm_set_l2_policy(int policy);
  * `on` is a bit set: 1 = record; 2 = ablation, issue no MMAs (operand loads and
  * barriers only); 4 = ablation, issue no operand loads (MMAs and barriers only,
  * on whatever shared memory holds); 8 = the epilogue's waits back off with
- * nanosleep instead of polling.  With bit 2 or 4 set C is garbage; the bits
- * exist to attribute cycles to the load path or the MMA path.
+ * nanosleep instead of polling; 16 = failure drill: one operand slot of the
+ * first tile is never filled, so the kernel's bounded waits (2 s) must expire,
+ * record a code for gemm_last_device_status, drain and return -- the call takes
+ * a few seconds, C is garbage and the context stays usable.  With bit 2, 4 or
+ * 16 set C is garbage; 2 and 4 exist to attribute cycles to the load path or
+ * the MMA path.
  */
 int gemm_trace_enable(int on);
 int gemm_trace_read(unsigned long long* out, int max_ctas);

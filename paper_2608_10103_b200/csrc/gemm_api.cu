@@ -281,7 +281,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.col_scale = out.col_scale;
   p.status = s->status_ptr;
   p.trace = (g_trace_on & 1) ? s->trace_ptr : nullptr;
-  p.ablate = (g_trace_on >> 1) & 7;
+  p.ablate = (g_trace_on >> 1) & 15;
   p.l2_policy = g_l2_policy & 3;
   p.serpentine_k = (g_l2_policy & 4) ? 0 : 1;
   p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
@@ -640,7 +640,7 @@ int gemm_set_l2_policy(int policy) {
 
 int gemm_trace_enable(int on) {
   std::lock_guard<std::mutex> lock(g_mutex);
-  g_trace_on = on & 15;
+  g_trace_on = on & 31;
   return GEMM_OK;
 }
 

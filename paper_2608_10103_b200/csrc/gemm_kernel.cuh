@@ -87,7 +87,10 @@ struct GemmParams {
   // K range its predecessor (same A rows) touched last and finds it still in L2.
   int serpentine_k;
   // Ablation switches for cycle accounting runs (results are then meaningless):
-  // bit 0 = issue no MMAs (loads + barriers only), bit 1 = issue no loads (MMAs + barriers only).
+  // bit 0 = issue no MMAs (loads + barriers only), bit 1 = issue no loads (MMAs + barriers only),
+  // bit 2 = epilogue waits back off with nanosleep, bit 3 = host-requested failure drill: the
+  // producer of CTA 0 leaves out the 3rd ring slot of its first tile, so the consumers' bounded
+  // waits must expire, record a status code and let the kernel drain and return.
   int ablate;
 };
 
@@ -288,6 +291,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const uint32_t b_dst = a_dst + KB * L::A_BYTES;
           if (!elected) {
             // nothing to issue in this lane
+          } else if ((p.ablate & 8) && blockIdx.x == 0 && t == first_tile && ks == 2) {
+            // failure drill: this slot is never filled
           } else if (p.ablate & 2) {
             if (leader) ptx::mbar_arrive(full_bar(stage));
           } else if constexpr (CTA_GROUP == 1) {

@@ -1,0 +1,43 @@
+"""The kernels never wait without a limit.  This drill makes one operand slot stay empty
+(a host-requested switch; nothing faults, traps or spins forever): the waits must run out
+after their 2 s limit, the kernel must record a status code, drain and return, and the
+next call on the same context must work."""
+import time
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_10103_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("cta_group", [1, 2])
+def test_expired_wait_is_reported_and_the_context_survives(cta_group):
+    M, N, K = 256, 256, 1024                      # one tile, 16 k-blocks (> ring depth)
+    A, B = synth.s8_uniform(M, N, K, seed=9)
+    dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    C = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    assert binding.gemm_last_device_status() == 0
+    binding.gemm_set_config_override(256, 0, cta_group)
+    try:
+        binding.gemm_trace_enable(16)
+        t0 = time.time()
+        binding.gemm_s8(dA, dB, C)
+        torch.cuda.synchronize()                  # returns: the kernel gave up by itself
+        took = time.time() - t0
+        binding.gemm_trace_enable(0)
+        status = binding.gemm_last_device_status()
+        assert status in (1, 2, 3), "expected a recorded wait expiry, got %d" % status
+        assert 1.5 < took < 30.0
+        assert binding.gemm_last_device_status() == 0        # reading clears it
+        # the context is intact: the same call now gives the right answer
+        binding.gemm_s8(dA, dB, C)
+        torch.cuda.synchronize()
+        assert np.array_equal(C.cpu().numpy(), oracle.gemm_s8(A, B))
+        assert binding.gemm_last_device_status() == 0
+    finally:
+        binding.gemm_trace_enable(0)
+        binding.gemm_set_config_override(0, 0, 0)
