@@ -21,6 +21,14 @@
  * enqueue nothing.  M and N are arbitrary; K carries an alignment rule because
  * operand rows are fetched by TMA (row pitch must be a multiple of 16 bytes).
  *
+ * Split-K.  The study runs squares only and names non-square shapes as future
+ * work (Sec. VI).  When a problem has fewer C tiles than the GPU has SMs (small
+ * M, as in LLM decoding, or small squares) the selector lets several work units
+ * share one tile over disjoint K ranges: C is zeroed on the stream and every
+ * unit ADDS its partial tile (TMA reduction).  INT32 results stay exact; FP32
+ * results then depend on the order the partial sums land, i.e. two runs can
+ * differ in the last bits, always inside the stated bound.
+ *
  * All functions return GEMM_OK (0) or a negative GEMM_ERR_* code.
  * A process may call from several host threads; calls that share a stream are
  * ordered by it.
@@ -208,12 +216,16 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len);
 
 /*
  * Overrides the selector for later calls from this process: tile width BN
- * (0 = automatic), raster band height in tiles (0 = automatic) and the number
+ * (0 = automatic), raster band height in tiles (0 = automatic), the number
  * of CTAs that share one tile (0 = automatic, 1 = 128 x BN tile per CTA, 2 =
- * 256 x BN tile per CTA pair).  For ablation sweeps in the spirit of the
- * paper's Run 4.  Returns GEMM_ERR_INVALID_ARG for a shape that is not built.
+ * 256 x BN tile per CTA pair) and the split-K factor (0 = automatic, 1 = off,
+ * s = every C tile is computed by s work units over disjoint K ranges; capped
+ * at the number of 128-byte K blocks; honoured only by gemm_fp16 / gemm_s8 /
+ * gemm_s4*, whose 32-bit results can be summed in place).  For ablation sweeps
+ * in the spirit of the paper's Run 4.  Returns GEMM_ERR_INVALID_ARG for a shape
+ * that is not built.
  */
-int gemm_set_config_override(int bn, int group_m, int cta_group);
+int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k);
 
 /*
  * Kernels never spin forever: a barrier wait that exceeds its limit makes the

@@ -69,7 +69,7 @@ def lib() -> ctypes.CDLL:
         L.gemm_unpack_s4.argtypes = [i, i, vp, vp, sz, vp]
         L.gemm_mma_peak_probe.argtypes = [i, i, i, i, ctypes.POINTER(ctypes.c_double), vp]
         L.gemm_query_config.argtypes = [i, i, i, i, ctypes.c_char_p, i]
-        L.gemm_set_config_override.argtypes = [i, i, i]
+        L.gemm_set_config_override.argtypes = [i, i, i, i]
         L.gemm_set_l2_policy.argtypes = [i]
         L.gemm_trace_enable.argtypes = [i]
         L.gemm_trace_read.argtypes = [ctypes.POINTER(ctypes.c_ulonglong), i]
@@ -265,8 +265,9 @@ def gemm_query_config(precision: str, M: int, N: int, K: int) -> str:
     return buf.value.decode()
 
 
-def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0):
-    _check(lib().gemm_set_config_override(bn, group_m, cta_group), "gemm_set_config_override")
+def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0, split_k: int = 0):
+    _check(lib().gemm_set_config_override(bn, group_m, cta_group, split_k),
+           "gemm_set_config_override")
 
 
 def gemm_set_l2_policy(policy: int = 11):

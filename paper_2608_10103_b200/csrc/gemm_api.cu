@@ -40,6 +40,7 @@ int g_last_cuda_error = 0;
 int g_override_bn = 0;
 int g_override_group_m = 0;
 int g_override_cta_group = 0;
+int g_override_splits = 0;
 int g_trace_on = 0;
 int g_l2_policy = 11;  // keep A, B normal, serpentine K, C stores evict-first
 
@@ -109,13 +110,13 @@ int encode_operand_map(CUtensorMap* map, CUtensorMapDataType type, int elem_byte
 
 // C (row-major, 32- or 16-bit elements) for the epilogue's TMA stores: boxes of 32 rows x
 // 128 bytes, 128-byte swizzle.  Needs a 16-byte aligned base and pitch.
-int encode_c_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, int elem_bytes) {
+int encode_c_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, int elem_bytes,
+                 CUtensorMapDataType reduce_type = CU_TENSOR_MAP_DATA_TYPE_UINT32) {
   cuuint64_t dims[2] = {cols, rows};
   cuuint64_t strides[1] = {cols * static_cast<uint64_t>(elem_bytes)};
   cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elem_bytes), 32};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(map, elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
-                                             : CU_TENSOR_MAP_DATA_TYPE_UINT16,
+  CUresult r = g_encode(map, elem_bytes == 4 ? reduce_type : CU_TENSOR_MAP_DATA_TYPE_UINT16,
                         2, const_cast<void*>(ptr), dims,
                         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
@@ -133,6 +134,7 @@ struct TileConfig {
   int cta_group;  // 1: one CTA per 128 x bn tile; 2: a CTA pair per 256 x bn tile
   int stages;
   int group_m;
+  int splits;     // split-K factor (1 = off)
 };
 
 constexpr int kWidths[] = {256, 128, 64, 32};
@@ -157,27 +159,58 @@ bool variant_exists(int bn, int cta_group) {
 
 int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b); }
 
-// Picks the C-tile shape.  The paper fixes one tiling for all sizes (Sec.
-// III-A); on 148 SMs small problems need smaller tiles to fill the machine and
-// large ones want the CTA-pair tile, which halves the B bytes each SM pulls
-// from L2.  Cost model: waves of tiles x (tile width + a fixed per-tile
-// overhead), with a discount for the pair shape.
-TileConfig select_config(int M, int N, int num_sms, int min_bn = 32) {
-  TileConfig best{256, 2, 6, 8};
+// Picks the C-tile shape and the split-K factor.  The paper fixes one tiling for all
+// sizes (Sec. III-A) and lists non-square shapes as future work (Sec. VI); on 148 SMs small
+// problems need more work units than they have tiles, and large ones want the CTA-pair
+// tile, which halves the B bytes each SM pulls from L2.
+// Cost model, in SM cycles, fitted to the cycle accounting of the kernel: a k-block (128
+// bytes of K) costs the slowest of the tensor pipe (2*bn: a 128-row MMA of width bn occupies
+// it bn/2 cycles, 4 per k-block), the issuing thread (~450) and the SM's L2 port
+// ((128 + bn/cta_group) rows x 128 bytes at ~66 bytes/cycle); units run in waves over the SMs
+// (or SM pairs); the last epilogue (~16 cycles per column), set-up (~3000) and a pair's
+// cluster launch (~2500) are paid once; split-K adds zeroing C and adding into it.
+TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 32,
+                         bool allow_split = false) {
+  TileConfig best{256, 2, 6, 8, 1};
   long long best_cost = -1;
   for (int cg = 2; cg >= 1; --cg) {
     if (g_override_cta_group && cg != g_override_cta_group) continue;
     for (int bn : kWidths) {
       if (g_override_bn && bn != g_override_bn) continue;
       if (!variant_exists(bn, cg) || bn < min_bn) continue;
-      long long tiles = static_cast<long long>(ceil_div(M, BM * cg)) * ceil_div(N, bn);
-      long long units = num_sms / cg;
-      long long waves = (tiles + units - 1) / units;
-      long long cost = waves * (bn + 160) * (cg == 2 ? 85 : 100);
-      if (best_cost < 0 || cost < best_cost) {
-        best_cost = cost;
-        best.bn = bn;
-        best.cta_group = cg;
+      const long long tiles = static_cast<long long>(ceil_div(M, BM * cg)) * ceil_div(N, bn);
+      const long long units = num_sms / cg;
+      int max_split = 1;
+      if (allow_split) {
+        max_split = static_cast<int>(units / tiles);
+        if (max_split > k_blocks / 2) max_split = k_blocks / 2;  // at least 2 k-blocks each
+        if (max_split > 32) max_split = 32;
+        if (max_split < 1) max_split = 1;
+      }
+      if (g_override_splits) {
+        // forced: the largest factor <= the request that leaves no K range empty
+        max_split = g_override_splits < k_blocks ? g_override_splits : k_blocks;
+        while (max_split > 1 &&
+               static_cast<long long>(max_split - 1) * ceil_div(k_blocks, max_split) >= k_blocks)
+          --max_split;
+        if (!allow_split) max_split = 1;
+      }
+      for (int sp = g_override_splits ? max_split : 1; sp <= max_split; ++sp) {
+        const int per = ceil_div(k_blocks, sp);
+        if (static_cast<long long>(sp - 1) * per >= k_blocks) continue;  // an empty K range
+        const long long waves = (tiles * sp + units - 1) / units;
+        long long per_kb = 2 * bn;
+        if (per_kb < 450) per_kb = 450;
+        const long long port = (128 + bn / cg) * 128 / 66;
+        if (per_kb < port) per_kb = port;
+        long long cost = waves * per * per_kb + 3000 + 16 * bn + (cg == 2 ? 2500 : 0);
+        if (sp > 1) cost += 6000 + static_cast<long long>(M) * N / 250;  // zeroing C + adding into it
+        if (best_cost < 0 || cost < best_cost) {
+          best_cost = cost;
+          best.bn = bn;
+          best.cta_group = cg;
+          best.splits = sp;
+        }
       }
     }
   }
@@ -211,7 +244,7 @@ int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUt
     if (e != cudaSuccess) return cuda_fail(e);
     s->attr_set[variant >> 6] |= 1ull << (variant & 63);
   }
-  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
+  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.splits;
   const long long units = s->num_sms / CTA_GROUP;
   const int grid = static_cast<int>((tiles < units ? tiles : units) * CTA_GROUP);
   cudaLaunchConfig_t cfg = {};
@@ -250,7 +283,9 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   constexpr int C_ELEM = (EPI == EPI_OUT16) ? 2 : 4;
   const CUtensorMapDataType type =
       (KIND == ptx::KIND_F16) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
-  const TileConfig cfg = select_config(M, N, s->num_sms, EPI == EPI_OUT16 ? 64 : 32);
+  const int k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
+  const TileConfig cfg = select_config(M, N, s->num_sms, k_blocks, EPI == EPI_OUT16 ? 64 : 32,
+                                       EPI == EPI_RAW32);
   if (cfg.bn == 0) return GEMM_ERR_INVALID_ARG;  // override asks for a shape this mode lacks
 
   CUtensorMap ta, tb;
@@ -267,11 +302,16 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.tiles_m = ceil_div(M, BM * cfg.cta_group);
   p.tiles_n = ceil_div(N, cfg.bn);
   p.group_m = cfg.group_m;
-  p.k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
+  p.k_blocks = k_blocks;
+  p.splits = cfg.splits;
   p.c_vec_ok = (N % (16 / C_ELEM) == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
   CUtensorMap tc;
   if (p.c_vec_ok) {
-    rc = encode_c_map(&tc, C, M, N, C_ELEM);
+    // split-K adds into C by TMA reduction, which takes the element type from the map
+    rc = encode_c_map(&tc, C, M, N, C_ELEM,
+                      cfg.splits == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
+                      : KIND == ptx::KIND_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                              : CU_TENSOR_MAP_DATA_TYPE_INT32);
     if (rc != GEMM_OK) return rc;
   } else {
     tc = ta;  // unused by the kernel on the plain-store path
@@ -286,6 +326,10 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.serpentine_k = (g_l2_policy & 4) ? 0 : 1;
   p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
 
+  if (cfg.splits > 1) {
+    cudaError_t e = cudaMemsetAsync(C, 0, static_cast<size_t>(M) * N * C_ELEM, stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
   const int vbase = ((KIND == ptx::KIND_F16) ? 0 : 32) + EPI * 8;  // bit index in attr_set
   if (cfg.cta_group == 2) {
     switch (cfg.bn) {
@@ -582,22 +626,27 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
     if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < MAX_DEVICES && g_dev[dev].ready)
       num_sms = g_dev[dev].num_sms;
   }
-  const TileConfig c = select_config(M, N, num_sms);
   const int elem = precision == GEMM_PREC_FP16 ? 2 : 1;
+  const TileConfig c =
+      select_config(M, N, num_sms, ceil_div(static_cast<long long>(K) * elem, BK_BYTES), 32, true);
+  if (c.bn == 0) return GEMM_ERR_INVALID_ARG;
   const long long tiles =
       static_cast<long long>(ceil_div(M, BM * c.cta_group)) * ceil_div(N, c.bn);
   const long long units = num_sms / c.cta_group;
   snprintf(buf, static_cast<size_t>(len),
-           "BM=%d BN=%d BK=%d cta_group=%d stages=%d group_m=%d tiles=%lld ctas=%lld kind=%s%s",
-           BM * c.cta_group, c.bn, atoms_for(c.bn, c.cta_group) * BK_BYTES / elem, c.cta_group, c.stages, c.group_m, tiles,
-           (tiles < units ? tiles : units) * c.cta_group,
+           "BM=%d BN=%d BK=%d cta_group=%d stages=%d group_m=%d split_k=%d tiles=%lld ctas=%lld "
+           "kind=%s%s",
+           BM * c.cta_group, c.bn, atoms_for(c.bn, c.cta_group) * BK_BYTES / elem, c.cta_group,
+           c.stages, c.group_m, c.splits, tiles,
+           (tiles * c.splits < units ? tiles * c.splits : units) * c.cta_group,
            precision == GEMM_PREC_FP16 ? "f16" : "i8",
            precision == GEMM_PREC_S4 ? " prepass=unpack_s4" : "");
   return GEMM_OK;
 }
 
-int gemm_set_config_override(int bn, int group_m, int cta_group) {
-  if (group_m < 0 || cta_group < 0 || cta_group > 2) return GEMM_ERR_INVALID_ARG;
+int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k) {
+  if (group_m < 0 || cta_group < 0 || cta_group > 2 || split_k < 0 || split_k > 64)
+    return GEMM_ERR_INVALID_ARG;
   bool ok = false;
   for (int cg = 1; cg <= 2; ++cg) {
     if (cta_group && cg != cta_group) continue;
@@ -611,6 +660,7 @@ int gemm_set_config_override(int bn, int group_m, int cta_group) {
   g_override_bn = bn;
   g_override_group_m = group_m;
   g_override_cta_group = cta_group;
+  g_override_splits = split_k;
   return GEMM_OK;
 }
 

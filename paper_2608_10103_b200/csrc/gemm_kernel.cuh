@@ -71,6 +71,8 @@ struct GemmParams {
   int tiles_m, tiles_n;  // number of C tiles (128*CTA_GROUP x BN) along M and N
   int group_m;           // raster: tiles are walked in bands of `group_m` tile rows
   int k_blocks;          // ceil(K bytes / BK_BYTES): 128-byte K atoms to cover K
+  int splits;            // split-K: each C tile is computed by `splits` work units over disjoint
+                         // K ranges and ADDED into a zeroed C (EPI_RAW32 only); 1 = off
   int c_vec_ok;          // 1 if C rows allow 16-byte accesses (N % 4 == 0, base 16-byte aligned):
                          // the epilogue then stages C in shared memory and stores it by TMA
   uint32_t* C;           // element size 4 bytes, or 2 with EPI_OUT16
@@ -218,8 +220,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   const int lane = threadIdx.x & 31;
   const uint32_t cta_rank = (CTA_GROUP == 2) ? ptx::cluster_ctarank() : 0u;
   const bool leader = (cta_rank == 0);
-  const int num_tiles = p.tiles_m * p.tiles_n;
-  const int k_slots = (p.k_blocks + KB - 1) / KB;  // ring slots per tile; a K tail is zero-filled
+  // Work units: unit u = (tile u % tiles, K range u / tiles).  `num_tiles` counts units.
+  const int real_tiles = p.tiles_m * p.tiles_n;
+  const int num_tiles = real_tiles * p.splits;
+  const int k_slots_all = (p.k_blocks + KB - 1) / KB;  // ring slots per tile; a K tail is zero-filled
+  const int k_per_split = (k_slots_all + p.splits - 1) / p.splits;
   const int first_tile = static_cast<int>(blockIdx.x) / CTA_GROUP;
   const int tile_stride = static_cast<int>(gridDim.x) / CTA_GROUP;
   unsigned long long* const trace =
@@ -277,10 +282,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       bool backward = false;
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
         int tm, tn;
-        tile_coords(p, t, tm, tn);
+        tile_coords(p, t % real_tiles, tm, tn);
+        const int k_begin = (t / real_tiles) * k_per_split;
+        const int k_end = min(k_begin + k_per_split, k_slots_all);
         const int a_row = tm * TILE_M + static_cast<int>(cta_rank) * BM;
         const int b_row = tn * BN + static_cast<int>(cta_rank) * L::B_ROWS;
-        for (int ks = 0; ks < k_slots; ++ks) {
+        for (int ks = k_begin; ks < k_end; ++ks) {
           const long long w0 = trace ? clock64() : 0;
           ok = wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status,
                             DEV_TIMEOUT_PRODUCER);
@@ -291,7 +298,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const uint32_t b_dst = a_dst + KB * L::A_BYTES;
           if (!elected) {
             // nothing to issue in this lane
-          } else if ((p.ablate & 8) && blockIdx.x == 0 && t == first_tile && ks == 2) {
+          } else if ((p.ablate & 8) && blockIdx.x == 0 && t == first_tile && ks == k_begin + 2) {
             // failure drill: this slot is never filled
           } else if (p.ablate & 2) {
             if (leader) ptx::mbar_arrive(full_bar(stage));
@@ -299,7 +306,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             ptx::mbar_arrive_expect_tx(full_bar(stage), L::STAGE_BYTES);
 #pragma unroll
             for (int a = 0; a < KB; ++a) {
-              const int k0 = ((backward ? k_slots - 1 - ks : ks) * KB + a) * BK_ELEMS;
+              const int k0 = ((backward ? k_begin + k_end - 1 - ks : ks) * KB + a) * BK_ELEMS;
               ptx::tma_load_2d(a_dst + a * L::A_BYTES, &tmap_a, k0, a_row, full_bar(stage), pol_a);
               ptx::tma_load_2d(b_dst + a * L::B_BYTES, &tmap_b, k0, b_row, full_bar(stage), pol_b);
             }
@@ -309,7 +316,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             const uint32_t lead_full = ptx::map_to_cta(full_bar(stage), 0);
 #pragma unroll
             for (int a = 0; a < KB; ++a) {
-              const int k0 = ((backward ? k_slots - 1 - ks : ks) * KB + a) * BK_ELEMS;
+              const int k0 = ((backward ? k_begin + k_end - 1 - ks : ks) * KB + a) * BK_ELEMS;
               ptx::tma_load_2d_pair(a_dst + a * L::A_BYTES, &tmap_a, k0, a_row, lead_full, pol_a);
               ptx::tma_load_2d_pair(b_dst + a * L::B_BYTES, &tmap_b, k0, b_row, lead_full, pol_b);
             }
@@ -356,7 +363,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         if (!ok) break;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
-        for (int ks = 0; ks < k_slots; ++ks) {
+        const int k_begin = (t / real_tiles) * k_per_split;
+        const int k_end = min(k_begin + k_per_split, k_slots_all);
+        for (int ks = k_begin; ks < k_end; ++ks) {
           const long long w1 = trace ? clock64() : 0;
           ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
           const long long w2 = trace ? clock64() : 0;
@@ -377,7 +386,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                 const uint64_t b_step =
                     static_cast<uint64_t>((a * L::B_BYTES + kk * MMA_K_BYTES) >> 4);
                 ptx::mma_ss<KIND, CTA_GROUP>(d_tmem, a_desc + a_step, b_desc + b_step, idesc,
-                                             (ks > 0 || a > 0 || kk > 0) ? 1u : 0u);
+                                             (ks > k_begin || a > 0 || kk > 0) ? 1u : 0u);
               }
             }
           }
@@ -433,7 +442,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     long long epi_wait = 0, epi_busy = 0, tiles_done = 0;
     for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
       int tm, tn;
-      tile_coords(p, t, tm, tn);
+      tile_coords(p, t % real_tiles, tm, tn);
       const long long w0 = trace ? clock64() : 0;
       ok = wait_bounded<true>(acc_full_bar(acc), acc_phase, abort_flag, p.status,
                               DEV_TIMEOUT_EPILOGUE, (p.ablate & 4) ? 500u : 0u);
@@ -508,7 +517,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           // close a (then empty) group so that "one group per block" keeps the buffer
           // reuse rule above exact.
           if (lane == 0) {
-            if (row0 < p.M && col < p.N) ptx::tma_store_2d(&tmap_c, col, row0, buf, pol_c);
+            if (row0 < p.M && col < p.N) {
+              if (EPI == EPI_RAW32 && p.splits > 1)
+                ptx::tma_reduce_add_2d(&tmap_c, col, row0, buf);
+              else
+                ptx::tma_store_2d(&tmap_c, col, row0, buf, pol_c);
+            }
             ptx::bulk_commit_group();
           }
         } else if (row < p.M) {
@@ -521,9 +535,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                 crow[col + v] = static_cast<uint16_t>(w[v / 2] >> (16 * (v & 1)));
           } else {
             uint32_t* crow = p.C + static_cast<size_t>(row) * p.N;
+            if (EPI == EPI_RAW32 && p.splits > 1) {
 #pragma unroll
-            for (int v = 0; v < 32; ++v)
-              if (col + v < p.N) crow[col + v] = w[v];
+              for (int v = 0; v < 32; ++v) {
+                if (col + v >= p.N) continue;
+                if constexpr (KIND == ptx::KIND_F16)
+                  atomicAdd(reinterpret_cast<float*>(crow + col + v), __uint_as_float(w[v]));
+                else
+                  atomicAdd(reinterpret_cast<int*>(crow + col + v), static_cast<int>(w[v]));
+              }
+            } else {
+#pragma unroll
+              for (int v = 0; v < 32; ++v)
+                if (col + v < p.N) crow[col + v] = w[v];
+            }
           }
         }
       }

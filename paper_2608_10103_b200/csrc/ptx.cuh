@@ -171,6 +171,17 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, int c0, int c
       : "memory");
 }
 
+// 2-D tiled reduction shared -> global: every element of the box is ADDED to the tensor
+// element (type taken from the tensor map: FP32 or INT32 here), atomically per element.
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* m, int c0, int c1,
+                                                  uint32_t src) {
+  asm volatile(
+      "cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];" ::
+          "l"(reinterpret_cast<uint64_t>(m)),
+      "r"(c0), "r"(c1), "r"(src)
+      : "memory");
+}
+
 __device__ __forceinline__ void bulk_commit_group() {
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }

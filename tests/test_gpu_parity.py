@@ -263,3 +263,39 @@ def test_argument_errors_enqueue_nothing():
     torch.cuda.synchronize()
     assert int((C != 5).sum()) == 0
     assert L.gemm_status_string(-3).decode().startswith("K too large")
+
+
+# ----------------------------------------------------------------------- split-K
+@pytest.mark.parametrize("splits", [2, 3, 5, 8])
+@pytest.mark.parametrize("prec", synth.PRECISIONS)
+def test_split_k_forced(prec, splits):
+    M, N, K = 300, 520, 2080                      # 65 resp. 33 k-blocks: uneven K ranges
+    A, B = synth.make(prec, M, N, K, seed=splits)
+    ref, S = oracle_block(prec, A, B)
+    for bn, cta_group in [(256, 2), (256, 1), (64, 1)]:
+        binding.gemm_set_config_override(bn, 0, cta_group, splits)
+        cfg = binding.gemm_query_config(prec, M, N, K)
+        got = int(cfg.split("split_k=")[1].split()[0])
+        assert 2 <= got <= splits, cfg            # capped so that no K range is empty
+        C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
+        assert_block(prec, C, ref, S, "bn=%d cta_group=%d" % (bn, cta_group))
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 4096, 4096), (16, 8192, 8192), (64, 4096, 16384),
+                                   (128, 1030, 4128), (40, 70, 8192), (8, 33, 1024)])
+def test_small_m_shapes_pick_split_k(M, N, K):
+    """Decode-like shapes: few C tiles, long K.  The selector splits K on its own; rows of C
+    that are not 16-byte multiples take the atomic-add path."""
+    for prec in synth.PRECISIONS:
+        A, B = synth.make(prec, M, N, K, seed=M + N)
+        if K >= 4096:
+            assert "split_k=1 " not in binding.gemm_query_config(prec, M, N, K)
+        C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
+        check_against_oracle(prec, A, B, C, force_full=True)
+
+
+def test_split_k_more_ranges_than_blocks_is_capped():
+    A, B = synth.s8_uniform(130, 260, 256, seed=1)      # 2 k-blocks
+    binding.gemm_set_config_override(0, 0, 0, 8)
+    assert "split_k=2 " in binding.gemm_query_config("s8", 130, 260, 256)
+    check_against_oracle("s8", A, B, run_gpu("s8", A, B, fill=-7), force_full=True)

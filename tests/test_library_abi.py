@@ -57,10 +57,11 @@ def test_argument_validation_needs_no_gpu(lib):
     assert lib.gemm_unpack_s4(4, 48, 16, 16, 48, None) == -2
     assert lib.gemm_mma_peak_probe(2, 10, 256, 0, ctypes.pointer(ctypes.c_double(0)), None) == -1
     assert lib.gemm_mma_peak_probe(0, 10, 24, 0, ctypes.pointer(ctypes.c_double(0)), None) == -1
-    assert lib.gemm_set_config_override(48, 0, 0) == -1
-    assert lib.gemm_set_config_override(32, 0, 2) == -1          # no 32-wide pair tile
-    assert lib.gemm_set_config_override(0, 0, 3) == -1
-    assert lib.gemm_set_config_override(0, 0, 0) == 0
+    assert lib.gemm_set_config_override(48, 0, 0, 0) == -1
+    assert lib.gemm_set_config_override(32, 0, 2, 0) == -1          # no 32-wide pair tile
+    assert lib.gemm_set_config_override(0, 0, 3, 0) == -1
+    assert lib.gemm_set_config_override(0, 0, 0, 0) == 0
+    assert lib.gemm_set_config_override(0, 0, 0, 65) == -1
 
 
 def test_workspace_size(lib):
