@@ -141,15 +141,17 @@ constexpr int kWidths[] = {256, 128, 64, 32};
 
 // Ring depth and 128-byte K atoms per slot of each built shape.
 int stages_for(int bn, int cta_group) {
-  if (cta_group == 2) return bn == 256 ? 6 : 8;
+  if (cta_group == 2) return bn == 256 ? 6 : 4;
   switch (bn) {
     case 256: return 4;
-    case 128: return 6;
-    default: return 8;
+    case 128: return 3;
+    default: return 4;
   }
 }
 
-int atoms_for(int, int) { return 1; }
+// 256-wide tiles are bound by the tensor pipe and want many small slots; narrower tiles are
+// bound by the issuing thread and get two K atoms per slot (one wait + one commit per 8 MMAs).
+int atoms_for(int bn, int) { return bn == 256 ? 1 : 2; }
 
 bool variant_exists(int bn, int cta_group) {
   if (cta_group == 1) return bn == 256 || bn == 128 || bn == 64 || bn == 32;
@@ -180,6 +182,8 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
       if (!variant_exists(bn, cg) || bn < min_bn) continue;
       const long long tiles = static_cast<long long>(ceil_div(M, BM * cg)) * ceil_div(N, bn);
       const long long units = num_sms / cg;
+      const int atoms = atoms_for(bn, cg);
+      const int slots = ceil_div(k_blocks, atoms);  // K is split in whole ring slots
       int max_split = 1;
       if (allow_split) {
         max_split = static_cast<int>(units / tiles);
@@ -189,15 +193,16 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
       }
       if (g_override_splits) {
         // forced: the largest factor <= the request that leaves no K range empty
-        max_split = g_override_splits < k_blocks ? g_override_splits : k_blocks;
+        max_split = g_override_splits < slots ? g_override_splits : slots;
         while (max_split > 1 &&
-               static_cast<long long>(max_split - 1) * ceil_div(k_blocks, max_split) >= k_blocks)
+               static_cast<long long>(max_split - 1) * ceil_div(slots, max_split) >= slots)
           --max_split;
         if (!allow_split) max_split = 1;
       }
+      if (max_split > slots) max_split = slots;
       for (int sp = g_override_splits ? max_split : 1; sp <= max_split; ++sp) {
-        const int per = ceil_div(k_blocks, sp);
-        if (static_cast<long long>(sp - 1) * per >= k_blocks) continue;  // an empty K range
+        if (static_cast<long long>(sp - 1) * ceil_div(slots, sp) >= slots) continue;  // empty range
+        const int per = ceil_div(slots, sp) * atoms;  // k-blocks per unit
         const long long waves = (tiles * sp + units - 1) / units;
         long long per_kb = 2 * bn;
         if (per_kb < 450) per_kb = 450;
@@ -334,18 +339,18 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   if (cfg.cta_group == 2) {
     switch (cfg.bn) {
       case 256: return launch_variant<KIND, 256, 6, 2, 1, EPI>(s, vbase + 4, ta, tb, tc, p, stream);
-      case 128: return launch_variant<KIND, 128, 8, 2, 1, EPI>(s, vbase + 5, ta, tb, tc, p, stream);
-      case 64: return launch_variant<KIND, 64, 8, 2, 1, EPI>(s, vbase + 6, ta, tb, tc, p, stream);
+      case 128: return launch_variant<KIND, 128, 4, 2, 2, EPI>(s, vbase + 5, ta, tb, tc, p, stream);
+      case 64: return launch_variant<KIND, 64, 4, 2, 2, EPI>(s, vbase + 6, ta, tb, tc, p, stream);
       default: return GEMM_ERR_INVALID_ARG;
     }
   }
   switch (cfg.bn) {
     case 256: return launch_variant<KIND, 256, 4, 1, 1, EPI>(s, vbase + 0, ta, tb, tc, p, stream);
-    case 128: return launch_variant<KIND, 128, 6, 1, 1, EPI>(s, vbase + 1, ta, tb, tc, p, stream);
-    case 64: return launch_variant<KIND, 64, 8, 1, 1, EPI>(s, vbase + 2, ta, tb, tc, p, stream);
+    case 128: return launch_variant<KIND, 128, 3, 1, 2, EPI>(s, vbase + 1, ta, tb, tc, p, stream);
+    case 64: return launch_variant<KIND, 64, 4, 1, 2, EPI>(s, vbase + 2, ta, tb, tc, p, stream);
     case 32:
       if constexpr (EPI != EPI_OUT16)
-        return launch_variant<KIND, 32, 8, 1, 1, EPI>(s, vbase + 3, ta, tb, tc, p, stream);
+        return launch_variant<KIND, 32, 4, 1, 2, EPI>(s, vbase + 3, ta, tb, tc, p, stream);
       return GEMM_ERR_INVALID_ARG;
     default: return GEMM_ERR_INVALID_ARG;
   }

@@ -451,6 +451,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       epi_wait += w1 - w0;
       if (!ok) break;
       ptx::tc_fence_after_sync();
+      // A split-K unit whose K range is empty (the host never creates one) contributes nothing.
+      const bool empty_range = (t / real_tiles) * k_per_split >= k_slots_all;
       const int row0 = tm * TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
       const int row = row0 + lane;
       const int col0 = tn * BN;
@@ -517,7 +519,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           // close a (then empty) group so that "one group per block" keeps the buffer
           // reuse rule above exact.
           if (lane == 0) {
-            if (row0 < p.M && col < p.N) {
+            if (row0 < p.M && col < p.N && !empty_range) {
               if (EPI == EPI_RAW32 && p.splits > 1)
                 ptx::tma_reduce_add_2d(&tmap_c, col, row0, buf);
               else
@@ -525,7 +527,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             }
             ptx::bulk_commit_group();
           }
-        } else if (row < p.M) {
+        } else if (row < p.M && !empty_range) {
           // C rows are not 16-byte multiples: plain predicated stores.
           if constexpr (EPI == EPI_OUT16) {
             uint16_t* crow = reinterpret_cast<uint16_t*>(p.C) + static_cast<size_t>(row) * p.N;

@@ -296,6 +296,8 @@ def test_small_m_shapes_pick_split_k(M, N, K):
 
 def test_split_k_more_ranges_than_blocks_is_capped():
     A, B = synth.s8_uniform(130, 260, 256, seed=1)      # 2 k-blocks
-    binding.gemm_set_config_override(0, 0, 0, 8)
-    assert "split_k=2 " in binding.gemm_query_config("s8", 130, 260, 256)
-    check_against_oracle("s8", A, B, run_gpu("s8", A, B, fill=-7), force_full=True)
+    for bn in (0, 256, 64):
+        binding.gemm_set_config_override(bn, 0, 0, 8)
+        cfg = binding.gemm_query_config("s8", 130, 260, 256)
+        assert int(cfg.split("split_k=")[1].split()[0]) <= 2, cfg     # never more ranges than slots
+        check_against_oracle("s8", A, B, run_gpu("s8", A, B, fill=-7), force_full=True)
