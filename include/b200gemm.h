@@ -139,6 +139,32 @@ int gemm_s4_dequant(int M, int N, int K, const uint8_t* A, const uint8_t* B,
                     gemm_stream_t stream);
 
 /*
+ * The same GEMM for operands and result in HOST memory (the end-to-end path:
+ * the study times kernels only, Sec. III-B; a caller whose data lives on the
+ * host also pays the PCIe transfers).  A, B, C are HOST pointers with the
+ * layouts above (A: M x K, B: N x K, C: M x N 32-bit; for GEMM_PREC_S4 A and B
+ * are packed, K/2 bytes per row).  precision = GEMM_PREC_FP16 / _S8 / _S4.
+ *
+ * The call cuts A and B into blocks of 2048 rows, sends them to the device in an
+ * order that lets C blocks start early, multiplies each C block on `stream` as
+ * soon as its two operand blocks have arrived and sends finished C blocks back
+ * while later ones are still being multiplied, using two internal copy streams.
+ * Everything is enqueued asynchronously: C is complete when `stream` has passed
+ * the call.  Use page-locked (pinned) host memory; with pageable memory the
+ * copies are staged by the driver, block the calling thread and run slower.
+ * The library keeps grow-only device copies of A, B and C per device
+ * (cudaMalloc on first use / growth, which synchronises the device);
+ * gemm_host_release frees them.  Calls through this entry point on one device
+ * share those buffers and must be ordered by the caller (same stream, or
+ * events).  K rules as for the device entry points; at most 64 x 64 blocks.
+ */
+int gemm_host(int precision, int M, int N, int K, const void* A, const void* B, void* C,
+              gemm_stream_t stream);
+
+/* Frees the device buffers, streams and events behind gemm_host (synchronises). */
+int gemm_host_release(void);
+
+/*
  * gemm_s4 for callers that cannot allocate device memory.  (The paper has no
  * counterpart: its INT4 kernels need no scratch.)
  *

@@ -21,7 +21,7 @@ PRECISION_ID = {"fp16": PREC_FP16, "s8": PREC_S8, "s4": PREC_S4}
 
 EXPORTS = (
     "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
-    "gemm_fp16_f16out", "gemm_s8_dequant", "gemm_s4_dequant",
+    "gemm_fp16_f16out", "gemm_s8_dequant", "gemm_s4_dequant", "gemm_host", "gemm_host_release",
     "gemm_s4_static", "gemm_s4_static_capacity", "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
     "gemm_set_config_override", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_last_device_status", "gemm_last_cuda_error",
     "gemm_status_string", "gemm_version",
@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.gemm_s4.argtypes = [i, i, i, vp, vp, vp, vp]
         L.gemm_s4_ws.argtypes = [i, i, i, vp, vp, vp, vp, sz, vp]
         L.gemm_fp16_f16out.argtypes = [i, i, i, vp, vp, vp, vp]
+        L.gemm_host.argtypes = [i, i, i, i, vp, vp, vp, vp]
         L.gemm_s8_dequant.argtypes = [i, i, i, vp, vp, vp, vp, vp, i, vp]
         L.gemm_s4_dequant.argtypes = [i, i, i, vp, vp, vp, vp, vp, i, vp]
         L.gemm_s4_workspace_bytes.argtypes = [i, i, i]
@@ -148,6 +149,35 @@ def gemm_s4(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor | None = None, str
     _check(lib().gemm_s4(M, N, 2 * Kh, _dev_ptr(A, torch.uint8, "A"), _dev_ptr(B, torch.uint8, "B"),
                          _dev_ptr(C, torch.int32, "C"), _stream_handle(stream)), "gemm_s4")
     return C
+
+
+_HOST_DTYPES = {"fp16": (torch.float16, torch.float32), "s8": (torch.int8, torch.int32),
+                "s4": (torch.uint8, torch.int32)}
+
+
+def gemm_host(precision: str, A: torch.Tensor, B: torch.Tensor, C: torch.Tensor | None = None,
+              stream=None):
+    """C = A @ B^T for HOST tensors (pinned memory recommended).  Returns C (host); it is
+    complete once `stream` (default: the current stream) has been synchronised."""
+    in_dtype, out_dtype = _HOST_DTYPES[precision]
+    for t, what in ((A, "A"), (B, "B")):
+        if not isinstance(t, torch.Tensor) or t.is_cuda or t.dtype != in_dtype or not t.is_contiguous():
+            raise TypeError("%s must be a contiguous CPU tensor of dtype %s" % (what, in_dtype))
+    M, N = A.shape[0], B.shape[0]
+    if A.shape[1] != B.shape[1]:
+        raise ValueError("A and B disagree on K")
+    K = A.shape[1] * (2 if precision == "s4" else 1)
+    if C is None:
+        C = torch.empty((M, N), dtype=out_dtype, pin_memory=True)
+    elif C.is_cuda or C.dtype != out_dtype or tuple(C.shape) != (M, N) or not C.is_contiguous():
+        raise TypeError("C must be a contiguous CPU tensor (%d, %d) of dtype %s" % (M, N, out_dtype))
+    _check(lib().gemm_host(PRECISION_ID[precision], M, N, K, A.data_ptr(), B.data_ptr(),
+                           C.data_ptr(), _stream_handle(stream)), "gemm_host")
+    return C
+
+
+def gemm_host_release():
+    _check(lib().gemm_host_release(), "gemm_host_release")
 
 
 def gemm_fp16_f16out(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor | None = None, stream=None):

@@ -76,6 +76,7 @@ struct GemmParams {
   int c_vec_ok;          // 1 if C rows allow 16-byte accesses (N % 4 == 0, base 16-byte aligned):
                          // the epilogue then stages C in shared memory and stores it by TMA
   uint32_t* C;           // element size 4 bytes, or 2 with EPI_OUT16
+  long long ldc;         // row pitch of C in elements (N for a dense C)
   const float* row_scale;  // EPI_OUT16 (integer kinds) / EPI_F32_SCALED: M per-row factors
   const float* col_scale;  // and N per-column factors; both null = no scaling (FP16 kind)
   int* status;           // device status word (0 = ok)
@@ -530,13 +531,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         } else if (row < p.M && !empty_range) {
           // C rows are not 16-byte multiples: plain predicated stores.
           if constexpr (EPI == EPI_OUT16) {
-            uint16_t* crow = reinterpret_cast<uint16_t*>(p.C) + static_cast<size_t>(row) * p.N;
+            uint16_t* crow = reinterpret_cast<uint16_t*>(p.C) + static_cast<size_t>(row) * p.ldc;
 #pragma unroll
             for (int v = 0; v < 64; ++v)
               if (col + v < p.N)
                 crow[col + v] = static_cast<uint16_t>(w[v / 2] >> (16 * (v & 1)));
           } else {
-            uint32_t* crow = p.C + static_cast<size_t>(row) * p.N;
+            uint32_t* crow = p.C + static_cast<size_t>(row) * p.ldc;
             if (EPI == EPI_RAW32 && p.splits > 1) {
 #pragma unroll
               for (int v = 0; v < 32; ++v) {
