@@ -294,19 +294,41 @@ def run_ours(args, rank, world):
     total_ms = times[0]
     worst = dict(zip(precs, times[1:]))
 
-    # ---- MMA-issue-only peak of this machine, per kind (same run, same clocks regime)
-    mma_peak = {}
+    # ---- cycle-based view (independent of the power-capped clock): one traced launch per
+    #      precision gives the SM cycles it took and the SM clock it ran at
+    cycles = {}
+    flop_per_clk = {"fp16": 8192, "s8": 16384, "s4": 16384}   # per SM, dense, from the probe below
+    binding.gemm_trace_enable(1)
+    for p in precs:
+        binding.gemm(p, dev[p][0], dev[p][1], out[p], stream)
+        tr = binding.gemm_trace_read(148)
+        cyc = max(t["cycles"] for t in tr)
+        mhz = statistics.median(t["cycles"] / t["nanos"] * 1e3 for t in tr if t["nanos"])
+        cycles[p] = {"sm_cycles": cyc, "sm_mhz_during_kernel": mhz,
+                     "pipe_utilisation": ops / (148 * flop_per_clk[p]) / cyc}
+    binding.gemm_trace_enable(0)
+
+    # ---- MMA-issue-only peak of this machine, per kind (same run, same power regime): rate by
+    #      CUDA events, cycles per 128x256x(32 B) MMA and clock by the probe's own counters
+    mma_peak, mma_detail = {}, {}
     for kind in (() if args.no_peak_probe else ("fp16", "s8")):
         binding.gemm_mma_peak_probe(kind, 2048)
         torch.cuda.synchronize()
+        binding.gemm_trace_enable(1)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         pops = binding.gemm_mma_peak_probe(kind, 200000)
         e1.record(stream)
         torch.cuda.synchronize()
+        tr = binding.gemm_trace_read(148)
+        binding.gemm_trace_enable(0)
         mma_peak[kind] = pops / (e0.elapsed_time(e1) * 1e-3) / 1e12
+        mma_detail[kind] = {
+            "cycles_per_mma": statistics.mean(t["cycles"] for t in tr) / 200000,
+            "sm_mhz_during_probe": statistics.median(t["cycles"] / t["nanos"] * 1e3 for t in tr)}
     if mma_peak:
         mma_peak["s4"] = mma_peak["s8"]
+        mma_detail["s4"] = mma_detail["s8"]
 
     # ---- end to end: FP16 GEMM through the host-buffer entry point (pinned A, B, C):
     #      H2D of the operands, the kernels and D2H of C are all inside the timed region
@@ -349,7 +371,9 @@ def run_ours(args, rank, world):
             "value": rate, "unit": UNIT[p], "ms": worst[p], "best_ms_rank0": best_ms[p],
             "frac_of_spec_peak": rate / world / SPEC_PEAK[p], "spec_peak": SPEC_PEAK[p],
             "frac_of_mma_only_peak": rate / world / mma_peak[p] if mma_peak else None,
-            "mma_only_peak": mma_peak.get(p),
+            "mma_only_peak": mma_peak.get(p), "mma_only_probe": mma_detail.get(p),
+            "sm_cycles": cycles[p]["sm_cycles"], "pipe_utilisation": cycles[p]["pipe_utilisation"],
+            "sm_mhz_during_kernel": cycles[p]["sm_mhz_during_kernel"],
             "config": binding.gemm_query_config(p, N, N, N),
         }
     if "s4" in worst and "s8" in worst:
