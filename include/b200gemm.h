@@ -286,8 +286,9 @@ int gemm_set_l2_policy(int policy);
  * cycles the producer waited for a free slot [2], the MMA issuer waited for
  * operands [3] and for a free accumulator [4], one epilogue warp waited for a
  * finished accumulator [5] and spent draining [6], the tile count [7], and the
- * issuer's cycles inside tcgen05.mma [8], tcgen05.commit [9] and fence +
- * descriptor set-up [10], and the producer's cycles issuing loads [11].
+ * issuer's cycles inside tcgen05.mma [8] and tcgen05.commit [9], the cycles
+ * the CTA spent setting up barriers and tensor memory [10], and the producer's
+ * cycles issuing loads [11].
  * gemm_trace_read synchronises the device, copies the words of the first
  * min(max_ctas, 160) CTAs of the last traced launch to `out` (host memory,
  * 12 * max_ctas words) and returns that CTA count.  Off by default; the cost

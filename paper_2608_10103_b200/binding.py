@@ -308,7 +308,7 @@ def gemm_set_l2_policy(policy: int = 11):
 
 
 TRACE_FIELDS = ("cycles", "nanos", "producer_wait", "mma_wait_operands", "mma_wait_accumulator",
-                "epilogue_wait", "epilogue_busy", "tiles", "mma_issue", "mma_commit", "mma_fence",
+                "epilogue_wait", "epilogue_busy", "tiles", "mma_issue", "mma_commit", "setup",
                 "producer_issue")
 TRACE_SLOTS = len(TRACE_FIELDS)
 

@@ -109,7 +109,7 @@ enum TraceSlot {
   TRACE_TILES = 7,          // tiles this CTA worked on
   TRACE_MMA_ISSUE = 8,      // MMA issuer: cycles inside the tcgen05.mma issue instructions
   TRACE_MMA_COMMIT = 9,     // MMA issuer: cycles inside tcgen05.commit
-  TRACE_MMA_FENCE = 10,     // MMA issuer: cycles in the fence + descriptor set-up
+  TRACE_SETUP = 10,         // cycles from kernel start until barriers and TMEM are set up
   TRACE_PROD_ISSUE = 11,    // producer: cycles issuing expect_tx + TMA loads
   TRACE_SLOTS = 12
 };
@@ -262,6 +262,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   }
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
+  if (trace && threadIdx.x == 0)
+    trace[TRACE_SETUP] = static_cast<unsigned long long>(clock64() - clk_start);
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -355,7 +357,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      long long wait_full = 0, wait_acc = 0, t_fence = 0, t_issue = 0, t_commit = 0;
+      long long wait_full = 0, wait_acc = 0, t_issue = 0, t_commit = 0;
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
         const long long w0 = trace ? clock64() : 0;
         ok = wait_bounded(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, p.status,
@@ -419,7 +421,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         trace[TRACE_MMA_WAIT_ACC] = static_cast<unsigned long long>(wait_acc);
         trace[TRACE_MMA_ISSUE] = static_cast<unsigned long long>(t_issue);
         trace[TRACE_MMA_COMMIT] = static_cast<unsigned long long>(t_commit);
-        trace[TRACE_MMA_FENCE] = static_cast<unsigned long long>(t_fence);
       }
       if (!ok && elected) {
         // Gave up: wait for the MMAs already issued before TMEM is released.
@@ -570,8 +571,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
-    // C stores still in flight read this CTA's shared memory: wait before leaving.
-    if (lane == 0) ptx::bulk_wait_group<0>();
+    // C stores still in flight read this CTA's shared memory: wait until they have read it
+    // (their global writes complete on their own before the grid counts as finished).
+    if (lane == 0) ptx::bulk_wait_group_read<0>();
     __syncwarp();
     if (trace && warp == 2 && lane == 0) {
       trace[TRACE_EPI_WAIT] = static_cast<unsigned long long>(epi_wait);
