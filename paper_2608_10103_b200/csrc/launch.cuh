@@ -1,0 +1,246 @@
+// Launch plumbing: one kernel variant per (kind, tile shape, output mode), argument checks
+// shared by the entry points, the INT4 pre-pass and its workspaces.
+#pragma once
+
+#include "runtime.cuh"
+#include "selector.cuh"
+#include "unpack_s4.cuh"
+
+namespace b200gemm {
+namespace {
+
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI>
+int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUtensorMap& tb,
+                   const CUtensorMap& tc, const GemmParams& p, cudaStream_t stream) {
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB>;
+  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI>;
+  if (!(s->attr_set[variant >> 6] & (1ull << (variant & 63)))) {
+    cudaError_t e =
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
+    if (e != cudaSuccess) return cuda_fail(e);
+    s->attr_set[variant >> 6] |= 1ull << (variant & 63);
+  }
+  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.splits;
+  const long long units = s->num_sms / CTA_GROUP;
+  const int grid = static_cast<int>((tiles < units ? tiles : units) * CTA_GROUP);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = L::DYN_BYTES;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTA_GROUP;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, tc, p);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return GEMM_OK;
+}
+
+// Output options of one GEMM call.
+struct OutputSpec {
+  int epi = EPI_RAW32;
+  const float* row_scale = nullptr;
+  const float* col_scale = nullptr;
+  long long ldc = 0;        // row pitch of C in elements; 0 = dense (N)
+  bool no_split = false;    // C is a block of a larger matrix: never zero / add into it
+};
+
+// A, B already in the element type of KIND (fp16 or int8), pitches in bytes.
+template <int KIND, int EPI>
+int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const void* B,
+                    size_t b_pitch, void* C, const OutputSpec& out, cudaStream_t stream) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceState* s = nullptr;
+  int rc = device_state(&s);
+  if (rc != GEMM_OK) return rc;
+  constexpr int ELEM = (KIND == ptx::KIND_F16) ? 2 : 1;
+  constexpr int C_ELEM = (EPI == EPI_OUT16) ? 2 : 4;
+  const CUtensorMapDataType type =
+      (KIND == ptx::KIND_F16) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+  const int k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
+  const TileConfig cfg = select_config(M, N, s->num_sms, k_blocks, EPI == EPI_OUT16 ? 64 : 32,
+                                       EPI == EPI_RAW32 && !out.no_split);
+  const long long ldc = out.ldc ? out.ldc : N;
+  if (cfg.bn == 0) return GEMM_ERR_INVALID_ARG;  // override asks for a shape this mode lacks
+
+  CUtensorMap ta, tb;
+  const bool promote = !(g_l2_policy & 16);
+  rc = encode_operand_map(&ta, type, ELEM, A, M, K, a_pitch, BM, promote);
+  if (rc != GEMM_OK) return rc;
+  rc = encode_operand_map(&tb, type, ELEM, B, N, K, b_pitch, cfg.bn / cfg.cta_group, promote);
+  if (rc != GEMM_OK) return rc;
+
+  GemmParams p;
+  p.M = M;
+  p.N = N;
+  p.K = K;
+  p.tiles_m = ceil_div(M, BM * cfg.cta_group);
+  p.tiles_n = ceil_div(N, cfg.bn);
+  p.group_m = cfg.group_m;
+  p.k_blocks = k_blocks;
+  p.splits = cfg.splits;
+  p.ldc = ldc;
+  p.c_vec_ok = (ldc % (16 / C_ELEM) == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+  CUtensorMap tc;
+  if (p.c_vec_ok) {
+    // split-K adds into C by TMA reduction, which takes the element type from the map
+    rc = encode_c_map(&tc, C, M, N, ldc, C_ELEM,
+                      cfg.splits == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
+                      : KIND == ptx::KIND_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                              : CU_TENSOR_MAP_DATA_TYPE_INT32);
+    if (rc != GEMM_OK) return rc;
+  } else {
+    tc = ta;  // unused by the kernel on the plain-store path
+  }
+  p.C = static_cast<uint32_t*>(C);
+  p.row_scale = out.row_scale;
+  p.col_scale = out.col_scale;
+  p.status = s->status_ptr;
+  p.trace = (g_trace_on & 1) ? s->trace_ptr : nullptr;
+  p.ablate = (g_trace_on >> 1) & 15;
+  p.l2_policy = g_l2_policy & 3;
+  p.serpentine_k = (g_l2_policy & 4) ? 0 : 1;
+  p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
+
+  if (cfg.splits > 1) {  // only with a dense C (no_split is set for blocks of a larger matrix)
+    cudaError_t e = cudaMemsetAsync(C, 0, static_cast<size_t>(M) * N * C_ELEM, stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  const int vbase = ((KIND == ptx::KIND_F16) ? 0 : 32) + EPI * 8;  // bit index in attr_set
+  if (cfg.cta_group == 2) {
+    switch (cfg.bn) {
+      case 256: return launch_variant<KIND, 256, 6, 2, 1, EPI>(s, vbase + 4, ta, tb, tc, p, stream);
+      case 128: return launch_variant<KIND, 128, 4, 2, 2, EPI>(s, vbase + 5, ta, tb, tc, p, stream);
+      case 64: return launch_variant<KIND, 64, 4, 2, 2, EPI>(s, vbase + 6, ta, tb, tc, p, stream);
+      default: return GEMM_ERR_INVALID_ARG;
+    }
+  }
+  switch (cfg.bn) {
+    case 256: return launch_variant<KIND, 256, 4, 1, 1, EPI>(s, vbase + 0, ta, tb, tc, p, stream);
+    case 128: return launch_variant<KIND, 128, 3, 1, 2, EPI>(s, vbase + 1, ta, tb, tc, p, stream);
+    case 64: return launch_variant<KIND, 64, 4, 1, 2, EPI>(s, vbase + 2, ta, tb, tc, p, stream);
+    case 32:
+      if constexpr (EPI != EPI_OUT16)
+        return launch_variant<KIND, 32, 4, 1, 2, EPI>(s, vbase + 3, ta, tb, tc, p, stream);
+      return GEMM_ERR_INVALID_ARG;
+    default: return GEMM_ERR_INVALID_ARG;
+  }
+}
+
+template <int KIND>
+int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* B, size_t b_pitch,
+                void* C, cudaStream_t stream, const OutputSpec& out = OutputSpec()) {
+  switch (out.epi) {
+    case EPI_RAW32:
+      return launch_gemm_epi<KIND, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+    case EPI_OUT16:
+      return launch_gemm_epi<KIND, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+    case EPI_F32_SCALED:
+      if constexpr (KIND == ptx::KIND_I8)
+        return launch_gemm_epi<KIND, EPI_F32_SCALED>(M, N, K, A, a_pitch, B, b_pitch, C, out,
+                                                     stream);
+      return GEMM_ERR_INVALID_ARG;
+    default: return GEMM_ERR_INVALID_ARG;
+  }
+}
+
+int check_common(int M, int N, int K, const void* A, const void* B, const void* C) {
+  if (M <= 0 || N <= 0 || K <= 0 || !A || !B || !C) return GEMM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) |
+       reinterpret_cast<uintptr_t>(C)) & 15)
+    return GEMM_ERR_MISALIGNED;
+  return GEMM_OK;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Unpacks one or two packed matrices (rows_b may be 0) with the same K and output pitch.
+int launch_unpack(long long rows_a, const uint8_t* packed_a, int8_t* out_a, long long rows_b,
+                  const uint8_t* packed_b, int8_t* out_b, int K, size_t out_pitch,
+                  cudaStream_t stream) {
+  UnpackJob a{reinterpret_cast<const uint4*>(packed_a), out_a, rows_a * (K / 32)};
+  UnpackJob b{reinterpret_cast<const uint4*>(packed_b), out_b, rows_b * (K / 32)};
+  const long long chunks = a.chunks + b.chunks;
+  long long blocks = (chunks + 255) / 256;
+  if (blocks > 148 * 32) blocks = 148 * 32;
+  if (blocks < 1) blocks = 1;
+  unpack_s4_kernel<<<static_cast<int>(blocks), 256, 0, stream>>>(
+      a, b, K / 32, static_cast<long long>(out_pitch));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return GEMM_OK;
+}
+
+int check_s4(int M, int N, int K, const void* A, const void* B, const void* C) {
+  int rc = check_common(M, N, K, A, B, C);
+  if (rc != GEMM_OK) return rc;
+  if (K % 32) return GEMM_ERR_MISALIGNED;
+  if (K > K_LIMIT_INT) return GEMM_ERR_K_TOO_LARGE;
+  return GEMM_OK;
+}
+
+size_t s4_workspace_need(int M, int N, int K) {
+  return align_up(static_cast<size_t>(M) * K, 256) + align_up(static_cast<size_t>(N) * K, 256);
+}
+
+// INT4 GEMM through caller-visible scratch: unpack A and B to int8, then the INT8 kernel.
+int s4_with_workspace(int M, int N, int K, const uint8_t* A, const uint8_t* B, void* C,
+                      void* workspace, size_t workspace_bytes, const OutputSpec& out,
+                      cudaStream_t st) {
+  if (!workspace) return GEMM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < s4_workspace_need(M, N, K))
+    return GEMM_ERR_WORKSPACE;
+  int8_t* a8 = static_cast<int8_t*>(workspace);
+  int8_t* b8 = a8 + align_up(static_cast<size_t>(M) * K, 256);
+  int rc;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState* s = nullptr;
+    rc = device_state(&s);
+    if (rc != GEMM_OK) return rc;
+  }
+  rc = launch_unpack(M, A, a8, N, B, b8, K, static_cast<size_t>(K), st);
+  if (rc != GEMM_OK) return rc;
+  return launch_gemm<ptx::KIND_I8>(M, N, K, a8, static_cast<size_t>(K), b8, static_cast<size_t>(K),
+                                   C, st, out);
+}
+
+// The library's own grow-only scratch for the current device (cudaMalloc on growth).
+int s4_internal_workspace(size_t need, void** ws, size_t* ws_bytes) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceState* s = nullptr;
+  int rc = device_state(&s);
+  if (rc != GEMM_OK) return rc;
+  if (s->s4_workspace_bytes < need) {
+    // Grow: earlier launches may still read the old buffer.
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (s->s4_workspace) cudaFree(s->s4_workspace);
+    s->s4_workspace = nullptr;
+    s->s4_workspace_bytes = 0;
+    e = cudaMalloc(&s->s4_workspace, need);
+    if (e != cudaSuccess) return cuda_fail(e);
+    s->s4_workspace_bytes = need;
+  }
+  *ws = s->s4_workspace;
+  *ws_bytes = s->s4_workspace_bytes;
+  return GEMM_OK;
+}
+
+int check_scales(const float* row_scale, const float* col_scale, const void* C, int c_is_fp16,
+                 OutputSpec* out) {
+  if (!row_scale || !col_scale || !C || (c_is_fp16 != 0 && c_is_fp16 != 1))
+    return GEMM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(row_scale) | reinterpret_cast<uintptr_t>(col_scale)) & 3)
+    return GEMM_ERR_MISALIGNED;
+  out->epi = c_is_fp16 ? EPI_OUT16 : EPI_F32_SCALED;
+  out->row_scale = row_scale;
+  out->col_scale = col_scale;
+  return GEMM_OK;
+}
+}  // namespace
+}  // namespace b200gemm
