@@ -448,6 +448,33 @@ def run_sweep(args):
         torch.cuda.current_stream().wait_stream(side)
         return g
 
+    # the box's own CPU rate beside the GPU numbers: the oracle, as it stands, on the full
+    # N = 1024 problem of each precision (a fraction of a second each)
+    import oracle
+    cpu_rate = {}
+    for prec in synth.PRECISIONS:
+        A, B = synth.make(prec, 1024, 1024, 1024, synth.sweep_seed(prec, 1024))
+        t0 = time.perf_counter()
+        if prec == "fp16":
+            oracle.gemm_fp16(A, B)
+        elif prec == "s8":
+            oracle.gemm_s8_i64(A, B)
+        else:
+            oracle.gemm_s4_i64(A, B, 1024)
+        cpu_rate[prec] = synth.gemm_ops(1024, 1024, 1024) / (time.perf_counter() - t0) / 1e9
+    # MMA-issue-only rate of this machine, per kind, measured once before the sweep
+    mma_peak = {}
+    for kind in ("fp16", "s8"):
+        binding.gemm_mma_peak_probe(kind, 2048)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        pops = binding.gemm_mma_peak_probe(kind, 200000)
+        e1.record()
+        torch.cuda.synchronize()
+        mma_peak[kind] = pops / (e0.elapsed_time(e1) * 1e-3) / 1e12
+    mma_peak["s4"] = mma_peak["s8"]
+
     for prec in synth.PRECISIONS:
         for N in synth.SWEEP_SIZES:
             A, B = synth.make(prec, N, N, N, synth.sweep_seed(prec, N))
@@ -476,6 +503,8 @@ def run_sweep(args):
                 "host_us_per_call": host_us,
                 "value": rate, "unit": UNIT[prec], "frac_of_spec_peak": rate / SPEC_PEAK[prec],
                 "frac_of_cublas_bf16_burst_scaled": rate / ref,
+                "frac_of_mma_only_peak": rate / mma_peak[prec], "mma_only_peak": mma_peak[prec],
+                "cpu_oracle_gops_n1024": cpu_rate[prec], "cpu_cores": oracle.threads(),
                 "config": binding.gemm_query_config(prec, N, N, N)}), flush=True)
     if binding.gemm_last_device_status() != 0:
         raise SystemExit("bench.py: a kernel reported a barrier timeout")
