@@ -301,3 +301,53 @@ def test_split_k_more_ranges_than_blocks_is_capped():
         cfg = binding.gemm_query_config("s8", 130, 260, 256)
         assert int(cfg.split("split_k=")[1].split()[0]) <= 2, cfg     # never more ranges than slots
         check_against_oracle("s8", A, B, run_gpu("s8", A, B, fill=-7), force_full=True)
+
+
+# ------------------------------------------------------------ size and host-side edges
+def test_large_m_and_n_small_k():
+    """Many tiles (157 x 79 of the 128 x 256 shape), ragged both ways, C = 1.6 GB."""
+    M, N, K = 20001, 20004, 64
+    for prec in ("s8", "fp16"):
+        A, B = synth.make(prec, M, N, K, seed=123)
+        C = run_gpu(prec, A, B)
+        check_against_oracle(prec, A, B, C, seed=123)          # 256 rows + 256 columns + edges
+        if prec == "s8":
+            freivalds(prec, A, B, C, seed=123, vectors=2)
+        del C
+
+
+def test_two_host_threads_on_two_streams():
+    import threading
+    A, B = synth.s8_uniform(1024, 768, 2048, seed=31)
+    ref = oracle.gemm_s8(A, B)
+    dA, dB = to_dev(A), to_dev(B)
+    results, errors = {}, []
+
+    def worker(tag):
+        try:
+            st = torch.cuda.Stream()
+            with torch.cuda.stream(st):
+                outs = [binding.gemm_s8(dA, dB, stream=st) for _ in range(20)]
+            st.synchronize()
+            results[tag] = [o.cpu().numpy() for o in outs[-3:]]
+        except Exception as e:          # noqa: BLE001 - reported below
+            errors.append(e)
+
+    torch.cuda.synchronize()
+    threads = [threading.Thread(target=worker, args=(t,)) for t in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for tag in range(2):
+        for C in results[tag]:
+            assert np.array_equal(C, ref)
+
+
+def test_transpose_symmetry_on_gpu():
+    """gemm(A, B) == gemm(B, A)^T exactly for the integer paths (different tiles, same sums)."""
+    A, B = synth.s8_uniform(700, 300, 1024, seed=41)
+    assert np.array_equal(run_gpu("s8", A, B), run_gpu("s8", B, A).T)
+    A4, B4 = synth.s4_uniform(700, 300, 1024, seed=42)
+    assert np.array_equal(run_gpu("s4", A4, B4), run_gpu("s4", B4, A4).T)
