@@ -533,7 +533,8 @@ def run_ablation(args):
                  ("L2: default + 128-byte promotion", (0, 0, 0), 27, 1),
                  ("ablate: no MMAs (loads + barriers only)", (0, 0, 0), 11, 3),
                  ("ablate: no loads (MMAs + barriers only)", (0, 0, 0), 11, 5),
-                 ("epilogue waits with nanosleep back-off", (0, 0, 0), 11, 9)]
+                 ("epilogue waits with nanosleep back-off", (0, 0, 0), 11, 9),
+                 ("epilogue: direct register -> global stores", (0, 0, 0), 11, 33)]
     for prec in ("fp16", "s8"):
         dA, dB = (torch.from_numpy(x).cuda() for x in data[prec])
         C = torch.empty((N, N), dtype=torch.float32 if prec == "fp16" else torch.int32,
@@ -572,7 +573,7 @@ def run_ablation(args):
                     "producer_wait": float(a["producer_wait"].mean() / kb_total),
                     "producer_issue": float(a["producer_issue"].mean() / kb_total)},
                 "epilogue_busy_frac": float(a["epilogue_busy"].mean() / a["cycles"].mean()),
-                "result_valid": trace in (1, 9)}), flush=True)
+                "result_valid": trace in (1, 9, 33)}), flush=True)
     binding.gemm_set_config_override(0, 0, 0)
     binding.gemm_set_l2_policy(11)
     binding.gemm_trace_enable(0)

@@ -299,7 +299,9 @@ int gemm_set_l2_policy(int policy);
  * nanosleep instead of polling; 16 = failure drill: one operand slot of the
  * first tile is never filled, so the kernel's bounded waits (2 s) must expire,
  * record a code for gemm_last_device_status, drain and return -- the call takes
- * a few seconds, C is garbage and the context stays usable.  With bit 2, 4 or
+ * a few seconds, C is garbage and the context stays usable; 32 = the epilogue
+ * writes C straight from registers (16 bytes per thread and store) instead of
+ * staging it in shared memory for TMA stores (results unchanged).  With bit 2, 4 or
  * 16 set C is garbage; 2 and 4 exist to attribute cycles to the load path or
  * the MMA path.
  */

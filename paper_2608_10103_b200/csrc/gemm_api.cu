@@ -241,7 +241,7 @@ int gemm_set_l2_policy(int policy) {
 
 int gemm_trace_enable(int on) {
   std::lock_guard<std::mutex> lock(g_mutex);
-  g_trace_on = on & 31;
+  g_trace_on = on & 63;
   return GEMM_OK;
 }
 

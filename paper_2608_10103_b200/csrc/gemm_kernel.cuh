@@ -91,6 +91,7 @@ struct GemmParams {
   int serpentine_k;
   // Ablation switches for cycle accounting runs (results are then meaningless):
   // bit 0 = issue no MMAs (loads + barriers only), bit 1 = issue no loads (MMAs + barriers only),
+  // bit 4 = epilogue stores C straight from registers (no staging, no TMA store),
   // bit 2 = epilogue waits back off with nanosleep, bit 3 = host-requested failure drill: the
   // producer of CTA 0 leaves out the 3rd ring slot of its first tile, so the consumers' bounded
   // waits must expire, record a status code and let the kernel drain and return.
@@ -504,7 +505,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             }
           }
         }
-        if (p.c_vec_ok) {
+        if (EPI == EPI_RAW32 && (p.ablate & 16) && p.c_vec_ok && p.splits == 1) {
+          // ablation: straight from registers, 8 x 16 bytes per thread into its own C row
+          if (row < p.M) {
+            uint32_t* crow = p.C + static_cast<size_t>(row) * p.ldc;
+            if (col + 32 <= p.N) {
+              uint4* dst = reinterpret_cast<uint4*>(crow + col);
+#pragma unroll
+              for (int v = 0; v < 8; ++v)
+                dst[v] = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
+            } else {
+#pragma unroll
+              for (int v = 0; v < 32; ++v)
+                if (col + v < p.N) crow[col + v] = w[v];
+            }
+          }
+        } else if (p.c_vec_ok) {
           // registers -> swizzled shared memory -> one TMA store per block
           const uint32_t buf = epi_base + static_cast<uint32_t>((c & 1) * L::EPI_BUF_BYTES);
           // the store issued from this buffer two blocks ago must have read it

@@ -101,7 +101,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.col_scale = out.col_scale;
   p.status = s->status_ptr;
   p.trace = (g_trace_on & 1) ? s->trace_ptr : nullptr;
-  p.ablate = (g_trace_on >> 1) & 15;
+  p.ablate = (g_trace_on >> 1) & 31;
   p.l2_policy = g_l2_policy & 3;
   p.serpentine_k = (g_l2_policy & 4) ? 0 : 1;
   p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
