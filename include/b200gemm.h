@@ -235,7 +235,8 @@ int gemm_mma_peak_probe(int precision, int iters, int n_cols, int commit_every, 
 
 /*
  * Writes a human-readable description of the tile configuration the selector
- * picks for this problem ("BM=128 BN=256 stages=4 ...") into buf (NUL
+ * picks for this problem ("BM=256 BN=256 BK=64 cta_group=2 stages=6 group_m=12
+ * split_k=1 tiles=1024 ctas=148 kind=f16") into buf (NUL
  * terminated, truncated to len).  Host only, no GPU work.
  */
 int gemm_query_config(int precision, int M, int N, int K, char* buf, int len);
