@@ -185,11 +185,15 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
       static_cast<long long>(ceil_div(M, BM * c.cta_group)) * ceil_div(N, c.bn);
   const long long units = num_sms / c.cta_group;
   snprintf(buf, static_cast<size_t>(len),
-           "BM=%d BN=%d BK=%d cta_group=%d stages=%d group_m=%d split_k=%d tiles=%lld ctas=%lld "
-           "kind=%s%s",
+           "BM=%d BN=%d BK=%d cta_group=%d stages=%d group_m=%d split_k=%d split_tiles=%d "
+           "tiles=%lld ctas=%lld kind=%s%s",
            BM * c.cta_group, c.bn, atoms_for(c.bn, c.cta_group) * BK_BYTES / elem, c.cta_group,
-           c.stages, c.group_m, c.splits, tiles,
-           (tiles * c.splits < units ? tiles * c.splits : units) * c.cta_group,
+           c.stages, c.group_m, c.splits, c.splits > 1 ? c.split_tiles : 0, tiles,
+           (tiles + (c.splits > 1 ? static_cast<long long>(c.split_tiles) * (c.splits - 1) : 0) <
+                    units
+                ? tiles + (c.splits > 1 ? static_cast<long long>(c.split_tiles) * (c.splits - 1) : 0)
+                : units) *
+               c.cta_group,
            precision == GEMM_PREC_FP16 ? "f16" : "i8",
            precision == GEMM_PREC_S4 ? " prepass=unpack_s4" : "");
   return GEMM_OK;

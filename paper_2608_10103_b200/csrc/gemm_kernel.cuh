@@ -71,8 +71,11 @@ struct GemmParams {
   int tiles_m, tiles_n;  // number of C tiles (128*CTA_GROUP x BN) along M and N
   int group_m;           // raster: tiles are walked in bands of `group_m` tile rows
   int k_blocks;          // ceil(K bytes / BK_BYTES): 128-byte K atoms to cover K
-  int splits;            // split-K: each C tile is computed by `splits` work units over disjoint
-                         // K ranges and ADDED into a zeroed C (EPI_RAW32 only); 1 = off
+  int splits;            // split-K: each C tile from `split_from` on is computed by `splits` work
+                         // units over disjoint K ranges and ADDED into a zeroed C (EPI_RAW32
+                         // only); 1 = off
+  int split_from;        // first split tile in raster order: 0 splits every tile (few tiles, long
+                         // K); tiles - r splits only the last, partly filled wave of tiles
   int c_vec_ok;          // 1 if C rows allow 16-byte accesses (N % 4 == 0, base 16-byte aligned):
                          // the epilogue then stages C in shared memory and stores it by TMA
   uint32_t* C;           // element size 4 bytes, or 2 with EPI_OUT16
@@ -222,11 +225,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   const int lane = threadIdx.x & 31;
   const uint32_t cta_rank = (CTA_GROUP == 2) ? ptx::cluster_ctarank() : 0u;
   const bool leader = (cta_rank == 0);
-  // Work units: unit u = (tile u % tiles, K range u / tiles).  `num_tiles` counts units.
+  // Work units (`num_tiles` counts units): unit u < split_from is the whole tile u; the
+  // remaining tiles are each covered by `splits` units, one per K range.
   const int real_tiles = p.tiles_m * p.tiles_n;
-  const int num_tiles = real_tiles * p.splits;
+  const int split_tiles = real_tiles - p.split_from;
+  const int num_tiles = p.split_from + split_tiles * p.splits;
   const int k_slots_all = (p.k_blocks + KB - 1) / KB;  // ring slots per tile; a K tail is zero-filled
   const int k_per_split = (k_slots_all + p.splits - 1) / p.splits;
+  // unit -> tile, K range (in ring slots) and whether its result is added into C
+  auto decode_unit = [&](int u, int& tile, int& k_begin, int& k_end, bool& add) {
+    if (u < p.split_from) {
+      tile = u;
+      k_begin = 0;
+      k_end = k_slots_all;
+      add = false;
+    } else {
+      const int r = u - p.split_from;
+      tile = p.split_from + r % split_tiles;
+      k_begin = (r / split_tiles) * k_per_split;
+      k_end = min(k_begin + k_per_split, k_slots_all);
+      add = p.splits > 1;
+    }
+  };
   const int first_tile = static_cast<int>(blockIdx.x) / CTA_GROUP;
   const int tile_stride = static_cast<int>(gridDim.x) / CTA_GROUP;
   unsigned long long* const trace =
@@ -285,10 +305,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                                                                      : ptx::policy_evict_last();
       bool backward = false;
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
-        int tm, tn;
-        tile_coords(p, t % real_tiles, tm, tn);
-        const int k_begin = (t / real_tiles) * k_per_split;
-        const int k_end = min(k_begin + k_per_split, k_slots_all);
+        int tm, tn, tile, k_begin, k_end;
+        bool add;
+        decode_unit(t, tile, k_begin, k_end, add);
+        tile_coords(p, tile, tm, tn);
         const int a_row = tm * TILE_M + static_cast<int>(cta_rank) * BM;
         const int b_row = tn * BN + static_cast<int>(cta_rank) * L::B_ROWS;
         for (int ks = k_begin; ks < k_end; ++ks) {
@@ -367,8 +387,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         if (!ok) break;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
-        const int k_begin = (t / real_tiles) * k_per_split;
-        const int k_end = min(k_begin + k_per_split, k_slots_all);
+        int tile, k_begin, k_end;
+        bool add;
+        decode_unit(t, tile, k_begin, k_end, add);
         for (int ks = k_begin; ks < k_end; ++ks) {
           const long long w1 = trace ? clock64() : 0;
           ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
@@ -444,8 +465,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     bool ok = true;
     long long epi_wait = 0, epi_busy = 0, tiles_done = 0;
     for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
-      int tm, tn;
-      tile_coords(p, t % real_tiles, tm, tn);
+      int tm, tn, tile, k_begin, k_end;
+      bool add;
+      decode_unit(t, tile, k_begin, k_end, add);
+      tile_coords(p, tile, tm, tn);
       const long long w0 = trace ? clock64() : 0;
       ok = wait_bounded<true>(acc_full_bar(acc), acc_phase, abort_flag, p.status,
                               DEV_TIMEOUT_EPILOGUE, (p.ablate & 4) ? 500u : 0u);
@@ -455,7 +478,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       if (!ok) break;
       ptx::tc_fence_after_sync();
       // A split-K unit whose K range is empty (the host never creates one) contributes nothing.
-      const bool empty_range = (t / real_tiles) * k_per_split >= k_slots_all;
+      const bool empty_range = k_begin >= k_end;
       const int row0 = tm * TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
       const int row = row0 + lane;
       const int col0 = tn * BN;
@@ -505,7 +528,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             }
           }
         }
-        if (EPI == EPI_RAW32 && (p.ablate & 16) && p.c_vec_ok && p.splits == 1) {
+        if (EPI == EPI_RAW32 && (p.ablate & 16) && p.c_vec_ok && !add) {
           // ablation: straight from registers, 8 x 16 bytes per thread into its own C row
           if (row < p.M) {
             uint32_t* crow = p.C + static_cast<size_t>(row) * p.ldc;
@@ -538,7 +561,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           // reuse rule above exact.
           if (lane == 0) {
             if (row0 < p.M && col < p.N && !empty_range) {
-              if (EPI == EPI_RAW32 && p.splits > 1)
+              if (EPI == EPI_RAW32 && add)
                 ptx::tma_reduce_add_2d(&tmap_c, col, row0, buf);
               else
                 ptx::tma_store_2d(&tmap_c, col, row0, buf, pol_c);
@@ -555,7 +578,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                 crow[col + v] = static_cast<uint16_t>(w[v / 2] >> (16 * (v & 1)));
           } else {
             uint32_t* crow = p.C + static_cast<size_t>(row) * p.ldc;
-            if (EPI == EPI_RAW32 && p.splits > 1) {
+            if (EPI == EPI_RAW32 && add) {
 #pragma unroll
               for (int v = 0; v < 32; ++v) {
                 if (col + v >= p.N) continue;

@@ -20,7 +20,8 @@ int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUt
     if (e != cudaSuccess) return cuda_fail(e);
     s->attr_set[variant >> 6] |= 1ull << (variant & 63);
   }
-  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.splits;
+  const long long all_tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
+  const long long tiles = p.split_from + (all_tiles - p.split_from) * p.splits;  // work units
   const long long units = s->num_sms / CTA_GROUP;
   const int grid = static_cast<int>((tiles < units ? tiles : units) * CTA_GROUP);
   cudaLaunchConfig_t cfg = {};
@@ -83,6 +84,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.group_m = cfg.group_m;
   p.k_blocks = k_blocks;
   p.splits = cfg.splits;
+  p.split_from = p.tiles_m * p.tiles_n - (cfg.splits > 1 ? cfg.split_tiles : 0);
   p.ldc = ldc;
   p.c_vec_ok = (ldc % (16 / C_ELEM) == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
   CUtensorMap tc;
@@ -107,7 +109,38 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
 
   if (cfg.splits > 1) {  // only with a dense C (no_split is set for blocks of a larger matrix)
-    cudaError_t e = cudaMemsetAsync(C, 0, static_cast<size_t>(M) * N * C_ELEM, stream);
+    // Split tiles add into C: zero them first.  All tiles: one memset.  The last wave only:
+    // the bounding rectangle of those tiles (other tiles inside it are overwritten later).
+    cudaError_t e;
+    if (p.split_from == 0) {
+      e = cudaMemsetAsync(C, 0, static_cast<size_t>(M) * N * C_ELEM, stream);
+    } else {
+      int tm_lo = p.tiles_m, tm_hi = -1, tn_lo = p.tiles_n, tn_hi = -1;
+      for (int t = p.split_from; t < p.tiles_m * p.tiles_n; ++t) {
+        // the kernel's raster (tile_coords), on the host
+        const int band_tiles = p.group_m * p.tiles_n;
+        const int band = t / band_tiles;
+        const int first_m = band * p.group_m;
+        const int rows_in_band =
+            p.group_m < p.tiles_m - first_m ? p.group_m : p.tiles_m - first_m;
+        const int r = t - band * band_tiles;
+        const int tm = first_m + r % rows_in_band, tn = r / rows_in_band;
+        tm_lo = tm < tm_lo ? tm : tm_lo;
+        tm_hi = tm > tm_hi ? tm : tm_hi;
+        tn_lo = tn < tn_lo ? tn : tn_lo;
+        tn_hi = tn > tn_hi ? tn : tn_hi;
+      }
+      const long long row_lo = static_cast<long long>(tm_lo) * BM * cfg.cta_group;
+      long long row_hi = static_cast<long long>(tm_hi + 1) * BM * cfg.cta_group;
+      const long long col_lo = static_cast<long long>(tn_lo) * cfg.bn;
+      long long col_hi = static_cast<long long>(tn_hi + 1) * cfg.bn;
+      if (row_hi > M) row_hi = M;
+      if (col_hi > N) col_hi = N;
+      e = cudaMemset2DAsync(static_cast<uint8_t*>(C) + (row_lo * ldc + col_lo) * C_ELEM,
+                            static_cast<size_t>(ldc) * C_ELEM, 0,
+                            static_cast<size_t>(col_hi - col_lo) * C_ELEM,
+                            static_cast<size_t>(row_hi - row_lo), stream);
+    }
     if (e != cudaSuccess) return cuda_fail(e);
   }
   const int vbase = ((KIND == ptx::KIND_F16) ? 0 : 32) + EPI * 8;  // bit index in attr_set

@@ -13,6 +13,8 @@ struct TileConfig {
   int stages;
   int group_m;
   int splits;     // split-K factor (1 = off)
+  int split_tiles;  // how many tiles, counted from the end of the raster, are split
+                    // (all of them, or only the last partly filled wave)
 };
 
 constexpr int kWidths[] = {256, 128, 64, 32};
@@ -51,7 +53,7 @@ int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b
 // cluster launch (~2500) are paid once; split-K adds zeroing C and adding into it.
 TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 32,
                          bool allow_split = false) {
-  TileConfig best{256, 2, 6, 8, 1};
+  TileConfig best{256, 2, 6, 8, 1, 0};
   long long best_cost = -1;
   for (int cg = 2; cg >= 1; --cg) {
     if (g_override_cta_group && cg != g_override_cta_group) continue;
@@ -100,6 +102,29 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
   if (best_cost < 0) {  // the override names a shape this output mode does not have
     best.bn = 0;
     return best;
+  }
+  {
+    // Split-K of every tile, or -- when the tiles fill at least one wave and the last wave
+    // is at most half full -- of the last wave only: its r tiles become r * s units over
+    // disjoint K ranges, so the tail costs 1/s of a tile time instead of a whole one.
+    const long long tiles =
+        static_cast<long long>(ceil_div(M, BM * best.cta_group)) * ceil_div(N, best.bn);
+    const long long units = num_sms / best.cta_group;
+    const int slots = ceil_div(k_blocks, atoms_for(best.bn, best.cta_group));
+    best.split_tiles = best.splits > 1 ? static_cast<int>(tiles) : 0;
+    const long long r = tiles % units;
+    if (allow_split && best.splits == 1 && g_override_splits == 0 && tiles > units && r > 0 &&
+        2 * r <= units && slots >= 64) {  // measured: pays off (+2-3 %) only for long K
+      int sp = static_cast<int>(units / r);
+      if (sp > 4) sp = 4;
+      while (sp > 1 && (slots / sp < 32 ||
+                        static_cast<long long>(sp - 1) * ceil_div(slots, sp) >= slots))
+        --sp;
+      if (sp > 1) {
+        best.splits = sp;
+        best.split_tiles = static_cast<int>(r);
+      }
+    }
   }
   best.stages = stages_for(best.bn, best.cta_group);
   // Band height: one wave of tiles about twice as tall as wide in operand bytes (measured

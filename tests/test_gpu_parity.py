@@ -351,3 +351,22 @@ def test_transpose_symmetry_on_gpu():
     assert np.array_equal(run_gpu("s8", A, B), run_gpu("s8", B, A).T)
     A4, B4 = synth.s4_uniform(700, 300, 1024, seed=42)
     assert np.array_equal(run_gpu("s4", A4, B4), run_gpu("s4", B4, A4).T)
+
+
+def test_tail_wave_split():
+    """4096^2 x 8192 FP16: 256 tiles on 74 SM pairs leave a last wave of 34 tiles, which the
+    selector splits in two along K (adds into a zeroed rectangle of C); ragged variant too."""
+    for M, N, K in ((4096, 4096, 8192), (4000, 3900, 8200)):
+        cfg = binding.gemm_query_config("fp16", M, N, K)
+        assert "split_k=2 " in cfg and "split_tiles=0 " not in cfg, cfg
+        A, B = synth.fp16_uniform(M, N, K, seed=77)
+        C = run_gpu("fp16", A, B, fill=float("nan"))
+        check_against_oracle("fp16", A, B, C, seed=77)
+        freivalds("fp16", A, B, C, seed=77, vectors=4)
+    # the integer kernel takes the same path when K is long enough
+    M, N, K = 4096, 4096, 8192
+    assert "split_k=2 " in binding.gemm_query_config("s8", M, N, K)
+    A, B = synth.s8_uniform(M, N, K, seed=78)
+    C = run_gpu("s8", A, B, fill=-7)
+    check_against_oracle("s8", A, B, C, seed=78)
+    freivalds("s8", A, B, C, seed=78, vectors=4)
