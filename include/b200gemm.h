@@ -25,7 +25,10 @@
  * work (Sec. VI).  When a problem has fewer C tiles than the GPU has SMs (small
  * M, as in LLM decoding, or small squares) the selector lets several work units
  * share one tile over disjoint K ranges: C is zeroed on the stream and every
- * unit ADDS its partial tile (TMA reduction).  INT32 results stay exact; FP32
+ * unit ADDS its partial tile (TMA reduction).  When the tiles fill more than one
+ * wave of SMs but the last wave is at most half full and K is long, only that
+ * last wave's tiles are split (and only their part of C is zeroed first).
+ * INT32 results stay exact; FP32
  * results then depend on the order the partial sums land, i.e. two runs can
  * differ in the last bits, always inside the stated bound.
  *
@@ -236,7 +239,7 @@ int gemm_mma_peak_probe(int precision, int iters, int n_cols, int commit_every, 
 /*
  * Writes a human-readable description of the tile configuration the selector
  * picks for this problem ("BM=256 BN=256 BK=64 cta_group=2 stages=6 group_m=12
- * split_k=1 tiles=1024 ctas=148 kind=f16") into buf (NUL
+ * split_k=1 split_tiles=0 tiles=1024 ctas=148 kind=f16") into buf (NUL
  * terminated, truncated to len).  Host only, no GPU work.
  */
 int gemm_query_config(int precision, int M, int N, int K, char* buf, int len);
