@@ -102,3 +102,55 @@ def test_product_path_never_touches_the_oracle():
         if f.endswith((".py", ".c")):
             text = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2608_10103_b200" not in text and "b200gemm" not in text, f
+
+
+def _parse(cfg):
+    out = {}
+    for tok in cfg.split():
+        if "=" in tok:
+            k, v = tok.split("=", 1)
+            out[k] = int(v) if v.lstrip("-").isdigit() else v
+    return out
+
+
+def test_selector_invariants_over_many_shapes(lib):
+    """Host logic only: whatever the selector picks must be a built shape, its split-K
+    factor must leave no K range empty, and the CTA count must fit the machine."""
+    import itertools
+    dims = [1, 7, 128, 129, 256, 300, 512, 1000, 2048, 2560, 4096, 5120, 8192, 20001]
+    ks = [32, 64, 160, 512, 1056, 4096, 8192, 16384, 131040]
+    built = {(1, 256), (1, 128), (1, 64), (1, 32), (2, 256), (2, 128), (2, 64)}
+    for prec, elem in (("fp16", 2), ("s8", 1), ("s4", 1)):
+        for M, N, K in itertools.product(dims, dims, ks):
+            c = _parse(binding.gemm_query_config(prec, M, N, K))
+            cg, bn, sp = c["cta_group"], c["BN"], c["split_k"]
+            assert (cg, bn) in built and c["BM"] == 128 * cg
+            atoms = c["BK"] * elem // 128
+            assert atoms in (1, 2)
+            slots = -(-(-(-K * elem // 128)) // atoms)
+            tiles = -(-M // c["BM"]) * -(-N // bn)
+            assert c["tiles"] == tiles
+            assert 1 <= sp <= 32 and sp <= slots
+            assert (sp - 1) * -(-slots // sp) < slots, (prec, M, N, K, c)
+            if sp > 1:
+                assert 0 < c["split_tiles"] <= tiles
+                units = tiles + c["split_tiles"] * (sp - 1)
+            else:
+                assert c["split_tiles"] == 0
+                units = tiles
+            assert c["ctas"] == min(units, 148 // cg) * cg
+            assert 1 <= c["group_m"] <= -(-M // c["BM"])
+
+
+def test_selector_headline_choices(lib):
+    big = _parse(binding.gemm_query_config("fp16", 8192, 8192, 8192))
+    assert (big["BM"], big["BN"], big["cta_group"], big["split_k"], big["stages"]) == (256, 256, 2, 1, 6)
+    dec = _parse(binding.gemm_query_config("s8", 16, 8192, 8192))
+    assert dec["split_k"] > 1 and dec["split_tiles"] == dec["tiles"]
+    tail = _parse(binding.gemm_query_config("fp16", 4096, 4096, 8192))
+    assert tail["split_k"] == 2 and tail["split_tiles"] == 256 % 74
+    binding.gemm_set_config_override(0, 0, 0, 1)
+    try:
+        assert _parse(binding.gemm_query_config("fp16", 4096, 4096, 8192))["split_k"] == 1
+    finally:
+        binding.gemm_set_config_override(0, 0, 0, 0)
