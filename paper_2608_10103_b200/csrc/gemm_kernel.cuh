@@ -464,6 +464,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     uint32_t acc_phase = 0;
     bool ok = true;
     long long epi_wait = 0, epi_busy = 0, tiles_done = 0;
+    uint32_t staged_blocks = 0;  // blocks sent through the staging buffers so far
     for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
       int tm, tn, tile, k_begin, k_end;
       bool add;
@@ -545,8 +546,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           }
         } else if (p.c_vec_ok) {
           // registers -> swizzled shared memory -> one TMA store per block
-          const uint32_t buf = epi_base + static_cast<uint32_t>((c & 1) * L::EPI_BUF_BYTES);
-          // the store issued from this buffer two blocks ago must have read it
+          // The two staging buffers alternate per BLOCK, counted across tiles (a tile may
+          // have an odd number of blocks): the store issued from this buffer two blocks ago
+          // must have read it
+          const uint32_t buf = epi_base + static_cast<uint32_t>((staged_blocks & 1) * L::EPI_BUF_BYTES);
+          ++staged_blocks;
           if (lane == 0) ptx::bulk_wait_group_read<1>();
           __syncwarp();
           const uint32_t row_addr = buf + static_cast<uint32_t>(lane * 128);

@@ -54,6 +54,20 @@ def test_fp16_out_every_tile_shape(bn, cta_group):
     assert ok, "error %.3g x bound" % worst
 
 
+
+@pytest.mark.parametrize("bn,cta_group", SHAPES16)
+def test_fp16_out_many_short_tiles_per_cta(bn, cta_group):
+    """Short mainloop, several tiles per CTA: consecutive tiles' stores overlap (the 64-wide
+    tile has a single 16-bit store block per tile)."""
+    M, N, K = 3000, 1000, 32
+    A, B = synth.fp16_normal_clipped(M, N, K, seed=bn)
+    ref, S = oracle.gemm_fp16(A, B)
+    binding.gemm_set_config_override(bn, 0, cta_group, 1)
+    for rep in range(3):
+        ok, worst = oracle.fp16_out_check(run_f16out(A, B), ref, S)
+        assert ok, "repeat %d: error %.3g x bound" % (rep, worst)
+
+
 def test_fp16_out_rejects_the_32_wide_tile():
     A, B = synth.fp16_uniform(64, 64, 64, seed=1)
     binding.gemm_set_config_override(32, 0, 1)
@@ -111,6 +125,20 @@ def test_dequant_every_tile_shape(bn, cta_group):
     assert oracle.dequant_check(run_dequant("s8", A, B, rs, cs, torch.float32), ref, False)[0]
     if bn >= 64:
         assert oracle.dequant_check(run_dequant("s8", A, B, rs, cs, torch.float16), ref, True)[0]
+
+
+
+@pytest.mark.parametrize("bn,cta_group", [(32, 1), (64, 1), (64, 2), (256, 2)])
+def test_dequant_many_short_tiles_per_cta(bn, cta_group):
+    M, N, K = 1024, 4096, 32
+    A, B = synth.s8_uniform(M, N, K, seed=bn)
+    rs, cs = scales(M, N, seed=bn)
+    ref = oracle.dequant_ref(oracle.gemm_s8_i64(A, B), rs, cs)
+    binding.gemm_set_config_override(bn, 0, cta_group, 1)
+    for rep in range(2):
+        assert oracle.dequant_check(run_dequant("s8", A, B, rs, cs, torch.float32), ref, False)[0]
+        if bn >= 64:
+            assert oracle.dequant_check(run_dequant("s8", A, B, rs, cs, torch.float16), ref, True)[0]
 
 
 def test_dequant_with_unit_scales_is_the_exact_integer():

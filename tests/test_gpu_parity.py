@@ -114,6 +114,22 @@ def test_every_tile_shape(prec, bn, cta_group):
     check_against_oracle(prec, A, B, C, force_full=True)
 
 
+@pytest.mark.parametrize("bn,cta_group", SHAPES)
+@pytest.mark.parametrize("prec,M,N,K", [("fp16", 3000, 1000, 32), ("s8", 1024, 4096, 32),
+                                        ("s4", 1500, 2304, 32), ("s8", 1500, 4096, 512)])
+def test_many_short_tiles_per_cta(prec, M, N, K, bn, cta_group):
+    """Several tiles per CTA with a mainloop far shorter than the epilogue: the stores of
+    consecutive tiles overlap, so a staging buffer reused too early shows as wrong values
+    (a tile whose epilogue has an odd number of store blocks is the critical case).
+    Repeated calls, compared in full."""
+    A, B = synth.make(prec, M, N, K, seed=K + bn)
+    binding.gemm_set_config_override(bn, 0, cta_group, 1)
+    ref, S = oracle_block(prec, A, B)
+    for rep in range(3):
+        C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
+        assert_block(prec, C, ref, S, "repeat %d" % rep)
+
+
 @pytest.mark.parametrize("group_m", [1, 2, 3, 7, 64])
 def test_raster_band_heights(group_m):
     M, N, K = 1300, 1500, 256
