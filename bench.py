@@ -521,7 +521,8 @@ def run_ablation(args):
     N = args.size
     ops = synth.gemm_ops(N, N, N)
     data = {"fp16": synth.fp16_normal_clipped(N, N, N, seed=3),
-            "s8": synth.s8_uniform(N, N, N, seed=synth.sweep_seed("s8", 8192))}
+            "s8": synth.s8_uniform(N, N, N, seed=synth.sweep_seed("s8", 8192)),
+            "s4": synth.s4_uniform(N, N, N, seed=synth.sweep_seed("s4", 8192))}
     variants = [("baseline (selector default)", (0, 0, 0), 11, 1)]
     variants += [("tile 128x%d, one CTA" % bn, (bn, 0, 1), 11, 1) for bn in (256, 128, 64, 32)]
     variants += [("tile 256x%d, CTA pair" % bn, (bn, 0, 2), 11, 1) for bn in (256, 128, 64)]
@@ -535,12 +536,20 @@ def run_ablation(args):
                  ("ablate: no loads (MMAs + barriers only)", (0, 0, 0), 11, 5),
                  ("epilogue waits with nanosleep back-off", (0, 0, 0), 11, 9),
                  ("epilogue: direct register -> global stores", (0, 0, 0), 11, 33)]
-    for prec in ("fp16", "s8"):
+    # INT4: how the nibbles reach the int8 tensor-core path (the traced launch is the GEMM;
+    # the pre-pass launch of route 0 is inside the timed loop but not in the cycle accounting)
+    s4_variants = [("INT4 route 0: pre-pass to int8 + INT8 GEMM (default)", (0, 0, 0), 11, 1, 0),
+                   ("INT4 route 1: nibbles expanded inside the GEMM kernel", (0, 0, 0), 11, 1, 1),
+                   ("INT4 route 1, ablate: no MMAs", (0, 0, 0), 11, 3, 1),
+                   ("INT4 route 1, ablate: no operand loads", (0, 0, 0), 11, 5, 1)]
+    for prec in ("fp16", "s8", "s4"):
         dA, dB = (torch.from_numpy(x).cuda() for x in data[prec])
         C = torch.empty((N, N), dtype=torch.float32 if prec == "fp16" else torch.int32,
                         device="cuda")
         flop_per_clk = 8192 if prec == "fp16" else 16384
-        for name, override, policy, trace in variants:
+        for v in (s4_variants if prec == "s4" else variants):
+            name, override, policy, trace = v[:4]
+            binding.gemm_set_s4_scheme(v[4] if len(v) > 4 else 0)
             binding.gemm_set_config_override(*override)
             binding.gemm_set_l2_policy(policy)
             binding.gemm_trace_enable(trace)
@@ -560,6 +569,12 @@ def run_ablation(args):
             a = {k: np.array([t[k] for t in tr], dtype=np.float64) for k in binding.TRACE_FIELDS}
             lead = a["mma_issue"] > 0
             kb_total = a["tiles"].mean() * (N * (2 if prec == "fp16" else 1) // 128)
+            unpack = {}
+            if a["unpack_busy"].max() > 0:
+                unpack = {"unpack_cycles_per_kblock": {
+                    k: float(a[f].mean() / kb_total) for k, f in (
+                        ("wait_packed_operands", "unpack_wait_packed"),
+                        ("wait_free_int8_slot", "unpack_wait_slot"), ("expanding", "unpack_busy"))}}
             cyc = float(a["cycles"].max())
             print(json.dumps({
                 "ablation": name, "precision": prec, "N": N, "config": cfg,
@@ -573,7 +588,8 @@ def run_ablation(args):
                     "producer_wait": float(a["producer_wait"].mean() / kb_total),
                     "producer_issue": float(a["producer_issue"].mean() / kb_total)},
                 "epilogue_busy_frac": float(a["epilogue_busy"].mean() / a["cycles"].mean()),
-                "result_valid": trace in (1, 9, 33)}), flush=True)
+                "result_valid": trace in (1, 9, 33), **unpack}), flush=True)
+    binding.gemm_set_s4_scheme(0)
     binding.gemm_set_config_override(0, 0, 0)
     binding.gemm_set_l2_policy(11)
     binding.gemm_trace_enable(0)

@@ -261,9 +261,31 @@ int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k);
  * Kernels never spin forever: a barrier wait that exceeds its limit makes the
  * kernel record a non-zero code and drain.  This reads that code for the
  * current device (synchronises the device) and clears it.  0 = no event;
- * 1/2/3 = producer / MMA / epilogue wait expired.
+ * 1/2/3 = producer / MMA / epilogue wait expired, 5 = a wait of the INT4
+ * expansion warps expired.
  */
 int gemm_last_device_status(void);
+
+/*
+ * Route of later gemm_s4 / gemm_s4_dequant calls.  tcgen05 has no signed 4-bit
+ * integer kind (the paper's kernels feed mma.sync m16n8k64 .s4 operands
+ * directly, Listing 2c), so the nibbles are expanded to int8 either
+ *   0 (default): by a streaming pre-pass kernel into an int8 scratch, followed
+ *     by the INT8 GEMM; or
+ *   1: inside the GEMM kernel ("fused") where that variant applies, i.e. where
+ *     the selector picks the 256 x 256 CTA-pair tile without split-K (large
+ *     problems), else as 0.  Packed tiles are loaded as they are and eight extra
+ *     warps per CTA expand them in shared memory into the slots the MMAs read:
+ *     no scratch and half the operand bytes through L2 and HBM, but half as much
+ *     shared-memory traffic again per unit of math, and shared-memory bandwidth
+ *     is what bounds this kernel: at N = 8192 it is about 1.35x slower than
+ *     route 0.  Kept as the measured alternative of the INT4 ablation.
+ * gemm_s4_ws and gemm_s4_static always take route 0.  Results are identical,
+ * bit for bit.  gemm_query_config shows the route.  The paper has no
+ * counterpart; its Run 4 ablates how the operands reach the tensor cores, of
+ * which this is the analogue here.
+ */
+int gemm_set_s4_scheme(int scheme);
 
 /*
  * L2 behaviour of later calls, a bit set (the paper's Run 4 ablates the
@@ -285,17 +307,19 @@ int gemm_set_l2_policy(int policy);
 /*
  * Cycle accounting, in the spirit of the counter attribution the paper does
  * with its profiler (Sec. III-B).  gemm_trace_enable(1) makes later GEMM
- * launches record, per CTA, 12 unsigned 64-bit words: [0] SM cycles and [1]
+ * launches record, per CTA, 16 unsigned 64-bit words: [0] SM cycles and [1]
  * nanoseconds the CTA ran (their ratio is the SM clock during the kernel),
  * cycles the producer waited for a free slot [2], the MMA issuer waited for
  * operands [3] and for a free accumulator [4], one epilogue warp waited for a
  * finished accumulator [5] and spent draining [6], the tile count [7], and the
  * issuer's cycles inside tcgen05.mma [8] and tcgen05.commit [9], the cycles
  * the CTA spent setting up barriers and tensor memory [10], and the producer's
- * cycles issuing loads [11].
+ * cycles issuing loads [11]; fused INT4 only, one expansion warp: cycles
+ * waiting for packed operands [12], for a free int8 slot [13] and spent
+ * expanding [14]; [15] is unused.
  * gemm_trace_read synchronises the device, copies the words of the first
  * min(max_ctas, 160) CTAs of the last traced launch to `out` (host memory,
- * 12 * max_ctas words) and returns that CTA count.  Off by default; the cost
+ * 16 * max_ctas words) and returns that CTA count.  Off by default; the cost
  * when on is a few clock reads per k-block.
  * `on` is a bit set: 1 = record; 2 = ablation, issue no MMAs (operand loads and
  * barriers only); 4 = ablation, issue no operand loads (MMAs and barriers only,

@@ -23,7 +23,7 @@ EXPORTS = (
     "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
     "gemm_fp16_f16out", "gemm_s8_dequant", "gemm_s4_dequant", "gemm_host", "gemm_host_release",
     "gemm_s4_static", "gemm_s4_static_capacity", "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
-    "gemm_set_config_override", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_last_device_status", "gemm_last_cuda_error",
+    "gemm_set_config_override", "gemm_set_s4_scheme", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_last_device_status", "gemm_last_cuda_error",
     "gemm_status_string", "gemm_version",
 )
 
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.gemm_mma_peak_probe.argtypes = [i, i, i, i, ctypes.POINTER(ctypes.c_double), vp]
         L.gemm_query_config.argtypes = [i, i, i, i, ctypes.c_char_p, i]
         L.gemm_set_config_override.argtypes = [i, i, i, i]
+        L.gemm_set_s4_scheme.argtypes = [i]
         L.gemm_set_l2_policy.argtypes = [i]
         L.gemm_trace_enable.argtypes = [i]
         L.gemm_trace_read.argtypes = [ctypes.POINTER(ctypes.c_ulonglong), i]
@@ -300,6 +301,13 @@ def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0, 
            "gemm_set_config_override")
 
 
+def gemm_set_s4_scheme(scheme: int = 0):
+    """Route of gemm_s4 / gemm_s4_dequant: 0 = pre-pass to int8 + INT8 GEMM (default); 1 =
+    nibbles expanded inside the GEMM kernel where that variant applies (256 x 256 CTA-pair
+    tile, no split-K), else the pre-pass."""
+    _check(lib().gemm_set_s4_scheme(int(scheme)), "gemm_set_s4_scheme")
+
+
 def gemm_set_l2_policy(policy: int = 11):
     """Bit set: bits 0-1 operand eviction priority (0 normal, 1 keep A / stream B, 2 keep
     both, 3 keep A), +4 serpentine K order off, +8 C stores evict-first, +16 128-byte L2
@@ -309,7 +317,7 @@ def gemm_set_l2_policy(policy: int = 11):
 
 TRACE_FIELDS = ("cycles", "nanos", "producer_wait", "mma_wait_operands", "mma_wait_accumulator",
                 "epilogue_wait", "epilogue_busy", "tiles", "mma_issue", "mma_commit", "setup",
-                "producer_issue")
+                "producer_issue", "unpack_wait_packed", "unpack_wait_slot", "unpack_busy", "unused15")
 TRACE_SLOTS = len(TRACE_FIELDS)
 
 

@@ -57,12 +57,7 @@ int gemm_s4(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t* C,
             gemm_stream_t stream) {
   int rc = check_s4(M, N, K, A, B, C);
   if (rc != GEMM_OK) return rc;
-  void* ws = nullptr;
-  size_t ws_bytes = 0;
-  rc = s4_internal_workspace(s4_workspace_need(M, N, K), &ws, &ws_bytes);
-  if (rc != GEMM_OK) return rc;
-  return s4_with_workspace(M, N, K, A, B, C, ws, ws_bytes, OutputSpec(),
-                           reinterpret_cast<cudaStream_t>(stream));
+  return s4_auto(M, N, K, A, B, C, OutputSpec(), reinterpret_cast<cudaStream_t>(stream));
 }
 
 int gemm_fp16_f16out(int M, int N, int K, const void* A, const void* B, void* C,
@@ -98,12 +93,7 @@ int gemm_s4_dequant(int M, int N, int K, const uint8_t* A, const uint8_t* B,
   OutputSpec out;
   rc = check_scales(row_scale, col_scale, C, c_is_fp16, &out);
   if (rc != GEMM_OK) return rc;
-  void* ws = nullptr;
-  size_t ws_bytes = 0;
-  rc = s4_internal_workspace(s4_workspace_need(M, N, K), &ws, &ws_bytes);
-  if (rc != GEMM_OK) return rc;
-  return s4_with_workspace(M, N, K, A, B, C, ws, ws_bytes, out,
-                           reinterpret_cast<cudaStream_t>(stream));
+  return s4_auto(M, N, K, A, B, C, out, reinterpret_cast<cudaStream_t>(stream));
 }
 
 int gemm_release_workspaces(void) {
@@ -195,7 +185,10 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
                 : units) *
                c.cta_group,
            precision == GEMM_PREC_FP16 ? "f16" : "i8",
-           precision == GEMM_PREC_S4 ? " prepass=unpack_s4" : "");
+           precision != GEMM_PREC_S4 ? ""
+           : (g_s4_scheme == 1 && c.bn == 256 && c.cta_group == 2 && c.splits == 1)
+               ? " s4=fused_unpack(4+2 slots)"
+               : " prepass=unpack_s4");
   return GEMM_OK;
 }
 
@@ -236,6 +229,13 @@ int gemm_last_device_status(void) {
   return v;
 }
 
+int gemm_set_s4_scheme(int scheme) {
+  if (scheme < 0 || scheme > 1) return GEMM_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  g_s4_scheme = scheme;
+  return GEMM_OK;
+}
+
 int gemm_set_l2_policy(int policy) {
   if (policy < 0 || policy > 31) return GEMM_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
@@ -250,7 +250,7 @@ int gemm_trace_enable(int on) {
 }
 
 int gemm_trace_read(unsigned long long* out, int max_ctas) {
-  static_assert(TRACE_SLOTS == 12, "header documents 12 words per CTA");
+  static_assert(TRACE_SLOTS == 16, "header documents 16 words per CTA");
   if (!out || max_ctas <= 0) return GEMM_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
   DeviceState* s = nullptr;

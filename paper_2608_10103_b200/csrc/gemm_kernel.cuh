@@ -27,6 +27,15 @@
 //   commits signal `empty` / `acc_full` in both CTAs; both epilogues report to the
 //   leader's `acc_empty`.
 //
+// PSTAGES > 0 (fused INT4): A and B hold packed signed 4-bit values (Listing 2c's s4
+//   operands).  The producer lands PACKED tiles (rows x 128 bytes = 256 nibbles of K) in a
+//   second ring of PSTAGES slots; warps 6..9 expand each packed slot into two int8 slots of
+//   the ring the MMA issuer reads, every value multiplied by 16 (nibble moved to the high
+//   half of its byte, low half zero), so the accumulators hold 256 * C and the epilogue
+//   shifts them right by 8, exactly.  The order in which K values land in the int8 slots
+//   differs from their order in memory, identically for A and B, which leaves every dot
+//   product unchanged.
+//
 // A is M x K row-major, B is N x K with K contiguous (the paper's ".row.col"
 // operand layout, Listing 2c); C is M x N row-major, 32-bit, overwritten.
 // Tiles outside M, N or K are zero-filled by the TMA loads and clipped by the
@@ -47,6 +56,8 @@ constexpr int BK_BYTES = 128;     // K extent of one pipeline slot, in bytes (on
 constexpr int MMA_K_BYTES = 32;   // K extent of one tcgen05.mma, in bytes
 constexpr int NUM_THREADS = 192;  // 6 warps: producer, MMA, 4 x epilogue
 constexpr int EPI_WARPS = 4;
+constexpr int UNPACK_WARPS = 8;   // fused INT4 only: warps 6..13
+constexpr int NUM_THREADS_FUSED = NUM_THREADS + 32 * UNPACK_WARPS;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // every barrier wait gives up after 2 s
 
 // Device status codes written to the status word when a wait gives up.
@@ -56,6 +67,7 @@ enum DeviceStatus {
   DEV_TIMEOUT_MMA = 2,
   DEV_TIMEOUT_EPILOGUE = 3,
   DEV_TIMEOUT_DRAIN = 4,
+  DEV_TIMEOUT_UNPACK = 5,
 };
 
 // What the epilogue writes.
@@ -115,27 +127,34 @@ enum TraceSlot {
   TRACE_MMA_COMMIT = 9,     // MMA issuer: cycles inside tcgen05.commit
   TRACE_SETUP = 10,         // cycles from kernel start until barriers and TMEM are set up
   TRACE_PROD_ISSUE = 11,    // producer: cycles issuing expect_tx + TMA loads
-  TRACE_SLOTS = 12
+  TRACE_UNPACK_WAIT_IN = 12,   // fused INT4, unpack warp 6: cycles waiting for packed operands
+  TRACE_UNPACK_WAIT_OUT = 13,  // ... waiting for a free int8 slot
+  TRACE_UNPACK_BUSY = 14,      // ... expanding nibbles
+  TRACE_SLOTS = 16
 };
 
 // One ring slot holds KB "atoms" per operand; an atom is a tile of rows x 128
 // bytes of K in the 128-byte-swizzle layout (the widest a swizzled TMA box can
 // be).  KB = 2 halves the per-slot barrier work (one wait, one commit per 8 MMAs)
 // of the single issuing thread, whose instruction time is the scarce resource.
-template <int BN, int STAGES, int CTA_GROUP, int KB>
+template <int BN, int STAGES, int CTA_GROUP, int KB, int PSTAGES = 0>
 struct SmemLayout {
   static constexpr int B_ROWS = BN / CTA_GROUP;  // B rows each CTA loads
   static constexpr int A_BYTES = BM * BK_BYTES;       // one A atom
   static constexpr int B_BYTES = B_ROWS * BK_BYTES;   // one B atom
   static constexpr int STAGE_BYTES = KB * (A_BYTES + B_BYTES);
-  static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
+  // Fused INT4: PSTAGES more slots, each one packed atom per operand (256 nibbles of K per row).
+  static constexpr int P_STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int P_OFFSET = STAGES * STAGE_BYTES;
+  static constexpr int RING_BYTES = STAGES * STAGE_BYTES + PSTAGES * P_STAGE_BYTES;
   // Epilogue staging: per epilogue warp two buffers of 32 rows x 128 bytes (32 x 32 C values).
   static constexpr int EPI_BUF_BYTES = 32 * 128;
   static constexpr int EPI_OFFSET = RING_BYTES;
   static constexpr int EPI_BYTES = EPI_WARPS * 2 * EPI_BUF_BYTES;
   static constexpr int BAR_OFFSET = EPI_OFFSET + EPI_BYTES;
-  // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], drain
-  static constexpr int NUM_BARS = 2 * STAGES + 5;
+  // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], drain, p_full[PSTAGES], p_empty[PSTAGES]
+  // fused INT4 adds ready[STAGES]
+  static constexpr int NUM_BARS = 2 * STAGES + 5 + 2 * PSTAGES + (PSTAGES > 0 ? STAGES : 0);
   static constexpr int MISC_OFFSET = BAR_OFFSET + NUM_BARS * 8;
   static constexpr int TOTAL = MISC_OFFSET + 16;
   static constexpr int DYN_BYTES = TOTAL + 1024;  // slack to align the ring to 1024 bytes
@@ -194,11 +213,13 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32, int PSTAGES = 0>
+__global__ void __launch_bounds__(PSTAGES > 0 ? NUM_THREADS_FUSED : NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
-  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB>;
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES>;
+  constexpr bool FUSED = PSTAGES > 0;  // packed INT4 operands, expanded on the way to the MMAs
+  static_assert(!FUSED || (KIND == ptx::KIND_I8 && KB == 1), "fused INT4: int8 MMAs, one atom per slot");
   constexpr int ELEM_BYTES = (KIND == ptx::KIND_F16) ? 2 : 1;
   constexpr int BK_ELEMS = BK_BYTES / ELEM_BYTES;
   constexpr int TILE_M = BM * CTA_GROUP;
@@ -218,6 +239,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   auto acc_full_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
   auto acc_empty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
   const uint32_t drain_bar = bar0 + 8u * (2 * STAGES + 4);
+  auto p_full_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 5 + s); };
+  auto p_empty_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 5 + PSTAGES + s); };
+  // fused INT4: int8 slot s of THIS CTA has been written by all its unpack warps.  The leader's
+  // MMA issuer waits for its own `ready` and, in a pair, for `full`, on which the peer's
+  // otherwise idle warp 1 relays the peer's `ready` (one remote arrive per slot: a remote
+  // arrive with release semantics straight from the writing warps costs each of them
+  // hundreds of cycles).
+  auto ready_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 5 + 2 * PSTAGES + s); };
   volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(base_ptr + L::MISC_OFFSET);
   volatile uint32_t* abort_flag = tmem_holder + 1;
 
@@ -259,6 +288,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     for (int s = 0; s < STAGES; ++s) {
       ptx::mbar_init(full_bar(s), 1);
       ptx::mbar_init(empty_bar(s), 1);
+      if constexpr (FUSED) ptx::mbar_init(ready_bar(s), UNPACK_WARPS);
+    }
+    for (int s = 0; s < PSTAGES; ++s) {
+      ptx::mbar_init(p_full_bar(s), 1);
+      ptx::mbar_init(p_empty_bar(s), UNPACK_WARPS);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(acc_full_bar(a), 1);
@@ -304,7 +338,45 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                              : p.l2_policy == 1                      ? ptx::policy_evict_first()
                                                                      : ptx::policy_evict_last();
       bool backward = false;
-      for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
+      constexpr int RING = FUSED ? PSTAGES : STAGES;  // slots of the ring this role fills
+      for (int t = first_tile; FUSED && t < num_tiles && ok; t += tile_stride) {
+        // Fused INT4: every CTA fills its own ring of packed slots and counts its own bytes;
+        // one packed slot (128 bytes = 256 values of K per row) feeds two int8 slots.
+        int tm, tn, tile, k_begin, k_end;
+        bool add;
+        decode_unit(t, tile, k_begin, k_end, add);
+        tile_coords(p, tile, tm, tn);
+        const int a_row = tm * TILE_M + static_cast<int>(cta_rank) * BM;
+        const int b_row = tn * BN + static_cast<int>(cta_rank) * L::B_ROWS;
+        const int ps_begin = k_begin / 2, ps_end = k_end / 2;
+        for (int ps = ps_begin; ps < ps_end; ++ps) {
+          const long long w0 = trace ? clock64() : 0;
+          ok = wait_bounded(p_empty_bar(stage), phase ^ 1u, abort_flag, p.status,
+                            DEV_TIMEOUT_PRODUCER);
+          const long long w9 = trace ? clock64() : 0;
+          if (trace) waited += w9 - w0;
+          if (!ok) break;
+          const uint32_t a_dst = base + L::P_OFFSET + stage * L::P_STAGE_BYTES;
+          const uint32_t b_dst = a_dst + L::A_BYTES;
+          if (!elected) {
+            // nothing to issue in this lane
+          } else if ((p.ablate & 8) && blockIdx.x == 0 && t == first_tile && ps == ps_begin + 2) {
+            // failure drill: this slot is never filled
+          } else if (p.ablate & 2) {
+            ptx::mbar_arrive(p_full_bar(stage));
+          } else {
+            const int k0 = (backward ? ps_begin + ps_end - 1 - ps : ps) * BK_BYTES;  // packed bytes
+            ptx::mbar_arrive_expect_tx(p_full_bar(stage), L::P_STAGE_BYTES);
+            ptx::tma_load_2d(a_dst, &tmap_a, k0, a_row, p_full_bar(stage), pol_a);
+            ptx::tma_load_2d(b_dst, &tmap_b, k0, b_row, p_full_bar(stage), pol_b);
+          }
+          ++issued;
+          if (trace) prod_issue += clock64() - w9;
+          if (++stage == RING) { stage = 0; phase ^= 1u; }
+        }
+        if (p.serpentine_k) backward = !backward;
+      }
+      for (int t = first_tile; !FUSED && t < num_tiles && ok; t += tile_stride) {
         int tm, tn, tile, k_begin, k_end;
         bool add;
         decode_unit(t, tile, k_begin, k_end, add);
@@ -355,13 +427,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         trace[TRACE_PROD_WAIT] = static_cast<unsigned long long>(waited);
         trace[TRACE_PROD_ISSUE] = static_cast<unsigned long long>(prod_issue);
       }
-      if (!ok && elected && (CTA_GROUP == 1 || leader)) {
+      if (!ok && elected && (FUSED || CTA_GROUP == 1 || leader)) {
         // Gave up: let the copies already in flight land before the CTA exits.
-        int n = issued < STAGES ? issued : STAGES;
+        int n = issued < RING ? issued : RING;
         for (int i = 0; i < n; ++i) {
-          if (--stage < 0) { stage = STAGES - 1; phase ^= 1u; }
+          if (--stage < 0) { stage = RING - 1; phase ^= 1u; }
           uint64_t t0 = ptx::globaltimer_ns();
-          while (!ptx::mbar_try_wait(full_bar(stage), phase) &&
+          while (!ptx::mbar_try_wait(FUSED ? p_full_bar(stage) : full_bar(stage), phase) &&
                  ptx::globaltimer_ns() - t0 < WAIT_LIMIT_NS) {
           }
         }
@@ -392,7 +464,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         decode_unit(t, tile, k_begin, k_end, add);
         for (int ks = k_begin; ks < k_end; ++ks) {
           const long long w1 = trace ? clock64() : 0;
-          ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
+          if constexpr (FUSED) {
+            ok = wait_bounded(ready_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
+            if (ok && CTA_GROUP == 2)
+              ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
+          } else {
+            ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
+          }
           const long long w2 = trace ? clock64() : 0;
           if (trace) wait_full += w2 - w1;
           if (!ok) break;
@@ -451,10 +529,111 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         while (!ptx::mbar_try_wait(drain_bar, 0) && ptx::globaltimer_ns() - t0 < WAIT_LIMIT_NS) {
         }
       }
+    } else if constexpr (FUSED && CTA_GROUP == 2) {
+      // Peer CTA, fused INT4: relay "my int8 slot is written" to the leader's `full` barrier.
+      const bool elected = ptx::elect_one();
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
+        int tile, k_begin, k_end;
+        bool add;
+        decode_unit(t, tile, k_begin, k_end, add);
+        for (int ks = k_begin; ks < k_end; ++ks) {
+          ok = wait_bounded(ready_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
+          if (!ok) break;
+          // The leader does not read this CTA's shared memory itself: the MMAs it issues make
+          // this SM's tensor core read it, after the writers' proxy fences.
+          if (elected) ptx::mbar_arrive_remote(ptx::map_to_cta(full_bar(stage), 0));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (FUSED && warp >= 2 + EPI_WARPS) {
+    // ------------------------------------------------- fused INT4: nibble expansion
+    // One packed slot holds, per operand row, 128 bytes = 8 chunks of 16 bytes (32 values of K
+    // each), chunk c stored at position c ^ (row & 7) by the 128-byte swizzle.  Chunks 0..3 feed
+    // int8 slot "h = 0", chunks 4..7 slot "h = 1".  A chunk's even-k values (low nibbles) become
+    // int8 chunk c & 3 of the row, its odd-k values chunk (c & 3) + 4, both in the same swizzle;
+    // in byte offsets inside the operand tile that is x ^ (h * 64) resp. x ^ (h * 64) ^ 64 for a
+    // chunk read at offset x.  Lane -> (row, chunk) is chosen so that each quarter-warp reads
+    // and writes all 32 banks once.
+    if constexpr (FUSED) {
+      const int uw = warp - (2 + EPI_WARPS);
+      const int c = lane & 3;
+      const int row_in_8 = (lane >> 3) + 4 * ((lane >> 2) & 1);
+      constexpr uint32_t HI = 0xF0F0F0F0u;
+      int pstage = 0, ustage = 0;
+      uint32_t pphase = 0, uphase = 0;
+      bool ok = true;
+      long long wait_in = 0, wait_out = 0, busy = 0;
+      for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
+        int tile, k_begin, k_end;
+        bool add;
+        decode_unit(t, tile, k_begin, k_end, add);
+        for (int ps = k_begin / 2; ps < k_end / 2 && ok; ++ps) {
+          const long long w0 = trace ? clock64() : 0;
+          ok = wait_bounded(p_full_bar(pstage), pphase, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
+          ok = __all_sync(0xffffffffu, ok);
+          if (trace) wait_in += clock64() - w0;
+          if (!ok) break;
+          const uint32_t src = base + L::P_OFFSET + pstage * L::P_STAGE_BYTES;
+#pragma unroll 1
+          for (int h = 0; h < 2; ++h) {
+            const long long w1 = trace ? clock64() : 0;
+            ok = wait_bounded(empty_bar(ustage), uphase ^ 1u, abort_flag, p.status,
+                              DEV_TIMEOUT_UNPACK);
+            ok = __all_sync(0xffffffffu, ok);
+            const long long w2 = trace ? clock64() : 0;
+            if (trace) wait_out += w2 - w1;
+            if (!ok) break;
+            const uint32_t dst = base + ustage * L::STAGE_BYTES;
+            const uint32_t x0 = static_cast<uint32_t>(row_in_8 * 128 + (((4 * h + c) ^ row_in_8) << 4));
+            const uint32_t flip = static_cast<uint32_t>(h) << 6;
+            // A rows first, then the B rows (the B tile follows the A tile in both rings); all
+            // loads are issued before the first store so that their latencies overlap
+            constexpr int TASKS = (BM + L::B_ROWS) / (8 * UNPACK_WARPS);
+            uint32_t wv[TASKS][4];
+#pragma unroll
+            for (int i = 0; i < TASKS; ++i)
+              ptx::ld_shared_v4(src + x0 + static_cast<uint32_t>((i * UNPACK_WARPS + uw) * 8 * 128),
+                                wv[i][0], wv[i][1], wv[i][2], wv[i][3]);
+#pragma unroll
+            for (int i = 0; i < TASKS; ++i) {
+              const uint32_t x = x0 + static_cast<uint32_t>((i * UNPACK_WARPS + uw) * 8 * 128);
+              ptx::st_shared_v4(dst + (x ^ flip), (wv[i][0] << 4) & HI, (wv[i][1] << 4) & HI,
+                                (wv[i][2] << 4) & HI, (wv[i][3] << 4) & HI);
+              ptx::st_shared_v4(dst + (x ^ flip ^ 64u), wv[i][0] & HI, wv[i][1] & HI, wv[i][2] & HI,
+                                wv[i][3] & HI);
+            }
+            // the tensor cores read shared memory through the async proxy
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ready_bar(ustage));
+            if (trace) busy += clock64() - w2;
+            if (++ustage == STAGES) { ustage = 0; uphase ^= 1u; }
+          }
+          if (!ok) break;
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(p_empty_bar(pstage));  // every lane has read its chunks
+          if (++pstage == PSTAGES) { pstage = 0; pphase ^= 1u; }
+        }
+      }
+      if (trace && uw == 0 && lane == 0) {
+        trace[TRACE_UNPACK_WAIT_IN] = static_cast<unsigned long long>(wait_in);
+        trace[TRACE_UNPACK_WAIT_OUT] = static_cast<unsigned long long>(wait_out);
+        trace[TRACE_UNPACK_BUSY] = static_cast<unsigned long long>(busy);
+      }
     }
     __syncwarp();
   } else {
     // ---------------------------------------------------------------- epilogue
+    // Fused INT4 accumulators hold 256 * C: an arithmetic shift restores C exactly.
+    auto fix = [](uint32_t bits) -> uint32_t {
+      if constexpr (FUSED) return static_cast<uint32_t>(static_cast<int32_t>(bits) >> 8);
+      return bits;
+    };
     const int quarter = warp & 3;  // TMEM lane quarter this warp may read
     const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
     const uint32_t epi_base =
@@ -501,6 +680,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           ptx::tmem_ld_32x32b_x32(
               tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), w);
           ptx::tmem_wait_ld();
+          if constexpr (FUSED) {
+#pragma unroll
+            for (int v = 0; v < 32; ++v) w[v] = fix(w[v]);
+          }
         } else if constexpr (EPI == EPI_F32_SCALED) {
           ptx::tmem_ld_32x32b_x32(
               tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), w);
@@ -508,7 +691,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 #pragma unroll
           for (int v = 0; v < 32; ++v) {
             const float cs = (col + v < p.N) ? __ldg(p.col_scale + col + v) : 0.0f;
-            w[v] = __float_as_uint(acc_to_float<KIND>(w[v]) * rs * cs);
+            w[v] = __float_as_uint(acc_to_float<KIND>(fix(w[v])) * rs * cs);
           }
         } else {
 #pragma unroll
@@ -519,7 +702,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             ptx::tmem_wait_ld();
 #pragma unroll
             for (int v = 0; v < 32; v += 2) {
-              float x0 = acc_to_float<KIND>(r[v]), x1 = acc_to_float<KIND>(r[v + 1]);
+              float x0 = acc_to_float<KIND>(fix(r[v])), x1 = acc_to_float<KIND>(fix(r[v + 1]));
               if (p.col_scale) {
                 const int cc = col + h * 32 + v;
                 x0 *= rs * ((cc < p.N) ? __ldg(p.col_scale + cc) : 0.0f);
@@ -606,7 +789,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         if constexpr (CTA_GROUP == 1) {
           ptx::mbar_arrive(acc_empty_bar(acc));
         } else {
-          ptx::mbar_arrive_cluster(ptx::map_to_cta(acc_empty_bar(acc), 0));
+          // CTA-scope release on the leader's barrier: the accumulator reads above are complete
+          // (tcgen05.wait::ld) and ordered by the tcgen05 fence; nothing else has to be made
+          // visible cluster-wide, and a cluster-scope release would stall this lane for
+          // hundreds of cycles per tile.
+          ptx::mbar_arrive_remote(ptx::map_to_cta(acc_empty_bar(acc), 0));
         }
       }
       if (trace) epi_busy += clock64() - w1;

@@ -9,11 +9,11 @@
 namespace b200gemm {
 namespace {
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI>
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI, int PSTAGES = 0>
 int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUtensorMap& tb,
                    const CUtensorMap& tc, const GemmParams& p, cudaStream_t stream) {
-  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB>;
-  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI>;
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES>;
+  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI, PSTAGES>;
   if (!(s->attr_set[variant >> 6] & (1ull << (variant & 63)))) {
     cudaError_t e =
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
@@ -26,7 +26,7 @@ int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUt
   const int grid = static_cast<int>((tiles < units ? tiles : units) * CTA_GROUP);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid, 1, 1);
-  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.blockDim = dim3(PSTAGES > 0 ? NUM_THREADS_FUSED : NUM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = L::DYN_BYTES;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -50,10 +50,19 @@ struct OutputSpec {
   bool no_split = false;    // C is a block of a larger matrix: never zero / add into it
 };
 
-// A, B already in the element type of KIND (fp16 or int8), pitches in bytes.
+// Returned (never to the caller of the library) when the fused INT4 kernel does not cover the
+// shape the selector picked: the entry point then takes the pre-pass route.
+constexpr int GEMM_NOT_FUSED = 1;
+
+// A, B in the element type of KIND (fp16 or int8), pitches in bytes.  packed_s4 (KIND_I8
+// only): A and B hold packed signed 4-bit values, K/2 bytes per row, and go to the kernel
+// variant that expands them on the way to the MMAs; that variant exists for the 256 x 256
+// CTA-pair tile without split-K, for any other choice GEMM_NOT_FUSED comes back and nothing
+// has been enqueued.
 template <int KIND, int EPI>
 int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const void* B,
-                    size_t b_pitch, void* C, const OutputSpec& out, cudaStream_t stream) {
+                    size_t b_pitch, void* C, const OutputSpec& out, cudaStream_t stream,
+                    bool packed_s4 = false) {
   std::lock_guard<std::mutex> lock(g_mutex);
   DeviceState* s = nullptr;
   int rc = device_state(&s);
@@ -62,17 +71,25 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   constexpr int C_ELEM = (EPI == EPI_OUT16) ? 2 : 4;
   const CUtensorMapDataType type =
       (KIND == ptx::KIND_F16) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
-  const int k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
+  // the selector sees the int8 problem either way, so both INT4 routes get the same tile
+  int k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
   const TileConfig cfg = select_config(M, N, s->num_sms, k_blocks, EPI == EPI_OUT16 ? 64 : 32,
                                        EPI == EPI_RAW32 && !out.no_split);
   const long long ldc = out.ldc ? out.ldc : N;
   if (cfg.bn == 0) return GEMM_ERR_INVALID_ARG;  // override asks for a shape this mode lacks
+  if (packed_s4) {
+    if (KIND != ptx::KIND_I8 || cfg.bn != 256 || cfg.cta_group != 2 || cfg.splits != 1)
+      return GEMM_NOT_FUSED;
+    k_blocks = 2 * ceil_div(K, 2 * BK_BYTES);  // one packed slot (256 values of K) = two int8 slots
+  }
 
   CUtensorMap ta, tb;
   const bool promote = !(g_l2_policy & 16);
-  rc = encode_operand_map(&ta, type, ELEM, A, M, K, a_pitch, BM, promote);
+  // packed: the tensor is K/2 bytes wide; boxes stay 128 bytes
+  const uint64_t k_cols = packed_s4 ? static_cast<uint64_t>(K) / 2 : static_cast<uint64_t>(K);
+  rc = encode_operand_map(&ta, type, ELEM, A, M, k_cols, a_pitch, BM, promote);
   if (rc != GEMM_OK) return rc;
-  rc = encode_operand_map(&tb, type, ELEM, B, N, K, b_pitch, cfg.bn / cfg.cta_group, promote);
+  rc = encode_operand_map(&tb, type, ELEM, B, N, k_cols, b_pitch, cfg.bn / cfg.cta_group, promote);
   if (rc != GEMM_OK) return rc;
 
   GemmParams p;
@@ -144,6 +161,11 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     if (e != cudaSuccess) return cuda_fail(e);
   }
   const int vbase = ((KIND == ptx::KIND_F16) ? 0 : 32) + EPI * 8;  // bit index in attr_set
+  if (packed_s4) {
+    if constexpr (KIND == ptx::KIND_I8)
+      return launch_variant<KIND, 256, 4, 2, 1, EPI, 2>(s, vbase + 7, ta, tb, tc, p, stream);
+    return GEMM_ERR_INVALID_ARG;
+  }
   if (cfg.cta_group == 2) {
     switch (cfg.bn) {
       case 256: return launch_variant<KIND, 256, 6, 2, 1, EPI>(s, vbase + 4, ta, tb, tc, p, stream);
@@ -166,16 +188,19 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
 
 template <int KIND>
 int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* B, size_t b_pitch,
-                void* C, cudaStream_t stream, const OutputSpec& out = OutputSpec()) {
+                void* C, cudaStream_t stream, const OutputSpec& out = OutputSpec(),
+                bool packed_s4 = false) {
   switch (out.epi) {
     case EPI_RAW32:
-      return launch_gemm_epi<KIND, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+      return launch_gemm_epi<KIND, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream,
+                                              packed_s4);
     case EPI_OUT16:
-      return launch_gemm_epi<KIND, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+      return launch_gemm_epi<KIND, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream,
+                                              packed_s4);
     case EPI_F32_SCALED:
       if constexpr (KIND == ptx::KIND_I8)
         return launch_gemm_epi<KIND, EPI_F32_SCALED>(M, N, K, A, a_pitch, B, b_pitch, C, out,
-                                                     stream);
+                                                     stream, packed_s4);
       return GEMM_ERR_INVALID_ARG;
     default: return GEMM_ERR_INVALID_ARG;
   }
@@ -262,6 +287,22 @@ int s4_internal_workspace(size_t need, void** ws, size_t* ws_bytes) {
   *ws = s->s4_workspace;
   *ws_bytes = s->s4_workspace_bytes;
   return GEMM_OK;
+}
+
+// INT4 GEMM by the route gemm_set_s4_scheme selected: the fused kernel if asked for and
+// applicable, else the pre-pass through the library's own workspace.
+int s4_auto(int M, int N, int K, const uint8_t* A, const uint8_t* B, void* C, const OutputSpec& out,
+            cudaStream_t st) {
+  if (g_s4_scheme == 1) {
+    const int rc = launch_gemm<ptx::KIND_I8>(M, N, K, A, static_cast<size_t>(K) / 2, B,
+                                             static_cast<size_t>(K) / 2, C, st, out, true);
+    if (rc != GEMM_NOT_FUSED) return rc;
+  }
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  int rc = s4_internal_workspace(s4_workspace_need(M, N, K), &ws, &ws_bytes);
+  if (rc != GEMM_OK) return rc;
+  return s4_with_workspace(M, N, K, A, B, C, ws, ws_bytes, out, st);
 }
 
 int check_scales(const float* row_scale, const float* col_scale, const void* C, int c_is_fp16,

@@ -39,6 +39,7 @@ int g_override_group_m = 0;
 int g_override_cta_group = 0;
 int g_override_splits = 0;
 int g_trace_on = 0;
+int g_s4_scheme = 0;   // INT4 route: 0 = pre-pass + INT8 GEMM, 1 = fused kernel where it applies
 int g_l2_policy = 11;  // keep A, B normal, serpentine K, C stores evict-first
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,

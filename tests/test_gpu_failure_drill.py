@@ -41,3 +41,34 @@ def test_expired_wait_is_reported_and_the_context_survives(cta_group):
     finally:
         binding.gemm_trace_enable(0)
         binding.gemm_set_config_override(0, 0, 0)
+
+
+def test_expired_wait_in_the_fused_int4_kernel():
+    """Same drill through the kernel variant with the extra nibble-expansion warps and the
+    second (packed) ring: a packed slot of CTA 0 is never filled."""
+    M, N, K = 256, 256, 2048                      # one tile, 8 packed slots (> ring depth 2)
+    A, B = synth.s4_uniform(M, N, K, seed=10)
+    dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    C = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    assert binding.gemm_last_device_status() == 0
+    binding.gemm_set_config_override(256, 0, 2, 1)
+    binding.gemm_set_s4_scheme(1)
+    try:
+        assert "fused_unpack" in binding.gemm_query_config("s4", M, N, K)
+        binding.gemm_trace_enable(16)
+        t0 = time.time()
+        binding.gemm_s4(dA, dB, C)
+        torch.cuda.synchronize()
+        took = time.time() - t0
+        binding.gemm_trace_enable(0)
+        status = binding.gemm_last_device_status()
+        assert status in (1, 2, 3, 5), "expected a recorded wait expiry, got %d" % status
+        assert 1.5 < took < 30.0
+        binding.gemm_s4(dA, dB, C)
+        torch.cuda.synchronize()
+        assert np.array_equal(C.cpu().numpy(), oracle.gemm_s4(A, B, K))
+        assert binding.gemm_last_device_status() == 0
+    finally:
+        binding.gemm_trace_enable(0)
+        binding.gemm_set_s4_scheme(0)
+        binding.gemm_set_config_override(0, 0, 0)
