@@ -538,10 +538,10 @@ def run_ablation(args):
                  ("epilogue: direct register -> global stores", (0, 0, 0), 11, 33)]
     # INT4: how the nibbles reach the int8 tensor-core path (the traced launch is the GEMM;
     # the pre-pass launch of route 0 is inside the timed loop but not in the cycle accounting)
-    s4_variants = [("INT4 route 0: pre-pass to int8 + INT8 GEMM (default)", (0, 0, 0), 11, 1, 0),
-                   ("INT4 route 1: nibbles expanded inside the GEMM kernel", (0, 0, 0), 11, 1, 1),
-                   ("INT4 route 1, ablate: no MMAs", (0, 0, 0), 11, 3, 1),
-                   ("INT4 route 1, ablate: no operand loads", (0, 0, 0), 11, 5, 1)]
+    s4_variants = [("INT4 route 0: pre-pass to int8 + INT8 GEMM (default at this size)", (0, 0, 0), 11, 1, 1),
+                   ("INT4 route 1: nibbles expanded inside the GEMM kernel", (0, 0, 0), 11, 1, 2),
+                   ("INT4 route 1, ablate: no MMAs", (0, 0, 0), 11, 3, 2),
+                   ("INT4 route 1, ablate: no operand loads", (0, 0, 0), 11, 5, 2)]
     for prec in ("fp16", "s8", "s4"):
         dA, dB = (torch.from_numpy(x).cuda() for x in data[prec])
         C = torch.empty((N, N), dtype=torch.float32 if prec == "fp16" else torch.int32,

@@ -270,20 +270,24 @@ int gemm_last_device_status(void);
  * Route of later gemm_s4 / gemm_s4_dequant calls.  tcgen05 has no signed 4-bit
  * integer kind (the paper's kernels feed mma.sync m16n8k64 .s4 operands
  * directly, Listing 2c), so the nibbles are expanded to int8 either
- *   0 (default): by a streaming pre-pass kernel into an int8 scratch, followed
- *     by the INT8 GEMM; or
- *   1: inside the GEMM kernel ("fused") where that variant applies, i.e. where
- *     the selector picks the 256 x 256 CTA-pair tile without split-K (large
- *     problems), else as 0.  Packed tiles are loaded as they are and eight extra
- *     warps per CTA expand them in shared memory into the slots the MMAs read:
- *     no scratch and half the operand bytes through L2 and HBM, but half as much
- *     shared-memory traffic again per unit of math, and shared-memory bandwidth
- *     is what bounds this kernel: at N = 8192 it is about 1.35x slower than
- *     route 0.  Kept as the measured alternative of the INT4 ablation.
- * gemm_s4_ws and gemm_s4_static always take route 0.  Results are identical,
- * bit for bit.  gemm_query_config shows the route.  The paper has no
- * counterpart; its Run 4 ablates how the operands reach the tensor cores, of
- * which this is the analogue here.
+ *   - by a streaming pre-pass kernel into an int8 scratch, followed by the
+ *     INT8 GEMM ("pre-pass"): each operand element is expanded once; or
+ *   - inside the GEMM kernel ("fused"): packed tiles are loaded as they are and
+ *     eight extra warps per CTA expand them in shared memory into the slots the
+ *     MMAs read.  No scratch, and a quarter of the pre-pass route's HBM bytes
+ *     for an operand that is read once; but half as much shared-memory traffic
+ *     again per unit of math, which is what bounds the large-tile kernel.
+ * Measured: at M = N = K = 8192 the pre-pass route is 1.1-1.35x faster; for
+ * M = 16, N = K = 8192 (bound by the bytes of B) the fused route is several
+ * times faster and faster than the INT8 GEMM on pre-expanded operands.
+ * scheme 0 (default, automatic): fused where the selector picks a one-CTA tile
+ * and M <= 128 or N <= 128, else the pre-pass; 1: always the pre-pass; 2: fused
+ * wherever a fused variant is built (every one-CTA tile, and the 256 x 256 CTA
+ * pair without split-K), else the pre-pass.  gemm_s4_ws and gemm_s4_static
+ * always use the pre-pass.  Results are identical, bit for bit.
+ * gemm_query_config shows the route.  The paper has no counterpart; its Run 4
+ * ablates how the operands reach the tensor cores, of which this is the
+ * analogue here.
  */
 int gemm_set_s4_scheme(int scheme);
 

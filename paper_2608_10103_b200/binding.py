@@ -302,9 +302,9 @@ def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0, 
 
 
 def gemm_set_s4_scheme(scheme: int = 0):
-    """Route of gemm_s4 / gemm_s4_dequant: 0 = pre-pass to int8 + INT8 GEMM (default); 1 =
-    nibbles expanded inside the GEMM kernel where that variant applies (256 x 256 CTA-pair
-    tile, no split-K), else the pre-pass."""
+    """Route of gemm_s4 / gemm_s4_dequant: 0 = automatic (nibbles expanded inside the GEMM
+    kernel for problems with few rows on one side, else a pre-pass to int8 + the INT8 GEMM);
+    1 = always the pre-pass; 2 = inside the GEMM kernel wherever such a variant is built."""
     _check(lib().gemm_set_s4_scheme(int(scheme)), "gemm_set_s4_scheme")
 
 

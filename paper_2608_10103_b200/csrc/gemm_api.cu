@@ -168,8 +168,15 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
       num_sms = g_dev[dev].num_sms;
   }
   const int elem = precision == GEMM_PREC_FP16 ? 2 : 1;
-  const TileConfig c =
-      select_config(M, N, num_sms, ceil_div(static_cast<long long>(K) * elem, BK_BYTES), 32, true);
+  const int kb = ceil_div(static_cast<long long>(K) * elem, BK_BYTES);
+  TileConfig c;
+  bool fused = false;
+  if (precision == GEMM_PREC_S4 && g_s4_scheme != 1) {  // the decision of s4_auto / launch_gemm_epi
+    c = select_config(M, N, num_sms, kb, 32, true, 2);
+    fused = c.bn != 0 && fused_s4_variant_exists(c.bn, c.cta_group, c.splits) &&
+            s4_fused_wanted(M, N, c);
+  }
+  if (!fused) c = select_config(M, N, num_sms, kb, 32, true);
   if (c.bn == 0) return GEMM_ERR_INVALID_ARG;
   const long long tiles =
       static_cast<long long>(ceil_div(M, BM * c.cta_group)) * ceil_div(N, c.bn);
@@ -185,10 +192,7 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
                 : units) *
                c.cta_group,
            precision == GEMM_PREC_FP16 ? "f16" : "i8",
-           precision != GEMM_PREC_S4 ? ""
-           : (g_s4_scheme == 1 && c.bn == 256 && c.cta_group == 2 && c.splits == 1)
-               ? " s4=fused_unpack(4+2 slots)"
-               : " prepass=unpack_s4");
+           precision != GEMM_PREC_S4 ? "" : fused ? " s4=fused_unpack" : " prepass=unpack_s4");
   return GEMM_OK;
 }
 
@@ -230,7 +234,7 @@ int gemm_last_device_status(void) {
 }
 
 int gemm_set_s4_scheme(int scheme) {
-  if (scheme < 0 || scheme > 1) return GEMM_ERR_INVALID_ARG;
+  if (scheme < 0 || scheme > 2) return GEMM_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
   g_s4_scheme = scheme;
   return GEMM_OK;

@@ -29,7 +29,7 @@
 //
 // PSTAGES > 0 (fused INT4): A and B hold packed signed 4-bit values (Listing 2c's s4
 //   operands).  The producer lands PACKED tiles (rows x 128 bytes = 256 nibbles of K) in a
-//   second ring of PSTAGES slots; warps 6..9 expand each packed slot into two int8 slots of
+//   second ring of PSTAGES slots; warps 6..13 expand each packed slot into two int8 slots of
 //   the ring the MMA issuer reads, every value multiplied by 16 (nibble moved to the high
 //   half of its byte, low half zero), so the accumulators hold 256 * C and the epilogue
 //   shifts them right by 8, exactly.  The order in which K values land in the int8 slots
@@ -260,7 +260,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   const int split_tiles = real_tiles - p.split_from;
   const int num_tiles = p.split_from + split_tiles * p.splits;
   const int k_slots_all = (p.k_blocks + KB - 1) / KB;  // ring slots per tile; a K tail is zero-filled
-  const int k_per_split = (k_slots_all + p.splits - 1) / p.splits;
+  // (fused INT4: K is split in whole packed slots = pairs of int8 slots)
+  const int k_per_split = FUSED ? 2 * ((k_slots_all / 2 + p.splits - 1) / p.splits)
+                                : (k_slots_all + p.splits - 1) / p.splits;
   // unit -> tile, K range (in ring slots) and whether its result is added into C
   auto decode_unit = [&](int u, int& tile, int& k_begin, int& k_end, bool& add) {
     if (u < p.split_from) {
@@ -569,9 +571,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       bool ok = true;
       long long wait_in = 0, wait_out = 0, busy = 0;
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
-        int tile, k_begin, k_end;
+        int tm, tn, tile, k_begin, k_end;
         bool add;
         decode_unit(t, tile, k_begin, k_end, add);
+        tile_coords(p, tile, tm, tn);
+        // Rows of the tile beyond M resp. N are not expanded: the accumulator rows and columns
+        // they feed are never stored, so whatever the int8 slot holds there does no harm, and a
+        // problem with few rows (M = 16) skips most of the A tile.
+        const int a_valid = p.M - (tm * TILE_M + static_cast<int>(cta_rank) * BM);
+        const int b_valid = p.N - (tn * BN + static_cast<int>(cta_rank) * L::B_ROWS);
+        constexpr int TASKS = (BM + L::B_ROWS + 8 * UNPACK_WARPS - 1) / (8 * UNPACK_WARPS);
+        bool active[TASKS];
+#pragma unroll
+        for (int i = 0; i < TASKS; ++i) {
+          const int row8 = (i * UNPACK_WARPS + uw) * 8;  // first row of this lane's group of 8
+          active[i] = row8 < BM ? row8 < a_valid : (row8 < BM + L::B_ROWS && row8 - BM < b_valid);
+        }
         for (int ps = k_begin / 2; ps < k_end / 2 && ok; ++ps) {
           const long long w0 = trace ? clock64() : 0;
           ok = wait_bounded(p_full_bar(pstage), pphase, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
@@ -593,14 +608,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             const uint32_t flip = static_cast<uint32_t>(h) << 6;
             // A rows first, then the B rows (the B tile follows the A tile in both rings); all
             // loads are issued before the first store so that their latencies overlap
-            constexpr int TASKS = (BM + L::B_ROWS) / (8 * UNPACK_WARPS);
             uint32_t wv[TASKS][4];
 #pragma unroll
             for (int i = 0; i < TASKS; ++i)
-              ptx::ld_shared_v4(src + x0 + static_cast<uint32_t>((i * UNPACK_WARPS + uw) * 8 * 128),
-                                wv[i][0], wv[i][1], wv[i][2], wv[i][3]);
+              if (active[i])
+                ptx::ld_shared_v4(src + x0 + static_cast<uint32_t>((i * UNPACK_WARPS + uw) * 8 * 128),
+                                  wv[i][0], wv[i][1], wv[i][2], wv[i][3]);
 #pragma unroll
             for (int i = 0; i < TASKS; ++i) {
+              if (!active[i]) continue;
               const uint32_t x = x0 + static_cast<uint32_t>((i * UNPACK_WARPS + uw) * 8 * 128);
               ptx::st_shared_v4(dst + (x ^ flip), (wv[i][0] << 4) & HI, (wv[i][1] << 4) & HI,
                                 (wv[i][2] << 4) & HI, (wv[i][3] << 4) & HI);

@@ -50,6 +50,16 @@ struct OutputSpec {
   bool no_split = false;    // C is a block of a larger matrix: never zero / add into it
 };
 
+// Whether the packed route is taken for the tile the selector picked.  Scheme 2 forces it
+// wherever a variant exists; scheme 0 (automatic) takes it where the operands cannot be
+// re-used enough to pay for a pre-pass over them: problems with few rows on one side
+// (LLM decoding), which are bound by the bytes of the other operand.
+bool s4_fused_wanted(int M, int N, const TileConfig& cfg) {
+  if (g_s4_scheme == 2) return true;
+  if (g_s4_scheme == 1) return false;
+  return cfg.cta_group == 1 && (M <= 128 || N <= 128);
+}
+
 // Returned (never to the caller of the library) when the fused INT4 kernel does not cover the
 // shape the selector picked: the entry point then takes the pre-pass route.
 constexpr int GEMM_NOT_FUSED = 1;
@@ -74,11 +84,12 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   // the selector sees the int8 problem either way, so both INT4 routes get the same tile
   int k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
   const TileConfig cfg = select_config(M, N, s->num_sms, k_blocks, EPI == EPI_OUT16 ? 64 : 32,
-                                       EPI == EPI_RAW32 && !out.no_split);
+                                       EPI == EPI_RAW32 && !out.no_split, packed_s4 ? 2 : 0);
   const long long ldc = out.ldc ? out.ldc : N;
   if (cfg.bn == 0) return GEMM_ERR_INVALID_ARG;  // override asks for a shape this mode lacks
   if (packed_s4) {
-    if (KIND != ptx::KIND_I8 || cfg.bn != 256 || cfg.cta_group != 2 || cfg.splits != 1)
+    if (KIND != ptx::KIND_I8 || !fused_s4_variant_exists(cfg.bn, cfg.cta_group, cfg.splits) ||
+        !s4_fused_wanted(M, N, cfg))
       return GEMM_NOT_FUSED;
     k_blocks = 2 * ceil_div(K, 2 * BK_BYTES);  // one packed slot (256 values of K) = two int8 slots
   }
@@ -162,8 +173,23 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   }
   const int vbase = ((KIND == ptx::KIND_F16) ? 0 : 32) + EPI * 8;  // bit index in attr_set
   if (packed_s4) {
-    if constexpr (KIND == ptx::KIND_I8)
-      return launch_variant<KIND, 256, 4, 2, 1, EPI, 2>(s, vbase + 7, ta, tb, tc, p, stream);
+    // fused INT4 variants: (int8 slots, packed slots) sized to fill shared memory; attr_set
+    // bits 64.. (one per tile shape and output mode)
+    if constexpr (KIND == ptx::KIND_I8) {
+      const int fb = 64 + EPI * 8;
+      if (cfg.cta_group == 2)
+        return launch_variant<KIND, 256, 4, 2, 1, EPI, 2>(s, fb + 0, ta, tb, tc, p, stream);
+      switch (cfg.bn) {
+        case 256: return launch_variant<KIND, 256, 2, 1, 1, EPI, 2>(s, fb + 1, ta, tb, tc, p, stream);
+        case 128: return launch_variant<KIND, 128, 3, 1, 1, EPI, 3>(s, fb + 2, ta, tb, tc, p, stream);
+        case 64: return launch_variant<KIND, 64, 3, 1, 1, EPI, 4>(s, fb + 3, ta, tb, tc, p, stream);
+        case 32:
+          if constexpr (EPI != EPI_OUT16)
+            return launch_variant<KIND, 32, 3, 1, 1, EPI, 5>(s, fb + 4, ta, tb, tc, p, stream);
+          return GEMM_ERR_INVALID_ARG;
+        default: return GEMM_ERR_INVALID_ARG;
+      }
+    }
     return GEMM_ERR_INVALID_ARG;
   }
   if (cfg.cta_group == 2) {
@@ -293,7 +319,7 @@ int s4_internal_workspace(size_t need, void** ws, size_t* ws_bytes) {
 // applicable, else the pre-pass through the library's own workspace.
 int s4_auto(int M, int N, int K, const uint8_t* A, const uint8_t* B, void* C, const OutputSpec& out,
             cudaStream_t st) {
-  if (g_s4_scheme == 1) {
+  if (g_s4_scheme != 1) {
     const int rc = launch_gemm<ptx::KIND_I8>(M, N, K, A, static_cast<size_t>(K) / 2, B,
                                              static_cast<size_t>(K) / 2, C, st, out, true);
     if (rc != GEMM_NOT_FUSED) return rc;

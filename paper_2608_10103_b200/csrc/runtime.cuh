@@ -28,7 +28,7 @@ struct DeviceState {
   unsigned long long* trace_ptr = nullptr;
   void* s4_workspace = nullptr;
   size_t s4_workspace_bytes = 0;
-  uint64_t attr_set[2] = {0, 0};  // bit i: dynamic-smem attribute set for kernel variant i
+  uint64_t attr_set[3] = {0, 0, 0};  // bit i: dynamic-smem attribute set for kernel variant i
 };
 
 std::mutex g_mutex;
@@ -39,7 +39,7 @@ int g_override_group_m = 0;
 int g_override_cta_group = 0;
 int g_override_splits = 0;
 int g_trace_on = 0;
-int g_s4_scheme = 0;   // INT4 route: 0 = pre-pass + INT8 GEMM, 1 = fused kernel where it applies
+int g_s4_scheme = 0;   // INT4 route: 0 = automatic, 1 = always the pre-pass, 2 = fused wherever built
 int g_l2_policy = 11;  // keep A, B normal, serpentine K, C stores evict-first
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,

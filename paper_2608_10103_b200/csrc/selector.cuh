@@ -39,6 +39,12 @@ bool variant_exists(int bn, int cta_group) {
   return false;
 }
 
+// Kernel variants that take packed INT4 operands and expand them on the way to the MMAs.
+bool fused_s4_variant_exists(int bn, int cta_group, int splits) {
+  if (cta_group == 2) return bn == 256 && splits == 1;
+  return bn == 256 || bn == 128 || bn == 64 || bn == 32;
+}
+
 int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b); }
 
 // Picks the C-tile shape and the split-K factor.  The paper fixes one tiling for all
@@ -51,8 +57,10 @@ int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b
 // ((128 + bn/cta_group) rows x 128 bytes at ~66 bytes/cycle); units run in waves over the SMs
 // (or SM pairs); the last epilogue (~16 cycles per column), set-up (~3000) and a pair's
 // cluster launch (~2500) are paid once; split-K adds zeroing C and adding into it.
+// force_atoms: K atoms per split unit whatever the tile (the fused INT4 kernel splits K in
+// packed slots = 2 int8 k-blocks); 0 = the tile's own ring slot.
 TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 32,
-                         bool allow_split = false) {
+                         bool allow_split = false, int force_atoms = 0) {
   TileConfig best{256, 2, 6, 8, 1, 0};
   long long best_cost = -1;
   for (int cg = 2; cg >= 1; --cg) {
@@ -62,7 +70,7 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
       if (!variant_exists(bn, cg) || bn < min_bn) continue;
       const long long tiles = static_cast<long long>(ceil_div(M, BM * cg)) * ceil_div(N, bn);
       const long long units = num_sms / cg;
-      const int atoms = atoms_for(bn, cg);
+      const int atoms = force_atoms ? force_atoms : atoms_for(bn, cg);
       const int slots = ceil_div(k_blocks, atoms);  // K is split in whole ring slots
       int max_split = 1;
       if (allow_split) {
@@ -110,7 +118,8 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
     const long long tiles =
         static_cast<long long>(ceil_div(M, BM * best.cta_group)) * ceil_div(N, best.bn);
     const long long units = num_sms / best.cta_group;
-    const int slots = ceil_div(k_blocks, atoms_for(best.bn, best.cta_group));
+    const int slots =
+        ceil_div(k_blocks, force_atoms ? force_atoms : atoms_for(best.bn, best.cta_group));
     best.split_tiles = best.splits > 1 ? static_cast<int>(tiles) : 0;
     const long long r = tiles % units;
     if (allow_split && best.splits == 1 && g_override_splits == 0 && tiles > units && r > 0 &&

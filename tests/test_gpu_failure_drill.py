@@ -52,7 +52,7 @@ def test_expired_wait_in_the_fused_int4_kernel():
     C = torch.zeros((M, N), dtype=torch.int32, device="cuda")
     assert binding.gemm_last_device_status() == 0
     binding.gemm_set_config_override(256, 0, 2, 1)
-    binding.gemm_set_s4_scheme(1)
+    binding.gemm_set_s4_scheme(2)
     try:
         assert "fused_unpack" in binding.gemm_query_config("s4", M, N, K)
         binding.gemm_trace_enable(16)

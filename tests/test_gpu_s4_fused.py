@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 @pytest.fixture(autouse=True)
 def _fused_route():
     binding.gemm_set_config_override(0, 0, 0, 0)
-    binding.gemm_set_s4_scheme(1)
+    binding.gemm_set_s4_scheme(2)
     yield
     binding.gemm_set_s4_scheme(0)
     binding.gemm_set_config_override(0, 0, 0, 0)
@@ -49,10 +49,40 @@ def test_fused_is_what_the_selector_reports_and_runs_at_2048():
 
 
 def test_fused_falls_back_where_the_variant_does_not_apply():
-    M, N, K = 64, 512, 4096          # the selector takes a narrow tile with split-K here
+    M, N, K = 640, 512, 1056
+    binding.gemm_set_config_override(128, 0, 2, 1)      # no fused variant for this pair tile
     cfg = binding.gemm_query_config("s4", M, N, K)
     assert "prepass" in cfg and "fused" not in cfg
     A, B = synth.s4_uniform(M, N, K, seed=6)
+    check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), force_full=True)
+
+
+@pytest.mark.parametrize("split_k", [1, 3])
+@pytest.mark.parametrize("bn", [256, 128, 64, 32])
+@pytest.mark.parametrize("M,N,K", [(16, 520, 1056), (130, 300, 2048), (1, 64, 96), (400, 700, 512)])
+def test_fused_one_cta_tiles_with_split_k(M, N, K, bn, split_k):
+    """Every one-CTA fused variant, with K split over several CTAs (each partial holds a
+    multiple of 256 and is shifted before it is added into C) and with tiles whose rows beyond
+    M or N are not expanded at all."""
+    binding.gemm_set_config_override(bn, 0, 1, split_k)
+    cfg = binding.gemm_query_config("s4", M, N, K)
+    assert "fused_unpack" in cfg and ("BN=%d " % bn) in cfg
+    A, B = synth.s4_uniform(M, N, K, seed=bn + split_k)
+    for rep in range(2):
+        check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), force_full=True)
+
+
+def test_automatic_route_by_shape():
+    binding.gemm_set_s4_scheme(0)
+    assert "fused_unpack" in binding.gemm_query_config("s4", 16, 8192, 8192)
+    assert "fused_unpack" in binding.gemm_query_config("s4", 8192, 64, 4096)
+    assert "prepass" in binding.gemm_query_config("s4", 8192, 8192, 8192)
+    assert "prepass" in binding.gemm_query_config("s4", 2048, 2048, 2048)
+    binding.gemm_set_s4_scheme(1)
+    assert "prepass" in binding.gemm_query_config("s4", 16, 8192, 8192)
+    binding.gemm_set_s4_scheme(0)
+    M, N, K = 16, 4096, 8192
+    A, B = synth.s4_uniform(M, N, K, seed=11)
     check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), force_full=True)
 
 
