@@ -292,6 +292,22 @@ int gemm_last_device_status(void);
 int gemm_set_s4_scheme(int scheme);
 
 /*
+ * Whether later calls run the kernel on exchanged operands: its 128-row tile
+ * side then holds rows of B (the caller's N), its narrow side rows of A, and C
+ * is written by plain stores that are contiguous along N.  For problems with
+ * few rows (M = 1..64, LLM decoding) this keeps 128 - M rows of zero fill out
+ * of shared memory, of the ring depth and -- on the fused INT4 route -- of the
+ * expansion work.  mode 0 (default, automatic): on the fused INT4 route when
+ * M <= 64 and N >= 512; 1: never; 2: always (any shape and precision; for tests
+ * and measurements).  Results: integers identical; FP16 within the bound;
+ * dequantised outputs multiply the two scales in the other order (last-bit
+ * differences).  gemm_query_config shows "swap_ab" and then describes the tile
+ * in the kernel's orientation.  The paper has no counterpart (square sizes
+ * only, Sec. VI).
+ */
+int gemm_set_swap_ab(int mode);
+
+/*
  * L2 behaviour of later calls, a bit set (the paper's Run 4 ablates the
  * analogous .ca / .cg cache policy of cp.async).  Bits 0-1, eviction priority
  * of the operand loads: 0 = normal for A and B; 1 = A "evict last" (kept), B

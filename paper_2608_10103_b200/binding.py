@@ -23,7 +23,7 @@ EXPORTS = (
     "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
     "gemm_fp16_f16out", "gemm_s8_dequant", "gemm_s4_dequant", "gemm_host", "gemm_host_release",
     "gemm_s4_static", "gemm_s4_static_capacity", "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
-    "gemm_set_config_override", "gemm_set_s4_scheme", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_last_device_status", "gemm_last_cuda_error",
+    "gemm_set_config_override", "gemm_set_s4_scheme", "gemm_set_swap_ab", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_last_device_status", "gemm_last_cuda_error",
     "gemm_status_string", "gemm_version",
 )
 
@@ -72,6 +72,7 @@ def lib() -> ctypes.CDLL:
         L.gemm_query_config.argtypes = [i, i, i, i, ctypes.c_char_p, i]
         L.gemm_set_config_override.argtypes = [i, i, i, i]
         L.gemm_set_s4_scheme.argtypes = [i]
+        L.gemm_set_swap_ab.argtypes = [i]
         L.gemm_set_l2_policy.argtypes = [i]
         L.gemm_trace_enable.argtypes = [i]
         L.gemm_trace_read.argtypes = [ctypes.POINTER(ctypes.c_ulonglong), i]
@@ -306,6 +307,12 @@ def gemm_set_s4_scheme(scheme: int = 0):
     kernel for problems with few rows on one side, else a pre-pass to int8 + the INT8 GEMM);
     1 = always the pre-pass; 2 = inside the GEMM kernel wherever such a variant is built."""
     _check(lib().gemm_set_s4_scheme(int(scheme)), "gemm_set_s4_scheme")
+
+
+def gemm_set_swap_ab(mode: int = 0):
+    """Run the kernel on exchanged operands (long operand on the 128-row tile side, C stored
+    along N by plain stores): 0 = automatic (fused INT4 route, M <= 64), 1 = never, 2 = always."""
+    _check(lib().gemm_set_swap_ab(int(mode)), "gemm_set_swap_ab")
 
 
 def gemm_set_l2_policy(policy: int = 11):

@@ -170,20 +170,30 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
   const int elem = precision == GEMM_PREC_FP16 ? 2 : 1;
   const int kb = ceil_div(static_cast<long long>(K) * elem, BK_BYTES);
   TileConfig c;
-  bool fused = false;
-  if (precision == GEMM_PREC_S4 && g_s4_scheme != 1) {  // the decision of s4_auto / launch_gemm_epi
-    c = select_config(M, N, num_sms, kb, 32, true, 2);
+  bool fused = false, swap = false;
+  const int user_m = M, user_n = N;
+  if (precision == GEMM_PREC_S4 && g_s4_scheme != 1) {  // the decisions of s4_auto / launch_gemm_epi
+    swap = swap_ab_wanted(M, N, true, OutputSpec());
+    c = swap ? select_config(N, M, num_sms, kb, 32, true, 2)
+             : select_config(M, N, num_sms, kb, 32, true, 2);
     fused = c.bn != 0 && fused_s4_variant_exists(c.bn, c.cta_group, c.splits) &&
-            s4_fused_wanted(M, N, c);
+            s4_fused_wanted(user_m, user_n, c);
   }
-  if (!fused) c = select_config(M, N, num_sms, kb, 32, true);
+  if (!fused) {
+    swap = swap_ab_wanted(M, N, false, OutputSpec());
+    c = swap ? select_config(N, M, num_sms, kb, 32, true) : select_config(M, N, num_sms, kb, 32, true);
+  }
   if (c.bn == 0) return GEMM_ERR_INVALID_ARG;
+  if (swap) {  // the tile counts below are the kernel's
+    M = user_n;
+    N = user_m;
+  }
   const long long tiles =
       static_cast<long long>(ceil_div(M, BM * c.cta_group)) * ceil_div(N, c.bn);
   const long long units = num_sms / c.cta_group;
   snprintf(buf, static_cast<size_t>(len),
            "BM=%d BN=%d BK=%d cta_group=%d stages=%d group_m=%d split_k=%d split_tiles=%d "
-           "tiles=%lld ctas=%lld kind=%s%s",
+           "tiles=%lld ctas=%lld kind=%s%s%s",
            BM * c.cta_group, c.bn, atoms_for(c.bn, c.cta_group) * BK_BYTES / elem, c.cta_group,
            c.stages, c.group_m, c.splits, c.splits > 1 ? c.split_tiles : 0, tiles,
            (tiles + (c.splits > 1 ? static_cast<long long>(c.split_tiles) * (c.splits - 1) : 0) <
@@ -192,7 +202,8 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
                 : units) *
                c.cta_group,
            precision == GEMM_PREC_FP16 ? "f16" : "i8",
-           precision != GEMM_PREC_S4 ? "" : fused ? " s4=fused_unpack" : " prepass=unpack_s4");
+           precision != GEMM_PREC_S4 ? "" : fused ? " s4=fused_unpack" : " prepass=unpack_s4",
+           swap ? " swap_ab" : "");
   return GEMM_OK;
 }
 
@@ -237,6 +248,13 @@ int gemm_set_s4_scheme(int scheme) {
   if (scheme < 0 || scheme > 2) return GEMM_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
   g_s4_scheme = scheme;
+  return GEMM_OK;
+}
+
+int gemm_set_swap_ab(int mode) {
+  if (mode < 0 || mode > 2) return GEMM_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  g_swap_ab = mode;
   return GEMM_OK;
 }
 

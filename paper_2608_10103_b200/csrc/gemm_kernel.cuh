@@ -92,6 +92,12 @@ struct GemmParams {
                          // the epilogue then stages C in shared memory and stores it by TMA
   uint32_t* C;           // element size 4 bytes, or 2 with EPI_OUT16
   long long ldc;         // row pitch of C in elements (N for a dense C)
+  // 1: the caller's A and B have changed places (the kernel's rows are the caller's columns), so
+  // element (row, col) of the kernel's result belongs at C[col * ldc + row].  Used for problems
+  // with few rows: the long operand then fills the 128-row side of the tile, and a warp's 32
+  // lanes (32 consecutive kernel rows) store 32 consecutive elements of a row of C.  Always
+  // with c_vec_ok = 0 (plain stores).
+  int transpose_c;
   const float* row_scale;  // EPI_OUT16 (integer kinds) / EPI_F32_SCALED: M per-row factors
   const float* col_scale;  // and N per-column factors; both null = no scaling (FP16 kind)
   int* status;           // device status word (0 = ok)
@@ -219,7 +225,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
   using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES>;
   constexpr bool FUSED = PSTAGES > 0;  // packed INT4 operands, expanded on the way to the MMAs
-  static_assert(!FUSED || (KIND == ptx::KIND_I8 && KB == 1), "fused INT4: int8 MMAs, one atom per slot");
+  static_assert(!FUSED || (KIND == ptx::KIND_I8 && KB == 1 && STAGES >= 2),
+                "fused INT4: int8 MMAs, one atom per slot, a packed slot fills two int8 slots at once");
   constexpr int ELEM_BYTES = (KIND == ptx::KIND_F16) ? 2 : 1;
   constexpr int BK_ELEMS = BK_BYTES / ELEM_BYTES;
   constexpr int TILE_M = BM * CTA_GROUP;
@@ -594,16 +601,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           if (trace) wait_in += clock64() - w0;
           if (!ok) break;
           const uint32_t src = base + L::P_OFFSET + pstage * L::P_STAGE_BYTES;
-#pragma unroll 1
+          // Both int8 slots this packed slot feeds are taken at once, so that one proxy fence
+          // (a few hundred cycles per warp) covers both.
+          const int u0 = ustage, u1 = (ustage + 1 == STAGES) ? 0 : ustage + 1;
+          const uint32_t ph0 = uphase, ph1 = (ustage + 1 == STAGES) ? (uphase ^ 1u) : uphase;
+          const long long w1 = trace ? clock64() : 0;
+          ok = wait_bounded(empty_bar(u0), ph0 ^ 1u, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
+          if (ok) ok = wait_bounded(empty_bar(u1), ph1 ^ 1u, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
+          ok = __all_sync(0xffffffffu, ok);
+          const long long w2 = trace ? clock64() : 0;
+          if (trace) wait_out += w2 - w1;
+          if (!ok) break;
+#pragma unroll
           for (int h = 0; h < 2; ++h) {
-            const long long w1 = trace ? clock64() : 0;
-            ok = wait_bounded(empty_bar(ustage), uphase ^ 1u, abort_flag, p.status,
-                              DEV_TIMEOUT_UNPACK);
-            ok = __all_sync(0xffffffffu, ok);
-            const long long w2 = trace ? clock64() : 0;
-            if (trace) wait_out += w2 - w1;
-            if (!ok) break;
-            const uint32_t dst = base + ustage * L::STAGE_BYTES;
+            const uint32_t dst = base + (h ? u1 : u0) * L::STAGE_BYTES;
             const uint32_t x0 = static_cast<uint32_t>(row_in_8 * 128 + (((4 * h + c) ^ row_in_8) << 4));
             const uint32_t flip = static_cast<uint32_t>(h) << 6;
             // A rows first, then the B rows (the B tile follows the A tile in both rings); all
@@ -623,13 +634,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
               ptx::st_shared_v4(dst + (x ^ flip ^ 64u), wv[i][0] & HI, wv[i][1] & HI, wv[i][2] & HI,
                                 wv[i][3] & HI);
             }
-            // the tensor cores read shared memory through the async proxy
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ready_bar(ustage));
-            if (trace) busy += clock64() - w2;
-            if (++ustage == STAGES) { ustage = 0; uphase ^= 1u; }
           }
+          // the tensor cores read shared memory through the async proxy
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            ptx::mbar_arrive(ready_bar(u0));
+            ptx::mbar_arrive(ready_bar(u1));
+          }
+          if (trace) busy += clock64() - w2;
+          ustage += 2;
+          if (ustage >= STAGES) { ustage -= STAGES; uphase ^= 1u; }
           if (!ok) break;
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(p_empty_bar(pstage));  // every lane has read its chunks
@@ -773,27 +788,30 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           }
         } else if (row < p.M && !empty_range) {
           // C rows are not 16-byte multiples: plain predicated stores.
+          // element (row, col + v) sits at row * rstep + (col + v) * cstep
+          const size_t rstep = p.transpose_c ? 1 : static_cast<size_t>(p.ldc);
+          const size_t cstep = p.transpose_c ? static_cast<size_t>(p.ldc) : 1;
           if constexpr (EPI == EPI_OUT16) {
-            uint16_t* crow = reinterpret_cast<uint16_t*>(p.C) + static_cast<size_t>(row) * p.ldc;
+            uint16_t* crow = reinterpret_cast<uint16_t*>(p.C) + static_cast<size_t>(row) * rstep;
 #pragma unroll
             for (int v = 0; v < 64; ++v)
               if (col + v < p.N)
-                crow[col + v] = static_cast<uint16_t>(w[v / 2] >> (16 * (v & 1)));
+                crow[(col + v) * cstep] = static_cast<uint16_t>(w[v / 2] >> (16 * (v & 1)));
           } else {
-            uint32_t* crow = p.C + static_cast<size_t>(row) * p.ldc;
+            uint32_t* crow = p.C + static_cast<size_t>(row) * rstep;
             if (EPI == EPI_RAW32 && add) {
 #pragma unroll
               for (int v = 0; v < 32; ++v) {
                 if (col + v >= p.N) continue;
                 if constexpr (KIND == ptx::KIND_F16)
-                  atomicAdd(reinterpret_cast<float*>(crow + col + v), __uint_as_float(w[v]));
+                  atomicAdd(reinterpret_cast<float*>(crow + (col + v) * cstep), __uint_as_float(w[v]));
                 else
-                  atomicAdd(reinterpret_cast<int*>(crow + col + v), static_cast<int>(w[v]));
+                  atomicAdd(reinterpret_cast<int*>(crow + (col + v) * cstep), static_cast<int>(w[v]));
               }
             } else {
 #pragma unroll
               for (int v = 0; v < 32; ++v)
-                if (col + v < p.N) crow[col + v] = w[v];
+                if (col + v < p.N) crow[(col + v) * cstep] = w[v];
             }
           }
         }

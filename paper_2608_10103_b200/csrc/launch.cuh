@@ -2,6 +2,8 @@
 // shared by the entry points, the INT4 pre-pass and its workspaces.
 #pragma once
 
+#include <utility>
+
 #include "runtime.cuh"
 #include "selector.cuh"
 #include "unpack_s4.cuh"
@@ -60,6 +62,18 @@ bool s4_fused_wanted(int M, int N, const TileConfig& cfg) {
   return cfg.cta_group == 1 && (M <= 128 || N <= 128);
 }
 
+// Whether the kernel runs on exchanged operands (its rows = the caller's N side).  The 128-row
+// side of a tile is then filled by the long operand of a problem with few rows (LLM decoding:
+// M = 1..64), instead of 128 - M rows of zero fill taking shared memory, ring depth and, on
+// the fused INT4 route, expansion work; C goes out by plain stores that are contiguous along
+// the caller's N.  Automatic: on the fused INT4 route only, where it was measured to pay.
+bool swap_ab_wanted(int M, int N, bool packed_s4, const OutputSpec& out) {
+  if (out.no_split || out.ldc) return false;  // C is a block of a larger matrix
+  if (g_swap_ab == 1) return false;
+  if (g_swap_ab == 2) return true;
+  return packed_s4 && M <= 64 && N >= 512;
+}
+
 // Returned (never to the caller of the library) when the fused INT4 kernel does not cover the
 // shape the selector picked: the entry point then takes the pre-pass route.
 constexpr int GEMM_NOT_FUSED = 1;
@@ -79,17 +93,24 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   if (rc != GEMM_OK) return rc;
   constexpr int ELEM = (KIND == ptx::KIND_F16) ? 2 : 1;
   constexpr int C_ELEM = (EPI == EPI_OUT16) ? 2 : 4;
+  const long long ldc = out.ldc ? out.ldc : N;
+  const int user_m = M, user_n = N;
+  const bool swap = swap_ab_wanted(M, N, packed_s4, out);
+  if (swap) {  // from here on M, N, A, B are the kernel's
+    std::swap(M, N);
+    std::swap(A, B);
+    std::swap(a_pitch, b_pitch);
+  }
   const CUtensorMapDataType type =
       (KIND == ptx::KIND_F16) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
   // the selector sees the int8 problem either way, so both INT4 routes get the same tile
   int k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
   const TileConfig cfg = select_config(M, N, s->num_sms, k_blocks, EPI == EPI_OUT16 ? 64 : 32,
                                        EPI == EPI_RAW32 && !out.no_split, packed_s4 ? 2 : 0);
-  const long long ldc = out.ldc ? out.ldc : N;
   if (cfg.bn == 0) return GEMM_ERR_INVALID_ARG;  // override asks for a shape this mode lacks
   if (packed_s4) {
     if (KIND != ptx::KIND_I8 || !fused_s4_variant_exists(cfg.bn, cfg.cta_group, cfg.splits) ||
-        !s4_fused_wanted(M, N, cfg))
+        !s4_fused_wanted(user_m, user_n, cfg))
       return GEMM_NOT_FUSED;
     k_blocks = 2 * ceil_div(K, 2 * BK_BYTES);  // one packed slot (256 values of K) = two int8 slots
   }
@@ -114,7 +135,8 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.splits = cfg.splits;
   p.split_from = p.tiles_m * p.tiles_n - (cfg.splits > 1 ? cfg.split_tiles : 0);
   p.ldc = ldc;
-  p.c_vec_ok = (ldc % (16 / C_ELEM) == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+  p.transpose_c = swap ? 1 : 0;
+  p.c_vec_ok = !swap && (ldc % (16 / C_ELEM) == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
   CUtensorMap tc;
   if (p.c_vec_ok) {
     // split-K adds into C by TMA reduction, which takes the element type from the map
@@ -127,8 +149,8 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     tc = ta;  // unused by the kernel on the plain-store path
   }
   p.C = static_cast<uint32_t*>(C);
-  p.row_scale = out.row_scale;
-  p.col_scale = out.col_scale;
+  p.row_scale = swap ? out.col_scale : out.row_scale;  // indexed by the kernel's rows
+  p.col_scale = swap ? out.row_scale : out.col_scale;
   p.status = s->status_ptr;
   p.trace = (g_trace_on & 1) ? s->trace_ptr : nullptr;
   p.ablate = (g_trace_on >> 1) & 31;
@@ -140,7 +162,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     // Split tiles add into C: zero them first.  All tiles: one memset.  The last wave only:
     // the bounding rectangle of those tiles (other tiles inside it are overwritten later).
     cudaError_t e;
-    if (p.split_from == 0) {
+    if (p.split_from == 0 || swap) {
       e = cudaMemsetAsync(C, 0, static_cast<size_t>(M) * N * C_ELEM, stream);
     } else {
       int tm_lo = p.tiles_m, tm_hi = -1, tn_lo = p.tiles_n, tn_hi = -1;

@@ -40,6 +40,7 @@ int g_override_cta_group = 0;
 int g_override_splits = 0;
 int g_trace_on = 0;
 int g_s4_scheme = 0;   // INT4 route: 0 = automatic, 1 = always the pre-pass, 2 = fused wherever built
+int g_swap_ab = 0;     // 0 = automatic, 1 = never, 2 = always exchange A and B inside the library
 int g_l2_policy = 11;  // keep A, B normal, serpentine K, C stores evict-first
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
