@@ -11,11 +11,12 @@
 namespace b200gemm {
 namespace {
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI, int PSTAGES = 0>
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI, int PSTAGES = 0,
+          int AMODE = 0>
 int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUtensorMap& tb,
                    const CUtensorMap& tc, const GemmParams& p, cudaStream_t stream) {
-  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES>;
-  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI, PSTAGES>;
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, AMODE>;
+  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI, PSTAGES, AMODE>;
   if (!(s->attr_set[variant >> 6] & (1ull << (variant & 63)))) {
     cudaError_t e =
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
@@ -57,7 +58,7 @@ struct OutputSpec {
 // re-used enough to pay for a pre-pass over them: problems with few rows on one side
 // (LLM decoding), which are bound by the bytes of the other operand.
 bool s4_fused_wanted(int M, int N, const TileConfig& cfg) {
-  if (g_s4_scheme == 2) return true;
+  if (g_s4_scheme >= 2) return true;
   if (g_s4_scheme == 1) return false;
   return cfg.cta_group == 1 && (M <= 128 || N <= 128);
 }
@@ -71,7 +72,7 @@ bool swap_ab_wanted(int M, int N, bool packed_s4, const OutputSpec& out) {
   if (out.no_split || out.ldc) return false;  // C is a block of a larger matrix
   if (g_swap_ab == 1) return false;
   if (g_swap_ab == 2) return true;
-  return packed_s4 && M <= 64 && N >= 512;
+  return packed_s4 ? (M <= 64 && N >= 512) : (M <= 32 && N >= 1024);
 }
 
 // Returned (never to the caller of the library) when the fused INT4 kernel does not cover the
@@ -201,6 +202,14 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
       const int fb = 64 + EPI * 8;
       if (cfg.cta_group == 2)
         return launch_variant<KIND, 256, 4, 2, 1, EPI, 2>(s, fb + 0, ta, tb, tc, p, stream);
+      if (swap && cfg.bn <= 64 && g_s4_scheme != 3) {
+        // exchanged operands, narrow tile: the expanded 128-row tile goes to tensor memory
+        if (cfg.bn == 64)
+          return launch_variant<KIND, 64, 4, 1, 1, EPI, 6, 1>(s, fb + 5, ta, tb, tc, p, stream);
+        if constexpr (EPI != EPI_OUT16)
+          return launch_variant<KIND, 32, 4, 1, 1, EPI, 8, 1>(s, fb + 6, ta, tb, tc, p, stream);
+        return GEMM_ERR_INVALID_ARG;
+      }
       switch (cfg.bn) {
         case 256: return launch_variant<KIND, 256, 2, 1, 1, EPI, 2>(s, fb + 1, ta, tb, tc, p, stream);
         case 128: return launch_variant<KIND, 128, 3, 1, 1, EPI, 3>(s, fb + 2, ta, tb, tc, p, stream);
