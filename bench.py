@@ -14,6 +14,10 @@ FP16 GEMM with pinned host buffers and both copies inside the timed region.
 
 Prints ONE JSON line on rank 0.  Under torchrun each rank runs an independent
 replica of the same workload (no data-path collective; weak scaling).
+
+Other modes (1 GPU, one JSON line per measurement): --sweep (precision x size,
+N = 512..8192), --ablation (tile / raster / L2 / INT4 route at --size, with the
+kernel's cycle accounting), --few-rows (M = 1..128 against the HBM roofline).
 """
 from __future__ import annotations
 
@@ -510,6 +514,69 @@ def run_sweep(args):
         raise SystemExit("bench.py: a kernel reported a barrier timeout")
 
 
+def run_few_rows(args):
+    """Problems with few rows (the shapes of LLM decoding, which the paper lists as the use it
+    has in mind but does not measure, Sec. VI): bound by the bytes of B, so the roofline is HBM.
+    One JSON line per (shape, precision, route): CUDA-graph replay of 10 calls after an L2
+    flush (256 MB write), median of 7, every launch of a call included (split-K's zeroing of C,
+    the INT4 pre-pass).  `achieved` = algorithmic bytes (A, B as stored, C once) / time."""
+    import numpy as np
+    import torch
+    from paper_2608_10103_b200 import binding, synth
+    torch.cuda.set_device(0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    hbm = measured_peaks()["hbm_gbs"]
+    shapes = [(1, 8192, 8192), (16, 8192, 8192), (64, 8192, 8192), (16, 4096, 16384),
+              (128, 16384, 4096), (32, 28672, 8192)]
+    routes = {"fp16": [("selector default", 0, 0), ("operands not exchanged", 0, 1)],
+              "s8": [("selector default", 0, 0), ("operands not exchanged", 0, 1)],
+              "s4": [("selector default", 0, 0), ("pre-pass + INT8 GEMM", 1, 1),
+                     ("expanded in the kernel, through shared memory only", 3, 1)]}
+    for M, N, K in shapes:
+        for prec in synth.PRECISIONS:
+            A, B = synth.make(prec, M, N, K, seed=M + N)
+            dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+            C = torch.empty((M, N), dtype=torch.float32 if prec == "fp16" else torch.int32,
+                            device="cuda")
+            algo_bytes = A.nbytes + B.nbytes + M * N * 4
+            for name, scheme, swap in routes[prec]:
+                binding.gemm_set_s4_scheme(scheme)
+                binding.gemm_set_swap_ab(swap)
+                for _ in range(3):
+                    binding.gemm(prec, dA, dB, C)
+                torch.cuda.synchronize()
+                g = torch.cuda.CUDAGraph()
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    with torch.cuda.graph(g, stream=side):
+                        for _ in range(10):
+                            binding.gemm(prec, dA, dB, C, stream=side)
+                torch.cuda.current_stream().wait_stream(side)
+                ts = []
+                for _ in range(7):
+                    flush.fill_(1)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    g.replay()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ts.append(e0.elapsed_time(e1) / 10)
+                us = float(np.median(ts)) * 1e3
+                gbs = algo_bytes / us / 1e3
+                print(json.dumps({
+                    "few_rows": True, "M": M, "N": N, "K": K, "precision": prec, "route": name,
+                    "us": us, "value": synth.gemm_ops(M, N, K) / us / 1e6, "unit": UNIT[prec],
+                    "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s",
+                                 "frac": gbs / hbm, "traffic": None},
+                    "algorithmic_bytes": algo_bytes,
+                    "config": binding.gemm_query_config(prec, M, N, K)}), flush=True)
+    binding.gemm_set_s4_scheme(0)
+    binding.gemm_set_swap_ab(0)
+    if binding.gemm_last_device_status() != 0:
+        raise SystemExit("bench.py: a kernel reported a barrier timeout")
+
+
 def run_ablation(args):
     """One-variable-at-a-time ablation at N = args.size (the analogue of the paper's Run 4):
     tile shape, raster band height, L2 policy, and load-only / MMA-only runs, each with
@@ -608,6 +675,9 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-peak-probe", action="store_true")
+    ap.add_argument("--few-rows", action="store_true",
+                    help="few-row (LLM decoding) shapes, every precision and INT4 route, against the "
+                         "HBM roofline (1 GPU)")
     ap.add_argument("--ablation", action="store_true",
                     help="tile / raster / L2 / load-vs-MMA ablation with cycle accounting (1 GPU)")
     ap.add_argument("--sweep", action="store_true",
@@ -624,6 +694,9 @@ def main():
     if args.ablation:
         if rank == 0:
             run_ablation(args)
+    elif args.few_rows:
+        if rank == 0:
+            run_few_rows(args)
     elif args.sweep:
         if rank == 0:
             run_sweep(args)
