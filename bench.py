@@ -528,12 +528,14 @@ def run_few_rows(args):
     hbm = measured_peaks()["hbm_gbs"]
     shapes = [(1, 8192, 8192), (16, 8192, 8192), (64, 8192, 8192), (16, 4096, 16384),
               (128, 16384, 4096), (32, 28672, 8192)]
+    if args.shape:
+        shapes = [tuple(int(x) for x in args.shape.split(","))]
     routes = {"fp16": [("selector default", 0, 0), ("operands not exchanged", 0, 1)],
               "s8": [("selector default", 0, 0), ("operands not exchanged", 0, 1)],
               "s4": [("selector default", 0, 0), ("pre-pass + INT8 GEMM", 1, 1),
                      ("expanded in the kernel, through shared memory only", 3, 1)]}
     for M, N, K in shapes:
-        for prec in synth.PRECISIONS:
+        for prec in [q for q in synth.PRECISIONS if q in args.precisions.split(",")]:
             A, B = synth.make(prec, M, N, K, seed=M + N)
             dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
             C = torch.empty((M, N), dtype=torch.float32 if prec == "fp16" else torch.int32,
@@ -609,7 +611,7 @@ def run_ablation(args):
                    ("INT4 route 1: nibbles expanded inside the GEMM kernel", (0, 0, 0), 11, 1, 2),
                    ("INT4 route 1, ablate: no MMAs", (0, 0, 0), 11, 3, 2),
                    ("INT4 route 1, ablate: no operand loads", (0, 0, 0), 11, 5, 2)]
-    for prec in ("fp16", "s8", "s4"):
+    for prec in [q for q in ("fp16", "s8", "s4") if q in args.precisions.split(",")]:
         dA, dB = (torch.from_numpy(x).cuda() for x in data[prec])
         C = torch.empty((N, N), dtype=torch.float32 if prec == "fp16" else torch.int32,
                         device="cuda")
@@ -678,6 +680,7 @@ def main():
     ap.add_argument("--few-rows", action="store_true",
                     help="few-row (LLM decoding) shapes, every precision and INT4 route, against the "
                          "HBM roofline (1 GPU)")
+    ap.add_argument("--shape", default="", help="--few-rows: only this M,N,K")
     ap.add_argument("--ablation", action="store_true",
                     help="tile / raster / L2 / load-vs-MMA ablation with cycle accounting (1 GPU)")
     ap.add_argument("--sweep", action="store_true",
