@@ -43,18 +43,26 @@ def test_expired_wait_is_reported_and_the_context_survives(cta_group):
         binding.gemm_set_config_override(0, 0, 0)
 
 
-def test_expired_wait_in_the_fused_int4_kernel():
-    """Same drill through the kernel variant with the extra nibble-expansion warps and the
+@pytest.mark.parametrize("variant", ["pair tile, expansion through shared memory",
+                                     "exchanged operands, expanded tile in tensor memory"])
+def test_expired_wait_in_the_fused_int4_kernels(variant):
+    """Same drill through the kernel variants with the extra nibble-expansion warps and the
     second (packed) ring: a packed slot of CTA 0 is never filled."""
-    M, N, K = 256, 256, 2048                      # one tile, 8 packed slots (> ring depth 2)
+    if variant.startswith("pair"):
+        M, N, K = 256, 256, 2048                  # one tile, 8 packed slots (> ring depth 2)
+        override, swap, tag = (256, 0, 2, 1), 1, "fused_unpack"
+    else:
+        M, N, K = 16, 128, 4096                   # one tile, 16 packed slots (> ring depth 8)
+        override, swap, tag = (32, 0, 1, 1), 2, "A via TMEM"
     A, B = synth.s4_uniform(M, N, K, seed=10)
     dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
     C = torch.zeros((M, N), dtype=torch.int32, device="cuda")
     assert binding.gemm_last_device_status() == 0
-    binding.gemm_set_config_override(256, 0, 2, 1)
+    binding.gemm_set_config_override(*override)
     binding.gemm_set_s4_scheme(2)
+    binding.gemm_set_swap_ab(swap)
     try:
-        assert "fused_unpack" in binding.gemm_query_config("s4", M, N, K)
+        assert tag in binding.gemm_query_config("s4", M, N, K)
         binding.gemm_trace_enable(16)
         t0 = time.time()
         binding.gemm_s4(dA, dB, C)
@@ -71,4 +79,5 @@ def test_expired_wait_in_the_fused_int4_kernel():
     finally:
         binding.gemm_trace_enable(0)
         binding.gemm_set_s4_scheme(0)
+        binding.gemm_set_swap_ab(0)
         binding.gemm_set_config_override(0, 0, 0)
