@@ -3,12 +3,13 @@
 // Roles of the paper's double/triple-buffered cp.async -> ldmatrix -> mma.sync
 // loop (Sec. III-A, Listings 1 and 3), re-cast for Blackwell:
 //
-//   warp 0, one lane   : TMA producer.  One tensor copy per operand per
-//                        k-block lands a 128 x 128-byte A tile and a
-//                        B_ROWS x 128-byte B tile (128-byte swizzle) in a ring
-//                        of STAGES shared-memory slots; completion is counted
-//                        in bytes on the slot's `full` mbarrier.
-//   warp 1, one lane   : MMA issuer.  Waits `full`, issues 4 tcgen05.mma
+//   warp 0             : TMA producer (all lanes walk the loops, one elected lane
+//                        issues).  One tensor copy per operand per k-block lands a
+//                        128 x 128-byte A tile and a B_ROWS x 128-byte B tile
+//                        (128-byte swizzle) in a ring of STAGES shared-memory
+//                        slots; completion is counted in bytes on the slot's
+//                        `full` mbarrier.
+//   warp 1             : MMA issuer (likewise).  Waits `full`, issues 4 tcgen05.mma
 //                        (each consumes 32 bytes of K) accumulating into one of
 //                        two TMEM accumulator buffers, then commits to the
 //                        slot's `empty` barrier so the producer may refill it.
@@ -35,6 +36,11 @@
 //   shifts them right by 8, exactly.  The order in which K values land in the int8 slots
 //   differs from their order in memory, identically for A and B, which leaves every dot
 //   product unchanged.
+//   AMODE = 1 (with PSTAGES > 0, one CTA, BN <= 64): the expanded A tile is written to
+//   tensor memory instead (tcgen05.st, thread = row = TMEM lane) and the MMAs take their
+//   A operand from there; shared memory then carries A once, packed.  The host uses it with
+//   exchanged operands (GemmParams::transpose_c) for problems with few rows, where the
+//   kernel's A is the caller's long operand.
 //
 // A is M x K row-major, B is N x K with K contiguous (the paper's ".row.col"
 // operand layout, Listing 2c); C is M x N row-major, 32-bit, overwritten.
