@@ -278,16 +278,12 @@ int gemm_last_device_status(void);
  *     for an operand that is read once; but half as much shared-memory traffic
  *     again per unit of math, which is what bounds the large-tile kernel.
  * Measured: at M = N = K = 8192 the pre-pass route is 1.1-1.35x faster; for
- * M = 16, N = K = 8192 (bound by the bytes of B) the fused route takes 15 us
+ * M = 16, N = K = 8192 (bound by the bytes of B) the fused route takes 18.6 us
  * instead of 33.
  * scheme 0 (default, automatic): fused where the selector picks a one-CTA tile
  * and M <= 128 or N <= 128, else the pre-pass; 1: always the pre-pass; 2: fused
  * wherever a fused variant is built (every one-CTA tile, and the 256 x 256 CTA
- * pair without split-K), else the pre-pass; 3: as 2, but without the variant
- * described next.  When the operands are exchanged (gemm_set_swap_ab) and the
- * tile is 32 or 64 wide, the expanded 128-row tile is written to tensor memory
- * (tcgen05.st) and the MMAs read it from there, so that it crosses shared
- * memory once, packed, instead of three times.  gemm_s4_ws and gemm_s4_static
+ * pair without split-K), else the pre-pass.  gemm_s4_ws and gemm_s4_static
  * always use the pre-pass.  Results are identical, bit for bit.
  * gemm_query_config shows the route.  The paper has no counterpart; its Run 4
  * ablates how the operands reach the tensor cores, of which this is the
@@ -301,14 +297,13 @@ int gemm_set_s4_scheme(int scheme);
  * is written by plain stores that are contiguous along N.  For problems with
  * few rows (M = 1..64, LLM decoding) this keeps 128 - M rows of zero fill out
  * of shared memory, of the ring depth and -- on the fused INT4 route -- of the
- * expansion work.  mode 0 (default, automatic): on the fused INT4 route when
- * M <= 64 and N >= 512, for the other kernels when M <= 32 and N >= 1024 (measured
- * 5-11 % faster there); 1: never; 2: always (any shape and precision; for tests
- * and measurements).  Results: integers identical; FP16 within the bound;
- * dequantised outputs multiply the two scales in the other order (last-bit
- * differences).  gemm_query_config shows "swap_ab" and then describes the tile
- * in the kernel's orientation.  The paper has no counterpart (square sizes
- * only, Sec. VI).
+ * expansion work.  mode 0 (default, automatic): for the FP16 and INT8 kernels
+ * when M <= 32 and N >= 1024 (measured 5-11 % faster there); 1: never; 2: always
+ * (any shape, precision and INT4 route; for tests and measurements).  Results:
+ * integers identical; FP16 within the bound; dequantised outputs multiply the
+ * two scales in the other order (last-bit differences).  gemm_query_config
+ * shows "swap_ab" and then describes the tile in the kernel's orientation.  The
+ * paper has no counterpart (square sizes only, Sec. VI).
  */
 int gemm_set_swap_ab(int mode);
 

@@ -305,15 +305,13 @@ def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0, 
 def gemm_set_s4_scheme(scheme: int = 0):
     """Route of gemm_s4 / gemm_s4_dequant: 0 = automatic (nibbles expanded inside the GEMM
     kernel for problems with few rows on one side, else a pre-pass to int8 + the INT8 GEMM);
-    1 = always the pre-pass; 2 = inside the GEMM kernel wherever such a variant is built; 3 = as 2
-    but never the variant that keeps the expanded tile in tensor memory."""
+    1 = always the pre-pass; 2 = inside the GEMM kernel wherever such a variant is built."""
     _check(lib().gemm_set_s4_scheme(int(scheme)), "gemm_set_s4_scheme")
 
 
 def gemm_set_swap_ab(mode: int = 0):
     """Run the kernel on exchanged operands (long operand on the 128-row tile side, C stored
-    along N by plain stores): 0 = automatic (few rows: M <= 64 on the fused INT4 route, M <= 32 otherwise), 1 = never,
-    2 = always."""
+    along N by plain stores): 0 = automatic (FP16 / INT8 problems with M <= 32), 1 = never, 2 = always."""
     _check(lib().gemm_set_swap_ab(int(mode)), "gemm_set_swap_ab")
 
 

@@ -202,11 +202,7 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
                 : units) *
                c.cta_group,
            precision == GEMM_PREC_FP16 ? "f16" : "i8",
-           precision != GEMM_PREC_S4 ? ""
-           : !fused                    ? " prepass=unpack_s4"
-           : (swap && c.cta_group == 1 && c.bn <= 64 && g_s4_scheme != 3)
-               ? " s4=fused_unpack(A via TMEM)"
-               : " s4=fused_unpack",
+           precision != GEMM_PREC_S4 ? "" : fused ? " s4=fused_unpack" : " prepass=unpack_s4",
            swap ? " swap_ab" : "");
   return GEMM_OK;
 }
@@ -249,7 +245,7 @@ int gemm_last_device_status(void) {
 }
 
 int gemm_set_s4_scheme(int scheme) {
-  if (scheme < 0 || scheme > 3) return GEMM_ERR_INVALID_ARG;
+  if (scheme < 0 || scheme > 2) return GEMM_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
   g_s4_scheme = scheme;
   return GEMM_OK;

@@ -36,11 +36,6 @@
 //   shifts them right by 8, exactly.  The order in which K values land in the int8 slots
 //   differs from their order in memory, identically for A and B, which leaves every dot
 //   product unchanged.
-//   AMODE = 1 (with PSTAGES > 0, one CTA, BN <= 64): the expanded A tile is written to
-//   tensor memory instead (tcgen05.st, thread = row = TMEM lane) and the MMAs take their
-//   A operand from there; shared memory then carries A once, packed.  The host uses it with
-//   exchanged operands (GemmParams::transpose_c) for problems with few rows, where the
-//   kernel's A is the caller's long operand.
 //
 // A is M x K row-major, B is N x K with K contiguous (the paper's ".row.col"
 // operand layout, Listing 2c); C is M x N row-major, 32-bit, overwritten.
@@ -104,6 +99,9 @@ struct GemmParams {
   // lanes (32 consecutive kernel rows) store 32 consecutive elements of a row of C.  Always
   // with c_vec_ok = 0 (plain stores).
   int transpose_c;
+  // 1: this grid was launched to start while the kernel that zeroes C for split-K may still
+  // run (programmatic dependent launch); whoever adds into C waits for that kernel first.
+  int wait_prior_grid;
   const float* row_scale;  // EPI_OUT16 (integer kinds) / EPI_F32_SCALED: M per-row factors
   const float* col_scale;  // and N per-column factors; both null = no scaling (FP16 kind)
   int* status;           // device status word (0 = ok)
@@ -149,15 +147,12 @@ enum TraceSlot {
 // bytes of K in the 128-byte-swizzle layout (the widest a swizzled TMA box can
 // be).  KB = 2 halves the per-slot barrier work (one wait, one commit per 8 MMAs)
 // of the single issuing thread, whose instruction time is the scarce resource.
-template <int BN, int STAGES, int CTA_GROUP, int KB, int PSTAGES = 0, int AMODE = 0>
+template <int BN, int STAGES, int CTA_GROUP, int KB, int PSTAGES = 0>
 struct SmemLayout {
   static constexpr int B_ROWS = BN / CTA_GROUP;  // B rows each CTA loads
   static constexpr int A_BYTES = BM * BK_BYTES;       // one A atom
   static constexpr int B_BYTES = B_ROWS * BK_BYTES;   // one B atom
-  // AMODE = 1 (fused INT4 only): the expanded A tile goes to tensor memory, so a slot of the
-  // ring the MMAs read holds B alone
-  static constexpr int A8_BYTES = AMODE ? 0 : A_BYTES;
-  static constexpr int STAGE_BYTES = KB * (A8_BYTES + B_BYTES);
+  static constexpr int STAGE_BYTES = KB * (A_BYTES + B_BYTES);
   // Fused INT4: PSTAGES more slots, each one packed atom per operand (256 nibbles of K per row).
   static constexpr int P_STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int P_OFFSET = STAGES * STAGE_BYTES;
@@ -228,26 +223,18 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32, int PSTAGES = 0,
-          int AMODE = 0>
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32, int PSTAGES = 0>
 __global__ void __launch_bounds__(PSTAGES > 0 ? NUM_THREADS_FUSED : NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
-  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, AMODE>;
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES>;
   constexpr bool FUSED = PSTAGES > 0;  // packed INT4 operands, expanded on the way to the MMAs
-  // The expanded A tile lives in tensor memory (STAGES buffers of 32 columns behind the two
-  // accumulators) and the MMAs take it from there: no shared-memory write or read for A.
-  constexpr bool TMEM_A = FUSED && AMODE == 1;
-  static_assert(AMODE == 0 || (FUSED && CTA_GROUP == 1 && BN <= 64), "A via TMEM: fused INT4, one CTA, narrow tile");
-  constexpr uint32_t ACC_COLS = 2 * BN;
   static_assert(!FUSED || (KIND == ptx::KIND_I8 && KB == 1 && STAGES >= 2),
                 "fused INT4: int8 MMAs, one atom per slot, a packed slot fills two int8 slots at once");
   constexpr int ELEM_BYTES = (KIND == ptx::KIND_F16) ? 2 : 1;
   constexpr int BK_ELEMS = BK_BYTES / ELEM_BYTES;
   constexpr int TILE_M = BM * CTA_GROUP;
-  constexpr uint32_t TMEM_COLS =   // two accumulator buffers (+ the A buffers), a power of two
-      TMEM_A ? ((ACC_COLS + STAGES * 32 <= 256) ? 256u : 512u) : ((2 * BN <= 32) ? 32u : 2u * BN);
-  static_assert(!TMEM_A || ACC_COLS + STAGES * 32 <= 512, "A buffers must fit behind the accumulators");
+  constexpr uint32_t TMEM_COLS = (2 * BN <= 32) ? 32 : 2 * BN;  // two accumulator buffers
   static_assert(CTA_GROUP == 1 || CTA_GROUP == 2, "CTA_GROUP is 1 or 2");
   static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "BN must be a multiple of 32 up to 256");
   static_assert((TMEM_COLS & (TMEM_COLS - 1)) == 0 && TMEM_COLS <= 512, "TMEM columns: power of 2");
@@ -503,7 +490,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           ptx::tc_fence_after_sync();
           const uint32_t a_src = base + stage * L::STAGE_BYTES;
           const uint64_t a_desc = ptx::smem_desc_sw128(a_src);
-          const uint64_t b_desc = ptx::smem_desc_sw128(a_src + KB * L::A8_BYTES);
+          const uint64_t b_desc = ptx::smem_desc_sw128(a_src + KB * L::A_BYTES);
           if (elected && !(p.ablate & 1)) {
 #pragma unroll
             for (int a = 0; a < KB; ++a) {
@@ -514,14 +501,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     static_cast<uint64_t>((a * L::A_BYTES + kk * MMA_K_BYTES) >> 4);
                 const uint64_t b_step =
                     static_cast<uint64_t>((a * L::B_BYTES + kk * MMA_K_BYTES) >> 4);
-                if constexpr (TMEM_A) {
-                  ptx::mma_ts_i8(d_tmem,
-                                 tmem_base + ACC_COLS + static_cast<uint32_t>(stage * 32 + kk * 8),
-                                 b_desc + b_step, idesc, (ks > k_begin || kk > 0) ? 1u : 0u);
-                } else {
-                  ptx::mma_ss<KIND, CTA_GROUP>(d_tmem, a_desc + a_step, b_desc + b_step, idesc,
-                                               (ks > k_begin || a > 0 || kk > 0) ? 1u : 0u);
-                }
+                ptx::mma_ss<KIND, CTA_GROUP>(d_tmem, a_desc + a_step, b_desc + b_step, idesc,
+                                             (ks > k_begin || a > 0 || kk > 0) ? 1u : 0u);
               }
             }
           }
@@ -635,62 +616,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const long long w2 = trace ? clock64() : 0;
           if (trace) wait_out += w2 - w1;
           if (!ok) break;
-          if constexpr (TMEM_A) {
-            // A: warps 6..9 take int8 slot u0 (packed chunks 0..3 of every row), warps 10..13
-            // slot u1 (chunks 4..7); lane = row within the TMEM lane quarter this warp may
-            // touch.  A thread reads its row's four chunks, and writes the 128 bytes of the
-            // int8 row -- even-k values of the four chunks, then their odd-k values, the
-            // order the B tile has in shared memory -- to 32 TMEM columns of its lane.
-            {
-              const int h = uw >> 2;
-              const int r = (warp & 3) * 32 + lane;
-              uint32_t regs[32];
-              if (r < a_valid) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  uint32_t w0_, w1_, w2_, w3_;
-                  ptx::ld_shared_v4(src + static_cast<uint32_t>(r * 128 + (((4 * h + j) ^ (r & 7)) << 4)),
-                                    w0_, w1_, w2_, w3_);
-                  regs[4 * j + 0] = (w0_ << 4) & HI;
-                  regs[4 * j + 1] = (w1_ << 4) & HI;
-                  regs[4 * j + 2] = (w2_ << 4) & HI;
-                  regs[4 * j + 3] = (w3_ << 4) & HI;
-                  regs[16 + 4 * j + 0] = w0_ & HI;
-                  regs[16 + 4 * j + 1] = w1_ & HI;
-                  regs[16 + 4 * j + 2] = w2_ & HI;
-                  regs[16 + 4 * j + 3] = w3_ & HI;
-                }
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) regs[j] = 0;
-              }
-              ptx::tmem_st_32x32b_x32(tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) +
-                                          ACC_COLS + static_cast<uint32_t>((h ? u1 : u0) * 32),
-                                      regs);
-            }
-            // B: BN rows x 8 chunks over the 256 threads; chunk at physical position pc of row
-            // rb is logical chunk pc ^ (rb & 7) and feeds int8 slot (logical chunk) / 4
-            {
-              const int t = uw * 32 + lane;
-#pragma unroll
-              for (int i = 0; i < BN / 32; ++i) {
-                const int rb = i * 32 + (t >> 3);
-                if (rb >= b_valid) continue;
-                const uint32_t xb = static_cast<uint32_t>(rb * 128 + ((t & 7) << 4));
-                const uint32_t hb = ((static_cast<uint32_t>(t) ^ static_cast<uint32_t>(rb)) >> 2) & 1u;
-                uint32_t w0_, w1_, w2_, w3_;
-                ptx::ld_shared_v4(src + L::A_BYTES + xb, w0_, w1_, w2_, w3_);
-                const uint32_t dst = base + (hb ? u1 : u0) * L::STAGE_BYTES;
-                ptx::st_shared_v4(dst + (xb ^ (hb << 6)), (w0_ << 4) & HI, (w1_ << 4) & HI,
-                                  (w2_ << 4) & HI, (w3_ << 4) & HI);
-                ptx::st_shared_v4(dst + (xb ^ (hb << 6) ^ 64u), w0_ & HI, w1_ & HI, w2_ & HI, w3_ & HI);
-              }
-            }
-            ptx::tmem_wait_st();
-            ptx::tc_fence_before_sync();
-          }
-#pragma unroll
-          for (int h = 0; h < 2 && !TMEM_A; ++h) {
+          for (int h = 0; h < 2; ++h) {
             const uint32_t dst = base + (h ? u1 : u0) * L::STAGE_BYTES;
             const uint32_t x0 = static_cast<uint32_t>(row_in_8 * 128 + (((4 * h + c) ^ row_in_8) << 4));
             const uint32_t flip = static_cast<uint32_t>(h) << 6;
@@ -752,6 +679,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     bool ok = true;
     long long epi_wait = 0, epi_busy = 0, tiles_done = 0;
     uint32_t staged_blocks = 0;  // blocks sent through the staging buffers so far
+    bool prior_grid_done = false;
     for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
       int tm, tn, tile, k_begin, k_end;
       bool add;
@@ -767,6 +695,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::tc_fence_after_sync();
       // A split-K unit whose K range is empty (the host never creates one) contributes nothing.
       const bool empty_range = k_begin >= k_end;
+      if (p.wait_prior_grid && !prior_grid_done) {  // C must have been zeroed before anything lands in it
+        ptx::grid_dep_wait();
+        prior_grid_done = true;
+      }
       const int row0 = tm * TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
       const int row = row0 + lane;
       const int col0 = tn * BN;

@@ -11,12 +11,23 @@
 namespace b200gemm {
 namespace {
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI, int PSTAGES = 0,
-          int AMODE = 0>
+// Zeroes C ahead of a split-K GEMM.  It lets the GEMM start at once (the GEMM's mainloop does
+// not touch C; its epilogue waits for this grid before it adds), which takes the launch
+// latency of the GEMM and the gap between two dependent launches off the critical path of
+// the small, latency-bound problems that split K.
+__global__ void zero_c_kernel(uint4* c16, size_t n16, uint32_t* tail, int tail_words) {
+  ptx::grid_dep_launch_dependents();
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n16; i += stride)
+    c16[i] = make_uint4(0, 0, 0, 0);
+  if (blockIdx.x == 0 && static_cast<int>(threadIdx.x) < tail_words) tail[threadIdx.x] = 0;
+}
+
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI, int PSTAGES = 0>
 int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUtensorMap& tb,
                    const CUtensorMap& tc, const GemmParams& p, cudaStream_t stream) {
-  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, AMODE>;
-  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI, PSTAGES, AMODE>;
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES>;
+  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI, PSTAGES>;
   if (!(s->attr_set[variant >> 6] & (1ull << (variant & 63)))) {
     cudaError_t e =
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
@@ -32,13 +43,15 @@ int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUt
   cfg.blockDim = dim3(PSTAGES > 0 ? NUM_THREADS_FUSED : NUM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = L::DYN_BYTES;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CTA_GROUP;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = p.wait_prior_grid ? 2 : 1;  // may start while zero_c_kernel still runs
   cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, tc, p);
   if (e != cudaSuccess) return cuda_fail(e);
   return GEMM_OK;
@@ -58,7 +71,7 @@ struct OutputSpec {
 // re-used enough to pay for a pre-pass over them: problems with few rows on one side
 // (LLM decoding), which are bound by the bytes of the other operand.
 bool s4_fused_wanted(int M, int N, const TileConfig& cfg) {
-  if (g_s4_scheme >= 2) return true;
+  if (g_s4_scheme == 2) return true;
   if (g_s4_scheme == 1) return false;
   return cfg.cta_group == 1 && (M <= 128 || N <= 128);
 }
@@ -67,12 +80,13 @@ bool s4_fused_wanted(int M, int N, const TileConfig& cfg) {
 // side of a tile is then filled by the long operand of a problem with few rows (LLM decoding:
 // M = 1..64), instead of 128 - M rows of zero fill taking shared memory, ring depth and, on
 // the fused INT4 route, expansion work; C goes out by plain stores that are contiguous along
-// the caller's N.  Automatic: on the fused INT4 route only, where it was measured to pay.
+// the caller's N.  Automatic for the FP16 / INT8 kernels when M <= 32 (measured 5-11 % faster);
+// the fused INT4 kernel gains nothing from it (bound by its expansion traffic either way).
 bool swap_ab_wanted(int M, int N, bool packed_s4, const OutputSpec& out) {
   if (out.no_split || out.ldc) return false;  // C is a block of a larger matrix
   if (g_swap_ab == 1) return false;
   if (g_swap_ab == 2) return true;
-  return packed_s4 ? (M <= 64 && N >= 512) : (M <= 32 && N >= 1024);
+  return !packed_s4 && M <= 32 && N >= 1024;
 }
 
 // Returned (never to the caller of the library) when the fused INT4 kernel does not cover the
@@ -137,6 +151,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.split_from = p.tiles_m * p.tiles_n - (cfg.splits > 1 ? cfg.split_tiles : 0);
   p.ldc = ldc;
   p.transpose_c = swap ? 1 : 0;
+  p.wait_prior_grid = 0;
   p.c_vec_ok = !swap && (ldc % (16 / C_ELEM) == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
   CUtensorMap tc;
   if (p.c_vec_ok) {
@@ -164,7 +179,16 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     // the bounding rectangle of those tiles (other tiles inside it are overwritten later).
     cudaError_t e;
     if (p.split_from == 0 || swap) {
-      e = cudaMemsetAsync(C, 0, static_cast<size_t>(M) * N * C_ELEM, stream);
+      const size_t bytes = static_cast<size_t>(M) * N * C_ELEM;  // a multiple of 4 (32-bit C only)
+      const size_t n16 = bytes / 16;
+      size_t blocks = (n16 + 255) / 256;
+      if (blocks > static_cast<size_t>(s->num_sms) * 4) blocks = static_cast<size_t>(s->num_sms) * 4;
+      if (blocks < 1) blocks = 1;
+      zero_c_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+          static_cast<uint4*>(C), n16, reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(C) + n16 * 16),
+          static_cast<int>((bytes % 16) / 4));
+      e = cudaGetLastError();
+      p.wait_prior_grid = 1;
     } else {
       int tm_lo = p.tiles_m, tm_hi = -1, tn_lo = p.tiles_n, tn_hi = -1;
       for (int t = p.split_from; t < p.tiles_m * p.tiles_n; ++t) {
@@ -202,14 +226,6 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
       const int fb = 64 + EPI * 8;
       if (cfg.cta_group == 2)
         return launch_variant<KIND, 256, 4, 2, 1, EPI, 2>(s, fb + 0, ta, tb, tc, p, stream);
-      if (swap && cfg.bn <= 64 && g_s4_scheme != 3) {
-        // exchanged operands, narrow tile: the expanded 128-row tile goes to tensor memory
-        if (cfg.bn == 64)
-          return launch_variant<KIND, 64, 4, 1, 1, EPI, 6, 1>(s, fb + 5, ta, tb, tc, p, stream);
-        if constexpr (EPI != EPI_OUT16)
-          return launch_variant<KIND, 32, 4, 1, 1, EPI, 8, 1>(s, fb + 6, ta, tb, tc, p, stream);
-        return GEMM_ERR_INVALID_ARG;
-      }
       switch (cfg.bn) {
         case 256: return launch_variant<KIND, 256, 2, 1, 1, EPI, 2>(s, fb + 1, ta, tb, tc, p, stream);
         case 128: return launch_variant<KIND, 128, 3, 1, 1, EPI, 3>(s, fb + 2, ta, tb, tc, p, stream);

@@ -39,8 +39,7 @@ int g_override_group_m = 0;
 int g_override_cta_group = 0;
 int g_override_splits = 0;
 int g_trace_on = 0;
-int g_s4_scheme = 0;   // INT4 route: 0 = automatic, 1 = always the pre-pass, 2 = fused wherever built,
-                       // 3 = as 2 but never the variant that keeps the expanded A tile in TMEM
+int g_s4_scheme = 0;   // INT4 route: 0 = automatic, 1 = always the pre-pass, 2 = fused wherever built
 int g_swap_ab = 0;     // 0 = automatic, 1 = never, 2 = always exchange A and B inside the library
 int g_l2_policy = 11;  // keep A, B normal, serpentine K, C stores evict-first
 

@@ -43,8 +43,7 @@ def test_expired_wait_is_reported_and_the_context_survives(cta_group):
         binding.gemm_set_config_override(0, 0, 0)
 
 
-@pytest.mark.parametrize("variant", ["pair tile, expansion through shared memory",
-                                     "exchanged operands, expanded tile in tensor memory"])
+@pytest.mark.parametrize("variant", ["pair tile", "one-CTA tile, exchanged operands"])
 def test_expired_wait_in_the_fused_int4_kernels(variant):
     """Same drill through the kernel variants with the extra nibble-expansion warps and the
     second (packed) ring: a packed slot of CTA 0 is never filled."""
@@ -52,8 +51,8 @@ def test_expired_wait_in_the_fused_int4_kernels(variant):
         M, N, K = 256, 256, 2048                  # one tile, 8 packed slots (> ring depth 2)
         override, swap, tag = (256, 0, 2, 1), 1, "fused_unpack"
     else:
-        M, N, K = 16, 128, 4096                   # one tile, 16 packed slots (> ring depth 8)
-        override, swap, tag = (32, 0, 1, 1), 2, "A via TMEM"
+        M, N, K = 16, 128, 4096                   # one tile, 16 packed slots (> ring depth 5)
+        override, swap, tag = (32, 0, 1, 1), 2, "swap_ab"
     A, B = synth.s4_uniform(M, N, K, seed=10)
     dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
     C = torch.zeros((M, N), dtype=torch.int32, device="cuda")

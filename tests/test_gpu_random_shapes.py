@@ -72,7 +72,7 @@ def test_random_shapes_configs_and_entry_points(seed):
             stream = side if g.integers(2) else None
             what = "%s %s M=%d N=%d K=%d cfg=%s side_stream=%s" % (prec, mode, M, N, K, cfg, stream is not None)
             binding.gemm_set_config_override(*cfg)
-            binding.gemm_set_s4_scheme(int(g.integers(4)))   # automatic / pre-pass / fused / fused, no TMEM
+            binding.gemm_set_s4_scheme(int(g.integers(3)))   # automatic / pre-pass / fused
             binding.gemm_set_swap_ab(int(g.integers(3)))     # automatic / never / always
             out_dtype = {"raw": torch.float32 if prec == "fp16" else torch.int32, "ws": torch.int32,
                          "static": torch.int32, "out16": torch.float16, "deq32": torch.float32,

@@ -35,17 +35,14 @@ def test_swapped_full_compare(prec, M, N, K):
         check_against_oracle(prec, A, B, C, force_full=True)
 
 
-@pytest.mark.parametrize("scheme", [1, 2, 3])
+@pytest.mark.parametrize("scheme", [1, 2])
 @pytest.mark.parametrize("bn,split_k", [(32, 1), (32, 4), (64, 3), (128, 2), (256, 1)])
 def test_swapped_int4_routes_tiles_and_split_k(bn, split_k, scheme):
-    """Pre-pass, fused (the expanded 128-row tile in tensor memory for the 32- and 64-wide
-    tiles) and fused through shared memory only."""
     M, N, K = 24, 1300, 2048
     binding.gemm_set_s4_scheme(scheme)
     binding.gemm_set_config_override(bn, 0, 1, split_k)
     cfg = binding.gemm_query_config("s4", M, N, K)
-    assert "swap_ab" in cfg and ("fused_unpack" in cfg) == (scheme >= 2)
-    assert ("A via TMEM" in cfg) == (scheme == 2 and bn <= 64)
+    assert "swap_ab" in cfg and ("fused_unpack" in cfg) == (scheme == 2)
     A, B = synth.s4_uniform(M, N, K, seed=bn + split_k)
     check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), force_full=True)
 
@@ -78,15 +75,16 @@ def test_swapped_output_variants():
 def test_automatic_choice_for_few_rows():
     binding.gemm_set_swap_ab(0)
     cfg = binding.gemm_query_config("s4", 16, 8192, 8192)
-    assert "swap_ab" in cfg and "fused_unpack" in cfg
-    assert "swap_ab" not in binding.gemm_query_config("s4", 2048, 2048, 2048)
-    assert "A via TMEM" in cfg
+    assert "fused_unpack" in cfg and "swap_ab" not in cfg
     assert "swap_ab" in binding.gemm_query_config("s8", 16, 8192, 8192)
     assert "swap_ab" in binding.gemm_query_config("fp16", 16, 8192, 8192)
     assert "swap_ab" not in binding.gemm_query_config("fp16", 128, 8192, 8192)
     assert "swap_ab" not in binding.gemm_query_config("s8", 16, 512, 8192)
+    assert "swap_ab" not in binding.gemm_query_config("s8", 2048, 2048, 2048)
     M, N, K = 16, 8192, 4096
-    A, B = synth.s4_uniform(M, N, K, seed=12)
-    check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), force_full=True)
+    for prec in synth.PRECISIONS:
+        A, B = synth.make(prec, M, N, K, seed=12)
+        C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
+        check_against_oracle(prec, A, B, C, force_full=True)
     binding.gemm_set_swap_ab(1)
-    assert "swap_ab" not in binding.gemm_query_config("s4", 16, 8192, 8192)
+    assert "swap_ab" not in binding.gemm_query_config("s8", 16, 8192, 8192)

@@ -1,0 +1,23 @@
+"""Collected after every other GPU test file but the last: the launch with the most tiles per
+CTA and the shortest mainloop (84 tiles of one k-block per CTA pair, 1.6 GB of C) must still be
+right after every other kernel variant of the library has run in this process.  (A kernel
+variant that kept an operand tile in tensor memory once made exactly this launch fail when it
+had run earlier in the process; the fixed-order suite did not show it.)"""
+import pytest
+
+from paper_2608_10103_b200 import binding, synth
+from gpu_util import check_against_oracle, freivalds, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def test_many_short_tiles_after_everything_else():
+    binding.gemm_set_config_override(0, 0, 0, 0)
+    binding.gemm_set_s4_scheme(0)
+    binding.gemm_set_swap_ab(0)
+    M, N, K = 20001, 20004, 64
+    A, B = synth.s8_uniform(M, N, K, seed=321)
+    C = run_gpu("s8", A, B)
+    check_against_oracle("s8", A, B, C, seed=321)
+    freivalds("s8", A, B, C, seed=321, vectors=2)
+    assert binding.gemm_last_device_status() == 0
