@@ -317,8 +317,15 @@ int gemm_set_swap_ab(int mode);
  * on the K range its predecessor, which shares its A rows, read last and still
  * finds in L2).  Bit 3 (8): mark the C stores "evict first" (written once,
  * never re-read).  Bit 4 (16): fetch operands with 128-byte instead of 256-byte
- * L2 promotion.  Default 11 = 3 + 8 with the serpentine order on, which gave
- * the lowest DRAM traffic at N = 8192.  Integer results never depend on any of
+ * L2 promotion.  Bit 5 (32): launch in plain stream order.  By default a GEMM
+ * of this library is launched so that it may begin while the kernel in front of
+ * it in the stream is still running (programmatic dependent launch): its set-up
+ * (barriers, tensor memory, descriptor prefetch) and the launch latency overlap
+ * that kernel's tail, and it waits for that kernel to complete before its first
+ * load and its first store; a GEMM of this library lets its successor begin as
+ * soon as it runs itself.  Stream semantics are unchanged; back-to-back small
+ * GEMMs get 15-25 % faster (N = 512: 5.1 -> 4.0 us).  Default 11 = 3 + 8 with
+ * the serpentine order on, which gave the lowest DRAM traffic at N = 8192.  Integer results never depend on any of
  * this; FP16 results may differ in the last bits (summation order) within the
  * bound.
  */

@@ -318,7 +318,7 @@ def gemm_set_swap_ab(mode: int = 0):
 def gemm_set_l2_policy(policy: int = 11):
     """Bit set: bits 0-1 operand eviction priority (0 normal, 1 keep A / stream B, 2 keep
     both, 3 keep A), +4 serpentine K order off, +8 C stores evict-first, +16 128-byte L2
-    promotion.  Default 11."""
+    promotion, +32 plain stream order (no programmatic dependent launch).  Default 11."""
     _check(lib().gemm_set_l2_policy(int(policy)), "gemm_set_l2_policy")
 
 

@@ -259,7 +259,7 @@ int gemm_set_swap_ab(int mode) {
 }
 
 int gemm_set_l2_policy(int policy) {
-  if (policy < 0 || policy > 31) return GEMM_ERR_INVALID_ARG;
+  if (policy < 0 || policy > 63) return GEMM_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
   g_l2_policy = policy;
   return GEMM_OK;

@@ -99,8 +99,13 @@ struct GemmParams {
   // lanes (32 consecutive kernel rows) store 32 consecutive elements of a row of C.  Always
   // with c_vec_ok = 0 (plain stores).
   int transpose_c;
-  // 1: this grid was launched to start while the kernel that zeroes C for split-K may still
-  // run (programmatic dependent launch); whoever adds into C waits for that kernel first.
+  // 1: this grid was launched to start before the grid in front of it in the stream has
+  // drained (programmatic dependent launch): its set-up overlaps that grid's tail, and whoever
+  // touches global memory (the producer before its first load, the epilogue before its first
+  // store) waits for that grid first.  In front may be another GEMM of this library, which
+  // lets its successor start as soon as it runs itself, or (value 2) the kernel that zeroes C for
+  // split-K: that one starts only when everything in front of it has completed, so the operands
+  // are ready when this grid starts and only the epilogue has to wait.
   int wait_prior_grid;
   const float* row_scale;  // EPI_OUT16 (integer kinds) / EPI_F32_SCALED: M per-row factors
   const float* col_scale;  // and N per-column factors; both null = no scaling (FP16 kind)
@@ -294,6 +299,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   unsigned long long* const trace =
       p.trace ? p.trace + static_cast<size_t>(blockIdx.x) * TRACE_SLOTS : nullptr;
   if (trace && threadIdx.x < TRACE_SLOTS) trace[threadIdx.x] = 0;  // roles that do not run leave 0
+  if (threadIdx.x == 0) ptx::grid_dep_launch_dependents();  // a following GEMM may set up now
   const long long clk_start = trace ? clock64() : 0;
   const uint64_t ns_start = trace ? ptx::globaltimer_ns() : 0;
 
@@ -341,6 +347,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       // issues the copies.  Nothing inside the loops is warp-collective, so a lane whose
       // wait gives up can leave on its own.
       const bool elected = ptx::elect_one();
+      if (p.wait_prior_grid == 1) ptx::grid_dep_wait();  // the operands may come from the grid in front
       int stage = 0;
       uint32_t phase = 0;
       int issued = 0;
@@ -695,7 +702,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::tc_fence_after_sync();
       // A split-K unit whose K range is empty (the host never creates one) contributes nothing.
       const bool empty_range = k_begin >= k_end;
-      if (p.wait_prior_grid && !prior_grid_done) {  // C must have been zeroed before anything lands in it
+      if (p.wait_prior_grid && !prior_grid_done) {  // C may be read, written or zeroed by the grid in front
         ptx::grid_dep_wait();
         prior_grid_done = true;
       }

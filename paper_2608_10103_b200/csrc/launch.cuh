@@ -11,10 +11,10 @@
 namespace b200gemm {
 namespace {
 
-// Zeroes C ahead of a split-K GEMM.  It lets the GEMM start at once (the GEMM's mainloop does
-// not touch C; its epilogue waits for this grid before it adds), which takes the launch
-// latency of the GEMM and the gap between two dependent launches off the critical path of
-// the small, latency-bound problems that split K.
+// Zeroes C ahead of a split-K GEMM.  It lets the GEMM start at once (the GEMM waits for this
+// grid before its first global access), which takes the launch latency of the GEMM and the
+// gap between two dependent launches off the critical path of the small, latency-bound
+// problems that split K.
 __global__ void zero_c_kernel(uint4* c16, size_t n16, uint32_t* tail, int tail_words) {
   ptx::grid_dep_launch_dependents();
   const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
@@ -51,7 +51,7 @@ int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUt
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = p.wait_prior_grid ? 2 : 1;  // may start while zero_c_kernel still runs
+  cfg.numAttrs = p.wait_prior_grid ? 2 : 1;  // may start while the grid in front still runs
   cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, tc, p);
   if (e != cudaSuccess) return cuda_fail(e);
   return GEMM_OK;
@@ -151,7 +151,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.split_from = p.tiles_m * p.tiles_n - (cfg.splits > 1 ? cfg.split_tiles : 0);
   p.ldc = ldc;
   p.transpose_c = swap ? 1 : 0;
-  p.wait_prior_grid = 0;
+  p.wait_prior_grid = (g_l2_policy & 32) ? 0 : 1;  // policy bit 32: plain stream order
   p.c_vec_ok = !swap && (ldc % (16 / C_ELEM) == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
   CUtensorMap tc;
   if (p.c_vec_ok) {
@@ -188,7 +188,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
           static_cast<uint4*>(C), n16, reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(C) + n16 * 16),
           static_cast<int>((bytes % 16) / 4));
       e = cudaGetLastError();
-      p.wait_prior_grid = 1;
+      if (p.wait_prior_grid) p.wait_prior_grid = 2;
     } else {
       int tm_lo = p.tiles_m, tm_hi = -1, tn_lo = p.tiles_n, tn_hi = -1;
       for (int t = p.split_from; t < p.tiles_m * p.tiles_n; ++t) {
