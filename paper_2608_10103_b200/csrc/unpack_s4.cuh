@@ -38,6 +38,8 @@ struct UnpackJob {
 
 __global__ void __launch_bounds__(256)
 unpack_s4_kernel(UnpackJob a, UnpackJob b, int chunks_per_row, long long out_pitch) {
+  // the GEMM behind this kernel may set up now; it waits for this grid before its first load
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const long long total = a.chunks + b.chunks;
   const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
   for (long long g = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; g < total;
