@@ -405,7 +405,10 @@ def run_ours(args, rank, world):
         },
         "clocks": clocks,
         "e2e": e2e,
-        "gpu_launches": args.steps * sum(KERNEL_LAUNCHES[p] for p in precs),
+        # INT4: pre-pass + GEMM, or the one fused kernel where the library picks that route
+        "gpu_launches": args.steps * sum(
+            1 if "fused_unpack" in binding.gemm_query_config(p, N, N, N) else KERNEL_LAUNCHES[p]
+            for p in precs),
     }
     if not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(N, host["fp16"][0], host["fp16"][1])

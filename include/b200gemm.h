@@ -280,8 +280,11 @@ int gemm_last_device_status(void);
  * Measured: at M = N = K = 8192 the pre-pass route is 1.1-1.35x faster; for
  * M = 16, N = K = 8192 (bound by the bytes of B) the fused route takes 18.6 us
  * instead of 33.
+ * Small problems, bound by launches and latencies, save one launch with the
+ * fused route (10-26 % up to 1024 x 1024 outputs).
  * scheme 0 (default, automatic): fused where the selector picks a one-CTA tile
- * and M <= 128 or N <= 128, else the pre-pass; 1: always the pre-pass; 2: fused
+ * and M <= 128 or N <= 128 or both <= 1024, or a single wave of CTA-pair tiles
+ * (e.g. 2048^3), else the pre-pass; 1: always the pre-pass; 2: fused
  * wherever a fused variant is built (every one-CTA tile, and the 256 x 256 CTA
  * pair without split-K), else the pre-pass.  gemm_s4_ws and gemm_s4_static
  * always use the pre-pass.  Results are identical, bit for bit.

@@ -177,7 +177,7 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
     c = swap ? select_config(N, M, num_sms, kb, 32, true, 2)
              : select_config(M, N, num_sms, kb, 32, true, 2);
     fused = c.bn != 0 && fused_s4_variant_exists(c.bn, c.cta_group, c.splits) &&
-            s4_fused_wanted(user_m, user_n, c);
+            s4_fused_wanted(user_m, user_n, c, num_sms);
   }
   if (!fused) {
     swap = swap_ab_wanted(M, N, false, OutputSpec());

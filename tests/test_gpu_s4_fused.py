@@ -43,7 +43,7 @@ def test_fused_is_what_the_selector_reports_and_runs_at_2048():
     A, B = synth.s4_uniform(M, N, K, seed=5)
     C = run_gpu("s4", A, B, fill=-7)
     check_against_oracle("s4", A, B, C, force_full=True)
-    binding.gemm_set_s4_scheme(0)
+    binding.gemm_set_s4_scheme(1)
     assert "prepass" in binding.gemm_query_config("s4", M, N, K)
     assert np.array_equal(C, run_gpu("s4", A, B, fill=-7))
 
@@ -74,10 +74,13 @@ def test_fused_one_cta_tiles_with_split_k(M, N, K, bn, split_k):
 
 def test_automatic_route_by_shape():
     binding.gemm_set_s4_scheme(0)
-    assert "fused_unpack" in binding.gemm_query_config("s4", 16, 8192, 8192)
+    assert "fused_unpack" in binding.gemm_query_config("s4", 16, 8192, 8192)      # few rows
     assert "fused_unpack" in binding.gemm_query_config("s4", 8192, 64, 4096)
+    assert "fused_unpack" in binding.gemm_query_config("s4", 512, 512, 512)       # small
+    assert "fused_unpack" in binding.gemm_query_config("s4", 2048, 2048, 2048)    # one wave of pair tiles
     assert "prepass" in binding.gemm_query_config("s4", 8192, 8192, 8192)
-    assert "prepass" in binding.gemm_query_config("s4", 2048, 2048, 2048)
+    assert "prepass" in binding.gemm_query_config("s4", 4096, 4096, 4096)
+    assert "prepass" in binding.gemm_query_config("s4", 512, 4096, 4096)
     binding.gemm_set_s4_scheme(1)
     assert "prepass" in binding.gemm_query_config("s4", 16, 8192, 8192)
     binding.gemm_set_s4_scheme(0)
