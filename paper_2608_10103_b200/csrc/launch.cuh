@@ -86,13 +86,13 @@ bool s4_fused_wanted(int M, int N, const TileConfig& cfg, int num_sms) {
 // side of a tile is then filled by the long operand of a problem with few rows (LLM decoding:
 // M = 1..64), instead of 128 - M rows of zero fill taking shared memory, ring depth and, on
 // the fused INT4 route, expansion work; C goes out by plain stores that are contiguous along
-// the caller's N.  Automatic when M <= 32 and N >= 1024 (measured 2-12 % faster on every route).
+// the caller's N.  Automatic when N >= 1024 and M <= 32 (M <= 64 on the fused INT4 route): measured
+// 2-12 % faster there.
 bool swap_ab_wanted(int M, int N, bool packed_s4, const OutputSpec& out) {
   if (out.no_split || out.ldc) return false;  // C is a block of a larger matrix
   if (g_swap_ab == 1) return false;
   if (g_swap_ab == 2) return true;
-  (void)packed_s4;
-  return M <= 32 && N >= 1024;
+  return N >= 1024 && M <= (packed_s4 ? 64 : 32);
 }
 
 // Returned (never to the caller of the library) when the fused INT4 kernel does not cover the
@@ -235,10 +235,10 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
       switch (cfg.bn) {
         case 256: return launch_variant<KIND, 256, 2, 1, 1, EPI, 2>(s, fb + 1, ta, tb, tc, p, stream);
         case 128: return launch_variant<KIND, 128, 3, 1, 1, EPI, 3>(s, fb + 2, ta, tb, tc, p, stream);
-        case 64: return launch_variant<KIND, 64, 3, 1, 1, EPI, 4>(s, fb + 3, ta, tb, tc, p, stream);
+        case 64: return launch_variant<KIND, 64, 4, 1, 1, EPI, 4>(s, fb + 3, ta, tb, tc, p, stream);
         case 32:
           if constexpr (EPI != EPI_OUT16)
-            return launch_variant<KIND, 32, 3, 1, 1, EPI, 5>(s, fb + 4, ta, tb, tc, p, stream);
+            return launch_variant<KIND, 32, 4, 1, 1, EPI, 5>(s, fb + 4, ta, tb, tc, p, stream);
           return GEMM_ERR_INVALID_ARG;
         default: return GEMM_ERR_INVALID_ARG;
       }

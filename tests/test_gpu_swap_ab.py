@@ -76,7 +76,9 @@ def test_automatic_choice_for_few_rows():
     binding.gemm_set_swap_ab(0)
     cfg = binding.gemm_query_config("s4", 16, 8192, 8192)
     assert "fused_unpack" in cfg and "swap_ab" in cfg
-    assert "swap_ab" not in binding.gemm_query_config("s4", 64, 8192, 8192)
+    assert "swap_ab" in binding.gemm_query_config("s4", 64, 8192, 8192)
+    assert "swap_ab" not in binding.gemm_query_config("s4", 128, 8192, 8192)
+    assert "swap_ab" not in binding.gemm_query_config("s8", 64, 8192, 8192)
     assert "swap_ab" in binding.gemm_query_config("s8", 16, 8192, 8192)
     assert "swap_ab" in binding.gemm_query_config("fp16", 16, 8192, 8192)
     assert "swap_ab" not in binding.gemm_query_config("fp16", 128, 8192, 8192)
