@@ -234,7 +234,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
         return launch_variant<KIND, 256, 4, 2, 1, EPI, 2>(s, fb + 0, ta, tb, tc, p, stream);
       switch (cfg.bn) {
         case 256: return launch_variant<KIND, 256, 2, 1, 1, EPI, 2>(s, fb + 1, ta, tb, tc, p, stream);
-        case 128: return launch_variant<KIND, 128, 3, 1, 1, EPI, 3>(s, fb + 2, ta, tb, tc, p, stream);
+        case 128: return launch_variant<KIND, 128, 4, 1, 1, EPI, 2>(s, fb + 2, ta, tb, tc, p, stream);
         case 64: return launch_variant<KIND, 64, 4, 1, 1, EPI, 4>(s, fb + 3, ta, tb, tc, p, stream);
         case 32:
           if constexpr (EPI != EPI_OUT16)
