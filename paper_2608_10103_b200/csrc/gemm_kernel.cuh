@@ -102,10 +102,9 @@ struct GemmParams {
   // 1: this grid was launched to start before the grid in front of it in the stream has
   // drained (programmatic dependent launch): its set-up overlaps that grid's tail, and whoever
   // touches global memory (the producer before its first load, the epilogue before its first
-  // store) waits for that grid first.  In front may be another GEMM of this library, which
-  // lets its successor start as soon as it runs itself, or (value 2) the kernel that zeroes C for
-  // split-K: that one starts only when everything in front of it has completed, so the operands
-  // are ready when this grid starts and only the epilogue has to wait.
+  // store) waits for that grid first.  In front may be another GEMM of this library or the
+  // kernel that zeroes C for split-K, both of which let their successor start as soon as they
+  // run themselves (and wait for their own predecessor in the same way).
   int wait_prior_grid;
   const float* row_scale;  // EPI_OUT16 (integer kinds) / EPI_F32_SCALED: M per-row factors
   const float* col_scale;  // and N per-column factors; both null = no scaling (FP16 kind)
@@ -347,7 +346,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       // issues the copies.  Nothing inside the loops is warp-collective, so a lane whose
       // wait gives up can leave on its own.
       const bool elected = ptx::elect_one();
-      if (p.wait_prior_grid == 1) ptx::grid_dep_wait();  // the operands may come from the grid in front
+      if (p.wait_prior_grid) ptx::grid_dep_wait();  // the operands may come from a grid in front
       int stage = 0;
       uint32_t phase = 0;
       int issued = 0;

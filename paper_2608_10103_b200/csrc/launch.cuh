@@ -11,12 +11,14 @@
 namespace b200gemm {
 namespace {
 
-// Zeroes C ahead of a split-K GEMM.  It lets the GEMM start at once (the GEMM waits for this
-// grid before its first global access), which takes the launch latency of the GEMM and the
-// gap between two dependent launches off the critical path of the small, latency-bound
-// problems that split K.
-__global__ void zero_c_kernel(uint4* c16, size_t n16, uint32_t* tail, int tail_words) {
+// Zeroes C ahead of a split-K GEMM.  Like the GEMMs it is launched to start early and lets its
+// successor start early: the launch latencies of the zeroing and of the GEMM behind it overlap
+// the tail of whatever runs in front, and each waits for its predecessor to complete before
+// it touches global memory -- which takes two launch gaps off the critical path of the small,
+// latency-bound problems that split K.
+__global__ void zero_c_kernel(uint4* c16, size_t n16, uint32_t* tail, int tail_words, int chained) {
   ptx::grid_dep_launch_dependents();
+  if (chained) ptx::grid_dep_wait();  // launched early itself: the grid in front may still use C
   const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
   for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n16; i += stride)
     c16[i] = make_uint4(0, 0, 0, 0);
@@ -190,11 +192,18 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
       size_t blocks = (n16 + 255) / 256;
       if (blocks > static_cast<size_t>(s->num_sms) * 4) blocks = static_cast<size_t>(s->num_sms) * 4;
       if (blocks < 1) blocks = 1;
-      zero_c_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-          static_cast<uint4*>(C), n16, reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(C) + n16 * 16),
-          static_cast<int>((bytes % 16) / 4));
-      e = cudaGetLastError();
-      if (p.wait_prior_grid) p.wait_prior_grid = 2;
+      cudaLaunchConfig_t zc = {};
+      zc.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+      zc.blockDim = dim3(256, 1, 1);
+      zc.stream = stream;
+      cudaLaunchAttribute za[1];
+      za[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      za[0].val.programmaticStreamSerializationAllowed = 1;
+      zc.attrs = za;
+      zc.numAttrs = p.wait_prior_grid ? 1 : 0;
+      e = cudaLaunchKernelEx(&zc, zero_c_kernel, static_cast<uint4*>(C), n16,
+                             reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(C) + n16 * 16),
+                             static_cast<int>((bytes % 16) / 4), p.wait_prior_grid);
     } else {
       int tm_lo = p.tiles_m, tm_hi = -1, tn_lo = p.tiles_n, tn_hi = -1;
       for (int t = p.split_from; t < p.tiles_m * p.tiles_n; ++t) {
