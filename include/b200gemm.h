@@ -347,6 +347,8 @@ int gemm_set_l2_policy(int policy);
  * cycles issuing loads [11]; fused INT4 only, one expansion warp: cycles
  * waiting for packed operands [12], for a free int8 slot [13] and spent
  * expanding [14]; [15] is unused.
+ * Traced launches run in plain stream order (no early start, see
+ * gemm_set_l2_policy bit 5), so that the cycle counts are the kernel's own.
  * gemm_trace_read synchronises the device, copies the words of the first
  * min(max_ctas, 160) CTAs of the last traced launch to `out` (host memory,
  * 16 * max_ctas words) and returns that CTA count.  Off by default; the cost

@@ -159,7 +159,9 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.split_from = p.tiles_m * p.tiles_n - (cfg.splits > 1 ? cfg.split_tiles : 0);
   p.ldc = ldc;
   p.transpose_c = swap ? 1 : 0;
-  p.wait_prior_grid = (g_l2_policy & 32) ? 0 : 1;  // policy bit 32: plain stream order
+  // policy bit 32: plain stream order; so are traced launches, whose cycle counts would
+  // otherwise include the time spent waiting for the predecessor's tail
+  p.wait_prior_grid = ((g_l2_policy & 32) || (g_trace_on & 1)) ? 0 : 1;
   p.c_vec_ok = !swap && (ldc % (16 / C_ELEM) == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
   CUtensorMap tc;
   if (p.c_vec_ok) {
