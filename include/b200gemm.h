@@ -328,7 +328,10 @@ int gemm_set_swap_ab(int mode);
  * load and its first store; a GEMM of this library lets its successor begin as
  * soon as it runs itself.  Stream semantics are unchanged; back-to-back small
  * GEMMs get 15-25 % faster (N = 512: 5.1 -> 4.0 us).  Default 11 = 3 + 8 with
- * the serpentine order on, which gave the lowest DRAM traffic at N = 8192.  Integer results never depend on any of
+ * the serpentine order on, which gave the lowest DRAM traffic at N = 8192; with
+ * the default, problems that are one tile wide or one tile tall (few rows on one
+ * side) use 2 for bits 0-1, so that the short operand every CTA re-reads is not
+ * pushed out of L2 by the long one streaming past.  Integer results never depend on any of
  * this; FP16 results may differ in the last bits (summation order) within the
  * bound.
  */
