@@ -117,7 +117,11 @@ int gemm_s4_ws(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t*
  * accumulators; here only the stored result is narrowed, so the error is the
  * FP32 path's plus one half-precision rounding.)  C: M x N binary16, row-major.
  * Alignment as gemm_fp16; rows of C that are not 16-byte multiples (N % 8 != 0)
- * take a slower scalar store path.
+ * take a slower scalar store path.  A 16-bit (or scaled) result cannot be
+ * accumulated in C, so where the plain GEMMs split K over CTAs that add into C,
+ * this entry point and the dequantising ones split K between the two CTAs of a
+ * cluster, which hand partial sums over through shared memory (narrow one-CTA
+ * tiles, factor 2: M = 16, N = 4096, K = 16384: 48.8 -> 39.3 us).
  */
 int gemm_fp16_f16out(int M, int N, int K, const void* A, const void* B, void* C,
                      gemm_stream_t stream);
@@ -331,7 +335,8 @@ int gemm_set_swap_ab(int mode);
  * the serpentine order on, which gave the lowest DRAM traffic at N = 8192; with
  * the default, problems that are one tile wide or one tile tall (few rows on one
  * side) use 2 for bits 0-1, so that the short operand every CTA re-reads is not
- * pushed out of L2 by the long one streaming past.  Integer results never depend on any of
+ * pushed out of L2 by the long one streaming past.  Bit 6 (64): no split-K
+ * inside a cluster (see gemm_fp16_f16out / the dequantising entry points).  Integer results never depend on any of
  * this; FP16 results may differ in the last bits (summation order) within the
  * bound.
  */
@@ -350,7 +355,8 @@ int gemm_set_l2_policy(int policy);
  * cycles issuing loads [11]; fused INT4 only, one expansion warp: cycles
  * waiting for packed operands [12], for a free int8 slot [13] and spent
  * expanding [14]; [15] is unused.
- * Traced launches run in plain stream order (no early start, see
+ * Switching recording on (bit 1 from 0 to 1) synchronises the device and clears
+ * all records.  Traced launches run in plain stream order (no early start, see
  * gemm_set_l2_policy bit 5), so that the cycle counts are the kernel's own.
  * gemm_trace_read synchronises the device, copies the words of the first
  * min(max_ctas, 160) CTAs of the last traced launch to `out` (host memory,

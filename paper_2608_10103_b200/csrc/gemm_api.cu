@@ -193,7 +193,7 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
   const long long units = num_sms / c.cta_group;
   snprintf(buf, static_cast<size_t>(len),
            "BM=%d BN=%d BK=%d cta_group=%d stages=%d group_m=%d split_k=%d split_tiles=%d "
-           "tiles=%lld ctas=%lld kind=%s%s%s",
+           "tiles=%lld ctas=%lld kind=%s%s%s%s",
            BM * c.cta_group, c.bn, atoms_for(c.bn, c.cta_group) * BK_BYTES / elem, c.cta_group,
            c.stages, c.group_m, c.splits, c.splits > 1 ? c.split_tiles : 0, tiles,
            (tiles + (c.splits > 1 ? static_cast<long long>(c.split_tiles) * (c.splits - 1) : 0) <
@@ -203,7 +203,8 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
                c.cta_group,
            precision == GEMM_PREC_FP16 ? "f16" : "i8",
            precision != GEMM_PREC_S4 ? "" : fused ? " s4=fused_unpack" : " prepass=unpack_s4",
-           swap ? " swap_ab" : "");
+           swap ? " swap_ab" : "",
+           "");  // (the raw outputs this function describes never split inside a cluster)
   return GEMM_OK;
 }
 
@@ -259,7 +260,7 @@ int gemm_set_swap_ab(int mode) {
 }
 
 int gemm_set_l2_policy(int policy) {
-  if (policy < 0 || policy > 63) return GEMM_ERR_INVALID_ARG;
+  if (policy < 0 || policy > 127) return GEMM_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
   g_l2_policy = policy;
   return GEMM_OK;
@@ -267,6 +268,16 @@ int gemm_set_l2_policy(int policy) {
 
 int gemm_trace_enable(int on) {
   std::lock_guard<std::mutex> lock(g_mutex);
+  if ((on & 1) && !(g_trace_on & 1)) {
+    // recording starts: clear the records, so that CTAs a later launch does not have read 0
+    DeviceState* s = nullptr;
+    int rc = device_state(&s);
+    if (rc != GEMM_OK) return rc;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess)
+      e = cudaMemset(s->trace_ptr, 0, sizeof(unsigned long long) * TRACE_SLOTS * TRACE_MAX_CTAS);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
   g_trace_on = on & 63;
   return GEMM_OK;
 }

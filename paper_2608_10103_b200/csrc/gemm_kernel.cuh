@@ -151,7 +151,7 @@ enum TraceSlot {
 // bytes of K in the 128-byte-swizzle layout (the widest a swizzled TMA box can
 // be).  KB = 2 halves the per-slot barrier work (one wait, one commit per 8 MMAs)
 // of the single issuing thread, whose instruction time is the scarce resource.
-template <int BN, int STAGES, int CTA_GROUP, int KB, int PSTAGES = 0>
+template <int BN, int STAGES, int CTA_GROUP, int KB, int PSTAGES = 0, int CSPLIT = 1>
 struct SmemLayout {
   static constexpr int B_ROWS = BN / CTA_GROUP;  // B rows each CTA loads
   static constexpr int A_BYTES = BM * BK_BYTES;       // one A atom
@@ -165,10 +165,15 @@ struct SmemLayout {
   static constexpr int EPI_BUF_BYTES = 32 * 128;
   static constexpr int EPI_OFFSET = RING_BYTES;
   static constexpr int EPI_BYTES = EPI_WARPS * 2 * EPI_BUF_BYTES;
-  static constexpr int BAR_OFFSET = EPI_OFFSET + EPI_BYTES;
+  // Cluster split-K: the CTA of cluster rank 0 receives the other CTA's 128 x BN partial
+  // accumulators (32-bit) here.
+  static constexpr int X_OFFSET = EPI_OFFSET + EPI_BYTES;
+  static constexpr int X_BYTES = CSPLIT > 1 ? BM * BN * 4 : 0;
+  static constexpr int BAR_OFFSET = X_OFFSET + X_BYTES;
   // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], drain, p_full[PSTAGES], p_empty[PSTAGES]
-  // fused INT4 adds ready[STAGES]
-  static constexpr int NUM_BARS = 2 * STAGES + 5 + 2 * PSTAGES + (PSTAGES > 0 ? STAGES : 0);
+  // fused INT4 adds ready[STAGES]; cluster split-K adds part_full, part_free
+  static constexpr int NUM_BARS =
+      2 * STAGES + 5 + 2 * PSTAGES + (PSTAGES > 0 ? STAGES : 0) + (CSPLIT > 1 ? 2 : 0);
   static constexpr int MISC_OFFSET = BAR_OFFSET + NUM_BARS * 8;
   static constexpr int TOTAL = MISC_OFFSET + 16;
   static constexpr int DYN_BYTES = TOTAL + 1024;  // slack to align the ring to 1024 bytes
@@ -178,15 +183,19 @@ struct SmemLayout {
 
 // Bounded wait: polls the barrier; after the limit (or once another role has
 // given up) records `code` and returns false.  The caller then leaves its loop.
-template <bool BACKOFF = false>
+template <bool BACKOFF = false, bool ACQUIRE_CLUSTER = false>
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity,
                                              volatile uint32_t* abort_flag, int* status, int code,
                                              uint32_t backoff_ns = 0) {
-  if (ptx::mbar_try_wait(bar, parity)) return true;
+  auto done = [&]() {
+    if constexpr (ACQUIRE_CLUSTER) return ptx::mbar_try_wait_acquire_cluster(bar, parity);
+    return ptx::mbar_try_wait(bar, parity);
+  };
+  if (done()) return true;
   uint64_t t0 = 0;
   uint32_t spins = 0;
   while (true) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if (done()) return true;
     if (BACKOFF && backoff_ns) __nanosleep(backoff_ns);
     if ((++spins & 255u) == 0) {
       if (*abort_flag) return false;
@@ -227,12 +236,20 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32, int PSTAGES = 0>
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32, int PSTAGES = 0,
+          int CSPLIT = 1>
 __global__ void __launch_bounds__(PSTAGES > 0 ? NUM_THREADS_FUSED : NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
-  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES>;
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, CSPLIT>;
   constexpr bool FUSED = PSTAGES > 0;  // packed INT4 operands, expanded on the way to the MMAs
+  // CSPLIT = 2 (cluster split-K): a cluster of two single CTAs owns every tile; each takes half
+  // of K into its own accumulator, the CTA of rank 1 hands its 128 x BN partial sums to rank 0
+  // through the cluster's shared-memory window, and rank 0 adds them to its own on the way
+  // out.  Unlike split-K through C this needs no zeroed C and no adds in global memory, so it
+  // also serves the 16-bit and scaled outputs, and a call is a single launch.
+  static_assert(CSPLIT == 1 || (CSPLIT == 2 && CTA_GROUP == 1 && !FUSED && BN <= 64),
+                "cluster split-K: two single CTAs, narrow tile");
   static_assert(!FUSED || (KIND == ptx::KIND_I8 && KB == 1 && STAGES >= 2),
                 "fused INT4: int8 MMAs, one atom per slot, a packed slot fills two int8 slots at once");
   constexpr int ELEM_BYTES = (KIND == ptx::KIND_F16) ? 2 : 1;
@@ -262,6 +279,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   // arrive with release semantics straight from the writing warps costs each of them
   // hundreds of cycles).
   auto ready_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 5 + 2 * PSTAGES + s); };
+  // cluster split-K: `part_full` lives in rank 0 (rank 1's partial sums of a tile have landed),
+  // `part_free` in rank 1 (rank 0 has consumed them, the buffer may be overwritten)
+  const uint32_t part_full_bar = bar0 + 8u * (L::NUM_BARS - 2);
+  const uint32_t part_free_bar = bar0 + 8u * (L::NUM_BARS - 1);
   volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(base_ptr + L::MISC_OFFSET);
   volatile uint32_t* abort_flag = tmem_holder + 1;
 
@@ -269,6 +290,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   const int lane = threadIdx.x & 31;
   const uint32_t cta_rank = (CTA_GROUP == 2) ? ptx::cluster_ctarank() : 0u;
   const bool leader = (cta_rank == 0);
+  const uint32_t krank = (CSPLIT > 1) ? ptx::cluster_ctarank() : 0u;  // which part of K this CTA takes
   // Work units (`num_tiles` counts units): unit u < split_from is the whole tile u; the
   // remaining tiles are each covered by `splits` units, one per K range.
   const int real_tiles = p.tiles_m * p.tiles_n;
@@ -280,7 +302,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                                 : (k_slots_all + p.splits - 1) / p.splits;
   // unit -> tile, K range (in ring slots) and whether its result is added into C
   auto decode_unit = [&](int u, int& tile, int& k_begin, int& k_end, bool& add) {
-    if (u < p.split_from) {
+    if constexpr (CSPLIT > 1) {  // every unit is a whole tile; K is divided inside the cluster
+      const int per = (k_slots_all + CSPLIT - 1) / CSPLIT;
+      tile = u;
+      k_begin = static_cast<int>(krank) * per;
+      k_end = min(k_begin + per, k_slots_all);
+      add = false;
+    } else if (u < p.split_from) {
       tile = u;
       k_begin = 0;
       k_end = k_slots_all;
@@ -293,8 +321,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       add = p.splits > 1;
     }
   };
-  const int first_tile = static_cast<int>(blockIdx.x) / CTA_GROUP;
-  const int tile_stride = static_cast<int>(gridDim.x) / CTA_GROUP;
+  const int first_tile = static_cast<int>(blockIdx.x) / (CTA_GROUP * CSPLIT);
+  const int tile_stride = static_cast<int>(gridDim.x) / (CTA_GROUP * CSPLIT);
   unsigned long long* const trace =
       p.trace ? p.trace + static_cast<size_t>(blockIdx.x) * TRACE_SLOTS : nullptr;
   if (trace && threadIdx.x < TRACE_SLOTS) trace[threadIdx.x] = 0;  // roles that do not run leave 0
@@ -317,6 +345,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::mbar_init(acc_empty_bar(a), EPI_WARPS * CTA_GROUP);
     }
     ptx::mbar_init(drain_bar, 1);
+    if constexpr (CSPLIT > 1) {
+      ptx::mbar_init(part_full_bar, EPI_WARPS);
+      ptx::mbar_init(part_free_bar, EPI_WARPS);
+    }
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmap_a);
@@ -328,7 +360,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     ptx::tmem_relinquish<CTA_GROUP>();
   }
   ptx::tc_fence_before_sync();
-  if constexpr (CTA_GROUP == 2) {
+  if constexpr (CTA_GROUP == 2 || CSPLIT > 1) {
     ptx::cluster_sync();  // the peer's barriers must exist before anything signals them
   } else {
     __syncthreads();
@@ -686,6 +718,32 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     long long epi_wait = 0, epi_busy = 0, tiles_done = 0;
     uint32_t staged_blocks = 0;  // blocks sent through the staging buffers so far
     bool prior_grid_done = false;
+    uint32_t xphase = 0;         // cluster split-K: parity of the partial-sum hand-over
+    const bool xpeer = CSPLIT > 1 && krank != 0;  // this CTA only contributes partial sums
+    // Cluster split-K, rank 0: adds the other CTA's partial sums for accumulator columns
+    // [32 * b32, 32 * b32 + 32) of this thread's row to the 32 raw accumulators in r.
+    auto add_partial = [&](uint32_t (&r)[32], int b32) {
+      if constexpr (CSPLIT > 1) {
+        const uint32_t xsrc = base + L::X_OFFSET +
+                              static_cast<uint32_t>(quarter * (32 * BN * 4) + b32 * 4096 + lane * 128);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          uint32_t t0, t1, t2, t3;
+          ptx::ld_shared_v4(xsrc + static_cast<uint32_t>(((j ^ (lane & 7)) * 16)), t0, t1, t2, t3);
+          if constexpr (KIND == ptx::KIND_F16) {
+            r[4 * j + 0] = __float_as_uint(__uint_as_float(r[4 * j + 0]) + __uint_as_float(t0));
+            r[4 * j + 1] = __float_as_uint(__uint_as_float(r[4 * j + 1]) + __uint_as_float(t1));
+            r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + __uint_as_float(t2));
+            r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + __uint_as_float(t3));
+          } else {
+            r[4 * j + 0] += t0;
+            r[4 * j + 1] += t1;
+            r[4 * j + 2] += t2;
+            r[4 * j + 3] += t3;
+          }
+        }
+      }
+    };
     for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
       int tm, tn, tile, k_begin, k_end;
       bool add;
@@ -699,6 +757,38 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       epi_wait += w1 - w0;
       if (!ok) break;
       ptx::tc_fence_after_sync();
+      if constexpr (CSPLIT > 1) {
+        if (xpeer) {
+          // Rank 1: once rank 0 has consumed the previous tile's partial sums, write this
+          // tile's (raw 32-bit accumulators, one 128-byte row piece per thread and 32 columns,
+          // swizzled like the staging buffers) into rank 0's shared memory and tell it.
+          ok = wait_bounded<false, true>(part_free_bar, xphase ^ 1u, abort_flag, p.status,
+                                         DEV_TIMEOUT_EPILOGUE);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          const uint32_t xdst = ptx::map_to_cta(base + L::X_OFFSET, 0) +
+                                static_cast<uint32_t>(quarter * (32 * BN * 4) + lane * 128);
+#pragma unroll 1
+          for (int b = 0; b < BN / 32; ++b) {
+            uint32_t r[32];
+            ptx::tmem_ld_32x32b_x32(tmem_base + lane_base + static_cast<uint32_t>(acc * BN + b * 32), r);
+            ptx::tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              ptx::st_shared_cluster_v4(xdst + static_cast<uint32_t>(b * 4096 + ((j ^ (lane & 7)) * 16)),
+                                        r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+          }
+          ptx::fence_acq_rel_cluster();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_release_cluster(ptx::map_to_cta(part_full_bar, 0));
+        } else {
+          ok = wait_bounded<false, true>(part_full_bar, xphase, abort_flag, p.status,
+                                         DEV_TIMEOUT_EPILOGUE);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+        }
+        xphase ^= 1u;
+      }
       // A split-K unit whose K range is empty (the host never creates one) contributes nothing.
       const bool empty_range = k_begin >= k_end;
       if (p.wait_prior_grid && !prior_grid_done) {  // C may be read, written or zeroed by the grid in front
@@ -719,13 +809,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       constexpr int BLOCK_COLS = (EPI == EPI_OUT16) ? 64 : 32;
       static_assert(BN % BLOCK_COLS == 0, "tile width must be a multiple of the store block");
 #pragma unroll 1
-      for (int c = 0; c < BN / BLOCK_COLS; ++c) {
+      for (int c = 0; c < BN / BLOCK_COLS && !xpeer; ++c) {
         const int col = col0 + c * BLOCK_COLS;
         uint32_t w[32];  // the thread's 128 bytes of output
         if constexpr (EPI == EPI_RAW32) {
           ptx::tmem_ld_32x32b_x32(
               tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), w);
           ptx::tmem_wait_ld();
+          add_partial(w, c);
           if constexpr (FUSED) {
 #pragma unroll
             for (int v = 0; v < 32; ++v) w[v] = fix(w[v]);
@@ -734,6 +825,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           ptx::tmem_ld_32x32b_x32(
               tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), w);
           ptx::tmem_wait_ld();
+          add_partial(w, c);
 #pragma unroll
           for (int v = 0; v < 32; ++v) {
             const float cs = (col + v < p.N) ? __ldg(p.col_scale + col + v) : 0.0f;
@@ -746,6 +838,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             ptx::tmem_ld_32x32b_x32(
                 tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 64 + h * 32), r);
             ptx::tmem_wait_ld();
+            add_partial(r, c * 2 + h);
 #pragma unroll
             for (int v = 0; v < 32; v += 2) {
               float x0 = acc_to_float<KIND>(fix(r[v])), x1 = acc_to_float<KIND>(fix(r[v + 1]));
@@ -831,6 +924,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           }
         }
       }
+      if constexpr (CSPLIT > 1) {
+        if (!xpeer) {  // the partial sums have been read: rank 1 may send the next tile's
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_release_cluster(ptx::map_to_cta(part_free_bar, 1));
+        }
+      }
       // Hand the accumulator buffer back to the (leader's) MMA issuer.
       ptx::tc_fence_before_sync();
       __syncwarp();
@@ -864,7 +963,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   // Teardown: every role gets here (all waits are bounded).  In a pair neither
   // CTA may release TMEM or exit while the other can still touch its memory.
   ptx::tc_fence_before_sync();
-  if constexpr (CTA_GROUP == 2) {
+  if constexpr (CTA_GROUP == 2 || CSPLIT > 1) {
     __syncwarp();
     ptx::cluster_sync();
   } else {

@@ -25,11 +25,12 @@ __global__ void zero_c_kernel(uint4* c16, size_t n16, uint32_t* tail, int tail_w
   if (blockIdx.x == 0 && static_cast<int>(threadIdx.x) < tail_words) tail[threadIdx.x] = 0;
 }
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI, int PSTAGES = 0>
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI, int PSTAGES = 0,
+          int CSPLIT = 1>
 int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUtensorMap& tb,
                    const CUtensorMap& tc, const GemmParams& p, cudaStream_t stream) {
-  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES>;
-  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI, PSTAGES>;
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, CSPLIT>;
+  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI, PSTAGES, CSPLIT>;
   if (!(s->attr_set[variant >> 6] & (1ull << (variant & 63)))) {
     cudaError_t e =
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
@@ -38,8 +39,9 @@ int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUt
   }
   const long long all_tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   const long long tiles = p.split_from + (all_tiles - p.split_from) * p.splits;  // work units
-  const long long units = s->num_sms / CTA_GROUP;
-  const int grid = static_cast<int>((tiles < units ? tiles : units) * CTA_GROUP);
+  constexpr int CLUSTER = CTA_GROUP * CSPLIT;  // CTAs that work on one unit together
+  const long long units = s->num_sms / CLUSTER;
+  const int grid = static_cast<int>((tiles < units ? tiles : units) * CLUSTER);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid, 1, 1);
   cfg.blockDim = dim3(PSTAGES > 0 ? NUM_THREADS_FUSED : NUM_THREADS, 1, 1);
@@ -47,7 +49,7 @@ int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUt
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = CTA_GROUP;
+  attr[0].val.clusterDim.x = CLUSTER;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -67,6 +69,12 @@ struct OutputSpec {
   long long ldc = 0;        // row pitch of C in elements; 0 = dense (N)
   bool no_split = false;    // C is a block of a larger matrix: never zero / add into it
 };
+
+// Whether the selector's choice can run as split-K inside a cluster of two CTAs.
+bool cluster_split_ok(const TileConfig& c, int M, int N) {
+  const long long tiles = static_cast<long long>(ceil_div(M, BM * c.cta_group)) * ceil_div(N, c.bn);
+  return c.cta_group == 1 && c.bn <= 64 && c.splits == 2 && c.split_tiles == tiles;
+}
 
 // Whether the packed route is taken for the tile the selector picked.  Scheme 2 forces it
 // wherever a variant exists; scheme 0 (automatic) takes it where a pre-pass over the operands
@@ -128,9 +136,24 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
       (KIND == ptx::KIND_F16) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
   // the selector sees the int8 problem either way, so both INT4 routes get the same tile
   int k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
-  const TileConfig cfg = select_config(M, N, s->num_sms, k_blocks, EPI == EPI_OUT16 ? 64 : 32,
-                                       EPI == EPI_RAW32 && !out.no_split, packed_s4 ? 2 : 0);
+  const int min_bn = EPI == EPI_OUT16 ? 64 : 32;
+  const bool split_through_c = EPI == EPI_RAW32 && !out.no_split;
+  TileConfig cfg =
+      select_config(M, N, s->num_sms, k_blocks, min_bn, split_through_c, packed_s4 ? 2 : 0);
   if (cfg.bn == 0) return GEMM_ERR_INVALID_ARG;  // override asks for a shape this mode lacks
+  // Outputs that cannot be split through C (16-bit, scaled, blocks of a larger C): split-K
+  // inside a cluster of two CTAs where the kernel has that variant (one-CTA tiles up to 64
+  // wide, every tile split in two) -- no zeroing of C, no adds in global memory.  Where the
+  // raw 32-bit output can split through C that stays the choice: with the launches chained it
+  // measured ~1 us faster per call than the hand-over inside the cluster.
+  bool csplit = false;
+  if (!packed_s4 && !split_through_c && !(g_l2_policy & 64)) {
+    const TileConfig c2 = select_config(M, N, s->num_sms, k_blocks, min_bn, true, 0, 2);
+    if (c2.bn != 0 && cluster_split_ok(c2, M, N)) {
+      cfg = c2;
+      csplit = true;
+    }
+  }
   if (packed_s4) {
     if (KIND != ptx::KIND_I8 || !fused_s4_variant_exists(cfg.bn, cfg.cta_group, cfg.splits) ||
         !s4_fused_wanted(user_m, user_n, cfg, s->num_sms))
@@ -155,8 +178,8 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.tiles_n = ceil_div(N, cfg.bn);
   p.group_m = cfg.group_m;
   p.k_blocks = k_blocks;
-  p.splits = cfg.splits;
-  p.split_from = p.tiles_m * p.tiles_n - (cfg.splits > 1 ? cfg.split_tiles : 0);
+  p.splits = csplit ? 1 : cfg.splits;
+  p.split_from = p.tiles_m * p.tiles_n - ((cfg.splits > 1 && !csplit) ? cfg.split_tiles : 0);
   p.ldc = ldc;
   p.transpose_c = swap ? 1 : 0;
   // policy bit 32: plain stream order; so are traced launches, whose cycle counts would
@@ -190,7 +213,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.serpentine_k = (g_l2_policy & 4) ? 0 : 1;
   p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
 
-  if (cfg.splits > 1) {  // only with a dense C (no_split is set for blocks of a larger matrix)
+  if (cfg.splits > 1 && !csplit) {  // only with a dense C (no_split is set for blocks of a larger matrix)
     // Split tiles add into C: zero them first.  All tiles: one memset.  The last wave only:
     // the bounding rectangle of those tiles (other tiles inside it are overwritten later).
     cudaError_t e;
@@ -240,6 +263,14 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
                             static_cast<size_t>(row_hi - row_lo), stream);
     }
     if (e != cudaSuccess) return cuda_fail(e);
+  }
+  if (csplit) {  // attr_set bits 96..: kind, output mode, width
+    const int cb = 96 + ((KIND == ptx::KIND_F16) ? 0 : 16) + EPI * 2;
+    if (cfg.bn == 64)
+      return launch_variant<KIND, 64, 3, 1, 2, EPI, 0, 2>(s, cb + 1, ta, tb, tc, p, stream);
+    if constexpr (EPI != EPI_OUT16)
+      return launch_variant<KIND, 32, 4, 1, 2, EPI, 0, 2>(s, cb, ta, tb, tc, p, stream);
+    return GEMM_ERR_INVALID_ARG;
   }
   const int vbase = ((KIND == ptx::KIND_F16) ? 0 : 32) + EPI * 8;  // bit index in attr_set
   if (packed_s4) {

@@ -59,8 +59,9 @@ int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b
 // cluster launch (~2500) are paid once; split-K adds zeroing C and adding into it.
 // force_atoms: K atoms per split unit whatever the tile (the fused INT4 kernel splits K in
 // packed slots = 2 int8 k-blocks); 0 = the tile's own ring slot.
+// split_cap: upper limit of the split-K factor (0 = none).
 TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 32,
-                         bool allow_split = false, int force_atoms = 0) {
+                         bool allow_split = false, int force_atoms = 0, int split_cap = 0) {
   TileConfig best{256, 2, 6, 8, 1, 0};
   long long best_cost = -1;
   for (int cg = 2; cg >= 1; --cg) {
@@ -77,6 +78,7 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
         max_split = static_cast<int>(units / tiles);
         if (max_split > k_blocks / 2) max_split = k_blocks / 2;  // at least 2 k-blocks each
         if (max_split > 32) max_split = 32;
+        if (split_cap && max_split > split_cap) max_split = split_cap;
         if (max_split < 1) max_split = 1;
       }
       if (g_override_splits) {

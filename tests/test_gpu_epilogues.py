@@ -170,3 +170,60 @@ def test_dequant_argument_errors():
     assert L.gemm_s8_dequant(64, 64, 24, p, p, s, s, c, 0, None) == -2
     assert L.gemm_s4_dequant(64, 64, 48, p, p, s, s, c, 0, None) == -2
     assert L.gemm_fp16_f16out(64, 64, 12, p, p, c, None) == -2
+
+
+# ------------------------------------------------ split-K inside a cluster of two CTAs
+def _ctas_of_last_launch():
+    return sum(1 for t in binding.gemm_trace_read(160) if t["cycles"] > 0)
+
+
+@pytest.mark.parametrize("swap", [1, 2])
+@pytest.mark.parametrize("M,N,K,bn,tiles", [(16, 2048, 4096, 64, 16), (1, 1030, 2080, 64, 9),
+                                            (40, 12800, 1056, 64, 100), (24, 640, 8192, 32, 5)])
+def test_cluster_split_k_for_16_bit_and_scaled_outputs(M, N, K, bn, tiles, swap):
+    """The outputs that cannot be split through C (binary16, dequantised) split K between the
+    two CTAs of a cluster, which exchange partial sums through shared memory: twice as many
+    CTAs as tiles work on the problem (checked through the cycle-accounting records), also when
+    a cluster has several tiles in a row (100 tiles on 74 clusters) and the hand-over buffer is
+    reused."""
+    binding.gemm_set_swap_ab(swap)
+    try:
+        kernel_tiles = tiles if swap == 2 else -(-M // 128) * -(-N // bn)
+        binding.gemm_set_config_override(bn, 0, 1, 2)
+        g = np.random.Generator(np.random.PCG64(M + N))
+        rs = (g.uniform(0.5, 2.0, M) * 1e-2).astype(np.float32)
+        cs = (g.uniform(0.5, 2.0, N) * 1e-1).astype(np.float32)
+        A, B = synth.s8_uniform(M, N, K, seed=M)
+        ref = oracle.dequant_ref(oracle.gemm_s8_i64(A, B), rs, cs)
+        for out_dtype in ((torch.float32, torch.float16) if bn == 64 else (torch.float32,)):
+            binding.gemm_trace_enable(1)
+            got = run_dequant("s8", A, B, rs, cs, out_dtype)
+            ctas = _ctas_of_last_launch()
+            binding.gemm_trace_enable(0)
+            assert ctas == min(2 * kernel_tiles, 148), (ctas, kernel_tiles)
+            ok, worst = oracle.dequant_check(got, ref, out_dtype == torch.float16)
+            assert ok, "%s: %.3g x bound" % (out_dtype, worst)
+        if bn == 64:
+            A, B = synth.fp16_normal_clipped(M, N, K, seed=N)
+            ref, S = oracle.gemm_fp16(A, B)
+            for rep in range(2):
+                ok, worst = oracle.fp16_out_check(run_f16out(A, B), ref, S)
+                assert ok, "fp16 out: %.3g x bound" % worst
+    finally:
+        binding.gemm_set_swap_ab(0)
+        binding.gemm_trace_enable(0)
+
+
+def test_cluster_split_k_is_the_automatic_choice_for_few_rows():
+    M, N, K = 16, 4096, 8192                      # 32 kernel tiles for 148 SMs
+    A, B = synth.s8_uniform(M, N, K, seed=77)
+    g = np.random.Generator(np.random.PCG64(77))
+    rs = (g.uniform(0.5, 2.0, M) * 1e-2).astype(np.float32)
+    cs = (g.uniform(0.5, 2.0, N) * 1e-1).astype(np.float32)
+    ref = oracle.dequant_ref(oracle.gemm_s8_i64(A, B), rs, cs)
+    binding.gemm_trace_enable(1)
+    got = run_dequant("s8", A, B, rs, cs, torch.float16)
+    ctas = _ctas_of_last_launch()
+    binding.gemm_trace_enable(0)
+    assert ctas == 64, ctas
+    assert oracle.dequant_check(got, ref, True)[0]
