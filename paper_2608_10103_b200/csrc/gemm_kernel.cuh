@@ -248,7 +248,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   // through the cluster's shared-memory window, and rank 0 adds them to its own on the way
   // out.  Unlike split-K through C this needs no zeroed C and no adds in global memory, so it
   // also serves the 16-bit and scaled outputs, and a call is a single launch.
-  static_assert(CSPLIT == 1 || (CSPLIT == 2 && CTA_GROUP == 1 && !FUSED && BN <= 64),
+  static_assert(CSPLIT == 1 || (CSPLIT == 2 && CTA_GROUP == 1 && BN <= 64),
                 "cluster split-K: two single CTAs, narrow tile");
   static_assert(!FUSED || (KIND == ptx::KIND_I8 && KB == 1 && STAGES >= 2),
                 "fused INT4: int8 MMAs, one atom per slot, a packed slot fills two int8 slots at once");
@@ -303,7 +303,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   // unit -> tile, K range (in ring slots) and whether its result is added into C
   auto decode_unit = [&](int u, int& tile, int& k_begin, int& k_end, bool& add) {
     if constexpr (CSPLIT > 1) {  // every unit is a whole tile; K is divided inside the cluster
-      const int per = (k_slots_all + CSPLIT - 1) / CSPLIT;
+      // (fused INT4: in whole packed slots = pairs of int8 slots)
+      const int per = FUSED ? 2 * ((k_slots_all / 2 + CSPLIT - 1) / CSPLIT)
+                            : (k_slots_all + CSPLIT - 1) / CSPLIT;
       tile = u;
       k_begin = static_cast<int>(krank) * per;
       k_end = min(k_begin + per, k_slots_all);

@@ -147,15 +147,17 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   // raw 32-bit output can split through C that stays the choice: with the launches chained it
   // measured ~1 us faster per call than the hand-over inside the cluster.
   bool csplit = false;
-  if (!packed_s4 && !split_through_c && !(g_l2_policy & 64)) {
-    const TileConfig c2 = select_config(M, N, s->num_sms, k_blocks, min_bn, true, 0, 2);
+  if (!split_through_c && !(g_l2_policy & 64)) {
+    const TileConfig c2 =
+        select_config(M, N, s->num_sms, k_blocks, min_bn, true, packed_s4 ? 2 : 0, 2);
     if (c2.bn != 0 && cluster_split_ok(c2, M, N)) {
       cfg = c2;
       csplit = true;
     }
   }
   if (packed_s4) {
-    if (KIND != ptx::KIND_I8 || !fused_s4_variant_exists(cfg.bn, cfg.cta_group, cfg.splits) ||
+    if (KIND != ptx::KIND_I8 ||
+        !(csplit || fused_s4_variant_exists(cfg.bn, cfg.cta_group, cfg.splits)) ||
         !s4_fused_wanted(user_m, user_n, cfg, s->num_sms))
       return GEMM_NOT_FUSED;
     k_blocks = 2 * ceil_div(K, 2 * BK_BYTES);  // one packed slot (256 values of K) = two int8 slots
@@ -263,6 +265,16 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
                             static_cast<size_t>(row_hi - row_lo), stream);
     }
     if (e != cudaSuccess) return cuda_fail(e);
+  }
+  if (csplit && packed_s4) {  // attr_set bits 128..
+    if constexpr (KIND == ptx::KIND_I8) {
+      const int cb = 128 + EPI * 2;
+      if (cfg.bn == 64)
+        return launch_variant<KIND, 64, 4, 1, 1, EPI, 2, 2>(s, cb + 1, ta, tb, tc, p, stream);
+      if constexpr (EPI != EPI_OUT16)
+        return launch_variant<KIND, 32, 4, 1, 1, EPI, 4, 2>(s, cb, ta, tb, tc, p, stream);
+    }
+    return GEMM_ERR_INVALID_ARG;
   }
   if (csplit) {  // attr_set bits 96..: kind, output mode, width
     const int cb = 96 + ((KIND == ptx::KIND_F16) ? 0 : 16) + EPI * 2;

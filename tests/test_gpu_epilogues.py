@@ -227,3 +227,32 @@ def test_cluster_split_k_is_the_automatic_choice_for_few_rows():
     binding.gemm_trace_enable(0)
     assert ctas == 64, ctas
     assert oracle.dequant_check(got, ref, True)[0]
+
+
+@pytest.mark.parametrize("scheme", [1, 2])
+@pytest.mark.parametrize("M,N,K,bn", [(16, 2048, 4096, 64), (24, 640, 8192, 32), (40, 12800, 1056, 64)])
+def test_cluster_split_k_dequantised_int4(M, N, K, bn, scheme):
+    """The same for packed INT4 operands, on the pre-pass route (INT8 kernel) and on the fused
+    route (nibbles expanded inside the kernel, K divided in whole packed slots)."""
+    binding.gemm_set_swap_ab(2)
+    binding.gemm_set_s4_scheme(scheme)
+    try:
+        binding.gemm_set_config_override(bn, 0, 1, 2)
+        g = np.random.Generator(np.random.PCG64(M + N))
+        rs = (g.uniform(0.5, 2.0, M) * 1e-2).astype(np.float32)
+        cs = (g.uniform(0.5, 2.0, N) * 1e-1).astype(np.float32)
+        A, B = synth.s4_uniform(M, N, K, seed=M)
+        ref = oracle.dequant_ref(oracle.gemm_s4_i64(A, B, K), rs, cs)
+        kernel_tiles = -(-N // 128)
+        for out_dtype in ((torch.float32, torch.float16) if bn == 64 else (torch.float32,)):
+            binding.gemm_trace_enable(1)
+            got = run_dequant("s4", A, B, rs, cs, out_dtype)
+            ctas = _ctas_of_last_launch()
+            binding.gemm_trace_enable(0)
+            assert ctas == min(2 * kernel_tiles, 148), (ctas, kernel_tiles)
+            ok, worst = oracle.dequant_check(got, ref, out_dtype == torch.float16)
+            assert ok, "%s: %.3g x bound" % (out_dtype, worst)
+    finally:
+        binding.gemm_set_swap_ab(0)
+        binding.gemm_set_s4_scheme(0)
+        binding.gemm_trace_enable(0)
