@@ -40,7 +40,7 @@ KERNEL_LAUNCHES = {"fp16": 1, "s8": 1, "s4": 2}            # s4: unpack launch +
 # DRAM bytes per launch of the FP16 GEMM kernel (dram__bytes_read.sum + dram__bytes_write.sum
 # from one ncu capture of this workload; profiles/gemm_kernels_n8192_ncu_metrics.md and
 # profiles/gemm_kernel_fp16_n4096_ncu_full.md).  Sizes that were not captured report null.
-NCU_TRAFFIC_BYTES = {"fp16": {8192: 900832256 + 253492480, 4096: 96256000 + 41258496}}
+NCU_TRAFFIC_BYTES = {"fp16": {8192: 835034880 + 253426176, 4096: 104337920 + 40935936}}
 
 
 def measured_peaks():
