@@ -85,10 +85,13 @@ int gemm_s8(int M, int N, int K, const int8_t* A, const int8_t* B, int32_t* C,
  * bytes, B: N rows of K/2 bytes; element k of a row is bits [4*(k&1), 4*(k&1)+4)
  * of byte k>>1 (low nibble first), two's complement.
  *
- * Blackwell's tcgen05.mma has no 4-bit integer kind, so the operands are first
- * sign-extended to int8 by a streaming pre-pass into a workspace of
- * gemm_s4_workspace_bytes(M, N, K) bytes and then multiplied by the INT8
- * kernel.  gemm_s4 keeps one grow-only workspace per device inside the library:
+ * Blackwell's tcgen05.mma has no 4-bit integer kind.  Large problems: the
+ * operands are first sign-extended to int8 by a streaming pre-pass into a
+ * workspace of gemm_s4_workspace_bytes(M, N, K) bytes and then multiplied by the
+ * INT8 kernel.  Small problems and problems with few rows: a kernel variant
+ * expands the nibbles on the way to the MMAs and needs no workspace (see
+ * gemm_set_s4_scheme for the rule and the switch).  For the pre-pass gemm_s4
+ * keeps one grow-only workspace per device inside the library:
  * the first call on a device (and any call that needs a larger one) allocates
  * with cudaMalloc, which synchronises the device; the buffer is reused by later
  * calls, so concurrent gemm_s4 calls on different streams of one device must be
@@ -244,7 +247,11 @@ int gemm_mma_peak_probe(int precision, int iters, int n_cols, int commit_every, 
  * Writes a human-readable description of the tile configuration the selector
  * picks for this problem ("BM=256 BN=256 BK=64 cta_group=2 stages=6 group_m=12
  * split_k=1 split_tiles=0 tiles=1024 ctas=148 kind=f16") into buf (NUL
- * terminated, truncated to len).  Host only, no GPU work.
+ * terminated, truncated to len); for INT4 followed by the route
+ * (" prepass=unpack_s4" or " s4=fused_unpack"), and by " swap_ab" when the
+ * kernel runs on exchanged operands (the tile is then described in the
+ * kernel's orientation).  Describes the raw 32-bit outputs (gemm_fp16,
+ * gemm_s8, gemm_s4).  Host only, no GPU work.
  */
 int gemm_query_config(int precision, int M, int N, int K, char* buf, int len);
 
