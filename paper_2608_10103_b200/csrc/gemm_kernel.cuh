@@ -808,7 +808,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       // 16-bit results.  Thread `lane` owns row `lane`; 16-byte chunk j of the row goes to
       // chunk j ^ (lane & 7), the 128-byte swizzle the C tensor map expects, which also
       // spreads the warp's 16-byte stores over all banks.
-      constexpr int BLOCK_COLS = (EPI == EPI_OUT16) ? 64 : 32;
+      // (The 32-wide tile with 16-bit output has no staging form -- a block would be 64 bytes
+      // wide -- and only ever runs with plain stores: c_vec_ok = 0, set by the host.)
+      constexpr int BLOCK_COLS = (EPI == EPI_OUT16 && BN >= 64) ? 64 : 32;
       static_assert(BN % BLOCK_COLS == 0, "tile width must be a multiple of the store block");
 #pragma unroll 1
       for (int c = 0; c < BN / BLOCK_COLS && !xpeer; ++c) {
@@ -835,12 +837,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           }
         } else {
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
+          for (int h = 0; h < BLOCK_COLS / 32; ++h) {
             uint32_t r[32];
             ptx::tmem_ld_32x32b_x32(
-                tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 64 + h * 32), r);
+                tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * BLOCK_COLS + h * 32), r);
             ptx::tmem_wait_ld();
-            add_partial(r, c * 2 + h);
+            add_partial(r, c * (BLOCK_COLS / 32) + h);
 #pragma unroll
             for (int v = 0; v < 32; v += 2) {
               float x0 = acc_to_float<KIND>(fix(r[v])), x1 = acc_to_float<KIND>(fix(r[v + 1]));
@@ -904,7 +906,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           if constexpr (EPI == EPI_OUT16) {
             uint16_t* crow = reinterpret_cast<uint16_t*>(p.C) + static_cast<size_t>(row) * rstep;
 #pragma unroll
-            for (int v = 0; v < 64; ++v)
+            for (int v = 0; v < BLOCK_COLS; ++v)
               if (col + v < p.N)
                 crow[(col + v) * cstep] = static_cast<uint16_t>(w[v / 2] >> (16 * (v & 1)));
           } else {

@@ -136,7 +136,9 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
       (KIND == ptx::KIND_F16) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
   // the selector sees the int8 problem either way, so both INT4 routes get the same tile
   int k_blocks = ceil_div(static_cast<long long>(K) * ELEM, BK_BYTES);
-  const int min_bn = EPI == EPI_OUT16 ? 64 : 32;
+  // 16-bit outputs are staged 64 columns at a time; with exchanged operands C goes out by
+  // plain stores and the 32-wide tile serves them too
+  const int min_bn = (EPI == EPI_OUT16 && !swap) ? 64 : 32;
   const bool split_through_c = EPI == EPI_RAW32 && !out.no_split;
   TileConfig cfg =
       select_config(M, N, s->num_sms, k_blocks, min_bn, split_through_c, packed_s4 ? 2 : 0);
@@ -271,7 +273,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
       const int cb = 128 + EPI * 2;
       if (cfg.bn == 64)
         return launch_variant<KIND, 64, 4, 1, 1, EPI, 2, 2>(s, cb + 1, ta, tb, tc, p, stream);
-      if constexpr (EPI != EPI_OUT16)
+      if (EPI != EPI_OUT16 || swap)
         return launch_variant<KIND, 32, 4, 1, 1, EPI, 4, 2>(s, cb, ta, tb, tc, p, stream);
     }
     return GEMM_ERR_INVALID_ARG;
@@ -280,7 +282,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     const int cb = 96 + ((KIND == ptx::KIND_F16) ? 0 : 16) + EPI * 2;
     if (cfg.bn == 64)
       return launch_variant<KIND, 64, 3, 1, 2, EPI, 0, 2>(s, cb + 1, ta, tb, tc, p, stream);
-    if constexpr (EPI != EPI_OUT16)
+    if (EPI != EPI_OUT16 || swap)
       return launch_variant<KIND, 32, 4, 1, 2, EPI, 0, 2>(s, cb, ta, tb, tc, p, stream);
     return GEMM_ERR_INVALID_ARG;
   }
@@ -297,7 +299,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
         case 128: return launch_variant<KIND, 128, 4, 1, 1, EPI, 2>(s, fb + 2, ta, tb, tc, p, stream);
         case 64: return launch_variant<KIND, 64, 4, 1, 1, EPI, 4>(s, fb + 3, ta, tb, tc, p, stream);
         case 32:
-          if constexpr (EPI != EPI_OUT16)
+          if (EPI != EPI_OUT16 || swap)
             return launch_variant<KIND, 32, 4, 1, 1, EPI, 5>(s, fb + 4, ta, tb, tc, p, stream);
           return GEMM_ERR_INVALID_ARG;
         default: return GEMM_ERR_INVALID_ARG;
@@ -318,7 +320,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     case 128: return launch_variant<KIND, 128, 3, 1, 2, EPI>(s, vbase + 1, ta, tb, tc, p, stream);
     case 64: return launch_variant<KIND, 64, 4, 1, 2, EPI>(s, vbase + 2, ta, tb, tc, p, stream);
     case 32:
-      if constexpr (EPI != EPI_OUT16)
+      if (EPI != EPI_OUT16 || swap)
         return launch_variant<KIND, 32, 4, 1, 2, EPI>(s, vbase + 3, ta, tb, tc, p, stream);
       return GEMM_ERR_INVALID_ARG;
     default: return GEMM_ERR_INVALID_ARG;

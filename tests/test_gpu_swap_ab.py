@@ -91,3 +91,33 @@ def test_automatic_choice_for_few_rows():
         check_against_oracle(prec, A, B, C, force_full=True)
     binding.gemm_set_swap_ab(1)
     assert "swap_ab" not in binding.gemm_query_config("s8", 16, 8192, 8192)
+
+
+@pytest.mark.parametrize("split_k", [1, 2])
+def test_swapped_16_bit_outputs_on_the_32_wide_tile(split_k):
+    """With exchanged operands C goes out by plain stores, so the 32-wide tile, which has no
+    64-column staging block, serves the binary16 outputs too (with and without the split of K
+    inside a cluster)."""
+    M, N, K = 24, 1300, 2080
+    binding.gemm_set_config_override(32, 0, 1, split_k)
+    A, B = synth.fp16_normal_clipped(M, N, K, seed=8)
+    ref, S = oracle.gemm_fp16(A, B)
+    C = torch.full((M, N), float("nan"), dtype=torch.float16, device="cuda")
+    binding.gemm_fp16_f16out(to_dev(A), to_dev(B), C)
+    torch.cuda.synchronize()
+    ok, worst = oracle.fp16_out_check(C.cpu().numpy(), ref, S)
+    assert ok, "fp16 out: %.3g x bound" % worst
+    g = np.random.Generator(np.random.PCG64(8))
+    rs = (g.uniform(0.5, 2.0, M) * 1e-2).astype(np.float32)
+    cs = (g.uniform(0.5, 2.0, N) * 1e-1).astype(np.float32)
+    for prec, scheme in (("s8", 0), ("s4", 1), ("s4", 2)):
+        binding.gemm_set_s4_scheme(scheme)
+        A, B = synth.make(prec, M, N, K, seed=9)
+        exact = oracle.gemm_s8_i64(A, B) if prec == "s8" else oracle.gemm_s4_i64(A, B, K)
+        ref = oracle.dequant_ref(exact, rs, cs)
+        fn = binding.gemm_s8_dequant if prec == "s8" else binding.gemm_s4_dequant
+        C = torch.full((M, N), float("nan"), dtype=torch.float16, device="cuda")
+        fn(to_dev(A), to_dev(B), to_dev(rs), to_dev(cs), C, torch.float16)
+        torch.cuda.synchronize()
+        ok, worst = oracle.dequant_check(C.cpu().numpy(), ref, True)
+        assert ok, "%s scheme %d: %.3g x bound" % (prec, scheme, worst)
