@@ -535,10 +535,13 @@ def run_few_rows(args):
               (128, 16384, 4096), (32, 28672, 8192)]
     if args.shape:
         shapes = [tuple(int(x) for x in args.shape.split(","))]
-    routes = {"fp16": [("selector default", 0, 0), ("operands not exchanged", 0, 1)],
-              "s8": [("selector default", 0, 0), ("operands not exchanged", 0, 1)],
-              "s4": [("selector default", 0, 0), ("pre-pass + INT8 GEMM", 1, 1),
-                     ("expanded in the kernel, operands exchanged", 2, 2)]}
+    routes = {"fp16": [("selector default", 0, 0, "raw"), ("operands not exchanged", 0, 1, "raw"),
+                       ("FP16 output, selector default", 0, 0, "out16")],
+              "s8": [("selector default", 0, 0, "raw"), ("operands not exchanged", 0, 1, "raw"),
+                     ("dequantised to FP16, selector default", 0, 0, "out16")],
+              "s4": [("selector default", 0, 0, "raw"), ("pre-pass + INT8 GEMM", 1, 1, "raw"),
+                     ("expanded in the kernel, operands exchanged", 2, 2, "raw"),
+                     ("dequantised to FP16, selector default", 0, 0, "out16")]}
     for M, N, K in shapes:
         for prec in [q for q in synth.PRECISIONS if q in args.precisions.split(",")]:
             A, B = synth.make(prec, M, N, K, seed=M + N)
@@ -546,14 +549,28 @@ def run_few_rows(args):
             copies = max(2, -(-(256 << 20) // B.nbytes))
             dBs = [torch.from_numpy(B).cuda() for _ in range(copies)]
             dB = dBs[0]
-            C = torch.empty((M, N), dtype=torch.float32 if prec == "fp16" else torch.int32,
-                            device="cuda")
-            algo_bytes = A.nbytes + B.nbytes + M * N * 4
-            for name, scheme, swap in routes[prec]:
+            C32 = torch.empty((M, N), dtype=torch.float32 if prec == "fp16" else torch.int32,
+                              device="cuda")
+            C16 = torch.empty((M, N), dtype=torch.float16, device="cuda")
+            rs = torch.rand(M, device="cuda") + 0.5
+            cs = torch.rand(N, device="cuda") + 0.5
+
+            def call(mode, b, stream=None):
+                if mode == "raw":
+                    binding.gemm(prec, dA, b, C32, stream=stream)
+                elif prec == "fp16":
+                    binding.gemm_fp16_f16out(dA, b, C16, stream=stream)
+                elif prec == "s8":
+                    binding.gemm_s8_dequant(dA, b, rs, cs, C16, torch.float16, stream=stream)
+                else:
+                    binding.gemm_s4_dequant(dA, b, rs, cs, C16, torch.float16, stream=stream)
+
+            for name, scheme, swap, mode in routes[prec]:
+                algo_bytes = A.nbytes + B.nbytes + M * N * (4 if mode == "raw" else 2)
                 binding.gemm_set_s4_scheme(scheme)
                 binding.gemm_set_swap_ab(swap)
                 for _ in range(3):
-                    binding.gemm(prec, dA, dB, C)
+                    call(mode, dB)
                 torch.cuda.synchronize()
                 g = torch.cuda.CUDAGraph()
                 side = torch.cuda.Stream()
@@ -561,7 +578,7 @@ def run_few_rows(args):
                 with torch.cuda.stream(side):
                     with torch.cuda.graph(g, stream=side):
                         for i in range(12):
-                            binding.gemm(prec, dA, dBs[i % copies], C, stream=side)
+                            call(mode, dBs[i % copies], side)
                 torch.cuda.current_stream().wait_stream(side)
                 ts = []
                 for _ in range(7):
@@ -580,7 +597,8 @@ def run_few_rows(args):
                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s",
                                  "frac": gbs / hbm, "traffic": None},
                     "algorithmic_bytes": algo_bytes, "b_copies_rotated": copies,
-                    "config": binding.gemm_query_config(prec, M, N, K)}), flush=True)
+                    "config": binding.gemm_query_config(prec, M, N, K) if mode == "raw" else None}),
+                    flush=True)
     binding.gemm_set_s4_scheme(0)
     binding.gemm_set_swap_ab(0)
     if binding.gemm_last_device_status() != 0:
