@@ -122,9 +122,10 @@ int gemm_s4_ws(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t*
  * Alignment as gemm_fp16; rows of C that are not 16-byte multiples (N % 8 != 0)
  * take a slower scalar store path.  A 16-bit (or scaled) result cannot be
  * accumulated in C, so where the plain GEMMs split K over CTAs that add into C,
- * this entry point and the dequantising ones split K between the two CTAs of a
- * cluster, which hand partial sums over through shared memory (narrow one-CTA
- * tiles, factor 2: M = 16, N = 4096, K = 16384: 46 -> 32 us).
+ * this entry point and the dequantising ones split K between the two or four
+ * CTAs of a cluster, which send their partial sums to the first one as bulk
+ * copies between shared memories (narrow one-CTA tiles: M = 16, N = 4096,
+ * K = 16384: 46 -> 28 us).
  */
 int gemm_fp16_f16out(int M, int N, int K, const void* A, const void* B, void* C,
                      gemm_stream_t stream);
@@ -343,8 +344,8 @@ int gemm_set_swap_ab(int mode);
  * the default, problems that are one tile wide or one tile tall (few rows on one
  * side) use 2 for bits 0-1, so that the short operand every CTA re-reads is not
  * pushed out of L2 by the long one streaming past.  Bit 6 (64): no split-K
- * inside a cluster (see gemm_fp16_f16out / the dequantising entry points).  Integer results never depend on any of
- * this; FP16 results may differ in the last bits (summation order) within the
+ * inside a cluster (see gemm_fp16_f16out / the dequantising entry points).
+ * Integer results never depend on any of this; FP16 results may differ in the last bits (summation order) within the
  * bound.
  */
 int gemm_set_l2_policy(int policy);

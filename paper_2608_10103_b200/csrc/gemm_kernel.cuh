@@ -165,10 +165,11 @@ struct SmemLayout {
   static constexpr int EPI_BUF_BYTES = 32 * 128;
   static constexpr int EPI_OFFSET = RING_BYTES;
   static constexpr int EPI_BYTES = EPI_WARPS * 2 * EPI_BUF_BYTES;
-  // Cluster split-K: the CTA of cluster rank 0 receives the other CTA's 128 x BN partial
-  // accumulators (32-bit) here.
+  // Cluster split-K: the CTA of cluster rank 0 receives the other CTAs' 128 x BN partial
+  // accumulators (32-bit) here, one buffer per sender.
   static constexpr int X_OFFSET = EPI_OFFSET + EPI_BYTES;
-  static constexpr int X_BYTES = CSPLIT > 1 ? BM * BN * 4 : 0;
+  static constexpr int X_PEER_BYTES = BM * BN * 4;  // one buffer per contributing CTA
+  static constexpr int X_BYTES = CSPLIT > 1 ? (CSPLIT - 1) * X_PEER_BYTES : 0;
   static constexpr int BAR_OFFSET = X_OFFSET + X_BYTES;
   // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], drain, p_full[PSTAGES], p_empty[PSTAGES]
   // fused INT4 adds ready[STAGES]; cluster split-K adds part_full, part_free
@@ -183,14 +184,11 @@ struct SmemLayout {
 
 // Bounded wait: polls the barrier; after the limit (or once another role has
 // given up) records `code` and returns false.  The caller then leaves its loop.
-template <bool BACKOFF = false, bool ACQUIRE_CLUSTER = false>
+template <bool BACKOFF = false>
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity,
                                              volatile uint32_t* abort_flag, int* status, int code,
                                              uint32_t backoff_ns = 0) {
-  auto done = [&]() {
-    if constexpr (ACQUIRE_CLUSTER) return ptx::mbar_try_wait_acquire_cluster(bar, parity);
-    return ptx::mbar_try_wait(bar, parity);
-  };
+  auto done = [&]() { return ptx::mbar_try_wait(bar, parity); };
   if (done()) return true;
   uint64_t t0 = 0;
   uint32_t spins = 0;
@@ -243,13 +241,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
   using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, CSPLIT>;
   constexpr bool FUSED = PSTAGES > 0;  // packed INT4 operands, expanded on the way to the MMAs
-  // CSPLIT = 2 (cluster split-K): a cluster of two single CTAs owns every tile; each takes half
-  // of K into its own accumulator, the CTA of rank 1 hands its 128 x BN partial sums to rank 0
-  // through the cluster's shared-memory window, and rank 0 adds them to its own on the way
-  // out.  Unlike split-K through C this needs no zeroed C and no adds in global memory, so it
+  // CSPLIT = 2 or 4 (cluster split-K): a cluster of CSPLIT single CTAs owns every tile; each
+  // takes its share of K into its own accumulator, the CTAs of rank 1.. hand their 128 x BN
+  // partial sums to rank 0 through the cluster's shared-memory window (one buffer each), and
+  // rank 0 adds them to its own on the way out.  Unlike split-K through C this needs no zeroed C and no adds in global memory, so it
   // also serves the 16-bit and scaled outputs, and a call is a single launch.
-  static_assert(CSPLIT == 1 || (CSPLIT == 2 && CTA_GROUP == 1 && BN <= 64),
-                "cluster split-K: two single CTAs, narrow tile");
+  static_assert(CSPLIT == 1 || ((CSPLIT == 2 || CSPLIT == 4) && CTA_GROUP == 1 && BN <= 64),
+                "cluster split-K: two or four single CTAs, narrow tile");
   static_assert(!FUSED || (KIND == ptx::KIND_I8 && KB == 1 && STAGES >= 2),
                 "fused INT4: int8 MMAs, one atom per slot, a packed slot fills two int8 slots at once");
   constexpr int ELEM_BYTES = (KIND == ptx::KIND_F16) ? 2 : 1;
@@ -279,8 +277,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   // arrive with release semantics straight from the writing warps costs each of them
   // hundreds of cycles).
   auto ready_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 5 + 2 * PSTAGES + s); };
-  // cluster split-K: `part_full` lives in rank 0 (rank 1's partial sums of a tile have landed),
-  // `part_free` in rank 1 (rank 0 has consumed them, the buffer may be overwritten)
+  // cluster split-K: `part_full` lives in rank 0 (the other ranks' partial sums of a tile have
+  // all landed), `part_free` in every other rank (rank 0 has consumed them, the buffer may be
+  // overwritten)
   const uint32_t part_full_bar = bar0 + 8u * (L::NUM_BARS - 2);
   const uint32_t part_free_bar = bar0 + 8u * (L::NUM_BARS - 1);
   volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(base_ptr + L::MISC_OFFSET);
@@ -348,7 +347,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     }
     ptx::mbar_init(drain_bar, 1);
     if constexpr (CSPLIT > 1) {
-      ptx::mbar_init(part_full_bar, EPI_WARPS);
+      ptx::mbar_init(part_full_bar, 1);  // rank 0's own announcement; the rest is a byte count
       ptx::mbar_init(part_free_bar, EPI_WARPS);
     }
     *abort_flag = 0;
@@ -722,12 +721,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     bool prior_grid_done = false;
     uint32_t xphase = 0;         // cluster split-K: parity of the partial-sum hand-over
     const bool xpeer = CSPLIT > 1 && krank != 0;  // this CTA only contributes partial sums
-    // Cluster split-K, rank 0: adds the other CTA's partial sums for accumulator columns
+    // Cluster split-K, rank 0: adds the other CTAs' partial sums for accumulator columns
     // [32 * b32, 32 * b32 + 32) of this thread's row to the 32 raw accumulators in r.
     auto add_partial = [&](uint32_t (&r)[32], int b32) {
       if constexpr (CSPLIT > 1) {
+#pragma unroll
+        for (int peer = 0; peer < CSPLIT - 1; ++peer) {
         const uint32_t xsrc = base + L::X_OFFSET +
-                              static_cast<uint32_t>(quarter * (32 * BN * 4) + b32 * 4096 + lane * 128);
+                              static_cast<uint32_t>(peer * L::X_PEER_BYTES + quarter * (32 * BN * 4) +
+                                                    b32 * 4096 + lane * 128);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           uint32_t t0, t1, t2, t3;
@@ -744,6 +746,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             r[4 * j + 3] += t3;
           }
         }
+        }
       }
     };
     for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
@@ -751,6 +754,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       bool add;
       decode_unit(t, tile, k_begin, k_end, add);
       tile_coords(p, tile, tm, tn);
+      const int row0 = tm * TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
+      const int row = row0 + lane;
+      const int col0 = tn * BN;
+      float rs = 1.0f;
+      if constexpr (EPI != EPI_RAW32) {
+        // The scale factors are fetched while the mainloop still runs: this thread's row
+        // factor into a register, the tile's column factors into L1 (one line per lane).
+        // They may come from the grid in front, so its end is awaited first -- the producer
+        // waits for the same before its first load, so no accumulator could be ready earlier.
+        if (p.row_scale || p.col_scale) {
+          if (p.wait_prior_grid && !prior_grid_done) {
+            ptx::grid_dep_wait();
+            prior_grid_done = true;
+          }
+          if (p.row_scale && row < p.M) rs = __ldg(p.row_scale + row);
+          if (p.col_scale && lane * 32 < BN && col0 + lane * 32 < p.N)
+            ptx::prefetch_l1(p.col_scale + col0 + lane * 32);
+        }
+      }
       const long long w0 = trace ? clock64() : 0;
       ok = wait_bounded<true>(acc_full_bar(acc), acc_phase, abort_flag, p.status,
                               DEV_TIMEOUT_EPILOGUE, (p.ablate & 4) ? 500u : 0u);
@@ -761,15 +783,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::tc_fence_after_sync();
       if constexpr (CSPLIT > 1) {
         if (xpeer) {
-          // Rank 1: once rank 0 has consumed the previous tile's partial sums, write this
-          // tile's (raw 32-bit accumulators, one 128-byte row piece per thread and 32 columns,
-          // swizzled like the staging buffers) into rank 0's shared memory and tell it.
-          ok = wait_bounded<false, true>(part_free_bar, xphase ^ 1u, abort_flag, p.status,
-                                         DEV_TIMEOUT_EPILOGUE);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          const uint32_t xdst = ptx::map_to_cta(base + L::X_OFFSET, 0) +
-                                static_cast<uint32_t>(quarter * (32 * BN * 4) + lane * 128);
+          // Ranks 1..: write this tile's raw 32-bit accumulators (one 128-byte row piece per
+          // thread and 32 columns, swizzled like the staging buffers) into this CTA's own
+          // hand-over buffer, then -- once rank 0 has consumed the previous tile's partial
+          // sums -- send the warp's 32 rows to rank 0's buffer for this rank as one bulk copy,
+          // whose bytes are counted on rank 0's `part_full`.  (No cluster-scope fence or
+          // release: the copy engine orders the data before the byte count.)
+          if (lane == 0) ptx::bulk_wait_group_read<0>();  // the previous copy has read the buffer
+          __syncwarp();
+          const uint32_t xown = base + L::X_OFFSET + static_cast<uint32_t>(quarter * (32 * BN * 4));
 #pragma unroll 1
           for (int b = 0; b < BN / 32; ++b) {
             uint32_t r[32];
@@ -777,15 +799,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             ptx::tmem_wait_ld();
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-              ptx::st_shared_cluster_v4(xdst + static_cast<uint32_t>(b * 4096 + ((j ^ (lane & 7)) * 16)),
-                                        r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+              ptx::st_shared_v4(xown + static_cast<uint32_t>(b * 4096 + lane * 128 + ((j ^ (lane & 7)) * 16)),
+                                r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
           }
-          ptx::fence_acq_rel_cluster();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive_release_cluster(ptx::map_to_cta(part_full_bar, 0));
+          ptx::fence_proxy_async_smem();
+          ok = wait_bounded(part_free_bar, xphase ^ 1u, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          if (lane == 0) {
+            ptx::bulk_copy_to_cluster(
+                ptx::map_to_cta(base + L::X_OFFSET, 0) +
+                    static_cast<uint32_t>((krank - 1) * L::X_PEER_BYTES + quarter * (32 * BN * 4)),
+                xown, 32 * BN * 4, ptx::map_to_cta(part_full_bar, 0));
+            ptx::bulk_commit_group();
+          }
         } else {
-          ok = wait_bounded<false, true>(part_full_bar, xphase, abort_flag, p.status,
-                                         DEV_TIMEOUT_EPILOGUE);
+          // rank 0: one thread announces the bytes the other ranks will send for this tile
+          if (warp == 2 && lane == 0)
+            ptx::mbar_arrive_expect_tx(part_full_bar, (CSPLIT - 1) * L::X_PEER_BYTES);
+          ok = wait_bounded(part_full_bar, xphase, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
         }
@@ -796,13 +828,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       if (p.wait_prior_grid && !prior_grid_done) {  // C may be read, written or zeroed by the grid in front
         ptx::grid_dep_wait();
         prior_grid_done = true;
-      }
-      const int row0 = tm * TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
-      const int row = row0 + lane;
-      const int col0 = tn * BN;
-      float rs = 1.0f;
-      if constexpr (EPI != EPI_RAW32) {
-        if (p.row_scale && row < p.M) rs = __ldg(p.row_scale + row);
       }
       // One staging block = 32 rows x 128 bytes = 32 columns of 32-bit or 64 columns of
       // 16-bit results.  Thread `lane` owns row `lane`; 16-byte chunk j of the row goes to
@@ -929,9 +954,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         }
       }
       if constexpr (CSPLIT > 1) {
-        if (!xpeer) {  // the partial sums have been read: rank 1 may send the next tile's
+        if (!xpeer) {  // the partial sums have been read: the others may send the next tile's
+          // (a plain arrive: the receiver reads nothing this CTA wrote, and this warp's loads
+          // from the buffer have returned their values)
           __syncwarp();
-          if (lane == 0) ptx::mbar_arrive_release_cluster(ptx::map_to_cta(part_free_bar, 1));
+          if (lane == 0) {
+#pragma unroll
+            for (int peer = 1; peer < CSPLIT; ++peer)
+              ptx::mbar_arrive_remote(ptx::map_to_cta(part_free_bar, peer));
+          }
         }
       }
       // Hand the accumulator buffer back to the (leader's) MMA issuer.
@@ -954,8 +985,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       if (acc == 0) acc_phase ^= 1u;
     }
     // C stores still in flight read this CTA's shared memory: wait until they have read it
-    // (their global writes complete on their own before the grid counts as finished).
-    if (lane == 0) ptx::bulk_wait_group_read<0>();
+    // (their global writes complete on their own before the grid counts as finished).  A
+    // hand-over copy into rank 0's shared memory has to have landed as well.
+    if (lane == 0) {
+      if (xpeer) ptx::bulk_wait_group_all();
+      else ptx::bulk_wait_group_read<0>();
+    }
     __syncwarp();
     if (trace && warp == 2 && lane == 0) {
       trace[TRACE_EPI_WAIT] = static_cast<unsigned long long>(epi_wait);

@@ -70,10 +70,51 @@ struct OutputSpec {
   bool no_split = false;    // C is a block of a larger matrix: never zero / add into it
 };
 
-// Whether the selector's choice can run as split-K inside a cluster of two CTAs.
+// Index in attr_set of the unfused cluster split-K variants: 96.., by kind, output mode, width.
+template <int KIND, int EPI>
+constexpr int csplit_variant_base() {
+  return 96 + ((KIND == ptx::KIND_F16) ? 0 : 16) + EPI * 2;
+}
+
+// How many clusters of four CTAs of the 4-way cluster split-K kernel the device holds at once.
+// (Clusters are placed inside one GPC, so this is less than SMs / 4 when a GPC's SM count is
+// not a multiple of four: a tile more than that would wait for a second wave.)
+template <int KIND, int EPI>
+int quad_clusters_resident(DeviceState* s, int variant) {
+  int& cached = s->quad_clusters[KIND == ptx::KIND_F16 ? 0 : 1][EPI];
+  if (cached) return cached;
+  using L = SmemLayout<32, 3, 1, 2, 0, 4>;
+  auto kernel = gemm_kernel<KIND, 32, 3, 1, 2, EPI, 0, 4>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) !=
+      cudaSuccess)
+    return 0;
+  s->attr_set[variant >> 6] |= 1ull << (variant & 63);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(s->num_sms / 4 * 4), 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = L::DYN_BYTES;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 4;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) {
+    (void)cudaGetLastError();
+    n = s->num_sms / 8;  // unknown: assume half
+  }
+  cached = n;
+  return n;
+}
+
+// Whether the selector's choice can run as split-K inside a cluster of two or four CTAs
+// (four only for the 32-wide tile, where the buffers fit).
 bool cluster_split_ok(const TileConfig& c, int M, int N) {
   const long long tiles = static_cast<long long>(ceil_div(M, BM * c.cta_group)) * ceil_div(N, c.bn);
-  return c.cta_group == 1 && c.bn <= 64 && c.splits == 2 && c.split_tiles == tiles;
+  if (c.cta_group != 1 || c.bn > 64 || c.split_tiles != tiles) return false;
+  return c.splits == 2 || (c.splits == 4 && c.bn == 32);
 }
 
 // Whether the packed route is taken for the tile the selector picked.  Scheme 2 forces it
@@ -144,15 +185,24 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
       select_config(M, N, s->num_sms, k_blocks, min_bn, split_through_c, packed_s4 ? 2 : 0);
   if (cfg.bn == 0) return GEMM_ERR_INVALID_ARG;  // override asks for a shape this mode lacks
   // Outputs that cannot be split through C (16-bit, scaled, blocks of a larger C): split-K
-  // inside a cluster of two CTAs where the kernel has that variant (one-CTA tiles up to 64
-  // wide, every tile split in two) -- no zeroing of C, no adds in global memory.  Where the
+  // inside a cluster of two or four CTAs where the kernel has that variant (one-CTA tiles up
+  // to 64 wide, every tile split the same way) -- no zeroing of C, no adds in global memory.  Where the
   // raw 32-bit output can split through C that stays the choice: with the launches chained it
   // measured ~1 us faster per call than the hand-over inside the cluster.
   bool csplit = false;
   if (!split_through_c && !(g_l2_policy & 64)) {
-    const TileConfig c2 =
-        select_config(M, N, s->num_sms, k_blocks, min_bn, true, packed_s4 ? 2 : 0, 2);
-    if (c2.bn != 0 && cluster_split_ok(c2, M, N)) {
+    // try up to four CTAs per tile (all clusters at once, unless the split is forced), then two
+    for (int cap = 4; cap >= 2 && !csplit; cap -= 2) {
+      const TileConfig c2 =
+          select_config(M, N, s->num_sms, k_blocks, min_bn, true, packed_s4 ? 2 : 0, cap);
+      if (c2.bn == 0 || !cluster_split_ok(c2, M, N)) continue;
+      if (c2.splits == 4 && (EPI != EPI_OUT16 || swap)) {
+        if (!g_override_splits &&
+            c2.split_tiles > quad_clusters_resident<KIND, EPI>(s, csplit_variant_base<KIND, EPI>() + 8))
+          continue;
+      } else if (c2.splits == 4) {
+        continue;  // 16-bit outputs take the 32-wide tile only with exchanged operands
+      }
       cfg = c2;
       csplit = true;
     }
@@ -273,17 +323,23 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
       const int cb = 128 + EPI * 2;
       if (cfg.bn == 64)
         return launch_variant<KIND, 64, 4, 1, 1, EPI, 2, 2>(s, cb + 1, ta, tb, tc, p, stream);
-      if (EPI != EPI_OUT16 || swap)
+      if (EPI != EPI_OUT16 || swap) {
+        if (cfg.splits == 4)
+          return launch_variant<KIND, 32, 4, 1, 1, EPI, 3, 4>(s, 136 + EPI, ta, tb, tc, p, stream);
         return launch_variant<KIND, 32, 4, 1, 1, EPI, 4, 2>(s, cb, ta, tb, tc, p, stream);
+      }
     }
     return GEMM_ERR_INVALID_ARG;
   }
   if (csplit) {  // attr_set bits 96..: kind, output mode, width
-    const int cb = 96 + ((KIND == ptx::KIND_F16) ? 0 : 16) + EPI * 2;
+    const int cb = csplit_variant_base<KIND, EPI>();
     if (cfg.bn == 64)
       return launch_variant<KIND, 64, 3, 1, 2, EPI, 0, 2>(s, cb + 1, ta, tb, tc, p, stream);
-    if (EPI != EPI_OUT16 || swap)
+    if (EPI != EPI_OUT16 || swap) {
+      if (cfg.splits == 4)
+        return launch_variant<KIND, 32, 3, 1, 2, EPI, 0, 4>(s, cb + 8, ta, tb, tc, p, stream);
       return launch_variant<KIND, 32, 4, 1, 2, EPI, 0, 2>(s, cb, ta, tb, tc, p, stream);
+    }
     return GEMM_ERR_INVALID_ARG;
   }
   const int vbase = ((KIND == ptx::KIND_F16) ? 0 : 32) + EPI * 8;  // bit index in attr_set

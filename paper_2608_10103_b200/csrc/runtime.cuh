@@ -29,6 +29,9 @@ struct DeviceState {
   void* s4_workspace = nullptr;
   size_t s4_workspace_bytes = 0;
   uint64_t attr_set[3] = {0, 0, 0};  // bit i: dynamic-smem attribute set for kernel variant i
+  // clusters of four CTAs (cluster split-K) the device runs at once, per kind and output
+  // mode; 0 = not asked yet
+  int quad_clusters[2][4] = {};
 };
 
 std::mutex g_mutex;

@@ -225,8 +225,52 @@ def test_cluster_split_k_is_the_automatic_choice_for_few_rows():
     got = run_dequant("s8", A, B, rs, cs, torch.float16)
     ctas = _ctas_of_last_launch()
     binding.gemm_trace_enable(0)
-    assert ctas == 64, ctas
+    assert ctas in (64, 128), ctas              # 32 tiles x 2 or 4 CTAs
     assert oracle.dequant_check(got, ref, True)[0]
+
+
+@pytest.mark.parametrize("prec", ["s8", "s4", "s4 fused", "fp16"])
+@pytest.mark.parametrize("M,N,K", [(16, 1536, 16384),    # 12 tiles x 4 CTAs
+                                   (24, 5000, 4128),     # clusters take several tiles in a row
+                                   (8, 128, 640)])       # fewer ring slots than would fill the ranks
+def test_cluster_split_k_four_ways(prec, M, N, K):
+    """Few tiles and a long K: four CTAs of a cluster share a 32-wide tile (exchanged
+    operands), ranks 1..3 each hand their partial sums to rank 0 in a buffer of their own."""
+    g = np.random.Generator(np.random.PCG64(M + N))
+    rs = (g.uniform(0.5, 2.0, M) * 1e-2).astype(np.float32)
+    cs = (g.uniform(0.5, 2.0, N) * 1e-1).astype(np.float32)
+    # packed INT4 through the pre-pass (the INT8 kernel) or expanded inside the kernel
+    binding.gemm_set_s4_scheme(2 if prec == "s4 fused" else 1)
+    prec = prec.split()[0]
+    binding.gemm_set_config_override(32, 0, 1, 4)
+    binding.gemm_set_swap_ab(2)
+    try:
+        if prec == "fp16":
+            A, B = synth.fp16_normal_clipped(M, N, K, seed=N)
+            ref, S = oracle.gemm_fp16(A, B)
+        else:
+            A, B = synth.make(prec, M, N, K, seed=M)
+            exact = oracle.gemm_s8_i64(A, B) if prec == "s8" else oracle.gemm_s4_i64(A, B, K)
+            ref = oracle.dequant_ref(exact, rs, cs)
+        for rep in range(2):
+            binding.gemm_trace_enable(1)
+            if prec == "fp16":
+                got = run_f16out(A, B)
+            else:
+                got = run_dequant(prec, A, B, rs, cs, torch.float16)
+            ctas = _ctas_of_last_launch()
+            binding.gemm_trace_enable(0)
+            if M == 16:
+                assert ctas == 48, ctas
+            if prec == "fp16":
+                ok, worst = oracle.fp16_out_check(got, ref, S)
+            else:
+                ok, worst = oracle.dequant_check(got, ref, True)
+            assert ok, "%s: %.3g x bound" % (prec, worst)
+    finally:
+        binding.gemm_set_s4_scheme(0)
+        binding.gemm_set_swap_ab(0)
+        binding.gemm_trace_enable(0)
 
 
 @pytest.mark.parametrize("scheme", [1, 2])

@@ -80,3 +80,41 @@ def test_expired_wait_in_the_fused_int4_kernels(variant):
         binding.gemm_set_s4_scheme(0)
         binding.gemm_set_swap_ab(0)
         binding.gemm_set_config_override(0, 0, 0)
+
+
+def test_expired_wait_in_the_cluster_split_k_kernel():
+    """Same drill where four CTAs of a cluster share a tile and hand partial sums to rank 0
+    through shared memory: rank 0 of the first cluster never gets one operand slot, gives up,
+    and the other three (whose copies have long landed) leave with it."""
+    M, N, K = 16, 1536, 8192
+    A, B = synth.s8_uniform(M, N, K, seed=11)
+    g = np.random.Generator(np.random.PCG64(11))
+    rs = (g.uniform(0.5, 2.0, M) * 1e-2).astype(np.float32)
+    cs = (g.uniform(0.5, 2.0, N) * 1e-1).astype(np.float32)
+    dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    d_rs, d_cs = torch.from_numpy(rs).cuda(), torch.from_numpy(cs).cuda()
+    C = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+    assert binding.gemm_last_device_status() == 0
+    binding.gemm_set_config_override(32, 0, 1, 4)
+    binding.gemm_set_swap_ab(2)
+    try:
+        binding.gemm_trace_enable(17)              # drill + cycle records
+        t0 = time.time()
+        binding.gemm_s8_dequant(dA, dB, d_rs, d_cs, C, torch.float16)
+        torch.cuda.synchronize()
+        took = time.time() - t0
+        ctas = sum(1 for t in binding.gemm_trace_read(160) if t["cycles"] > 0)
+        binding.gemm_trace_enable(0)
+        assert ctas == 48, ctas                    # 12 tiles x 4 CTAs: the cluster split-K kernel ran
+        status = binding.gemm_last_device_status()
+        assert status in (1, 2, 3), "expected a recorded wait expiry, got %d" % status
+        assert 1.5 < took < 30.0
+        binding.gemm_s8_dequant(dA, dB, d_rs, d_cs, C, torch.float16)
+        torch.cuda.synchronize()
+        ref = oracle.dequant_ref(oracle.gemm_s8_i64(A, B), rs, cs)
+        assert oracle.dequant_check(C.cpu().numpy(), ref, True)[0]
+        assert binding.gemm_last_device_status() == 0
+    finally:
+        binding.gemm_trace_enable(0)
+        binding.gemm_set_swap_ab(0)
+        binding.gemm_set_config_override(0, 0, 0)

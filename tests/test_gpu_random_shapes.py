@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 # (bn, group_m, cta_group, split_k); 0 = let the selector decide
 CONFIGS = [(0, 0, 0, 0), (0, 0, 0, 1), (256, 0, 2, 0), (256, 0, 1, 1), (128, 0, 2, 1), (64, 0, 1, 1),
            (32, 0, 1, 1), (128, 0, 1, 0), (64, 0, 2, 0), (256, 3, 2, 2), (0, 0, 0, 3), (128, 1, 2, 4),
-           (64, 5, 1, 2), (256, 0, 2, 8), (32, 0, 1, 5)]
+           (64, 5, 1, 2), (256, 0, 2, 8), (32, 0, 1, 5), (32, 0, 1, 4)]
 MS = [1, 2, 17, 127, 128, 129, 255, 256, 300, 511, 777, 1024, 1500, 2048, 3000]
 NS = [1, 3, 8, 64, 100, 256, 260, 512, 1000, 1024, 2304, 4096]
 KS = [32, 64, 96, 128, 160, 256, 512, 1056, 2048, 4128]
