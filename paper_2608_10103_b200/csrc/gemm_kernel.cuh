@@ -851,18 +851,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             for (int v = 0; v < 32; ++v) w[v] = fix(w[v]);
           }
         } else if constexpr (EPI == EPI_F32_SCALED) {
+          // Column factors: one coalesced load per 32 columns (lane v fetches column v's),
+          // handed round by shuffles -- a load per element, even from L1, made this loop
+          // wait ~25 cycles per column.
+          const float cs_mine = (col + lane < p.N) ? __ldg(p.col_scale + col + lane) : 0.0f;
           ptx::tmem_ld_32x32b_x32(
               tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), w);
           ptx::tmem_wait_ld();
           add_partial(w, c);
 #pragma unroll
           for (int v = 0; v < 32; ++v) {
-            const float cs = (col + v < p.N) ? __ldg(p.col_scale + col + v) : 0.0f;
+            const float cs = __shfl_sync(0xffffffffu, cs_mine, v);
             w[v] = __float_as_uint(acc_to_float<KIND>(fix(w[v])) * rs * cs);
           }
         } else {
 #pragma unroll
           for (int h = 0; h < BLOCK_COLS / 32; ++h) {
+            const int cc = col + h * 32 + lane;
+            const float cs_mine = (p.col_scale && cc < p.N) ? __ldg(p.col_scale + cc) : 0.0f;
             uint32_t r[32];
             ptx::tmem_ld_32x32b_x32(
                 tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * BLOCK_COLS + h * 32), r);
@@ -871,10 +877,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 #pragma unroll
             for (int v = 0; v < 32; v += 2) {
               float x0 = acc_to_float<KIND>(fix(r[v])), x1 = acc_to_float<KIND>(fix(r[v + 1]));
-              if (p.col_scale) {
-                const int cc = col + h * 32 + v;
-                x0 *= rs * ((cc < p.N) ? __ldg(p.col_scale + cc) : 0.0f);
-                x1 *= rs * ((cc + 1 < p.N) ? __ldg(p.col_scale + cc + 1) : 0.0f);
+              if (p.col_scale) {  // same for the whole warp
+                x0 *= rs * __shfl_sync(0xffffffffu, cs_mine, v);
+                x1 *= rs * __shfl_sync(0xffffffffu, cs_mine, v + 1);
               }
               w[h * 16 + v / 2] = pack_half2(x0, x1);
             }
