@@ -296,9 +296,13 @@ int gemm_last_device_status(void);
  * fused route (10-26 % up to 1024 x 1024 outputs).
  * scheme 0 (default, automatic): fused where the selector picks a one-CTA tile
  * and M <= 128 or N <= 128 or both <= 1024, or a single wave of CTA-pair tiles
- * (e.g. 2048^3), else the pre-pass; 1: always the pre-pass; 2: fused
- * wherever a fused variant is built (every one-CTA tile, and the 256 x 256 CTA
- * pair without split-K), else the pre-pass.  gemm_s4_ws and gemm_s4_static
+ * (e.g. 2048^3); also for problems with a short side, where the pre-pass (cost:
+ * the bytes of both operands) is dear next to the GEMM: M N / (M + N) <= 384
+ * with the best tile the fused kernel has, and up to 1024 rows or columns with
+ * its CTA-pair tile if the tiles fill their waves to 75 % (256 x 28672 x 8192:
+ * 119 -> 67 us; 512 x 16384 x 4096: 44 -> 35 us); else the pre-pass.  1: always
+ * the pre-pass; 2: fused wherever a fused variant is built (every one-CTA tile,
+ * and the 256 x 256 CTA pair without split-K), else the pre-pass.  gemm_s4_ws and gemm_s4_static
  * always use the pre-pass.  Results are identical, bit for bit.
  * gemm_query_config shows the route.  The paper has no counterpart; its Run 4
  * ablates how the operands reach the tensor cores, of which this is the

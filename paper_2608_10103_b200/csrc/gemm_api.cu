@@ -174,10 +174,8 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
   const int user_m = M, user_n = N;
   if (precision == GEMM_PREC_S4 && g_s4_scheme != 1) {  // the decisions of s4_auto / launch_gemm_epi
     swap = swap_ab_wanted(M, N, true, OutputSpec());
-    c = swap ? select_config(N, M, num_sms, kb, 32, true, 2)
-             : select_config(M, N, num_sms, kb, 32, true, 2);
-    fused = c.bn != 0 && fused_s4_variant_exists(c.bn, c.cta_group, c.splits) &&
-            s4_fused_wanted(user_m, user_n, c, num_sms);
+    fused = swap ? select_fused_s4(N, M, user_m, user_n, num_sms, kb, 32, true, &c)
+                 : select_fused_s4(M, N, user_m, user_n, num_sms, kb, 32, true, &c);
   }
   if (!fused) {
     swap = swap_ab_wanted(M, N, false, OutputSpec());

@@ -133,6 +133,49 @@ bool s4_fused_wanted(int M, int N, const TileConfig& cfg, int num_sms) {
   return M <= 128 || N <= 128 || (M <= 1024 && N <= 1024);
 }
 
+// The INT4 route of a problem (M, N: the kernel's, user_m/user_n: the caller's): true, with
+// the tile in *out, when the nibbles are expanded inside the GEMM kernel.  First the selector's
+// free choice, taken if the fused kernel has that shape and s4_fused_wanted agrees.  Then
+// problems with a short side: the pre-pass costs the bytes of BOTH operands, (M + N) K, the
+// expansion inside the kernel costs shared-memory time that grows with the work, M N K, so
+// what decides is M N / (M + N).  Up to 384 the selector's best choice among all the shapes
+// the fused kernel has is taken; up to 1024 rows or columns its CTA-pair shape, the efficient
+// one, where the tiles fill their waves to 75 % (it cannot split K).  Measured, packed B
+// from HBM: 256 x 28672 x 8192 119 -> 67 us, 512 x 16384 x 4096 44 -> 35 us, 256 x 8192 x 8192
+// 35 -> 31 us, 1024 x 8192 x 8192 63 -> 60 us; the one-CTA shapes at 640-1024 x 2048 x 8192
+// would lose 15-35 %, and from 1280 rows on the pre-pass is even or ahead.
+bool select_fused_s4(int M, int N, int user_m, int user_n, int num_sms, int k_blocks, int min_bn,
+                     bool allow_split, TileConfig* out) {
+  if (g_s4_scheme == 1) return false;
+  const TileConfig c = select_config(M, N, num_sms, k_blocks, min_bn, allow_split, 2);
+  if (c.bn != 0 && fused_s4_variant_exists(c.bn, c.cta_group, c.splits) &&
+      s4_fused_wanted(user_m, user_n, c, num_sms)) {
+    *out = c;
+    return true;
+  }
+  const long long mn = static_cast<long long>(user_m) * user_n;
+  if (g_s4_scheme == 2 || mn <= 384ll * (user_m + user_n)) {
+    const TileConfig f = select_config(M, N, num_sms, k_blocks, min_bn, allow_split, 2, 0, 1);
+    if (f.bn != 0) {
+      *out = f;
+      return true;
+    }
+  }
+  if (user_m <= 1024 || user_n <= 1024) {
+    const TileConfig f = select_config(M, N, num_sms, k_blocks, min_bn, allow_split, 2, 0, 2);
+    if (f.bn != 0) {
+      const long long tiles = static_cast<long long>(ceil_div(M, 2 * BM)) * ceil_div(N, f.bn);
+      const long long pairs = num_sms / 2;
+      const long long waves = (tiles + pairs - 1) / pairs;
+      if (4 * tiles >= 3 * waves * pairs) {
+        *out = f;
+        return true;
+      }
+    }
+  }
+  return false;
+}
+
 // Whether the kernel runs on exchanged operands (its rows = the caller's N side).  The 128-row
 // side of a tile is then filled by the long operand of a problem with few rows (LLM decoding:
 // M = 1..64), instead of 128 - M rows of zero fill taking shared memory, ring depth and, on
@@ -181,8 +224,11 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   // plain stores and the 32-wide tile serves them too
   const int min_bn = (EPI == EPI_OUT16 && !swap) ? 64 : 32;
   const bool split_through_c = EPI == EPI_RAW32 && !out.no_split;
-  TileConfig cfg =
-      select_config(M, N, s->num_sms, k_blocks, min_bn, split_through_c, packed_s4 ? 2 : 0);
+  TileConfig cfg = select_config(M, N, s->num_sms, k_blocks, min_bn, split_through_c);
+  bool fused_cfg = false;
+  if (packed_s4)
+    fused_cfg = select_fused_s4(M, N, user_m, user_n, s->num_sms, k_blocks, min_bn,
+                                split_through_c, &cfg);
   if (cfg.bn == 0) return GEMM_ERR_INVALID_ARG;  // override asks for a shape this mode lacks
   // Outputs that cannot be split through C (16-bit, scaled, blocks of a larger C): split-K
   // inside a cluster of two or four CTAs where the kernel has that variant (one-CTA tiles up
@@ -208,9 +254,8 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     }
   }
   if (packed_s4) {
-    if (KIND != ptx::KIND_I8 ||
-        !(csplit || fused_s4_variant_exists(cfg.bn, cfg.cta_group, cfg.splits)) ||
-        !s4_fused_wanted(user_m, user_n, cfg, s->num_sms))
+    if (KIND != ptx::KIND_I8) return GEMM_NOT_FUSED;
+    if (csplit ? !s4_fused_wanted(user_m, user_n, cfg, s->num_sms) : !fused_cfg)
       return GEMM_NOT_FUSED;
     k_blocks = 2 * ceil_div(K, 2 * BK_BYTES);  // one packed slot (256 values of K) = two int8 slots
   }

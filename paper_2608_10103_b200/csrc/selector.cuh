@@ -60,12 +60,15 @@ int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b
 // force_atoms: K atoms per split unit whatever the tile (the fused INT4 kernel splits K in
 // packed slots = 2 int8 k-blocks); 0 = the tile's own ring slot.
 // split_cap: upper limit of the split-K factor (0 = none).
+// fused_only: 1 = only shapes the fused INT4 kernel is built for, 2 = only its CTA-pair shape.
 TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 32,
-                         bool allow_split = false, int force_atoms = 0, int split_cap = 0) {
+                         bool allow_split = false, int force_atoms = 0, int split_cap = 0,
+                         int fused_only = 0) {
   TileConfig best{256, 2, 6, 8, 1, 0};
   long long best_cost = -1;
   for (int cg = 2; cg >= 1; --cg) {
     if (g_override_cta_group && cg != g_override_cta_group) continue;
+    if (fused_only == 2 && cg != 2) continue;
     for (int bn : kWidths) {
       if (g_override_bn && bn != g_override_bn) continue;
       if (!variant_exists(bn, cg) || bn < min_bn) continue;
@@ -92,6 +95,7 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
       if (max_split > slots) max_split = slots;
       for (int sp = g_override_splits ? max_split : 1; sp <= max_split; ++sp) {
         if (static_cast<long long>(sp - 1) * ceil_div(slots, sp) >= slots) continue;  // empty range
+        if (fused_only && !fused_s4_variant_exists(bn, cg, sp)) continue;
         const int per = ceil_div(slots, sp) * atoms;  // k-blocks per unit
         const long long waves = (tiles * sp + units - 1) / units;
         long long per_kb = 2 * bn;
@@ -125,7 +129,7 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
     best.split_tiles = best.splits > 1 ? static_cast<int>(tiles) : 0;
     const long long r = tiles % units;
     if (allow_split && best.splits == 1 && g_override_splits == 0 && tiles > units && r > 0 &&
-        2 * r <= units && slots >= 64) {  // measured: pays off (+2-3 %) only for long K
+        2 * r <= units && slots >= 64 && !(fused_only && best.cta_group == 2)) {  // measured: pays off (+2-3 %) only for long K
       int sp = static_cast<int>(units / r);
       if (sp > 4) sp = 4;
       while (sp > 1 && (slots / sp < 32 ||
