@@ -81,12 +81,24 @@ def test_automatic_route_by_shape():
     assert "prepass" in binding.gemm_query_config("s4", 8192, 8192, 8192)
     assert "prepass" in binding.gemm_query_config("s4", 4096, 4096, 4096)
     assert "prepass" in binding.gemm_query_config("s4", 512, 4096, 4096)
+    # a short side against a large N K: M N / (M + N) <= 384, or <= 1024 rows on well-filled pair tiles
+    assert "fused_unpack" in binding.gemm_query_config("s4", 256, 28672, 8192)
+    assert "fused_unpack" in binding.gemm_query_config("s4", 28672, 256, 8192)
+    assert "fused_unpack" in binding.gemm_query_config("s4", 384, 4096, 16384)
+    assert "fused_unpack" in binding.gemm_query_config("s4", 1024, 8192, 8192)
+    assert "prepass" in binding.gemm_query_config("s4", 640, 8192, 8192)           # pair tiles fill 65 %
+    assert "prepass" in binding.gemm_query_config("s4", 896, 2048, 8192)
+    assert "prepass" in binding.gemm_query_config("s4", 2048, 8192, 8192)
     binding.gemm_set_s4_scheme(1)
     assert "prepass" in binding.gemm_query_config("s4", 16, 8192, 8192)
     binding.gemm_set_s4_scheme(0)
     M, N, K = 16, 4096, 8192
     A, B = synth.s4_uniform(M, N, K, seed=11)
     check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), force_full=True)
+    for M, N, K in [(200, 20000, 2080), (300, 5000, 1056)]:   # two waves of pair tiles; one-CTA tiles
+        assert "fused_unpack" in binding.gemm_query_config("s4", M, N, K)
+        A, B = synth.s4_uniform(M, N, K, seed=M)
+        check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), seed=M)
 
 
 def test_fused_extreme_values_and_nibble_positions():
