@@ -178,7 +178,7 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
                  : select_fused_s4(M, N, user_m, user_n, num_sms, kb, 32, true, &c);
   }
   if (!fused) {
-    swap = swap_ab_wanted(M, N, false, OutputSpec());
+    swap = swap_ab_wanted(M, N, precision != GEMM_PREC_FP16, OutputSpec());
     c = swap ? select_config(N, M, num_sms, kb, 32, true) : select_config(M, N, num_sms, kb, 32, true);
   }
   if (c.bn == 0) return GEMM_ERR_INVALID_ARG;

@@ -180,13 +180,14 @@ bool select_fused_s4(int M, int N, int user_m, int user_n, int num_sms, int k_bl
 // side of a tile is then filled by the long operand of a problem with few rows (LLM decoding:
 // M = 1..64), instead of 128 - M rows of zero fill taking shared memory, ring depth and, on
 // the fused INT4 route, expansion work; C goes out by plain stores that are contiguous along
-// the caller's N.  Automatic when N >= 1024 and M <= 32 (M <= 64 on the fused INT4 route): measured
-// 2-12 % faster there.
-bool swap_ab_wanted(int M, int N, bool packed_s4, const OutputSpec& out) {
+// the caller's N.  Automatic when N >= 1024 and M <= 32 (FP16) or M <= 64 (the integer kinds,
+// both INT4 routes): measured 2-12 % faster there (INT8, M = 48-64: 3-8 %; FP16 even; from
+// M = 80 on, where the narrow side needs the 128-wide tile, 4-20 % slower).
+bool swap_ab_wanted(int M, int N, bool integer_kind, const OutputSpec& out) {
   if (out.no_split || out.ldc) return false;  // C is a block of a larger matrix
   if (g_swap_ab == 1) return false;
   if (g_swap_ab == 2) return true;
-  return N >= 1024 && M <= (packed_s4 ? 64 : 32);
+  return N >= 1024 && M <= (integer_kind ? 64 : 32);
 }
 
 // Returned (never to the caller of the library) when the fused INT4 kernel does not cover the
@@ -210,7 +211,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   constexpr int C_ELEM = (EPI == EPI_OUT16) ? 2 : 4;
   const long long ldc = out.ldc ? out.ldc : N;
   const int user_m = M, user_n = N;
-  const bool swap = swap_ab_wanted(M, N, packed_s4, out);
+  const bool swap = swap_ab_wanted(M, N, KIND == ptx::KIND_I8, out);
   if (swap) {  // from here on M, N, A, B are the kernel's
     std::swap(M, N);
     std::swap(A, B);

@@ -78,7 +78,9 @@ def test_automatic_choice_for_few_rows():
     assert "fused_unpack" in cfg and "swap_ab" in cfg
     assert "swap_ab" in binding.gemm_query_config("s4", 64, 8192, 8192)
     assert "swap_ab" not in binding.gemm_query_config("s4", 128, 8192, 8192)
-    assert "swap_ab" not in binding.gemm_query_config("s8", 64, 8192, 8192)
+    assert "swap_ab" in binding.gemm_query_config("s8", 64, 8192, 8192)
+    assert "swap_ab" not in binding.gemm_query_config("s8", 80, 8192, 8192)
+    assert "swap_ab" not in binding.gemm_query_config("fp16", 64, 8192, 8192)
     assert "swap_ab" in binding.gemm_query_config("s8", 16, 8192, 8192)
     assert "swap_ab" in binding.gemm_query_config("fp16", 16, 8192, 8192)
     assert "swap_ab" not in binding.gemm_query_config("fp16", 128, 8192, 8192)
