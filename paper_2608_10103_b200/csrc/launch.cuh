@@ -126,9 +126,9 @@ bool cluster_split_ok(const TileConfig& c, int M, int N) {
 bool s4_fused_wanted(int M, int N, const TileConfig& cfg, int num_sms) {
   if (g_s4_scheme == 2) return true;
   if (g_s4_scheme == 1) return false;
-  if (cfg.cta_group == 2) {
+  if (cfg.cta_group == 2) {  // (the 128-wide pair tile only comes in through select_fused_s4)
     const long long tiles = static_cast<long long>(ceil_div(M, 2 * BM)) * ceil_div(N, cfg.bn);
-    return tiles <= num_sms / 2;
+    return cfg.bn == 256 && tiles <= num_sms / 2;
   }
   return M <= 128 || N <= 128 || (M <= 1024 && N <= 1024);
 }
@@ -139,8 +139,8 @@ bool s4_fused_wanted(int M, int N, const TileConfig& cfg, int num_sms) {
 // problems with a short side: the pre-pass costs the bytes of BOTH operands, (M + N) K, the
 // expansion inside the kernel costs shared-memory time that grows with the work, M N K, so
 // what decides is M N / (M + N).  Up to 384 the selector's best choice among all the shapes
-// the fused kernel has is taken; up to 1024 rows or columns its CTA-pair shape, the efficient
-// one, where the tiles fill their waves to 75 % (it cannot split K).  Measured, packed B
+// the fused kernel has is taken; up to 1024 rows or columns its 256-wide CTA-pair shape, the
+// efficient one, where the tiles fill their waves to 75 % (it cannot split K).  Measured, packed B
 // from HBM: 256 x 28672 x 8192 119 -> 67 us, 512 x 16384 x 4096 44 -> 35 us, 256 x 8192 x 8192
 // 35 -> 31 us, 1024 x 8192 x 8192 63 -> 60 us; the one-CTA shapes at 640-1024 x 2048 x 8192
 // would lose 15-35 %, and from 1280 rows on the pre-pass is even or ahead.
@@ -394,8 +394,11 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     // bits 64.. (one per tile shape and output mode)
     if constexpr (KIND == ptx::KIND_I8) {
       const int fb = 64 + EPI * 8;
-      if (cfg.cta_group == 2)
+      if (cfg.cta_group == 2) {
+        if (cfg.bn == 128)
+          return launch_variant<KIND, 128, 4, 2, 1, EPI, 3>(s, fb + 5, ta, tb, tc, p, stream);
         return launch_variant<KIND, 256, 4, 2, 1, EPI, 2>(s, fb + 0, ta, tb, tc, p, stream);
+      }
       switch (cfg.bn) {
         case 256: return launch_variant<KIND, 256, 2, 1, 1, EPI, 2>(s, fb + 1, ta, tb, tc, p, stream);
         case 128: return launch_variant<KIND, 128, 4, 1, 1, EPI, 2>(s, fb + 2, ta, tb, tc, p, stream);

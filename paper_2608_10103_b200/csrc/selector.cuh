@@ -41,7 +41,7 @@ bool variant_exists(int bn, int cta_group) {
 
 // Kernel variants that take packed INT4 operands and expand them on the way to the MMAs.
 bool fused_s4_variant_exists(int bn, int cta_group, int splits) {
-  if (cta_group == 2) return bn == 256 && splits == 1;
+  if (cta_group == 2) return (bn == 256 || bn == 128) && splits == 1;
   return bn == 256 || bn == 128 || bn == 64 || bn == 32;
 }
 
@@ -60,7 +60,8 @@ int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b
 // force_atoms: K atoms per split unit whatever the tile (the fused INT4 kernel splits K in
 // packed slots = 2 int8 k-blocks); 0 = the tile's own ring slot.
 // split_cap: upper limit of the split-K factor (0 = none).
-// fused_only: 1 = only shapes the fused INT4 kernel is built for, 2 = only its CTA-pair shape.
+// fused_only: 1 = only shapes the fused INT4 kernel is built for, 2 = only its 256-wide
+// CTA-pair shape.
 TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 32,
                          bool allow_split = false, int force_atoms = 0, int split_cap = 0,
                          int fused_only = 0) {
@@ -72,6 +73,7 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
     for (int bn : kWidths) {
       if (g_override_bn && bn != g_override_bn) continue;
       if (!variant_exists(bn, cg) || bn < min_bn) continue;
+      if (fused_only == 2 && bn != 256) continue;
       const long long tiles = static_cast<long long>(ceil_div(M, BM * cg)) * ceil_div(N, bn);
       const long long units = num_sms / cg;
       const int atoms = force_atoms ? force_atoms : atoms_for(bn, cg);

@@ -21,16 +21,17 @@ def _fused_route():
     assert binding.gemm_last_device_status() == 0
 
 
-def _force_pair_tile():
-    binding.gemm_set_config_override(256, 0, 2, 1)   # the only tile the fused variant has
+def _force_pair_tile(bn=256):
+    binding.gemm_set_config_override(bn, 0, 2, 1)    # the pair tiles of the fused variant: 256, 128 wide
 
 
 # K = 32: a single 16-byte chunk per row; 96/160: partly filled packed slots; 256/512: whole
 # slots; 1056, 4128: ragged tails; M, N not tile multiples
 @pytest.mark.parametrize("M,N,K", [(256, 256, 32), (256, 256, 256), (130, 70, 96), (300, 500, 160),
                                    (512, 768, 512), (640, 1100, 1056), (1, 8, 64), (1000, 1000, 4128)])
-def test_fused_full_compare(M, N, K):
-    _force_pair_tile()
+@pytest.mark.parametrize("bn", [256, 128])
+def test_fused_full_compare(M, N, K, bn):
+    _force_pair_tile(bn)
     assert "fused_unpack" in binding.gemm_query_config("s4", M, N, K)
     A, B = synth.s4_uniform(M, N, K, seed=M + K)
     for rep in range(2):
@@ -50,7 +51,7 @@ def test_fused_is_what_the_selector_reports_and_runs_at_2048():
 
 def test_fused_falls_back_where_the_variant_does_not_apply():
     M, N, K = 640, 512, 1056
-    binding.gemm_set_config_override(128, 0, 2, 1)      # no fused variant for this pair tile
+    binding.gemm_set_config_override(64, 0, 2, 1)       # no fused variant for this pair tile
     cfg = binding.gemm_query_config("s4", M, N, K)
     assert "prepass" in cfg and "fused" not in cfg
     A, B = synth.s4_uniform(M, N, K, seed=6)
