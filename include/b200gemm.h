@@ -302,8 +302,7 @@ int gemm_last_device_status(void);
  * its CTA-pair tile if the tiles fill their waves to 75 % (256 x 28672 x 8192:
  * 119 -> 67 us; 512 x 16384 x 4096: 44 -> 35 us); else the pre-pass.  1: always
  * the pre-pass; 2: fused wherever a fused variant is built (every one-CTA tile,
- * and the 256 x 256 and 256 x 128 CTA pairs without split-K), else the
- * pre-pass.  gemm_s4_ws and gemm_s4_static
+ * and the 256 x 256 and 256 x 128 CTA pairs), else the pre-pass.  gemm_s4_ws and gemm_s4_static
  * always use the pre-pass.  Results are identical, bit for bit.
  * gemm_query_config shows the route.  The paper has no counterpart; its Run 4
  * ablates how the operands reach the tensor cores, of which this is the

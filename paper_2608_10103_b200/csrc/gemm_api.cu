@@ -174,8 +174,10 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
   const int user_m = M, user_n = N;
   if (precision == GEMM_PREC_S4 && g_s4_scheme != 1) {  // the decisions of s4_auto / launch_gemm_epi
     swap = swap_ab_wanted(M, N, true, OutputSpec());
-    fused = swap ? select_fused_s4(N, M, user_m, user_n, num_sms, kb, 32, true, &c)
-                 : select_fused_s4(M, N, user_m, user_n, num_sms, kb, 32, true, &c);
+    const TileConfig i8 =
+        swap ? select_config(N, M, num_sms, kb, 32, true) : select_config(M, N, num_sms, kb, 32, true);
+    fused = swap ? select_fused_s4(N, M, user_m, user_n, num_sms, kb, 32, true, i8, &c)
+                 : select_fused_s4(M, N, user_m, user_n, num_sms, kb, 32, true, i8, &c);
   }
   if (!fused) {
     swap = swap_ab_wanted(M, N, precision != GEMM_PREC_FP16, OutputSpec());

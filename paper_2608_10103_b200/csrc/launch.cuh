@@ -140,16 +140,21 @@ bool s4_fused_wanted(int M, int N, const TileConfig& cfg, int num_sms) {
 // expansion inside the kernel costs shared-memory time that grows with the work, M N K, so
 // what decides is M N / (M + N).  Up to 384 the selector's best choice among all the shapes
 // the fused kernel has is taken; up to 1024 rows or columns its 256-wide CTA-pair shape, the
-// efficient one, where the tiles fill their waves to 75 % (it cannot split K).  Measured, packed B
-// from HBM: 256 x 28672 x 8192 119 -> 67 us, 512 x 16384 x 4096 44 -> 35 us, 256 x 8192 x 8192
-// 35 -> 31 us, 1024 x 8192 x 8192 63 -> 60 us; the one-CTA shapes at 640-1024 x 2048 x 8192
-// would lose 15-35 %, and from 1280 rows on the pre-pass is even or ahead.
+// efficient one, where the work units fill their waves to 75 %.  A pair tile that would have
+// to split K where the INT8 kernel behind the pre-pass (`int8_choice`) would not is left to
+// the pre-pass (1024 x 2048 x 8192: 24.1 against 22.5 us).  Measured, packed B from HBM:
+// 256 x 28672 x 8192 119 -> 67 us, 512 x 16384 x 4096 44 -> 35 us, 256 x 8192 x 8192 35 -> 28 us,
+// 512 x 4096 x 16384 49 -> 38 us, 1024 x 8192 x 8192 63 -> 60 us; the one-CTA shapes at
+// 640-1024 x 2048 x 8192 would lose 15-35 %, and from 1280 rows on the pre-pass is even or ahead.
 bool select_fused_s4(int M, int N, int user_m, int user_n, int num_sms, int k_blocks, int min_bn,
-                     bool allow_split, TileConfig* out) {
+                     bool allow_split, const TileConfig& int8_choice, TileConfig* out) {
   if (g_s4_scheme == 1) return false;
   const TileConfig c = select_config(M, N, num_sms, k_blocks, min_bn, allow_split, 2);
+  const auto pair_split_only_here = [&](const TileConfig& f) {
+    return g_s4_scheme == 0 && f.cta_group == 2 && f.splits > 1 && int8_choice.splits == 1;
+  };
   if (c.bn != 0 && fused_s4_variant_exists(c.bn, c.cta_group, c.splits) &&
-      s4_fused_wanted(user_m, user_n, c, num_sms)) {
+      s4_fused_wanted(user_m, user_n, c, num_sms) && !pair_split_only_here(c)) {
     *out = c;
     return true;
   }
@@ -164,10 +169,12 @@ bool select_fused_s4(int M, int N, int user_m, int user_n, int num_sms, int k_bl
   if (user_m <= 1024 || user_n <= 1024) {
     const TileConfig f = select_config(M, N, num_sms, k_blocks, min_bn, allow_split, 2, 0, 2);
     if (f.bn != 0) {
-      const long long tiles = static_cast<long long>(ceil_div(M, 2 * BM)) * ceil_div(N, f.bn);
+      // work units: tiles, those of a split-K part counted once per K range
+      const long long tiles = static_cast<long long>(ceil_div(M, 2 * BM)) * ceil_div(N, f.bn) +
+                              static_cast<long long>(f.split_tiles) * (f.splits - 1);
       const long long pairs = num_sms / 2;
       const long long waves = (tiles + pairs - 1) / pairs;
-      if (4 * tiles >= 3 * waves * pairs) {
+      if (4 * tiles >= 3 * waves * pairs && !pair_split_only_here(f)) {
         *out = f;
         return true;
       }
@@ -196,9 +203,8 @@ constexpr int GEMM_NOT_FUSED = 1;
 
 // A, B in the element type of KIND (fp16 or int8), pitches in bytes.  packed_s4 (KIND_I8
 // only): A and B hold packed signed 4-bit values, K/2 bytes per row, and go to the kernel
-// variant that expands them on the way to the MMAs; that variant exists for the 256 x 256
-// CTA-pair tile without split-K, for any other choice GEMM_NOT_FUSED comes back and nothing
-// has been enqueued.
+// variant that expands them on the way to the MMAs; where select_fused_s4 leaves the problem
+// to the pre-pass GEMM_NOT_FUSED comes back and nothing has been enqueued.
 template <int KIND, int EPI>
 int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const void* B,
                     size_t b_pitch, void* C, const OutputSpec& out, cudaStream_t stream,
@@ -229,7 +235,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   bool fused_cfg = false;
   if (packed_s4)
     fused_cfg = select_fused_s4(M, N, user_m, user_n, s->num_sms, k_blocks, min_bn,
-                                split_through_c, &cfg);
+                                split_through_c, TileConfig(cfg), &cfg);
   if (cfg.bn == 0) return GEMM_ERR_INVALID_ARG;  // override asks for a shape this mode lacks
   // Outputs that cannot be split through C (16-bit, scaled, blocks of a larger C): split-K
   // inside a cluster of two or four CTAs where the kernel has that variant (one-CTA tiles up

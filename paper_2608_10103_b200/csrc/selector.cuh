@@ -41,7 +41,7 @@ bool variant_exists(int bn, int cta_group) {
 
 // Kernel variants that take packed INT4 operands and expand them on the way to the MMAs.
 bool fused_s4_variant_exists(int bn, int cta_group, int splits) {
-  if (cta_group == 2) return (bn == 256 || bn == 128) && splits == 1;
+  if (cta_group == 2) return bn == 256 || bn == 128;
   return bn == 256 || bn == 128 || bn == 64 || bn == 32;
 }
 
@@ -131,7 +131,7 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
     best.split_tiles = best.splits > 1 ? static_cast<int>(tiles) : 0;
     const long long r = tiles % units;
     if (allow_split && best.splits == 1 && g_override_splits == 0 && tiles > units && r > 0 &&
-        2 * r <= units && slots >= 64 && !(fused_only && best.cta_group == 2)) {  // measured: pays off (+2-3 %) only for long K
+        2 * r <= units && slots >= 64) {  // measured: pays off (+2-3 %) only for long K
       int sp = static_cast<int>(units / r);
       if (sp > 4) sp = 4;
       while (sp > 1 && (slots / sp < 32 ||

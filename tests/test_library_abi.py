@@ -134,10 +134,12 @@ def test_selector_invariants_over_many_shapes(lib):
             if "fused_unpack" in text:   # K is split in packed slots of 256 values
                 # a problem with a short side, or a single wave of pair tiles
                 tiles2 = -(-M // 256) * -(-N // bn)
-                assert (M * N <= 512 * (M + N) or (cg == 2 and tiles2 <= 74) or
-                        (cg == 2 and min(M, N) <= 1024 and 4 * tiles2 >= 3 * 74 * -(-tiles2 // 74)))
-                if cg == 2:              # the pair tile is never split
-                    assert bn in (256, 128) and sp == 1
+                units2 = tiles2 + c["split_tiles"] * (sp - 1)
+                assert (M * N <= 512 * (M + N) or (cg == 2 and bn == 256 and tiles2 <= 74) or
+                        (cg == 2 and bn == 256 and min(M, N) <= 1024 and
+                         4 * units2 >= 3 * 74 * -(-units2 // 74)))
+                if cg == 2:
+                    assert bn in (256, 128)
                 atoms = 2
             slots = -(-(-(-K * elem // 128)) // atoms)
             tiles = -(-M // c["BM"]) * -(-N // bn)
