@@ -73,6 +73,19 @@ def test_fused_one_cta_tiles_with_split_k(M, N, K, bn, split_k):
         check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), force_full=True)
 
 
+@pytest.mark.parametrize("split_k", [2, 3, 5])
+@pytest.mark.parametrize("bn", [256, 128])
+@pytest.mark.parametrize("M,N,K", [(300, 500, 1056), (512, 768, 2048), (256, 2048, 8192), (1000, 1000, 4128)])
+def test_fused_pair_tiles_with_split_k(M, N, K, bn, split_k):
+    """K divided in whole packed slots between CTA pairs that add into a zeroed C."""
+    binding.gemm_set_config_override(bn, 0, 2, split_k)
+    cfg = binding.gemm_query_config("s4", M, N, K)
+    assert "fused_unpack" in cfg and "cta_group=2" in cfg
+    A, B = synth.s4_uniform(M, N, K, seed=M + split_k)
+    for rep in range(2):
+        check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), force_full=True)
+
+
 def test_automatic_route_by_shape():
     binding.gemm_set_s4_scheme(0)
     assert "fused_unpack" in binding.gemm_query_config("s4", 16, 8192, 8192)      # few rows
