@@ -104,6 +104,10 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
         if (per_kb < 450) per_kb = 450;
         const long long port = (128 + bn / cg) * 128 / 66;
         if (per_kb < port) per_kb = port;
+        // measured: with a short K (up to 48 k-blocks) the 256 x 128 pair tile runs ahead of
+        // the port figure (2304^3 FP16: 24.4 us against 27.6 on the 256-wide tile, INT8 15.1 / 16.3;
+        // not so the fused INT4 kernel: 256 x 12288 x 1536 14.0 against 12.4 us)
+        if (cg == 2 && bn == 128 && k_blocks <= 48 && force_atoms == 0) per_kb = 320;
         long long cost = waves * per * per_kb + 3000 + 16 * bn + (cg == 2 ? 2500 : 0);
         if (sp > 1) cost += 6000 + static_cast<long long>(M) * N / 250;  // zeroing C + adding into it
         if (best_cost < 0 || cost < best_cost) {
