@@ -101,13 +101,7 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
         const int per = ceil_div(slots, sp) * atoms;  // k-blocks per unit
         const long long waves = (tiles * sp + units - 1) / units;
         long long per_kb = 2 * bn;
-        // the issuing thread: ~450 cycles per k-block on the one-CTA tiles (and in the fused INT4
-        // kernel), ~250 on the pair tiles, where one thread issues for two SMs' worth of operands
-        // (not applied to problems with a short side, which stream the other operand from HBM
-        // and are 5-9 % faster on one-CTA tiles: 16 x 8192 x 8192 exchanged, INT8 15.9 against
-        // 17.2 us; 64 x 8192 x 8192 with FP16 output 30.8 against 32.9 us)
-        const long long issue = (cg == 2 && force_atoms == 0 && N >= 256 && M > 128) ? 256 : 450;
-        if (per_kb < issue) per_kb = issue;
+        if (per_kb < 450) per_kb = 450;
         const long long port = (128 + bn / cg) * 128 / 66;
         if (per_kb < port) per_kb = port;
         // measured: with a short K (up to 48 k-blocks) the 256 x 128 pair tile runs ahead of
