@@ -605,6 +605,71 @@ def run_few_rows(args):
         raise SystemExit("bench.py: a kernel reported a barrier timeout")
 
 
+def run_selector_check(args):
+    """The selector's automatic choice against forced tile shapes and split-K factors: one JSON
+    line per (shape, precision) with the automatic time, the best forced time and configuration,
+    and the regret = automatic / best - 1.  CUDA-graph replay of 20 calls, median of 3, operands
+    seeded and resident (square and rectangular shapes between 256 and 4096; the few-row shapes
+    have a mode of their own)."""
+    import statistics
+    import torch
+    from paper_2608_10103_b200 import binding, synth
+    torch.cuda.set_device(0)
+    forced = [(256, 0, 2, 1), (128, 0, 2, 1), (64, 0, 2, 1), (256, 0, 1, 1), (128, 0, 1, 1),
+              (64, 0, 1, 1), (32, 0, 1, 1), (256, 0, 2, 2), (128, 0, 2, 2), (256, 0, 1, 2),
+              (128, 0, 1, 2), (64, 0, 1, 2), (256, 0, 2, 3), (128, 0, 1, 4), (64, 0, 1, 4), (32, 0, 1, 8)]
+    shapes = [(n, n, n) for n in (512, 768, 1024, 1280, 1536, 1792, 2048, 2304, 2560, 2816, 3072,
+                                  3584, 4096)]
+    shapes += [(512, 8192, 4096), (1024, 4096, 8192), (2048, 8192, 2048), (4096, 1024, 4096),
+               (2304, 2304, 8192), (2560, 2560, 1024), (1792, 3584, 4096), (3000, 3000, 1024),
+               (640, 1280, 2560), (384, 768, 4096), (512, 512, 8192), (768, 3072, 768)]
+    if args.shape:
+        shapes = [tuple(int(x) for x in args.shape.split(","))]
+
+    def timed(call, reps=20):
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for _ in range(reps):
+                call()
+        g.replay()
+        torch.cuda.synchronize()
+        out = []
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            out.append(e0.elapsed_time(e1) * 1e3 / reps)
+        return statistics.median(out)
+
+    for M, N, K in shapes:
+        for prec in [q for q in ("fp16", "s8") if q in args.precisions.split(",")]:
+            A, B = synth.make(prec, M, N, K, seed=M + N + K)
+            dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+            C = torch.empty((M, N), dtype=torch.float32 if prec == "fp16" else torch.int32, device="cuda")
+            binding.gemm_set_config_override(0, 0, 0, 0)
+            auto_us = timed(lambda: binding.gemm(prec, dA, dB, C))
+            chosen = binding.gemm_query_config(prec, M, N, K)
+            best_us, best_cfg = None, None
+            for cfg in forced:
+                binding.gemm_set_config_override(*cfg)
+                try:
+                    us = timed(lambda: binding.gemm(prec, dA, dB, C))
+                except binding.GemmError:
+                    continue
+                if best_us is None or us < best_us:
+                    best_us, best_cfg = us, cfg
+            binding.gemm_set_config_override(0, 0, 0, 0)
+            print(json.dumps({"selector_check": True, "M": M, "N": N, "K": K, "precision": prec,
+                              "auto_us": auto_us, "chosen": chosen, "best_forced_us": best_us,
+                              "best_forced": "BN=%d cta_group=%d split_k=%d" % (best_cfg[0], best_cfg[2], best_cfg[3]),
+                              "regret": auto_us / best_us - 1.0}), flush=True)
+
+
 def run_ablation(args):
     """One-variable-at-a-time ablation at N = args.size (the analogue of the paper's Run 4):
     tile shape, raster band height, L2 policy, and load-only / MMA-only runs, each with
@@ -709,6 +774,8 @@ def main():
     ap.add_argument("--shape", default="", help="--few-rows: only this M,N,K")
     ap.add_argument("--ablation", action="store_true",
                     help="tile / raster / L2 / load-vs-MMA ablation with cycle accounting (1 GPU)")
+    ap.add_argument("--selector-check", action="store_true",
+                    help="automatic tile / split-K choice against forced ones, one JSON line per shape")
     ap.add_argument("--sweep", action="store_true",
                     help="precision x size sweep N=512..8192, one JSON line per cell (1 GPU)")
     ap.add_argument("--precisions", default="fp16,s8,s4")
@@ -720,7 +787,10 @@ def main():
         args.warmup = 3
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.ablation:
+    if args.selector_check:
+        if rank == 0:
+            run_selector_check(args)
+    elif args.ablation:
         if rank == 0:
             run_ablation(args)
     elif args.few_rows:
