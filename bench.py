@@ -17,7 +17,9 @@ replica of the same workload (no data-path collective; weak scaling).
 
 Other modes (1 GPU, one JSON line per measurement): --sweep (precision x size,
 N = 512..8192), --ablation (tile / raster / L2 / INT4 route at --size, with the
-kernel's cycle accounting), --few-rows (M = 1..128 against the HBM roofline).
+kernel's cycle accounting), --few-rows (M = 1..128 against the HBM roofline;
+--shape M,N,K for any other shape), --selector-check (the automatic tile and
+split-K choice against forced ones).
 """
 from __future__ import annotations
 
