@@ -290,7 +290,7 @@ int gemm_last_device_status(void);
  *     for an operand that is read once; but half as much shared-memory traffic
  *     again per unit of math, which is what bounds the large-tile kernel.
  * Measured: at M = N = K = 8192 the pre-pass route is 1.1-1.35x faster; for
- * M = 16, N = K = 8192 (bound by the bytes of B) the fused route takes 16 us
+ * M = 16, N = K = 8192 (bound by the bytes of B) the fused route takes 15 us
  * instead of 33.
  * Small problems, bound by launches and latencies, save one launch with the
  * fused route (10-26 % up to 1024 x 1024 outputs).

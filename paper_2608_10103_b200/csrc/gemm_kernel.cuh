@@ -241,6 +241,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
   using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, CSPLIT>;
   constexpr bool FUSED = PSTAGES > 0;  // packed INT4 operands, expanded on the way to the MMAs
+  // fused INT4: the expansion warps work as one group of eight, or -- where both rings are at
+  // least four slots deep -- as two groups of four on alternate packed slots
+  constexpr int UNPACK_GROUPS = (STAGES >= 4 && PSTAGES >= 4) ? 2 : 1;
+  constexpr int GROUP_WARPS = UNPACK_WARPS / UNPACK_GROUPS;
   // CSPLIT = 2 or 4 (cluster split-K): a cluster of CSPLIT single CTAs owns every tile; each
   // takes its share of K into its own accumulator, the CTAs of rank 1.. hand their 128 x BN
   // partial sums to rank 0 through the cluster's shared-memory window (one buffer each), and
@@ -335,11 +339,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     for (int s = 0; s < STAGES; ++s) {
       ptx::mbar_init(full_bar(s), 1);
       ptx::mbar_init(empty_bar(s), 1);
-      if constexpr (FUSED) ptx::mbar_init(ready_bar(s), UNPACK_WARPS);
+      if constexpr (FUSED) ptx::mbar_init(ready_bar(s), GROUP_WARPS);
     }
     for (int s = 0; s < PSTAGES; ++s) {
       ptx::mbar_init(p_full_bar(s), 1);
-      ptx::mbar_init(p_empty_bar(s), UNPACK_WARPS);
+      ptx::mbar_init(p_empty_bar(s), GROUP_WARPS);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(acc_full_bar(a), 1);
@@ -612,7 +616,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     // chunk read at offset x.  Lane -> (row, chunk) is chosen so that each quarter-warp reads
     // and writes all 32 banks once.
     if constexpr (FUSED) {
-      const int uw = warp - (2 + EPI_WARPS);
+      // With deep rings (the narrow tiles of problems with few rows) the eight warps work as
+      // two groups on alternate packed slots: a slot's fixed costs -- three barrier waits, the
+      // proxy fence, the arrives: ~700 of the ~1300 cycles a slot took -- then overlap.
+      const int uw = (warp - (2 + EPI_WARPS)) % GROUP_WARPS;  // warp within its group
+      const int ugroup = (warp - (2 + EPI_WARPS)) / GROUP_WARPS;
+      int pcount = 0;                                          // packed slots so far, all tiles
       const int c = lane & 3;
       const int row_in_8 = (lane >> 3) + 4 * ((lane >> 2) & 1);
       constexpr uint32_t HI = 0xF0F0F0F0u;
@@ -630,14 +639,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         // problem with few rows (M = 16) skips most of the A tile.
         const int a_valid = p.M - (tm * TILE_M + static_cast<int>(cta_rank) * BM);
         const int b_valid = p.N - (tn * BN + static_cast<int>(cta_rank) * L::B_ROWS);
-        constexpr int TASKS = (BM + L::B_ROWS + 8 * UNPACK_WARPS - 1) / (8 * UNPACK_WARPS);
+        constexpr int TASKS = (BM + L::B_ROWS + 8 * GROUP_WARPS - 1) / (8 * GROUP_WARPS);
         bool active[TASKS];
 #pragma unroll
         for (int i = 0; i < TASKS; ++i) {
-          const int row8 = (i * UNPACK_WARPS + uw) * 8;  // first row of this lane's group of 8
+          const int row8 = (i * GROUP_WARPS + uw) * 8;  // first row of this lane's group of 8
           active[i] = row8 < BM ? row8 < a_valid : (row8 < BM + L::B_ROWS && row8 - BM < b_valid);
         }
-        for (int ps = k_begin / 2; ps < k_end / 2 && ok; ++ps) {
+        for (int ps = k_begin / 2; ps < k_end / 2 && ok; ++ps, ++pcount) {
+          if (UNPACK_GROUPS > 1 && pcount % UNPACK_GROUPS != ugroup) {
+            // the other group's slot: only keep the ring positions in step
+            ustage += 2;
+            if (ustage >= STAGES) { ustage -= STAGES; uphase ^= 1u; }
+            if (++pstage == PSTAGES) { pstage = 0; pphase ^= 1u; }
+            continue;
+          }
           const long long w0 = trace ? clock64() : 0;
           ok = wait_bounded(p_full_bar(pstage), pphase, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
           ok = __all_sync(0xffffffffu, ok);
@@ -666,12 +682,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 #pragma unroll
             for (int i = 0; i < TASKS; ++i)
               if (active[i])
-                ptx::ld_shared_v4(src + x0 + static_cast<uint32_t>((i * UNPACK_WARPS + uw) * 8 * 128),
+                ptx::ld_shared_v4(src + x0 + static_cast<uint32_t>((i * GROUP_WARPS + uw) * 8 * 128),
                                   wv[i][0], wv[i][1], wv[i][2], wv[i][3]);
 #pragma unroll
             for (int i = 0; i < TASKS; ++i) {
               if (!active[i]) continue;
-              const uint32_t x = x0 + static_cast<uint32_t>((i * UNPACK_WARPS + uw) * 8 * 128);
+              const uint32_t x = x0 + static_cast<uint32_t>((i * GROUP_WARPS + uw) * 8 * 128);
               ptx::st_shared_v4(dst + (x ^ flip), (wv[i][0] << 4) & HI, (wv[i][1] << 4) & HI,
                                 (wv[i][2] << 4) & HI, (wv[i][3] << 4) & HI);
               ptx::st_shared_v4(dst + (x ^ flip ^ 64u), wv[i][0] & HI, wv[i][1] & HI, wv[i][2] & HI,
@@ -694,7 +710,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           if (++pstage == PSTAGES) { pstage = 0; pphase ^= 1u; }
         }
       }
-      if (trace && uw == 0 && lane == 0) {
+      if (trace && uw == 0 && ugroup == 0 && lane == 0) {
         trace[TRACE_UNPACK_WAIT_IN] = static_cast<unsigned long long>(wait_in);
         trace[TRACE_UNPACK_WAIT_OUT] = static_cast<unsigned long long>(wait_out);
         trace[TRACE_UNPACK_BUSY] = static_cast<unsigned long long>(busy);
