@@ -311,7 +311,7 @@ def gemm_set_s4_scheme(scheme: int = 0):
 
 def gemm_set_swap_ab(mode: int = 0):
     """Run the kernel on exchanged operands (long operand on the 128-row tile side, C stored
-    along N by plain stores): 0 = automatic (N >= 1024 and M <= 32, M <= 64 for INT8 / INT4), 1 = never, 2 = always."""
+    along N by plain stores): 0 = automatic (N >= 1024 and M <= 32, M <= 64 for INT8 / INT4 / FP16 output), 1 = never, 2 = always."""
     _check(lib().gemm_set_swap_ab(int(mode)), "gemm_set_swap_ab")
 
 

@@ -187,14 +187,15 @@ bool select_fused_s4(int M, int N, int user_m, int user_n, int num_sms, int k_bl
 // side of a tile is then filled by the long operand of a problem with few rows (LLM decoding:
 // M = 1..64), instead of 128 - M rows of zero fill taking shared memory, ring depth and, on
 // the fused INT4 route, expansion work; C goes out by plain stores that are contiguous along
-// the caller's N.  Automatic when N >= 1024 and M <= 32 (FP16) or M <= 64 (the integer kinds,
-// both INT4 routes): measured 2-12 % faster there (INT8, M = 48-64: 3-8 %; FP16 even; from
-// M = 80 on, where the narrow side needs the 128-wide tile, 4-20 % slower).
+// the caller's N.  Automatic when N >= 1024 and M <= 32 (FP16 with FP32 output) or M <= 64 (the
+// integer kinds, both INT4 routes, and FP16 with FP16 output): measured 2-12 % faster there
+// (INT8, M = 48-64: 3-8 %; FP16 -> FP16, M = 40-64: 1-13 %; FP16 -> FP32 even; from M = 80 on,
+// where the narrow side needs the 128-wide tile, 4-20 % slower).
 bool swap_ab_wanted(int M, int N, bool integer_kind, const OutputSpec& out) {
   if (out.no_split || out.ldc) return false;  // C is a block of a larger matrix
   if (g_swap_ab == 1) return false;
   if (g_swap_ab == 2) return true;
-  return N >= 1024 && M <= (integer_kind ? 64 : 32);
+  return N >= 1024 && M <= ((integer_kind || out.epi == EPI_OUT16) ? 64 : 32);
 }
 
 // Returned (never to the caller of the library) when the fused INT4 kernel does not cover the
