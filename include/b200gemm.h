@@ -317,8 +317,8 @@ int gemm_set_s4_scheme(int scheme);
  * few rows (M = 1..64, LLM decoding) this keeps 128 - M rows of zero fill out
  * of shared memory, of the ring depth and -- on the fused INT4 route -- of the
  * expansion work.  mode 0 (default, automatic): when N >= 1024 and M <= 32
- * (gemm_fp16) or M <= 64 (INT8, INT4, gemm_fp16_f16out) (measured 2-12 % faster
- * there); 1: never; 2: always
+ * (gemm_fp16) or M <= 64 (INT8, INT4, gemm_fp16_f16out, and gemm_fp16 from
+ * N = 16384 on) (measured 2-12 % faster there); 1: never; 2: always
  * (any shape, precision and INT4 route; for tests and measurements).  Results:
  * integers identical; FP16 within the bound; dequantised outputs multiply the
  * two scales in the other order (last-bit differences).  gemm_query_config

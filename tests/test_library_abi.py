@@ -125,7 +125,7 @@ def test_selector_invariants_over_many_shapes(lib):
             text = binding.gemm_query_config(prec, M, N, K)
             c = _parse(text)
             if "swap_ab" in text:        # the tile is described in the kernel's orientation
-                assert N >= 1024 and M <= (32 if prec == "fp16" else 64)
+                assert N >= 1024 and M <= (32 if prec == "fp16" and N < 16384 else 64)
                 M, N = N, M
             cg, bn, sp = c["cta_group"], c["BN"], c["split_k"]
             assert (cg, bn) in built and c["BM"] == 128 * cg
