@@ -300,3 +300,35 @@ def test_cluster_split_k_dequantised_int4(M, N, K, bn, scheme):
         binding.gemm_set_swap_ab(0)
         binding.gemm_set_s4_scheme(0)
         binding.gemm_trace_enable(0)
+
+
+def test_cluster_split_k_and_fused_int4_share_the_gpu_from_two_streams():
+    """Clusters of four (INT8 dequantised to FP16) and the fused few-row INT4 kernel, enqueued
+    alternately on two streams without any synchronisation in between, so that CTAs of both are
+    resident at once: every result of both must be right."""
+    M, N, K = 16, 4096, 8192
+    g = np.random.Generator(np.random.PCG64(5))
+    rs = (g.uniform(0.5, 2.0, M) * 1e-2).astype(np.float32)
+    cs = (g.uniform(0.5, 2.0, N) * 1e-1).astype(np.float32)
+    A8, B8 = synth.s8_uniform(M, N, K, seed=51)
+    A4, B4 = synth.s4_uniform(M, N, K, seed=52)
+    ref8 = oracle.dequant_ref(oracle.gemm_s8_i64(A8, B8), rs, cs)
+    ref4 = oracle.gemm_s4(A4, B4, K)
+    dA8, dB8, dA4, dB4, d_rs, d_cs = (to_dev(x) for x in (A8, B8, A4, B4, rs, cs))
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs8, outs4 = [], []
+    for rep in range(12):
+        C8 = torch.full((M, N), float("nan"), dtype=torch.float16, device="cuda")
+        C4 = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
+        s1.wait_stream(torch.cuda.current_stream())
+        s2.wait_stream(torch.cuda.current_stream())
+        binding.gemm_s8_dequant(dA8, dB8, d_rs, d_cs, C8, torch.float16, stream=s1)
+        binding.gemm_s4(dA4, dB4, C4, stream=s2)
+        outs8.append(C8)
+        outs4.append(C4)
+    s1.synchronize()
+    s2.synchronize()
+    for C8, C4 in zip(outs8, outs4):
+        assert oracle.dequant_check(C8.cpu().numpy(), ref8, True)[0]
+        assert np.array_equal(C4.cpu().numpy(), ref4)
