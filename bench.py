@@ -39,10 +39,28 @@ if ROOT not in sys.path:
 SPEC_PEAK = {"fp16": 2250.0, "s8": 4500.0, "s4": 4500.0}   # vendor dense figures, T(FL)OP/s
 UNIT = {"fp16": "TFLOP/s", "s8": "TOP/s", "s4": "TOP/s"}
 KERNEL_LAUNCHES = {"fp16": 1, "s8": 1, "s4": 2}            # s4: unpack launch + GEMM
-# DRAM bytes per launch of the FP16 GEMM kernel (dram__bytes_read.sum + dram__bytes_write.sum
-# from one ncu capture of this workload; profiles/gemm_kernels_n8192_ncu_metrics.md and
-# profiles/gemm_kernel_fp16_n4096_ncu_full.md).  Sizes that were not captured report null.
-NCU_TRAFFIC_BYTES = {"fp16": {8192: 835034880 + 253426176, 4096: 104337920 + 40935936}}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic_fp16_gemm.txt")
+
+
+def captured_traffic(size, lib_version):
+    """DRAM bytes per launch of the FP16 GEMM kernel from the last profiler capture of this
+    workload (key = value lines written beside the capture's summary), or None when no capture
+    of this size exists or it was taken with another version of the library."""
+    try:
+        kv = {}
+        with open(TRAFFIC_FILE) as f:
+            for line in f:
+                if "=" in line and not line.lstrip().startswith("#"):
+                    k, v = line.split("=", 1)
+                    kv[k.strip()] = v.strip()
+        if int(kv["library_version"]) != lib_version:
+            return None, "capture is of library version %s" % kv["library_version"]
+        r, w = kv.get("n%d_dram_read_bytes" % size), kv.get("n%d_dram_write_bytes" % size)
+        if r is None or w is None:
+            return None, "no capture at this size"
+        return int(r) + int(w), kv.get("capture", "")
+    except (OSError, KeyError, ValueError):
+        return None, "no capture on file"
 
 
 def measured_peaks():
@@ -144,6 +162,10 @@ class ClockSampler:
                 "sm_min_mhz": min(self.sm) if self.sm else None,
                 "sm_max_mhz": self.sm_max,
                 "power_w_max": max(self.pw) if self.pw else None,
+                "power_w_mean": statistics.mean(self.pw) if self.pw else None,
+                # second half of the samples: the regime the region settled in
+                "sm_mhz_settled": statistics.median(self.sm[len(self.sm) // 2:]) if self.sm else None,
+                "power_w_settled": statistics.median(self.pw[len(self.pw) // 2:]) if self.pw else None,
                 "samples": len(self.sm),
                 "source": "nvml" if self.nvml is not None else "nvidia-smi",
                 "reasons": sorted(name for bit, name in self.REASONS if self.mask & bit)}
@@ -274,11 +296,11 @@ def run_ours(args, rank, world):
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()                       # before the warm-up, so that short runs get samples too
     for _ in range(args.warmup):
         step()
     barrier()
-    sampler = ClockSampler(physical_gpu_index(local))
-    sampler.start()
     evs = [{p: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
             for p in precs} for _ in range(args.steps)]
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -304,15 +326,43 @@ def run_ours(args, rank, world):
     #      precision gives the SM cycles it took and the SM clock it ran at
     cycles = {}
     flop_per_clk = {"fp16": 8192, "s8": 16384, "s4": 16384}   # per SM, dense, from the probe below
+    num_sms = torch.cuda.get_device_properties(local).multi_processor_count
     binding.gemm_trace_enable(1)
     for p in precs:
         binding.gemm(p, dev[p][0], dev[p][1], out[p], stream)
-        tr = binding.gemm_trace_read(148)
+        tr = binding.gemm_trace_read(num_sms)
         cyc = max(t["cycles"] for t in tr)
         mhz = statistics.median(t["cycles"] / t["nanos"] * 1e3 for t in tr if t["nanos"])
         cycles[p] = {"sm_cycles": cyc, "sm_mhz_during_kernel": mhz,
-                     "pipe_utilisation": ops / (148 * flop_per_clk[p]) / cyc}
+                     "pipe_utilisation": ops / (num_sms * flop_per_clk[p]) / cyc}
     binding.gemm_trace_enable(0)
+
+    # ---- the sustained regime: each precision alone, back to back for >= --sustain-seconds,
+    #      with the clock and power NVML saw meanwhile (energy per GEMM = mean power x time)
+    sustained = {}
+    if args.sustain_seconds > 0:
+        for p in precs:
+            n = max(args.steps, int(args.sustain_seconds * 1e3 / max(per_prec_ms[p], 1e-3)) + 1)
+            barrier()
+            s2 = ClockSampler(physical_gpu_index(local))
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s2.start()
+            e0.record(stream)
+            for _ in range(n):
+                binding.gemm(p, dev[p][0], dev[p][1], out[p], stream)
+            e1.record(stream)
+            barrier()
+            c2 = s2.stop()
+            ms = replicas.max_over_ranks([e0.elapsed_time(e1) / n], dist, "cuda")[0]
+            sustained[p] = {"launches": n, "seconds": ms * n * 1e-3, "ms": ms,
+                            "value": replicas.whole_job_rate(ops, world, ms), "unit": UNIT[p],
+                            "sm_mhz_settled": c2.get("sm_mhz_settled"),
+                            "power_w_settled": c2.get("power_w_settled"),
+                            "joules_per_gemm": (c2["power_w_mean"] * ms * 1e-3
+                                                if c2.get("power_w_mean") else None),
+                            "clock_samples": c2.get("samples"), "reasons": c2.get("reasons")}
+        if binding.gemm_last_device_status() != 0:
+            raise SystemExit("bench.py: a kernel reported a barrier timeout")
 
     # ---- MMA-issue-only peak of this machine, per kind (same run, same power regime): rate by
     #      CUDA events, cycles per 128x256x(32 B) MMA and clock by the probe's own counters
@@ -326,7 +376,7 @@ def run_ours(args, rank, world):
         pops = binding.gemm_mma_peak_probe(kind, 200000)
         e1.record(stream)
         torch.cuda.synchronize()
-        tr = binding.gemm_trace_read(148)
+        tr = binding.gemm_trace_read(num_sms)
         binding.gemm_trace_enable(0)
         mma_peak[kind] = pops / (e0.elapsed_time(e1) * 1e-3) / 1e12
         mma_detail[kind] = {
@@ -367,9 +417,6 @@ def run_ours(args, rank, world):
         return
 
     peaks = measured_peaks()
-    # the GEMMs are timed inside a long back-to-back loop -> sustained figure
-    ref_peak = {"fp16": peaks["bf16_sustained"], "s8": 2 * peaks["bf16_sustained"],
-                "s4": 2 * peaks["bf16_sustained"]}
     precisions = {}
     for p in precs:
         rate = replicas.whole_job_rate(ops, world, worst[p])
@@ -382,11 +429,25 @@ def run_ours(args, rank, world):
             "sm_mhz_during_kernel": cycles[p]["sm_mhz_during_kernel"],
             "config": binding.gemm_query_config(p, N, N, N),
         }
+        if p in sustained:
+            sus = dict(sustained[p])
+            sus["frac_of_spec_peak"] = sus["value"] / world / SPEC_PEAK[p]
+            precisions[p]["sustained"] = sus
     if "s4" in worst and "s8" in worst:
         precisions["s4"]["overhead_vs_s8"] = worst["s4"] / worst["s8"] - 1.0
 
     fp16_rate_1gpu = ops / (worst["fp16"] * 1e-3) / 1e12
-    traffic = NCU_TRAFFIC_BYTES["fp16"].get(N)
+    traffic, traffic_note = captured_traffic(N, binding.gemm_version())
+    # Which measured peak applies: the burst figure for a timed region shorter than a second
+    # (the clock has not settled under the power cap), the sustained one for longer regions.
+    region_s = total_ms * 1e-3
+    short = region_s < 1.0
+    frac_burst = fp16_rate_1gpu / peaks["bf16_burst"]
+    frac_sustained = None
+    if "fp16" in sustained:
+        frac_sustained = sustained["fp16"]["value"] / world / peaks["bf16_sustained"]
+    elif not short:
+        frac_sustained = fp16_rate_1gpu / peaks["bf16_sustained"]
     line = {
         "metric": "fp16_gemm_tflops_n%d" % N, "value": precisions["fp16"]["value"],
         "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -400,10 +461,23 @@ def run_ours(args, rank, world):
         },
         "precisions": precisions,
         "roofline": {
-            "bound": "tensor", "achieved": fp16_rate_1gpu, "peak": ref_peak["fp16"],
-            "unit": "TFLOP/s", "frac": fp16_rate_1gpu / ref_peak["fp16"], "traffic": traffic,
-            "peak_source": "%s cuBLAS bf16 sustained (kernel timed inside a long step)" % peaks["source"],
-            "kernel": "gemm_kernel<f16> N=%d, avg of %d launches" % (N, args.steps),
+            "bound": "tensor", "achieved": fp16_rate_1gpu,
+            "peak": peaks["bf16_burst"] if short else peaks["bf16_sustained"],
+            "unit": "TFLOP/s",
+            "frac": frac_burst if short else fp16_rate_1gpu / peaks["bf16_sustained"],
+            "frac_burst": frac_burst, "frac_sustained": frac_sustained,
+            "peak_burst": peaks["bf16_burst"], "peak_sustained": peaks["bf16_sustained"],
+            "peak_spec": SPEC_PEAK["fp16"], "frac_of_spec": fp16_rate_1gpu / SPEC_PEAK["fp16"],
+            "timed_region_s": region_s,
+            "traffic": traffic, "traffic_source": traffic_note,
+            "algorithmic_bytes": 2 * N * N * 2 + 4 * N * N,
+            "peak_source": "%s cuBLAS bf16 %s figure: the timed region lasted %.3f s (< 1 s: burst, "
+                           "else sustained); frac_sustained is the separate >= %.0f s FP16-only "
+                           "leg against the sustained figure"
+                           % (peaks["source"], "burst" if short else "sustained", region_s,
+                              args.sustain_seconds),
+            "kernel": "FP16 GEMM kernel N=%d (%s), avg of %d launches"
+                      % (N, precisions["fp16"]["config"].split(" kind")[0], args.steps),
         },
         "clocks": clocks,
         "e2e": e2e,
@@ -680,6 +754,7 @@ def run_ablation(args):
     import torch
     from paper_2608_10103_b200 import binding, synth
     torch.cuda.set_device(0)
+    num_sms = torch.cuda.get_device_properties(0).multi_processor_count
     N = args.size
     ops = synth.gemm_ops(N, N, N)
     data = {"fp16": synth.fp16_normal_clipped(N, N, N, seed=3),
@@ -727,7 +802,7 @@ def run_ablation(args):
             e1.record()
             torch.cuda.synchronize()
             ms = e0.elapsed_time(e1) / args.steps
-            tr = binding.gemm_trace_read(148)
+            tr = binding.gemm_trace_read(num_sms)
             a = {k: np.array([t[k] for t in tr], dtype=np.float64) for k in binding.TRACE_FIELDS}
             lead = a["mma_issue"] > 0
             kb_total = a["tiles"].mean() * (N * (2 if prec == "fp16" else 1) // 128)
@@ -741,7 +816,7 @@ def run_ablation(args):
             print(json.dumps({
                 "ablation": name, "precision": prec, "N": N, "config": cfg,
                 "ms": ms, "value": ops / (ms * 1e-3) / 1e12, "unit": UNIT[prec],
-                "sm_cycles": cyc, "pipe_utilisation": ops / (148 * flop_per_clk) / cyc,
+                "sm_cycles": cyc, "pipe_utilisation": ops / (num_sms * flop_per_clk) / cyc,
                 "sm_mhz_during_kernel": float(np.median(a["cycles"] / a["nanos"] * 1e3)),
                 "cycles_per_kblock": {
                     "mma_wait_operands": float(a["mma_wait_operands"][lead].mean() / kb_total),
@@ -767,6 +842,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--size", type=int, default=8192)
     ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--sustain-seconds", type=float, default=2.0,
+                    help="length of the per-precision back-to-back legs (0 = skip them)")
     ap.add_argument("--ref-rows", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-peak-probe", action="store_true")

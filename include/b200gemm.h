@@ -33,8 +33,11 @@
  * differ in the last bits, always inside the stated bound.
  *
  * All functions return GEMM_OK (0) or a negative GEMM_ERR_* code.
- * A process may call from several host threads; calls that share a stream are
- * ordered by it.
+ * A process may call from several host threads (the call path takes no global
+ * lock); calls that share a stream are ordered by it, and two threads that
+ * enqueue on the same stream at once get an unspecified order, as with any CUDA
+ * work.  Tensor-map descriptors are cached per thread, keyed on pointer, extents
+ * and pitch, so repeated calls on the same buffers skip their encoding.
  */
 #ifndef B200GEMM_H_
 #define B200GEMM_H_
@@ -90,12 +93,18 @@ int gemm_s8(int M, int N, int K, const int8_t* A, const int8_t* B, int32_t* C,
  * workspace of gemm_s4_workspace_bytes(M, N, K) bytes and then multiplied by the
  * INT8 kernel.  Small problems and problems with few rows: a kernel variant
  * expands the nibbles on the way to the MMAs and needs no workspace (see
- * gemm_set_s4_scheme for the rule and the switch).  For the pre-pass gemm_s4
- * keeps one grow-only workspace per device inside the library:
- * the first call on a device (and any call that needs a larger one) allocates
- * with cudaMalloc, which synchronises the device; the buffer is reused by later
- * calls, so concurrent gemm_s4 calls on different streams of one device must be
- * ordered by the caller.  Use gemm_s4_ws to supply the workspace yourself.
+ * gemm_set_s4_scheme in b200gemm_debug.h for the rule and the switch).  For
+ * the pre-pass the library leases a scratch buffer from a per-device pool for
+ * the call's stream: the first call on a stream (and any call that needs a
+ * larger one) allocates with cudaMallocAsync on that stream -- no device-wide
+ * synchronisation -- and later calls on the stream reuse it, so calls on
+ * different streams never share scratch.  A buffer whose last use has finished
+ * may move to another stream.  While a stream is being captured into a graph
+ * nothing can be allocated: make one call of the same size outside the capture
+ * first; the captured call then keeps using that buffer, and keeping replays of
+ * the graph apart from other gemm_s4 calls that may use it is the caller's job.
+ * gemm_release_workspaces frees the pool.  Use gemm_s4_ws to supply the scratch
+ * yourself.
  * Alignment: A, B, C 16-byte aligned; K % 32 == 0; K <= 131071.
  */
 int gemm_s4(int M, int N, int K, const uint8_t* A, const uint8_t* B, int32_t* C,
@@ -196,7 +205,13 @@ int gemm_host_release(void);
  *     process exits.
  *   - The first call on each device looks up the array's device address (one
  *     cudaGetSymbolAddress, with that device current).  Make that first call
- *     before starting any stream capture.
+ *     before starting any stream capture.  The array is part of the library's
+ *     device code image, which the CUDA runtime places in device memory when the
+ *     image is first needed on a device -- by any call of this library there.  A
+ *     process that is about to hand all remaining device memory to its own pool
+ *     should therefore make one call into the library on each device first (any
+ *     entry point that launches, e.g. a tiny gemm_s4_static), so that the image
+ *     and its 32 MiB are in place before the memory is gone.
  *   - All calls on a device share the one array: calls that may overlap on the
  *     GPU (different streams without an ordering between them) race on it and
  *     give wrong results.  Calls on one stream are safe.  The array keeps the
@@ -211,8 +226,9 @@ int gemm_s4_static(int M, int N, int K, const uint8_t* A, const uint8_t* B, int3
 size_t gemm_s4_static_capacity(void);
 
 /*
- * Frees the per-device workspaces held for gemm_s4 (synchronises).  Optional;
- * they are otherwise released when the process exits.
+ * Frees the scratch buffers the library holds for gemm_s4 / gemm_s4_dequant on
+ * every device (synchronises each device that has any).  Optional; they are
+ * otherwise released when the process exits.
  */
 int gemm_release_workspaces(void);
 
@@ -228,23 +244,6 @@ int gemm_unpack_s4(int rows, int K, const uint8_t* packed, int8_t* out, size_t o
                    gemm_stream_t stream);
 
 /*
- * Measurement aid (Sec. III-B profiles every kernel against the hardware's
- * limits): every SM issues `iters` back-to-back tcgen05.mma instructions of
- * shape 128 x n_cols x (32 bytes of K) on shared-memory operands that are never
- * reloaded, and the operation count performed is added to *ops_out (host
- * pointer).  n_cols: multiple of 16 up to 256 (256 = the production tile).
- * iters is rounded down to a multiple of 4 (MMAs are issued in groups of 4, one
- * k-block of the GEMM kernels).  commit_every: 0 = none inside the loop; c > 0 =
- * a tcgen05.commit after every c groups, as a pipelined GEMM does once per
- * k-block (c = 1).
- * Time it with events on `stream` for the MMA-issue-only rate of the given
- * precision (GEMM_PREC_FP16 or GEMM_PREC_S8); with tracing on, words [0] and
- * [1] of each CTA's trace record hold the cycles and nanoseconds of the loop.
- */
-int gemm_mma_peak_probe(int precision, int iters, int n_cols, int commit_every, double* ops_out,
-                        gemm_stream_t stream);
-
-/*
  * Writes a human-readable description of the tile configuration the selector
  * picks for this problem ("BM=256 BN=256 BK=64 cta_group=2 stages=6 group_m=12
  * split_k=1 split_tiles=0 tiles=1024 ctas=148 kind=f16") into buf (NUL
@@ -257,138 +256,19 @@ int gemm_mma_peak_probe(int precision, int iters, int n_cols, int commit_every, 
 int gemm_query_config(int precision, int M, int N, int K, char* buf, int len);
 
 /*
- * Overrides the selector for later calls from this process: tile width BN
- * (0 = automatic), raster band height in tiles (0 = automatic), the number
- * of CTAs that share one tile (0 = automatic, 1 = 128 x BN tile per CTA, 2 =
- * 256 x BN tile per CTA pair) and the split-K factor (0 = automatic, 1 = off,
- * s = every C tile is computed by s work units over disjoint K ranges; capped
- * at the number of 128-byte K blocks; honoured only by gemm_fp16 / gemm_s8 /
- * gemm_s4*, whose 32-bit results can be summed in place).  For ablation sweeps
- * in the spirit of the paper's Run 4.  Returns GEMM_ERR_INVALID_ARG for a shape
- * that is not built.
- */
-int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k);
-
-/*
- * Kernels never spin forever: a barrier wait that exceeds its limit makes the
- * kernel record a non-zero code and drain.  This reads that code for the
- * current device (synchronises the device) and clears it.  0 = no event;
- * 1/2/3 = producer / MMA / epilogue wait expired, 5 = a wait of the INT4
- * expansion warps expired.
+ * Kernels never spin forever: a barrier wait that exceeds its limit (2 s) makes
+ * the kernel record a non-zero code in a status word on the device, drain and
+ * return, leaving garbage in C -- the host call has long returned GEMM_OK by
+ * then.  A caller that must be sure of C therefore reads the word after the
+ * work: gemm_last_device_status reads it for the current device and clears it
+ * (it synchronises the device); gemm_read_device_status enqueues a copy of the
+ * word to `host_out` (host memory, page-locked for a truly asynchronous copy) on
+ * `stream`, in stream order behind the GEMMs enqueued there, without clearing.
+ * 0 = no event; 1/2/3 = producer / MMA / epilogue wait expired, 5 = a wait of the
+ * INT4 expansion warps expired.
  */
 int gemm_last_device_status(void);
-
-/*
- * Route of later gemm_s4 / gemm_s4_dequant calls.  tcgen05 has no signed 4-bit
- * integer kind (the paper's kernels feed mma.sync m16n8k64 .s4 operands
- * directly, Listing 2c), so the nibbles are expanded to int8 either
- *   - by a streaming pre-pass kernel into an int8 scratch, followed by the
- *     INT8 GEMM ("pre-pass"): each operand element is expanded once; or
- *   - inside the GEMM kernel ("fused"): packed tiles are loaded as they are and
- *     eight extra warps per CTA expand them in shared memory into the slots the
- *     MMAs read.  No scratch, and a quarter of the pre-pass route's HBM bytes
- *     for an operand that is read once; but half as much shared-memory traffic
- *     again per unit of math, which is what bounds the large-tile kernel.
- * Measured: at M = N = K = 8192 the pre-pass route is 1.1-1.35x faster; for
- * M = 16, N = K = 8192 (bound by the bytes of B) the fused route takes 15 us
- * instead of 33.
- * Small problems, bound by launches and latencies, save one launch with the
- * fused route (10-26 % up to 1024 x 1024 outputs).
- * scheme 0 (default, automatic): fused where the selector picks a one-CTA tile
- * and M <= 128 or N <= 128 or both <= 1024, or a single wave of CTA-pair tiles
- * (e.g. 2048^3); also for problems with a short side, where the pre-pass (cost:
- * the bytes of both operands) is dear next to the GEMM: M N / (M + N) <= 384
- * with the best tile the fused kernel has, and up to 1024 rows or columns with
- * its CTA-pair tile if the tiles fill their waves to 75 % (256 x 28672 x 8192:
- * 119 -> 67 us; 512 x 16384 x 4096: 44 -> 35 us); else the pre-pass.  1: always
- * the pre-pass; 2: fused wherever a fused variant is built (every one-CTA tile,
- * and the 256 x 256 and 256 x 128 CTA pairs), else the pre-pass.  gemm_s4_ws and gemm_s4_static
- * always use the pre-pass.  Results are identical, bit for bit.
- * gemm_query_config shows the route.  The paper has no counterpart; its Run 4
- * ablates how the operands reach the tensor cores, of which this is the
- * analogue here.
- */
-int gemm_set_s4_scheme(int scheme);
-
-/*
- * Whether later calls run the kernel on exchanged operands: its 128-row tile
- * side then holds rows of B (the caller's N), its narrow side rows of A, and C
- * is written by plain stores that are contiguous along N.  For problems with
- * few rows (M = 1..64, LLM decoding) this keeps 128 - M rows of zero fill out
- * of shared memory, of the ring depth and -- on the fused INT4 route -- of the
- * expansion work.  mode 0 (default, automatic): when N >= 1024 and M <= 32
- * (gemm_fp16) or M <= 64 (INT8, INT4, gemm_fp16_f16out, and gemm_fp16 from
- * N = 16384 on) (measured 2-12 % faster there); 1: never; 2: always
- * (any shape, precision and INT4 route; for tests and measurements).  Results:
- * integers identical; FP16 within the bound; dequantised outputs multiply the
- * two scales in the other order (last-bit differences).  gemm_query_config
- * shows "swap_ab" and then describes the tile in the kernel's orientation.  The
- * paper has no counterpart (square sizes only, Sec. VI).
- */
-int gemm_set_swap_ab(int mode);
-
-/*
- * L2 behaviour of later calls, a bit set (the paper's Run 4 ablates the
- * analogous .ca / .cg cache policy of cp.async).  Bits 0-1, eviction priority
- * of the operand loads: 0 = normal for A and B; 1 = A "evict last" (kept), B
- * "evict first" (streamed); 2 = both "evict last"; 3 = A "evict last", B
- * normal.  Bit 2 (4): turn OFF the serpentine K order (by default successive
- * tiles of a CTA walk K forward, backward, forward, ... so that a tile begins
- * on the K range its predecessor, which shares its A rows, read last and still
- * finds in L2).  Bit 3 (8): mark the C stores "evict first" (written once,
- * never re-read).  Bit 4 (16): fetch operands with 128-byte instead of 256-byte
- * L2 promotion.  Bit 5 (32): launch in plain stream order.  By default a GEMM
- * of this library is launched so that it may begin while the kernel in front of
- * it in the stream is still running (programmatic dependent launch): its set-up
- * (barriers, tensor memory, descriptor prefetch) and the launch latency overlap
- * that kernel's tail, and it waits for that kernel to complete before its first
- * load and its first store; a GEMM of this library lets its successor begin as
- * soon as it runs itself.  Stream semantics are unchanged; back-to-back small
- * GEMMs get 15-25 % faster (N = 512: 5.1 -> 4.0 us).  Default 11 = 3 + 8 with
- * the serpentine order on, which gave the lowest DRAM traffic at N = 8192; with
- * the default, problems that are one tile wide or one tile tall (few rows on one
- * side) use 2 for bits 0-1, so that the short operand every CTA re-reads is not
- * pushed out of L2 by the long one streaming past.  Bit 6 (64): no split-K
- * inside a cluster (see gemm_fp16_f16out / the dequantising entry points).
- * Integer results never depend on any of this; FP16 results may differ in the last bits (summation order) within the
- * bound.
- */
-int gemm_set_l2_policy(int policy);
-
-/*
- * Cycle accounting, in the spirit of the counter attribution the paper does
- * with its profiler (Sec. III-B).  gemm_trace_enable(1) makes later GEMM
- * launches record, per CTA, 16 unsigned 64-bit words: [0] SM cycles and [1]
- * nanoseconds the CTA ran (their ratio is the SM clock during the kernel),
- * cycles the producer waited for a free slot [2], the MMA issuer waited for
- * operands [3] and for a free accumulator [4], one epilogue warp waited for a
- * finished accumulator [5] and spent draining [6], the tile count [7], and the
- * issuer's cycles inside tcgen05.mma [8] and tcgen05.commit [9], the cycles
- * the CTA spent setting up barriers and tensor memory [10], and the producer's
- * cycles issuing loads [11]; fused INT4 only, one expansion warp: cycles
- * waiting for packed operands [12], for a free int8 slot [13] and spent
- * expanding [14]; [15] is unused.
- * Switching recording on (bit 1 from 0 to 1) synchronises the device and clears
- * all records.  Traced launches run in plain stream order (no early start, see
- * gemm_set_l2_policy bit 5), so that the cycle counts are the kernel's own.
- * gemm_trace_read synchronises the device, copies the words of the first
- * min(max_ctas, 160) CTAs of the last traced launch to `out` (host memory,
- * 16 * max_ctas words) and returns that CTA count.  Off by default; the cost
- * when on is a few clock reads per k-block.
- * `on` is a bit set: 1 = record; 2 = ablation, issue no MMAs (operand loads and
- * barriers only); 4 = ablation, issue no operand loads (MMAs and barriers only,
- * on whatever shared memory holds); 8 = the epilogue's waits back off with
- * nanosleep instead of polling; 16 = failure drill: one operand slot of the
- * first tile is never filled, so the kernel's bounded waits (2 s) must expire,
- * record a code for gemm_last_device_status, drain and return -- the call takes
- * a few seconds, C is garbage and the context stays usable; 32 = the epilogue
- * writes C straight from registers (16 bytes per thread and store) instead of
- * staging it in shared memory for TMA stores (results unchanged).  With bit 2, 4 or
- * 16 set C is garbage; 2 and 4 exist to attribute cycles to the load path or
- * the MMA path.
- */
-int gemm_trace_enable(int on);
-int gemm_trace_read(unsigned long long* out, int max_ctas);
+int gemm_read_device_status(int* host_out, gemm_stream_t stream);
 
 /* cudaError_t value of the last failed CUDA call made by this library, or 0. */
 int gemm_last_cuda_error(void);

@@ -23,7 +23,8 @@ EXPORTS = (
     "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
     "gemm_fp16_f16out", "gemm_s8_dequant", "gemm_s4_dequant", "gemm_host", "gemm_host_release",
     "gemm_s4_static", "gemm_s4_static_capacity", "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
-    "gemm_set_config_override", "gemm_set_s4_scheme", "gemm_set_swap_ab", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_last_device_status", "gemm_last_cuda_error",
+    "gemm_set_config_override", "gemm_set_kernel_family", "gemm_set_s4_scheme", "gemm_set_swap_ab", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_set_stages_override", "gemm_debug_counters",
+    "gemm_last_device_status", "gemm_read_device_status", "gemm_last_cuda_error",
     "gemm_status_string", "gemm_version",
 )
 
@@ -72,6 +73,10 @@ def lib() -> ctypes.CDLL:
         L.gemm_query_config.argtypes = [i, i, i, i, ctypes.c_char_p, i]
         L.gemm_set_config_override.argtypes = [i, i, i, i]
         L.gemm_set_s4_scheme.argtypes = [i]
+        L.gemm_set_kernel_family.argtypes = [i]
+        L.gemm_set_stages_override.argtypes = [i]
+        L.gemm_debug_counters.argtypes = [ctypes.POINTER(ctypes.c_longlong), i]
+        L.gemm_read_device_status.argtypes = [vp, vp]
         L.gemm_set_swap_ab.argtypes = [i]
         L.gemm_set_l2_policy.argtypes = [i]
         L.gemm_trace_enable.argtypes = [i]
@@ -302,6 +307,33 @@ def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0, 
            "gemm_set_config_override")
 
 
+def gemm_set_kernel_family(family: int = 0):
+    """Kernel for large problems: 0 = automatic, 1 = 256 x 256 tile per CTA pair, 2 = 512 x 256."""
+    _check(lib().gemm_set_kernel_family(int(family)), "gemm_set_kernel_family")
+
+
+def gemm_set_stages_override(stages: int = 0):
+    """Ring depth of the 256 x 256 CTA-pair kernel (raw outputs): 0 = shipped (6), or 3..6."""
+    _check(lib().gemm_set_stages_override(int(stages)), "gemm_set_stages_override")
+
+
+def gemm_debug_counters() -> dict:
+    """Host-side counters: tensor maps encoded so far, scratch buffers pooled on the current
+    device, whether this thread's last INT4 call ran the overlapped pre-pass."""
+    buf = (ctypes.c_longlong * 3)()
+    _check(lib().gemm_debug_counters(buf, 3), "gemm_debug_counters")
+    return {"map_encodes": int(buf[0]), "pool_buffers": int(buf[1]), "s4_overlapped": int(buf[2])}
+
+
+def gemm_read_device_status(host_out: torch.Tensor, stream=None):
+    """Enqueues a copy of the device status word into `host_out` (a pinned int32 CPU tensor of
+    one element) on `stream`; the value is there once the stream has passed the copy."""
+    if host_out.is_cuda or host_out.dtype != torch.int32 or host_out.numel() < 1:
+        raise TypeError("host_out must be an int32 CPU tensor")
+    _check(lib().gemm_read_device_status(host_out.data_ptr(), _stream_handle(stream)),
+           "gemm_read_device_status")
+
+
 def gemm_set_s4_scheme(scheme: int = 0):
     """Route of gemm_s4 / gemm_s4_dequant: 0 = automatic (nibbles expanded inside the GEMM
     kernel for problems with few rows on one side, else a pre-pass to int8 + the INT8 GEMM);
@@ -324,7 +356,7 @@ def gemm_set_l2_policy(policy: int = 11):
 
 TRACE_FIELDS = ("cycles", "nanos", "producer_wait", "mma_wait_operands", "mma_wait_accumulator",
                 "epilogue_wait", "epilogue_busy", "tiles", "mma_issue", "mma_commit", "setup",
-                "producer_issue", "unpack_wait_packed", "unpack_wait_slot", "unpack_busy", "unused15")
+                "producer_issue", "unpack_wait_packed", "unpack_wait_slot", "unpack_busy", "mma_wait_accumulator1")
 TRACE_SLOTS = len(TRACE_FIELDS)
 
 

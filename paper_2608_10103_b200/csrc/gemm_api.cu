@@ -97,18 +97,19 @@ int gemm_s4_dequant(int M, int N, int K, const uint8_t* A, const uint8_t* B,
 }
 
 int gemm_release_workspaces(void) {
-  std::lock_guard<std::mutex> lock(g_mutex);
   int cur = 0;
   if (cudaGetDevice(&cur) != cudaSuccess) cur = -1;
   int rc = GEMM_OK;
   for (int d = 0; d < MAX_DEVICES; ++d) {
-    if (!g_dev[d].s4_workspace) continue;
+    if (g_pool[d].buffers() == 0) continue;
     cudaError_t e = cudaSetDevice(d);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
-    if (e == cudaSuccess) e = cudaFree(g_dev[d].s4_workspace);
-    if (e != cudaSuccess) rc = cuda_fail(e);
-    g_dev[d].s4_workspace = nullptr;
-    g_dev[d].s4_workspace_bytes = 0;
+    if (e != cudaSuccess) {
+      rc = cuda_fail(e);
+      continue;
+    }
+    const int r = g_pool[d].release_all();
+    if (r != 0) rc = cuda_fail(static_cast<cudaError_t>(r));
   }
   if (cur >= 0) cudaSetDevice(cur);
   return rc;
@@ -129,7 +130,6 @@ int gemm_mma_peak_probe(int precision, int iters, int n_cols, int commit_every, 
   if (iters <= 0 || !ops_out || (precision != GEMM_PREC_FP16 && precision != GEMM_PREC_S8) ||
       n_cols < 16 || n_cols > PROBE_BN || n_cols % 16 || commit_every < 0)
     return GEMM_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(g_mutex);
   DeviceState* s = nullptr;
   int rc = device_state(&s);
   if (rc != GEMM_OK) return rc;
@@ -160,13 +160,7 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
   if (!buf || len <= 0 || M <= 0 || N <= 0 || K <= 0 || precision < GEMM_PREC_FP16 ||
       precision > GEMM_PREC_S4)
     return GEMM_ERR_INVALID_ARG;
-  int num_sms = 148;
-  {
-    std::lock_guard<std::mutex> lock(g_mutex);
-    int dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < MAX_DEVICES && g_dev[dev].ready)
-      num_sms = g_dev[dev].num_sms;
-  }
+  const int num_sms = known_sm_count();
   const int elem = precision == GEMM_PREC_FP16 ? 2 : 1;
   const int kb = ceil_div(static_cast<long long>(K) * elem, BK_BYTES);
   TileConfig c;
@@ -188,13 +182,24 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
     M = user_n;
     N = user_m;
   }
+  const bool wide = wide_wanted(c, M, N, num_sms, swap, false, fused);
+  if (wide) {
+    c.bn = WIDE_BN;
+    c.cta_group = 2;
+    c.splits = 1;
+    c.split_tiles = 0;
+    c.stages = WIDE_STAGES;
+    c.group_m = band_height(M, WIDE_TILE_M, WIDE_BN, num_sms / 2);
+  }
+  const int rows_per_cta = wide ? WIDE_CTA_ROWS : BM;
   const long long tiles =
-      static_cast<long long>(ceil_div(M, BM * c.cta_group)) * ceil_div(N, c.bn);
+      static_cast<long long>(ceil_div(M, rows_per_cta * c.cta_group)) * ceil_div(N, c.bn);
   const long long units = num_sms / c.cta_group;
   snprintf(buf, static_cast<size_t>(len),
            "BM=%d BN=%d BK=%d cta_group=%d stages=%d group_m=%d split_k=%d split_tiles=%d "
            "tiles=%lld ctas=%lld kind=%s%s%s%s",
-           BM * c.cta_group, c.bn, atoms_for(c.bn, c.cta_group) * BK_BYTES / elem, c.cta_group,
+           rows_per_cta * c.cta_group, c.bn,
+           (wide ? 1 : atoms_for(c.bn, c.cta_group)) * BK_BYTES / elem, c.cta_group,
            c.stages, c.group_m, c.splits, c.splits > 1 ? c.split_tiles : 0, tiles,
            (tiles + (c.splits > 1 ? static_cast<long long>(c.split_tiles) * (c.splits - 1) : 0) <
                     units
@@ -220,7 +225,6 @@ int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k) {
     }
   }
   if (!ok) return GEMM_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(g_mutex);
   g_override_bn = bn;
   g_override_group_m = group_m;
   g_override_cta_group = cta_group;
@@ -229,7 +233,6 @@ int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k) {
 }
 
 int gemm_last_device_status(void) {
-  std::lock_guard<std::mutex> lock(g_mutex);
   DeviceState* s = nullptr;
   int rc = device_state(&s);
   if (rc != GEMM_OK) return rc;
@@ -245,29 +248,58 @@ int gemm_last_device_status(void) {
   return v;
 }
 
+int gemm_set_kernel_family(int family) {
+  if (family < 0 || family > 2) return GEMM_ERR_INVALID_ARG;
+  g_family = family;
+  return GEMM_OK;
+}
+
 int gemm_set_s4_scheme(int scheme) {
   if (scheme < 0 || scheme > 2) return GEMM_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(g_mutex);
   g_s4_scheme = scheme;
   return GEMM_OK;
 }
 
 int gemm_set_swap_ab(int mode) {
   if (mode < 0 || mode > 2) return GEMM_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(g_mutex);
   g_swap_ab = mode;
   return GEMM_OK;
 }
 
 int gemm_set_l2_policy(int policy) {
   if (policy < 0 || policy > 127) return GEMM_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(g_mutex);
   g_l2_policy = policy;
   return GEMM_OK;
 }
 
+int gemm_set_stages_override(int stages) {
+  if (stages != 0 && (stages < 3 || stages > 6)) return GEMM_ERR_INVALID_ARG;
+  g_override_stages = stages;
+  return GEMM_OK;
+}
+
+int gemm_debug_counters(long long* out, int n) {
+  if (!out || n <= 0) return GEMM_ERR_INVALID_ARG;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) dev = 0;
+  const long long v[3] = {g_map_encodes.load(), static_cast<long long>(g_pool[dev].buffers()),
+                          t_last_s4_overlapped};
+  for (int i = 0; i < n; ++i) out[i] = i < 3 ? v[i] : 0;
+  return GEMM_OK;
+}
+
+int gemm_read_device_status(int* host_out, gemm_stream_t stream) {
+  if (!host_out) return GEMM_ERR_INVALID_ARG;
+  DeviceState* s = nullptr;
+  int rc = device_state(&s);
+  if (rc != GEMM_OK) return rc;
+  cudaError_t e = cudaMemcpyAsync(host_out, s->status_ptr, sizeof(int), cudaMemcpyDeviceToHost,
+                                  reinterpret_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e);
+  return GEMM_OK;
+}
+
 int gemm_trace_enable(int on) {
-  std::lock_guard<std::mutex> lock(g_mutex);
   if ((on & 1) && !(g_trace_on & 1)) {
     // recording starts: clear the records, so that CTAs a later launch does not have read 0
     DeviceState* s = nullptr;
@@ -285,7 +317,6 @@ int gemm_trace_enable(int on) {
 int gemm_trace_read(unsigned long long* out, int max_ctas) {
   static_assert(TRACE_SLOTS == 16, "header documents 16 words per CTA");
   if (!out || max_ctas <= 0) return GEMM_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(g_mutex);
   DeviceState* s = nullptr;
   int rc = device_state(&s);
   if (rc != GEMM_OK) return rc;
@@ -298,7 +329,7 @@ int gemm_trace_read(unsigned long long* out, int max_ctas) {
   return n;
 }
 
-int gemm_last_cuda_error(void) { return g_last_cuda_error; }
+int gemm_last_cuda_error(void) { return g_last_cuda_error.load(); }
 
 const char* gemm_status_string(int status) {
   switch (status) {
@@ -314,7 +345,7 @@ const char* gemm_status_string(int status) {
   }
 }
 
-int gemm_version(void) { return 1000; }
+int gemm_version(void) { return 2000; }
 
 }  // extern "C"
 

@@ -144,6 +144,7 @@ enum TraceSlot {
   TRACE_UNPACK_WAIT_IN = 12,   // fused INT4, unpack warp 6: cycles waiting for packed operands
   TRACE_UNPACK_WAIT_OUT = 13,  // ... waiting for a free int8 slot
   TRACE_UNPACK_BUSY = 14,      // ... expanding nibbles
+  TRACE_MMA_WAIT_ACC1 = 15,    // wide kernel: MMA issuer waiting for the tile's second accumulator
   TRACE_SLOTS = 16
 };
 
@@ -234,13 +235,16 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+// DBG: the measurement and drill switches of GemmParams::ablate are compiled in (the product
+// instantiations leave them out of their loops).
 template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32, int PSTAGES = 0,
-          int CSPLIT = 1>
+          int CSPLIT = 1, bool DBG = false>
 __global__ void __launch_bounds__(PSTAGES > 0 ? NUM_THREADS_FUSED : NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
   using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, CSPLIT>;
   constexpr bool FUSED = PSTAGES > 0;  // packed INT4 operands, expanded on the way to the MMAs
+  const int ablate = DBG ? p.ablate : 0;
   // fused INT4: the expansion warps work as one group of eight, or -- where both rings are at
   // least four slots deep -- as two groups of four on alternate packed slots
   constexpr int UNPACK_GROUPS = (STAGES >= 4 && PSTAGES >= 4) ? 2 : 1;
@@ -416,9 +420,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const uint32_t b_dst = a_dst + L::A_BYTES;
           if (!elected) {
             // nothing to issue in this lane
-          } else if ((p.ablate & 8) && blockIdx.x == 0 && t == first_tile && ps == ps_begin + 2) {
+          } else if ((ablate & 8) && blockIdx.x == 0 && t == first_tile && ps == ps_begin + 2) {
             // failure drill: this slot is never filled
-          } else if (p.ablate & 2) {
+          } else if (ablate & 2) {
             ptx::mbar_arrive(p_full_bar(stage));
           } else {
             const int k0 = (backward ? ps_begin + ps_end - 1 - ps : ps) * BK_BYTES;  // packed bytes
@@ -450,9 +454,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const uint32_t b_dst = a_dst + KB * L::A_BYTES;
           if (!elected) {
             // nothing to issue in this lane
-          } else if ((p.ablate & 8) && blockIdx.x == 0 && t == first_tile && ks == k_begin + 2) {
+          } else if ((ablate & 8) && blockIdx.x == 0 && t == first_tile && ks == k_begin + 2) {
             // failure drill: this slot is never filled
-          } else if (p.ablate & 2) {
+          } else if (ablate & 2) {
             if (leader) ptx::mbar_arrive(full_bar(stage));
           } else if constexpr (CTA_GROUP == 1) {
             ptx::mbar_arrive_expect_tx(full_bar(stage), L::STAGE_BYTES);
@@ -534,7 +538,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const uint32_t a_src = base + stage * L::STAGE_BYTES;
           const uint64_t a_desc = ptx::smem_desc_sw128(a_src);
           const uint64_t b_desc = ptx::smem_desc_sw128(a_src + KB * L::A_BYTES);
-          if (elected && !(p.ablate & 1)) {
+          if (elected && !(ablate & 1)) {
 #pragma unroll
             for (int a = 0; a < KB; ++a) {
 #pragma unroll
@@ -791,7 +795,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       }
       const long long w0 = trace ? clock64() : 0;
       ok = wait_bounded<true>(acc_full_bar(acc), acc_phase, abort_flag, p.status,
-                              DEV_TIMEOUT_EPILOGUE, (p.ablate & 4) ? 500u : 0u);
+                              DEV_TIMEOUT_EPILOGUE, (ablate & 4) ? 500u : 0u);
       ok = __all_sync(0xffffffffu, ok);
       const long long w1 = trace ? clock64() : 0;
       epi_wait += w1 - w0;
@@ -901,7 +905,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             }
           }
         }
-        if (EPI == EPI_RAW32 && (p.ablate & 16) && p.c_vec_ok && !add) {
+        if (EPI == EPI_RAW32 && (ablate & 16) && p.c_vec_ok && !add) {
           // ablation: straight from registers, 8 x 16 bytes per thread into its own C row
           if (row < p.M) {
             uint32_t* crow = p.C + static_cast<size_t>(row) * p.ldc;

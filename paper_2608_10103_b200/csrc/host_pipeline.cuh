@@ -15,18 +15,24 @@ struct HostPipe {
   size_t cap[4] = {0, 0, 0, 0};
   cudaEvent_t ev[3 + 2 * 64 + 64 * 64] = {};
   int num_ev = 0;
+  bool used_before = false;  // ev[1] marks the end of the previous call
 };
 HostPipe g_pipe[MAX_DEVICES];
 std::mutex g_pipe_mutex;
 
-int pipe_grow(HostPipe& p, int which, size_t need) {
+// Grows buffer `which`, stream-ordered on `st` (no device-wide synchronisation).  `st` has been
+// made to wait for the previous call through this pipe, so nothing uses the old buffer any more
+// once `st` gets here.
+int pipe_grow(HostPipe& p, int which, size_t need, cudaStream_t st) {
   if (p.cap[which] >= need) return GEMM_OK;
-  cudaError_t e = cudaDeviceSynchronize();  // earlier calls may still use the old buffer
-  if (e != cudaSuccess) return cuda_fail(e);
-  if (p.buf[which]) cudaFree(p.buf[which]);
+  cudaError_t e;
+  if (p.buf[which]) {
+    e = cudaFreeAsync(p.buf[which], st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
   p.buf[which] = nullptr;
   p.cap[which] = 0;
-  e = cudaMalloc(&p.buf[which], need);
+  e = cudaMallocAsync(&p.buf[which], need, st);
   if (e != cudaSuccess) return cuda_fail(e);
   p.cap[which] = need;
   return GEMM_OK;
@@ -73,24 +79,26 @@ int gemm_host(int precision, int M, int N, int K, const void* A, const void* B, 
   GEMM_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= MAX_DEVICES) return GEMM_ERR_UNSUPPORTED_DEVICE;
   {
-    std::lock_guard<std::mutex> lock(g_mutex);
     DeviceState* s = nullptr;
     int rc = device_state(&s);
     if (rc != GEMM_OK) return rc;
   }
   std::lock_guard<std::mutex> lock(g_pipe_mutex);
   HostPipe& p = g_pipe[dev];
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (!p.h2d) GEMM_CUDA_TRY(cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking));
   if (!p.d2h) GEMM_CUDA_TRY(cudaStreamCreateWithFlags(&p.d2h, cudaStreamNonBlocking));
-  int rc = pipe_grow(p, 0, align_up(static_cast<size_t>(M) * row_bytes, 256));
-  if (rc == GEMM_OK) rc = pipe_grow(p, 1, align_up(static_cast<size_t>(N) * row_bytes, 256));
-  if (rc == GEMM_OK) rc = pipe_grow(p, 2, align_up(static_cast<size_t>(M) * N * 4, 256));
+  // The previous call through this pipe (possibly on another stream) must have finished with
+  // the device buffers before this one refills -- or frees -- them.
+  if (p.used_before) GEMM_CUDA_TRY(cudaStreamWaitEvent(st, p.ev[1], 0));
+  int rc = pipe_grow(p, 0, align_up(static_cast<size_t>(M) * row_bytes, 256), st);
+  if (rc == GEMM_OK) rc = pipe_grow(p, 1, align_up(static_cast<size_t>(N) * row_bytes, 256), st);
+  if (rc == GEMM_OK) rc = pipe_grow(p, 2, align_up(static_cast<size_t>(M) * N * 4, 256), st);
   if (rc == GEMM_OK && precision == GEMM_PREC_S4)
     rc = pipe_grow(p, 3, align_up(static_cast<size_t>(M) * K, 256) +
-                             align_up(static_cast<size_t>(N) * K, 256));
+                             align_up(static_cast<size_t>(N) * K, 256), st);
   if (rc != GEMM_OK) return rc;
 
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const uint8_t* hA = static_cast<const uint8_t*>(A);
   const uint8_t* hB = static_cast<const uint8_t*>(B);
   uint8_t* dA = static_cast<uint8_t*>(p.buf[0]);
@@ -174,6 +182,7 @@ int gemm_host(int precision, int M, int N, int K, const void* A, const void* B, 
   }
   GEMM_CUDA_TRY(cudaEventRecord(ev_done, p.d2h));
   GEMM_CUDA_TRY(cudaStreamWaitEvent(st, ev_done, 0));
+  p.used_before = true;
   return GEMM_OK;
 }
 
@@ -195,6 +204,7 @@ int gemm_host_release(void) {
     }
     for (int k = 0; k < p.num_ev; ++k) cudaEventDestroy(p.ev[k]);
     p.num_ev = 0;
+    p.used_before = false;
     if (p.h2d) cudaStreamDestroy(p.h2d);
     if (p.d2h) cudaStreamDestroy(p.d2h);
     p.h2d = p.d2h = nullptr;

@@ -4,6 +4,7 @@
 
 #include <utility>
 
+#include "gemm_wide.cuh"
 #include "runtime.cuh"
 #include "selector.cuh"
 #include "unpack_s4.cuh"
@@ -25,31 +26,45 @@ __global__ void zero_c_kernel(uint4* c16, size_t n16, uint32_t* tail, int tail_w
   if (blockIdx.x == 0 && static_cast<int>(threadIdx.x) < tail_words) tail[threadIdx.x] = 0;
 }
 
-template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI, int PSTAGES = 0,
-          int CSPLIT = 1>
-int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUtensorMap& tb,
-                   const CUtensorMap& tc, const GemmParams& p, cudaStream_t stream) {
-  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, CSPLIT>;
-  auto kernel = gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI, PSTAGES, CSPLIT>;
-  if (!(s->attr_set[variant >> 6] & (1ull << (variant & 63)))) {
+// Kernel variants that also exist with the measurement / drill switches compiled in, and the
+// attr_set bit of that twin (208..): the two 256-wide tiles of the raw outputs, two of the
+// fused INT4 kernels and the 4-way cluster split-K kernel -- the ones the ablation runs and
+// the failure drills use.
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI, int PSTAGES, int CSPLIT>
+constexpr int dbg_twin_bit() {
+  if (EPI == EPI_RAW32 && CSPLIT == 1 && PSTAGES == 0 && BN == 256 &&
+      ((CTA_GROUP == 1 && STAGES == 4) || (CTA_GROUP == 2 && STAGES == 6)))
+    return 208 + (KIND == ptx::KIND_F16 ? 0 : 2) + (CTA_GROUP - 1);
+  if (KIND == ptx::KIND_I8 && EPI == EPI_RAW32 && CSPLIT == 1 && PSTAGES > 0 && BN == 256 &&
+      CTA_GROUP == 2)
+    return 212;
+  if (KIND == ptx::KIND_I8 && EPI == EPI_RAW32 && CSPLIT == 1 && PSTAGES > 0 && BN == 32) return 213;
+  if (KIND == ptx::KIND_I8 && EPI == EPI_OUT16 && CSPLIT == 4 && PSTAGES == 0) return 214;
+  return -1;
+}
+
+template <class Kernel>
+int launch_kernel(DeviceState* s, Kernel kernel, int variant, int dyn_bytes, int threads,
+                  int cluster, const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc,
+                  const GemmParams& p, cudaStream_t stream) {
+  if (!(s->attr_set[variant >> 6].load(std::memory_order_relaxed) & (1ull << (variant & 63)))) {
     cudaError_t e =
-        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES);
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_bytes);
     if (e != cudaSuccess) return cuda_fail(e);
-    s->attr_set[variant >> 6] |= 1ull << (variant & 63);
+    s->attr_set[variant >> 6].fetch_or(1ull << (variant & 63), std::memory_order_relaxed);
   }
   const long long all_tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   const long long tiles = p.split_from + (all_tiles - p.split_from) * p.splits;  // work units
-  constexpr int CLUSTER = CTA_GROUP * CSPLIT;  // CTAs that work on one unit together
-  const long long units = s->num_sms / CLUSTER;
-  const int grid = static_cast<int>((tiles < units ? tiles : units) * CLUSTER);
+  const long long units = s->num_sms / cluster;
+  const int grid = static_cast<int>((tiles < units ? tiles : units) * cluster);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid, 1, 1);
-  cfg.blockDim = dim3(PSTAGES > 0 ? NUM_THREADS_FUSED : NUM_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = L::DYN_BYTES;
+  cfg.blockDim = dim3(threads, 1, 1);
+  cfg.dynamicSmemBytes = dyn_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = CLUSTER;
+  attr[0].val.clusterDim.x = cluster;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -59,6 +74,94 @@ int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUt
   cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, tc, p);
   if (e != cudaSuccess) return cuda_fail(e);
   return GEMM_OK;
+}
+
+template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI, int PSTAGES = 0,
+          int CSPLIT = 1>
+int launch_variant(DeviceState* s, int variant, const CUtensorMap& ta, const CUtensorMap& tb,
+                   const CUtensorMap& tc, const GemmParams& p, cudaStream_t stream) {
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, CSPLIT>;
+  constexpr int THREADS = PSTAGES > 0 ? NUM_THREADS_FUSED : NUM_THREADS;
+  constexpr int CLUSTER = CTA_GROUP * CSPLIT;  // CTAs that work on one unit together
+  if (p.ablate) {
+    constexpr int twin = dbg_twin_bit<KIND, BN, STAGES, CTA_GROUP, KB, EPI, PSTAGES, CSPLIT>();
+    if constexpr (twin >= 0) {
+      return launch_kernel(s, gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI, PSTAGES, CSPLIT, true>,
+                           twin, L::DYN_BYTES, THREADS, CLUSTER, ta, tb, tc, p, stream);
+    } else {
+      return GEMM_ERR_INVALID_ARG;  // this variant is not built with the switches
+    }
+  }
+  return launch_kernel(s, gemm_kernel<KIND, BN, STAGES, CTA_GROUP, KB, EPI, PSTAGES, CSPLIT>,
+                       variant, L::DYN_BYTES, THREADS, CLUSTER, ta, tb, tc, p, stream);
+}
+
+// The 512 x 256 CTA-pair kernel for large problems (gemm_wide.cuh).  attr_set bits 160..
+template <int KIND, int EPI>
+int launch_wide(DeviceState* s, const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p,
+                cudaStream_t stream) {
+  const bool dbg = p.ablate != 0;
+  if (dbg && EPI != EPI_RAW32) return GEMM_ERR_INVALID_ARG;  // switches exist for the raw outputs
+  const int variant = 160 + ((KIND == ptx::KIND_F16) ? 0 : 8) + EPI * 2 + (dbg ? 1 : 0);
+  void (*kernel)(CUtensorMap, CUtensorMap, GemmParams) = gemm_wide_kernel<KIND, EPI, false>;
+  if constexpr (EPI == EPI_RAW32) {
+    if (dbg) kernel = gemm_wide_kernel<KIND, EPI, true>;
+  }
+  if (!(s->attr_set[variant >> 6].load(std::memory_order_relaxed) & (1ull << (variant & 63)))) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         WideSmem::DYN_BYTES);
+    if (e != cudaSuccess) return cuda_fail(e);
+    s->attr_set[variant >> 6].fetch_or(1ull << (variant & 63), std::memory_order_relaxed);
+  }
+  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
+  const long long pairs = s->num_sms / 2;
+  const int grid = static_cast<int>((tiles < pairs ? tiles : pairs) * 2);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(WIDE_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = WideSmem::DYN_BYTES;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.wait_prior_grid ? 2 : 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, p);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return GEMM_OK;
+}
+
+// Band height (in tiles) of the raster for a tile of `rows_per_tile` x `bn`: one wave of tiles
+// about twice as tall as wide in operand bytes, then evened out over the bands so that no
+// short last band streams the other operand for little work.
+int band_height(int M, int rows_per_tile, int bn, int units) {
+  int g = 1;
+  while ((g + 1) * (g + 1) * rows_per_tile <= 2 * units * bn) ++g;
+  if (g_override_group_m) g = g_override_group_m;
+  const int tiles_m = ceil_div(M, rows_per_tile);
+  if (g > tiles_m) g = tiles_m;
+  if (g < 1) g = 1;
+  if (!g_override_group_m) g = ceil_div(tiles_m, ceil_div(tiles_m, g));
+  return g;
+}
+
+// Whether a problem goes to the 512 x 256 kernel.  It needs the same number of SM cycles as the
+// 256 x 256 pair tile but a quarter fewer operand bytes from L2, which buys clock on a
+// power-capped part; its tiles are twice as large, so it needs enough of them to fill its waves.
+bool wide_wanted(const TileConfig& cfg, int M, int N, int num_sms, bool swap, bool csplit,
+                 bool packed_s4) {
+  if (swap || csplit || packed_s4 || g_family == 1) return false;
+  if (g_family == 2) return !(g_override_bn && g_override_bn != 256) && g_override_cta_group != 1 &&
+                            g_override_splits <= 1;
+  if (cfg.bn != 256 || cfg.cta_group != 2 || cfg.splits != 1) return false;
+  const long long tiles = static_cast<long long>(ceil_div(M, WIDE_TILE_M)) * ceil_div(N, WIDE_BN);
+  const long long pairs = num_sms / 2;
+  const long long waves = (tiles + pairs - 1) / pairs;
+  return tiles >= 2 * pairs && 10 * tiles >= 9 * waves * pairs;  // waves at least 90 % full
 }
 
 // Output options of one GEMM call.
@@ -81,14 +184,14 @@ constexpr int csplit_variant_base() {
 // not a multiple of four: a tile more than that would wait for a second wave.)
 template <int KIND, int EPI>
 int quad_clusters_resident(DeviceState* s, int variant) {
-  int& cached = s->quad_clusters[KIND == ptx::KIND_F16 ? 0 : 1][EPI];
-  if (cached) return cached;
+  std::atomic<int>& cached = s->quad_clusters[KIND == ptx::KIND_F16 ? 0 : 1][EPI];
+  if (cached.load()) return cached.load();
   using L = SmemLayout<32, 3, 1, 2, 0, 4>;
   auto kernel = gemm_kernel<KIND, 32, 3, 1, 2, EPI, 0, 4>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) !=
       cudaSuccess)
     return 0;
-  s->attr_set[variant >> 6] |= 1ull << (variant & 63);
+  s->attr_set[variant >> 6].fetch_or(1ull << (variant & 63), std::memory_order_relaxed);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(s->num_sms / 4 * 4), 1, 1);
   cfg.blockDim = dim3(NUM_THREADS, 1, 1);
@@ -105,7 +208,7 @@ int quad_clusters_resident(DeviceState* s, int variant) {
     (void)cudaGetLastError();
     n = s->num_sms / 8;  // unknown: assume half
   }
-  cached = n;
+  cached.store(n);
   return n;
 }
 
@@ -211,7 +314,6 @@ template <int KIND, int EPI>
 int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const void* B,
                     size_t b_pitch, void* C, const OutputSpec& out, cudaStream_t stream,
                     bool packed_s4 = false) {
-  std::lock_guard<std::mutex> lock(g_mutex);
   DeviceState* s = nullptr;
   int rc = device_state(&s);
   if (rc != GEMM_OK) return rc;
@@ -269,11 +371,20 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     k_blocks = 2 * ceil_div(K, 2 * BK_BYTES);  // one packed slot (256 values of K) = two int8 slots
   }
 
+  const bool wide = wide_wanted(cfg, M, N, s->num_sms, swap, csplit, packed_s4);
+  if (wide) {
+    cfg.bn = WIDE_BN;
+    cfg.cta_group = 2;
+    cfg.splits = 1;
+    cfg.split_tiles = 0;
+    cfg.group_m = band_height(M, WIDE_TILE_M, WIDE_BN, s->num_sms / 2);
+  }
+  const int rows_per_cta = wide ? WIDE_CTA_ROWS : BM;
   CUtensorMap ta, tb;
   const bool promote = !(g_l2_policy & 16);
   // packed: the tensor is K/2 bytes wide; boxes stay 128 bytes
   const uint64_t k_cols = packed_s4 ? static_cast<uint64_t>(K) / 2 : static_cast<uint64_t>(K);
-  rc = encode_operand_map(&ta, type, ELEM, A, M, k_cols, a_pitch, BM, promote);
+  rc = encode_operand_map(&ta, type, ELEM, A, M, k_cols, a_pitch, rows_per_cta, promote);
   if (rc != GEMM_OK) return rc;
   rc = encode_operand_map(&tb, type, ELEM, B, N, k_cols, b_pitch, cfg.bn / cfg.cta_group, promote);
   if (rc != GEMM_OK) return rc;
@@ -282,7 +393,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.M = M;
   p.N = N;
   p.K = K;
-  p.tiles_m = ceil_div(M, BM * cfg.cta_group);
+  p.tiles_m = ceil_div(M, rows_per_cta * cfg.cta_group);
   p.tiles_n = ceil_div(N, cfg.bn);
   p.group_m = cfg.group_m;
   p.k_blocks = k_blocks;
@@ -294,8 +405,11 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   // otherwise include the time spent waiting for the predecessor's tail
   p.wait_prior_grid = ((g_l2_policy & 32) || (g_trace_on & 1)) ? 0 : 1;
   p.c_vec_ok = !swap && (ldc % (16 / C_ELEM) == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+  if (wide && N % (16 / C_ELEM)) p.c_vec_ok = 0;  // its 16-byte stores must end on a row's end
   CUtensorMap tc;
-  if (p.c_vec_ok) {
+  if (wide) {
+    tc = ta;  // the wide kernel writes C with plain stores
+  } else if (p.c_vec_ok) {
     // split-K adds into C by TMA reduction, which takes the element type from the map
     rc = encode_c_map(&tc, C, M, N, ldc, C_ELEM,
                       cfg.splits == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
@@ -321,6 +435,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.serpentine_k = (g_l2_policy & 4) ? 0 : 1;
   p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
 
+  if (wide) return launch_wide<KIND, EPI>(s, ta, tb, p, stream);
   if (cfg.splits > 1 && !csplit) {  // only with a dense C (no_split is set for blocks of a larger matrix)
     // Split tiles add into C: zero them first.  All tiles: one memset.  The last wave only:
     // the bounding rectangle of those tiles (other tiles inside it are overwritten later).
@@ -422,7 +537,15 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   }
   if (cfg.cta_group == 2) {
     switch (cfg.bn) {
-      case 256: return launch_variant<KIND, 256, 6, 2, 1, EPI>(s, vbase + 4, ta, tb, tc, p, stream);
+      case 256:
+        if constexpr (EPI == EPI_RAW32) {
+          // ring depth as an ablation variable (gemm_set_stages_override); attr_set bits 216..
+          const int sb = 216 + (KIND == ptx::KIND_F16 ? 0 : 4);
+          if (cfg.stages == 3) return launch_variant<KIND, 256, 3, 2, 1, EPI>(s, sb + 0, ta, tb, tc, p, stream);
+          if (cfg.stages == 4) return launch_variant<KIND, 256, 4, 2, 1, EPI>(s, sb + 1, ta, tb, tc, p, stream);
+          if (cfg.stages == 5) return launch_variant<KIND, 256, 5, 2, 1, EPI>(s, sb + 2, ta, tb, tc, p, stream);
+        }
+        return launch_variant<KIND, 256, 6, 2, 1, EPI>(s, vbase + 4, ta, tb, tc, p, stream);
       case 128: return launch_variant<KIND, 128, 4, 2, 2, EPI>(s, vbase + 5, ta, tb, tc, p, stream);
       case 64: return launch_variant<KIND, 64, 4, 2, 2, EPI>(s, vbase + 6, ta, tb, tc, p, stream);
       default: return GEMM_ERR_INVALID_ARG;
@@ -476,9 +599,12 @@ int launch_unpack(long long rows_a, const uint8_t* packed_a, int8_t* out_a, long
                   cudaStream_t stream) {
   UnpackJob a{reinterpret_cast<const uint4*>(packed_a), out_a, rows_a * (K / 32)};
   UnpackJob b{reinterpret_cast<const uint4*>(packed_b), out_b, rows_b * (K / 32)};
+  DeviceState* s = nullptr;
+  int rc = device_state(&s);
+  if (rc != GEMM_OK) return rc;
   const long long chunks = a.chunks + b.chunks;
   long long blocks = (chunks + 255) / 256;
-  if (blocks > 148 * 32) blocks = 148 * 32;
+  if (blocks > static_cast<long long>(s->num_sms) * 32) blocks = static_cast<long long>(s->num_sms) * 32;
   if (blocks < 1) blocks = 1;
   unpack_s4_kernel<<<static_cast<int>(blocks), 256, 0, stream>>>(
       a, b, K / 32, static_cast<long long>(out_pitch));
@@ -509,54 +635,45 @@ int s4_with_workspace(int M, int N, int K, const uint8_t* A, const uint8_t* B, v
   int8_t* a8 = static_cast<int8_t*>(workspace);
   int8_t* b8 = a8 + align_up(static_cast<size_t>(M) * K, 256);
   int rc;
-  {
-    std::lock_guard<std::mutex> lock(g_mutex);
-    DeviceState* s = nullptr;
-    rc = device_state(&s);
-    if (rc != GEMM_OK) return rc;
-  }
   rc = launch_unpack(M, A, a8, N, B, b8, K, static_cast<size_t>(K), st);
   if (rc != GEMM_OK) return rc;
   return launch_gemm<ptx::KIND_I8>(M, N, K, a8, static_cast<size_t>(K), b8, static_cast<size_t>(K),
                                    C, st, out);
 }
 
-// The library's own grow-only scratch for the current device (cudaMalloc on growth).
-int s4_internal_workspace(size_t need, void** ws, size_t* ws_bytes) {
-  std::lock_guard<std::mutex> lock(g_mutex);
-  DeviceState* s = nullptr;
-  int rc = device_state(&s);
-  if (rc != GEMM_OK) return rc;
-  if (s->s4_workspace_bytes < need) {
-    // Grow: earlier launches may still read the old buffer.
-    cudaError_t e = cudaDeviceSynchronize();
-    if (e != cudaSuccess) return cuda_fail(e);
-    if (s->s4_workspace) cudaFree(s->s4_workspace);
-    s->s4_workspace = nullptr;
-    s->s4_workspace_bytes = 0;
-    e = cudaMalloc(&s->s4_workspace, need);
-    if (e != cudaSuccess) return cuda_fail(e);
-    s->s4_workspace_bytes = need;
-  }
-  *ws = s->s4_workspace;
-  *ws_bytes = s->s4_workspace_bytes;
-  return GEMM_OK;
+// Zero-initialised bookkeeping bytes in front of a pool buffer of `need` data bytes (ready
+// flags of the overlapped pre-pass: one word per 32 rows x 512 columns of int8, both operands).
+size_t s4_head_bytes(int M, int N, int K) {
+  const size_t flags = (static_cast<size_t>(ceil_div(M, 32)) + ceil_div(N, 32)) * ceil_div(K, 512);
+  return align_up(256 + 4 * flags, 256);
 }
 
+thread_local int t_last_s4_overlapped = 0;
+
 // INT4 GEMM by the route gemm_set_s4_scheme selected: the fused kernel if asked for and
-// applicable, else the pre-pass through the library's own workspace.
+// applicable, else the pre-pass through a scratch buffer leased from the device's pool for
+// this stream (allocated stream-ordered on first use or growth: no device-wide
+// synchronisation, and calls on different streams never share a buffer).
 int s4_auto(int M, int N, int K, const uint8_t* A, const uint8_t* B, void* C, const OutputSpec& out,
             cudaStream_t st) {
+  t_last_s4_overlapped = 0;
   if (g_s4_scheme != 1) {
     const int rc = launch_gemm<ptx::KIND_I8>(M, N, K, A, static_cast<size_t>(K) / 2, B,
                                              static_cast<size_t>(K) / 2, C, st, out, true);
     if (rc != GEMM_NOT_FUSED) return rc;
   }
-  void* ws = nullptr;
-  size_t ws_bytes = 0;
-  int rc = s4_internal_workspace(s4_workspace_need(M, N, K), &ws, &ws_bytes);
+  DeviceState* s = nullptr;
+  int dev = 0;
+  int rc = device_state(&s, &dev);
   if (rc != GEMM_OK) return rc;
-  return s4_with_workspace(M, N, K, A, B, C, ws, ws_bytes, out, st);
+  ScratchPool::Lease lease;
+  const int prc = g_pool[dev].acquire(st, s4_workspace_need(M, N, K), s4_head_bytes(M, N, K), &lease);
+  if (prc != 0) return pool_fail(prc);
+  rc = s4_with_workspace(M, N, K, A, B, C, static_cast<uint8_t*>(lease.ptr) + lease.head_bytes,
+                         lease.bytes, out, st);
+  const int qrc = g_pool[dev].release(lease, st);
+  if (rc == GEMM_OK && qrc != 0) rc = pool_fail(qrc);
+  return rc;
 }
 
 int check_scales(const float* row_scale, const float* col_scale, const void* C, int c_is_fp16,

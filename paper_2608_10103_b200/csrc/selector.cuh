@@ -21,7 +21,11 @@ constexpr int kWidths[] = {256, 128, 64, 32};
 
 // Ring depth and 128-byte K atoms per slot of each built shape.
 int stages_for(int bn, int cta_group) {
-  if (cta_group == 2) return bn == 256 ? 6 : 4;
+  if (cta_group == 2 && bn == 256) {
+    const int o = g_override_stages;
+    return (o >= 3 && o <= 6) ? o : 6;
+  }
+  if (cta_group == 2) return 4;
   switch (bn) {
     case 256: return 4;
     case 128: return 3;
@@ -67,11 +71,14 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
                          int fused_only = 0) {
   TileConfig best{256, 2, 6, 8, 1, 0};
   long long best_cost = -1;
+  // the ablation overrides, read once
+  const int o_bn = g_override_bn, o_cta_group = g_override_cta_group;
+  const int o_splits = g_override_splits, o_group_m = g_override_group_m;
   for (int cg = 2; cg >= 1; --cg) {
-    if (g_override_cta_group && cg != g_override_cta_group) continue;
+    if (o_cta_group && cg != o_cta_group) continue;
     if (fused_only == 2 && cg != 2) continue;
     for (int bn : kWidths) {
-      if (g_override_bn && bn != g_override_bn) continue;
+      if (o_bn && bn != o_bn) continue;
       if (!variant_exists(bn, cg) || bn < min_bn) continue;
       if (fused_only == 2 && bn != 256) continue;
       const long long tiles = static_cast<long long>(ceil_div(M, BM * cg)) * ceil_div(N, bn);
@@ -86,16 +93,16 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
         if (split_cap && max_split > split_cap) max_split = split_cap;
         if (max_split < 1) max_split = 1;
       }
-      if (g_override_splits) {
+      if (o_splits) {
         // forced: the largest factor <= the request that leaves no K range empty
-        max_split = g_override_splits < slots ? g_override_splits : slots;
+        max_split = o_splits < slots ? o_splits : slots;
         while (max_split > 1 &&
                static_cast<long long>(max_split - 1) * ceil_div(slots, max_split) >= slots)
           --max_split;
         if (!allow_split) max_split = 1;
       }
       if (max_split > slots) max_split = slots;
-      for (int sp = g_override_splits ? max_split : 1; sp <= max_split; ++sp) {
+      for (int sp = o_splits ? max_split : 1; sp <= max_split; ++sp) {
         if (static_cast<long long>(sp - 1) * ceil_div(slots, sp) >= slots) continue;  // empty range
         if (fused_only && !fused_s4_variant_exists(bn, cg, sp)) continue;
         const int per = ceil_div(slots, sp) * atoms;  // k-blocks per unit
@@ -134,7 +141,7 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
         ceil_div(k_blocks, force_atoms ? force_atoms : atoms_for(best.bn, best.cta_group));
     best.split_tiles = best.splits > 1 ? static_cast<int>(tiles) : 0;
     const long long r = tiles % units;
-    if (allow_split && best.splits == 1 && g_override_splits == 0 && tiles > units && r > 0 &&
+    if (allow_split && best.splits == 1 && o_splits == 0 && tiles > units && r > 0 &&
         2 * r <= units && slots >= 64) {  // measured: pays off (+2-3 %) only for long K
       int sp = static_cast<int>(units / r);
       if (sp > 4) sp = 4;
@@ -154,7 +161,7 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
   int units = num_sms / best.cta_group;
   int g = 1;
   while ((g + 1) * (g + 1) * rows_per_tile <= 2 * units * best.bn) ++g;
-  if (g_override_group_m) g = g_override_group_m;
+  if (o_group_m) g = o_group_m;
   int tiles_m = ceil_div(M, rows_per_tile);
   if (g > tiles_m) g = tiles_m;
   if (g < 1) g = 1;

@@ -67,7 +67,7 @@ def test_random_shapes_configs_and_entry_points(seed):
         for trial in range(3):
             cfg = CONFIGS[int(g.integers(len(CONFIGS)))]
             mode = str(g.choice(_modes(prec)))
-            if mode == "static" and (M + N) * K > binding.gemm_s4_static_capacity():
+            if mode == "static" and binding.gemm_s4_workspace_bytes(M, N, K) > binding.gemm_s4_static_capacity():
                 mode = "raw"
             stream = side if g.integers(2) else None
             what = "%s %s M=%d N=%d K=%d cfg=%s side_stream=%s" % (prec, mode, M, N, K, cfg, stream is not None)

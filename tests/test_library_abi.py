@@ -9,7 +9,8 @@ import pytest
 from paper_2608_10103_b200 import binding, build as lib_build
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-HEADER = os.path.join(ROOT, "include", "b200gemm.h")
+HEADERS = [os.path.join(ROOT, "include", "b200gemm.h"),
+           os.path.join(ROOT, "include", "b200gemm_debug.h")]
 
 
 @pytest.fixture(scope="module")
@@ -19,7 +20,7 @@ def lib():
 
 
 def declared_functions():
-    text = open(HEADER).read()
+    text = "".join(open(h).read() for h in HEADERS)
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     names = re.findall(r"\b(gemm_[a-z0-9_]+)\s*\(", text)
     return sorted(set(names))
@@ -128,7 +129,11 @@ def test_selector_invariants_over_many_shapes(lib):
                 assert N >= 1024 and M <= (32 if prec == "fp16" and N < 16384 else 64)
                 M, N = N, M
             cg, bn, sp = c["cta_group"], c["BN"], c["split_k"]
-            assert (cg, bn) in built and c["BM"] == 128 * cg
+            wide = c["BM"] == 512            # the 512 x 256 CTA-pair kernel for large problems
+            assert (cg, bn) in built and (c["BM"] == 128 * cg or (wide and (cg, bn) == (2, 256)))
+            if wide:
+                assert sp == 1 and "swap_ab" not in text and "fused_unpack" not in text
+                assert -(-M // 512) * -(-N // 256) >= 2 * 74 and c["stages"] == 4
             atoms = c["BK"] * elem // 128
             assert atoms in (1, 2)
             if "fused_unpack" in text:   # K is split in packed slots of 256 values
@@ -158,7 +163,13 @@ def test_selector_invariants_over_many_shapes(lib):
 
 def test_selector_headline_choices(lib):
     big = _parse(binding.gemm_query_config("fp16", 8192, 8192, 8192))
-    assert (big["BM"], big["BN"], big["cta_group"], big["split_k"], big["stages"]) == (256, 256, 2, 1, 6)
+    assert (big["BM"], big["BN"], big["cta_group"], big["split_k"], big["stages"]) == (512, 256, 2, 1, 4)
+    binding.gemm_set_kernel_family(1)
+    try:
+        classic = _parse(binding.gemm_query_config("fp16", 8192, 8192, 8192))
+        assert (classic["BM"], classic["BN"], classic["cta_group"], classic["stages"]) == (256, 256, 2, 6)
+    finally:
+        binding.gemm_set_kernel_family(0)
     dec = _parse(binding.gemm_query_config("s8", 16, 8192, 8192))
     assert dec["split_k"] > 1 and dec["split_tiles"] == dec["tiles"]
     tail = _parse(binding.gemm_query_config("fp16", 4096, 4096, 8192))

@@ -1,8 +1,8 @@
 """Collected after every other GPU test file but the last: the launch with the most tiles per
 CTA and the shortest mainloop (84 tiles of one k-block per CTA pair, 1.6 GB of C) must still be
-right after every other kernel variant of the library has run in this process.  (A kernel
-variant that kept an operand tile in tensor memory once made exactly this launch fail when it
-had run earlier in the process; the fixed-order suite did not show it.)"""
+right after every other kernel variant of the library has run in this process, i.e. no
+variant may leave anything behind (tensor memory, barriers, device-side state) that a later,
+unrelated launch trips over."""
 import pytest
 
 from paper_2608_10103_b200 import binding, synth
