@@ -19,7 +19,8 @@ Other modes (1 GPU, one JSON line per measurement): --sweep (precision x size,
 N = 512..8192), --ablation (tile / raster / L2 / INT4 route at --size, with the
 kernel's cycle accounting), --few-rows (M = 1..128 against the HBM roofline;
 --shape M,N,K for any other shape), --selector-check (the automatic tile and
-split-K choice against forced ones).
+split-K choice against forced ones), --capture (the launches the profiler summaries under
+profiles/ were taken from).
 """
 from __future__ import annotations
 
@@ -358,8 +359,8 @@ def run_ours(args, rank, world):
                             "value": replicas.whole_job_rate(ops, world, ms), "unit": UNIT[p],
                             "sm_mhz_settled": c2.get("sm_mhz_settled"),
                             "power_w_settled": c2.get("power_w_settled"),
-                            "joules_per_gemm": (c2["power_w_mean"] * ms * 1e-3
-                                                if c2.get("power_w_mean") else None),
+                            "joules_per_gemm": (c2["power_w_settled"] * ms * 1e-3
+                                                if c2.get("power_w_settled") else None),
                             "clock_samples": c2.get("samples"), "reasons": c2.get("reasons")}
         if binding.gemm_last_device_status() != 0:
             raise SystemExit("bench.py: a kernel reported a barrier timeout")
@@ -573,6 +574,15 @@ def run_sweep(args):
                 call(stream)
             host_us = (time.perf_counter() - t0) / 200 * 1e6
             torch.cuda.synchronize()
+            # the library's own share of that: the C entry point called with arguments that
+            # are already marshalled (what a C or C++ caller pays, plus one ctypes dispatch)
+            fn = getattr(binding.lib(), {"fp16": "gemm_fp16", "s8": "gemm_s8", "s4": "gemm_s4"}[prec])
+            c_args = (N, N, N, dA.data_ptr(), dB.data_ptr(), C.data_ptr(), int(stream.cuda_stream))
+            t0 = time.perf_counter()
+            for _ in range(200):
+                fn(*c_args)
+            host_us_c = (time.perf_counter() - t0) / 200 * 1e6
+            torch.cuda.synchronize()
             reps = max(5, min(100, int(20.0 / max(timed(lambda: call(stream), 5), 1e-3))))
             g_many, g_one = graph_of(call, reps), graph_of(call, 1)
             warm = float(np.median([timed(g_many.replay, 1) for _ in range(5)])) / reps
@@ -583,7 +593,7 @@ def run_sweep(args):
             print(json.dumps({
                 "sweep": True, "precision": prec, "N": N, "seed": synth.sweep_seed(prec, N),
                 "ms": warm, "reps": reps, "ms_cold_single_launch": cold,
-                "host_us_per_call": host_us,
+                "host_us_per_call": host_us, "host_us_c_abi": host_us_c,
                 "value": rate, "unit": UNIT[prec], "frac_of_spec_peak": rate / SPEC_PEAK[prec],
                 "frac_of_cublas_bf16_burst_scaled": rate / ref,
                 "frac_of_mma_only_peak": rate / mma_peak[prec], "mma_only_peak": mma_peak[prec],
@@ -760,33 +770,46 @@ def run_ablation(args):
     data = {"fp16": synth.fp16_normal_clipped(N, N, N, seed=3),
             "s8": synth.s8_uniform(N, N, N, seed=synth.sweep_seed("s8", 8192)),
             "s4": synth.s4_uniform(N, N, N, seed=synth.sweep_seed("s4", 8192))}
-    variants = [("baseline (selector default)", (0, 0, 0), 11, 1)]
-    variants += [("tile 128x%d, one CTA" % bn, (bn, 0, 1), 11, 1) for bn in (256, 128, 64, 32)]
-    variants += [("tile 256x%d, CTA pair" % bn, (bn, 0, 2), 11, 1) for bn in (256, 128, 64)]
-    variants += [("band height %d" % g, (256, g, 2), 11, 1) for g in (2, 4, 8, 16, 32)]
-    variants += [("L2: no hints, forward K only", (0, 0, 0), 4, 1),
-                 ("L2: no hints, serpentine K", (0, 0, 0), 0, 1),
-                 ("L2: keep A, stream B", (0, 0, 0), 1, 1),
-                 ("L2: keep A and B", (0, 0, 0), 2, 1),
-                 ("L2: default + 128-byte promotion", (0, 0, 0), 27, 1),
-                 ("ablate: no MMAs (loads + barriers only)", (0, 0, 0), 11, 3),
-                 ("ablate: no loads (MMAs + barriers only)", (0, 0, 0), 11, 5),
-                 ("epilogue waits with nanosleep back-off", (0, 0, 0), 11, 9),
-                 ("epilogue: direct register -> global stores", (0, 0, 0), 11, 33)]
-    # INT4: how the nibbles reach the int8 tensor-core path (the traced launch is the GEMM;
-    # the pre-pass launch of route 0 is inside the timed loop but not in the cycle accounting)
-    s4_variants = [("INT4 route 0: pre-pass to int8 + INT8 GEMM (default at this size)", (0, 0, 0), 11, 1, 1),
-                   ("INT4 route 1: nibbles expanded inside the GEMM kernel", (0, 0, 0), 11, 1, 2),
-                   ("INT4 route 1, ablate: no MMAs", (0, 0, 0), 11, 3, 2),
-                   ("INT4 route 1, ablate: no operand loads", (0, 0, 0), 11, 5, 2)]
+    # (name, (BN, band height, CTAs per tile), L2 policy, trace bits, INT4 route, kernel family,
+    #  ring depth); family 1 = the 256 x 256 pair tile, 2 = the 512 x 256 tile, 0 = automatic
+    def V(name, override=(0, 0, 0), policy=11, trace=1, scheme=0, family=1, stages=0):
+        return (name, override, policy, trace, scheme, family, stages)
+    variants = [V("baseline (automatic choice)", family=0),
+                V("kernel: 256x256 tile per CTA pair, 2 accumulator buffers"),
+                V("kernel: 512x256 tile per CTA pair, accumulators fill TMEM", family=2)]
+    variants += [V("tile 128x%d, one CTA" % bn, (bn, 0, 1)) for bn in (256, 128, 64, 32)]
+    variants += [V("tile 256x%d, CTA pair" % bn, (bn, 0, 2)) for bn in (256, 128, 64)]
+    variants += [V("256x256 pair tile, ring depth %d" % st, (256, 0, 2), stages=st) for st in (3, 4, 5, 6)]
+    variants += [V("band height %d" % g, (256, g, 2)) for g in (2, 4, 8, 16, 32)]
+    variants += [V("512x256 tile, band height %d" % g, (0, g, 0), family=2) for g in (2, 4, 6, 8, 16)]
+    variants += [V("L2: no hints, forward K only", policy=4),
+                 V("L2: no hints, serpentine K", policy=0),
+                 V("L2: keep A, stream B", policy=1),
+                 V("L2: keep A and B", policy=2),
+                 V("L2: default + 128-byte promotion", policy=27),
+                 V("ablate: no MMAs (loads + barriers only)", trace=3),
+                 V("ablate: no loads (MMAs + barriers only)", trace=5),
+                 V("epilogue waits with nanosleep back-off", trace=9),
+                 V("epilogue: direct register -> global stores", trace=33),
+                 V("512x256 tile, ablate: no MMAs", trace=3, family=2),
+                 V("512x256 tile, ablate: no loads", trace=5, family=2)]
+    # INT4: how the nibbles reach the int8 tensor-core path (the traced launch is the GEMM; a
+    # separate pre-pass launch is inside the timed loop but not in the cycle accounting)
+    s4_variants = [V("INT4 route 0: pre-pass launch to int8 + INT8 GEMM (default at this size)", family=0),
+                   V("INT4 route 0': pre-pass inside the INT8 GEMM kernel, ahead of its tiles", scheme=4, family=0),
+                   V("INT4 route 1: nibbles expanded in shared memory inside the GEMM kernel", scheme=2),
+                   V("INT4 route 1, ablate: no MMAs", trace=3, scheme=2),
+                   V("INT4 route 1, ablate: no operand loads", trace=5, scheme=2)]
     for prec in [q for q in ("fp16", "s8", "s4") if q in args.precisions.split(",")]:
         dA, dB = (torch.from_numpy(x).cuda() for x in data[prec])
         C = torch.empty((N, N), dtype=torch.float32 if prec == "fp16" else torch.int32,
                         device="cuda")
         flop_per_clk = 8192 if prec == "fp16" else 16384
         for v in (s4_variants if prec == "s4" else variants):
-            name, override, policy, trace = v[:4]
-            binding.gemm_set_s4_scheme(v[4] if len(v) > 4 else 0)
+            name, override, policy, trace, scheme, family, stages = v
+            binding.gemm_set_s4_scheme(scheme)
+            binding.gemm_set_kernel_family(family)
+            binding.gemm_set_stages_override(stages)
             binding.gemm_set_config_override(*override)
             binding.gemm_set_l2_policy(policy)
             binding.gemm_trace_enable(trace)
@@ -822,14 +845,55 @@ def run_ablation(args):
                     "mma_wait_operands": float(a["mma_wait_operands"][lead].mean() / kb_total),
                     "mma_issue": float(a["mma_issue"][lead].mean() / kb_total),
                     "mma_commit": float(a["mma_commit"][lead].mean() / kb_total),
+                    "mma_wait_accumulators": float((a["mma_wait_accumulator"][lead].mean() +
+                                                    a["mma_wait_accumulator1"][lead].mean()) / kb_total),
                     "producer_wait": float(a["producer_wait"].mean() / kb_total),
                     "producer_issue": float(a["producer_issue"].mean() / kb_total)},
                 "epilogue_busy_frac": float(a["epilogue_busy"].mean() / a["cycles"].mean()),
                 "result_valid": trace in (1, 9, 33), **unpack}), flush=True)
     binding.gemm_set_s4_scheme(0)
+    binding.gemm_set_kernel_family(0)
+    binding.gemm_set_stages_override(0)
     binding.gemm_set_config_override(0, 0, 0)
     binding.gemm_set_l2_policy(11)
     binding.gemm_trace_enable(0)
+    if binding.gemm_last_device_status() != 0:
+        raise SystemExit("bench.py: a kernel reported a barrier timeout")
+
+
+def run_capture(args):
+    """Workload for profiler captures (the summaries under profiles/ name the full command): the
+    FP16 GEMM at --size (seed 3) on both kernel families and a few raster band heights, two
+    launches each, inside a cudaProfilerStart/Stop range, so that `ncu --profile-from-start off`
+    sees exactly these launches.  Prints which configuration each pair of launches ran."""
+    import torch
+    from paper_2608_10103_b200 import binding, synth
+    torch.cuda.set_device(0)
+    N = args.size
+    A, B = synth.fp16_normal_clipped(N, N, N, seed=3)
+    dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    C = torch.empty((N, N), dtype=torch.float32, device="cuda")
+    cases = [("automatic", 0, 0), ("256x256 pair tile", 1, 0), ("512x256 tile, band 4", 2, 4),
+             ("512x256 tile, band 5", 2, 5), ("512x256 tile, band 6", 2, 6), ("512x256 tile, band 8", 2, 8)]
+
+    def setup(fam, g):
+        binding.gemm_set_kernel_family(fam)
+        binding.gemm_set_config_override(0, g, 0, 0)
+
+    for _, fam, g in cases:
+        setup(fam, g)
+        binding.gemm_fp16(dA, dB, C)
+    torch.cuda.synchronize()
+    torch.cuda.profiler.start()
+    for name, fam, g in cases:
+        setup(fam, g)
+        for _ in range(2):
+            binding.gemm_fp16(dA, dB, C)
+        print(json.dumps({"capture": name, "config": binding.gemm_query_config("fp16", N, N, N)}),
+              flush=True)
+    torch.cuda.synchronize()
+    torch.cuda.profiler.stop()
+    setup(0, 0)
     if binding.gemm_last_device_status() != 0:
         raise SystemExit("bench.py: a kernel reported a barrier timeout")
 
@@ -855,6 +919,9 @@ def main():
                     help="tile / raster / L2 / load-vs-MMA ablation with cycle accounting (1 GPU)")
     ap.add_argument("--selector-check", action="store_true",
                     help="automatic tile / split-K choice against forced ones, one JSON line per shape")
+    ap.add_argument("--capture", action="store_true",
+                    help="profiler workload: FP16 GEMM at --size, both kernel families and band "
+                         "heights, inside a profiler range (1 GPU)")
     ap.add_argument("--sweep", action="store_true",
                     help="precision x size sweep N=512..8192, one JSON line per cell (1 GPU)")
     ap.add_argument("--precisions", default="fp16,s8,s4")
@@ -866,7 +933,10 @@ def main():
         args.warmup = 3
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.selector_check:
+    if args.capture:
+        if rank == 0:
+            run_capture(args)
+    elif args.selector_check:
         if rank == 0:
             run_selector_check(args)
     elif args.ablation:

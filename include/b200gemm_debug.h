@@ -87,8 +87,15 @@ int gemm_set_kernel_family(int family);
  * its CTA-pair tile if the tiles fill their waves to 75 % (256 x 28672 x 8192:
  * 119 -> 67 us; 512 x 16384 x 4096: 44 -> 35 us); else the pre-pass.  1: always
  * the pre-pass; 2: fused wherever a fused variant is built (every one-CTA tile,
- * and the 256 x 256 and 256 x 128 CTA pairs), else the pre-pass.  gemm_s4_ws and gemm_s4_static
- * always use the pre-pass.  Results are identical, bit for bit.
+ * and the 256 x 256 and 256 x 128 CTA pairs), else the pre-pass.  4: the
+ * pre-pass, but where the INT8 GEMM runs on the 256 x 256 CTA-pair tile over at
+ * least two waves its own epilogue warps expand the operands inside that
+ * kernel, chunk by chunk ahead of the tiles that read them (no separate launch;
+ * measured slower than 1 -- N = 8192: 574 k SM cycles against 496 k plus a
+ * 36 us pre-pass -- because that kernel already keeps the SM's L2 port and
+ * shared-memory pipe full; kept as the ablation's third INT4 route).  3 = 1.
+ * gemm_s4_ws and gemm_s4_static always use the pre-pass launch.  Results are
+ * identical, bit for bit.
  * gemm_query_config shows the route.  The paper has no counterpart; its Run 4
  * ablates how the operands reach the tensor cores, of which this is the
  * analogue here.

@@ -337,7 +337,8 @@ def gemm_read_device_status(host_out: torch.Tensor, stream=None):
 def gemm_set_s4_scheme(scheme: int = 0):
     """Route of gemm_s4 / gemm_s4_dequant: 0 = automatic (nibbles expanded inside the GEMM
     kernel for problems with few rows on one side, else a pre-pass to int8 + the INT8 GEMM);
-    1 = always the pre-pass; 2 = inside the GEMM kernel wherever such a variant is built."""
+    1 = always the pre-pass; 2 = inside the GEMM kernel wherever such a variant is built;
+    4 = the pre-pass done by the INT8 GEMM kernel's own epilogue warps where that applies."""
     _check(lib().gemm_set_s4_scheme(int(scheme)), "gemm_set_s4_scheme")
 
 

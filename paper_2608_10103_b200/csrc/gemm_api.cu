@@ -166,7 +166,7 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
   TileConfig c;
   bool fused = false, swap = false;
   const int user_m = M, user_n = N;
-  if (precision == GEMM_PREC_S4 && g_s4_scheme != 1) {  // the decisions of s4_auto / launch_gemm_epi
+  if (precision == GEMM_PREC_S4 && !s4_prepass_forced()) {  // the decisions of s4_auto / launch_gemm_epi
     swap = swap_ab_wanted(M, N, true, OutputSpec());
     const TileConfig i8 =
         swap ? select_config(N, M, num_sms, kb, 32, true) : select_config(M, N, num_sms, kb, 32, true);
@@ -182,7 +182,7 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
     M = user_n;
     N = user_m;
   }
-  const bool wide = wide_wanted(c, M, N, num_sms, swap, false, fused);
+  const bool wide = wide_wanted(c, M, N, num_sms, swap, false, fused, precision == GEMM_PREC_FP16);
   if (wide) {
     c.bn = WIDE_BN;
     c.cta_group = 2;
@@ -255,7 +255,7 @@ int gemm_set_kernel_family(int family) {
 }
 
 int gemm_set_s4_scheme(int scheme) {
-  if (scheme < 0 || scheme > 2) return GEMM_ERR_INVALID_ARG;
+  if (scheme < 0 || scheme > 4) return GEMM_ERR_INVALID_ARG;
   g_s4_scheme = scheme;
   return GEMM_OK;
 }

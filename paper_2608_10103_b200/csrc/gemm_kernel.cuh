@@ -49,6 +49,7 @@
 #include <stdint.h>
 
 #include "ptx.cuh"
+#include "s4_ahead.cuh"
 
 namespace b200gemm {
 
@@ -125,6 +126,9 @@ struct GemmParams {
   // producer of CTA 0 leaves out the 3rd ring slot of its first tile, so the consumers' bounded
   // waits must expire, record a status code and let the kernel drain and return.
   int ablate;
+  // Overlapped INT4 pre-pass (kernel variants built with AHEAD): the int8 operands this GEMM
+  // reads are produced by its own epilogue warps from the packed ones named here.
+  S4Ahead ahead;
 };
 
 // Trace slots written per CTA when GemmParams::trace is set.
@@ -238,7 +242,7 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
 // DBG: the measurement and drill switches of GemmParams::ablate are compiled in (the product
 // instantiations leave them out of their loops).
 template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32, int PSTAGES = 0,
-          int CSPLIT = 1, bool DBG = false>
+          int CSPLIT = 1, bool DBG = false, bool AHEAD = false>
 __global__ void __launch_bounds__(PSTAGES > 0 ? NUM_THREADS_FUSED : NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
@@ -256,6 +260,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   // also serves the 16-bit and scaled outputs, and a call is a single launch.
   static_assert(CSPLIT == 1 || ((CSPLIT == 2 || CSPLIT == 4) && CTA_GROUP == 1 && BN <= 64),
                 "cluster split-K: two or four single CTAs, narrow tile");
+  static_assert(!AHEAD || (KIND == ptx::KIND_I8 && !FUSED && KB == 1 && CSPLIT == 1),
+                "overlapped INT4 pre-pass: the plain int8 kernel, one atom per slot");
   static_assert(!FUSED || (KIND == ptx::KIND_I8 && KB == 1 && STAGES >= 2),
                 "fused INT4: int8 MMAs, one atom per slot, a packed slot fills two int8 slots at once");
   constexpr int ELEM_BYTES = (KIND == ptx::KIND_F16) ? 2 : 1;
@@ -392,7 +398,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       uint32_t phase = 0;
       int issued = 0;
       bool ok = true;
-      long long waited = 0, prod_issue = 0;
+      long long waited = 0, prod_issue = 0, flag_wait = 0;
       const uint64_t pol_a = p.l2_policy == 0 ? ptx::policy_evict_normal() : ptx::policy_evict_last();
       const uint64_t pol_b = (p.l2_policy == 0 || p.l2_policy == 3) ? ptx::policy_evict_normal()
                              : p.l2_policy == 1                      ? ptx::policy_evict_first()
@@ -436,6 +442,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         }
         if (p.serpentine_k) backward = !backward;
       }
+      // overlapped INT4 pre-pass: the int8 rows behind a box must have been produced
+      const uint32_t ahead_epoch = AHEAD ? s4a_epoch(p.ahead) : 0u;
+      bool ahead_all = !AHEAD;
       for (int t = first_tile; !FUSED && t < num_tiles && ok; t += tile_stride) {
         int tm, tn, tile, k_begin, k_end;
         bool add;
@@ -443,10 +452,29 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         tile_coords(p, tile, tm, tn);
         const int a_row = tm * TILE_M + static_cast<int>(cta_rank) * BM;
         const int b_row = tn * BN + static_cast<int>(cta_rank) * L::B_ROWS;
+        int ahead_kc = -1;
         for (int ks = k_begin; ks < k_end; ++ks) {
           const long long w0 = trace ? clock64() : 0;
           ok = wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status,
                             DEV_TIMEOUT_PRODUCER);
+          if constexpr (AHEAD) {
+            const int kc = (backward ? k_begin + k_end - 1 - ks : ks) * BK_BYTES / S4A_CHUNK_COLS;
+            const long long f0 = trace ? clock64() : 0;
+            if (ok && !ahead_all && kc != ahead_kc) {
+              ahead_kc = kc;
+              if (ld_acquire_u32(p.ahead.sync + S4A_ALL_DONE) == ahead_epoch) {
+                ahead_all = true;
+              } else {
+                ok = s4a_wait_ready(p.ahead, ahead_epoch, a_row, BM / S4A_CHUNK_ROWS, b_row,
+                                    L::B_ROWS / S4A_CHUNK_ROWS, kc, lane, abort_flag, WAIT_LIMIT_NS);
+                if (!ok) {
+                  *abort_flag = 1;
+                  atomicCAS(p.status, 0, DEV_TIMEOUT_PRODUCER);
+                }
+              }
+            }
+            if (trace) flag_wait += clock64() - f0;
+          }
           const long long w9 = trace ? clock64() : 0;
           if (trace) waited += w9 - w0;
           if (!ok) break;
@@ -486,6 +514,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       if (trace && elected) {
         trace[TRACE_PROD_WAIT] = static_cast<unsigned long long>(waited);
         trace[TRACE_PROD_ISSUE] = static_cast<unsigned long long>(prod_issue);
+        if (AHEAD) trace[TRACE_UNPACK_WAIT_IN] = static_cast<unsigned long long>(flag_wait);
       }
       if (!ok && elected && (FUSED || CTA_GROUP == 1 || leader)) {
         // Gave up: let the copies already in flight land before the CTA exits.
@@ -739,6 +768,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     long long epi_wait = 0, epi_busy = 0, tiles_done = 0;
     uint32_t staged_blocks = 0;  // blocks sent through the staging buffers so far
     bool prior_grid_done = false;
+    uint32_t ahead_epoch = 0;    // overlapped INT4 pre-pass: 0 = not read yet (epochs start at 1)
+    bool ahead_more = AHEAD;     // ... chunks may be left to claim
+    long long ahead_busy = 0;
     uint32_t xphase = 0;         // cluster split-K: parity of the partial-sum hand-over
     const bool xpeer = CSPLIT > 1 && krank != 0;  // this CTA only contributes partial sums
     // Cluster split-K, rank 0: adds the other CTAs' partial sums for accumulator columns
@@ -791,6 +823,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           if (p.row_scale && row < p.M) rs = __ldg(p.row_scale + row);
           if (p.col_scale && lane * 32 < BN && col0 + lane * 32 < p.N)
             ptx::prefetch_l1(p.col_scale + col0 + lane * 32);
+        }
+      }
+      if constexpr (AHEAD) {
+        // while the accumulator is not ready: expand packed INT4 chunks for the tiles to come
+        if (ahead_more) {
+          if (p.wait_prior_grid && !prior_grid_done) {  // the scratch may be in use by the grid in front
+            ptx::grid_dep_wait();
+            prior_grid_done = true;
+          }
+          if (ahead_epoch == 0) ahead_epoch = s4a_epoch(p.ahead);
+          const long long u0 = trace ? clock64() : 0;
+          ahead_more = s4a_work(p.ahead, ahead_epoch, lane, [&]() {
+            return __any_sync(0xffffffffu, ptx::mbar_test_wait(acc_full_bar(acc), acc_phase));
+          });
+          if (trace) ahead_busy += clock64() - u0;
         }
       }
       const long long w0 = trace ? clock64() : 0;
@@ -1009,6 +1056,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
+    if constexpr (AHEAD) {
+      // no tile left for this CTA, but the list may not be exhausted: other CTAs' tiles wait
+      // for these chunks
+      if (ok && ahead_more) {
+        if (ahead_epoch == 0) {
+          if (p.wait_prior_grid && !prior_grid_done) ptx::grid_dep_wait();
+          ahead_epoch = s4a_epoch(p.ahead);
+        }
+        s4a_work(p.ahead, ahead_epoch, lane, []() { return false; });
+      }
+    }
     // C stores still in flight read this CTA's shared memory: wait until they have read it
     // (their global writes complete on their own before the grid counts as finished).  A
     // hand-over copy into rank 0's shared memory has to have landed as well.
@@ -1021,6 +1079,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       trace[TRACE_EPI_WAIT] = static_cast<unsigned long long>(epi_wait);
       trace[TRACE_EPI_BUSY] = static_cast<unsigned long long>(epi_busy);
       trace[TRACE_TILES] = static_cast<unsigned long long>(tiles_done);
+      if (AHEAD) trace[TRACE_UNPACK_BUSY] = static_cast<unsigned long long>(ahead_busy);
     }
   }
 
@@ -1036,6 +1095,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc<CTA_GROUP>(tmem_base, TMEM_COLS);
+  }
+  if constexpr (AHEAD) {
+    if (threadIdx.x == 0) s4a_cta_exit(p.ahead);  // every claim of this CTA lies before the barrier above
   }
   if (trace && threadIdx.x == 0) {
     trace[TRACE_CYCLES] = static_cast<unsigned long long>(clock64() - clk_start);

@@ -46,8 +46,8 @@ struct WideSmem {
   static constexpr int EPI_OFFSET = RING_BYTES;
   static constexpr int EPI_BYTES = WIDE_EPI_WARPS * EPI_BUF_BYTES;
   static constexpr int BAR_OFFSET = EPI_OFFSET + EPI_BYTES;
-  // full[STAGES], empty[STAGES], acc_full, acc_empty[2], drain
-  static constexpr int NUM_BARS = 2 * WIDE_STAGES + 4;
+  // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], drain
+  static constexpr int NUM_BARS = 2 * WIDE_STAGES + 5;
   static constexpr int MISC_OFFSET = BAR_OFFSET + NUM_BARS * 8;
   static constexpr int TOTAL = MISC_OFFSET + 16;
   static constexpr int DYN_BYTES = TOTAL + 1024;
@@ -91,9 +91,9 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
   const uint32_t bar0 = base + L::BAR_OFFSET;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
-  const uint32_t acc_full_bar = bar0 + 8u * (2 * STAGES);
-  auto acc_empty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 1 + a); };
-  const uint32_t drain_bar = bar0 + 8u * (2 * STAGES + 3);
+  auto acc_full_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto acc_empty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * STAGES + 4);
   volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(base_ptr + L::MISC_OFFSET);
   volatile uint32_t* abort_flag = tmem_holder + 1;
 
@@ -117,7 +117,8 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
       ptx::mbar_init(full_bar(s), 1);
       ptx::mbar_init(empty_bar(s), 1);
     }
-    ptx::mbar_init(acc_full_bar, 1);
+    ptx::mbar_init(acc_full_bar(0), 1);
+    ptx::mbar_init(acc_full_bar(1), 1);
     ptx::mbar_init(acc_empty_bar(0), 2 * WIDE_EPI_WARPS);
     ptx::mbar_init(acc_empty_bar(1), 2 * WIDE_EPI_WARPS);
     ptx::mbar_init(drain_bar, 1);
@@ -229,36 +230,37 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
       auto advance = [&](int& s, uint32_t& ph) {
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       };
-      for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
-        // The first accumulator is free: run ahead on it while the second is being read out.
-        long long w0 = trace ? clock64() : 0;
-        ok = wait_bounded(acc_empty_bar(0), acc_phase ^ 1u, abort_flag, p.status, DEV_TIMEOUT_MMA);
-        if (trace) wait_acc0 += clock64() - w0;
-        if (!ok) break;
-        ptx::tc_fence_after_sync();
-        const int ahead = k_slots < STAGES ? k_slots : STAGES;
+      // One pass over `n` consecutive ring slots for accumulator 0 (waiting for their operands),
+      // then a second pass over the same slots for accumulator 1, which also frees them.
+      // Used at both ends of a tile: at its start accumulator 0 is handed back first and the
+      // tensor pipe gets going on it while accumulator 1 is still being read out; at its end
+      // accumulator 0 finishes n k-blocks' worth of MMA time before accumulator 1, so its
+      // rows are on their way out while the pipe is still busy.
+      auto two_pass = [&](int n, bool first_of_tile, bool last_of_tile) {
         int s = stage;
         uint32_t ph = phase;
-        for (int i = 0; i < ahead && ok; ++i) {
+        for (int i = 0; i < n && ok; ++i) {
           const long long w1 = trace ? clock64() : 0;
           ok = wait_bounded(full_bar(s), ph, abort_flag, p.status, DEV_TIMEOUT_MMA);
           const long long w2 = trace ? clock64() : 0;
           if (trace) wait_full += w2 - w1;
-          if (!ok) break;
+          if (!ok) return;
           ptx::tc_fence_after_sync();
-          issue_half(s, 0, i == 0);
+          issue_half(s, 0, first_of_tile && i == 0);
           if (trace) t_issue += clock64() - w2;
           advance(s, ph);
         }
-        if (!ok) break;
-        w0 = trace ? clock64() : 0;
-        ok = wait_bounded(acc_empty_bar(1), acc_phase ^ 1u, abort_flag, p.status, DEV_TIMEOUT_MMA);
-        if (trace) wait_acc1 += clock64() - w0;
-        if (!ok) break;
-        ptx::tc_fence_after_sync();
-        for (int i = 0; i < ahead; ++i) {
+        if (last_of_tile && elected) ptx::mma_commit_pair(acc_full_bar(0), 0x3);
+        if (first_of_tile) {
+          const long long w0 = trace ? clock64() : 0;
+          ok = wait_bounded(acc_empty_bar(1), acc_phase ^ 1u, abort_flag, p.status, DEV_TIMEOUT_MMA);
+          if (trace) wait_acc1 += clock64() - w0;
+          if (!ok) return;
+          ptx::tc_fence_after_sync();
+        }
+        for (int i = 0; i < n; ++i) {
           const long long w2 = trace ? clock64() : 0;
-          issue_half(stage, 1, i == 0);
+          issue_half(stage, 1, first_of_tile && i == 0);
           const long long w4 = trace ? clock64() : 0;
           if (elected) ptx::mma_commit_pair(empty_bar(stage), 0x3);
           if (trace) {
@@ -267,7 +269,19 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
           }
           advance(stage, phase);
         }
-        for (int ks = ahead; ks < k_slots; ++ks) {
+        if (last_of_tile && elected) ptx::mma_commit_pair(acc_full_bar(1), 0x3);
+      };
+      for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
+        const long long w0 = trace ? clock64() : 0;
+        ok = wait_bounded(acc_empty_bar(0), acc_phase ^ 1u, abort_flag, p.status, DEV_TIMEOUT_MMA);
+        if (trace) wait_acc0 += clock64() - w0;
+        if (!ok) break;
+        ptx::tc_fence_after_sync();
+        const int head = k_slots < STAGES ? k_slots : STAGES;
+        const int tail = (k_slots - head) < STAGES ? (k_slots - head) : STAGES;
+        two_pass(head, true, tail == 0);
+        if (!ok) break;
+        for (int ks = head; ks < k_slots - tail; ++ks) {
           const long long w1 = trace ? clock64() : 0;
           ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
           const long long w2 = trace ? clock64() : 0;
@@ -285,7 +299,8 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
           advance(stage, phase);
         }
         if (!ok) break;
-        if (elected) ptx::mma_commit_pair(acc_full_bar, 0x3);
+        if (tail > 0) two_pass(tail, false, true);
+        if (!ok) break;
         acc_phase ^= 1u;
       }
       if (trace && elected) {
@@ -343,24 +358,28 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
             ptx::prefetch_l1(p.col_scale + col_base + lane * 32);
         }
       }
-      const long long w0 = trace ? clock64() : 0;
-      ok = wait_bounded<true>(acc_full_bar, acc_phase, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE,
-                              (DBG && (ablate & 4)) ? 500u : 0u);
-      ok = __all_sync(0xffffffffu, ok);
-      const long long w1 = trace ? clock64() : 0;
-      if (trace) epi_wait += w1 - w0;
-      if (!ok) break;
-      ptx::tc_fence_after_sync();
-      if (p.wait_prior_grid && !prior_grid_done) {  // C may still be in use by the grid in front
-        ptx::grid_dep_wait();
-        prior_grid_done = true;
-      }
+      long long w1 = 0;
 #pragma unroll 1
       for (int a = 0; a < 2; ++a) {
         const int row0 = cta_row0 + a * BM + quarter * 32;
         const int row = row0 + lane;
         const float rs_a = a ? rs[1] : rs[0];
         const uint32_t t_acc = tmem_base + lane_base + static_cast<uint32_t>(a * WIDE_BN + half * 128);
+        const long long w0 = trace ? clock64() : 0;
+        ok = wait_bounded<true>(acc_full_bar(a), acc_phase, abort_flag, p.status, DEV_TIMEOUT_EPILOGUE,
+                                (DBG && (ablate & 4)) ? 500u : 0u);
+        ok = __all_sync(0xffffffffu, ok);
+        if (trace) {
+          const long long now = clock64();
+          epi_wait += now - w0;
+          if (a == 0) w1 = now;
+        }
+        if (!ok) break;
+        ptx::tc_fence_after_sync();
+        if (p.wait_prior_grid && !prior_grid_done) {  // C may still be in use by the grid in front
+          ptx::grid_dep_wait();
+          prior_grid_done = true;
+        }
         // This warp's whole share of the accumulator (its row x 128 columns) goes to registers
         // at once and the accumulator is handed back to the (leader's) MMA issuer before
         // anything is written out: with every CTA of the grid storing its tile at the same
@@ -435,6 +454,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
           }
         }
       }
+      if (!ok) break;
       if (trace) epi_busy += clock64() - w1;
       ++tiles_done;
       acc_phase ^= 1u;

@@ -153,11 +153,14 @@ int band_height(int M, int rows_per_tile, int bn, int units) {
 // 256 x 256 pair tile but a quarter fewer operand bytes from L2, which buys clock on a
 // power-capped part; its tiles are twice as large, so it needs enough of them to fill its waves.
 bool wide_wanted(const TileConfig& cfg, int M, int N, int num_sms, bool swap, bool csplit,
-                 bool packed_s4) {
+                 bool packed_s4, bool fp16_kind) {
   if (swap || csplit || packed_s4 || g_family == 1) return false;
   if (g_family == 2) return !(g_override_bn && g_override_bn != 256) && g_override_cta_group != 1 &&
                             g_override_splits <= 1;
-  if (cfg.bn != 256 || cfg.cta_group != 2 || cfg.splits != 1) return false;
+  // The integer kinds stay on the 256 x 256 tile: their tiles take half as long for the same C
+  // bytes, so the hand-over between tiles, which only this kernel exposes, weighs twice as much
+  // (N = 8192 INT8: 517 k against 499 k SM cycles, no gain in time).
+  if (!fp16_kind || cfg.bn != 256 || cfg.cta_group != 2 || cfg.splits != 1) return false;
   const long long tiles = static_cast<long long>(ceil_div(M, WIDE_TILE_M)) * ceil_div(N, WIDE_BN);
   const long long pairs = num_sms / 2;
   const long long waves = (tiles + pairs - 1) / pairs;
@@ -172,6 +175,21 @@ struct OutputSpec {
   long long ldc = 0;        // row pitch of C in elements; 0 = dense (N)
   bool no_split = false;    // C is a block of a larger matrix: never zero / add into it
 };
+
+// Overlapped INT4 pre-pass: A and B of the call are the (not yet written) int8 images in a
+// scratch buffer, these are the packed operands they are to be made from inside the GEMM
+// kernel, and `sync` its bookkeeping words (see s4_ahead.cuh).
+struct S4AheadReq {
+  const uint8_t* packed_a;
+  const uint8_t* packed_b;
+  uint32_t* sync;
+};
+
+// Returned (never to the caller of the library) when a call with an S4AheadReq is not one the
+// overlapped kernel takes: nothing has been enqueued, the caller runs the pre-pass launch.
+constexpr int GEMM_NOT_AHEAD = 2;
+
+thread_local int t_last_s4_overlapped = 0;
 
 // Index in attr_set of the unfused cluster split-K variants: 96.., by kind, output mode, width.
 template <int KIND, int EPI>
@@ -228,7 +246,7 @@ bool cluster_split_ok(const TileConfig& c, int M, int N) {
 // of pair tiles such as 2048^3, even or slower beyond).
 bool s4_fused_wanted(int M, int N, const TileConfig& cfg, int num_sms) {
   if (g_s4_scheme == 2) return true;
-  if (g_s4_scheme == 1) return false;
+  if (s4_prepass_forced()) return false;
   if (cfg.cta_group == 2) {  // (the 128-wide pair tile only comes in through select_fused_s4)
     const long long tiles = static_cast<long long>(ceil_div(M, 2 * BM)) * ceil_div(N, cfg.bn);
     return cfg.bn == 256 && tiles <= num_sms / 2;
@@ -251,7 +269,7 @@ bool s4_fused_wanted(int M, int N, const TileConfig& cfg, int num_sms) {
 // 640-1024 x 2048 x 8192 would lose 15-35 %, and from 1280 rows on the pre-pass is even or ahead.
 bool select_fused_s4(int M, int N, int user_m, int user_n, int num_sms, int k_blocks, int min_bn,
                      bool allow_split, const TileConfig& int8_choice, TileConfig* out) {
-  if (g_s4_scheme == 1) return false;
+  if (s4_prepass_forced()) return false;
   const TileConfig c = select_config(M, N, num_sms, k_blocks, min_bn, allow_split, 2);
   const auto pair_split_only_here = [&](const TileConfig& f) {
     return g_s4_scheme == 0 && f.cta_group == 2 && f.splits > 1 && int8_choice.splits == 1;
@@ -313,7 +331,7 @@ constexpr int GEMM_NOT_FUSED = 1;
 template <int KIND, int EPI>
 int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const void* B,
                     size_t b_pitch, void* C, const OutputSpec& out, cudaStream_t stream,
-                    bool packed_s4 = false) {
+                    bool packed_s4 = false, const S4AheadReq* req = nullptr) {
   DeviceState* s = nullptr;
   int rc = device_state(&s);
   if (rc != GEMM_OK) return rc;
@@ -371,7 +389,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     k_blocks = 2 * ceil_div(K, 2 * BK_BYTES);  // one packed slot (256 values of K) = two int8 slots
   }
 
-  const bool wide = wide_wanted(cfg, M, N, s->num_sms, swap, csplit, packed_s4);
+  const bool wide = wide_wanted(cfg, M, N, s->num_sms, swap, csplit, packed_s4, KIND == ptx::KIND_F16);
   if (wide) {
     cfg.bn = WIDE_BN;
     cfg.cta_group = 2;
@@ -380,6 +398,20 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     cfg.group_m = band_height(M, WIDE_TILE_M, WIDE_BN, s->num_sms / 2);
   }
   const int rows_per_cta = wide ? WIDE_CTA_ROWS : BM;
+  bool ahead = false;
+  if (req) {
+    // The overlapped pre-pass rides on the 256 x 256 pair-tile kernel of large problems: at
+    // least two waves of tiles, so that the expansion is done long before the GEMM is.  Only on
+    // request (scheme 4): measured, it loses to the separate launch -- that kernel already keeps
+    // the SM's L2 port and shared-memory pipe full, and the loads and stores of the expansion
+    // slow its mainloop by more than the pre-pass takes on its own (N = 8192: 574 k SM cycles
+    // against 496 k + a 36 us pre-pass).
+    const long long tiles = static_cast<long long>(ceil_div(M, 2 * BM)) * ceil_div(N, 256);
+    ahead = KIND == ptx::KIND_I8 && !wide && !swap && !csplit && !packed_s4 && cfg.bn == 256 &&
+            cfg.cta_group == 2 && cfg.stages == 6 && g_s4_scheme == 4 && (g_trace_on >> 1) == 0 &&
+            tiles >= 2 * (s->num_sms / 2);
+    if (!ahead) return GEMM_NOT_AHEAD;
+  }
   CUtensorMap ta, tb;
   const bool promote = !(g_l2_policy & 16);
   // packed: the tensor is K/2 bytes wide; boxes stay 128 bytes
@@ -434,6 +466,29 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   if (p.l2_policy == 3 && (p.tiles_n == 1 || p.tiles_m == 1)) p.l2_policy = 2;
   p.serpentine_k = (g_l2_policy & 4) ? 0 : 1;
   p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
+  p.ahead = S4Ahead();
+  if (ahead) {
+    p.ahead.packed_a = reinterpret_cast<const uint4*>(req->packed_a);
+    p.ahead.packed_b = reinterpret_cast<const uint4*>(req->packed_b);
+    p.ahead.a8 = static_cast<int8_t*>(const_cast<void*>(A));
+    p.ahead.b8 = static_cast<int8_t*>(const_cast<void*>(B));
+    p.ahead.sync = req->sync;
+    p.ahead.M = M;
+    p.ahead.N = N;
+    p.ahead.K = K;
+    S4AheadPlan& pl = p.ahead.plan;
+    pl.ra = ceil_div(M, S4A_CHUNK_ROWS);
+    pl.rb = ceil_div(N, S4A_CHUNK_ROWS);
+    pl.kc = ceil_div(K, S4A_CHUNK_COLS);
+    pl.ga = 2 * BM / S4A_CHUNK_ROWS;
+    pl.gb = 256 / S4A_CHUNK_ROWS;
+    // what the first wave of tiles reads: the first band's rows of A, and as many tile columns
+    // of B as one wave of CTA pairs covers in that band
+    const int band = p.group_m < p.tiles_m ? p.group_m : p.tiles_m;
+    const int first_cols = ceil_div(s->num_sms / 2, band);
+    pl.ra1 = band * pl.ga < pl.ra ? band * pl.ga : pl.ra;
+    pl.rb1 = first_cols * pl.gb < pl.rb ? first_cols * pl.gb : pl.rb;
+  }
 
   if (wide) return launch_wide<KIND, EPI>(s, ta, tb, p, stream);
   if (cfg.splits > 1 && !csplit) {  // only with a dense C (no_split is set for blocks of a larger matrix)
@@ -538,6 +593,14 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   if (cfg.cta_group == 2) {
     switch (cfg.bn) {
       case 256:
+        if constexpr (KIND == ptx::KIND_I8) {
+          if (ahead) {  // attr_set bits 224..
+            t_last_s4_overlapped = 1;
+            using L = SmemLayout<256, 6, 2, 1, 0, 1>;
+            return launch_kernel(s, gemm_kernel<KIND, 256, 6, 2, 1, EPI, 0, 1, false, true>, 224 + EPI,
+                                 L::DYN_BYTES, NUM_THREADS, 2, ta, tb, tc, p, stream);
+          }
+        }
         if constexpr (EPI == EPI_RAW32) {
           // ring depth as an ablation variable (gemm_set_stages_override); attr_set bits 216..
           const int sb = 216 + (KIND == ptx::KIND_F16 ? 0 : 4);
@@ -566,18 +629,18 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
 template <int KIND>
 int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* B, size_t b_pitch,
                 void* C, cudaStream_t stream, const OutputSpec& out = OutputSpec(),
-                bool packed_s4 = false) {
+                bool packed_s4 = false, const S4AheadReq* req = nullptr) {
   switch (out.epi) {
     case EPI_RAW32:
       return launch_gemm_epi<KIND, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream,
-                                              packed_s4);
+                                              packed_s4, req);
     case EPI_OUT16:
       return launch_gemm_epi<KIND, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream,
-                                              packed_s4);
+                                              packed_s4, req);
     case EPI_F32_SCALED:
       if constexpr (KIND == ptx::KIND_I8)
         return launch_gemm_epi<KIND, EPI_F32_SCALED>(M, N, K, A, a_pitch, B, b_pitch, C, out,
-                                                     stream, packed_s4);
+                                                     stream, packed_s4, req);
       return GEMM_ERR_INVALID_ARG;
     default: return GEMM_ERR_INVALID_ARG;
   }
@@ -626,15 +689,23 @@ size_t s4_workspace_need(int M, int N, int K) {
 }
 
 // INT4 GEMM through caller-visible scratch: unpack A and B to int8, then the INT8 kernel.
+// `sync`: bookkeeping words of the overlapped pre-pass in front of a pool buffer, or null
+// (caller-supplied scratch, whose surroundings the library knows nothing about).
 int s4_with_workspace(int M, int N, int K, const uint8_t* A, const uint8_t* B, void* C,
                       void* workspace, size_t workspace_bytes, const OutputSpec& out,
-                      cudaStream_t st) {
+                      cudaStream_t st, uint32_t* sync = nullptr) {
   if (!workspace) return GEMM_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < s4_workspace_need(M, N, K))
     return GEMM_ERR_WORKSPACE;
   int8_t* a8 = static_cast<int8_t*>(workspace);
   int8_t* b8 = a8 + align_up(static_cast<size_t>(M) * K, 256);
   int rc;
+  if (sync) {
+    const S4AheadReq req{A, B, sync};
+    rc = launch_gemm<ptx::KIND_I8>(M, N, K, a8, static_cast<size_t>(K), b8, static_cast<size_t>(K),
+                                   C, st, out, false, &req);
+    if (rc != GEMM_NOT_AHEAD) return rc;
+  }
   rc = launch_unpack(M, A, a8, N, B, b8, K, static_cast<size_t>(K), st);
   if (rc != GEMM_OK) return rc;
   return launch_gemm<ptx::KIND_I8>(M, N, K, a8, static_cast<size_t>(K), b8, static_cast<size_t>(K),
@@ -645,10 +716,8 @@ int s4_with_workspace(int M, int N, int K, const uint8_t* A, const uint8_t* B, v
 // flags of the overlapped pre-pass: one word per 32 rows x 512 columns of int8, both operands).
 size_t s4_head_bytes(int M, int N, int K) {
   const size_t flags = (static_cast<size_t>(ceil_div(M, 32)) + ceil_div(N, 32)) * ceil_div(K, 512);
-  return align_up(256 + 4 * flags, 256);
+  return align_up(4 * (S4A_SYNC_WORDS + flags), 256);
 }
-
-thread_local int t_last_s4_overlapped = 0;
 
 // INT4 GEMM by the route gemm_set_s4_scheme selected: the fused kernel if asked for and
 // applicable, else the pre-pass through a scratch buffer leased from the device's pool for
@@ -657,7 +726,7 @@ thread_local int t_last_s4_overlapped = 0;
 int s4_auto(int M, int N, int K, const uint8_t* A, const uint8_t* B, void* C, const OutputSpec& out,
             cudaStream_t st) {
   t_last_s4_overlapped = 0;
-  if (g_s4_scheme != 1) {
+  if (!s4_prepass_forced()) {
     const int rc = launch_gemm<ptx::KIND_I8>(M, N, K, A, static_cast<size_t>(K) / 2, B,
                                              static_cast<size_t>(K) / 2, C, st, out, true);
     if (rc != GEMM_NOT_FUSED) return rc;
@@ -670,7 +739,7 @@ int s4_auto(int M, int N, int K, const uint8_t* A, const uint8_t* B, void* C, co
   const int prc = g_pool[dev].acquire(st, s4_workspace_need(M, N, K), s4_head_bytes(M, N, K), &lease);
   if (prc != 0) return pool_fail(prc);
   rc = s4_with_workspace(M, N, K, A, B, C, static_cast<uint8_t*>(lease.ptr) + lease.head_bytes,
-                         lease.bytes, out, st);
+                         lease.bytes, out, st, static_cast<uint32_t*>(lease.ptr));
   const int qrc = g_pool[dev].release(lease, st);
   if (rc == GEMM_OK && qrc != 0) rc = pool_fail(qrc);
   return rc;
