@@ -263,6 +263,8 @@ def run_ours(args, rank, world):
         binding.gemm_set_config_override(*[int(x) for x in args.override.split(",")])
     if args.l2_policy >= 0:
         binding.gemm_set_l2_policy(args.l2_policy)
+    if args.family:
+        binding.gemm_set_kernel_family(args.family)
     N = args.size
     ops = synth.gemm_ops(N, N, N)
     stream = torch.cuda.current_stream()
@@ -926,6 +928,8 @@ def main():
                     help="precision x size sweep N=512..8192, one JSON line per cell (1 GPU)")
     ap.add_argument("--precisions", default="fp16,s8,s4")
     ap.add_argument("--l2-policy", type=int, default=-1, help="ablation: gemm_set_l2_policy")
+    ap.add_argument("--family", type=int, default=0,
+                    help="ablation: gemm_set_kernel_family (1 = 256x256 pair tile, 2 = 512x256)")
     ap.add_argument("--override", default="",
                     help="ablation: BN,GROUP_M,CTA_GROUP passed to gemm_set_config_override")
     args = ap.parse_args()

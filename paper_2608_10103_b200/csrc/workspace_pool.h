@@ -62,8 +62,9 @@ class WorkspacePool {
       Entry& e = entries_[i];
       if (!e.leased && e.stream == s && fits(e, need, head)) pick = static_cast<int>(i);
     }
-    // 2. a buffer nobody is using any more
-    for (size_t i = 0; i < entries_.size() && pick < 0; ++i) {
+    // 2. a buffer nobody is using any more (not asked during capture: querying an event is
+    //    not allowed then, and says nothing about when the captured work will run)
+    for (size_t i = 0; i < entries_.size() && pick < 0 && !cap; ++i) {
       Entry& e = entries_[i];
       if (!e.leased && !e.shared && fits(e, need, head) && backend_.event_done(e.event))
         pick = static_cast<int>(i);

@@ -19,6 +19,7 @@ struct FakeState {
   std::map<int, bool> event_done;                  // event id -> done
   std::set<int> capturing;
   int allocs = 0, clears = 0, next_event = 1;
+  bool queried_during_capture = false;
 };
 
 struct FakeBackend {
@@ -58,6 +59,7 @@ struct FakeBackend {
   }
   bool event_done(Event e) {
     std::lock_guard<std::mutex> l(st->m);
+    if (!st->capturing.empty()) st->queried_during_capture = true;  // not allowed in a capture
     return st->event_done[e];
   }
   bool capturing(Stream s) {
@@ -132,6 +134,7 @@ int main() {
   EXPECT(pool.acquire(7, 4000, 256, &g) == 0);
   EXPECT(st.allocs == allocs_before);
   EXPECT(pool.release(g, 7) == 0);
+  EXPECT(!st.queried_during_capture);
   // a shared buffer never moves to another stream through the "completed" rule
   for (auto& e : st.event_done) e.second = true;
   Pool::Lease k;

@@ -40,3 +40,15 @@ def test_reference_arm_other_ranks_exit_quietly():
                          timeout=600, cwd=ROOT, env=env)
     assert out.returncode == 0, out.stderr[-2000:]
     assert not [l for l in out.stdout.splitlines() if l.startswith("{")]
+
+
+def test_traffic_comes_from_the_capture_file_and_only_for_the_same_library_version():
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2608_10103_b200 import binding
+    version = binding.gemm_version()
+    total, source = bench.captured_traffic(8192, version)
+    assert total is not None and total > 2 * 8192 * 8192 * 2 + 4 * 8192 * 8192   # above the algorithmic bytes
+    assert "bench.py --capture" in source and "ncu" in source
+    assert bench.captured_traffic(8192, version + 1)[0] is None      # stale capture: no number
+    assert bench.captured_traffic(12345, version)[0] is None         # size never captured

@@ -15,7 +15,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 def test_bench_line_has_the_contract_keys():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--size", "2048",
-                          "--steps", "5", "--warmup", "3", "--e2e-steps", "2"],
+                          "--steps", "5", "--warmup", "3", "--e2e-steps", "2", "--sustain-seconds", "0.5"],
                          capture_output=True, text=True, timeout=900, cwd=ROOT)
     assert out.returncode == 0, out.stderr[-2000:]
     lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
@@ -30,6 +30,13 @@ def test_bench_line_has_the_contract_keys():
     r = d["roofline"]
     assert r["bound"] == "tensor" and r["unit"] == "TFLOP/s" and r["peak"] > 0
     assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
+    # the denominator follows the length of the timed region: a few milliseconds here
+    assert r["timed_region_s"] < 1.0 and r["peak"] == r["peak_burst"] and r["frac"] == r["frac_burst"]
+    assert r["frac_sustained"] is not None and r["peak_sustained"] > 0
+    assert r["traffic"] is None and r["algorithmic_bytes"] == 2 * 2048 * 2048 * 2 + 4 * 2048 * 2048
+    for p in ("fp16", "s8", "s4"):
+        sus = d["precisions"][p]["sustained"]
+        assert sus["seconds"] >= 0.5 and sus["value"] > 0 and sus["launches"] >= 5
     e = d["e2e"]
     assert e["value"] > 0 and e["h2d_bytes_per_step"] == 2 * 2048 * 2048 * 2
     assert e["d2h_bytes_per_step"] == 2048 * 2048 * 4 and e["value"] < d["value"]
