@@ -531,6 +531,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     __syncwarp();
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
+    // A grid launched to start early counts its 2 s wait limits only from the moment the grid
+    // in front has completed: no operand can arrive before the producer has passed the same
+    // point, and the time spent behind a long predecessor must not look like a stuck barrier.
+    if (p.wait_prior_grid) ptx::grid_dep_wait();
     if (leader) {  // whole warp walks the loops, the lane elected once issues (see producer)
       const bool elected = ptx::elect_one();
       constexpr uint32_t idesc = ptx::make_idesc<KIND>(TILE_M, BN);
@@ -649,6 +653,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     // chunk read at offset x.  Lane -> (row, chunk) is chosen so that each quarter-warp reads
     // and writes all 32 banks once.
     if constexpr (FUSED) {
+      if (p.wait_prior_grid) ptx::grid_dep_wait();  // wait limits count from the predecessor's end
       // With deep rings (the narrow tiles of problems with few rows) the eight warps work as
       // two groups on alternate packed slots: a slot's fixed costs -- three barrier waits, the
       // proxy fence, the arrives: ~700 of the ~1300 cycles a slot took -- then overlap.
@@ -767,7 +772,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     bool ok = true;
     long long epi_wait = 0, epi_busy = 0, tiles_done = 0;
     uint32_t staged_blocks = 0;  // blocks sent through the staging buffers so far
-    bool prior_grid_done = false;
+    // (see the MMA issuer: wait limits count from the end of the grid in front; also C, the
+    // scale factors and the INT4 scratch may still be in use by it)
+    if (p.wait_prior_grid) ptx::grid_dep_wait();
+    bool prior_grid_done = true;
     uint32_t ahead_epoch = 0;    // overlapped INT4 pre-pass: 0 = not read yet (epochs start at 1)
     bool ahead_more = AHEAD;     // ... chunks may be left to claim
     long long ahead_busy = 0;

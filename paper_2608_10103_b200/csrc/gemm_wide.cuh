@@ -204,6 +204,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
     __syncwarp();
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
+    if (p.wait_prior_grid) ptx::grid_dep_wait();  // wait limits count from the predecessor's end
     if (leader) {
       const bool elected = ptx::elect_one();
       constexpr uint32_t idesc = ptx::make_idesc<KIND>(2 * BM, WIDE_BN);
@@ -333,7 +334,10 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const size_t pitch = static_cast<size_t>(p.ldc) * C_ELEM;
     uint32_t acc_phase = 0;
     bool ok = true;
-    bool prior_grid_done = false;
+    // wait limits count from the end of the grid in front, which may also still use C and the
+    // scale factors
+    if (p.wait_prior_grid) ptx::grid_dep_wait();
+    bool prior_grid_done = true;
     long long epi_wait = 0, epi_busy = 0, tiles_done = 0;
     for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
       int tm, tn;
