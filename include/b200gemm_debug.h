@@ -57,8 +57,9 @@ int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k);
  * overlaps the next tile; 2 = the 512 x 256 tile per CTA pair wherever the
  * problem's layout allows it (plain orientation, no split-K), whose two
  * accumulators fill tensor memory and which moves a quarter fewer operand
- * bytes per unit of math.  The automatic rule takes 2 when its tiles fill at
- * least two waves of CTA pairs to 90 %.  The paper fixes one tiling for every
+ * bytes per unit of math.  The automatic rule takes 2 for FP16 inputs when its
+ * tiles fill at least two waves of CTA pairs to 90 % and K covers at least 96
+ * blocks of 128 bytes (K >= 6144).  The paper fixes one tiling for every
  * size (Sec. III-A); this is the corresponding ablation axis here.
  */
 int gemm_set_kernel_family(int family);
@@ -89,11 +90,12 @@ int gemm_set_kernel_family(int family);
  * the pre-pass; 2: fused wherever a fused variant is built (every one-CTA tile,
  * and the 256 x 256 and 256 x 128 CTA pairs), else the pre-pass.  4: the
  * pre-pass, but where the INT8 GEMM runs on the 256 x 256 CTA-pair tile over at
- * least two waves its own epilogue warps expand the operands inside that
- * kernel, chunk by chunk ahead of the tiles that read them (no separate launch;
- * measured slower than 1 -- N = 8192: 574 k SM cycles against 496 k plus a
- * 36 us pre-pass -- because that kernel already keeps the SM's L2 port and
- * shared-memory pipe full; kept as the ablation's third INT4 route).  3 = 1.
+ * least two waves, four extra warps per CTA of that kernel expand the operands
+ * inside it, chunk by chunk ahead of the tiles that read them (no separate
+ * launch; measured slower than 1 -- N = 8192: 573 k SM cycles against 495 k plus
+ * a 36 us pre-pass -- because that kernel already keeps the SM's L2 port and
+ * shared-memory pipe full and runs at ~60 % speed while the expansion is in
+ * progress; kept as the ablation's third INT4 route).  3 = 1.
  * gemm_s4_ws and gemm_s4_static always use the pre-pass launch.  Results are
  * identical, bit for bit.
  * gemm_query_config shows the route.  The paper has no counterpart; its Run 4

@@ -182,7 +182,7 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
     M = user_n;
     N = user_m;
   }
-  const bool wide = wide_wanted(c, M, N, num_sms, swap, false, fused, precision == GEMM_PREC_FP16);
+  const bool wide = wide_wanted(c, M, N, kb, num_sms, swap, false, fused, precision == GEMM_PREC_FP16);
   if (wide) {
     c.bn = WIDE_BN;
     c.cta_group = 2;

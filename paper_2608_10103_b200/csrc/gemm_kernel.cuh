@@ -60,6 +60,8 @@ constexpr int NUM_THREADS = 192;  // 6 warps: producer, MMA, 4 x epilogue
 constexpr int EPI_WARPS = 4;
 constexpr int UNPACK_WARPS = 8;   // fused INT4 only: warps 6..13
 constexpr int NUM_THREADS_FUSED = NUM_THREADS + 32 * UNPACK_WARPS;
+constexpr int AHEAD_WARPS = 4;    // overlapped INT4 pre-pass only: warps 6..9
+constexpr int NUM_THREADS_AHEAD = NUM_THREADS + 32 * AHEAD_WARPS;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // every barrier wait gives up after 2 s
 
 // Device status codes written to the status word when a wait gives up.
@@ -243,7 +245,7 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
 // instantiations leave them out of their loops).
 template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32, int PSTAGES = 0,
           int CSPLIT = 1, bool DBG = false, bool AHEAD = false>
-__global__ void __launch_bounds__(PSTAGES > 0 ? NUM_THREADS_FUSED : NUM_THREADS, 1)
+__global__ void __launch_bounds__(PSTAGES > 0 ? NUM_THREADS_FUSED : (AHEAD ? NUM_THREADS_AHEAD : NUM_THREADS), 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
   using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, CSPLIT>;
@@ -643,6 +645,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       }
     }
     __syncwarp();
+  } else if (AHEAD && warp >= 2 + EPI_WARPS) {
+    // ------------------------------------- overlapped INT4 pre-pass: int8 chunks for the tiles to come
+    // Warps of their own: a chunk takes thousands of cycles inside a busy GEMM (its loads and
+    // stores queue behind the operand tiles), and a warp with another duty -- an epilogue that
+    // became due meanwhile -- would be late for it by that much.
+    if constexpr (AHEAD) {
+      if (p.wait_prior_grid) ptx::grid_dep_wait();  // the scratch may be in use by the grid in front
+      const uint32_t epoch = s4a_epoch(p.ahead);
+      const long long u0 = trace ? clock64() : 0;
+      s4a_work(p.ahead, epoch, lane, [&]() { return *abort_flag != 0; });
+      if (trace && warp == 2 + EPI_WARPS && lane == 0)
+        trace[TRACE_UNPACK_BUSY] = static_cast<unsigned long long>(clock64() - u0);
+    }
+    __syncwarp();
   } else if (FUSED && warp >= 2 + EPI_WARPS) {
     // ------------------------------------------------- fused INT4: nibble expansion
     // One packed slot holds, per operand row, 128 bytes = 8 chunks of 16 bytes (32 values of K
@@ -776,9 +792,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     // scale factors and the INT4 scratch may still be in use by it)
     if (p.wait_prior_grid) ptx::grid_dep_wait();
     bool prior_grid_done = true;
-    uint32_t ahead_epoch = 0;    // overlapped INT4 pre-pass: 0 = not read yet (epochs start at 1)
-    bool ahead_more = AHEAD;     // ... chunks may be left to claim
-    long long ahead_busy = 0;
     uint32_t xphase = 0;         // cluster split-K: parity of the partial-sum hand-over
     const bool xpeer = CSPLIT > 1 && krank != 0;  // this CTA only contributes partial sums
     // Cluster split-K, rank 0: adds the other CTAs' partial sums for accumulator columns
@@ -831,21 +844,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           if (p.row_scale && row < p.M) rs = __ldg(p.row_scale + row);
           if (p.col_scale && lane * 32 < BN && col0 + lane * 32 < p.N)
             ptx::prefetch_l1(p.col_scale + col0 + lane * 32);
-        }
-      }
-      if constexpr (AHEAD) {
-        // while the accumulator is not ready: expand packed INT4 chunks for the tiles to come
-        if (ahead_more) {
-          if (p.wait_prior_grid && !prior_grid_done) {  // the scratch may be in use by the grid in front
-            ptx::grid_dep_wait();
-            prior_grid_done = true;
-          }
-          if (ahead_epoch == 0) ahead_epoch = s4a_epoch(p.ahead);
-          const long long u0 = trace ? clock64() : 0;
-          ahead_more = s4a_work(p.ahead, ahead_epoch, lane, [&]() {
-            return __any_sync(0xffffffffu, ptx::mbar_test_wait(acc_full_bar(acc), acc_phase));
-          });
-          if (trace) ahead_busy += clock64() - u0;
         }
       }
       const long long w0 = trace ? clock64() : 0;
@@ -1064,17 +1062,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
-    if constexpr (AHEAD) {
-      // no tile left for this CTA, but the list may not be exhausted: other CTAs' tiles wait
-      // for these chunks
-      if (ok && ahead_more) {
-        if (ahead_epoch == 0) {
-          if (p.wait_prior_grid && !prior_grid_done) ptx::grid_dep_wait();
-          ahead_epoch = s4a_epoch(p.ahead);
-        }
-        s4a_work(p.ahead, ahead_epoch, lane, []() { return false; });
-      }
-    }
     // C stores still in flight read this CTA's shared memory: wait until they have read it
     // (their global writes complete on their own before the grid counts as finished).  A
     // hand-over copy into rank 0's shared memory has to have landed as well.
@@ -1087,7 +1074,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       trace[TRACE_EPI_WAIT] = static_cast<unsigned long long>(epi_wait);
       trace[TRACE_EPI_BUSY] = static_cast<unsigned long long>(epi_busy);
       trace[TRACE_TILES] = static_cast<unsigned long long>(tiles_done);
-      if (AHEAD) trace[TRACE_UNPACK_BUSY] = static_cast<unsigned long long>(ahead_busy);
     }
   }
 

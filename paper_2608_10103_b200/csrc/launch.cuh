@@ -152,8 +152,8 @@ int band_height(int M, int rows_per_tile, int bn, int units) {
 // Whether a problem goes to the 512 x 256 kernel.  It needs the same number of SM cycles as the
 // 256 x 256 pair tile but a quarter fewer operand bytes from L2, which buys clock on a
 // power-capped part; its tiles are twice as large, so it needs enough of them to fill its waves.
-bool wide_wanted(const TileConfig& cfg, int M, int N, int num_sms, bool swap, bool csplit,
-                 bool packed_s4, bool fp16_kind) {
+bool wide_wanted(const TileConfig& cfg, int M, int N, int k_blocks, int num_sms, bool swap,
+                 bool csplit, bool packed_s4, bool fp16_kind) {
   if (swap || csplit || packed_s4 || g_family == 1) return false;
   if (g_family == 2) return !(g_override_bn && g_override_bn != 256) && g_override_cta_group != 1 &&
                             g_override_splits <= 1;
@@ -164,7 +164,10 @@ bool wide_wanted(const TileConfig& cfg, int M, int N, int num_sms, bool swap, bo
   const long long tiles = static_cast<long long>(ceil_div(M, WIDE_TILE_M)) * ceil_div(N, WIDE_BN);
   const long long pairs = num_sms / 2;
   const long long waves = (tiles + pairs - 1) / pairs;
-  return tiles >= 2 * pairs && 10 * tiles >= 9 * waves * pairs;  // waves at least 90 % full
+  // at least two waves, at least 90 % full, and tiles long enough that the hand-over between
+  // them (~4.5 k cycles per tile that the 256 x 256 kernel does not have) stays small: measured
+  // +3 % at K = 8192, +2 % at 6144, even at 4096, -2 % at 2048 (FP16, 8192 x 8192 outputs)
+  return tiles >= 2 * pairs && 10 * tiles >= 9 * waves * pairs && k_blocks >= 96;
 }
 
 // Output options of one GEMM call.
@@ -389,7 +392,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     k_blocks = 2 * ceil_div(K, 2 * BK_BYTES);  // one packed slot (256 values of K) = two int8 slots
   }
 
-  const bool wide = wide_wanted(cfg, M, N, s->num_sms, swap, csplit, packed_s4, KIND == ptx::KIND_F16);
+  const bool wide = wide_wanted(cfg, M, N, k_blocks, s->num_sms, swap, csplit, packed_s4, KIND == ptx::KIND_F16);
   if (wide) {
     cfg.bn = WIDE_BN;
     cfg.cta_group = 2;
@@ -397,15 +400,17 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     cfg.split_tiles = 0;
     cfg.group_m = band_height(M, WIDE_TILE_M, WIDE_BN, s->num_sms / 2);
   }
-  const int rows_per_cta = wide ? WIDE_CTA_ROWS : BM;
   bool ahead = false;
+  const int rows_per_cta = wide ? WIDE_CTA_ROWS : BM;
   if (req) {
     // The overlapped pre-pass rides on the 256 x 256 pair-tile kernel of large problems: at
     // least two waves of tiles, so that the expansion is done long before the GEMM is.  Only on
-    // request (scheme 4): measured, it loses to the separate launch -- that kernel already keeps
-    // the SM's L2 port and shared-memory pipe full, and the loads and stores of the expansion
-    // slow its mainloop by more than the pre-pass takes on its own (N = 8192: 574 k SM cycles
-    // against 496 k + a 36 us pre-pass).
+    // request (scheme 4): measured, it loses to the separate launch.  While the four pre-pass
+    // warps per CTA are at work (the first ~130 k cycles at N = 8192) the GEMM's mainloop runs at
+    // ~60 % of its speed -- that kernel keeps the SM's L2 port and shared-memory pipe full with
+    // operand tiles already -- and the first wave starts a batch of chunks late: 573 k SM cycles
+    // against 495 k + a 36 us (~50 k cycle) pre-pass.  The same role inside the 512 x 256 kernel,
+    // whose L2 port has a quarter to spare, measured no better (596 k against ~520 k).
     const long long tiles = static_cast<long long>(ceil_div(M, 2 * BM)) * ceil_div(N, 256);
     ahead = KIND == ptx::KIND_I8 && !wide && !swap && !csplit && !packed_s4 && cfg.bn == 256 &&
             cfg.cta_group == 2 && cfg.stages == 6 && g_s4_scheme == 4 && (g_trace_on >> 1) == 0 &&
@@ -598,7 +603,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
             t_last_s4_overlapped = 1;
             using L = SmemLayout<256, 6, 2, 1, 0, 1>;
             return launch_kernel(s, gemm_kernel<KIND, 256, 6, 2, 1, EPI, 0, 1, false, true>, 224 + EPI,
-                                 L::DYN_BYTES, NUM_THREADS, 2, ta, tb, tc, p, stream);
+                                 L::DYN_BYTES, NUM_THREADS_AHEAD, 2, ta, tb, tc, p, stream);
           }
         }
         if constexpr (EPI == EPI_RAW32) {

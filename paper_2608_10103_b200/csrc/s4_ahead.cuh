@@ -1,10 +1,10 @@
 // Device side of the overlapped INT4 pre-pass (work list: s4_ahead.h).
 //
-// The GEMM kernel that multiplies the int8 images of A and B also produces them: while its
-// epilogue warps wait for an accumulator they claim chunks (32 rows x 512 columns) of the work
-// list, expand the packed nibbles to sign-extended int8 (the paper's s4 operand format,
-// Listing 2c, which tcgen05 cannot take directly) and publish each chunk with a flag; the TMA
-// producer looks at the flags behind a box before it loads it.  Claims are dynamic, so a
+// The GEMM kernel that multiplies the int8 images of A and B also produces them: four warps of
+// their own per CTA claim chunks (32 rows x 512 columns) of the work list, expand the packed
+// nibbles to sign-extended int8 (the paper's s4 operand format, Listing 2c, which tcgen05 cannot
+// take directly) and publish each chunk with a flag; the TMA producer looks at the flags behind
+// a box before it loads it.  Claims are dynamic, so a
 // claimed chunk always belongs to a warp that is running and waits for nothing, and every
 // wait on a flag is bounded like the kernel's other waits.
 //
@@ -93,22 +93,23 @@ __device__ __forceinline__ S4AChunkRef s4a_chunk_ref(const S4Ahead& ah, int i, i
 // atomic takes a thousand cycles and more to come back (the SM's L2 port is full of operand
 // tiles), so a warp keeps all 32 loads of two chunks in flight and pays the round trips of
 // claiming, draining its stores and publishing once per pair.
-template <class Stop>
+template <int CHUNKS = 2, class Stop>
 __device__ __forceinline__ bool s4a_work(const S4Ahead& ah, uint32_t epoch, int lane, Stop stop) {
+  static_assert(CHUNKS == 1 || CHUNKS == 2, "one or two chunks in flight per warp");
   const int total = s4a_total(ah.plan);
   const int row_u4 = ah.K / 32;
   while (!stop()) {
     int i = 0;
-    if (lane == 0) i = static_cast<int>(atomicAdd(ah.sync + S4A_CLAIM, 2u));
+    if (lane == 0) i = static_cast<int>(atomicAdd(ah.sync + S4A_CLAIM, static_cast<uint32_t>(CHUNKS)));
     i = __shfl_sync(0xffffffffu, i, 0);
     if (i >= total) return false;
-    const int n = (i + 1 < total) ? 2 : 1;
-    S4AChunkRef ref[2];
+    const int n = (CHUNKS == 2 && i + 1 < total) ? 2 : 1;
+    S4AChunkRef ref[CHUNKS];
     ref[0] = s4a_chunk_ref(ah, i, lane);
-    ref[1] = s4a_chunk_ref(ah, n == 2 ? i + 1 : i, lane);
-    uint4 w[2][16];
+    if constexpr (CHUNKS == 2) ref[1] = s4a_chunk_ref(ah, n == 2 ? i + 1 : i, lane);
+    uint4 w[CHUNKS][16];
 #pragma unroll
-    for (int c = 0; c < 2; ++c) {
+    for (int c = 0; c < CHUNKS; ++c) {
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
         if (c < n && ref[c].col_ok && ref[c].row0 + 2 * j < ref[c].rows)
@@ -116,7 +117,7 @@ __device__ __forceinline__ bool s4a_work(const S4Ahead& ah, uint32_t epoch, int 
       }
     }
 #pragma unroll
-    for (int c = 0; c < 2; ++c) {
+    for (int c = 0; c < CHUNKS; ++c) {
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
         if (c < n && ref[c].col_ok && ref[c].row0 + 2 * j < ref[c].rows) {

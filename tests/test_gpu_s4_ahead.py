@@ -1,6 +1,6 @@
 """GPU parity of the overlapped INT4 pre-pass (gemm_set_s4_scheme(4), a measured alternative to
-the separate pre-pass launch): the INT8 kernel's own epilogue warps expand the packed operands
-into the int8 scratch, chunk by chunk, just ahead of the tiles that read them (ready flags,
+the separate pre-pass launch): four extra warps per CTA of the INT8 kernel expand the packed
+operands into the int8 scratch, chunk by chunk, just ahead of the tiles that read them (ready flags,
 dynamic claims, an epoch per call).  Everything through the C-ABI (gemm_s4 / gemm_s4_dequant)
 against the oracle, bit for bit."""
 import numpy as np
@@ -151,3 +151,4 @@ def test_overlapped_dequant(out_dtype):
     ref = oracle.dequant_ref(oracle.gemm_s4_i64(A, B, K, rows=rows), rs[rows], cs)
     ok, worst = oracle.dequant_check(C.cpu().numpy()[rows], ref, out_dtype == torch.float16)
     assert ok, "error %.3g x bound" % worst
+
