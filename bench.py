@@ -797,6 +797,7 @@ def run_ablation(args):
                  V("ablate: no loads (MMAs + barriers only)", trace=5),
                  V("epilogue waits with nanosleep back-off", trace=9),
                  V("epilogue: direct register -> global stores", trace=33),
+                 V("epilogue: 16x256b TMEM loads, sector-complete direct stores (no staging)", trace=65),
                  V("512x256 tile, ablate: no MMAs", trace=3, family=2),
                  V("512x256 tile, ablate: no loads", trace=5, family=2)]
     # INT4: how the nibbles reach the int8 tensor-core path (the traced launch is the GEMM; a
@@ -856,7 +857,7 @@ def run_ablation(args):
                     "producer_wait": float(a["producer_wait"].mean() / kb_total),
                     "producer_issue": float(a["producer_issue"].mean() / kb_total)},
                 "epilogue_busy_frac": float(a["epilogue_busy"].mean() / a["cycles"].mean()),
-                "result_valid": trace in (1, 9, 33), **unpack}), flush=True)
+                "result_valid": trace in (1, 9, 33, 65), **unpack}), flush=True)
     binding.gemm_set_s4_scheme(0)
     binding.gemm_set_kernel_family(0)
     binding.gemm_set_stages_override(0)

@@ -178,7 +178,13 @@ int gemm_set_l2_policy(int policy);
  * record a code for gemm_last_device_status, drain and return -- the call takes
  * a few seconds, C is garbage and the context stays usable; 32 = the epilogue
  * writes C straight from registers (16 bytes per thread and store) instead of
- * staging it in shared memory for TMA stores (results unchanged).  With bit 2, 4 or
+ * staging it in shared memory for TMA stores (results unchanged); 64 = the
+ * epilogue of the 128/256-row kernels reads the accumulator in the 16x256b shape,
+ * in which four neighbouring threads hold 32 contiguous bytes of a row, and
+ * stores whole 32-byte sectors straight to C: no staging, no shared-memory
+ * traffic beside the mainloop's (raw outputs with rows of whole 32-byte sectors;
+ * results unchanged; 2-4 % fewer SM cycles at N = 8192 and the same time, the
+ * part being power-capped).  With bit 2, 4 or
  * 16 set C is garbage; 2 and 4 exist to attribute cycles to the load path or
  * the MMA path.
  */

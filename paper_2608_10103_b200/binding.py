@@ -365,7 +365,7 @@ def gemm_trace_enable(flags: int = 1):
     """1 = record cycles; +2 = issue no MMAs; +4 = issue no operand loads; +8 = epilogue
     waits back off with nanosleep; +16 = failure drill (a slot is never filled: the bounded
     waits expire and the kernel reports it); +32 = epilogue stores C straight from registers;
-    0 = off."""
+    +64 = epilogue reads TMEM in the 16x256b shape and stores whole 32-byte sectors; 0 = off."""
     _check(lib().gemm_trace_enable(int(flags)), "gemm_trace_enable")
 
 

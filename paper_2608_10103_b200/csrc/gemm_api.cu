@@ -310,7 +310,7 @@ int gemm_trace_enable(int on) {
       e = cudaMemset(s->trace_ptr, 0, sizeof(unsigned long long) * TRACE_SLOTS * TRACE_MAX_CTAS);
     if (e != cudaSuccess) return cuda_fail(e);
   }
-  g_trace_on = on & 63;
+  g_trace_on = on & 127;
   return GEMM_OK;
 }
 

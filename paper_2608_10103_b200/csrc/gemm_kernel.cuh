@@ -123,13 +123,14 @@ struct GemmParams {
   int serpentine_k;
   // Ablation switches for cycle accounting runs (results are then meaningless):
   // bit 0 = issue no MMAs (loads + barriers only), bit 1 = issue no loads (MMAs + barriers only),
-  // bit 4 = epilogue stores C straight from registers (no staging, no TMA store),
+  // bit 4 = epilogue stores C straight from registers (no staging, no TMA store), bit 5 = the
+  // same from the 16x256b TMEM load shape, whole 32-byte sectors per four threads,
   // bit 2 = epilogue waits back off with nanosleep, bit 3 = host-requested failure drill: the
   // producer of CTA 0 leaves out the 3rd ring slot of its first tile, so the consumers' bounded
   // waits must expire, record a status code and let the kernel drain and return.
   int ablate;
   // Overlapped INT4 pre-pass (kernel variants built with AHEAD): the int8 operands this GEMM
-  // reads are produced by its own epilogue warps from the packed ones named here.
+  // reads are produced by four extra warps of its own CTAs from the packed ones named here.
   S4Ahead ahead;
 };
 
@@ -914,6 +915,33 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       for (int c = 0; c < BN / BLOCK_COLS && !xpeer; ++c) {
         const int col = col0 + c * BLOCK_COLS;
         uint32_t w[32];  // the thread's 128 bytes of output
+        if constexpr (EPI == EPI_RAW32 && CSPLIT == 1) {
+          if (DBG && (ablate & 32) && p.c_vec_ok && p.ldc % 8 == 0 && !add) {
+            // ablation: no staging at all -- read the block in the 16x256b shape, in which four
+            // neighbouring threads hold 32 contiguous bytes of a row, and store those straight
+            // to C: whole 32-byte sectors, no shared-memory traffic beside the mainloop's
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              uint32_t r16[16];
+              ptx::tmem_ld_16x256b_x4(tmem_base + lane_base + (static_cast<uint32_t>(h * 16) << 16) +
+                                          static_cast<uint32_t>(acc * BN + c * 32),
+                                      r16);
+              ptx::tmem_wait_ld();
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int cj = col + 8 * j + 2 * (lane & 3);
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                  const int rr = row0 + 16 * h + 8 * u + (lane >> 2);
+                  if (rr < p.M && cj < p.N && !empty_range)
+                    ptx::st_global_v2_hint(p.C + static_cast<size_t>(rr) * p.ldc + cj,
+                                           fix(r16[4 * j + 2 * u]), fix(r16[4 * j + 2 * u + 1]), pol_c);
+                }
+              }
+            }
+            continue;
+          }
+        }
         if constexpr (EPI == EPI_RAW32) {
           ptx::tmem_ld_32x32b_x32(
               tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), w);

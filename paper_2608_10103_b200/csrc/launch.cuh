@@ -461,7 +461,7 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.col_scale = swap ? out.row_scale : out.col_scale;
   p.status = s->status_ptr;
   p.trace = (g_trace_on & 1) ? s->trace_ptr : nullptr;
-  p.ablate = (g_trace_on >> 1) & 31;
+  p.ablate = (g_trace_on >> 1) & 63;
   p.l2_policy = g_l2_policy & 3;
   // Default policy, one tile column or one tile row (problems with few rows on one side): the
   // short operand, which every CTA re-reads, gets the same priority in L2 as the long one that

@@ -363,6 +363,27 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)
       : "memory");
 }
 
+// TMEM -> registers, shape 16x256b, four column groups: the warp reads 16 lanes (rows) x 32
+// consecutive 32-bit columns.  Thread t gets, for column group j (8 columns each), registers
+// 4j, 4j+1 = row t/4, columns 8j + 2(t%4) + {0,1} and 4j+2, 4j+3 = row t/4 + 8, same columns:
+// four neighbouring threads hold 32 contiguous bytes of one row.
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+__device__ __forceinline__ void st_global_v2_hint(void* p, uint32_t a, uint32_t b, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.v2.b32 [%0], {%1, %2}, %3;" ::"l"(p), "r"(a), "r"(b),
+               "l"(policy)
+               : "memory");
+}
+
 // Programmatic dependent launch.  launch_dependents: the next kernel in the stream, if it was
 // launched with the programmatic-serialization attribute, may start now instead of when this
 // grid has drained.  wait: blocks the calling thread until the grids this one depends on have

@@ -332,3 +332,26 @@ def test_cluster_split_k_and_fused_int4_share_the_gpu_from_two_streams():
     for C8, C4 in zip(outs8, outs4):
         assert oracle.dequant_check(C8.cpu().numpy(), ref8, True)[0]
         assert np.array_equal(C4.cpu().numpy(), ref4)
+
+
+@pytest.mark.parametrize("prec", ["fp16", "s8"])
+@pytest.mark.parametrize("cta_group", [1, 2])
+def test_sector_store_epilogue_switch_gives_the_same_results(prec, cta_group):
+    """Measurement switch 64: accumulators read in the 16x256b shape and stored as whole 32-byte
+    sectors, no staging.  Ragged in M, N a multiple of 8 (rows of whole sectors), several tiles."""
+    M, N, K = 700, 1032, 512
+    A, B = synth.make(prec, M, N, K, seed=5)
+    binding.gemm_set_config_override(256, 0, cta_group, 1)
+    try:
+        binding.gemm_trace_enable(64)
+        C = torch.full((M, N), -7, dtype=torch.float32 if prec == "fp16" else torch.int32, device="cuda")
+        binding.gemm(prec, to_dev(A), to_dev(B), C)
+        torch.cuda.synchronize()
+    finally:
+        binding.gemm_trace_enable(0)
+    got = C.cpu().numpy()
+    if prec == "s8":
+        assert np.array_equal(got, oracle.gemm_s8(A, B))
+    else:
+        ref, S = oracle.gemm_fp16(A, B)
+        assert oracle.fp16_check(got, ref, S)[0]
