@@ -589,6 +589,9 @@ def run_sweep(args):
                 fn(*c_args)
             host_us_c = (time.perf_counter() - t0) / 200 * 1e6
             torch.cuda.synchronize()
+            # ... and without that dispatch: the same 200 calls looped and timed inside the library
+            host_us_native = min(binding.gemm_debug_host_cost(prec, dA, dB, C, stream, 200)
+                                 for _ in range(3)) * 1e-3
             reps = max(5, min(100, int(20.0 / max(timed(lambda: call(stream), 5), 1e-3))))
             g_many, g_one = graph_of(call, reps), graph_of(call, 1)
             warm = float(np.median([timed(g_many.replay, 1) for _ in range(5)])) / reps
@@ -600,6 +603,7 @@ def run_sweep(args):
                 "sweep": True, "precision": prec, "N": N, "seed": synth.sweep_seed(prec, N),
                 "ms": warm, "reps": reps, "ms_cold_single_launch": cold,
                 "host_us_per_call": host_us, "host_us_c_abi": host_us_c,
+                "host_us_in_library": host_us_native,
                 "value": rate, "unit": UNIT[prec], "frac_of_spec_peak": rate / SPEC_PEAK[prec],
                 "frac_of_cublas_bf16_burst_scaled": rate / ref,
                 "frac_of_mma_only_peak": rate / mma_peak[prec], "mma_only_peak": mma_peak[prec],

@@ -208,6 +208,19 @@ int gemm_set_stages_override(int stages);
  */
 int gemm_debug_counters(long long* out, int n);
 
+/*
+ * Host time of one call of gemm_fp16 / gemm_s8 / gemm_s4 (precision = GEMM_PREC_*), measured
+ * inside the library so that no foreign-function dispatch is in it: synchronises `stream`,
+ * enqueues `calls` (1..512, below the depth of the launch queue, so that the device never
+ * holds the host back) identical calls back to back, and writes the wall time of that loop
+ * divided by `calls`, in nanoseconds, to *ns_per_call.  The calls are real: C is written.
+ * Returns the first non-zero code of a call, else 0.  A measurement aid (the paper does not
+ * discuss host cost; its sizes start at 512, where a call is a few microseconds on the device
+ * and the enqueue rate of the host bounds a stream of them).
+ */
+int gemm_debug_host_cost(int precision, int M, int N, int K, const void* A, const void* B, void* C,
+                         gemm_stream_t stream, int calls, double* ns_per_call);
+
 #ifdef __cplusplus
 }
 #endif

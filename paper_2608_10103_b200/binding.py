@@ -23,7 +23,7 @@ EXPORTS = (
     "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
     "gemm_fp16_f16out", "gemm_s8_dequant", "gemm_s4_dequant", "gemm_host", "gemm_host_release",
     "gemm_s4_static", "gemm_s4_static_capacity", "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
-    "gemm_set_config_override", "gemm_set_kernel_family", "gemm_set_s4_scheme", "gemm_set_swap_ab", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_set_stages_override", "gemm_debug_counters",
+    "gemm_set_config_override", "gemm_set_kernel_family", "gemm_set_s4_scheme", "gemm_set_swap_ab", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_set_stages_override", "gemm_debug_counters", "gemm_debug_host_cost",
     "gemm_last_device_status", "gemm_read_device_status", "gemm_last_cuda_error",
     "gemm_status_string", "gemm_version",
 )
@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
         L.gemm_set_kernel_family.argtypes = [i]
         L.gemm_set_stages_override.argtypes = [i]
         L.gemm_debug_counters.argtypes = [ctypes.POINTER(ctypes.c_longlong), i]
+        L.gemm_debug_host_cost.argtypes = [i, i, i, i, vp, vp, vp, vp, i, ctypes.POINTER(ctypes.c_double)]
         L.gemm_read_device_status.argtypes = [vp, vp]
         L.gemm_set_swap_ab.argtypes = [i]
         L.gemm_set_l2_policy.argtypes = [i]
@@ -323,6 +324,19 @@ def gemm_debug_counters() -> dict:
     buf = (ctypes.c_longlong * 3)()
     _check(lib().gemm_debug_counters(buf, 3), "gemm_debug_counters")
     return {"map_encodes": int(buf[0]), "pool_buffers": int(buf[1]), "s4_overlapped": int(buf[2])}
+
+
+def gemm_debug_host_cost(precision: str, A: torch.Tensor, B: torch.Tensor, C: torch.Tensor,
+                         stream=None, calls: int = 200) -> float:
+    """Host nanoseconds per call of gemm_fp16 / gemm_s8 / gemm_s4 on these device tensors,
+    timed inside the library over `calls` (<= 512) back-to-back calls after a stream sync."""
+    M, N = A.shape[0], B.shape[0]
+    K = A.shape[1] * (2 if precision == "s4" else 1)
+    out = ctypes.c_double(0.0)
+    _check(lib().gemm_debug_host_cost(PRECISION_ID[precision], M, N, K, A.data_ptr(), B.data_ptr(),
+                                      C.data_ptr(), _stream_handle(stream), int(calls),
+                                      ctypes.byref(out)), "gemm_debug_host_cost")
+    return float(out.value)
 
 
 def gemm_read_device_status(host_out: torch.Tensor, stream=None):

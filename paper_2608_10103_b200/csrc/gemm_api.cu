@@ -9,6 +9,7 @@
 
 #include <mutex>
 
+#include <chrono>
 #include "../../include/b200gemm.h"
 #include "gemm_kernel.cuh"
 #include "launch.cuh"
@@ -285,6 +286,34 @@ int gemm_debug_counters(long long* out, int n) {
   const long long v[3] = {g_map_encodes.load(), static_cast<long long>(g_pool[dev].buffers()),
                           t_last_s4_overlapped};
   for (int i = 0; i < n; ++i) out[i] = i < 3 ? v[i] : 0;
+  return GEMM_OK;
+}
+
+int gemm_debug_host_cost(int precision, int M, int N, int K, const void* A, const void* B, void* C,
+                         gemm_stream_t stream, int calls, double* ns_per_call) {
+  if (!ns_per_call || calls < 1 || calls > 512) return GEMM_ERR_INVALID_ARG;
+  if (precision != GEMM_PREC_FP16 && precision != GEMM_PREC_S8 && precision != GEMM_PREC_S4)
+    return GEMM_ERR_INVALID_ARG;
+  auto one = [&]() {
+    switch (precision) {
+      case GEMM_PREC_FP16: return gemm_fp16(M, N, K, A, B, static_cast<float*>(C), stream);
+      case GEMM_PREC_S8:
+        return gemm_s8(M, N, K, static_cast<const int8_t*>(A), static_cast<const int8_t*>(B),
+                       static_cast<int32_t*>(C), stream);
+      default:
+        return gemm_s4(M, N, K, static_cast<const uint8_t*>(A), static_cast<const uint8_t*>(B),
+                       static_cast<int32_t*>(C), stream);
+    }
+  };
+  cudaError_t e = cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e);
+  const auto t0 = std::chrono::steady_clock::now();
+  for (int i = 0; i < calls; ++i) {
+    const int rc = one();
+    if (rc != GEMM_OK) return rc;
+  }
+  const auto t1 = std::chrono::steady_clock::now();
+  *ns_per_call = std::chrono::duration<double, std::nano>(t1 - t0).count() / calls;
   return GEMM_OK;
 }
 

@@ -116,3 +116,20 @@ def test_release_workspaces_empties_the_pool_and_calls_still_work():
     finally:
         binding.gemm_set_s4_scheme(0)
     assert np.array_equal(C.cpu().numpy(), oracle.gemm_s4(A, B, K))
+
+
+def test_host_cost_probe_runs_real_calls_and_rejects_bad_arguments():
+    """gemm_debug_host_cost loops the product entry point: C holds the result afterwards, the
+    figure is a plausible enqueue time, and counts outside 1..512 are refused."""
+    M, N, K = 256, 384, 512
+    A, B = synth.make("s8", M, N, K, seed=11)
+    dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    C = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    ns = binding.gemm_debug_host_cost("s8", dA, dB, C, calls=50)
+    torch.cuda.synchronize()
+    assert np.array_equal(C.cpu().numpy(), oracle.gemm_s8(A, B))
+    assert 200.0 < ns < 200000.0
+    for calls in (0, 513):
+        with pytest.raises(binding.GemmError) as e:
+            binding.gemm_debug_host_cost("s8", dA, dB, C, calls=calls)
+        assert e.value.code == -1
