@@ -872,6 +872,78 @@ def run_ablation(args):
         raise SystemExit("bench.py: a kernel reported a barrier timeout")
 
 
+def run_library_compare(args):
+    """Measurement only (no library kernel is on the product path): this library against the
+    vendor GEMM that PyTorch calls (cuBLAS / cuBLASLt) on the same box, same operand values,
+    at --size: alternating loops of >= --sustain-seconds each, after a 2 s pause, with the SM
+    clock and board power NVML saw in the second half of the loop and the energy per GEMM
+    (settled power x time per GEMM).  On a power-capped part time per GEMM is energy per GEMM
+    divided by the cap, so energy is the figure to compare.  A short leg (20 launches after the
+    pause: the burst regime) follows for FP16.  One JSON line per leg."""
+    import torch
+    from paper_2608_10103_b200 import binding, synth
+    torch.cuda.set_device(0)
+    N = args.size
+    A, B = synth.fp16_normal_clipped(N, N, N, seed=3)
+    dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    C32 = torch.empty((N, N), dtype=torch.float32, device="cuda")
+    C16 = torch.empty((N, N), dtype=torch.float16, device="cuda")
+    bA, bB = dA.to(torch.bfloat16), dB.to(torch.bfloat16)
+    Cb = torch.empty((N, N), dtype=torch.bfloat16, device="cuda")
+    A8, B8 = synth.s8_uniform(N, N, N, seed=19)
+    dA8, dB8 = torch.from_numpy(A8).cuda(), torch.from_numpy(B8).cuda()
+    Ci = torch.empty((N, N), dtype=torch.int32, device="cuda")
+    ops = synth.gemm_ops(N, N, N)
+    index = physical_gpu_index(0)
+
+    def leg(name, impl, fn, seconds, unit):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(5):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        n = 20 if seconds <= 0 else int(seconds * 1e3 / (e0.elapsed_time(e1) / 5) * 1.15) + 1
+        time.sleep(2.0)
+        sampler = ClockSampler(index)
+        sampler.start()
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        ms = e0.elapsed_time(e1) / n
+        pw = clocks.get("power_w_settled")
+        print(json.dumps({
+            "library_compare": True, "leg": name, "impl": impl, "N": N, "launches": n,
+            "seconds": ms * n * 1e-3, "ms": ms, "value": ops / (ms * 1e-3) / 1e12, "unit": unit,
+            "sm_mhz_settled": clocks.get("sm_mhz_settled"), "power_w_settled": pw,
+            "joule_per_gemm": pw * ms * 1e-3 if pw else None, "reasons": clocks.get("reasons")}),
+            flush=True)
+
+    S = args.sustain_seconds
+    dBt, bBt, dB8t = dB.t(), bB.t(), dB8.t()
+    legs = [
+        ("fp16 in, fp32 out", "this library", lambda: binding.gemm_fp16(dA, dB, C32), "TFLOP/s"),
+        ("fp16 in, fp16 out", "this library", lambda: binding.gemm_fp16_f16out(dA, dB, C16), "TFLOP/s"),
+        ("fp16 in, fp16 out", "torch.matmul", lambda: torch.matmul(dA, dBt, out=C16), "TFLOP/s"),
+        ("bf16 in, bf16 out (same values)", "torch.matmul", lambda: torch.matmul(bA, bBt, out=Cb), "TFLOP/s"),
+        ("int8 in, int32 out", "this library", lambda: binding.gemm_s8(dA8, dB8, Ci), "TOP/s"),
+        ("int8 in, int32 out", "torch._int_mm", lambda: torch._int_mm(dA8, dB8t, out=Ci), "TOP/s"),
+    ]
+    for rnd in range(2):  # twice round, so that a drift of the box shows
+        for name, impl, fn, unit in legs:
+            leg(name, impl, fn, S, unit)
+    for name, impl, fn, unit in legs[:4]:
+        leg(name + " (20 launches)", impl, fn, 0, unit)
+    if binding.gemm_last_device_status() != 0:
+        raise SystemExit("bench.py: a kernel reported a barrier timeout")
+
+
 def run_capture(args):
     """Workload for profiler captures (the summaries under profiles/ name the full command): the
     FP16 GEMM at --size (seed 3) on both kernel families and a few raster band heights, two
@@ -933,6 +1005,9 @@ def main():
     ap.add_argument("--capture", action="store_true",
                     help="profiler workload: FP16 GEMM at --size, both kernel families and band "
                          "heights, inside a profiler range (1 GPU)")
+    ap.add_argument("--library-compare", action="store_true",
+                    help="measurement only: this library against torch.matmul / torch._int_mm "
+                         "(the vendor GEMM) in alternating sustained loops with power and clock")
     ap.add_argument("--sweep", action="store_true",
                     help="precision x size sweep N=512..8192, one JSON line per cell (1 GPU)")
     ap.add_argument("--precisions", default="fp16,s8,s4")
@@ -949,6 +1024,9 @@ def main():
     if args.capture:
         if rank == 0:
             run_capture(args)
+    elif args.library_compare:
+        if rank == 0:
+            run_library_compare(args)
     elif args.selector_check:
         if rank == 0:
             run_selector_check(args)
