@@ -572,30 +572,36 @@ def run_sweep(args):
             C = torch.empty((N, N), dtype=torch.float32 if prec == "fp16" else torch.int32,
                             device="cuda")
             call = lambda st: binding.gemm(prec, dA, dB, C, st)
-            for _ in range(300):          # also lets the host core reach its working clock
+            # device time first (the host-cost loops below are a second of full-power work at
+            # N = 8192 and would push the timed replays into the power-capped regime), after a
+            # pause, so that every cell starts from the same power state
+            torch.cuda.synchronize()
+            time.sleep(1.0)
+            reps = max(5, min(100, int(20.0 / max(timed(lambda: call(stream), 5), 1e-3))))
+            g_many, g_one = graph_of(call, reps), graph_of(call, 1)
+            warm = float(np.median([timed(g_many.replay, 1) for _ in range(5)])) / reps
+            cold = float(np.median([timed(g_one.replay, 1) for _ in range(5)]))
+            n_host = 200 if N <= 2048 else 50
+            for _ in range(300 if N <= 2048 else 50):   # also lets the host core reach its working clock
                 call(stream)
             torch.cuda.synchronize()
             t0 = time.perf_counter()
-            for _ in range(200):
+            for _ in range(n_host):
                 call(stream)
-            host_us = (time.perf_counter() - t0) / 200 * 1e6
+            host_us = (time.perf_counter() - t0) / n_host * 1e6
             torch.cuda.synchronize()
             # the library's own share of that: the C entry point called with arguments that
             # are already marshalled (what a C or C++ caller pays, plus one ctypes dispatch)
             fn = getattr(binding.lib(), {"fp16": "gemm_fp16", "s8": "gemm_s8", "s4": "gemm_s4"}[prec])
             c_args = (N, N, N, dA.data_ptr(), dB.data_ptr(), C.data_ptr(), int(stream.cuda_stream))
             t0 = time.perf_counter()
-            for _ in range(200):
+            for _ in range(n_host):
                 fn(*c_args)
-            host_us_c = (time.perf_counter() - t0) / 200 * 1e6
+            host_us_c = (time.perf_counter() - t0) / n_host * 1e6
             torch.cuda.synchronize()
-            # ... and without that dispatch: the same 200 calls looped and timed inside the library
-            host_us_native = min(binding.gemm_debug_host_cost(prec, dA, dB, C, stream, 200)
+            # ... and without that dispatch: the same calls looped and timed inside the library
+            host_us_native = min(binding.gemm_debug_host_cost(prec, dA, dB, C, stream, n_host)
                                  for _ in range(3)) * 1e-3
-            reps = max(5, min(100, int(20.0 / max(timed(lambda: call(stream), 5), 1e-3))))
-            g_many, g_one = graph_of(call, reps), graph_of(call, 1)
-            warm = float(np.median([timed(g_many.replay, 1) for _ in range(5)])) / reps
-            cold = float(np.median([timed(g_one.replay, 1) for _ in range(5)]))
             ops = synth.gemm_ops(N, N, N)
             rate = ops / (warm * 1e-3) / 1e12
             ref = peaks["bf16_burst"] * (1 if prec == "fp16" else 2)

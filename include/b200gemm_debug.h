@@ -57,10 +57,11 @@ int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k);
  * overlaps the next tile; 2 = the 512 x 256 tile per CTA pair wherever the
  * problem's layout allows it (plain orientation, no split-K), whose two
  * accumulators fill tensor memory and which moves a quarter fewer operand
- * bytes per unit of math.  The automatic rule takes 2 for FP16 inputs when its
- * tiles fill at least two waves of CTA pairs to 90 % and K covers at least 96
- * blocks of 128 bytes (K >= 6144).  The paper fixes one tiling for every
- * size (Sec. III-A); this is the corresponding ablation axis here.
+ * bytes per unit of math.  The automatic rule takes 2 when its tiles fill at
+ * least two waves of CTA pairs to 90 % and K covers at least 96 blocks of 128
+ * bytes for FP16 (K >= 6144) or 64 for the integer kinds (K >= 8192; the INT4
+ * pre-pass route included).  The paper fixes one tiling for every size
+ * (Sec. III-A); this is the corresponding ablation axis here.
  */
 int gemm_set_kernel_family(int family);
 

@@ -157,17 +157,18 @@ bool wide_wanted(const TileConfig& cfg, int M, int N, int k_blocks, int num_sms,
   if (swap || csplit || packed_s4 || g_family == 1) return false;
   if (g_family == 2) return !(g_override_bn && g_override_bn != 256) && g_override_cta_group != 1 &&
                             g_override_splits <= 1;
-  // The integer kinds stay on the 256 x 256 tile: their tiles take half as long for the same C
-  // bytes, so the hand-over between tiles, which only this kernel exposes, weighs twice as much
-  // (N = 8192 INT8: 517 k against 499 k SM cycles, no gain in time).
-  if (!fp16_kind || cfg.bn != 256 || cfg.cta_group != 2 || cfg.splits != 1) return false;
+  if (cfg.bn != 256 || cfg.cta_group != 2 || cfg.splits != 1) return false;
   const long long tiles = static_cast<long long>(ceil_div(M, WIDE_TILE_M)) * ceil_div(N, WIDE_BN);
   const long long pairs = num_sms / 2;
   const long long waves = (tiles + pairs - 1) / pairs;
-  // at least two waves, at least 90 % full, and tiles long enough that the hand-over between
-  // them (~4.5 k cycles per tile that the 256 x 256 kernel does not have) stays small: measured
-  // +3 % at K = 8192, +2 % at 6144, even at 4096, -2 % at 2048 (FP16, 8192 x 8192 outputs)
-  return tiles >= 2 * pairs && 10 * tiles >= 9 * waves * pairs && k_blocks >= 96;
+  // At least two waves, at least 90 % full, and tiles long enough that the hand-over between
+  // them (~4.5 k cycles per tile that the 256 x 256 kernel does not have) stays small.  Measured
+  // in alternating sustained loops, FP16 with 8192 x 8192 outputs: +3 % at K = 8192, +2 % at
+  // 6144, even at 4096, -2 % at 2048.  The integer kinds' tiles take half as long for the same
+  // C bytes, so the hand-over weighs twice as much: the kernel needs more SM cycles there
+  // (N = 8192: 525 k against 496 k) and still wins on the power-capped part from K = 8192 on
+  // (8192^3 +1.8 %, 16384 x 8192 x 8192 +2.4 %, 8192 x 8192 x 16384 +5 %; 6144^3 -1 %).
+  return tiles >= 2 * pairs && 10 * tiles >= 9 * waves * pairs && k_blocks >= (fp16_kind ? 96 : 64);
 }
 
 // Output options of one GEMM call.
@@ -392,7 +393,9 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     k_blocks = 2 * ceil_div(K, 2 * BK_BYTES);  // one packed slot (256 values of K) = two int8 slots
   }
 
-  const bool wide = wide_wanted(cfg, M, N, k_blocks, s->num_sms, swap, csplit, packed_s4, KIND == ptx::KIND_F16);
+  // (a call that asks for the overlapped INT4 pre-pass stays on the kernel that has that role)
+  const bool wide = !req && wide_wanted(cfg, M, N, k_blocks, s->num_sms, swap, csplit, packed_s4,
+                                        KIND == ptx::KIND_F16);
   if (wide) {
     cfg.bn = WIDE_BN;
     cfg.cta_group = 2;
