@@ -183,7 +183,10 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
     M = user_n;
     N = user_m;
   }
-  const bool wide = wide_wanted(c, M, N, kb, num_sms, swap, false, fused, precision == GEMM_PREC_FP16);
+  // (the overlapped INT4 pre-pass, scheme 4, rides on the 256 x 256 kernel: every problem the
+  // 512 x 256 kernel would take qualifies for it)
+  const bool wide = !(precision == GEMM_PREC_S4 && g_s4_scheme == 4) &&
+                    wide_wanted(c, M, N, kb, num_sms, swap, false, fused, precision == GEMM_PREC_FP16);
   if (wide) {
     c.bn = WIDE_BN;
     c.cta_group = 2;
