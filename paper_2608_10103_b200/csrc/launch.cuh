@@ -677,9 +677,19 @@ int launch_unpack(long long rows_a, const uint8_t* packed_a, int8_t* out_a, long
   long long blocks = (chunks + 255) / 256;
   if (blocks > static_cast<long long>(s->num_sms) * 32) blocks = static_cast<long long>(s->num_sms) * 32;
   if (blocks < 1) blocks = 1;
-  unpack_s4_kernel<<<static_cast<int>(blocks), 256, 0, stream>>>(
-      a, b, K / 32, static_cast<long long>(out_pitch));
-  cudaError_t e = cudaGetLastError();
+  // policy bit 32 and traced launches: plain stream order, as for the GEMMs
+  const int chained = ((g_l2_policy & 32) || (g_trace_on & 1)) ? 0 : 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = chained ? 1 : 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, unpack_s4_kernel, a, b, K / 32,
+                                     static_cast<long long>(out_pitch), chained);
   if (e != cudaSuccess) return cuda_fail(e);
   return GEMM_OK;
 }

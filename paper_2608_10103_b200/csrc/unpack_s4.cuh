@@ -37,9 +37,12 @@ struct UnpackJob {
 };
 
 __global__ void __launch_bounds__(256)
-unpack_s4_kernel(UnpackJob a, UnpackJob b, int chunks_per_row, long long out_pitch) {
+unpack_s4_kernel(UnpackJob a, UnpackJob b, int chunks_per_row, long long out_pitch, int chained) {
   // the GEMM behind this kernel may set up now; it waits for this grid before its first load
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // launched early itself (its launch latency overlaps the tail of the grid in front): that grid
+  // may still read the scratch this kernel writes, or produce the packed operands it reads
+  if (chained) asm volatile("griddepcontrol.wait;" ::: "memory");
   const long long total = a.chunks + b.chunks;
   const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
   for (long long g = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; g < total;
