@@ -643,6 +643,7 @@ def run_few_rows(args):
                      ("dequantised to FP16, selector default", 0, 0, "out16")],
               "s4": [("selector default", 0, 0, "raw"), ("pre-pass + INT8 GEMM", 1, 1, "raw"),
                      ("expanded in the kernel, operands exchanged", 2, 2, "raw"),
+                     ("expanded in the kernel, both operands packed on CTA-pair tiles", 5, 0, "raw"),
                      ("dequantised to FP16, selector default", 0, 0, "out16")]}
     for M, N, K in shapes:
         for prec in [q for q in synth.PRECISIONS if q in args.precisions.split(",")]:

@@ -97,6 +97,14 @@ int gemm_set_kernel_family(int family);
  * a 36 us pre-pass -- because that kernel already keeps the SM's L2 port and
  * shared-memory pipe full and runs at ~60 % speed while the expansion is in
  * progress; kept as the ablation's third INT4 route).  3 = 1.
+ * On the CTA-pair tiles (plain operand order) the fused route has a hybrid
+ * form: B stays packed and is expanded inside the kernel, A -- the short operand
+ * there, which every tile column would otherwise expand again -- is turned into
+ * an int8 image once, by a small kernel in front, into scratch leased from the
+ * pool (gemm_query_config then shows "a=int8_image").  Taken where the 6-8 % it
+ * saves in the kernel outweigh that extra launch and the image's bytes, i.e. for
+ * large N K against a short M (256 x 28672 x 8192: 66 -> 61 us).  5 = as 2, but
+ * never the hybrid form; 6 = as 2, always the hybrid form where it exists.
  * gemm_s4_ws and gemm_s4_static always use the pre-pass launch.  Results are
  * identical, bit for bit.
  * gemm_query_config shows the route.  The paper has no counterpart; its Run 4

@@ -352,7 +352,9 @@ def gemm_set_s4_scheme(scheme: int = 0):
     """Route of gemm_s4 / gemm_s4_dequant: 0 = automatic (nibbles expanded inside the GEMM
     kernel for problems with few rows on one side, else a pre-pass to int8 + the INT8 GEMM);
     1 = always the pre-pass; 2 = inside the GEMM kernel wherever such a variant is built;
-    4 = the pre-pass done by the INT8 GEMM kernel's own epilogue warps where that applies."""
+    4 = the pre-pass done by extra warps of the INT8 GEMM kernel where that applies;
+    5 / 6 = as 2, never / always with A as an int8 image made beforehand on the CTA-pair tiles
+    (the automatic rule takes that form for large N x K against a short M)."""
     _check(lib().gemm_set_s4_scheme(int(scheme)), "gemm_set_s4_scheme")
 
 

@@ -213,7 +213,9 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
            precision == GEMM_PREC_FP16 ? "f16" : "i8",
            precision != GEMM_PREC_S4 ? "" : fused ? " s4=fused_unpack" : " prepass=unpack_s4",
            swap ? " swap_ab" : "",
-           "");  // (the raw outputs this function describes never split inside a cluster)
+           // hybrid form of the fused route: A as an int8 image made beforehand, B packed
+           // (the raw outputs this function describes never split inside a cluster)
+           (fused && !swap && c.cta_group == 2 && s4_hybrid_wanted(M, N, K)) ? " a=int8_image" : "");
   return GEMM_OK;
 }
 
@@ -259,7 +261,7 @@ int gemm_set_kernel_family(int family) {
 }
 
 int gemm_set_s4_scheme(int scheme) {
-  if (scheme < 0 || scheme > 4) return GEMM_ERR_INVALID_ARG;
+  if (scheme < 0 || scheme > 6) return GEMM_ERR_INVALID_ARG;
   g_s4_scheme = scheme;
   return GEMM_OK;
 }

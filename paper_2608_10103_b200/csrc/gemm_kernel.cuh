@@ -36,6 +36,12 @@
 //   shifts them right by 8, exactly.  The order in which K values land in the int8 slots
 //   differs from their order in memory, identically for A and B, which leaves every dot
 //   product unchanged.
+//   A8 (fused INT4, hybrid): only B arrives packed.  A is an int8 image made beforehand by a
+//   small pre-pass in exactly the form the expansion produces (16 * value, the same order of
+//   K inside a packed slot), and the first expansion warp of a group fetches the A half of
+//   each int8 slot by TMA as soon as the slot is free.  The short operand of a problem with
+//   M << N is otherwise expanded again for every tile column; this halves the expansion
+//   work and takes a sixth off the shared-memory traffic that bounds the fused kernel.
 //
 // A is M x K row-major, B is N x K with K contiguous (the paper's ".row.col"
 // operand layout, Listing 2c); C is M x N row-major, 32-bit, overwritten.
@@ -159,14 +165,15 @@ enum TraceSlot {
 // bytes of K in the 128-byte-swizzle layout (the widest a swizzled TMA box can
 // be).  KB = 2 halves the per-slot barrier work (one wait, one commit per 8 MMAs)
 // of the single issuing thread, whose instruction time is the scarce resource.
-template <int BN, int STAGES, int CTA_GROUP, int KB, int PSTAGES = 0, int CSPLIT = 1>
+template <int BN, int STAGES, int CTA_GROUP, int KB, int PSTAGES = 0, int CSPLIT = 1, bool A8 = false>
 struct SmemLayout {
   static constexpr int B_ROWS = BN / CTA_GROUP;  // B rows each CTA loads
   static constexpr int A_BYTES = BM * BK_BYTES;       // one A atom
   static constexpr int B_BYTES = B_ROWS * BK_BYTES;   // one B atom
   static constexpr int STAGE_BYTES = KB * (A_BYTES + B_BYTES);
   // Fused INT4: PSTAGES more slots, each one packed atom per operand (256 nibbles of K per row).
-  static constexpr int P_STAGE_BYTES = A_BYTES + B_BYTES;
+  // (hybrid: only B is packed, see A8 in the kernel's head comment)
+  static constexpr int P_STAGE_BYTES = (A8 ? 0 : A_BYTES) + B_BYTES;
   static constexpr int P_OFFSET = STAGES * STAGE_BYTES;
   static constexpr int RING_BYTES = STAGES * STAGE_BYTES + PSTAGES * P_STAGE_BYTES;
   // Epilogue staging: per epilogue warp two buffers of 32 rows x 128 bytes (32 x 32 C values).
@@ -180,9 +187,10 @@ struct SmemLayout {
   static constexpr int X_BYTES = CSPLIT > 1 ? (CSPLIT - 1) * X_PEER_BYTES : 0;
   static constexpr int BAR_OFFSET = X_OFFSET + X_BYTES;
   // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], drain, p_full[PSTAGES], p_empty[PSTAGES]
-  // fused INT4 adds ready[STAGES]; cluster split-K adds part_full, part_free
-  static constexpr int NUM_BARS =
-      2 * STAGES + 5 + 2 * PSTAGES + (PSTAGES > 0 ? STAGES : 0) + (CSPLIT > 1 ? 2 : 0);
+  // fused INT4 adds ready[STAGES], its hybrid form a_full[STAGES]; cluster split-K adds
+  // part_full, part_free (last two)
+  static constexpr int NUM_BARS = 2 * STAGES + 5 + 2 * PSTAGES + (PSTAGES > 0 ? STAGES : 0) +
+                                  (A8 ? STAGES : 0) + (CSPLIT > 1 ? 2 : 0);
   static constexpr int MISC_OFFSET = BAR_OFFSET + NUM_BARS * 8;
   static constexpr int TOTAL = MISC_OFFSET + 16;
   static constexpr int DYN_BYTES = TOTAL + 1024;  // slack to align the ring to 1024 bytes
@@ -245,12 +253,13 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
 // DBG: the measurement and drill switches of GemmParams::ablate are compiled in (the product
 // instantiations leave them out of their loops).
 template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32, int PSTAGES = 0,
-          int CSPLIT = 1, bool DBG = false, bool AHEAD = false>
+          int CSPLIT = 1, bool DBG = false, bool AHEAD = false, bool A8 = false>
 __global__ void __launch_bounds__(PSTAGES > 0 ? NUM_THREADS_FUSED : (AHEAD ? NUM_THREADS_AHEAD : NUM_THREADS), 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
-  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, CSPLIT>;
+  using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, CSPLIT, A8>;
   constexpr bool FUSED = PSTAGES > 0;  // packed INT4 operands, expanded on the way to the MMAs
+  static_assert(!A8 || (PSTAGES > 0 && CSPLIT == 1 && !DBG), "hybrid: a fused INT4 variant");
   const int ablate = DBG ? p.ablate : 0;
   // fused INT4: the expansion warps work as one group of eight, or -- where both rings are at
   // least four slots deep -- as two groups of four on alternate packed slots
@@ -294,6 +303,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   // arrive with release semantics straight from the writing warps costs each of them
   // hundreds of cycles).
   auto ready_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 5 + 2 * PSTAGES + s); };
+  // hybrid: the A half of int8 slot s (fetched by TMA) has landed
+  auto a_full_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 5 + 2 * PSTAGES + STAGES + s); };
   // cluster split-K: `part_full` lives in rank 0 (the other ranks' partial sums of a tile have
   // all landed), `part_free` in every other rank (rank 0 has consumed them, the buffer may be
   // overwritten)
@@ -353,6 +364,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::mbar_init(full_bar(s), 1);
       ptx::mbar_init(empty_bar(s), 1);
       if constexpr (FUSED) ptx::mbar_init(ready_bar(s), GROUP_WARPS);
+      if constexpr (A8) ptx::mbar_init(a_full_bar(s), 1);
     }
     for (int s = 0; s < PSTAGES; ++s) {
       ptx::mbar_init(p_full_bar(s), 1);
@@ -426,7 +438,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           if (trace) waited += w9 - w0;
           if (!ok) break;
           const uint32_t a_dst = base + L::P_OFFSET + stage * L::P_STAGE_BYTES;
-          const uint32_t b_dst = a_dst + L::A_BYTES;
+          const uint32_t b_dst = a_dst + (A8 ? 0 : L::A_BYTES);
           if (!elected) {
             // nothing to issue in this lane
           } else if ((ablate & 8) && blockIdx.x == 0 && t == first_tile && ps == ps_begin + 2) {
@@ -436,7 +448,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           } else {
             const int k0 = (backward ? ps_begin + ps_end - 1 - ps : ps) * BK_BYTES;  // packed bytes
             ptx::mbar_arrive_expect_tx(p_full_bar(stage), L::P_STAGE_BYTES);
-            ptx::tma_load_2d(a_dst, &tmap_a, k0, a_row, p_full_bar(stage), pol_a);
+            if constexpr (!A8) ptx::tma_load_2d(a_dst, &tmap_a, k0, a_row, p_full_bar(stage), pol_a);
             ptx::tma_load_2d(b_dst, &tmap_b, k0, b_row, p_full_bar(stage), pol_b);
           }
           ++issued;
@@ -683,7 +695,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       int pstage = 0, ustage = 0;
       uint32_t pphase = 0, uphase = 0;
       bool ok = true;
+      bool backward = false;  // hybrid: the producer's K direction for this tile (serpentine order)
+      int a_inflight[2] = {-1, -1};       // hybrid: int8 slots whose A halves this lane asked for last
+      uint32_t a_inflight_phase[2] = {0, 0};
       long long wait_in = 0, wait_out = 0, busy = 0;
+      // Rows this role expands: the whole packed slot (A rows, then B rows), or -- hybrid --
+      // only the B rows, which then start at row 0 of the packed slot and at row BM of the
+      // int8 slot.
+      constexpr int ROW0 = A8 ? BM : 0;
+      constexpr int ROWS = A8 ? L::B_ROWS : BM + L::B_ROWS;
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
         int tm, tn, tile, k_begin, k_end;
         bool add;
@@ -692,16 +712,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         // Rows of the tile beyond M resp. N are not expanded: the accumulator rows and columns
         // they feed are never stored, so whatever the int8 slot holds there does no harm, and a
         // problem with few rows (M = 16) skips most of the A tile.
-        const int a_valid = p.M - (tm * TILE_M + static_cast<int>(cta_rank) * BM);
+        const int a_row = tm * TILE_M + static_cast<int>(cta_rank) * BM;
+        const int a_valid = p.M - a_row;
         const int b_valid = p.N - (tn * BN + static_cast<int>(cta_rank) * L::B_ROWS);
-        constexpr int TASKS = (BM + L::B_ROWS + 8 * GROUP_WARPS - 1) / (8 * GROUP_WARPS);
+        constexpr int TASKS = (ROWS + 8 * GROUP_WARPS - 1) / (8 * GROUP_WARPS);
         bool active[TASKS];
 #pragma unroll
         for (int i = 0; i < TASKS; ++i) {
-          const int row8 = (i * GROUP_WARPS + uw) * 8;  // first row of this lane's group of 8
+          const int row8 = ROW0 + (i * GROUP_WARPS + uw) * 8;  // first row of this lane's group of 8
           active[i] = row8 < BM ? row8 < a_valid : (row8 < BM + L::B_ROWS && row8 - BM < b_valid);
         }
-        for (int ps = k_begin / 2; ps < k_end / 2 && ok; ++ps, ++pcount) {
+        const int ps_begin = k_begin / 2, ps_end = k_end / 2;
+        for (int ps = ps_begin; ps < ps_end && ok; ++ps, ++pcount) {
           if (UNPACK_GROUPS > 1 && pcount % UNPACK_GROUPS != ugroup) {
             // the other group's slot: only keep the ring positions in step
             ustage += 2;
@@ -726,9 +748,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const long long w2 = trace ? clock64() : 0;
           if (trace) wait_out += w2 - w1;
           if (!ok) break;
+          if constexpr (A8) {
+            // The two int8 slots are free: fetch their A halves (the int8 image of A, same K
+            // range as the packed B slot the producer sent: two 128-byte atoms of it).
+            if (uw == 0 && lane == 0) {
+              const int psk = backward ? ps_begin + ps_end - 1 - ps : ps;
+              const uint64_t pol = ptx::policy_evict_last();  // every tile column re-reads A
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                const int u = h ? u1 : u0;
+                ptx::mbar_arrive_expect_tx(a_full_bar(u), L::A_BYTES);
+                ptx::tma_load_2d(base + u * L::STAGE_BYTES, &tmap_a, (2 * psk + h) * BK_BYTES, a_row,
+                                 a_full_bar(u), pol);
+                a_inflight[h] = u;
+                a_inflight_phase[h] = h ? ph1 : ph0;
+              }
+            }
+          }
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
-            const uint32_t dst = base + (h ? u1 : u0) * L::STAGE_BYTES;
+            const uint32_t dst = base + (h ? u1 : u0) * L::STAGE_BYTES + ROW0 * BK_BYTES;
             const uint32_t x0 = static_cast<uint32_t>(row_in_8 * 128 + (((4 * h + c) ^ row_in_8) << 4));
             const uint32_t flip = static_cast<uint32_t>(h) << 6;
             // A rows first, then the B rows (the B tile follows the A tile in both rings); all
@@ -751,6 +790,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           }
           // the tensor cores read shared memory through the async proxy
           ptx::fence_proxy_async_smem();
+          if constexpr (A8) {
+            // the warp that fetched the A halves vouches for them with its own arrival
+            if (uw == 0) {
+              ok = wait_bounded(a_full_bar(u0), ph0, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
+              if (ok) ok = wait_bounded(a_full_bar(u1), ph1, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+            }
+          }
           __syncwarp();
           if (lane == 0) {
             ptx::mbar_arrive(ready_bar(u0));
@@ -763,6 +811,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(p_empty_bar(pstage));  // every lane has read its chunks
           if (++pstage == PSTAGES) { pstage = 0; pphase ^= 1u; }
+        }
+        if (p.serpentine_k) backward = !backward;
+      }
+      if constexpr (A8) {
+        if (!ok && uw == 0 && lane == 0) {
+          // Gave up: let the copies this lane asked for land before the CTA exits.
+          for (int h = 0; h < 2; ++h) {
+            if (a_inflight[h] < 0) continue;
+            const uint64_t t0 = ptx::globaltimer_ns();
+            while (!ptx::mbar_try_wait(a_full_bar(a_inflight[h]), a_inflight_phase[h]) &&
+                   ptx::globaltimer_ns() - t0 < WAIT_LIMIT_NS) {
+            }
+          }
         }
       }
       if (trace && uw == 0 && ugroup == 0 && lane == 0) {

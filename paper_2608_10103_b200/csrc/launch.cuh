@@ -195,6 +195,16 @@ constexpr int GEMM_NOT_AHEAD = 2;
 
 thread_local int t_last_s4_overlapped = 0;
 
+// Hybrid fused INT4 (CTA-pair tiles, plain orientation): B stays packed and is expanded inside
+// the kernel, A comes as the int8 image expand_s4_slots_kernel makes (rows of a8_pitch bytes,
+// K rounded up to 256).  A call that would take this form but was given no image enqueues
+// nothing and returns GEMM_WANT_A8; the caller makes the image and calls again.
+struct S4HybridReq {
+  const int8_t* a8;
+  size_t a8_pitch;
+};
+constexpr int GEMM_WANT_A8 = 3;
+
 // Index in attr_set of the unfused cluster split-K variants: 96.., by kind, output mode, width.
 template <int KIND, int EPI>
 constexpr int csplit_variant_base() {
@@ -249,7 +259,7 @@ bool cluster_split_ok(const TileConfig& c, int M, int N) {
 // which save one launch (measured: 10-26 % faster up to 1024^2 outputs, 8 % for a single wave
 // of pair tiles such as 2048^3, even or slower beyond).
 bool s4_fused_wanted(int M, int N, const TileConfig& cfg, int num_sms) {
-  if (g_s4_scheme == 2) return true;
+  if (s4_fused_forced()) return true;
   if (s4_prepass_forced()) return false;
   if (cfg.cta_group == 2) {  // (the 128-wide pair tile only comes in through select_fused_s4)
     const long long tiles = static_cast<long long>(ceil_div(M, 2 * BM)) * ceil_div(N, cfg.bn);
@@ -284,7 +294,7 @@ bool select_fused_s4(int M, int N, int user_m, int user_n, int num_sms, int k_bl
     return true;
   }
   const long long mn = static_cast<long long>(user_m) * user_n;
-  if (g_s4_scheme == 2 || mn <= 384ll * (user_m + user_n)) {
+  if (s4_fused_forced() || mn <= 384ll * (user_m + user_n)) {
     const TileConfig f = select_config(M, N, num_sms, k_blocks, min_bn, allow_split, 2, 0, 1);
     if (f.bn != 0) {
       *out = f;
@@ -306,6 +316,20 @@ bool select_fused_s4(int M, int N, int user_m, int user_n, int num_sms, int k_bl
     }
   }
   return false;
+}
+
+// Whether a fused INT4 call on a CTA-pair tile takes A as an int8 image made beforehand (the
+// hybrid form).  Measured, the kernel gains 6-8 % from not expanding A again for every tile
+// column; the image costs a launch in the chain (~2.5 us) plus its bytes (1/2 read + 1 written
+// per element at ~5 TB/s).  256 x 28672 x 8192: 66.4 -> 61.3 us, 512 x 28672 x 8192 116 -> 108,
+// 1024 x 28672 x 8192 190 -> 181; 1024 x 8192 x 8192 59.2 -> 59.9 and 2048^3 14.2 -> 16.9 are
+// the other side of the rule.  Scheme 5 never, scheme 6 always (tests, ablation).
+bool s4_hybrid_wanted(int M, int N, int K) {
+  if (g_s4_scheme == 5) return false;
+  if (g_s4_scheme == 6) return true;
+  const double gain = 0.065 * 2.0 * M * static_cast<double>(N) * K / 1.9e15;
+  const double cost = 2.5e-6 + 1.5 * M * static_cast<double>(K) / 5.0e12;
+  return gain > 1.2 * cost;
 }
 
 // Whether the kernel runs on exchanged operands (its rows = the caller's N side).  The 128-row
@@ -335,7 +359,8 @@ constexpr int GEMM_NOT_FUSED = 1;
 template <int KIND, int EPI>
 int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const void* B,
                     size_t b_pitch, void* C, const OutputSpec& out, cudaStream_t stream,
-                    bool packed_s4 = false, const S4AheadReq* req = nullptr) {
+                    bool packed_s4 = false, const S4AheadReq* req = nullptr,
+                    const S4HybridReq* hyb = nullptr) {
   DeviceState* s = nullptr;
   int rc = device_state(&s);
   if (rc != GEMM_OK) return rc;
@@ -392,6 +417,12 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
       return GEMM_NOT_FUSED;
     k_blocks = 2 * ceil_div(K, 2 * BK_BYTES);  // one packed slot (256 values of K) = two int8 slots
   }
+  // The CTA-pair fused tiles serve problems with a short M against a large N K (and single
+  // waves): every tile column would expand the same rows of A again, so A is expanded once,
+  // beforehand (scheme 5 keeps both operands packed; so do the runs with measurement switches).
+  const bool hybrid = packed_s4 && !swap && !csplit && cfg.cta_group == 2 && (g_trace_on >> 1) == 0 &&
+                      s4_hybrid_wanted(M, N, K);
+  if (hybrid && !hyb) return GEMM_WANT_A8;
 
   // (a call that asks for the overlapped INT4 pre-pass stays on the kernel that has that role)
   const bool wide = !req && wide_wanted(cfg, M, N, k_blocks, s->num_sms, swap, csplit, packed_s4,
@@ -424,7 +455,12 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   const bool promote = !(g_l2_policy & 16);
   // packed: the tensor is K/2 bytes wide; boxes stay 128 bytes
   const uint64_t k_cols = packed_s4 ? static_cast<uint64_t>(K) / 2 : static_cast<uint64_t>(K);
-  rc = encode_operand_map(&ta, type, ELEM, A, M, k_cols, a_pitch, rows_per_cta, promote);
+  if (hybrid) {
+    rc = encode_operand_map(&ta, type, ELEM, hyb->a8, M, static_cast<uint64_t>(k_blocks) * BK_BYTES,
+                            hyb->a8_pitch, rows_per_cta, promote);
+  } else {
+    rc = encode_operand_map(&ta, type, ELEM, A, M, k_cols, a_pitch, rows_per_cta, promote);
+  }
   if (rc != GEMM_OK) return rc;
   rc = encode_operand_map(&tb, type, ELEM, B, N, k_cols, b_pitch, cfg.bn / cfg.cta_group, promote);
   if (rc != GEMM_OK) return rc;
@@ -580,6 +616,16 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
     // bits 64.. (one per tile shape and output mode)
     if constexpr (KIND == ptx::KIND_I8) {
       const int fb = 64 + EPI * 8;
+      if (hybrid) {  // (int8 slots, packed B slots) = (4, 4): two groups of expansion warps
+        if (cfg.bn == 128) {
+          using L = SmemLayout<128, 4, 2, 1, 4, 1, true>;
+          return launch_kernel(s, gemm_kernel<KIND, 128, 4, 2, 1, EPI, 4, 1, false, false, true>, fb + 7,
+                               L::DYN_BYTES, NUM_THREADS_FUSED, 2, ta, tb, tc, p, stream);
+        }
+        using L = SmemLayout<256, 4, 2, 1, 4, 1, true>;
+        return launch_kernel(s, gemm_kernel<KIND, 256, 4, 2, 1, EPI, 4, 1, false, false, true>, fb + 6,
+                             L::DYN_BYTES, NUM_THREADS_FUSED, 2, ta, tb, tc, p, stream);
+      }
       if (cfg.cta_group == 2) {
         if (cfg.bn == 128)
           return launch_variant<KIND, 128, 4, 2, 1, EPI, 3>(s, fb + 5, ta, tb, tc, p, stream);
@@ -637,18 +683,19 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
 template <int KIND>
 int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* B, size_t b_pitch,
                 void* C, cudaStream_t stream, const OutputSpec& out = OutputSpec(),
-                bool packed_s4 = false, const S4AheadReq* req = nullptr) {
+                bool packed_s4 = false, const S4AheadReq* req = nullptr,
+                const S4HybridReq* hyb = nullptr) {
   switch (out.epi) {
     case EPI_RAW32:
       return launch_gemm_epi<KIND, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream,
-                                              packed_s4, req);
+                                              packed_s4, req, hyb);
     case EPI_OUT16:
       return launch_gemm_epi<KIND, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream,
-                                              packed_s4, req);
+                                              packed_s4, req, hyb);
     case EPI_F32_SCALED:
       if constexpr (KIND == ptx::KIND_I8)
         return launch_gemm_epi<KIND, EPI_F32_SCALED>(M, N, K, A, a_pitch, B, b_pitch, C, out,
-                                                     stream, packed_s4, req);
+                                                     stream, packed_s4, req, hyb);
       return GEMM_ERR_INVALID_ARG;
     default: return GEMM_ERR_INVALID_ARG;
   }
@@ -689,6 +736,29 @@ int launch_unpack(long long rows_a, const uint8_t* packed_a, int8_t* out_a, long
   cfg.attrs = attr;
   cfg.numAttrs = chained ? 1 : 0;
   cudaError_t e = cudaLaunchKernelEx(&cfg, unpack_s4_kernel, a, b, K / 32,
+                                     static_cast<long long>(out_pitch), chained);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return GEMM_OK;
+}
+
+// The int8 image of one packed operand for the hybrid fused kernel (expand_s4_slots_kernel).
+int launch_expand_slots(long long rows, const uint8_t* packed, int8_t* out, int K, size_t out_pitch,
+                        int num_sms, cudaStream_t stream) {
+  const long long chunks = rows * static_cast<long long>(out_pitch / 32);
+  long long blocks = (chunks + 255) / 256;
+  if (blocks > static_cast<long long>(num_sms) * 32) blocks = static_cast<long long>(num_sms) * 32;
+  if (blocks < 1) blocks = 1;
+  const int chained = ((g_l2_policy & 32) || (g_trace_on & 1)) ? 0 : 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = chained ? 1 : 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, expand_s4_slots_kernel, packed, out, rows, K / 2,
                                      static_cast<long long>(out_pitch), chained);
   if (e != cudaSuccess) return cuda_fail(e);
   return GEMM_OK;
@@ -744,15 +814,34 @@ size_t s4_head_bytes(int M, int N, int K) {
 int s4_auto(int M, int N, int K, const uint8_t* A, const uint8_t* B, void* C, const OutputSpec& out,
             cudaStream_t st) {
   t_last_s4_overlapped = 0;
-  if (!s4_prepass_forced()) {
-    const int rc = launch_gemm<ptx::KIND_I8>(M, N, K, A, static_cast<size_t>(K) / 2, B,
-                                             static_cast<size_t>(K) / 2, C, st, out, true);
-    if (rc != GEMM_NOT_FUSED) return rc;
-  }
   DeviceState* s = nullptr;
   int dev = 0;
   int rc = device_state(&s, &dev);
   if (rc != GEMM_OK) return rc;
+  if (!s4_prepass_forced()) {
+    rc = launch_gemm<ptx::KIND_I8>(M, N, K, A, static_cast<size_t>(K) / 2, B,
+                                   static_cast<size_t>(K) / 2, C, st, out, true);
+    if (rc == GEMM_WANT_A8) {
+      // hybrid: the int8 image of A (M rows of K rounded up to 256) in leased scratch, then the
+      // fused kernel on it and the packed B
+      const size_t pitch = align_up(static_cast<size_t>(K), 256);
+      ScratchPool::Lease lease;
+      const int prc = g_pool[dev].acquire(st, align_up(static_cast<size_t>(M) * pitch, 256),
+                                          s4_head_bytes(M, N, K), &lease);
+      if (prc != 0) return pool_fail(prc);
+      int8_t* a8 = reinterpret_cast<int8_t*>(static_cast<uint8_t*>(lease.ptr) + lease.head_bytes);
+      rc = launch_expand_slots(M, A, a8, K, pitch, s->num_sms, st);
+      if (rc == GEMM_OK) {
+        const S4HybridReq hyb{a8, pitch};
+        rc = launch_gemm<ptx::KIND_I8>(M, N, K, A, static_cast<size_t>(K) / 2, B,
+                                       static_cast<size_t>(K) / 2, C, st, out, true, nullptr, &hyb);
+      }
+      const int qrc = g_pool[dev].release(lease, st);
+      if (rc == GEMM_OK && qrc != 0) rc = pool_fail(qrc);
+      return rc;
+    }
+    if (rc != GEMM_NOT_FUSED) return rc;
+  }
   ScratchPool::Lease lease;
   const int prc = g_pool[dev].acquire(st, s4_workspace_need(M, N, K), s4_head_bytes(M, N, K), &lease);
   if (prc != 0) return pool_fail(prc);

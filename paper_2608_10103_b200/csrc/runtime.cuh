@@ -57,6 +57,7 @@ std::atomic<int> g_trace_on{0};
 // done inside the INT8 GEMM kernel ahead of its tiles where that variant applies (3 = 1)
 std::atomic<int> g_s4_scheme{0};
 bool s4_prepass_forced() { const int v = g_s4_scheme; return v == 1 || v == 3 || v == 4; }
+bool s4_fused_forced() { const int v = g_s4_scheme; return v == 2 || v == 5 || v == 6; }
 std::atomic<int> g_swap_ab{0};     // 0 = automatic, 1 = never, 2 = always exchange A and B inside the library
 std::atomic<int> g_family{0};      // kernel for large problems: 0 = automatic, 1 = 256 x 256 pair tile, 2 = 512 x 256
 std::atomic<int> g_l2_policy{11};  // keep A, B normal, serpentine K, C stores evict-first

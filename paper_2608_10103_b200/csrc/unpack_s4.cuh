@@ -70,4 +70,35 @@ unpack_s4_kernel(UnpackJob a, UnpackJob b, int chunks_per_row, long long out_pit
   }
 }
 
+// The int8 image of one packed operand in the form the fused INT4 kernel's expansion warps
+// produce in shared memory, for its hybrid variant (only the other operand expanded inside the
+// kernel): every value times 16 (nibble in the high half of its byte), and inside each run of
+// 256 values of K (one packed slot, 128 bytes; two int8 atoms of 128 bytes) the 16-byte packed
+// chunk j = 4h + c goes to atom h, its even-k values to chunk c, its odd-k values to chunk c + 4.
+// Rows are out_pitch bytes, a multiple of 256 (K rounded up; the excess is written as zeros).
+// One thread per packed chunk.
+__global__ void __launch_bounds__(256)
+expand_s4_slots_kernel(const uint8_t* packed, int8_t* out, long long rows, int k_bytes,
+                       long long out_pitch, int chained) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (chained) asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int chunks_per_row = static_cast<int>(out_pitch / 32);
+  const long long total = rows * chunks_per_row;
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  constexpr uint32_t HI = 0xF0F0F0F0u;
+  for (long long g = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; g < total;
+       g += stride) {
+    const long long row = g / chunks_per_row;
+    const int j = static_cast<int>(g - row * chunks_per_row);
+    uint4 w = make_uint4(0, 0, 0, 0);
+    if (j * 16 < k_bytes)
+      w = __ldg(reinterpret_cast<const uint4*>(packed + row * k_bytes + static_cast<long long>(j) * 16));
+    const int ps = j >> 3, h = (j >> 2) & 1, c = j & 3;
+    int8_t* dst = out + row * out_pitch + static_cast<long long>(ps) * 256 + h * 128 + c * 16;
+    *reinterpret_cast<uint4*>(dst) =
+        make_uint4((w.x << 4) & HI, (w.y << 4) & HI, (w.z << 4) & HI, (w.w << 4) & HI);
+    *reinterpret_cast<uint4*>(dst + 64) = make_uint4(w.x & HI, w.y & HI, w.z & HI, w.w & HI);
+  }
+}
+
 }  // namespace b200gemm
