@@ -93,8 +93,10 @@ int gemm_s8(int M, int N, int K, const int8_t* A, const int8_t* B, int32_t* C,
  * workspace of gemm_s4_workspace_bytes(M, N, K) bytes and then multiplied by the
  * INT8 kernel.  Small problems and problems with few rows: a kernel variant
  * expands the nibbles on the way to the MMAs and needs no workspace (see
- * gemm_set_s4_scheme in b200gemm_debug.h for the rule and the switch).  For
- * the pre-pass the library leases a scratch buffer from a per-device pool for
+ * gemm_set_s4_scheme in b200gemm_debug.h for the rule and the switch); for a
+ * short M against a large N x K that variant takes A as an int8 image made by
+ * a small kernel in front (M x K rounded up to 256 bytes of scratch).  For
+ * the pre-pass and that image the library leases a scratch buffer from a per-device pool for
  * the call's stream: the first call on a stream (and any call that needs a
  * larger one) allocates with cudaMallocAsync on that stream -- no device-wide
  * synchronisation -- and later calls on the stream reuse it, so calls on
