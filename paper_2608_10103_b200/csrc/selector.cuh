@@ -141,11 +141,17 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
         ceil_div(k_blocks, force_atoms ? force_atoms : atoms_for(best.bn, best.cta_group));
     best.split_tiles = best.splits > 1 ? static_cast<int>(tiles) : 0;
     const long long r = tiles % units;
+    const int atoms = force_atoms ? force_atoms : atoms_for(best.bn, best.cta_group);
     if (allow_split && best.splits == 1 && o_splits == 0 && tiles > units && r > 0 &&
-        2 * r <= units && slots >= 64) {  // measured: pays off (+2-3 %) only for long K
+        2 * r <= units && slots * atoms >= 64) {  // measured: pays off (+2-3 %) only for long K
       int sp = static_cast<int>(units / r);
-      if (sp > 4) sp = 4;
-      while (sp > 1 && (slots / sp < 32 ||
+      // A last wave of a few tiles only (224 tiles on 74 pairs leave 2) would cost a whole tile
+      // time: there the split goes as deep as the idle units allow, down to 8 k-blocks per
+      // unit.  Fuller last waves keep the measured rule: up to 4 ways, 32 k-blocks each.
+      const bool few = sp >= 5;
+      const int cap = few ? 16 : 4, min_kb = few ? 8 : 32;
+      if (sp > cap) sp = cap;
+      while (sp > 1 && (slots * atoms / sp < min_kb ||
                         static_cast<long long>(sp - 1) * ceil_div(slots, sp) >= slots))
         --sp;
       if (sp > 1) {

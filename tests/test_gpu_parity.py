@@ -386,3 +386,23 @@ def test_tail_wave_split():
     C = run_gpu("s8", A, B, fill=-7)
     check_against_oracle("s8", A, B, C, seed=78)
     freivalds("s8", A, B, C, seed=78, vectors=4)
+
+
+@pytest.mark.parametrize("prec", ["fp16", "s8", "s4"])
+def test_tail_wave_of_a_few_tiles_is_split_deep(prec):
+    """76 (ragged: 19 x 4) tiles of 256 x 256 on 74 SM pairs leave a last wave of two tiles: the
+    selector splits those as deep as the idle pairs allow (>= 8 k-blocks per unit) instead of
+    paying a whole tile time for them.  INT4 through the fused CTA-pair kernel in both forms."""
+    M, N, K = 1000, 4864, 8192 if prec != "fp16" else 4096
+    schemes = [0] if prec != "s4" else [5, 6]
+    A, B = synth.make(prec, M, N, K, seed=79)
+    for scheme in schemes:
+        binding.gemm_set_s4_scheme(scheme)
+        try:
+            cfg = binding.gemm_query_config(prec, M, N, K)
+            assert "split_k=8 " in cfg and "split_tiles=2 " in cfg and "tiles=76 " in cfg, cfg
+            C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
+        finally:
+            binding.gemm_set_s4_scheme(0)
+        check_against_oracle(prec, A, B, C, seed=79)
+        freivalds(prec, A, B, C, seed=79, vectors=4)
