@@ -153,6 +153,12 @@ int gemm_set_swap_ab(int mode);
  * side) use 2 for bits 0-1, so that the short operand every CTA re-reads is not
  * pushed out of L2 by the long one streaming past.  Bit 6 (64): no split-K
  * inside a cluster (see gemm_fp16_f16out / the dequantising entry points).
+ * Bit 7 (128): no even shares.  By default the one-CTA fused INT4 kernels (few
+ * rows on one side, raw output) cut the tiles' K ranges, laid end to end, into
+ * equal contiguous shares, one per SM, where that lowers the busiest SM's work by
+ * a fifth or more -- 224 tiles on 148 SMs make some SMs do two where the average
+ * is 1.5 -- instead of giving every SM whole tiles or equal parts of one tile;
+ * each piece is added into a zeroed C (gemm_query_config shows "even_share=").
  * Integer results never depend on any of this; FP16 results may differ in the last bits (summation order) within the
  * bound.
  */

@@ -199,23 +199,35 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
   const long long tiles =
       static_cast<long long>(ceil_div(M, rows_per_cta * c.cta_group)) * ceil_div(N, c.bn);
   const long long units = num_sms / c.cta_group;
+  char even[32] = "";
+  long long even_ctas = 0;
+  if (fused && c.cta_group == 1) {  // one-CTA fused INT4 tiles: equal contiguous shares of K
+    const int kb_fused = 2 * ceil_div(K, 2 * BK_BYTES);
+    const int share = s4_even_share(tiles, kb_fused, c.splits, c.split_tiles, num_sms);
+    if (share) {
+      snprintf(even, sizeof(even), " even_share=%d", share);
+      even_ctas = (tiles * (kb_fused / 2) + share - 1) / share;
+    }
+  }
   snprintf(buf, static_cast<size_t>(len),
            "BM=%d BN=%d BK=%d cta_group=%d stages=%d group_m=%d split_k=%d split_tiles=%d "
-           "tiles=%lld ctas=%lld kind=%s%s%s%s",
+           "tiles=%lld ctas=%lld kind=%s%s%s%s%s",
            rows_per_cta * c.cta_group, c.bn,
            (wide ? 1 : atoms_for(c.bn, c.cta_group)) * BK_BYTES / elem, c.cta_group,
            c.stages, c.group_m, c.splits, c.splits > 1 ? c.split_tiles : 0, tiles,
-           (tiles + (c.splits > 1 ? static_cast<long long>(c.split_tiles) * (c.splits - 1) : 0) <
-                    units
-                ? tiles + (c.splits > 1 ? static_cast<long long>(c.split_tiles) * (c.splits - 1) : 0)
-                : units) *
-               c.cta_group,
+           even_ctas ? even_ctas
+                     : (tiles + (c.splits > 1 ? static_cast<long long>(c.split_tiles) * (c.splits - 1) : 0) <
+                                units
+                            ? tiles + (c.splits > 1 ? static_cast<long long>(c.split_tiles) * (c.splits - 1) : 0)
+                            : units) *
+                           c.cta_group,
            precision == GEMM_PREC_FP16 ? "f16" : "i8",
            precision != GEMM_PREC_S4 ? "" : fused ? " s4=fused_unpack" : " prepass=unpack_s4",
            swap ? " swap_ab" : "",
            // hybrid form of the fused route: A as an int8 image made beforehand, B packed
            // (the raw outputs this function describes never split inside a cluster)
-           (fused && !swap && c.cta_group == 2 && s4_hybrid_wanted(M, N, K)) ? " a=int8_image" : "");
+           (fused && !swap && c.cta_group == 2 && s4_hybrid_wanted(M, N, K)) ? " a=int8_image" : "",
+           even);
   return GEMM_OK;
 }
 
@@ -273,7 +285,7 @@ int gemm_set_swap_ab(int mode) {
 }
 
 int gemm_set_l2_policy(int policy) {
-  if (policy < 0 || policy > 127) return GEMM_ERR_INVALID_ARG;
+  if (policy < 0 || policy > 255) return GEMM_ERR_INVALID_ARG;
   g_l2_policy = policy;
   return GEMM_OK;
 }

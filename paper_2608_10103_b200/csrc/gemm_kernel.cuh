@@ -102,6 +102,14 @@ struct GemmParams {
                          // the epilogue then stages C in shared memory and stores it by TMA
   uint32_t* C;           // element size 4 bytes, or 2 with EPI_OUT16
   long long ldc;         // row pitch of C in elements (N for a dense C)
+  // Even shares (0 = off; split-K through C only): the tiles' K ranges, laid end to end and
+  // counted in granules of one ring slot (fused INT4: one packed slot = two), are cut into
+  // contiguous shares of sk_share granules, one per CTA; a share covers the end of one tile,
+  // whole tiles, and the beginning of another, and every piece is ADDED into the zeroed C.
+  // Fills all SMs with equal work whatever the tile count (64 tiles x 2 halves occupy 128 of
+  // 148 SMs; 224 tiles make the busiest SM do two where the average is 1.5).
+  int sk_share;
+  long long sk_total;
   // 1: the caller's A and B have changed places (the kernel's rows are the caller's columns), so
   // element (row, col) of the kernel's result belongs at C[col * ldc + row].  Used for problems
   // with few rows: the long operand then fills the 128-row side of the tile, and a warp's 32
@@ -322,8 +330,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   // remaining tiles are each covered by `splits` units, one per K range.
   const int real_tiles = p.tiles_m * p.tiles_n;
   const int split_tiles = real_tiles - p.split_from;
-  const int num_tiles = p.split_from + split_tiles * p.splits;
   const int k_slots_all = (p.k_blocks + KB - 1) / KB;  // ring slots per tile; a K tail is zero-filled
+  // even shares: this CTA's (CTA pair's) contiguous range of granules and the pieces it is cut into
+  constexpr int SK_GRAN = FUSED ? 2 : 1;          // ring slots per granule
+  const int sk_tile = k_slots_all / SK_GRAN;      // granules per tile (fused INT4: k_slots_all is even)
+  const bool sk_on = CSPLIT == 1 && p.sk_share > 0;
+  const long long sk_begin =
+      sk_on ? static_cast<long long>(blockIdx.x / CTA_GROUP) * p.sk_share : 0;
+  const long long sk_end =
+      sk_on ? (sk_begin + p.sk_share < p.sk_total ? sk_begin + p.sk_share : p.sk_total) : 0;
+  const int sk_pieces =
+      sk_begin < sk_end ? static_cast<int>((sk_end - 1) / sk_tile - sk_begin / sk_tile) + 1 : 0;
+  const int num_tiles = sk_on ? sk_pieces : p.split_from + split_tiles * p.splits;
   // (fused INT4: K is split in whole packed slots = pairs of int8 slots)
   const int k_per_split = FUSED ? 2 * ((k_slots_all / 2 + p.splits - 1) / p.splits)
                                 : (k_slots_all + p.splits - 1) / p.splits;
@@ -337,6 +355,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       k_begin = static_cast<int>(krank) * per;
       k_end = min(k_begin + per, k_slots_all);
       add = false;
+    } else if (sk_on) {
+      const int first = static_cast<int>(sk_begin / sk_tile), last = static_cast<int>((sk_end - 1) / sk_tile);
+      tile = first + u;
+      k_begin = (u == 0 ? static_cast<int>(sk_begin - static_cast<long long>(first) * sk_tile) : 0) * SK_GRAN;
+      k_end = (tile == last ? static_cast<int>(sk_end - static_cast<long long>(last) * sk_tile) : sk_tile) * SK_GRAN;
+      add = true;
     } else if (u < p.split_from) {
       tile = u;
       k_begin = 0;
@@ -350,8 +374,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       add = p.splits > 1;
     }
   };
-  const int first_tile = static_cast<int>(blockIdx.x) / (CTA_GROUP * CSPLIT);
-  const int tile_stride = static_cast<int>(gridDim.x) / (CTA_GROUP * CSPLIT);
+  const int first_tile = sk_on ? 0 : static_cast<int>(blockIdx.x) / (CTA_GROUP * CSPLIT);
+  const int tile_stride = sk_on ? 1 : static_cast<int>(gridDim.x) / (CTA_GROUP * CSPLIT);
   unsigned long long* const trace =
       p.trace ? p.trace + static_cast<size_t>(blockIdx.x) * TRACE_SLOTS : nullptr;
   if (trace && threadIdx.x < TRACE_SLOTS) trace[threadIdx.x] = 0;  // roles that do not run leave 0

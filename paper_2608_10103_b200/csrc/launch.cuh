@@ -56,7 +56,9 @@ int launch_kernel(DeviceState* s, Kernel kernel, int variant, int dyn_bytes, int
   const long long all_tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   const long long tiles = p.split_from + (all_tiles - p.split_from) * p.splits;  // work units
   const long long units = s->num_sms / cluster;
-  const int grid = static_cast<int>((tiles < units ? tiles : units) * cluster);
+  int grid = static_cast<int>((tiles < units ? tiles : units) * cluster);
+  if (p.sk_share > 0)  // even shares: one CTA (pair) per share
+    grid = static_cast<int>((p.sk_total + p.sk_share - 1) / p.sk_share) * cluster;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid, 1, 1);
   cfg.blockDim = dim3(threads, 1, 1);
@@ -318,6 +320,30 @@ bool select_fused_s4(int M, int N, int user_m, int user_n, int num_sms, int k_bl
   return false;
 }
 
+// Even shares for the one-CTA fused INT4 tiles with split-K through C (problems with few rows,
+// bound by the shared-memory time of the expansion, i.e. by the busiest SM): returns the share
+// in packed slots per CTA, or 0 where whole tiles or equal tile parts do as well.  Taken when
+// the busiest SM's work falls by a fifth or more -- 150 or 224 tiles on 148 SMs make some SMs do
+// two tiles where the average is 1.0 or 1.5 (M = 32, N = 28672, K = 8192: 39.4 -> 35.5 us) --
+// and a share is at least 16 packed slots.  Smaller gains on paper are eaten by the second
+// piece a CTA then has (M = 16, N = K = 8192, 16 -> 14 slots per CTA: 15.2 -> 15.4 us).
+int s4_even_share(long long tiles, int k_blocks, int splits, long long split_tiles, int num_sms) {
+  if (g_l2_policy & 128) return 0;
+  const long long per_tile = k_blocks / 2;  // packed slots
+  const long long total = tiles * per_tile;
+  const long long cur_units = (splits > 1 && split_tiles == tiles) ? tiles * splits : tiles;
+  const long long cur = ((cur_units + num_sms - 1) / num_sms) *
+                        ((splits > 1 && split_tiles == tiles) ? (per_tile + splits - 1) / splits : per_tile);
+  const long long share = (total + num_sms - 1) / num_sms;
+  // short shares lose to the second piece (epilogue, adds, pipeline refill) a CTA then has:
+  // measured 16 x 24000 x 4096 (share 21) 23.0 -> 19.9 us, 8 x 29440 x 4096 (25) 23.1 -> 21.4,
+  // 24 x 26000 x 2048 (12) even, 64 x 21000 x 1056 (6) 13.8 -> 15.5 us
+  if (share < 16) return 0;
+  if (splits > 1 && split_tiles != tiles) return 0;  // a split of the last wave only stays as it is
+  if (splits == 1 && tiles <= num_sms) return 0;     // the selector found no split worth its cost
+  return share * 100 <= cur * 80 ? static_cast<int>(share) : 0;
+}
+
 // Whether a fused INT4 call on a CTA-pair tile takes A as an int8 image made beforehand (the
 // hybrid form).  Measured, the kernel gains 6-8 % from not expanding A again for every tile
 // column; the image costs a launch in the chain (~2.5 us) plus its bytes (1/2 read + 1 written
@@ -423,6 +449,15 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   const bool hybrid = packed_s4 && !swap && !csplit && cfg.cta_group == 2 && (g_trace_on >> 1) == 0 &&
                       s4_hybrid_wanted(M, N, K);
   if (hybrid && !hyb) return GEMM_WANT_A8;
+  int even_share = 0;
+  if (packed_s4 && !hybrid && !csplit && cfg.cta_group == 1 && split_through_c && (g_trace_on >> 1) == 0) {
+    const long long tiles = static_cast<long long>(ceil_div(M, BM)) * ceil_div(N, cfg.bn);
+    even_share = s4_even_share(tiles, k_blocks, cfg.splits, cfg.split_tiles, s->num_sms);
+    if (even_share) {  // every piece is added into a zeroed C
+      if (cfg.splits < 2) cfg.splits = 2;
+      cfg.split_tiles = static_cast<int>(tiles);
+    }
+  }
 
   // (a call that asks for the overlapped INT4 pre-pass stays on the kernel that has that role)
   const bool wide = !req && wide_wanted(cfg, M, N, k_blocks, s->num_sms, swap, csplit, packed_s4,
@@ -510,6 +545,8 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   if (p.l2_policy == 3 && (p.tiles_n == 1 || p.tiles_m == 1)) p.l2_policy = 2;
   p.serpentine_k = (g_l2_policy & 4) ? 0 : 1;
   p.c_evict_first = (g_l2_policy & 8) ? 1 : 0;
+  p.sk_share = even_share;
+  p.sk_total = even_share ? static_cast<long long>(p.tiles_m) * p.tiles_n * (k_blocks / 2) : 0;
   p.ahead = S4Ahead();
   if (ahead) {
     p.ahead.packed_a = reinterpret_cast<const uint4*>(req->packed_a);

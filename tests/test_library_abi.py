@@ -158,7 +158,14 @@ def test_selector_invariants_over_many_shapes(lib):
             else:
                 assert c["split_tiles"] == 0
                 units = tiles
-            assert c["ctas"] == min(units, 148 // cg) * cg
+            if "even_share" in text:     # fused INT4, one-CTA tiles: equal contiguous shares of K
+                share = int(text.split("even_share=")[1].split()[0])
+                slots = -(-K // 256)
+                assert "fused_unpack" in text and cg == 1 and share >= 16
+                assert c["ctas"] == -(-tiles * slots // share) <= 148
+                assert share == -(-tiles * slots // 148)
+            else:
+                assert c["ctas"] == min(units, 148 // cg) * cg
             assert 1 <= c["group_m"] <= -(-M // c["BM"])
 
 
