@@ -143,7 +143,8 @@ TileConfig select_config(int M, int N, int num_sms, int k_blocks, int min_bn = 3
     const long long r = tiles % units;
     const int atoms = force_atoms ? force_atoms : atoms_for(best.bn, best.cta_group);
     if (allow_split && best.splits == 1 && o_splits == 0 && tiles > units && r > 0 &&
-        2 * r <= units && slots * atoms >= 64) {  // measured: pays off (+2-3 %) only for long K
+        2 * r <= units && slots * atoms >= (units / r >= 5 ? 32 : 64)) {  // measured: a fuller last
+      // wave pays off (+2-3 %) only for long K
       int sp = static_cast<int>(units / r);
       // A last wave of a few tiles only (224 tiles on 74 pairs leave 2) would cost a whole tile
       // time: there the split goes as deep as the idle units allow, down to 8 k-blocks per

@@ -33,7 +33,7 @@ def _share(cfg):
 # 224 tiles on 148 SMs, unsplit (some SMs two, the average 1.5), with a ragged K whose last packed
 # slot is partly filled; 165 64-wide, 188 and 230 32-wide tiles; a long K; shares that start and
 # end inside tiles in every combination
-@pytest.mark.parametrize("M,N,K", [(32, 28672, 4128), (64, 21000, 4096), (16, 24000, 4128), (8, 29440, 8192)])
+@pytest.mark.parametrize("M,N,K", [(32, 28672, 4128), (64, 28000, 4096), (16, 24000, 4128), (8, 29440, 8192)])
 def test_even_shares_exact(M, N, K):
     cfg = binding.gemm_query_config("s4", M, N, K)
     assert "fused_unpack" in cfg and _share(cfg) >= 16, cfg
