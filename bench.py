@@ -815,9 +815,10 @@ def run_ablation(args):
     # separate pre-pass launch is inside the timed loop but not in the cycle accounting)
     s4_variants = [V("INT4 route 0: pre-pass launch to int8 + INT8 GEMM (default at this size)", family=0),
                    V("INT4 route 0': pre-pass inside the INT8 GEMM kernel, ahead of its tiles", scheme=4, family=0),
-                   V("INT4 route 1: nibbles expanded in shared memory inside the GEMM kernel", scheme=2),
-                   V("INT4 route 1, ablate: no MMAs", trace=3, scheme=2),
-                   V("INT4 route 1, ablate: no operand loads", trace=5, scheme=2)]
+                   V("INT4 route 1: nibbles expanded in shared memory inside the GEMM kernel", scheme=5),
+                   V("INT4 route 1': B expanded inside the kernel, A as an int8 image made in front", scheme=6),
+                   V("INT4 route 1, ablate: no MMAs", trace=3, scheme=5),
+                   V("INT4 route 1, ablate: no operand loads", trace=5, scheme=5)]
     for prec in [q for q in ("fp16", "s8", "s4") if q in args.precisions.split(",")]:
         dA, dB = (torch.from_numpy(x).cuda() for x in data[prec])
         C = torch.empty((N, N), dtype=torch.float32 if prec == "fp16" else torch.int32,

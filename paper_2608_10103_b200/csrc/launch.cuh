@@ -353,6 +353,9 @@ int s4_even_share(long long tiles, int k_blocks, int splits, long long split_til
 bool s4_hybrid_wanted(int M, int N, int K) {
   if (g_s4_scheme == 5) return false;
   if (g_s4_scheme == 6) return true;
+  // (with many tile rows the int8 ring, not the expansion, sets the pace: N = 8192 707 -> 689 k
+  // SM cycles only, less than the image costs)
+  if (M > 1024) return false;
   const double gain = 0.065 * 2.0 * M * static_cast<double>(N) * K / 1.9e15;
   const double cost = 2.5e-6 + 1.5 * M * static_cast<double>(K) / 5.0e12;
   return gain > 1.2 * cost;
