@@ -103,7 +103,9 @@ int gemm_s8(int M, int N, int K, const int8_t* A, const int8_t* B, int32_t* C,
  * different streams never share scratch.  A buffer whose last use has finished
  * may move to another stream.  While a stream is being captured into a graph
  * nothing can be allocated: make one call of the same size outside the capture
- * first; the captured call then keeps using that buffer, and keeping replays of
+ * first (a captured call that only wanted the image of A does without it and
+ * expands both operands in the kernel instead; one that needs the pre-pass
+ * fails); the captured call then keeps using that buffer, and keeping replays of
  * the graph apart from other gemm_s4 calls that may use it is the caller's job.
  * gemm_release_workspaces frees the pool.  Use gemm_s4_ws to supply the scratch
  * yourself.

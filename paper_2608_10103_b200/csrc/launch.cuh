@@ -449,9 +449,10 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   // The CTA-pair fused tiles serve problems with a short M against a large N K (and single
   // waves): every tile column would expand the same rows of A again, so A is expanded once,
   // beforehand (scheme 5 keeps both operands packed; so do the runs with measurement switches).
-  const bool hybrid = packed_s4 && !swap && !csplit && cfg.cta_group == 2 && (g_trace_on >> 1) == 0 &&
-                      s4_hybrid_wanted(M, N, K);
+  bool hybrid = packed_s4 && !swap && !csplit && cfg.cta_group == 2 && (g_trace_on >> 1) == 0 &&
+                s4_hybrid_wanted(M, N, K);
   if (hybrid && !hyb) return GEMM_WANT_A8;
+  if (hybrid && !hyb->a8) hybrid = false;  // the caller has no scratch for the image: both packed
   int even_share = 0;
   if (packed_s4 && !hybrid && !csplit && cfg.cta_group == 1 && split_through_c && (g_trace_on >> 1) == 0) {
     const long long tiles = static_cast<long long>(ceil_div(M, BM)) * ceil_div(N, cfg.bn);
@@ -868,6 +869,12 @@ int s4_auto(int M, int N, int K, const uint8_t* A, const uint8_t* B, void* C, co
       ScratchPool::Lease lease;
       const int prc = g_pool[dev].acquire(st, align_up(static_cast<size_t>(M) * pitch, 256),
                                           s4_head_bytes(M, N, K), &lease);
+      if (prc == ScratchPool::kNoAllocInCapture) {
+        // a stream being captured with no buffer from an earlier call: the form that needs none
+        const S4HybridReq none{nullptr, 0};
+        return launch_gemm<ptx::KIND_I8>(M, N, K, A, static_cast<size_t>(K) / 2, B,
+                                         static_cast<size_t>(K) / 2, C, st, out, true, nullptr, &none);
+      }
       if (prc != 0) return pool_fail(prc);
       int8_t* a8 = reinterpret_cast<int8_t*>(static_cast<uint8_t*>(lease.ptr) + lease.head_bytes);
       rc = launch_expand_slots(M, A, a8, K, pitch, s->num_sms, st);

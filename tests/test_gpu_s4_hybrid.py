@@ -140,3 +140,24 @@ def test_automatic_rule_takes_the_hybrid_form_for_a_short_m_against_a_large_n_k(
     A, B = synth.s4_uniform(M, N, K, seed=2)
     C = run_gpu("s4", A, B, fill=-7)
     check_against_oracle("s4", A, B, C)
+
+
+def test_hybrid_captured_without_an_earlier_call_falls_back_to_the_form_without_scratch():
+    """Nothing can be allocated while a stream is captured: with no pooled buffer from an earlier
+    call the captured call keeps both operands packed (no scratch at all) and is still exact."""
+    binding.gemm_release_workspaces()
+    binding.gemm_set_config_override(256, 0, 2, 1)
+    M, N, K = 300, 900, 1056
+    A, B = synth.s4_uniform(M, N, K, seed=21)
+    dA, dB = to_dev(A), to_dev(B)
+    C = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            binding.gemm_s4(dA, dB, C, stream=side)
+    assert binding.gemm_debug_counters()["pool_buffers"] == 0
+    g.replay()
+    torch.cuda.synchronize()
+    assert np.array_equal(C.cpu().numpy(), oracle.gemm_s4(A, B, K))
