@@ -488,9 +488,11 @@ def run_ours(args, rank, world):
         },
         "clocks": clocks,
         "e2e": e2e,
-        # INT4: pre-pass + GEMM, or the one fused kernel where the library picks that route
+        # INT4: pre-pass + GEMM; or the fused kernel, alone or behind the kernel that makes the
+        # int8 image of A, where the library picks that route
         "gpu_launches": args.steps * sum(
-            1 if "fused_unpack" in binding.gemm_query_config(p, N, N, N) else KERNEL_LAUNCHES[p]
+            (2 if "a=int8_image" in binding.gemm_query_config(p, N, N, N) else 1)
+            if "fused_unpack" in binding.gemm_query_config(p, N, N, N) else KERNEL_LAUNCHES[p]
             for p in precs),
     }
     if not args.no_cpu_baseline:

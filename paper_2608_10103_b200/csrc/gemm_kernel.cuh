@@ -38,10 +38,12 @@
 //   product unchanged.
 //   A8 (fused INT4, hybrid): only B arrives packed.  A is an int8 image made beforehand by a
 //   small pre-pass in exactly the form the expansion produces (16 * value, the same order of
-//   K inside a packed slot), and the first expansion warp of a group fetches the A half of
-//   each int8 slot by TMA as soon as the slot is free.  The short operand of a problem with
-//   M << N is otherwise expanded again for every tile column; this halves the expansion
-//   work and takes a sixth off the shared-memory traffic that bounds the fused kernel.
+//   K inside a packed slot).  Its 128-byte atoms have a ring of their own, filled by a warp of
+//   its own (warp 14) as soon as the MMAs release a slot, so that the loads run a full ring
+//   ahead of the MMAs; the int8 ring the expansion warps fill then holds B only.  The short
+//   operand of a problem with M << N is otherwise expanded again for every tile column; this
+//   halves the expansion work and takes a sixth off the shared-memory traffic that bounds
+//   the fused kernel.
 //
 // A is M x K row-major, B is N x K with K contiguous (the paper's ".row.col"
 // operand layout, Listing 2c); C is M x N row-major, 32-bit, overwritten.
@@ -66,6 +68,7 @@ constexpr int NUM_THREADS = 192;  // 6 warps: producer, MMA, 4 x epilogue
 constexpr int EPI_WARPS = 4;
 constexpr int UNPACK_WARPS = 8;   // fused INT4 only: warps 6..13
 constexpr int NUM_THREADS_FUSED = NUM_THREADS + 32 * UNPACK_WARPS;
+constexpr int NUM_THREADS_FUSED_A8 = NUM_THREADS_FUSED + 32;  // hybrid: warp 14 fetches the A image
 constexpr int AHEAD_WARPS = 4;    // overlapped INT4 pre-pass only: warps 6..9
 constexpr int NUM_THREADS_AHEAD = NUM_THREADS + 32 * AHEAD_WARPS;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // every barrier wait gives up after 2 s
@@ -178,12 +181,16 @@ struct SmemLayout {
   static constexpr int B_ROWS = BN / CTA_GROUP;  // B rows each CTA loads
   static constexpr int A_BYTES = BM * BK_BYTES;       // one A atom
   static constexpr int B_BYTES = B_ROWS * BK_BYTES;   // one B atom
-  static constexpr int STAGE_BYTES = KB * (A_BYTES + B_BYTES);
+  // (hybrid fused INT4, A8: the slots of this ring hold B only; A has the ring below)
+  static constexpr int STAGE_BYTES = A8 ? B_BYTES : KB * (A_BYTES + B_BYTES);
   // Fused INT4: PSTAGES more slots, each one packed atom per operand (256 nibbles of K per row).
   // (hybrid: only B is packed, see A8 in the kernel's head comment)
   static constexpr int P_STAGE_BYTES = (A8 ? 0 : A_BYTES) + B_BYTES;
   static constexpr int P_OFFSET = STAGES * STAGE_BYTES;
-  static constexpr int RING_BYTES = STAGES * STAGE_BYTES + PSTAGES * P_STAGE_BYTES;
+  // hybrid: ring of A atoms (int8 image), as many as fit beside the other two rings
+  static constexpr int A8_STAGES = A8 ? (BN >= 256 ? 4 : 6) : 0;
+  static constexpr int A8_OFFSET = P_OFFSET + PSTAGES * P_STAGE_BYTES;
+  static constexpr int RING_BYTES = STAGES * STAGE_BYTES + PSTAGES * P_STAGE_BYTES + A8_STAGES * A_BYTES;
   // Epilogue staging: per epilogue warp two buffers of 32 rows x 128 bytes (32 x 32 C values).
   static constexpr int EPI_BUF_BYTES = 32 * 128;
   static constexpr int EPI_OFFSET = RING_BYTES;
@@ -195,10 +202,10 @@ struct SmemLayout {
   static constexpr int X_BYTES = CSPLIT > 1 ? (CSPLIT - 1) * X_PEER_BYTES : 0;
   static constexpr int BAR_OFFSET = X_OFFSET + X_BYTES;
   // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], drain, p_full[PSTAGES], p_empty[PSTAGES]
-  // fused INT4 adds ready[STAGES], its hybrid form a_full[STAGES]; cluster split-K adds
-  // part_full, part_free (last two)
+  // fused INT4 adds ready[STAGES], its hybrid form a_full[A8_STAGES], a_empty[A8_STAGES];
+  // cluster split-K adds part_full, part_free (last two)
   static constexpr int NUM_BARS = 2 * STAGES + 5 + 2 * PSTAGES + (PSTAGES > 0 ? STAGES : 0) +
-                                  (A8 ? STAGES : 0) + (CSPLIT > 1 ? 2 : 0);
+                                  2 * A8_STAGES + (CSPLIT > 1 ? 2 : 0);
   static constexpr int MISC_OFFSET = BAR_OFFSET + NUM_BARS * 8;
   static constexpr int TOTAL = MISC_OFFSET + 16;
   static constexpr int DYN_BYTES = TOTAL + 1024;  // slack to align the ring to 1024 bytes
@@ -262,7 +269,8 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
 // instantiations leave them out of their loops).
 template <int KIND, int BN, int STAGES, int CTA_GROUP, int KB, int EPI = EPI_RAW32, int PSTAGES = 0,
           int CSPLIT = 1, bool DBG = false, bool AHEAD = false, bool A8 = false>
-__global__ void __launch_bounds__(PSTAGES > 0 ? NUM_THREADS_FUSED : (AHEAD ? NUM_THREADS_AHEAD : NUM_THREADS), 1)
+__global__ void __launch_bounds__(A8 ? NUM_THREADS_FUSED_A8
+                                     : PSTAGES > 0 ? NUM_THREADS_FUSED : (AHEAD ? NUM_THREADS_AHEAD : NUM_THREADS), 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
   using L = SmemLayout<BN, STAGES, CTA_GROUP, KB, PSTAGES, CSPLIT, A8>;
@@ -311,8 +319,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   // arrive with release semantics straight from the writing warps costs each of them
   // hundreds of cycles).
   auto ready_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 5 + 2 * PSTAGES + s); };
-  // hybrid: the A half of int8 slot s (fetched by TMA) has landed
+  // hybrid: slot s of the A ring holds its atom (both CTAs' bytes are counted on the leader's) /
+  // the MMAs that read it have retired
   auto a_full_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 5 + 2 * PSTAGES + STAGES + s); };
+  auto a_empty_bar = [&](int s) {
+    return bar0 + 8u * (2 * STAGES + 5 + 2 * PSTAGES + STAGES + L::A8_STAGES + s);
+  };
   // cluster split-K: `part_full` lives in rank 0 (the other ranks' partial sums of a tile have
   // all landed), `part_free` in every other rank (rank 0 has consumed them, the buffer may be
   // overwritten)
@@ -388,7 +400,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ptx::mbar_init(full_bar(s), 1);
       ptx::mbar_init(empty_bar(s), 1);
       if constexpr (FUSED) ptx::mbar_init(ready_bar(s), GROUP_WARPS);
-      if constexpr (A8) ptx::mbar_init(a_full_bar(s), 1);
+    }
+    for (int s = 0; s < L::A8_STAGES; ++s) {
+      ptx::mbar_init(a_full_bar(s), 1);
+      ptx::mbar_init(a_empty_bar(s), 1);
     }
     for (int s = 0; s < PSTAGES; ++s) {
       ptx::mbar_init(p_full_bar(s), 1);
@@ -581,6 +596,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
+      int astage = 0;          // hybrid fused INT4: the ring of A atoms
+      uint32_t aphase = 0;
       bool ok = true;
       long long wait_full = 0, wait_acc = 0, t_issue = 0, t_commit = 0;
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
@@ -600,6 +617,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             ok = wait_bounded(ready_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
             if (ok && CTA_GROUP == 2)
               ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
+            if constexpr (A8) {
+              if (ok) ok = wait_bounded(a_full_bar(astage), aphase, abort_flag, p.status, DEV_TIMEOUT_MMA);
+            }
           } else {
             ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
           }
@@ -607,9 +627,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           if (trace) wait_full += w2 - w1;
           if (!ok) break;
           ptx::tc_fence_after_sync();
-          const uint32_t a_src = base + stage * L::STAGE_BYTES;
+          const uint32_t a_src = A8 ? base + L::A8_OFFSET + astage * L::A_BYTES : base + stage * L::STAGE_BYTES;
           const uint64_t a_desc = ptx::smem_desc_sw128(a_src);
-          const uint64_t b_desc = ptx::smem_desc_sw128(a_src + KB * L::A_BYTES);
+          const uint64_t b_desc =
+              ptx::smem_desc_sw128(A8 ? base + stage * L::STAGE_BYTES : a_src + KB * L::A_BYTES);
           if (elected && !(ablate & 1)) {
 #pragma unroll
             for (int a = 0; a < KB; ++a) {
@@ -630,12 +651,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           if (elected) {
             if constexpr (CTA_GROUP == 1) {
               ptx::mma_commit<1>(empty_bar(stage));
+              if constexpr (A8) ptx::mma_commit<1>(a_empty_bar(astage));
             } else {
               ptx::mma_commit_pair(empty_bar(stage), 0x3);
+              if constexpr (A8) ptx::mma_commit_pair(a_empty_bar(astage), 0x3);
             }
           }
           if (trace) t_commit += clock64() - w4;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          if constexpr (A8) {
+            if (++astage == L::A8_STAGES) { astage = 0; aphase ^= 1u; }
+          }
         }
         if (!ok) break;
         if (elected) {
@@ -696,6 +722,60 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         trace[TRACE_UNPACK_BUSY] = static_cast<unsigned long long>(clock64() - u0);
     }
     __syncwarp();
+  } else if (A8 && warp == 2 + EPI_WARPS + UNPACK_WARPS) {
+    // ------------------------------------------ hybrid fused INT4: producer of the A image
+    // One 128-byte atom of the int8 image of A per k-block of the MMA issuer, into a ring of
+    // its own, in the order the packed B slots are sent (slot ps of a unit feeds k-blocks 2 ps
+    // and 2 ps + 1; with the serpentine order every other tile walks its slots backwards).
+    if constexpr (A8) {
+      const bool elected = ptx::elect_one();
+      if (p.wait_prior_grid) ptx::grid_dep_wait();  // the image comes from the grid in front
+      int astage = 0, issued = 0;
+      uint32_t aphase = 0;
+      bool ok = true, backward = false;
+      const uint64_t pol = ptx::policy_evict_last();  // every tile column re-reads A
+      for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
+        int tm, tn, tile, k_begin, k_end;
+        bool add;
+        decode_unit(t, tile, k_begin, k_end, add);
+        tile_coords(p, tile, tm, tn);
+        const int a_row = tm * TILE_M + static_cast<int>(cta_rank) * BM;
+        const int ps_begin = k_begin / 2, ps_end = k_end / 2;
+        for (int ks = k_begin; ks < k_end; ++ks) {
+          ok = wait_bounded(a_empty_bar(astage), aphase ^ 1u, abort_flag, p.status, DEV_TIMEOUT_PRODUCER);
+          if (!ok) break;
+          if (elected) {
+            const int ps = ks / 2;
+            const int atom = 2 * (backward ? ps_begin + ps_end - 1 - ps : ps) + (ks & 1);
+            const uint32_t dst = base + L::A8_OFFSET + astage * L::A_BYTES;
+            if constexpr (CTA_GROUP == 1) {
+              ptx::mbar_arrive_expect_tx(a_full_bar(astage), L::A_BYTES);
+              ptx::tma_load_2d(dst, &tmap_a, atom * BK_BYTES, a_row, a_full_bar(astage), pol);
+            } else {
+              // bytes of both CTAs are counted on the leader's barrier
+              if (leader) ptx::mbar_arrive_expect_tx(a_full_bar(astage), 2 * L::A_BYTES);
+              ptx::tma_load_2d_pair(dst, &tmap_a, atom * BK_BYTES, a_row,
+                                    ptx::map_to_cta(a_full_bar(astage), 0), pol);
+            }
+          }
+          ++issued;
+          if (++astage == L::A8_STAGES) { astage = 0; aphase ^= 1u; }
+        }
+        if (p.serpentine_k) backward = !backward;
+      }
+      if (!ok && elected && (CTA_GROUP == 1 || leader)) {
+        // Gave up: let the copies already in flight land before the CTA exits.
+        int n = issued < L::A8_STAGES ? issued : L::A8_STAGES;
+        for (int i = 0; i < n; ++i) {
+          if (--astage < 0) { astage = L::A8_STAGES - 1; aphase ^= 1u; }
+          const uint64_t t0 = ptx::globaltimer_ns();
+          while (!ptx::mbar_try_wait(a_full_bar(astage), aphase) &&
+                 ptx::globaltimer_ns() - t0 < WAIT_LIMIT_NS) {
+          }
+        }
+      }
+    }
+    __syncwarp();
   } else if (FUSED && warp >= 2 + EPI_WARPS) {
     // ------------------------------------------------- fused INT4: nibble expansion
     // One packed slot holds, per operand row, 128 bytes = 8 chunks of 16 bytes (32 values of K
@@ -719,13 +799,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       int pstage = 0, ustage = 0;
       uint32_t pphase = 0, uphase = 0;
       bool ok = true;
-      bool backward = false;  // hybrid: the producer's K direction for this tile (serpentine order)
-      int a_inflight[2] = {-1, -1};       // hybrid: int8 slots whose A halves this lane asked for last
-      uint32_t a_inflight_phase[2] = {0, 0};
       long long wait_in = 0, wait_out = 0, busy = 0;
       // Rows this role expands: the whole packed slot (A rows, then B rows), or -- hybrid --
-      // only the B rows, which then start at row 0 of the packed slot and at row BM of the
-      // int8 slot.
+      // only the B rows, which then start at row 0 of both the packed slot and the int8 slot
+      // (ROW0: what to add to a row of the slot to get its place in the A-then-B numbering
+      // that the validity test uses).
       constexpr int ROW0 = A8 ? BM : 0;
       constexpr int ROWS = A8 ? L::B_ROWS : BM + L::B_ROWS;
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
@@ -746,8 +824,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const int row8 = ROW0 + (i * GROUP_WARPS + uw) * 8;  // first row of this lane's group of 8
           active[i] = row8 < BM ? row8 < a_valid : (row8 < BM + L::B_ROWS && row8 - BM < b_valid);
         }
-        const int ps_begin = k_begin / 2, ps_end = k_end / 2;
-        for (int ps = ps_begin; ps < ps_end && ok; ++ps, ++pcount) {
+        for (int ps = k_begin / 2; ps < k_end / 2 && ok; ++ps, ++pcount) {
           if (UNPACK_GROUPS > 1 && pcount % UNPACK_GROUPS != ugroup) {
             // the other group's slot: only keep the ring positions in step
             ustage += 2;
@@ -772,26 +849,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const long long w2 = trace ? clock64() : 0;
           if (trace) wait_out += w2 - w1;
           if (!ok) break;
-          if constexpr (A8) {
-            // The two int8 slots are free: fetch their A halves (the int8 image of A, same K
-            // range as the packed B slot the producer sent: two 128-byte atoms of it).
-            if (uw == 0 && lane == 0) {
-              const int psk = backward ? ps_begin + ps_end - 1 - ps : ps;
-              const uint64_t pol = ptx::policy_evict_last();  // every tile column re-reads A
-#pragma unroll
-              for (int h = 0; h < 2; ++h) {
-                const int u = h ? u1 : u0;
-                ptx::mbar_arrive_expect_tx(a_full_bar(u), L::A_BYTES);
-                ptx::tma_load_2d(base + u * L::STAGE_BYTES, &tmap_a, (2 * psk + h) * BK_BYTES, a_row,
-                                 a_full_bar(u), pol);
-                a_inflight[h] = u;
-                a_inflight_phase[h] = h ? ph1 : ph0;
-              }
-            }
-          }
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
-            const uint32_t dst = base + (h ? u1 : u0) * L::STAGE_BYTES + ROW0 * BK_BYTES;
+            const uint32_t dst = base + (h ? u1 : u0) * L::STAGE_BYTES;
             const uint32_t x0 = static_cast<uint32_t>(row_in_8 * 128 + (((4 * h + c) ^ row_in_8) << 4));
             const uint32_t flip = static_cast<uint32_t>(h) << 6;
             // A rows first, then the B rows (the B tile follows the A tile in both rings); all
@@ -814,15 +874,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           }
           // the tensor cores read shared memory through the async proxy
           ptx::fence_proxy_async_smem();
-          if constexpr (A8) {
-            // the warp that fetched the A halves vouches for them with its own arrival
-            if (uw == 0) {
-              ok = wait_bounded(a_full_bar(u0), ph0, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
-              if (ok) ok = wait_bounded(a_full_bar(u1), ph1, abort_flag, p.status, DEV_TIMEOUT_UNPACK);
-              ok = __all_sync(0xffffffffu, ok);
-              if (!ok) break;
-            }
-          }
           __syncwarp();
           if (lane == 0) {
             ptx::mbar_arrive(ready_bar(u0));
@@ -835,19 +886,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(p_empty_bar(pstage));  // every lane has read its chunks
           if (++pstage == PSTAGES) { pstage = 0; pphase ^= 1u; }
-        }
-        if (p.serpentine_k) backward = !backward;
-      }
-      if constexpr (A8) {
-        if (!ok && uw == 0 && lane == 0) {
-          // Gave up: let the copies this lane asked for land before the CTA exits.
-          for (int h = 0; h < 2; ++h) {
-            if (a_inflight[h] < 0) continue;
-            const uint64_t t0 = ptx::globaltimer_ns();
-            while (!ptx::mbar_try_wait(a_full_bar(a_inflight[h]), a_inflight_phase[h]) &&
-                   ptx::globaltimer_ns() - t0 < WAIT_LIMIT_NS) {
-            }
-          }
         }
       }
       if (trace && uw == 0 && ugroup == 0 && lane == 0) {

@@ -317,6 +317,23 @@ bool select_fused_s4(int M, int N, int user_m, int user_n, int num_sms, int k_bl
       }
     }
   }
+  if (user_m > 1024 && user_n > 1024) {
+    // Large in both dimensions: the fused 256-wide CTA-pair kernel again, usually in its hybrid
+    // form.  Its mainloop needs more SM cycles than the INT8 kernel behind a pre-pass (N = 8192:
+    // 591 k against 528 k) but no pre-pass over both operands, and it draws less power, which on
+    // this power-capped part is clock: measured 20-launch / 0.4 s loops, pre-pass route ->
+    // fused, 8192^3 359 / 409 -> 337 / 379 us (INT8 on int8 operands: 342 / 385), 6144^3
+    // 165 / 187 -> 154 / 170, 4096^3 57.5 / 64.3 -> 57.7 / 56.9, 2048 x 8192 x 8192 110 / 124 ->
+    // 97 / 101, 8192 x 2048 x 8192 112 / 126 -> 101 / 101, 3072^3 28.4 / 29.3 -> 27.0 / 26.1;
+    // of fifteen shapes between 2048 and 16384 the pre-pass was ahead on none by more than 0.5 %.
+    // (at least one wave of pair tiles and K >= 2048: what was measured)
+    const TileConfig f = select_config(M, N, num_sms, k_blocks, min_bn, allow_split, 2, 0, 2);
+    const long long tiles = static_cast<long long>(ceil_div(M, 2 * BM)) * ceil_div(N, 256);
+    if (f.bn != 0 && tiles >= num_sms / 2 && k_blocks >= 16 && !pair_split_only_here(f)) {
+      *out = f;
+      return true;
+    }
+  }
   return false;
 }
 
@@ -345,20 +362,22 @@ int s4_even_share(long long tiles, int k_blocks, int splits, long long split_til
 }
 
 // Whether a fused INT4 call on a CTA-pair tile takes A as an int8 image made beforehand (the
-// hybrid form).  Measured, the kernel gains 6-8 % from not expanding A again for every tile
+// hybrid form).  Measured, the kernel gains 14-20 % from not expanding A again for every tile
 // column; the image costs a launch in the chain (~2.5 us) plus its bytes (1/2 read + 1 written
-// per element at ~5 TB/s).  256 x 28672 x 8192: 66.4 -> 61.3 us, 512 x 28672 x 8192 116 -> 108,
-// 1024 x 28672 x 8192 190 -> 181; 1024 x 8192 x 8192 59.2 -> 59.9 and 2048^3 14.2 -> 16.9 are
-// the other side of the rule.  Scheme 5 never, scheme 6 always (tests, ablation).
+// per element at ~5 TB/s).  256 / 512 / 1024 x 28672 x 8192: 66.5 -> 55.2, 102.0 -> 83.8,
+// 177.3 -> 149.1 us (the INT8 kernel on pre-expanded operands: 56.3, 86.9, 158.9);
+// 1024 x 8192 x 8192 59.7 -> 55.0, 512 x 16384 x 4096 35.4 -> 33.4; 256 x 8192 x 8192 and
+// 384 x 12288 x 4096 even, 2048^3 14.5 -> 16.5 are the other side of the rule; so are a
+// tall A against few tile columns (8192 x 2048 x 8192: 101 -> 112 us) and mid-sized squares
+// (4096^3 57.7 -> 59.6, 3072^3 27.0 -> 29.7), where the image costs more than it saves, while
+// 8192^3 gains 377 -> 337 us and 2048 x 8192 x 8192 108 -> 97.  Scheme 5 never, scheme 6 always
+// (tests, ablation).
 bool s4_hybrid_wanted(int M, int N, int K) {
   if (g_s4_scheme == 5) return false;
   if (g_s4_scheme == 6) return true;
-  // (with many tile rows the int8 ring, not the expansion, sets the pace: N = 8192 707 -> 689 k
-  // SM cycles only, less than the image costs)
-  if (M > 1024) return false;
-  const double gain = 0.065 * 2.0 * M * static_cast<double>(N) * K / 1.9e15;
+  const double gain = 0.14 * 2.0 * M * static_cast<double>(N) * K / 1.9e15;
   const double cost = 2.5e-6 + 1.5 * M * static_cast<double>(K) / 5.0e12;
-  return gain > 1.2 * cost;
+  return gain > 1.1 * cost + 2.0e-6;
 }
 
 // Whether the kernel runs on exchanged operands (its rows = the caller's N side).  The 128-row
@@ -661,11 +680,11 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
         if (cfg.bn == 128) {
           using L = SmemLayout<128, 4, 2, 1, 4, 1, true>;
           return launch_kernel(s, gemm_kernel<KIND, 128, 4, 2, 1, EPI, 4, 1, false, false, true>, fb + 7,
-                               L::DYN_BYTES, NUM_THREADS_FUSED, 2, ta, tb, tc, p, stream);
+                               L::DYN_BYTES, NUM_THREADS_FUSED_A8, 2, ta, tb, tc, p, stream);
         }
         using L = SmemLayout<256, 4, 2, 1, 4, 1, true>;
         return launch_kernel(s, gemm_kernel<KIND, 256, 4, 2, 1, EPI, 4, 1, false, false, true>, fb + 6,
-                             L::DYN_BYTES, NUM_THREADS_FUSED, 2, ta, tb, tc, p, stream);
+                             L::DYN_BYTES, NUM_THREADS_FUSED_A8, 2, ta, tb, tc, p, stream);
       }
       if (cfg.cta_group == 2) {
         if (cfg.bn == 128)

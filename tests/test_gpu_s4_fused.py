@@ -92,8 +92,15 @@ def test_automatic_route_by_shape():
     assert "fused_unpack" in binding.gemm_query_config("s4", 8192, 64, 4096)
     assert "fused_unpack" in binding.gemm_query_config("s4", 512, 512, 512)       # small
     assert "fused_unpack" in binding.gemm_query_config("s4", 2048, 2048, 2048)    # one wave of pair tiles
-    assert "prepass" in binding.gemm_query_config("s4", 8192, 8192, 8192)
-    assert "prepass" in binding.gemm_query_config("s4", 4096, 4096, 4096)
+    # large in both dimensions (at least a wave of pair tiles, K >= 2048): the fused pair kernel,
+    # with A as an int8 image where that pays
+    big = binding.gemm_query_config("s4", 8192, 8192, 8192)
+    assert "fused_unpack" in big and "a=int8_image" in big
+    mid = binding.gemm_query_config("s4", 4096, 4096, 4096)
+    assert "fused_unpack" in mid and "a=int8_image" not in mid
+    assert "fused_unpack" in binding.gemm_query_config("s4", 2048, 8192, 8192)
+    assert "prepass" in binding.gemm_query_config("s4", 8192, 8192, 1024)       # short K
+    assert "prepass" in binding.gemm_query_config("s4", 1536, 1536, 8192)       # less than a wave
     assert "prepass" in binding.gemm_query_config("s4", 512, 4096, 4096)
     # a short side against a large N K: M N / (M + N) <= 384, or <= 1024 rows on well-filled pair tiles
     assert "fused_unpack" in binding.gemm_query_config("s4", 256, 28672, 8192)
@@ -103,7 +110,6 @@ def test_automatic_route_by_shape():
     # 96 pair tiles on 74 pairs: the last 22 are split in two along K, which fills the waves to 80 %
     assert "fused_unpack" in binding.gemm_query_config("s4", 640, 8192, 8192)
     assert "prepass" in binding.gemm_query_config("s4", 896, 2048, 8192)
-    assert "prepass" in binding.gemm_query_config("s4", 2048, 8192, 8192)
     binding.gemm_set_s4_scheme(1)
     assert "prepass" in binding.gemm_query_config("s4", 16, 8192, 8192)
     binding.gemm_set_s4_scheme(0)

@@ -132,7 +132,11 @@ def test_automatic_rule_takes_the_hybrid_form_for_a_short_m_against_a_large_n_k(
     binding.gemm_set_s4_scheme(0)
     assert "a=int8_image" in binding.gemm_query_config("s4", 256, 28672, 8192)
     assert "a=int8_image" in binding.gemm_query_config("s4", 512, 28672, 8192)
-    assert "a=int8_image" not in binding.gemm_query_config("s4", 1024, 8192, 8192)
+    assert "a=int8_image" in binding.gemm_query_config("s4", 1024, 8192, 8192)
+    assert "a=int8_image" in binding.gemm_query_config("s4", 8192, 8192, 8192)
+    assert "a=int8_image" not in binding.gemm_query_config("s4", 8192, 2048, 8192)   # a tall A, few tile columns
+    assert "a=int8_image" not in binding.gemm_query_config("s4", 4096, 4096, 4096)
+    assert "a=int8_image" not in binding.gemm_query_config("s4", 256, 8192, 8192)
     assert "a=int8_image" not in binding.gemm_query_config("s4", 2048, 2048, 2048)
     assert "a=int8_image" not in binding.gemm_query_config("s4", 16, 8192, 8192)   # exchanged operands
     M, N, K = 256, 28672, 1056          # the rule's shape in M and N, a short K to keep the oracle quick

@@ -74,7 +74,8 @@ def test_workspace_size(lib):
 def test_selector_descriptions(lib):
     cfg = binding.gemm_query_config("fp16", 8192, 8192, 8192)
     assert "BN=256" in cfg and "cta_group=2" in cfg and "kind=f16" in cfg
-    assert "prepass=unpack_s4" in binding.gemm_query_config("s4", 4096, 4096, 4096)
+    assert "prepass=unpack_s4" in binding.gemm_query_config("s4", 1536, 1536, 8192)
+    assert "s4=fused_unpack" in binding.gemm_query_config("s4", 4096, 4096, 4096)
     binding.gemm_set_config_override(64, 3, 1)
     try:
         cfg = binding.gemm_query_config("s8", 1000, 1000, 1024)
@@ -141,9 +142,11 @@ def test_selector_invariants_over_many_shapes(lib):
                 # a problem with a short side, or a single wave of pair tiles
                 tiles2 = -(-M // 256) * -(-N // bn)
                 units2 = tiles2 + c["split_tiles"] * (sp - 1)
+                # ... or large in both dimensions: at least a wave of pair tiles, K >= 2048
                 assert (M * N <= 512 * (M + N) or (cg == 2 and bn == 256 and tiles2 <= 74) or
                         (cg == 2 and bn == 256 and min(M, N) <= 1024 and
-                         4 * units2 >= 3 * 74 * -(-units2 // 74)))
+                         4 * units2 >= 3 * 74 * -(-units2 // 74)) or
+                        (cg == 2 and bn == 256 and min(M, N) > 1024 and tiles2 >= 74 and K >= 2048))
                 if cg == 2:
                     assert bn in (256, 128)
                 atoms = 2
