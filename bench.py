@@ -815,10 +815,11 @@ def run_ablation(args):
                  V("512x256 tile, ablate: no loads", trace=5, family=2)]
     # INT4: how the nibbles reach the int8 tensor-core path (the traced launch is the GEMM; a
     # separate pre-pass launch is inside the timed loop but not in the cycle accounting)
-    s4_variants = [V("INT4 route 0: pre-pass launch to int8 + INT8 GEMM (default at this size)", family=0),
+    s4_variants = [V("INT4 route 0: pre-pass launch to int8 + INT8 GEMM", scheme=1, family=0),
                    V("INT4 route 0': pre-pass inside the INT8 GEMM kernel, ahead of its tiles", scheme=4, family=0),
                    V("INT4 route 1: nibbles expanded in shared memory inside the GEMM kernel", scheme=5),
-                   V("INT4 route 1': B expanded inside the kernel, A as an int8 image made in front", scheme=6),
+                   V("INT4 route 1': B expanded inside the kernel, A as an int8 image made in front "
+                     "(the automatic choice at this size)", scheme=0, family=0),
                    V("INT4 route 1, ablate: no MMAs", trace=3, scheme=5),
                    V("INT4 route 1, ablate: no operand loads", trace=5, scheme=5)]
     for prec in [q for q in ("fp16", "s8", "s4") if q in args.precisions.split(",")]:
