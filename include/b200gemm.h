@@ -88,13 +88,14 @@ int gemm_s8(int M, int N, int K, const int8_t* A, const int8_t* B, int32_t* C,
  * bytes, B: N rows of K/2 bytes; element k of a row is bits [4*(k&1), 4*(k&1)+4)
  * of byte k>>1 (low nibble first), two's complement.
  *
- * Blackwell's tcgen05.mma has no 4-bit integer kind.  Large problems: the
- * operands are first sign-extended to int8 by a streaming pre-pass into a
- * workspace of gemm_s4_workspace_bytes(M, N, K) bytes and then multiplied by the
- * INT8 kernel.  Small problems and problems with few rows: a kernel variant
- * expands the nibbles on the way to the MMAs and needs no workspace (see
- * gemm_set_s4_scheme in b200gemm_debug.h for the rule and the switch); for a
- * short M against a large N x K that variant takes A as an int8 image made by
+ * Blackwell's tcgen05.mma has no 4-bit integer kind.  Most problems: a kernel
+ * variant expands the nibbles on the way to the MMAs (see gemm_set_s4_scheme in
+ * b200gemm_debug.h for the rule and the switch).  The rest (a short K, less than
+ * a wave of tiles with more than 1024 rows and columns, a few in-between
+ * shapes): the operands are first sign-extended to int8 by a streaming pre-pass
+ * into a workspace of gemm_s4_workspace_bytes(M, N, K) bytes and then multiplied
+ * by the INT8 kernel.  Where A is re-read by many tile columns -- large problems,
+ * a short M against a large N x K -- the expanding variant takes A as an int8 image made by
  * a small kernel in front (M x K rounded up to 256 bytes of scratch).  For
  * the pre-pass and that image the library leases a scratch buffer from a per-device pool for
  * the call's stream: the first call on a stream (and any call that needs a

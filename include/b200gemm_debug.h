@@ -76,17 +76,24 @@ int gemm_set_kernel_family(int family);
  *     MMAs read.  No scratch, and a quarter of the pre-pass route's HBM bytes
  *     for an operand that is read once; but half as much shared-memory traffic
  *     again per unit of math, which is what bounds the large-tile kernel.
- * Measured: at M = N = K = 8192 the pre-pass route is 1.1-1.35x faster; for
- * M = 16, N = K = 8192 (bound by the bytes of B) the fused route takes 15 us
- * instead of 33.
+ * Measured: for M = 16, N = K = 8192 (bound by the bytes of B) the fused route
+ * takes 15 us instead of 33; at M = N = K = 8192 the fused CTA-pair kernel in
+ * its hybrid form (below) takes 337 us in a 20-launch loop and 379 us in a
+ * sustained one against 359 / 409 us for the pre-pass route -- its kernel needs
+ * 12 % more SM cycles but nothing expands B beforehand and it draws less power,
+ * which on a power-capped part is clock -- and the INT8 GEMM on int8 operands
+ * takes 342 / 385 us.
  * Small problems, bound by launches and latencies, save one launch with the
  * fused route (10-26 % up to 1024 x 1024 outputs).
  * scheme 0 (default, automatic): fused where the selector picks a one-CTA tile
  * and M <= 128 or N <= 128 or both <= 1024, or a single wave of CTA-pair tiles
- * (e.g. 2048^3); also for problems with a short side, where the pre-pass (cost:
+ * (e.g. 2048^3); for problems with a short side, where the pre-pass (cost:
  * the bytes of both operands) is dear next to the GEMM: M N / (M + N) <= 384
  * with the best tile the fused kernel has, and up to 1024 rows or columns with
- * its CTA-pair tile if the tiles fill their waves to 75 % (256 x 28672 x 8192:
+ * its CTA-pair tile if the tiles fill their waves to 75 %; and for problems that
+ * are large in both dimensions (more than 1024 rows and columns, at least one
+ * wave of 256 x 256 pair tiles, K >= 2048: fifteen shapes between 2048 and 16384
+ * measured, the pre-pass ahead on none) (256 x 28672 x 8192:
  * 119 -> 67 us; 512 x 16384 x 4096: 44 -> 35 us); else the pre-pass.  1: always
  * the pre-pass; 2: fused wherever a fused variant is built (every one-CTA tile,
  * and the 256 x 256 and 256 x 128 CTA pairs), else the pre-pass.  4: the
