@@ -165,3 +165,13 @@ def test_hybrid_captured_without_an_earlier_call_falls_back_to_the_form_without_
     g.replay()
     torch.cuda.synchronize()
     assert np.array_equal(C.cpu().numpy(), oracle.gemm_s4(A, B, K))
+
+
+def test_hybrid_long_k_many_laps_of_the_rings():
+    """K = 65568: 257 packed slots per tile, i.e. dozens of laps of the A ring, the packed ring and
+    the int8 ring, ending in a partly filled slot."""
+    M, N, K = 200, 520, 65568
+    binding.gemm_set_config_override(256, 0, 2, 1)
+    assert "a=int8_image" in binding.gemm_query_config("s4", M, N, K)
+    A, B = synth.s4_uniform(M, N, K, seed=65)
+    check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), force_full=True)
