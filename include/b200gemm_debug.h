@@ -184,7 +184,8 @@ int gemm_set_l2_policy(int policy);
  * cycles issuing loads [11]; fused INT4 only, one expansion warp: cycles
  * waiting for packed operands [12], for a free int8 slot [13] and spent
  * expanding [14]; 512 x 256 kernel only: cycles the MMA issuer waited for
- * the tile's second accumulator [15] ([4] is then the first).
+ * the tile's second accumulator [15] ([4] is then the first); hybrid fused INT4
+ * kernel: [15] is the part of [3] spent waiting for the atom of the A image.
  * Switching recording on (bit 1 from 0 to 1) synchronises the device and clears
  * all records.  Traced launches run in plain stream order (no early start, see
  * gemm_set_l2_policy bit 5), so that the cycle counts are the kernel's own.

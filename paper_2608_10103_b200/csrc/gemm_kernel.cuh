@@ -168,7 +168,8 @@ enum TraceSlot {
   TRACE_UNPACK_WAIT_IN = 12,   // fused INT4, unpack warp 6: cycles waiting for packed operands
   TRACE_UNPACK_WAIT_OUT = 13,  // ... waiting for a free int8 slot
   TRACE_UNPACK_BUSY = 14,      // ... expanding nibbles
-  TRACE_MMA_WAIT_ACC1 = 15,    // wide kernel: MMA issuer waiting for the tile's second accumulator
+  TRACE_MMA_WAIT_ACC1 = 15,    // wide kernel: MMA issuer waiting for the tile's second accumulator;
+                               // hybrid fused INT4: the part of [3] spent waiting for the A atom
   TRACE_SLOTS = 16
 };
 
@@ -599,7 +600,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       int astage = 0;          // hybrid fused INT4: the ring of A atoms
       uint32_t aphase = 0;
       bool ok = true;
-      long long wait_full = 0, wait_acc = 0, t_issue = 0, t_commit = 0;
+      long long wait_full = 0, wait_acc = 0, t_issue = 0, t_commit = 0, wait_a = 0;
       for (int t = first_tile; t < num_tiles && ok; t += tile_stride) {
         const long long w0 = trace ? clock64() : 0;
         ok = wait_bounded(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, p.status,
@@ -618,7 +619,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             if (ok && CTA_GROUP == 2)
               ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
             if constexpr (A8) {
+              const long long wa = trace ? clock64() : 0;
               if (ok) ok = wait_bounded(a_full_bar(astage), aphase, abort_flag, p.status, DEV_TIMEOUT_MMA);
+              if (trace) wait_a += clock64() - wa;
             }
           } else {
             ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, DEV_TIMEOUT_MMA);
@@ -679,6 +682,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         trace[TRACE_MMA_WAIT_ACC] = static_cast<unsigned long long>(wait_acc);
         trace[TRACE_MMA_ISSUE] = static_cast<unsigned long long>(t_issue);
         trace[TRACE_MMA_COMMIT] = static_cast<unsigned long long>(t_commit);
+        if (A8) trace[TRACE_MMA_WAIT_ACC1] = static_cast<unsigned long long>(wait_a);  // of wait_full: for the A atom
       }
       if (!ok && elected) {
         // Gave up: wait for the MMAs already issued before TMEM is released.
