@@ -1,0 +1,293 @@
+// Integer GEMM for problems with a few rows on one side (a handful of activations against a
+// large weight matrix): C = A B^T where one operand has at most 8 * NT rows.
+//
+// Such a call is bound by reading the long operand from HBM once, not by arithmetic, and the
+// tile kernels pay for staging it: every byte crosses shared memory several times (written by
+// the copy engine, read by the tensor core; the packed INT4 form is read, expanded and written
+// a second time), and that traffic, not HBM, sets their pace.  Here a warp feeds the operands
+// to the warp-level integer MMA (mma.sync m16n8k32, s8 x s8 -> s32: 16 rows of the long operand
+// against 8 rows of the short one per instruction) from registers, and every thread fetches
+// exactly the 16-byte pieces its own fragment registers need.
+//
+// Work split: one CTA per 16 rows of the long operand over the whole of K; its warps take the
+// 64-byte steps of K in turn (warp w: steps w, w + warps, ...), so that the CTA as a whole reads
+// a window of warps x depth x 64 contiguous bytes of each of its rows at any moment.  Every CTA
+// sums its warps' results in shared memory and writes its 16 columns (or rows) of C itself: no
+// zeroed C, no atomics, no second launch.
+//
+// Latency: a step's pieces travel by cp.async into a ring of `depth` slots that is private to the
+// thread (nobody else reads them, so no barrier is involved: the thread waits for its own copy
+// group and loads the pieces back), which keeps that many steps -- depth KB of the long operand per
+// warp -- in flight without holding registers.  (Fetching straight into registers, two steps
+// ahead, left the warps waiting on the loads for 33 of every 39 cycles and HBM at 31 %.)
+//
+// K order: a dot product may take K in any order as long as both operands use the same one.
+// Lane (g, t) = (lane / 4, lane % 4) fetches the 16 bytes at offset 16 t of a step from rows g
+// and g + 8 of the long operand and from row g of each group of eight short rows, and feeds
+// the four 32-bit words to successive MMAs: the K positions the instruction assigns to t are
+// filled from t's own words on both sides.
+//
+// Packed INT4 (two values per byte, K / 2 bytes per row): a 32-bit word holds eight values;
+// (w << 4) & 0xF0F0F0F0 is the four low nibbles as int8 values times 16, w & 0xF0F0F0F0 the
+// four high ones -- three ALU operations per word, no sign handling.  Both operands are
+// scaled alike, every product is 256 times the true one, and each warp's partial sum is an
+// exact multiple of 256 that an arithmetic shift brings back (|sum| <= 16384 K < 2^31 by the
+// library's limit on K).  (mma.sync m16n8k64 with .s4 operands compiles for sm_100a and gives
+// the same sums, but ran 4.5 times slower than this expansion: 50.9 against 11.3 us at
+// 16 x 8192 x 8192.)
+#pragma once
+
+#include <cstdint>
+#include <cuda_fp16.h>
+
+#include "gemm_kernel.cuh"
+#include "ptx.cuh"
+
+namespace b200gemm {
+
+struct FewRowsParams {
+  const uint8_t* L;     // long operand: rows_l rows of row_bytes bytes
+  const uint8_t* S;     // short operand: rows_s <= 8 NT rows
+  long long l_pitch;    // bytes between rows (multiples of 16, bases 16-byte aligned)
+  long long s_pitch;
+  int rows_l, rows_s;
+  int row_bytes;        // K (INT8) or K / 2 (INT4); a multiple of 16
+  void* C;              // element (short row s, long row l) at C[s * c_stride_s + l * c_stride_l]
+  long long c_stride_s, c_stride_l;  // in elements; one of them is 1
+  const float* scale_s; // per short row / per long row factors of the scaled outputs, or null
+  const float* scale_l;
+  int scale_s_first;    // 1: float(sum) * scale_s * scale_l, 0: float(sum) * scale_l * scale_s
+                        // (the caller's row factor is applied first either way)
+  int wait_prior_grid;  // launched to start early: wait for the grid in front before any access
+  int depth;            // ring slots per thread = steps in flight per warp, 2 .. FEW_ROWS_MAX_DEPTH
+};
+
+constexpr int FEW_ROWS_MAX_DEPTH = 8;
+
+// Words per short row in the reduction buffer: the block's long rows plus four, so that the
+// four lanes of a quad (short rows 2t) land 8 banks apart.
+__host__ __device__ constexpr int few_rows_red_pitch(int mt) { return 16 * mt + 4; }
+__host__ __device__ constexpr int few_rows_ring_bytes(int mt, int nt, int depth, int warps) {
+  return depth * (2 * mt + nt) * warps * 512;
+}
+__host__ __device__ constexpr int few_rows_red_bytes(int mt, int nt, int warps) {
+  return warps * 8 * nt * few_rows_red_pitch(mt) * 4;
+}
+
+namespace few_rows_detail {
+
+// 16 bytes global -> shared, asynchronously; bytes = 0 writes zeros and reads nothing.
+// cg: through L2 only (the long operand, read once); ca: kept in L1 too (the short operand,
+// which every CTA of the SM reads again).
+__device__ __forceinline__ void cp_async_16_cg(uint32_t dst, const uint8_t* src, int bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_16_ca(uint32_t dst, const uint8_t* src, int bytes) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() {
+  asm volatile("cp.async.commit_group;" ::: "memory");
+}
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
+}
+// The instruction takes its count as an immediate; pending is 1 .. FEW_ROWS_MAX_DEPTH - 1.
+__device__ __forceinline__ void cp_async_wait_all_but(int pending) {
+  switch (pending) {
+    case 1: cp_async_wait<1>(); break;
+    case 2: cp_async_wait<2>(); break;
+    case 3: cp_async_wait<3>(); break;
+    case 4: cp_async_wait<4>(); break;
+    case 5: cp_async_wait<5>(); break;
+    case 6: cp_async_wait<6>(); break;
+    default: cp_async_wait<7>(); break;
+  }
+}
+
+__device__ __forceinline__ void mma_s8_m16n8k32(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+      "{%8, %9}, {%0, %1, %2, %3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t word_of(const uint4& v, int i) {
+  return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
+}
+
+__device__ __forceinline__ uint32_t low_nibbles_x16(uint32_t w) { return (w << 4) & 0xF0F0F0F0u; }
+__device__ __forceinline__ uint32_t high_nibbles_x16(uint32_t w) { return w & 0xF0F0F0F0u; }
+
+}  // namespace few_rows_detail
+
+// S4: packed 4-bit operands (else int8).  MT: groups of 16 long rows per CTA (a warp holds the
+// fragments of all of them and uses each short fragment MT times: the short operand, fetched
+// again by every CTA, costs 8 NT / (16 MT) of the long operand's bytes in requests).  NT: groups
+// of eight short rows.  EPI: as for the tile kernels.
+// Dynamic shared memory: few_rows_ring_bytes + few_rows_red_bytes.  Any grid size: CTA c takes
+// the row blocks c, c + grid, ...; its copies run ahead across the block boundaries, so only
+// the first block of a CTA waits for the memory latency in full.
+template <bool S4, int MT, int NT, int EPI>
+__global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
+  using namespace few_rows_detail;
+  extern __shared__ __align__(16) unsigned char few_rows_smem[];
+  const int tid = static_cast<int>(threadIdx.x), threads = static_cast<int>(blockDim.x);
+  const int lane = tid & 31, warp = tid >> 5, warps = threads >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  constexpr int PIECES = 2 * MT + NT;      // 16-byte pieces per thread and step
+  constexpr int BLOCK_ROWS = 16 * MT;
+  constexpr int RED_PITCH = few_rows_red_pitch(MT);
+  // ring[slot][piece][thread]: a warp's 32 pieces of one kind are 512 contiguous bytes
+  const uint32_t ring = ptx::smem_addr(few_rows_smem) + static_cast<uint32_t>(tid) * 16u;
+  const uint32_t piece_pitch = static_cast<uint32_t>(threads) * 16u;
+  // behind the ring: [warps][8 NT][RED_PITCH] partial sums
+  const int depth = p.depth;
+  int* red = reinterpret_cast<int*>(few_rows_smem + few_rows_ring_bytes(MT, NT, depth, warps));
+
+  if (tid == 0) ptx::grid_dep_launch_dependents();
+  if (p.wait_prior_grid) ptx::grid_dep_wait();
+
+  // rows past the end are read as the last row (valid memory) and dropped at the store
+  const int last_l = p.rows_l - 1, last_s = p.rows_s - 1;
+  const uint8_t* sp[NT];
+#pragma unroll
+  for (int j = 0; j < NT; ++j) sp[j] = p.S + static_cast<long long>(min(8 * j + g, last_s)) * p.s_pitch;
+
+  const int blocks = (p.rows_l + BLOCK_ROWS - 1) / BLOCK_ROWS;
+  const int grid = static_cast<int>(gridDim.x);
+  const int my_blocks = (blocks - static_cast<int>(blockIdx.x) + grid - 1) / grid;
+  const int steps = (p.row_bytes + 63) >> 6;
+  const int my_steps = warp < steps ? (steps - warp + warps - 1) / warps : 0;
+
+  // The copies walk (block, step) in the order the arithmetic will; f_* is where they stand.
+  int f_block = 0, f_step = 0, f_slot = 0;
+  auto fetch = [&]() {  // this thread's pieces of the next step into the next ring slot
+    if (f_block < my_blocks && my_steps > 0) {
+      const int l0 = (static_cast<int>(blockIdx.x) + f_block * grid) * BLOCK_ROWS;
+      const int off = (warp + f_step * warps) * 64 + t * 16;
+      const bool in = off < p.row_bytes;  // rows are whole 16-byte pieces; beyond K: zeros
+      const int at = in ? off : 0, bytes = in ? 16 : 0;
+      const uint32_t slot = ring + static_cast<uint32_t>(f_slot * PIECES) * piece_pitch;
+#pragma unroll
+      for (int r = 0; r < 2 * MT; ++r)  // piece r: fragment rows g + 8 r
+        cp_async_16_cg(slot + static_cast<uint32_t>(r) * piece_pitch,
+                       p.L + static_cast<long long>(min(l0 + g + 8 * r, last_l)) * p.l_pitch + at, bytes);
+#pragma unroll
+      for (int j = 0; j < NT; ++j)
+        cp_async_16_ca(slot + static_cast<uint32_t>(2 * MT + j) * piece_pitch, sp[j] + at, bytes);
+      if (++f_step == my_steps) {
+        f_step = 0;
+        ++f_block;
+      }
+      f_slot = f_slot + 1 == depth ? 0 : f_slot + 1;
+    }
+    cp_async_commit();  // one group per call, empty or not, so that the counts below hold
+  };
+#pragma unroll 1
+  for (int d = 0; d < depth; ++d) fetch();
+
+  int c_slot = 0;
+#pragma unroll 1
+  for (int blk = 0; blk < my_blocks; ++blk) {
+    int acc[MT][NT][4];
+#pragma unroll
+    for (int m = 0; m < MT; ++m)
+#pragma unroll
+      for (int j = 0; j < NT; ++j)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[m][j][v] = 0;
+#pragma unroll 1
+    for (int i = 0; i < my_steps; ++i) {
+      cp_async_wait_all_but(depth - 1);  // all but the newest depth - 1 groups: this step has landed
+      const uint32_t slot = ring + static_cast<uint32_t>(c_slot * PIECES) * piece_pitch;
+      c_slot = c_slot + 1 == depth ? 0 : c_slot + 1;
+      uint4 a[2 * MT], b[NT];
+#pragma unroll
+      for (int r = 0; r < 2 * MT; ++r)
+        ptx::ld_shared_v4(slot + static_cast<uint32_t>(r) * piece_pitch, a[r].x, a[r].y, a[r].z, a[r].w);
+#pragma unroll
+      for (int j = 0; j < NT; ++j)
+        ptx::ld_shared_v4(slot + static_cast<uint32_t>(2 * MT + j) * piece_pitch, b[j].x, b[j].y,
+                          b[j].z, b[j].w);
+      if constexpr (S4) {
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          uint32_t b0[NT], b1[NT];
+#pragma unroll
+          for (int j = 0; j < NT; ++j) {
+            const uint32_t z = word_of(b[j], w);
+            b0[j] = low_nibbles_x16(z);
+            b1[j] = high_nibbles_x16(z);
+          }
+#pragma unroll
+          for (int m = 0; m < MT; ++m) {
+            const uint32_t x = word_of(a[2 * m], w), y = word_of(a[2 * m + 1], w);
+            const uint32_t a0 = low_nibbles_x16(x), a2 = high_nibbles_x16(x);
+            const uint32_t a1 = low_nibbles_x16(y), a3 = high_nibbles_x16(y);
+#pragma unroll
+            for (int j = 0; j < NT; ++j) mma_s8_m16n8k32(acc[m][j], a0, a1, a2, a3, b0[j], b1[j]);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int w = 0; w < 4; w += 2) {
+#pragma unroll
+          for (int m = 0; m < MT; ++m)
+#pragma unroll
+            for (int j = 0; j < NT; ++j)
+              mma_s8_m16n8k32(acc[m][j], word_of(a[2 * m], w), word_of(a[2 * m + 1], w),
+                              word_of(a[2 * m], w + 1), word_of(a[2 * m + 1], w + 1),
+                              word_of(b[j], w), word_of(b[j], w + 1));
+        }
+      }
+      // the slot just read is free again (its loads have delivered: their values were used)
+      fetch();
+    }
+
+    // accumulator fragment of group m: [0], [1] = long row 16 m + g, short rows 2t, 2t + 1;
+    // [2], [3] = long row 16 m + g + 8
+    int* mine = red + warp * (8 * NT * RED_PITCH);
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+#pragma unroll
+      for (int j = 0; j < NT; ++j) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const int s = 8 * j + 2 * t + (v & 1), l = 16 * m + g + 8 * (v >> 1);
+          mine[s * RED_PITCH + l] = S4 ? (acc[m][j][v] >> 8) : acc[m][j][v];
+        }
+      }
+    }
+    __syncthreads();
+    const int l0 = (static_cast<int>(blockIdx.x) + blk * grid) * BLOCK_ROWS;
+    const bool l_contiguous = p.c_stride_l == 1;
+    for (int idx = tid; idx < 8 * NT * BLOCK_ROWS; idx += threads) {
+      // consecutive threads along whichever index is contiguous in C
+      const int s = l_contiguous ? idx / BLOCK_ROWS : idx % (8 * NT);
+      const int l = l_contiguous ? idx % BLOCK_ROWS : idx / (8 * NT);
+      if (s >= p.rows_s || l0 + l >= p.rows_l) continue;
+      int sum = 0;
+      for (int w = 0; w < warps; ++w) sum += red[w * (8 * NT * RED_PITCH) + s * RED_PITCH + l];
+      const long long at = s * p.c_stride_s + static_cast<long long>(l0 + l) * p.c_stride_l;
+      if constexpr (EPI == EPI_RAW32) {
+        static_cast<int*>(p.C)[at] = sum;
+      } else {
+        const float fs = __ldg(p.scale_s + s), fl = __ldg(p.scale_l + l0 + l);
+        const float x = p.scale_s_first ? static_cast<float>(sum) * fs * fl
+                                        : static_cast<float>(sum) * fl * fs;
+        if constexpr (EPI == EPI_OUT16)
+          static_cast<__half*>(p.C)[at] = __float2half_rn(x);
+        else
+          static_cast<float*>(p.C)[at] = x;
+      }
+    }
+    __syncthreads();  // the sums are read: the next block's may be written
+  }
+  cp_async_wait<0>();
+}
+
+}  // namespace b200gemm

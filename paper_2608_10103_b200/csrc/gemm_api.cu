@@ -164,6 +164,17 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
   const int num_sms = known_sm_count();
   const int elem = precision == GEMM_PREC_FP16 ? 2 : 1;
   const int kb = ceil_div(static_cast<long long>(K) * elem, BK_BYTES);
+  if (precision != GEMM_PREC_FP16 &&
+      few_rows_wanted(M, N, K, precision == GEMM_PREC_S4, OutputSpec())) {
+    const int rows_l = M < N ? N : M;
+    const int row_bytes = precision == GEMM_PREC_S4 ? K / 2 : K;
+    const FewRowsShape f = few_rows_shape(rows_l, M < N ? M : N, row_bytes, num_sms);
+    snprintf(buf, static_cast<size_t>(len),
+             "few_rows rows_per_block=%d blocks=%d short_rows=%d warps=%d depth=%d ctas=%d kind=i8%s",
+             16 * f.mt, ceil_div(rows_l, 16 * f.mt), M < N ? M : N, f.warps, f.depth, f.grid,
+             precision == GEMM_PREC_S4 ? " s4=in_registers" : "");
+    return GEMM_OK;
+  }
   TileConfig c;
   bool fused = false, swap = false;
   const int user_m = M, user_n = N;
@@ -267,7 +278,7 @@ int gemm_last_device_status(void) {
 }
 
 int gemm_set_kernel_family(int family) {
-  if (family < 0 || family > 2) return GEMM_ERR_INVALID_ARG;
+  if (family < 0 || family > 3) return GEMM_ERR_INVALID_ARG;
   g_family = family;
   return GEMM_OK;
 }

@@ -4,6 +4,7 @@
 
 #include <utility>
 
+#include "few_rows.cuh"
 #include "gemm_wide.cuh"
 #include "runtime.cuh"
 #include "selector.cuh"
@@ -180,6 +181,7 @@ struct OutputSpec {
   const float* col_scale = nullptr;
   long long ldc = 0;        // row pitch of C in elements; 0 = dense (N)
   bool no_split = false;    // C is a block of a larger matrix: never zero / add into it
+  bool tiles_only = false;  // the GEMM of the INT4 pre-pass route: always a tile kernel
 };
 
 // Overlapped INT4 pre-pass: A and B of the call are the (not yet written) int8 images in a
@@ -740,11 +742,157 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   }
 }
 
+// Integer problems with a few rows on one side go to few_rows_kernel (the long operand from
+// global memory to MMA fragments without a pass through a shared tile, one launch, nothing
+// zeroed).  Automatic for a short side of up to 16 rows against 512 or more: INT4 always (it
+// measured 0.45-0.98 of the tile kernels' time for 2048 <= N <= 28672, K = 4096 / 8192: there the
+// tile kernels are bound by expanding the nibbles in shared memory); INT8 while the long operand
+// has at most 32 MB and, from nine rows on, at least 4096 rows (0.68-0.92 of the tile kernels'
+// time; level at 64 MB, and 1.1-1.3 x slower beyond, where the tile kernels' bulk copies reach
+// 0.86 of the HBM bandwidth and this kernel's 16-byte copies 0.7).  gemm_set_kernel_family(3)
+// takes it wherever it exists (a short side of up to 32 rows), families 1 and 2, forced tile
+// shapes, forced operand orders, every forced INT4 scheme and the traced runs never.
+constexpr int FEW_ROWS_AUTO = 16;
+constexpr int FEW_ROWS_MAX = 32;
+bool few_rows_wanted(int M, int N, int K, bool packed_s4, const OutputSpec& out) {
+  if (out.tiles_only || g_override_bn || g_override_cta_group || g_override_splits) return false;
+  if ((g_trace_on & 1) || (g_l2_policy & 64)) return false;  // measurement runs mean the tile kernels
+  if (g_swap_ab) return false;                                // so does a forced operand order
+  if (packed_s4 && g_s4_scheme != 0) return false;
+  const int fam = g_family;
+  const int shorter = M < N ? M : N, longer = M < N ? N : M;
+  if (fam == 3) return shorter <= FEW_ROWS_MAX;
+  if (fam != 0 || shorter > FEW_ROWS_AUTO || longer < 512) return false;
+  if (packed_s4) return true;
+  return static_cast<long long>(longer) * K <= (32LL << 20) && (shorter <= 8 || longer >= 4096);
+}
+
+// Shape of a few-rows launch.  MT groups of 16 long rows per CTA: two from nine short rows on,
+// so that the short operand's requests stay at half the long operand's.
+#ifndef FEW_ROWS_MT
+#define FEW_ROWS_MT(nt) ((nt) >= 2 ? 2 : 1)
+#endif
+
+struct FewRowsShape {
+  int mt, depth, warps, grid, smem;
+};
+
+constexpr int FEW_ROWS_SMEM_SM = 227 * 1024;  // shared memory of an SM; each CTA reserves 1 KB more
+
+// Warps per CTA share K (64 bytes per step): eight, fewer for a short K (two steps each at
+// least), sixteen while the SMs would have fewer than twelve warps each and K is long enough.
+// CTAs per SM: as many as hold every row block at once if the ring can still be two steps deep;
+// else fewer, with a ring of at least three steps, and a CTA walks the blocks c, c + grid, ...
+// The ring takes what shared memory there is (up to eight steps): the kernel is as fast as HBM
+// only while ~100 KB of the long operand per SM are in flight (warps x depth x MT KB per CTA).
+FewRowsShape few_rows_shape(int rows_l, int rows_s, int row_bytes, int num_sms) {
+  const int nt = rows_s <= 8 ? 1 : rows_s <= 16 ? 2 : 4;
+  FewRowsShape f;
+  f.mt = FEW_ROWS_MT(nt);
+  const int steps = ceil_div(row_bytes, 64);
+  const long long blocks = ceil_div(rows_l, 16 * f.mt);
+  f.warps = 8;
+  while (f.warps > 1 && steps < 2 * f.warps) f.warps /= 2;
+  if (f.warps == 8 && blocks * 8 < 12LL * num_sms && steps >= 64) f.warps = 16;
+  const int red = few_rows_red_bytes(f.mt, nt, f.warps);
+  const int slot = few_rows_ring_bytes(f.mt, nt, 1, f.warps);
+  int per_sm = static_cast<int>((blocks + num_sms - 1) / num_sms);
+  if (per_sm * f.warps > 64) per_sm = 64 / f.warps;  // warp slots of an SM
+  if (per_sm > 32) per_sm = 32;                      // and its CTA slots
+  for (;; --per_sm) {
+    f.depth = (FEW_ROWS_SMEM_SM / per_sm - 1024 - red) / slot;
+    const bool all_at_once = blocks <= static_cast<long long>(per_sm) * num_sms;
+    if (f.depth >= (all_at_once ? 2 : 3) || per_sm == 1) break;
+  }
+  if (f.depth > FEW_ROWS_MAX_DEPTH) f.depth = FEW_ROWS_MAX_DEPTH;
+  f.smem = few_rows_ring_bytes(f.mt, nt, f.depth, f.warps) + red;
+  const long long resident = static_cast<long long>(per_sm) * num_sms;
+  f.grid = static_cast<int>(blocks < resident ? blocks : resident);
+  return f;
+}
+
+template <bool S4, int NT, int EPI>
+int launch_few_rows_nt(DeviceState* s, FewRowsParams& p, const FewRowsShape& f,
+                       cudaStream_t stream) {
+  constexpr int MT = FEW_ROWS_MT(NT);
+  constexpr int variant = 224 + (S4 ? 9 : 0) + (NT == 1 ? 0 : NT == 2 ? 3 : 6) + EPI;
+  auto kernel = few_rows_kernel<S4, MT, NT, EPI>;
+  if (!(s->attr_set[variant >> 6].load(std::memory_order_relaxed) & (1ull << (variant & 63)))) {
+    const cudaError_t e = cudaFuncSetAttribute(
+        kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FEW_ROWS_SMEM_SM);
+    if (e != cudaSuccess) return cuda_fail(e);
+    s->attr_set[variant >> 6].fetch_or(1ull << (variant & 63), std::memory_order_relaxed);
+  }
+  p.depth = f.depth;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(f.grid), 1, 1);
+  cfg.blockDim = dim3(static_cast<unsigned>(f.warps * 32), 1, 1);
+  cfg.dynamicSmemBytes = static_cast<size_t>(f.smem);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.wait_prior_grid ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, p);
+  return e == cudaSuccess ? GEMM_OK : cuda_fail(e);
+}
+
+// A, B: int8 or packed INT4 rows, pitches in bytes.
+template <bool S4, int EPI>
+int launch_few_rows(int M, int N, int K, const void* A, size_t a_pitch, const void* B,
+                    size_t b_pitch, void* C, const OutputSpec& out, cudaStream_t stream) {
+  DeviceState* s = nullptr;
+  int rc = device_state(&s);
+  if (rc != GEMM_OK) return rc;
+  const long long ldc = out.ldc ? out.ldc : N;
+  const bool a_short = M <= N;
+  FewRowsParams p;
+  p.L = static_cast<const uint8_t*>(a_short ? B : A);
+  p.S = static_cast<const uint8_t*>(a_short ? A : B);
+  p.l_pitch = static_cast<long long>(a_short ? b_pitch : a_pitch);
+  p.s_pitch = static_cast<long long>(a_short ? a_pitch : b_pitch);
+  p.rows_l = a_short ? N : M;
+  p.rows_s = a_short ? M : N;
+  p.row_bytes = S4 ? K / 2 : K;
+  p.C = C;
+  p.c_stride_s = a_short ? ldc : 1;
+  p.c_stride_l = a_short ? 1 : ldc;
+  p.scale_s = a_short ? out.row_scale : out.col_scale;
+  p.scale_l = a_short ? out.col_scale : out.row_scale;
+  p.scale_s_first = a_short ? 1 : 0;
+  p.wait_prior_grid = (g_l2_policy & 32) ? 0 : 1;
+  const FewRowsShape f = few_rows_shape(p.rows_l, p.rows_s, p.row_bytes, s->num_sms);
+  switch (ceil_div(p.rows_s, 8)) {
+    case 1: return launch_few_rows_nt<S4, 1, EPI>(s, p, f, stream);
+    case 2: return launch_few_rows_nt<S4, 2, EPI>(s, p, f, stream);
+    case 3:
+    case 4: return launch_few_rows_nt<S4, 4, EPI>(s, p, f, stream);
+    default: return GEMM_ERR_INVALID_ARG;
+  }
+}
+
 template <int KIND>
 int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* B, size_t b_pitch,
                 void* C, cudaStream_t stream, const OutputSpec& out = OutputSpec(),
                 bool packed_s4 = false, const S4AheadReq* req = nullptr,
                 const S4HybridReq* hyb = nullptr) {
+  if constexpr (KIND == ptx::KIND_I8) {
+    if (!req && !hyb && few_rows_wanted(M, N, K, packed_s4, out)) {
+      switch (out.epi) {
+        case EPI_RAW32:
+          return packed_s4 ? launch_few_rows<true, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream)
+                           : launch_few_rows<false, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+        case EPI_OUT16:
+          return packed_s4 ? launch_few_rows<true, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream)
+                           : launch_few_rows<false, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+        case EPI_F32_SCALED:
+          return packed_s4 ? launch_few_rows<true, EPI_F32_SCALED>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream)
+                           : launch_few_rows<false, EPI_F32_SCALED>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+        default: return GEMM_ERR_INVALID_ARG;
+      }
+    }
+  }
   switch (out.epi) {
     case EPI_RAW32:
       return launch_gemm_epi<KIND, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream,
@@ -840,13 +988,15 @@ size_t s4_workspace_need(int M, int N, int K) {
 // `sync`: bookkeeping words of the overlapped pre-pass in front of a pool buffer, or null
 // (caller-supplied scratch, whose surroundings the library knows nothing about).
 int s4_with_workspace(int M, int N, int K, const uint8_t* A, const uint8_t* B, void* C,
-                      void* workspace, size_t workspace_bytes, const OutputSpec& out,
+                      void* workspace, size_t workspace_bytes, const OutputSpec& out_in,
                       cudaStream_t st, uint32_t* sync = nullptr) {
   if (!workspace) return GEMM_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < s4_workspace_need(M, N, K))
     return GEMM_ERR_WORKSPACE;
   int8_t* a8 = static_cast<int8_t*>(workspace);
   int8_t* b8 = a8 + align_up(static_cast<size_t>(M) * K, 256);
+  OutputSpec out = out_in;
+  out.tiles_only = true;
   int rc;
   if (sync) {
     const S4AheadReq req{A, B, sync};

@@ -1,0 +1,157 @@
+"""GPU parity of the kernel for integer problems with a few rows on one side (the long operand
+goes from global memory into warp-level MMA fragments; no tile, no split-K through C) against
+the oracle: both integer precisions, either operand as the short one, every output mode,
+ragged sizes, many row blocks per CTA, and bit-equality with the tile kernels.
+gemm_set_kernel_family(3) takes the kernel wherever it exists (a short side of up to 32 rows),
+family 1 never."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_10103_b200 import binding, synth
+from gpu_util import check_against_oracle, run_gpu, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def _few_rows_route():
+    binding.gemm_set_config_override(0, 0, 0, 0)
+    binding.gemm_set_s4_scheme(0)
+    binding.gemm_set_kernel_family(3)
+    yield
+    binding.gemm_set_kernel_family(0)
+    assert binding.gemm_last_device_status() == 0
+
+
+def _make(prec, M, N, K, seed):
+    return synth.s4_uniform(M, N, K, seed=seed) if prec == "s4" else synth.make(prec, M, N, K, seed=seed)
+
+
+# short side 1..32 (one, two and four groups of eight rows; 3, 12, 20 leave a group partly
+# filled), the long side ragged against the 16- and 32-row blocks, K from a single 16-byte piece
+# per row (32 packed values) over ragged steps (96, 160, 1056, 4128) to many steps per warp
+SHAPES = [(1, 1, 32), (1, 777, 512), (3, 100, 96), (8, 1000, 4128), (9, 530, 160), (12, 2049, 1056),
+          (16, 4100, 2048), (16, 31, 64), (20, 600, 1056), (32, 1500, 512),
+          (777, 1, 512), (1000, 8, 4128), (2049, 12, 1056), (530, 16, 160), (600, 29, 96)]
+
+
+@pytest.mark.parametrize("prec", ["s8", "s4"])
+@pytest.mark.parametrize("M,N,K", SHAPES)
+def test_few_rows_full_compare(prec, M, N, K):
+    assert binding.gemm_query_config(prec, M, N, K).startswith("few_rows")
+    A, B = _make(prec, M, N, K, seed=M + N + K)
+    for rep in range(2):
+        check_against_oracle(prec, A, B, run_gpu(prec, A, B, fill=-7), force_full=True)
+
+
+@pytest.mark.parametrize("prec", ["s8", "s4"])
+@pytest.mark.parametrize("M,N,K", [(8, 80000, 1056), (16, 160001, 256), (5, 200000, 64), (160000, 16, 512)])
+def test_few_rows_more_row_blocks_than_ctas(prec, M, N, K):
+    """More row blocks than CTAs fit the SMs: a CTA walks several, its copies running ahead
+    across the block boundaries."""
+    cfg = binding.gemm_query_config(prec, M, N, K)
+    ctas = int(cfg.split("ctas=")[1].split()[0])
+    blocks = int(cfg.split("blocks=")[1].split()[0])
+    assert cfg.startswith("few_rows") and ctas < blocks
+    A, B = _make(prec, M, N, K, seed=N)
+    check_against_oracle(prec, A, B, run_gpu(prec, A, B, fill=-7))
+
+
+@pytest.mark.parametrize("prec", ["s8", "s4"])
+def test_few_rows_equals_the_tile_kernels(prec):
+    for M, N, K in [(16, 3000, 4128), (7, 2500, 1056), (1500, 11, 2048)]:
+        A, B = _make(prec, M, N, K, seed=K)
+        got = run_gpu(prec, A, B, fill=-7)
+        binding.gemm_set_kernel_family(1)
+        assert not binding.gemm_query_config(prec, M, N, K).startswith("few_rows")
+        tiles = run_gpu(prec, A, B, fill=-7)
+        binding.gemm_set_kernel_family(3)
+        assert np.array_equal(got, tiles)
+
+
+def test_few_rows_extreme_values_at_the_longest_k():
+    """-8 x -8 over K = 131040 (the scaled products reach 16384 K = 2^31 - 524288 summed over the
+    warps of a CTA: each warp's partial sum is brought back to scale before they are added), and
+    -128 x -128 in INT8."""
+    M, N, K = 2, 40, 131040
+    A = np.full((M, K // 2), 0x88, dtype=np.uint8)
+    B = np.full((N, K // 2), 0x88, dtype=np.uint8)
+    assert np.all(run_gpu("s4", A, B, fill=-7) == 64 * K)
+    A8 = np.full((M, K), -128, dtype=np.int8)
+    B8 = np.full((N, K), -128, dtype=np.int8)
+    assert np.all(run_gpu("s8", A8, B8, fill=-7) == 16384 * K)
+
+
+def test_few_rows_one_hot_positions():
+    """Rows with a single non-zero value at every position of a 64-byte step: the order of K
+    inside the fragments must be the same on both sides."""
+    M, N, K = 16, 256, 512
+    vals_a = np.zeros((M, K), dtype=np.int8)
+    vals_b = np.zeros((N, K), dtype=np.int8)
+    for i in range(M):
+        vals_a[i, (37 * i) % K] = 1 + (i % 7)
+        vals_a[i, (37 * i + 129) % K] = -8
+    for j in range(N):
+        vals_b[j, j % K] = -3
+        vals_b[j, (j + 129) % K] = 7
+        if vals_b[j, (2 * j + 1) % K] == 0:
+            vals_b[j, (2 * j + 1) % K] = 2
+    A, B = synth.pack_s4(vals_a), synth.pack_s4(vals_b)
+    assert np.array_equal(run_gpu("s4", A, B, fill=-7), oracle.gemm_s4(A, B, K))
+    assert np.array_equal(run_gpu("s8", vals_a, vals_b, fill=-7), oracle.gemm_s8(vals_a, vals_b))
+
+
+@pytest.mark.parametrize("prec", ["s8", "s4"])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.float16])
+@pytest.mark.parametrize("M,N,K", [(12, 1300, 1056), (900, 5, 512)])
+def test_few_rows_dequantised_outputs(prec, out_dtype, M, N, K):
+    A, B = _make(prec, M, N, K, seed=8)
+    g = np.random.Generator(np.random.PCG64(8))
+    rs = (g.uniform(0.5, 2.0, M) * 1e-2).astype(np.float32)
+    cs = (g.uniform(0.5, 2.0, N) * 1e-2).astype(np.float32)
+    C = torch.full((M, N), float("nan"), dtype=out_dtype, device="cuda")
+    fn = binding.gemm_s4_dequant if prec == "s4" else binding.gemm_s8_dequant
+    fn(to_dev(A), to_dev(B), to_dev(rs), to_dev(cs), C, out_dtype)
+    torch.cuda.synchronize()
+    acc = oracle.gemm_s4_i64(A, B, K) if prec == "s4" else oracle.gemm_s8(A, B).astype(np.int64)
+    ok, worst = oracle.dequant_check(C.cpu().numpy(), oracle.dequant_ref(acc, rs, cs),
+                                     out_dtype == torch.float16)
+    assert ok, worst
+
+
+def test_few_rows_automatic_rule():
+    binding.gemm_set_kernel_family(0)
+    few = lambda prec, M, N, K: binding.gemm_query_config(prec, M, N, K).startswith("few_rows")
+    assert few("s4", 16, 8192, 8192) and few("s4", 1, 28672, 8192) and few("s4", 4096, 9, 1024)
+    assert not few("s4", 17, 8192, 8192) and not few("s4", 16, 500, 8192)
+    assert few("s8", 8, 2048, 4096) and few("s8", 16, 4096, 8192)
+    assert not few("s8", 16, 8192, 8192) and not few("s8", 16, 2048, 4096)
+    assert not few("fp16", 1, 8192, 8192)
+    binding.gemm_set_s4_scheme(2)          # a forced INT4 scheme means the tile kernels
+    assert not few("s4", 16, 8192, 8192)
+    binding.gemm_set_s4_scheme(0)
+    M, N, K = 16, 4096, 1056
+    A, B = synth.s4_uniform(M, N, K, seed=2)
+    check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7))
+
+
+def test_few_rows_in_a_cuda_graph():
+    """No scratch, no zeroing launch: a captured call is one kernel node and replays exactly."""
+    M, N, K = 16, 2100, 2048
+    A, B = synth.s4_uniform(M, N, K, seed=5)
+    dA, dB = to_dev(A), to_dev(B)
+    C = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            binding.gemm_s4(dA, dB, C, stream=side)
+    ref = oracle.gemm_s4(A, B, K)
+    for rep in range(3):
+        C.fill_(-7)
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(C.cpu().numpy(), ref)

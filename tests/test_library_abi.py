@@ -126,6 +126,23 @@ def test_selector_invariants_over_many_shapes(lib):
         for M, N, K in itertools.product(dims, dims, ks):
             text = binding.gemm_query_config(prec, M, N, K)
             c = _parse(text)
+            if text.startswith("few_rows"):   # the kernel for a short side of up to 16 rows
+                short, long_ = min(M, N), max(M, N)
+                assert prec != "fp16" and short <= 16 and long_ >= 512 and c["short_rows"] == short
+                if prec == "s8":
+                    assert long_ * K <= 32 << 20 and (short <= 8 or long_ >= 4096)
+                rows = c["rows_per_block"]
+                assert rows == (16 if short <= 8 else 32) and c["blocks"] == -(-long_ // rows)
+                row_bytes = K // 2 if prec == "s4" else K
+                w, d = c["warps"], c["depth"]
+                assert w in (1, 2, 4, 8, 16) and 2 <= d <= 8
+                assert w == 1 or -(-row_bytes // 64) >= 2 * w      # two 64-byte steps per warp
+                nt, mt = (1 if short <= 8 else 2), rows // 16
+                smem = d * (2 * mt + nt) * w * 512 + w * 8 * nt * (16 * mt + 4) * 4
+                per_sm = min((227 * 1024) // (smem + 1024), 64 // w, 32)
+                assert per_sm >= 1 and 1 <= c["ctas"] <= min(c["blocks"], per_sm * 148)
+                assert c["ctas"] == c["blocks"] or c["ctas"] % 148 == 0
+                continue
             if "swap_ab" in text:        # the tile is described in the kernel's orientation
                 assert N >= 1024 and M <= (32 if prec == "fp16" and N < 16384 else 64)
                 M, N = N, M
@@ -183,6 +200,11 @@ def test_selector_headline_choices(lib):
         binding.gemm_set_kernel_family(0)
     dec = _parse(binding.gemm_query_config("s8", 16, 8192, 8192))
     assert dec["split_k"] > 1 and dec["split_tiles"] == dec["tiles"]
+    few = binding.gemm_query_config("s4", 16, 8192, 8192)
+    assert few.startswith("few_rows") and "s4=in_registers" in few
+    assert binding.gemm_query_config("s8", 8, 4096, 4096).startswith("few_rows")
+    assert not binding.gemm_query_config("s8", 16, 28672, 8192).startswith("few_rows")
+    assert not binding.gemm_query_config("s4", 17, 8192, 8192).startswith("few_rows")
     tail = _parse(binding.gemm_query_config("fp16", 4096, 4096, 8192))
     assert tail["split_k"] == 2 and tail["split_tiles"] == 256 % 74
     binding.gemm_set_config_override(0, 0, 0, 1)
