@@ -815,7 +815,7 @@ template <bool S4, int NT, int EPI>
 int launch_few_rows_nt(DeviceState* s, FewRowsParams& p, const FewRowsShape& f,
                        cudaStream_t stream) {
   constexpr int MT = FEW_ROWS_MT(NT);
-  constexpr int variant = 224 + (S4 ? 9 : 0) + (NT == 1 ? 0 : NT == 2 ? 3 : 6) + EPI;
+  constexpr int variant = 256 + (S4 ? 9 : 0) + (NT == 1 ? 0 : NT == 2 ? 3 : 6) + EPI;  // attr_set bits 256..273
   auto kernel = few_rows_kernel<S4, MT, NT, EPI>;
   if (!(s->attr_set[variant >> 6].load(std::memory_order_relaxed) & (1ull << (variant & 63)))) {
     const cudaError_t e = cudaFuncSetAttribute(

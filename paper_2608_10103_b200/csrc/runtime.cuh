@@ -38,7 +38,7 @@ struct DeviceState {
   int* status_ptr = nullptr;
   unsigned long long* trace_ptr = nullptr;
   // bit i: dynamic-smem attribute set for kernel variant i (setting it twice is harmless)
-  std::atomic<uint64_t> attr_set[4] = {};
+  std::atomic<uint64_t> attr_set[5] = {};
   // clusters of four CTAs (cluster split-K) the device runs at once, per kind and output
   // mode; 0 = not asked yet
   std::atomic<int> quad_clusters[2][4] = {};

@@ -1,6 +1,6 @@
 """Seeded walk over shapes of the kind that trigger the selector's special cases in the automatic
 mode -- a sparsely filled last wave split along K, even shares, the hybrid INT4 form, exchanged
-operands, the pre-pass -- each result checked against the oracle on a sample of rows, and the
+operands, the pre-pass, the kernel for a few rows -- each result checked against the oracle on a sample of rows, and the
 walk as a whole checked to have met every one of those cases."""
 import numpy as np
 import pytest
@@ -17,7 +17,7 @@ def _shape(g):
     if kind == 5:      # INT4, a short M against a large N K: the hybrid form of the fused pair kernel
         return (int(g.choice([256, 384, 512])), int(g.integers(24000, 29000)), 8192), "s4"
     if kind == 4:      # INT4, few rows, 1.3 ... 1.9 tiles of 128 rows per SM: even shares
-        return (int(g.choice([8, 16, 32])), int(g.integers(24000, 30000)), int(g.choice([4096, 4128, 8192]))), "s4"
+        return (int(g.choice([24, 32, 32])), int(g.integers(24000, 30000)), int(g.choice([4096, 4128, 8192]))), "s4"
     if kind == 0:      # few rows against a wide N
         return (int(g.choice([1, 3, 8, 16, 24, 32, 48, 64, 100, 128])), int(g.integers(8000, 30000)),
                 int(g.choice([1024, 2048, 4096, 4128, 8192]))), None
@@ -49,10 +49,10 @@ def test_automatic_paths_over_a_seeded_walk_of_shapes():
         rows = np.unique(np.concatenate([g.choice(M, size=min(10, M), replace=False), [0, M - 1]])).astype(np.int32)
         cfg = binding.gemm_query_config(prec, M, N, K)
         m = dict(kv.split("=") for kv in cfg.split() if "=" in kv)
-        for f in ("even_share", "a=int8_image", "fused_unpack", "prepass", "swap_ab"):
+        for f in ("even_share", "a=int8_image", "fused_unpack", "prepass", "swap_ab", "few_rows"):
             if f in cfg:
                 met.add(f)
-        if int(m["split_k"]) > 1 and m["split_tiles"] != m["tiles"]:
+        if "few_rows" not in cfg and int(m["split_k"]) > 1 and m["split_tiles"] != m["tiles"]:
             met.add("tail_split_deep" if int(m["split_k"]) > 4 else "tail_split")
         C = torch.full((M, N), float("nan") if prec == "fp16" else -7,
                        dtype=torch.float32 if prec == "fp16" else torch.int32, device="cuda")
@@ -70,4 +70,4 @@ def test_automatic_paths_over_a_seeded_walk_of_shapes():
             assert np.array_equal(got.astype(np.int64), exact), what
     assert binding.gemm_last_device_status() == 0
     assert met >= {"even_share", "a=int8_image", "fused_unpack", "prepass", "swap_ab", "tail_split",
-                   "tail_split_deep"}, met
+                   "tail_split_deep", "few_rows"}, met

@@ -23,6 +23,7 @@ def _clean():
     binding.gemm_set_s4_scheme(0)
     binding.gemm_set_l2_policy(11)
     binding.gemm_set_swap_ab(0)
+    binding.gemm_set_kernel_family(0)
     assert binding.gemm_last_device_status() == 0
 
 
@@ -35,6 +36,8 @@ def _share(cfg):
 # end inside tiles in every combination
 @pytest.mark.parametrize("M,N,K", [(32, 28672, 4128), (64, 28000, 4096), (16, 24000, 4128), (8, 29440, 8192)])
 def test_even_shares_exact(M, N, K):
+    if M <= 16:       # the automatic route there is the kernel for a few rows: ask for the tiles
+        binding.gemm_set_kernel_family(1)
     cfg = binding.gemm_query_config("s4", M, N, K)
     assert "fused_unpack" in cfg and _share(cfg) >= 16, cfg
     A, B = synth.s4_uniform(M, N, K, seed=M + K)
@@ -65,7 +68,9 @@ def test_even_shares_with_operands_not_exchanged_and_forced_widths():
 
 def test_even_shares_not_taken_where_they_do_not_pay():
     assert _share(binding.gemm_query_config("s4", 256, 256, 8192)) == 0      # one tile, no split chosen
+    binding.gemm_set_kernel_family(1)
     assert _share(binding.gemm_query_config("s4", 16, 8192, 8192)) == 0      # 16 -> 14 slots per SM: not worth a second piece
+    binding.gemm_set_kernel_family(0)
     assert _share(binding.gemm_query_config("s4", 64, 21000, 1056)) == 0     # shares of 6 slots: measured slower
     assert _share(binding.gemm_query_config("s4", 8192, 8192, 8192)) == 0    # pre-pass route
     assert _share(binding.gemm_query_config("s4", 256, 28672, 8192)) == 0    # CTA-pair tiles

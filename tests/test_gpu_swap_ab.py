@@ -74,8 +74,9 @@ def test_swapped_output_variants():
 
 def test_automatic_choice_for_few_rows():
     binding.gemm_set_swap_ab(0)
-    cfg = binding.gemm_query_config("s4", 16, 8192, 8192)
+    cfg = binding.gemm_query_config("s4", 24, 8192, 8192)
     assert "fused_unpack" in cfg and "swap_ab" in cfg
+    assert binding.gemm_query_config("s4", 16, 8192, 8192).startswith("few_rows")
     assert "swap_ab" in binding.gemm_query_config("s4", 64, 8192, 8192)
     assert "swap_ab" not in binding.gemm_query_config("s4", 128, 8192, 8192)
     assert "swap_ab" in binding.gemm_query_config("s8", 64, 8192, 8192)
@@ -86,7 +87,7 @@ def test_automatic_choice_for_few_rows():
     assert "swap_ab" not in binding.gemm_query_config("fp16", 128, 8192, 8192)
     assert "swap_ab" not in binding.gemm_query_config("s8", 16, 512, 8192)
     assert "swap_ab" not in binding.gemm_query_config("s8", 2048, 2048, 2048)
-    M, N, K = 16, 8192, 4096
+    M, N, K = 24, 8192, 4096
     for prec in synth.PRECISIONS:
         A, B = synth.make(prec, M, N, K, seed=12)
         C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
