@@ -635,16 +635,19 @@ def run_few_rows(args):
     torch.cuda.set_device(0)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     hbm = measured_peaks()["hbm_gbs"]
-    shapes = [(1, 8192, 8192), (16, 8192, 8192), (64, 8192, 8192), (16, 4096, 16384),
-              (128, 16384, 4096), (32, 28672, 8192)]
+    shapes = [(1, 8192, 8192), (8, 8192, 8192), (16, 8192, 8192), (64, 8192, 8192), (16, 4096, 16384),
+              (8, 4096, 4096), (128, 16384, 4096), (16, 28672, 8192), (32, 28672, 8192)]
     if args.shape:
         shapes = [tuple(int(x) for x in args.shape.split(","))]
     routes = {"fp16": [("selector default", 0, 0, "raw"), ("operands not exchanged", 0, 1, "raw"),
                        ("FP16 output, selector default", 0, 0, "out16")],
               "s8": [("selector default", 0, 0, "raw"), ("operands not exchanged", 0, 1, "raw"),
+                     ("tile kernels, operands exchanged", 0, 2, "raw"),
+                     ("kernel for a few rows where it exists (up to 32)", 0, 0, "raw", 3),
                      ("dequantised to FP16, selector default", 0, 0, "out16")],
               "s4": [("selector default", 0, 0, "raw"), ("pre-pass + INT8 GEMM", 1, 1, "raw"),
-                     ("expanded in the kernel, operands exchanged", 2, 2, "raw"),
+                     ("tile kernels: expanded in the kernel, operands exchanged", 2, 2, "raw"),
+                     ("kernel for a few rows where it exists (up to 32)", 0, 0, "raw", 3),
                      ("expanded in the kernel, both operands packed on CTA-pair tiles", 5, 0, "raw"),
                      ("dequantised to FP16, selector default", 0, 0, "out16")]}
     for M, N, K in shapes:
@@ -670,10 +673,11 @@ def run_few_rows(args):
                 else:
                     binding.gemm_s4_dequant(dA, b, rs, cs, C16, torch.float16, stream=stream)
 
-            for name, scheme, swap, mode in routes[prec]:
+            for name, scheme, swap, mode, *rest in routes[prec]:
                 algo_bytes = A.nbytes + B.nbytes + M * N * (4 if mode == "raw" else 2)
                 binding.gemm_set_s4_scheme(scheme)
                 binding.gemm_set_swap_ab(swap)
+                binding.gemm_set_kernel_family(rest[0] if rest else 0)
                 for _ in range(3):
                     call(mode, dB)
                 torch.cuda.synchronize()
@@ -706,6 +710,7 @@ def run_few_rows(args):
                     flush=True)
     binding.gemm_set_s4_scheme(0)
     binding.gemm_set_swap_ab(0)
+    binding.gemm_set_kernel_family(0)
     if binding.gemm_last_device_status() != 0:
         raise SystemExit("bench.py: a kernel reported a barrier timeout")
 

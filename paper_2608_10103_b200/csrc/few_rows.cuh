@@ -163,25 +163,32 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   const int steps = (p.row_bytes + 63) >> 6;
   const int my_steps = warp < steps ? (steps - warp + warps - 1) / warps : 0;
 
-  // The copies walk (block, step) in the order the arithmetic will; f_* is where they stand.
+  // The copies walk (block, step) in the order the arithmetic will; f_* is where they stand,
+  // lrow[] this thread's rows of the block the copies are in (piece r: fragment rows g + 8 r).
   int f_block = 0, f_step = 0, f_slot = 0;
+  const uint8_t* lrow[2 * MT];
+  auto rows_of = [&](int block) {
+    const int l0 = (static_cast<int>(blockIdx.x) + block * grid) * BLOCK_ROWS;
+#pragma unroll
+    for (int r = 0; r < 2 * MT; ++r)
+      lrow[r] = p.L + static_cast<long long>(min(l0 + g + 8 * r, last_l)) * p.l_pitch;
+  };
+  rows_of(0);
   auto fetch = [&]() {  // this thread's pieces of the next step into the next ring slot
     if (f_block < my_blocks && my_steps > 0) {
-      const int l0 = (static_cast<int>(blockIdx.x) + f_block * grid) * BLOCK_ROWS;
       const int off = (warp + f_step * warps) * 64 + t * 16;
       const bool in = off < p.row_bytes;  // rows are whole 16-byte pieces; beyond K: zeros
       const int at = in ? off : 0, bytes = in ? 16 : 0;
       const uint32_t slot = ring + static_cast<uint32_t>(f_slot * PIECES) * piece_pitch;
 #pragma unroll
-      for (int r = 0; r < 2 * MT; ++r)  // piece r: fragment rows g + 8 r
-        cp_async_16_cg(slot + static_cast<uint32_t>(r) * piece_pitch,
-                       p.L + static_cast<long long>(min(l0 + g + 8 * r, last_l)) * p.l_pitch + at, bytes);
+      for (int r = 0; r < 2 * MT; ++r)
+        cp_async_16_cg(slot + static_cast<uint32_t>(r) * piece_pitch, lrow[r] + at, bytes);
 #pragma unroll
       for (int j = 0; j < NT; ++j)
         cp_async_16_ca(slot + static_cast<uint32_t>(2 * MT + j) * piece_pitch, sp[j] + at, bytes);
       if (++f_step == my_steps) {
         f_step = 0;
-        ++f_block;
+        rows_of(++f_block);  // (one block past the end on the last step: clamped, never read)
       }
       f_slot = f_slot + 1 == depth ? 0 : f_slot + 1;
     }
