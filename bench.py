@@ -664,7 +664,9 @@ def run_few_rows(args):
             cs = torch.rand(N, device="cuda") + 0.5
 
             def call(mode, b, stream=None):
-                if mode == "raw":
+                if mode == "probe":
+                    binding.gemm_debug_read_probe(b, stream=stream)
+                elif mode == "raw":
                     binding.gemm(prec, dA, b, C32, stream=stream)
                 elif prec == "fp16":
                     binding.gemm_fp16_f16out(dA, b, C16, stream=stream)
@@ -673,8 +675,11 @@ def run_few_rows(args):
                 else:
                     binding.gemm_s4_dequant(dA, b, rs, cs, C16, torch.float16, stream=stream)
 
-            for name, scheme, swap, mode, *rest in routes[prec]:
+            probe = ("read-only probe: a kernel that reads B once and does nothing else", 0, 0, "probe")
+            for name, scheme, swap, mode, *rest in routes[prec] + [probe]:
                 algo_bytes = A.nbytes + B.nbytes + M * N * (4 if mode == "raw" else 2)
+                if mode == "probe":
+                    algo_bytes = B.nbytes
                 binding.gemm_set_s4_scheme(scheme)
                 binding.gemm_set_swap_ab(swap)
                 binding.gemm_set_kernel_family(rest[0] if rest else 0)

@@ -88,7 +88,13 @@ int gemm_s8(int M, int N, int K, const int8_t* A, const int8_t* B, int32_t* C,
  * bytes, B: N rows of K/2 bytes; element k of a row is bits [4*(k&1), 4*(k&1)+4)
  * of byte k>>1 (low nibble first), two's complement.
  *
- * Blackwell's tcgen05.mma has no 4-bit integer kind.  Most problems: a kernel
+ * Blackwell's tcgen05.mma has no 4-bit integer kind.  A problem with at most 16
+ * rows on one side (M or N) against 512 or more on the other never reaches it:
+ * the long operand goes from global memory straight into the fragments of the
+ * warp-level integer MMA, its nibbles expanded in registers, in one launch that
+ * needs no scratch and zeroes nothing (gemm_s8 does the same while the long
+ * operand has at most 32 MB; see gemm_set_kernel_family in b200gemm_debug.h).
+ * Most other problems: a kernel
  * variant expands the nibbles on the way to the MMAs (see gemm_set_s4_scheme in
  * b200gemm_debug.h for the rule and the switch).  The rest (a short K, less than
  * a wave of tiles with more than 1024 rows and columns, a few in-between
@@ -255,8 +261,11 @@ int gemm_unpack_s4(int rows, int K, const uint8_t* packed, int8_t* out, size_t o
  * terminated, truncated to len); for INT4 followed by the route
  * (" prepass=unpack_s4" or " s4=fused_unpack"), and by " swap_ab" when the
  * kernel runs on exchanged operands (the tile is then described in the
- * kernel's orientation).  Describes the raw 32-bit outputs (gemm_fp16,
- * gemm_s8, gemm_s4).  Host only, no GPU work.
+ * kernel's orientation).  An integer problem that goes to the kernel for a few
+ * rows instead of a tile kernel reads "few_rows rows_per_block=32 blocks=256
+ * short_rows=16 warps=8 depth=3 ctas=256 kind=i8" (" s4=in_registers" for INT4).
+ * Describes the raw 32-bit outputs (gemm_fp16, gemm_s8, gemm_s4).  Host only,
+ * no GPU work.
  */
 int gemm_query_config(int precision, int M, int N, int K, char* buf, int len);
 

@@ -62,6 +62,20 @@ int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k);
  * bytes for FP16 (K >= 6144) or 64 for the integer kinds (K >= 8192; the INT4
  * pre-pass route included).  The paper fixes one tiling for every size
  * (Sec. III-A); this is the corresponding ablation axis here.
+ *
+ * The integer precisions have a third kernel, for problems with a few rows on
+ * one side, which are bound by reading the long operand once: every thread
+ * copies the 16-byte pieces its own mma.sync m16n8k32 (s8 x s8 -> s32) fragments
+ * need into a private ring in shared memory (cp.async, several steps ahead),
+ * loads them back and, for INT4, expands the nibbles in registers; a CTA owns
+ * 16 or 32 rows of the long operand over the whole of K, sums its warps'
+ * results and writes its part of C once.  Family 0 takes it for a short side
+ * of at most 16 rows against at least 512 -- INT4 always, INT8 while the long
+ * operand has at most 32 MB (and, from nine rows on, at least 4096 rows); 3 =
+ * wherever it exists (a short side of at most 32 rows); 1 and 2 never, nor do
+ * calls with a forced tile shape, operand order or INT4 scheme, or traced ones.
+ * gemm_query_config describes such a call as "few_rows rows_per_block=..
+ * blocks=.. short_rows=.. warps=.. depth=.. ctas=..".
  */
 int gemm_set_kernel_family(int family);
 
@@ -243,6 +257,18 @@ int gemm_debug_counters(long long* out, int n);
  */
 int gemm_debug_host_cost(int precision, int M, int N, int K, const void* A, const void* B, void* C,
                          gemm_stream_t stream, int calls, double* ns_per_call);
+
+/*
+ * Measurement aid for calls that are bound by reading one operand once (the
+ * problems with a few rows): enqueues a kernel on `stream` that reads `bytes`
+ * bytes (a multiple of 16) at `data` (device memory, 16-byte aligned) with
+ * 16-byte loads and keeps nothing.  Launched like the GEMMs (it may start while
+ * the grid in front drains and waits for it before its first load), so its
+ * time in a given harness -- launch, first-byte latency and tail included -- is
+ * what a GEMM call that only had to read that operand could at best take there.
+ * Writes nothing.
+ */
+int gemm_debug_read_probe(const void* data, size_t bytes, gemm_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -23,7 +23,7 @@ EXPORTS = (
     "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
     "gemm_fp16_f16out", "gemm_s8_dequant", "gemm_s4_dequant", "gemm_host", "gemm_host_release",
     "gemm_s4_static", "gemm_s4_static_capacity", "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
-    "gemm_set_config_override", "gemm_set_kernel_family", "gemm_set_s4_scheme", "gemm_set_swap_ab", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_set_stages_override", "gemm_debug_counters", "gemm_debug_host_cost",
+    "gemm_set_config_override", "gemm_set_kernel_family", "gemm_set_s4_scheme", "gemm_set_swap_ab", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_set_stages_override", "gemm_debug_counters", "gemm_debug_host_cost", "gemm_debug_read_probe",
     "gemm_last_device_status", "gemm_read_device_status", "gemm_last_cuda_error",
     "gemm_status_string", "gemm_version",
 )
@@ -77,6 +77,7 @@ def lib() -> ctypes.CDLL:
         L.gemm_set_stages_override.argtypes = [i]
         L.gemm_debug_counters.argtypes = [ctypes.POINTER(ctypes.c_longlong), i]
         L.gemm_debug_host_cost.argtypes = [i, i, i, i, vp, vp, vp, vp, i, ctypes.POINTER(ctypes.c_double)]
+        L.gemm_debug_read_probe.argtypes = [vp, sz, vp]
         L.gemm_read_device_status.argtypes = [vp, vp]
         L.gemm_set_swap_ab.argtypes = [i]
         L.gemm_set_l2_policy.argtypes = [i]
@@ -309,7 +310,9 @@ def gemm_set_config_override(bn: int = 0, group_m: int = 0, cta_group: int = 0, 
 
 
 def gemm_set_kernel_family(family: int = 0):
-    """Kernel for large problems: 0 = automatic, 1 = 256 x 256 tile per CTA pair, 2 = 512 x 256."""
+    """Kernel family: 0 = automatic, 1 = 256 x 256 tile per CTA pair, 2 = 512 x 256 (large
+    problems); 3 = the integer kernel for a few rows wherever it exists (a short side of up to
+    32 rows; 1 and 2 never take it)."""
     _check(lib().gemm_set_kernel_family(int(family)), "gemm_set_kernel_family")
 
 
@@ -337,6 +340,15 @@ def gemm_debug_host_cost(precision: str, A: torch.Tensor, B: torch.Tensor, C: to
                                       C.data_ptr(), _stream_handle(stream), int(calls),
                                       ctypes.byref(out)), "gemm_debug_host_cost")
     return float(out.value)
+
+
+def gemm_debug_read_probe(data: torch.Tensor, stream=None):
+    """Enqueues a kernel that reads `data` (device tensor, a multiple of 16 bytes) once and
+    keeps nothing: the time a call bound by reading that operand could at best take."""
+    if not data.is_cuda or not data.is_contiguous():
+        raise ValueError("data must be a contiguous CUDA tensor")
+    _check(lib().gemm_debug_read_probe(data.data_ptr(), data.numel() * data.element_size(),
+                                       _stream_handle(stream)), "gemm_debug_read_probe")
 
 
 def gemm_read_device_status(host_out: torch.Tensor, stream=None):

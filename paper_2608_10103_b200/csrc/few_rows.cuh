@@ -297,4 +297,31 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   cp_async_wait<0>();
 }
 
+// Measurement aid: reads `bytes` (a multiple of 16) once with 16-byte loads, eight in flight per
+// thread, and keeps nothing -- what a call bound by reading one operand could at best take in a
+// given harness (launch, first-byte latency and tail included).  `sink` is never written.
+__global__ void __launch_bounds__(256) read_probe_kernel(const uint8_t* data, size_t bytes,
+                                                         unsigned* sink, int wait_prior_grid) {
+  if (threadIdx.x == 0) ptx::grid_dep_launch_dependents();
+  if (wait_prior_grid) ptx::grid_dep_wait();
+  constexpr int U = 8;
+  const size_t per_cta = static_cast<size_t>(blockDim.x) * 16 * U;
+  unsigned acc = 0;
+  for (size_t base = blockIdx.x * per_cta; base < bytes; base += gridDim.x * per_cta) {
+    uint4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const size_t at = base + (static_cast<size_t>(u) * blockDim.x + threadIdx.x) * 16;
+      v[u] = make_uint4(0, 0, 0, 0);
+      if (at < bytes)
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(v[u].x), "=r"(v[u].y), "=r"(v[u].z), "=r"(v[u].w)
+                     : "l"(data + at));
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) acc += v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+  }
+  if (acc == 0x9e3779b9u && bytes == 1) *sink = acc;  // never true: keeps the loads alive
+}
+
 }  // namespace b200gemm

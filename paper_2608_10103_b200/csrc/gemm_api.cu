@@ -345,6 +345,27 @@ int gemm_debug_host_cost(int precision, int M, int N, int K, const void* A, cons
   return GEMM_OK;
 }
 
+int gemm_debug_read_probe(const void* data, size_t bytes, gemm_stream_t stream) {
+  if (!data || bytes == 0 || (bytes & 15) || (reinterpret_cast<uintptr_t>(data) & 15))
+    return GEMM_ERR_INVALID_ARG;
+  DeviceState* s = nullptr;
+  int rc = device_state(&s);
+  if (rc != GEMM_OK) return rc;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(8 * s->num_sms), 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = reinterpret_cast<cudaStream_t>(stream);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;  // launched like the GEMMs: may start early, waits for the grid in front
+  const cudaError_t e =
+      cudaLaunchKernelEx(&cfg, read_probe_kernel, static_cast<const uint8_t*>(data), bytes,
+                         reinterpret_cast<unsigned*>(s->status_ptr), 1);
+  return e == cudaSuccess ? GEMM_OK : cuda_fail(e);
+}
+
 int gemm_read_device_status(int* host_out, gemm_stream_t stream) {
   if (!host_out) return GEMM_ERR_INVALID_ARG;
   DeviceState* s = nullptr;

@@ -133,3 +133,18 @@ def test_host_cost_probe_runs_real_calls_and_rejects_bad_arguments():
         with pytest.raises(binding.GemmError) as e:
             binding.gemm_debug_host_cost("s8", dA, dB, C, calls=calls)
         assert e.value.code == -1
+
+
+def test_read_probe_reads_and_writes_nothing():
+    """The read-only probe takes any 16-byte multiple, leaves the data and the status word alone,
+    and rejects sizes and addresses that are not 16-byte multiples."""
+    data = torch.arange(1 << 20, dtype=torch.int32, device="cuda")
+    before = data.clone()
+    for n in (4, 4 * 37, 1 << 20):
+        binding.gemm_debug_read_probe(data[:n])
+    torch.cuda.synchronize()
+    assert torch.equal(data, before) and binding.gemm_last_device_status() == 0
+    with pytest.raises(binding.GemmError):
+        binding.gemm_debug_read_probe(data[:3])
+    with pytest.raises(binding.GemmError):
+        binding.gemm_debug_read_probe(data[1:5])
