@@ -9,11 +9,11 @@
 // against 8 rows of the short one per instruction) from registers, and every thread fetches
 // exactly the 16-byte pieces its own fragment registers need.
 //
-// Work split: one CTA per 16 rows of the long operand over the whole of K; its warps take the
-// 64-byte steps of K in turn (warp w: steps w, w + warps, ...), so that the CTA as a whole reads
-// a window of warps x depth x 64 contiguous bytes of each of its rows at any moment.  Every CTA
-// sums its warps' results in shared memory and writes its 16 columns (or rows) of C itself: no
-// zeroed C, no atomics, no second launch.
+// Work split: one CTA per 16 (32) rows of the long operand over the whole of K; its warps share
+// K in 64-byte steps, each warp a contiguous run of them (so that a warp streams 64 x steps
+// consecutive bytes of each of its rows: taking the steps in turn, warp w: w, w + warps, ...,
+// measured 2-8 % slower).  Every CTA sums its warps' results in shared memory and writes its 16
+// (32) columns (or rows) of C itself: no zeroed C, no atomics, no second launch.
 //
 // Latency: a step's pieces travel by cp.async into a ring of `depth` slots that is private to the
 // thread (nobody else reads them, so no barrier is involved: the thread waits for its own copy
@@ -161,7 +161,10 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   const int grid = static_cast<int>(gridDim.x);
   const int my_blocks = (blocks - static_cast<int>(blockIdx.x) + grid - 1) / grid;
   const int steps = (p.row_bytes + 63) >> 6;
-  const int my_steps = warp < steps ? (steps - warp + warps - 1) / warps : 0;
+  // warp w: the steps [w, w + 1) * ceil(steps / warps) -- a contiguous run of each row
+  const int per_warp = (steps + warps - 1) / warps;
+  const int first_step = warp * per_warp;
+  const int my_steps = max(0, min(steps, first_step + per_warp) - first_step);
 
   // The copies walk (block, step) in the order the arithmetic will; f_* is where they stand,
   // lrow[] this thread's rows of the block the copies are in (piece r: fragment rows g + 8 r).
@@ -176,7 +179,7 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   rows_of(0);
   auto fetch = [&]() {  // this thread's pieces of the next step into the next ring slot
     if (f_block < my_blocks && my_steps > 0) {
-      const int off = (warp + f_step * warps) * 64 + t * 16;
+      const int off = (first_step + f_step) * 64 + t * 16;
       const bool in = off < p.row_bytes;  // rows are whole 16-byte pieces; beyond K: zeros
       const int at = in ? off : 0, bytes = in ? 16 : 0;
       const uint32_t slot = ring + static_cast<uint32_t>(f_slot * PIECES) * piece_pitch;

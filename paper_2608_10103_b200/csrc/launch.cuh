@@ -747,11 +747,11 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
 // zeroed).  Automatic for a short side of up to 16 rows against 512 or more: INT4 always (it
 // measured 0.45-0.98 of the tile kernels' time for 2048 <= N <= 28672, K = 4096 / 8192: there the
 // tile kernels are bound by expanding the nibbles in shared memory); INT8 while the long operand
-// has at most 32 MB and, from nine rows on, at least 4096 rows (0.68-0.92 of the tile kernels'
-// time; level at 64 MB, and 1.1-1.3 x slower beyond, where the tile kernels' bulk copies reach
-// 0.86 of the HBM bandwidth and this kernel's 16-byte copies 0.7).  gemm_set_kernel_family(3)
-// takes it wherever it exists (a short side of up to 32 rows), families 1 and 2, forced tile
-// shapes, forced operand orders, every forced INT4 scheme and the traced runs never.
+// has at most 64 MB (0.65-0.96 of the tile kernels' time; level from there to 128 MB, and up to
+// 1.1 x slower beyond, where the tile kernels' bulk copies reach 0.86 of the HBM bandwidth).
+// gemm_set_kernel_family(3) takes it wherever it exists (a short side of up to 32 rows),
+// families 1 and 2, forced tile shapes, forced operand orders, every forced INT4 scheme and the
+// traced runs never.
 constexpr int FEW_ROWS_AUTO = 16;
 constexpr int FEW_ROWS_MAX = 32;
 bool few_rows_wanted(int M, int N, int K, bool packed_s4, const OutputSpec& out) {
@@ -764,7 +764,7 @@ bool few_rows_wanted(int M, int N, int K, bool packed_s4, const OutputSpec& out)
   if (fam == 3) return shorter <= FEW_ROWS_MAX;
   if (fam != 0 || shorter > FEW_ROWS_AUTO || longer < 512) return false;
   if (packed_s4) return true;
-  return static_cast<long long>(longer) * K <= (32LL << 20) && (shorter <= 8 || longer >= 4096);
+  return static_cast<long long>(longer) * K <= (64LL << 20);
 }
 
 // Shape of a few-rows launch.  MT groups of 16 long rows per CTA: two from nine short rows on,

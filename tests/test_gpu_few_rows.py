@@ -126,8 +126,8 @@ def test_few_rows_automatic_rule():
     few = lambda prec, M, N, K: binding.gemm_query_config(prec, M, N, K).startswith("few_rows")
     assert few("s4", 16, 8192, 8192) and few("s4", 1, 28672, 8192) and few("s4", 4096, 9, 1024)
     assert not few("s4", 17, 8192, 8192) and not few("s4", 16, 500, 8192)
-    assert few("s8", 8, 2048, 4096) and few("s8", 16, 4096, 8192)
-    assert not few("s8", 16, 8192, 8192) and not few("s8", 16, 2048, 4096)
+    assert few("s8", 8, 2048, 4096) and few("s8", 16, 4096, 8192) and few("s8", 16, 8192, 8192)
+    assert not few("s8", 16, 12288, 8192) and not few("s8", 17, 2048, 4096)
     assert not few("fp16", 1, 8192, 8192)
     binding.gemm_set_s4_scheme(2)          # a forced INT4 scheme means the tile kernels
     assert not few("s4", 16, 8192, 8192)
