@@ -87,6 +87,20 @@ __device__ __forceinline__ void cp_async_16_ca(uint32_t dst, const uint8_t* src,
   asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes)
                : "memory");
 }
+__device__ __forceinline__ uint4 ld_stream_16(const uint8_t* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint4 ld_cached_16(const uint8_t* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
 __device__ __forceinline__ void cp_async_commit() {
   asm volatile("cp.async.commit_group;" ::: "memory");
 }
@@ -127,11 +141,12 @@ __device__ __forceinline__ uint32_t high_nibbles_x16(uint32_t w) { return w & 0x
 // S4: packed 4-bit operands (else int8).  MT: groups of 16 long rows per CTA (a warp holds the
 // fragments of all of them and uses each short fragment MT times: the short operand, fetched
 // again by every CTA, costs 8 NT / (16 MT) of the long operand's bytes in requests).  NT: groups
-// of eight short rows.  EPI: as for the tile kernels.
+// of eight short rows.  EPI: as for the tile kernels.  HEAD: steps of the first block that go
+// through registers instead of the ring (costs 4 (2 MT + NT) registers each).
 // Dynamic shared memory: few_rows_ring_bytes + few_rows_red_bytes.  Any grid size: CTA c takes
 // the row blocks c, c + grid, ...; its copies run ahead across the block boundaries, so only
 // the first block of a CTA waits for the memory latency in full.
-template <bool S4, int MT, int NT, int EPI>
+template <bool S4, int MT, int NT, int EPI, int HEAD = 0>
 __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   using namespace few_rows_detail;
   extern __shared__ __align__(16) unsigned char few_rows_smem[];
@@ -177,6 +192,29 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
       lrow[r] = p.L + static_cast<long long>(min(l0 + g + 8 * r, last_l)) * p.l_pitch;
   };
   rows_of(0);
+  // The first HEAD steps of a CTA's first block travel through registers, on top of what the
+  // ring holds: that much more is in flight from the start, and the ring's first round trip
+  // begins one step further on.
+  constexpr int HN = HEAD > 0 ? HEAD : 1;
+  const int head = (HEAD > 0 && my_blocks > 0) ? min(HEAD, my_steps) : 0;
+  uint4 ha[HN][2 * MT], hb[HN][NT];
+  if constexpr (HEAD > 0) {
+#pragma unroll
+    for (int h = 0; h < HEAD; ++h) {
+      const int off = (first_step + h) * 64 + t * 16;
+      const bool in = h < head && off < p.row_bytes;
+#pragma unroll
+      for (int r = 0; r < 2 * MT; ++r)
+        ha[h][r] = in ? ld_stream_16(lrow[r] + off) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int j = 0; j < NT; ++j) hb[h][j] = in ? ld_cached_16(sp[j] + off) : make_uint4(0, 0, 0, 0);
+    }
+    f_step = head;
+    if (my_steps > 0 && f_step == my_steps) {
+      f_step = 0;
+      rows_of(++f_block);
+    }
+  }
   auto fetch = [&]() {  // this thread's pieces of the next step into the next ring slot
     if (f_block < my_blocks && my_steps > 0) {
       const int off = (first_step + f_step) * 64 + t * 16;
@@ -200,6 +238,41 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
 #pragma unroll 1
   for (int d = 0; d < depth; ++d) fetch();
 
+  // one step: the four words of every piece feed four (INT4) or two (INT8) rounds of MMAs
+  auto mac = [&](const uint4 (&a)[2 * MT], const uint4 (&b)[NT], int (&acc)[MT][NT][4]) {
+    if constexpr (S4) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        uint32_t b0[NT], b1[NT];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+          const uint32_t z = word_of(b[j], w);
+          b0[j] = low_nibbles_x16(z);
+          b1[j] = high_nibbles_x16(z);
+        }
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+          const uint32_t x = word_of(a[2 * m], w), y = word_of(a[2 * m + 1], w);
+          const uint32_t a0 = low_nibbles_x16(x), a2 = high_nibbles_x16(x);
+          const uint32_t a1 = low_nibbles_x16(y), a3 = high_nibbles_x16(y);
+#pragma unroll
+          for (int j = 0; j < NT; ++j) mma_s8_m16n8k32(acc[m][j], a0, a1, a2, a3, b0[j], b1[j]);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int w = 0; w < 4; w += 2) {
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+#pragma unroll
+          for (int j = 0; j < NT; ++j)
+            mma_s8_m16n8k32(acc[m][j], word_of(a[2 * m], w), word_of(a[2 * m + 1], w),
+                            word_of(a[2 * m], w + 1), word_of(a[2 * m + 1], w + 1),
+                            word_of(b[j], w), word_of(b[j], w + 1));
+      }
+    }
+  };
+
   int c_slot = 0;
 #pragma unroll 1
   for (int blk = 0; blk < my_blocks; ++blk) {
@@ -210,8 +283,17 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
       for (int j = 0; j < NT; ++j)
 #pragma unroll
         for (int v = 0; v < 4; ++v) acc[m][j][v] = 0;
+    int i0 = 0;
+    if constexpr (HEAD > 0) {
+      if (blk == 0) {
+#pragma unroll
+        for (int h = 0; h < HEAD; ++h)
+          if (h < head) mac(ha[h], hb[h], acc);
+        i0 = head;
+      }
+    }
 #pragma unroll 1
-    for (int i = 0; i < my_steps; ++i) {
+    for (int i = i0; i < my_steps; ++i) {
       cp_async_wait_all_but(depth - 1);  // all but the newest depth - 1 groups: this step has landed
       const uint32_t slot = ring + static_cast<uint32_t>(c_slot * PIECES) * piece_pitch;
       c_slot = c_slot + 1 == depth ? 0 : c_slot + 1;
@@ -223,37 +305,7 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
       for (int j = 0; j < NT; ++j)
         ptx::ld_shared_v4(slot + static_cast<uint32_t>(2 * MT + j) * piece_pitch, b[j].x, b[j].y,
                           b[j].z, b[j].w);
-      if constexpr (S4) {
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          uint32_t b0[NT], b1[NT];
-#pragma unroll
-          for (int j = 0; j < NT; ++j) {
-            const uint32_t z = word_of(b[j], w);
-            b0[j] = low_nibbles_x16(z);
-            b1[j] = high_nibbles_x16(z);
-          }
-#pragma unroll
-          for (int m = 0; m < MT; ++m) {
-            const uint32_t x = word_of(a[2 * m], w), y = word_of(a[2 * m + 1], w);
-            const uint32_t a0 = low_nibbles_x16(x), a2 = high_nibbles_x16(x);
-            const uint32_t a1 = low_nibbles_x16(y), a3 = high_nibbles_x16(y);
-#pragma unroll
-            for (int j = 0; j < NT; ++j) mma_s8_m16n8k32(acc[m][j], a0, a1, a2, a3, b0[j], b1[j]);
-          }
-        }
-      } else {
-#pragma unroll
-        for (int w = 0; w < 4; w += 2) {
-#pragma unroll
-          for (int m = 0; m < MT; ++m)
-#pragma unroll
-            for (int j = 0; j < NT; ++j)
-              mma_s8_m16n8k32(acc[m][j], word_of(a[2 * m], w), word_of(a[2 * m + 1], w),
-                              word_of(a[2 * m], w + 1), word_of(a[2 * m + 1], w + 1),
-                              word_of(b[j], w), word_of(b[j], w + 1));
-        }
-      }
+      mac(a, b, acc);
       // the slot just read is free again (its loads have delivered: their values were used)
       fetch();
     }

@@ -767,28 +767,31 @@ bool few_rows_wanted(int M, int N, int K, bool packed_s4, const OutputSpec& out)
   return static_cast<long long>(longer) * K <= (64LL << 20);
 }
 
-// Shape of a few-rows launch.  MT groups of 16 long rows per CTA: two from nine short rows on,
-// so that the short operand's requests stay at half the long operand's.
-#ifndef FEW_ROWS_MT
-#define FEW_ROWS_MT(nt) ((nt) >= 2 ? 2 : 1)
-#endif
+// Shape of a few-rows launch.  Two groups of 16 long rows per CTA (32-row blocks): the short
+// operand's requests are then at most half the long operand's, and 9-16 short rows measured
+// 10 %, up to 8 short rows 2-9 % faster than with 16-row blocks.
+constexpr int FEW_ROWS_MT = 2;
 
 struct FewRowsShape {
-  int mt, depth, warps, grid, smem;
+  int mt, depth, warps, grid, smem, head;
 };
 
 constexpr int FEW_ROWS_SMEM_SM = 227 * 1024;  // shared memory of an SM; each CTA reserves 1 KB more
+// What the CTAs of an SM take of it between them: the rest of the 256 KB stays L1, where the
+// short operand, which every CTA reads again, finds room (with all 227 KB given to deeper rings
+// up to 8 short rows ran 9.9 us instead of 9.2-9.4 at N = K = 8192, INT4; with 160 KB the
+// problems whose blocks outnumber the resident CTAs lost 15-20 %).
+constexpr int FEW_ROWS_SMEM_RING = 192 * 1024;
 
 // Warps per CTA share K (64 bytes per step): eight, fewer for a short K (two steps each at
 // least), sixteen while the SMs would have fewer than twelve warps each and K is long enough.
 // CTAs per SM: as many as hold every row block at once if the ring can still be two steps deep;
 // else fewer, with a ring of at least three steps, and a CTA walks the blocks c, c + grid, ...
-// The ring takes what shared memory there is (up to eight steps): the kernel is as fast as HBM
-// only while ~100 KB of the long operand per SM are in flight (warps x depth x MT KB per CTA).
+// The ring takes what is left of the SM's allotment (FEW_ROWS_SMEM_RING, up to eight steps).
 FewRowsShape few_rows_shape(int rows_l, int rows_s, int row_bytes, int num_sms) {
   const int nt = rows_s <= 8 ? 1 : rows_s <= 16 ? 2 : 4;
   FewRowsShape f;
-  f.mt = FEW_ROWS_MT(nt);
+  f.mt = FEW_ROWS_MT;
   const int steps = ceil_div(row_bytes, 64);
   const long long blocks = ceil_div(rows_l, 16 * f.mt);
   f.warps = 8;
@@ -800,7 +803,7 @@ FewRowsShape few_rows_shape(int rows_l, int rows_s, int row_bytes, int num_sms) 
   if (per_sm * f.warps > 64) per_sm = 64 / f.warps;  // warp slots of an SM
   if (per_sm > 32) per_sm = 32;                      // and its CTA slots
   for (;; --per_sm) {
-    f.depth = (FEW_ROWS_SMEM_SM / per_sm - 1024 - red) / slot;
+    f.depth = (FEW_ROWS_SMEM_RING / per_sm - 1024 - red) / slot;
     const bool all_at_once = blocks <= static_cast<long long>(per_sm) * num_sms;
     if (f.depth >= (all_at_once ? 2 : 3) || per_sm == 1) break;
   }
@@ -808,15 +811,20 @@ FewRowsShape few_rows_shape(int rows_l, int rows_s, int row_bytes, int num_sms) 
   f.smem = few_rows_ring_bytes(f.mt, nt, f.depth, f.warps) + red;
   const long long resident = static_cast<long long>(per_sm) * num_sms;
   f.grid = static_cast<int>(blocks < resident ? blocks : resident);
+  // One step through registers on top of the ring where the kernel variant exists (9-16 short
+  // rows: 10.1 -> 9.2 us at 16 x 8192 x 8192, INT4) and its ~96 registers per thread do not cost a
+  // resident CTA (three CTAs of eight warps per SM did: 13.7 -> 14.7 us at 16 x 12288 x 8192).
+  f.head = (nt == 2 && per_sm * f.warps <= 16) ? 1 : 0;
   return f;
 }
 
-template <bool S4, int NT, int EPI>
+template <bool S4, int NT, int EPI, int HEAD>
 int launch_few_rows_nt(DeviceState* s, FewRowsParams& p, const FewRowsShape& f,
                        cudaStream_t stream) {
-  constexpr int MT = FEW_ROWS_MT(NT);
-  constexpr int variant = 256 + (S4 ? 9 : 0) + (NT == 1 ? 0 : NT == 2 ? 3 : 6) + EPI;  // attr_set bits 256..273
-  auto kernel = few_rows_kernel<S4, MT, NT, EPI>;
+  // attr_set bits 256..273, with the register head 274..279
+  constexpr int variant = HEAD ? 274 + (S4 ? 3 : 0) + EPI
+                               : 256 + (S4 ? 9 : 0) + (NT == 1 ? 0 : NT == 2 ? 3 : 6) + EPI;
+  auto kernel = few_rows_kernel<S4, FEW_ROWS_MT, NT, EPI, HEAD>;
   if (!(s->attr_set[variant >> 6].load(std::memory_order_relaxed) & (1ull << (variant & 63)))) {
     const cudaError_t e = cudaFuncSetAttribute(
         kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FEW_ROWS_SMEM_SM);
@@ -864,10 +872,12 @@ int launch_few_rows(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.wait_prior_grid = (g_l2_policy & 32) ? 0 : 1;
   const FewRowsShape f = few_rows_shape(p.rows_l, p.rows_s, p.row_bytes, s->num_sms);
   switch (ceil_div(p.rows_s, 8)) {
-    case 1: return launch_few_rows_nt<S4, 1, EPI>(s, p, f, stream);
-    case 2: return launch_few_rows_nt<S4, 2, EPI>(s, p, f, stream);
+    case 1: return launch_few_rows_nt<S4, 1, EPI, 0>(s, p, f, stream);
+    case 2:
+      return f.head ? launch_few_rows_nt<S4, 2, EPI, 1>(s, p, f, stream)
+                    : launch_few_rows_nt<S4, 2, EPI, 0>(s, p, f, stream);
     case 3:
-    case 4: return launch_few_rows_nt<S4, 4, EPI>(s, p, f, stream);
+    case 4: return launch_few_rows_nt<S4, 4, EPI, 0>(s, p, f, stream);
     default: return GEMM_ERR_INVALID_ARG;
   }
 }
