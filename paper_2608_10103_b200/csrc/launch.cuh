@@ -811,18 +811,19 @@ FewRowsShape few_rows_shape(int rows_l, int rows_s, int row_bytes, int num_sms) 
   f.smem = few_rows_ring_bytes(f.mt, nt, f.depth, f.warps) + red;
   const long long resident = static_cast<long long>(per_sm) * num_sms;
   f.grid = static_cast<int>(blocks < resident ? blocks : resident);
-  // One step through registers on top of the ring where the kernel variant exists (9-16 short
-  // rows: 10.1 -> 9.2 us at 16 x 8192 x 8192, INT4) and its ~96 registers per thread do not cost a
-  // resident CTA (three CTAs of eight warps per SM did: 13.7 -> 14.7 us at 16 x 12288 x 8192).
-  f.head = (nt == 2 && per_sm * f.warps <= 16) ? 1 : 0;
+  // One step through registers on top of the ring (up to 16 short rows: 10.1 -> 9.2 us at
+  // 16 x 8192 x 8192, 9.2 -> 8.9 us at 1 x 8192 x 8192, INT4) where its registers, up to 128 per
+  // thread, do not cost a resident CTA (three CTAs of eight warps per SM did: 13.7 -> 14.7 us at
+  // 16 x 12288 x 8192).
+  f.head = (nt <= 2 && per_sm * f.warps <= 16) ? 1 : 0;
   return f;
 }
 
 template <bool S4, int NT, int EPI, int HEAD>
 int launch_few_rows_nt(DeviceState* s, FewRowsParams& p, const FewRowsShape& f,
                        cudaStream_t stream) {
-  // attr_set bits 256..273, with the register head 274..279
-  constexpr int variant = HEAD ? 274 + (S4 ? 3 : 0) + EPI
+  // attr_set bits 256..273, with the register head 274..285
+  constexpr int variant = HEAD ? 274 + (S4 ? 3 : 0) + EPI + (NT == 1 ? 6 : 0)
                                : 256 + (S4 ? 9 : 0) + (NT == 1 ? 0 : NT == 2 ? 3 : 6) + EPI;
   auto kernel = few_rows_kernel<S4, FEW_ROWS_MT, NT, EPI, HEAD>;
   if (!(s->attr_set[variant >> 6].load(std::memory_order_relaxed) & (1ull << (variant & 63)))) {
@@ -872,7 +873,9 @@ int launch_few_rows(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.wait_prior_grid = (g_l2_policy & 32) ? 0 : 1;
   const FewRowsShape f = few_rows_shape(p.rows_l, p.rows_s, p.row_bytes, s->num_sms);
   switch (ceil_div(p.rows_s, 8)) {
-    case 1: return launch_few_rows_nt<S4, 1, EPI, 0>(s, p, f, stream);
+    case 1:
+      return f.head ? launch_few_rows_nt<S4, 1, EPI, 1>(s, p, f, stream)
+                    : launch_few_rows_nt<S4, 1, EPI, 0>(s, p, f, stream);
     case 2:
       return f.head ? launch_few_rows_nt<S4, 2, EPI, 1>(s, p, f, stream)
                     : launch_few_rows_nt<S4, 2, EPI, 0>(s, p, f, stream);
