@@ -92,8 +92,9 @@ int gemm_s8(int M, int N, int K, const int8_t* A, const int8_t* B, int32_t* C,
  * rows on one side (M or N) against 512 or more on the other never reaches it:
  * the long operand goes from global memory straight into the fragments of the
  * warp-level integer MMA, its nibbles expanded in registers, in one launch that
- * needs no scratch and zeroes nothing (gemm_s8 does the same while the long
- * operand has at most 64 MB; see gemm_set_kernel_family in b200gemm_debug.h).
+ * needs no scratch and zeroes nothing (gemm_s8 does the same with up to 8
+ * such rows, and with 9-16 while the long operand has at most 64 MB; see
+ * gemm_set_kernel_family in b200gemm_debug.h).
  * Most other problems: a kernel
  * variant expands the nibbles on the way to the MMAs (see gemm_set_s4_scheme in
  * b200gemm_debug.h for the rule and the switch).  The rest (a short K, less than

@@ -70,8 +70,8 @@ int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k);
  * loads them back and, for INT4, expands the nibbles in registers; a CTA owns
  * 32 rows of the long operand over the whole of K, sums its warps'
  * results and writes its part of C once.  Family 0 takes it for a short side
- * of at most 16 rows against at least 512 -- INT4 always, INT8 while the long
- * operand has at most 64 MB; 3 =
+ * of at most 16 rows against at least 512 -- INT4 always, INT8 with up to 8
+ * rows always and with 9-16 while the long operand has at most 64 MB; 3 =
  * wherever it exists (a short side of at most 32 rows); 1 and 2 never, nor do
  * calls with a forced tile shape, operand order or INT4 scheme, or traced ones.
  * gemm_query_config describes such a call as "few_rows rows_per_block=..

@@ -63,6 +63,8 @@ struct FewRowsParams {
 };
 
 constexpr int FEW_ROWS_MAX_DEPTH = 8;
+// Operand kinds of few_rows_kernel: int8, packed signed 4-bit, binary16.
+constexpr int FEW_ROWS_S8 = 0, FEW_ROWS_S4 = 1, FEW_ROWS_F16 = 2;
 
 // Words per short row in the reduction buffer: the block's long rows plus four, so that the
 // four lanes of a quad (short rows 2t) land 8 banks apart.
@@ -129,6 +131,26 @@ __device__ __forceinline__ void mma_s8_m16n8k32(int (&d)[4], uint32_t a0, uint32
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// FP16 operands: 16 rows x 16 values against 8 rows per instruction, FP32 accumulators; a 32-bit
+// word holds two values, and words w, w + 1 of a thread's piece fill its K positions 2t, 2t + 1
+// and 2t + 8, 2t + 9 on both sides.
+__device__ __forceinline__ void mma_f16_m16n8k16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                 uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+      "{%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <bool F16>
+struct AccOf {
+  using type = int;
+};
+template <>
+struct AccOf<true> {
+  using type = float;
+};
+
 __device__ __forceinline__ uint32_t word_of(const uint4& v, int i) {
   return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
 }
@@ -138,7 +160,7 @@ __device__ __forceinline__ uint32_t high_nibbles_x16(uint32_t w) { return w & 0x
 
 }  // namespace few_rows_detail
 
-// S4: packed 4-bit operands (else int8).  MT: groups of 16 long rows per CTA (a warp holds the
+// KIND: int8, packed 4-bit or binary16 operands.  MT: groups of 16 long rows per CTA (a warp holds the
 // fragments of all of them and uses each short fragment MT times: the short operand, fetched
 // again by every CTA, costs 8 NT / (16 MT) of the long operand's bytes in requests).  NT: groups
 // of eight short rows.  EPI: as for the tile kernels.  HEAD: steps of the first block that go
@@ -146,9 +168,11 @@ __device__ __forceinline__ uint32_t high_nibbles_x16(uint32_t w) { return w & 0x
 // Dynamic shared memory: few_rows_ring_bytes + few_rows_red_bytes.  Any grid size: CTA c takes
 // the row blocks c, c + grid, ...; its copies run ahead across the block boundaries, so only
 // the first block of a CTA waits for the memory latency in full.
-template <bool S4, int MT, int NT, int EPI, int HEAD = 0>
+template <int KIND, int MT, int NT, int EPI, int HEAD = 0>
 __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   using namespace few_rows_detail;
+  constexpr bool S4 = KIND == FEW_ROWS_S4, F16 = KIND == FEW_ROWS_F16;
+  using Acc = typename AccOf<F16>::type;  // FP32 sums for FP16 operands, INT32 for the integer kinds
   extern __shared__ __align__(16) unsigned char few_rows_smem[];
   const int tid = static_cast<int>(threadIdx.x), threads = static_cast<int>(blockDim.x);
   const int lane = tid & 31, warp = tid >> 5, warps = threads >> 5;
@@ -161,7 +185,7 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   const uint32_t piece_pitch = static_cast<uint32_t>(threads) * 16u;
   // behind the ring: [warps][8 NT][RED_PITCH] partial sums
   const int depth = p.depth;
-  int* red = reinterpret_cast<int*>(few_rows_smem + few_rows_ring_bytes(MT, NT, depth, warps));
+  Acc* red = reinterpret_cast<Acc*>(few_rows_smem + few_rows_ring_bytes(MT, NT, depth, warps));
 
   if (tid == 0) ptx::grid_dep_launch_dependents();
   if (p.wait_prior_grid) ptx::grid_dep_wait();
@@ -239,8 +263,19 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   for (int d = 0; d < depth; ++d) fetch();
 
   // one step: the four words of every piece feed four (INT4) or two (INT8) rounds of MMAs
-  auto mac = [&](const uint4 (&a)[2 * MT], const uint4 (&b)[NT], int (&acc)[MT][NT][4]) {
-    if constexpr (S4) {
+  auto mac = [&](const uint4 (&a)[2 * MT], const uint4 (&b)[NT], Acc (&acc)[MT][NT][4]) {
+    if constexpr (F16) {
+#pragma unroll
+      for (int w = 0; w < 4; w += 2) {
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+#pragma unroll
+          for (int j = 0; j < NT; ++j)
+            mma_f16_m16n8k16(acc[m][j], word_of(a[2 * m], w), word_of(a[2 * m + 1], w),
+                             word_of(a[2 * m], w + 1), word_of(a[2 * m + 1], w + 1),
+                             word_of(b[j], w), word_of(b[j], w + 1));
+      }
+    } else if constexpr (S4) {
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
         uint32_t b0[NT], b1[NT];
@@ -276,7 +311,7 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   int c_slot = 0;
 #pragma unroll 1
   for (int blk = 0; blk < my_blocks; ++blk) {
-    int acc[MT][NT][4];
+    Acc acc[MT][NT][4];
 #pragma unroll
     for (int m = 0; m < MT; ++m)
 #pragma unroll
@@ -312,7 +347,7 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
 
     // accumulator fragment of group m: [0], [1] = long row 16 m + g, short rows 2t, 2t + 1;
     // [2], [3] = long row 16 m + g + 8
-    int* mine = red + warp * (8 * NT * RED_PITCH);
+    Acc* mine = red + warp * (8 * NT * RED_PITCH);
 #pragma unroll
     for (int m = 0; m < MT; ++m) {
 #pragma unroll
@@ -320,7 +355,10 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
           const int s = 8 * j + 2 * t + (v & 1), l = 16 * m + g + 8 * (v >> 1);
-          mine[s * RED_PITCH + l] = S4 ? (acc[m][j][v] >> 8) : acc[m][j][v];
+          if constexpr (S4)
+            mine[s * RED_PITCH + l] = acc[m][j][v] >> 8;
+          else
+            mine[s * RED_PITCH + l] = acc[m][j][v];
         }
       }
     }
@@ -332,11 +370,13 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
       const int s = l_contiguous ? idx / BLOCK_ROWS : idx % (8 * NT);
       const int l = l_contiguous ? idx % BLOCK_ROWS : idx / (8 * NT);
       if (s >= p.rows_s || l0 + l >= p.rows_l) continue;
-      int sum = 0;
+      Acc sum = 0;
       for (int w = 0; w < warps; ++w) sum += red[w * (8 * NT * RED_PITCH) + s * RED_PITCH + l];
       const long long at = s * p.c_stride_s + static_cast<long long>(l0 + l) * p.c_stride_l;
       if constexpr (EPI == EPI_RAW32) {
-        static_cast<int*>(p.C)[at] = sum;
+        static_cast<Acc*>(p.C)[at] = sum;
+      } else if constexpr (F16) {
+        static_cast<__half*>(p.C)[at] = __float2half_rn(sum);  // EPI_OUT16: rounded once
       } else {
         const float fs = __ldg(p.scale_s + s), fl = __ldg(p.scale_l + l0 + l);
         const float x = p.scale_s_first ? static_cast<float>(sum) * fs * fl

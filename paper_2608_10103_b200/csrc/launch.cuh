@@ -742,19 +742,23 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   }
 }
 
-// Integer problems with a few rows on one side go to few_rows_kernel (the long operand from
+// Problems with a few rows on one side go to few_rows_kernel (the long operand from
 // global memory to MMA fragments without a pass through a shared tile, one launch, nothing
 // zeroed).  Automatic for a short side of up to 16 rows against 512 or more: INT4 always (it
 // measured 0.45-0.98 of the tile kernels' time for 2048 <= N <= 28672, K = 4096 / 8192: there the
-// tile kernels are bound by expanding the nibbles in shared memory); INT8 while the long operand
-// has at most 64 MB (0.65-0.96 of the tile kernels' time; level from there to 128 MB, and up to
-// 1.1 x slower beyond, where the tile kernels' bulk copies reach 0.86 of the HBM bandwidth).
+// tile kernels are bound by expanding the nibbles in shared memory); INT8 with up to 8 short
+// rows always too (0.65-0.93 of the tile kernels' time, 0.94 of the HBM bandwidth at
+// 1 x 28672 x 8192), with 9-16 while the long operand has at most 64 MB (0.8-0.9; level at
+// 128 MB, 5-15 % slower at 96 and 235 MB, where the tile kernels' bulk copies reach 0.86-0.88 of
+// the HBM bandwidth); FP16 while the long operand has at most 64 M elements (128 MB: 0.78-0.96
+// of the tile kernels' time, level at 16 x 4096 x 16384; 4-17 % slower beyond).
 // gemm_set_kernel_family(3) takes it wherever it exists (a short side of up to 32 rows),
 // families 1 and 2, forced tile shapes, forced operand orders, every forced INT4 scheme and the
 // traced runs never.
 constexpr int FEW_ROWS_AUTO = 16;
 constexpr int FEW_ROWS_MAX = 32;
-bool few_rows_wanted(int M, int N, int K, bool packed_s4, const OutputSpec& out) {
+bool few_rows_wanted(int M, int N, int K, bool packed_s4, const OutputSpec& out,
+                     bool fp16 = false) {
   if (out.tiles_only || g_override_bn || g_override_cta_group || g_override_splits) return false;
   if ((g_trace_on & 1) || (g_l2_policy & 64)) return false;  // measurement runs mean the tile kernels
   if (g_swap_ab) return false;                                // so does a forced operand order
@@ -764,7 +768,8 @@ bool few_rows_wanted(int M, int N, int K, bool packed_s4, const OutputSpec& out)
   if (fam == 3) return shorter <= FEW_ROWS_MAX;
   if (fam != 0 || shorter > FEW_ROWS_AUTO || longer < 512) return false;
   if (packed_s4) return true;
-  return static_cast<long long>(longer) * K <= (64LL << 20);
+  if (fp16) return static_cast<long long>(longer) * K <= (64LL << 20);
+  return shorter <= 8 || static_cast<long long>(longer) * K <= (64LL << 20);
 }
 
 // Shape of a few-rows launch.  Two groups of 16 long rows per CTA (32-row blocks): the short
@@ -819,13 +824,13 @@ FewRowsShape few_rows_shape(int rows_l, int rows_s, int row_bytes, int num_sms) 
   return f;
 }
 
-template <bool S4, int NT, int EPI, int HEAD>
+template <int FKIND, int NT, int EPI, int HEAD>
 int launch_few_rows_nt(DeviceState* s, FewRowsParams& p, const FewRowsShape& f,
                        cudaStream_t stream) {
-  // attr_set bits 256..273, with the register head 274..285
-  constexpr int variant = HEAD ? 274 + (S4 ? 3 : 0) + EPI + (NT == 1 ? 6 : 0)
-                               : 256 + (S4 ? 9 : 0) + (NT == 1 ? 0 : NT == 2 ? 3 : 6) + EPI;
-  auto kernel = few_rows_kernel<S4, FEW_ROWS_MT, NT, EPI, HEAD>;
+  // attr_set bits 256..309: by operand kind, short-row groups, output mode, register head
+  constexpr int variant =
+      256 + ((FKIND * 3 + (NT == 1 ? 0 : NT == 2 ? 1 : 2)) * 3 + EPI) * 2 + HEAD;
+  auto kernel = few_rows_kernel<FKIND, FEW_ROWS_MT, NT, EPI, HEAD>;
   if (!(s->attr_set[variant >> 6].load(std::memory_order_relaxed) & (1ull << (variant & 63)))) {
     const cudaError_t e = cudaFuncSetAttribute(
         kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FEW_ROWS_SMEM_SM);
@@ -847,8 +852,8 @@ int launch_few_rows_nt(DeviceState* s, FewRowsParams& p, const FewRowsShape& f,
   return e == cudaSuccess ? GEMM_OK : cuda_fail(e);
 }
 
-// A, B: int8 or packed INT4 rows, pitches in bytes.
-template <bool S4, int EPI>
+// A, B: int8, packed INT4 or FP16 rows, pitches in bytes.
+template <int FKIND, int EPI>
 int launch_few_rows(int M, int N, int K, const void* A, size_t a_pitch, const void* B,
                     size_t b_pitch, void* C, const OutputSpec& out, cudaStream_t stream) {
   DeviceState* s = nullptr;
@@ -863,7 +868,7 @@ int launch_few_rows(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.s_pitch = static_cast<long long>(a_short ? a_pitch : b_pitch);
   p.rows_l = a_short ? N : M;
   p.rows_s = a_short ? M : N;
-  p.row_bytes = S4 ? K / 2 : K;
+  p.row_bytes = FKIND == FEW_ROWS_S4 ? K / 2 : FKIND == FEW_ROWS_F16 ? 2 * K : K;
   p.C = C;
   p.c_stride_s = a_short ? ldc : 1;
   p.c_stride_l = a_short ? 1 : ldc;
@@ -874,13 +879,13 @@ int launch_few_rows(int M, int N, int K, const void* A, size_t a_pitch, const vo
   const FewRowsShape f = few_rows_shape(p.rows_l, p.rows_s, p.row_bytes, s->num_sms);
   switch (ceil_div(p.rows_s, 8)) {
     case 1:
-      return f.head ? launch_few_rows_nt<S4, 1, EPI, 1>(s, p, f, stream)
-                    : launch_few_rows_nt<S4, 1, EPI, 0>(s, p, f, stream);
+      return f.head ? launch_few_rows_nt<FKIND, 1, EPI, 1>(s, p, f, stream)
+                    : launch_few_rows_nt<FKIND, 1, EPI, 0>(s, p, f, stream);
     case 2:
-      return f.head ? launch_few_rows_nt<S4, 2, EPI, 1>(s, p, f, stream)
-                    : launch_few_rows_nt<S4, 2, EPI, 0>(s, p, f, stream);
+      return f.head ? launch_few_rows_nt<FKIND, 2, EPI, 1>(s, p, f, stream)
+                    : launch_few_rows_nt<FKIND, 2, EPI, 0>(s, p, f, stream);
     case 3:
-    case 4: return launch_few_rows_nt<S4, 4, EPI, 0>(s, p, f, stream);
+    case 4: return launch_few_rows_nt<FKIND, 4, EPI, 0>(s, p, f, stream);
     default: return GEMM_ERR_INVALID_ARG;
   }
 }
@@ -894,16 +899,23 @@ int launch_gemm(int M, int N, int K, const void* A, size_t a_pitch, const void* 
     if (!req && !hyb && few_rows_wanted(M, N, K, packed_s4, out)) {
       switch (out.epi) {
         case EPI_RAW32:
-          return packed_s4 ? launch_few_rows<true, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream)
-                           : launch_few_rows<false, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+          return packed_s4 ? launch_few_rows<FEW_ROWS_S4, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream)
+                           : launch_few_rows<FEW_ROWS_S8, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
         case EPI_OUT16:
-          return packed_s4 ? launch_few_rows<true, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream)
-                           : launch_few_rows<false, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+          return packed_s4 ? launch_few_rows<FEW_ROWS_S4, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream)
+                           : launch_few_rows<FEW_ROWS_S8, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
         case EPI_F32_SCALED:
-          return packed_s4 ? launch_few_rows<true, EPI_F32_SCALED>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream)
-                           : launch_few_rows<false, EPI_F32_SCALED>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+          return packed_s4 ? launch_few_rows<FEW_ROWS_S4, EPI_F32_SCALED>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream)
+                           : launch_few_rows<FEW_ROWS_S8, EPI_F32_SCALED>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
         default: return GEMM_ERR_INVALID_ARG;
       }
+    }
+  } else {
+    if (!req && !hyb && !packed_s4 && few_rows_wanted(M, N, K, false, out, true)) {
+      if (out.epi == EPI_RAW32)
+        return launch_few_rows<FEW_ROWS_F16, EPI_RAW32>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
+      if (out.epi == EPI_OUT16)
+        return launch_few_rows<FEW_ROWS_F16, EPI_OUT16>(M, N, K, A, a_pitch, B, b_pitch, C, out, stream);
     }
   }
   switch (out.epi) {

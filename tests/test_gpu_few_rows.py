@@ -1,6 +1,6 @@
-"""GPU parity of the kernel for integer problems with a few rows on one side (the long operand
-goes from global memory into warp-level MMA fragments; no tile, no split-K through C) against
-the oracle: both integer precisions, either operand as the short one, every output mode,
+"""GPU parity of the kernel for problems with a few rows on one side (the long operand goes
+from global memory into warp-level MMA fragments; no tile, no split-K through C) against the
+oracle: every precision, either operand as the short one, every output mode,
 ragged sizes, many row blocks per CTA, and bit-equality with the tile kernels.
 gemm_set_kernel_family(3) takes the kernel wherever it exists (a short side of up to 32 rows),
 family 1 never."""
@@ -37,16 +37,17 @@ SHAPES = [(1, 1, 32), (1, 777, 512), (3, 100, 96), (8, 1000, 4128), (9, 530, 160
           (777, 1, 512), (1000, 8, 4128), (2049, 12, 1056), (530, 16, 160), (600, 29, 96)]
 
 
-@pytest.mark.parametrize("prec", ["s8", "s4"])
+@pytest.mark.parametrize("prec", ["fp16", "s8", "s4"])
 @pytest.mark.parametrize("M,N,K", SHAPES)
 def test_few_rows_full_compare(prec, M, N, K):
     assert binding.gemm_query_config(prec, M, N, K).startswith("few_rows")
     A, B = _make(prec, M, N, K, seed=M + N + K)
     for rep in range(2):
-        check_against_oracle(prec, A, B, run_gpu(prec, A, B, fill=-7), force_full=True)
+        C = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)
+        check_against_oracle(prec, A, B, C, force_full=True)
 
 
-@pytest.mark.parametrize("prec", ["s8", "s4"])
+@pytest.mark.parametrize("prec", ["fp16", "s8", "s4"])
 @pytest.mark.parametrize("M,N,K", [(8, 80000, 1056), (16, 160001, 256), (5, 200000, 64), (160000, 16, 512)])
 def test_few_rows_more_row_blocks_than_ctas(prec, M, N, K):
     """More row blocks than CTAs fit the SMs: a CTA walks several, its copies running ahead
@@ -56,7 +57,7 @@ def test_few_rows_more_row_blocks_than_ctas(prec, M, N, K):
     blocks = int(cfg.split("blocks=")[1].split()[0])
     assert cfg.startswith("few_rows") and ctas < blocks
     A, B = _make(prec, M, N, K, seed=N)
-    check_against_oracle(prec, A, B, run_gpu(prec, A, B, fill=-7))
+    check_against_oracle(prec, A, B, run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7))
 
 
 @pytest.mark.parametrize("prec", ["s8", "s4"])
@@ -121,14 +122,39 @@ def test_few_rows_dequantised_outputs(prec, out_dtype, M, N, K):
     assert ok, worst
 
 
+def test_few_rows_fp16_output_and_special_values():
+    """FP16 result rounded once from the FP32 sums; infinities and NaNs of the operands reach
+    the rows and columns they belong to and no others."""
+    M, N, K = 12, 1300, 1056
+    A, B = synth.fp16_normal_clipped(M, N, K, seed=3)
+    ref, S = oracle.gemm_fp16(A, B)
+    C = torch.full((M, N), float("nan"), dtype=torch.float16, device="cuda")
+    binding.gemm_fp16_f16out(to_dev(A), to_dev(B), C)
+    torch.cuda.synchronize()
+    ok, worst = oracle.fp16_out_check(C.cpu().numpy(), ref, S)
+    assert ok, "fp16 out: %.3g x bound" % worst
+    A = A.copy()
+    B = B.copy()
+    A[3, 700] = np.float16(np.inf)
+    B[77, 5] = np.float16(np.nan)
+    got = run_gpu("fp16", A, B, fill=0.0)
+    assert np.all(np.isnan(got[:, 77])) and np.all(np.isinf(got[3, :77]) | np.isnan(got[3, :77]))
+    clean = np.ones((M, N), dtype=bool)
+    clean[3, :] = False
+    clean[:, 77] = False
+    assert np.all(np.isfinite(got[clean]))
+
+
 def test_few_rows_automatic_rule():
     binding.gemm_set_kernel_family(0)
     few = lambda prec, M, N, K: binding.gemm_query_config(prec, M, N, K).startswith("few_rows")
     assert few("s4", 16, 8192, 8192) and few("s4", 1, 28672, 8192) and few("s4", 4096, 9, 1024)
     assert not few("s4", 17, 8192, 8192) and not few("s4", 16, 500, 8192)
     assert few("s8", 8, 2048, 4096) and few("s8", 16, 4096, 8192) and few("s8", 16, 8192, 8192)
+    assert few("s8", 8, 28672, 8192)
     assert not few("s8", 16, 12288, 8192) and not few("s8", 17, 2048, 4096)
-    assert not few("fp16", 1, 8192, 8192)
+    assert few("fp16", 1, 8192, 8192) and few("fp16", 16, 4096, 16384) and few("fp16", 3000, 7, 512)
+    assert not few("fp16", 16, 16384, 8192) and not few("fp16", 17, 8192, 8192)
     binding.gemm_set_s4_scheme(2)          # a forced INT4 scheme means the tile kernels
     assert not few("s4", 16, 8192, 8192)
     binding.gemm_set_s4_scheme(0)

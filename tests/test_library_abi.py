@@ -128,12 +128,14 @@ def test_selector_invariants_over_many_shapes(lib):
             c = _parse(text)
             if text.startswith("few_rows"):   # the kernel for a short side of up to 16 rows
                 short, long_ = min(M, N), max(M, N)
-                assert prec != "fp16" and short <= 16 and long_ >= 512 and c["short_rows"] == short
+                assert short <= 16 and long_ >= 512 and c["short_rows"] == short
                 if prec == "s8":
+                    assert short <= 8 or long_ * K <= 64 << 20
+                if prec == "fp16":
                     assert long_ * K <= 64 << 20
                 rows = c["rows_per_block"]
                 assert rows == 32 and c["blocks"] == -(-long_ // rows)
-                row_bytes = K // 2 if prec == "s4" else K
+                row_bytes = K // 2 if prec == "s4" else 2 * K if prec == "fp16" else K
                 w, d = c["warps"], c["depth"]
                 assert w in (1, 2, 4, 8, 16) and 2 <= d <= 8
                 assert w == 1 or -(-row_bytes // 64) >= 2 * w      # two 64-byte steps per warp
@@ -200,13 +202,16 @@ def test_selector_headline_choices(lib):
         assert (classic["BM"], classic["BN"], classic["cta_group"], classic["stages"]) == (256, 256, 2, 6)
     finally:
         binding.gemm_set_kernel_family(0)
-    dec = _parse(binding.gemm_query_config("fp16", 16, 8192, 8192))
+    dec = _parse(binding.gemm_query_config("fp16", 24, 8192, 8192))
     assert dec["split_k"] > 1 and dec["split_tiles"] == dec["tiles"]
+    assert binding.gemm_query_config("fp16", 16, 8192, 8192).startswith("few_rows")
+    assert not binding.gemm_query_config("fp16", 16, 16384, 8192).startswith("few_rows")
     few = binding.gemm_query_config("s4", 16, 8192, 8192)
     assert few.startswith("few_rows") and "s4=in_registers" in few
     assert binding.gemm_query_config("s8", 8, 4096, 4096).startswith("few_rows")
     assert binding.gemm_query_config("s8", 16, 8192, 8192).startswith("few_rows")
     assert not binding.gemm_query_config("s8", 16, 28672, 8192).startswith("few_rows")
+    assert binding.gemm_query_config("s8", 8, 28672, 8192).startswith("few_rows")
     assert not binding.gemm_query_config("s4", 17, 8192, 8192).startswith("few_rows")
     tail = _parse(binding.gemm_query_config("fp16", 4096, 4096, 8192))
     assert tail["split_k"] == 2 and tail["split_tiles"] == 256 % 74
