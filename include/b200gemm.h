@@ -71,6 +71,9 @@ enum { GEMM_PREC_FP16 = 0, GEMM_PREC_S8 = 1, GEMM_PREC_S4 = 2 };
  * A, B: IEEE binary16.  Accumulation order inside the tensor core is hardware
  * defined; results satisfy |C - exact| <= 1e-4 * sum_k|a*b| + 1e-6.
  * Alignment: A, B, C 16-byte aligned; K % 8 == 0.
+ * (A problem with at most 16 rows on one side against 512 or more on the
+ * other, and at most 32 M elements in the long operand, does not run on tiles:
+ * see gemm_set_kernel_family in b200gemm_debug.h.  Same bound.)
  */
 int gemm_fp16(int M, int N, int K, const void* A, const void* B, float* C, gemm_stream_t stream);
 
@@ -262,8 +265,8 @@ int gemm_unpack_s4(int rows, int K, const uint8_t* packed, int8_t* out, size_t o
  * terminated, truncated to len); for INT4 followed by the route
  * (" prepass=unpack_s4" or " s4=fused_unpack"), and by " swap_ab" when the
  * kernel runs on exchanged operands (the tile is then described in the
- * kernel's orientation).  An integer problem that goes to the kernel for a few
- * rows instead of a tile kernel reads "few_rows rows_per_block=32 blocks=256
+ * kernel's orientation).  A problem that goes to the kernel for a few rows
+ * instead of a tile kernel reads "few_rows rows_per_block=32 blocks=256
  * short_rows=16 warps=8 depth=3 head=1 ctas=256 kind=i8" (" s4=in_registers" for
  * INT4).
  * Describes the raw 32-bit outputs (gemm_fp16, gemm_s8, gemm_s4).  Host only,

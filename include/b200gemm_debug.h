@@ -63,15 +63,18 @@ int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k);
  * pre-pass route included).  The paper fixes one tiling for every size
  * (Sec. III-A); this is the corresponding ablation axis here.
  *
- * The integer precisions have a third kernel, for problems with a few rows on
- * one side, which are bound by reading the long operand once: every thread
- * copies the 16-byte pieces its own mma.sync m16n8k32 (s8 x s8 -> s32) fragments
- * need into a private ring in shared memory (cp.async, several steps ahead),
- * loads them back and, for INT4, expands the nibbles in registers; a CTA owns
+ * There is a third kernel, for problems with a few rows on one side, which
+ * are bound by reading the long operand once: every thread copies the 16-byte
+ * pieces its own warp-level MMA fragments need (mma.sync m16n8k32, s8 x s8 ->
+ * s32, or m16n8k16, f16 x f16 -> f32) into a private ring in shared memory
+ * (cp.async, several steps ahead), loads them back and, for INT4, expands the
+ * nibbles in registers; a CTA owns
  * 32 rows of the long operand over the whole of K, sums its warps'
  * results and writes its part of C once.  Family 0 takes it for a short side
  * of at most 16 rows against at least 512 -- INT4 always, INT8 with up to 8
- * rows always and with 9-16 while the long operand has at most 64 MB; 3 =
+ * rows always and with 9-16 while the long operand has at most 64 MB, FP16
+ * while it has at most 32 M elements (INT8 and FP16 only with at least six
+ * 32-row blocks per KB of a row); 3 =
  * wherever it exists (a short side of at most 32 rows); 1 and 2 never, nor do
  * calls with a forced tile shape, operand order or INT4 scheme, or traced ones.
  * gemm_query_config describes such a call as "few_rows rows_per_block=..

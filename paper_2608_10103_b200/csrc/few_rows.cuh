@@ -1,5 +1,6 @@
-// Integer GEMM for problems with a few rows on one side (a handful of activations against a
-// large weight matrix): C = A B^T where one operand has at most 8 * NT rows.
+// GEMM for problems with a few rows on one side (a handful of activations against a large
+// weight matrix): C = A B^T where one operand has at most 8 * NT rows.  Written out below for
+// the integer kinds; FP16 operands take the same path with mma.sync m16n8k16 and FP32 sums.
 //
 // Such a call is bound by reading the long operand from HBM once, not by arithmetic, and the
 // tile kernels pay for staging it: every byte crosses shared memory several times (written by

@@ -742,6 +742,11 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
   }
 }
 
+// Shape of a few-rows launch.  Two groups of 16 long rows per CTA (32-row blocks): the short
+// operand's requests are then at most half the long operand's, and 9-16 short rows measured
+// 10 %, up to 8 short rows 2-9 % faster than with 16-row blocks.
+constexpr int FEW_ROWS_MT = 2;
+
 // Problems with a few rows on one side go to few_rows_kernel (the long operand from
 // global memory to MMA fragments without a pass through a shared tile, one launch, nothing
 // zeroed).  Automatic for a short side of up to 16 rows against 512 or more: INT4 always (it
@@ -750,8 +755,10 @@ int launch_gemm_epi(int M, int N, int K, const void* A, size_t a_pitch, const vo
 // rows always too (0.65-0.93 of the tile kernels' time, 0.94 of the HBM bandwidth at
 // 1 x 28672 x 8192), with 9-16 while the long operand has at most 64 MB (0.8-0.9; level at
 // 128 MB, 5-15 % slower at 96 and 235 MB, where the tile kernels' bulk copies reach 0.86-0.88 of
-// the HBM bandwidth); FP16 while the long operand has at most 64 M elements (128 MB: 0.78-0.96
-// of the tile kernels' time, level at 16 x 4096 x 16384; 4-17 % slower beyond).
+// the HBM bandwidth); FP16 while the long operand has at most 32 M elements (64 MB: 0.82-0.95
+// of the tile kernels' time; level at 128 MB, 4-17 % slower beyond); INT8 and FP16 only with
+// at least six 32-row blocks per KB of a row (16 x 1024 x 8192 FP16 has 32 blocks of 16 KB rows
+// and ran 12.3 against 8.5 us: too few CTAs for rows that long).
 // gemm_set_kernel_family(3) takes it wherever it exists (a short side of up to 32 rows),
 // families 1 and 2, forced tile shapes, forced operand orders, every forced INT4 scheme and the
 // traced runs never.
@@ -768,14 +775,13 @@ bool few_rows_wanted(int M, int N, int K, bool packed_s4, const OutputSpec& out,
   if (fam == 3) return shorter <= FEW_ROWS_MAX;
   if (fam != 0 || shorter > FEW_ROWS_AUTO || longer < 512) return false;
   if (packed_s4) return true;
-  if (fp16) return static_cast<long long>(longer) * K <= (64LL << 20);
+  // A CTA's time grows with the length of a row (its 16 warps share it), the tile kernels
+  // split K over as many CTAs as it takes: few row blocks against long rows stay on tiles.
+  const long long row_bytes = fp16 ? 2LL * K : K;
+  if (ceil_div(longer, 16 * FEW_ROWS_MT) < 6 * ceil_div(row_bytes, 1024)) return false;
+  if (fp16) return static_cast<long long>(longer) * K <= (32LL << 20);
   return shorter <= 8 || static_cast<long long>(longer) * K <= (64LL << 20);
 }
-
-// Shape of a few-rows launch.  Two groups of 16 long rows per CTA (32-row blocks): the short
-// operand's requests are then at most half the long operand's, and 9-16 short rows measured
-// 10 %, up to 8 short rows 2-9 % faster than with 16-row blocks.
-constexpr int FEW_ROWS_MT = 2;
 
 struct FewRowsShape {
   int mt, depth, warps, grid, smem, head;

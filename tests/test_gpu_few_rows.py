@@ -151,10 +151,12 @@ def test_few_rows_automatic_rule():
     assert few("s4", 16, 8192, 8192) and few("s4", 1, 28672, 8192) and few("s4", 4096, 9, 1024)
     assert not few("s4", 17, 8192, 8192) and not few("s4", 16, 500, 8192)
     assert few("s8", 8, 2048, 4096) and few("s8", 16, 4096, 8192) and few("s8", 16, 8192, 8192)
+    assert few("s4", 16, 512, 8192)
     assert few("s8", 8, 28672, 8192)
     assert not few("s8", 16, 12288, 8192) and not few("s8", 17, 2048, 4096)
-    assert few("fp16", 1, 8192, 8192) and few("fp16", 16, 4096, 16384) and few("fp16", 3000, 7, 512)
-    assert not few("fp16", 16, 16384, 8192) and not few("fp16", 17, 8192, 8192)
+    assert few("fp16", 1, 4096, 8192) and few("fp16", 16, 8192, 4096) and few("fp16", 3000, 7, 512)
+    assert not few("fp16", 16, 8192, 8192) and not few("fp16", 17, 4096, 4096)
+    assert not few("fp16", 16, 1024, 8192) and not few("s8", 16, 512, 8192)   # few blocks, long rows
     binding.gemm_set_s4_scheme(2)          # a forced INT4 scheme means the tile kernels
     assert not few("s4", 16, 8192, 8192)
     binding.gemm_set_s4_scheme(0)

@@ -83,7 +83,7 @@ def test_automatic_choice_for_few_rows():
     assert "swap_ab" not in binding.gemm_query_config("s8", 80, 8192, 8192)
     assert "swap_ab" not in binding.gemm_query_config("fp16", 64, 8192, 8192)
     assert "swap_ab" in binding.gemm_query_config("s8", 24, 8192, 8192)
-    assert "swap_ab" in binding.gemm_query_config("fp16", 24, 8192, 8192)
+    assert "swap_ab" in binding.gemm_query_config("fp16", 16, 8192, 8192)
     assert "swap_ab" not in binding.gemm_query_config("fp16", 128, 8192, 8192)
     assert "swap_ab" not in binding.gemm_query_config("s8", 16, 512, 8192)
     assert "swap_ab" not in binding.gemm_query_config("s8", 2048, 2048, 2048)

@@ -132,7 +132,9 @@ def test_selector_invariants_over_many_shapes(lib):
                 if prec == "s8":
                     assert short <= 8 or long_ * K <= 64 << 20
                 if prec == "fp16":
-                    assert long_ * K <= 64 << 20
+                    assert long_ * K <= 32 << 20
+                if prec != "s4":       # enough row blocks for the length of a row
+                    assert -(-long_ // 32) >= 6 * -(-(K * (2 if prec == "fp16" else 1)) // 1024)
                 rows = c["rows_per_block"]
                 assert rows == 32 and c["blocks"] == -(-long_ // rows)
                 row_bytes = K // 2 if prec == "s4" else 2 * K if prec == "fp16" else K
@@ -202,10 +204,11 @@ def test_selector_headline_choices(lib):
         assert (classic["BM"], classic["BN"], classic["cta_group"], classic["stages"]) == (256, 256, 2, 6)
     finally:
         binding.gemm_set_kernel_family(0)
-    dec = _parse(binding.gemm_query_config("fp16", 24, 8192, 8192))
+    dec = _parse(binding.gemm_query_config("fp16", 16, 8192, 8192))
     assert dec["split_k"] > 1 and dec["split_tiles"] == dec["tiles"]
-    assert binding.gemm_query_config("fp16", 16, 8192, 8192).startswith("few_rows")
-    assert not binding.gemm_query_config("fp16", 16, 16384, 8192).startswith("few_rows")
+    assert binding.gemm_query_config("fp16", 16, 4096, 8192).startswith("few_rows")
+    assert not binding.gemm_query_config("fp16", 16, 8192, 8192).startswith("few_rows")
+    assert not binding.gemm_query_config("fp16", 16, 1024, 8192).startswith("few_rows")
     few = binding.gemm_query_config("s4", 16, 8192, 8192)
     assert few.startswith("few_rows") and "s4=in_registers" in few
     assert binding.gemm_query_config("s8", 8, 4096, 4096).startswith("few_rows")
