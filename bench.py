@@ -642,7 +642,7 @@ def run_few_rows(args):
     # The tile kernels load their long operand with L2 priority "evict last", and lines so marked
     # outlive the flush between replays: whatever ran after them found part of a B copy in L2
     # (FP16, M = 1, N = K = 8192, few-rows kernel: 25.8 us before the first tile route, 23.9 us
-    # after).  Hence the scrub in front of every route below.
+    # after).  Hence the reset in front of every route below.
     probe = ("read-only probe: a kernel that reads B once and does nothing else", 0, 0, "probe")
     few = ("kernel for a few rows where it exists (up to 32)", 0, 0, "raw", 3)
     routes = {"fp16": [probe, ("selector default", 0, 0, "raw"), few,
@@ -658,9 +658,6 @@ def run_few_rows(args):
                      ("tile kernels: expanded in the kernel, operands exchanged", 2, 2, "raw"),
                      ("tile kernels: expanded in the kernel, both operands packed on CTA-pair tiles", 5, 0, "raw"),
                      ("pre-pass + INT8 GEMM", 1, 1, "raw")]}
-    scrub_a = torch.zeros((16, 8192), dtype=torch.float16, device="cuda")
-    scrub_b = torch.zeros((16384, 8192), dtype=torch.float16, device="cuda")
-    scrub_c = torch.empty((16, 16384), dtype=torch.float32, device="cuda")
     for M, N, K in shapes:
         for prec in [q for q in synth.PRECISIONS if q in args.precisions.split(",")]:
             A, B = synth.make(prec, M, N, K, seed=M + N)
@@ -697,12 +694,9 @@ def run_few_rows(args):
                 algo_bytes = A.nbytes + B.nbytes + M * N * (4 if mode == "raw" else 2)
                 if mode == "probe":
                     algo_bytes = B.nbytes
-                # every route starts alike: whatever "evict last" lines the route before left in
-                # L2 are replaced by lines of an unrelated matrix (a tile-kernel call over 256 MB)
-                binding.gemm_set_s4_scheme(0)
-                binding.gemm_set_kernel_family(1)
-                binding.gemm_set_swap_ab(2)
-                binding.gemm_fp16(scrub_a, scrub_b, scrub_c)
+                # every route starts alike: the "evict last" lines the route before left in L2
+                # go back to normal status, so that the flush removes them
+                binding.gemm_debug_reset_l2()
                 binding.gemm_set_s4_scheme(scheme)
                 binding.gemm_set_swap_ab(swap)
                 binding.gemm_set_kernel_family(rest[0] if rest else 0)

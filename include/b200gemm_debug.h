@@ -273,6 +273,19 @@ int gemm_debug_host_cost(int precision, int M, int N, int K, const void* A, cons
  */
 int gemm_debug_read_probe(const void* data, size_t bytes, gemm_stream_t stream);
 
+/*
+ * Measurement aid: waits for the device and returns every L2 line that is held
+ * with raised priority to normal status (cudaCtxResetPersistingL2Cache).  The
+ * tile kernels load operands they re-read with the L2 priority "evict last",
+ * and lines so marked survive any amount of ordinary traffic: a timing harness
+ * that flushes L2 by writing a large buffer does not remove them, and whatever
+ * it times next may find part of its operands in L2 (measured: a kernel that
+ * reads a 128 MB operand once ran 25.1 us from a clean L2 and 23.4 us after a
+ * tile kernel had read the same operand).  Call it between the cases of a
+ * comparison.
+ */
+int gemm_debug_reset_l2(void);
+
 #ifdef __cplusplus
 }
 #endif

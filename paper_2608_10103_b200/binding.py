@@ -23,7 +23,7 @@ EXPORTS = (
     "gemm_fp16", "gemm_s8", "gemm_s4", "gemm_s4_workspace_bytes", "gemm_s4_ws",
     "gemm_fp16_f16out", "gemm_s8_dequant", "gemm_s4_dequant", "gemm_host", "gemm_host_release",
     "gemm_s4_static", "gemm_s4_static_capacity", "gemm_release_workspaces", "gemm_unpack_s4", "gemm_mma_peak_probe", "gemm_query_config",
-    "gemm_set_config_override", "gemm_set_kernel_family", "gemm_set_s4_scheme", "gemm_set_swap_ab", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_set_stages_override", "gemm_debug_counters", "gemm_debug_host_cost", "gemm_debug_read_probe",
+    "gemm_set_config_override", "gemm_set_kernel_family", "gemm_set_s4_scheme", "gemm_set_swap_ab", "gemm_set_l2_policy", "gemm_trace_enable", "gemm_trace_read", "gemm_set_stages_override", "gemm_debug_counters", "gemm_debug_host_cost", "gemm_debug_read_probe", "gemm_debug_reset_l2",
     "gemm_last_device_status", "gemm_read_device_status", "gemm_last_cuda_error",
     "gemm_status_string", "gemm_version",
 )
@@ -349,6 +349,12 @@ def gemm_debug_read_probe(data: torch.Tensor, stream=None):
         raise ValueError("data must be a contiguous CUDA tensor")
     _check(lib().gemm_debug_read_probe(data.data_ptr(), data.numel() * data.element_size(),
                                        _stream_handle(stream)), "gemm_debug_read_probe")
+
+
+def gemm_debug_reset_l2():
+    """Waits for the device and returns L2 lines held with raised priority ("evict last") to
+    normal status, so that a following measurement starts from an L2 an ordinary flush can clear."""
+    _check(lib().gemm_debug_reset_l2(), "gemm_debug_reset_l2")
 
 
 def gemm_read_device_status(host_out: torch.Tensor, stream=None):

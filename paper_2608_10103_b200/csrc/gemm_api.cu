@@ -346,6 +346,12 @@ int gemm_debug_host_cost(int precision, int M, int N, int K, const void* A, cons
   return GEMM_OK;
 }
 
+int gemm_debug_reset_l2(void) {
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaCtxResetPersistingL2Cache();
+  return e == cudaSuccess ? GEMM_OK : cuda_fail(e);
+}
+
 int gemm_debug_read_probe(const void* data, size_t bytes, gemm_stream_t stream) {
   if (!data || bytes == 0 || (bytes & 15) || (reinterpret_cast<uintptr_t>(data) & 15))
     return GEMM_ERR_INVALID_ARG;

@@ -148,3 +148,14 @@ def test_read_probe_reads_and_writes_nothing():
         binding.gemm_debug_read_probe(data[:3])
     with pytest.raises(binding.GemmError):
         binding.gemm_debug_read_probe(data[1:5])
+
+
+def test_reset_l2_is_harmless_between_calls():
+    A, B = synth.make("s8", 300, 500, 512, seed=4)
+    dA, dB = to_dev(A), to_dev(B)
+    C = torch.empty((300, 500), dtype=torch.int32, device="cuda")
+    binding.gemm_s8(dA, dB, C)
+    binding.gemm_debug_reset_l2()
+    binding.gemm_s8(dA, dB, C)
+    torch.cuda.synchronize()
+    assert np.array_equal(C.cpu().numpy(), oracle.gemm_s8(A, B))
