@@ -935,6 +935,9 @@ def run_library_compare(args):
     index = physical_gpu_index(0)
 
     def leg(name, impl, fn, seconds, unit):
+        # L2 lines this library's kernels marked "evict last" would stay through the other
+        # implementation's whole leg (ordinary traffic does not displace them)
+        binding.gemm_debug_reset_l2()
         for _ in range(3):
             fn()
         torch.cuda.synchronize()
