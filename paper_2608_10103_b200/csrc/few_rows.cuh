@@ -111,9 +111,11 @@ template <int PENDING>
 __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
 }
-// The instruction takes its count as an immediate; pending is 1 .. FEW_ROWS_MAX_DEPTH - 1.
+// The instruction takes its count as an immediate; pending is 0 .. FEW_ROWS_MAX_DEPTH - 1 (0, a
+// ring of one slot, is never launched but must not fall through to a wait that waits for less).
 __device__ __forceinline__ void cp_async_wait_all_but(int pending) {
   switch (pending) {
+    case 0: cp_async_wait<0>(); break;
     case 1: cp_async_wait<1>(); break;
     case 2: cp_async_wait<2>(); break;
     case 3: cp_async_wait<3>(); break;

@@ -808,6 +808,10 @@ FewRowsShape few_rows_shape(int rows_l, int rows_s, int row_bytes, int num_sms) 
   f.warps = 8;
   while (f.warps > 1 && steps < 2 * f.warps) f.warps /= 2;
   if (f.warps == 8 && blocks * 8 < 12LL * num_sms && steps >= 64) f.warps = 16;
+  // (17-32 short rows: sixteen warps' sums and two ring slots do not fit the allotment)
+  while (f.warps > 1 && few_rows_ring_bytes(f.mt, nt, 2, f.warps) + few_rows_red_bytes(f.mt, nt, f.warps) +
+                                1024 > FEW_ROWS_SMEM_RING)
+    f.warps /= 2;
   const int red = few_rows_red_bytes(f.mt, nt, f.warps);
   const int slot = few_rows_ring_bytes(f.mt, nt, 1, f.warps);
   int per_sm = static_cast<int>((blocks + num_sms - 1) / num_sms);
@@ -819,6 +823,7 @@ FewRowsShape few_rows_shape(int rows_l, int rows_s, int row_bytes, int num_sms) 
     if (f.depth >= (all_at_once ? 2 : 3) || per_sm == 1) break;
   }
   if (f.depth > FEW_ROWS_MAX_DEPTH) f.depth = FEW_ROWS_MAX_DEPTH;
+  if (f.depth < 2) f.depth = 2;  // (cannot happen after the loop above; the kernel needs two)
   f.smem = few_rows_ring_bytes(f.mt, nt, f.depth, f.warps) + red;
   const long long resident = static_cast<long long>(per_sm) * num_sms;
   f.grid = static_cast<int>(blocks < resident ? blocks : resident);

@@ -34,7 +34,10 @@ def _make(prec, M, N, K, seed):
 # per row (32 packed values) over ragged steps (96, 160, 1056, 4128) to many steps per warp
 SHAPES = [(1, 1, 32), (1, 777, 512), (3, 100, 96), (8, 1000, 4128), (9, 530, 160), (12, 2049, 1056),
           (16, 4100, 2048), (16, 31, 64), (20, 600, 1056), (32, 1500, 512),
-          (777, 1, 512), (1000, 8, 4128), (2049, 12, 1056), (530, 16, 160), (600, 29, 96)]
+          (777, 1, 512), (1000, 8, 4128), (2049, 12, 1056), (530, 16, 160), (600, 29, 96),
+          # few row blocks against a long K: sixteen warps per CTA (eight with 17-32 short rows,
+          # whose sums take the room of a ring slot)
+          (20, 2048, 8192), (32, 1024, 16384), (16, 2000, 8192), (5, 1500, 16384)]
 
 
 @pytest.mark.parametrize("prec", ["fp16", "s8", "s4"])

@@ -195,6 +195,26 @@ def test_selector_invariants_over_many_shapes(lib):
             assert 1 <= c["group_m"] <= -(-M // c["BM"])
 
 
+def test_few_rows_shapes_when_forced(lib):
+    """gemm_set_kernel_family(3) takes the few-rows kernel up to 32 short rows, whatever the other
+    sizes: its launch shape must fit an SM (ring of at least two slots plus the warps' sums)."""
+    binding.gemm_set_kernel_family(3)
+    try:
+        for prec in ("fp16", "s8", "s4"):
+            for short in (1, 8, 9, 16, 17, 24, 32):
+                for long_ in (33, 512, 2048, 4096, 20001):
+                    for K in (32, 512, 4096, 8192, 16384, 131040):
+                        c = _parse(binding.gemm_query_config(prec, short, long_, K))
+                        assert "rows_per_block" in c, (prec, short, long_, K)
+                        nt = 1 if short <= 8 else 2 if short <= 16 else 4
+                        w, d = c["warps"], c["depth"]
+                        smem = d * (4 + nt) * w * 512 + w * 8 * nt * 36 * 4
+                        assert w in (1, 2, 4, 8, 16) and 2 <= d <= 8 and smem + 1024 <= 227 * 1024
+                        assert c["head"] == 0 or nt <= 2
+    finally:
+        binding.gemm_set_kernel_family(0)
+
+
 def test_selector_headline_choices(lib):
     big = _parse(binding.gemm_query_config("fp16", 8192, 8192, 8192))
     assert (big["BM"], big["BN"], big["cta_group"], big["split_k"], big["stages"]) == (512, 256, 2, 1, 4)
