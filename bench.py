@@ -635,7 +635,8 @@ def run_few_rows(args):
     torch.cuda.set_device(0)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     hbm = measured_peaks()["hbm_gbs"]
-    shapes = [(1, 8192, 8192), (8, 8192, 8192), (16, 8192, 8192), (64, 8192, 8192), (16, 4096, 16384),
+    shapes = [(1, 8192, 8192), (8, 8192, 8192), (16, 8192, 8192), (32, 8192, 8192), (64, 8192, 8192),
+              (16, 4096, 16384),
               (8, 4096, 4096), (128, 16384, 4096), (16, 28672, 8192), (32, 28672, 8192)]
     if args.shape:
         shapes = [tuple(int(x) for x in args.shape.split(","))]

@@ -92,7 +92,8 @@ int gemm_s8(int M, int N, int K, const int8_t* A, const int8_t* B, int32_t* C,
  * of byte k>>1 (low nibble first), two's complement.
  *
  * Blackwell's tcgen05.mma has no 4-bit integer kind.  A problem with at most 16
- * rows on one side (M or N) against 512 or more on the other never reaches it:
+ * rows on one side (M or N) against 512 or more on the other (at most 32 rows
+ * against 512 ... 8192) never reaches it:
  * the long operand goes from global memory straight into the fragments of the
  * warp-level integer MMA, its nibbles expanded in registers, in one launch that
  * needs no scratch and zeroes nothing (gemm_s8 does the same with up to 8

@@ -71,7 +71,8 @@ int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k);
  * nibbles in registers; a CTA owns
  * 32 rows of the long operand over the whole of K, sums its warps'
  * results and writes its part of C once.  Family 0 takes it for a short side
- * of at most 16 rows against at least 512 -- INT4 always, INT8 with up to 8
+ * of at most 16 rows against at least 512 -- INT4 always (and with 17-32
+ * rows against at most 8192), INT8 with up to 8
  * rows always and with 9-16 while the long operand has at most 64 MB, FP16
  * while it has at most 32 M elements (INT8 and FP16 only with at least six
  * 32-row blocks per KB of a row); 3 =

@@ -749,7 +749,8 @@ constexpr int FEW_ROWS_MT = 2;
 
 // Problems with a few rows on one side go to few_rows_kernel (the long operand from
 // global memory to MMA fragments without a pass through a shared tile, one launch, nothing
-// zeroed).  Automatic for a short side of up to 16 rows against 512 or more: INT4 always (it
+// zeroed).  Automatic for a short side of up to 16 rows (INT4: 32 against at most 8192) against
+// 512 or more: INT4 always (it
 // measured 0.45-0.98 of the tile kernels' time for 2048 <= N <= 28672, K = 4096 / 8192: there the
 // tile kernels are bound by expanding the nibbles in shared memory); INT8 with up to 8 short
 // rows always too (0.65-0.93 of the tile kernels' time, 0.94 of the HBM bandwidth at
@@ -773,7 +774,12 @@ bool few_rows_wanted(int M, int N, int K, bool packed_s4, const OutputSpec& out,
   const int fam = g_family;
   const int shorter = M < N ? M : N, longer = M < N ? N : M;
   if (fam == 3) return shorter <= FEW_ROWS_MAX;
-  if (fam != 0 || shorter > FEW_ROWS_AUTO || longer < 512) return false;
+  if (fam != 0 || longer < 512) return false;
+  // INT4 with 17-32 rows (four groups of short rows per warp) against up to 8192: 3-33 % ahead of
+  // the tile kernels (32 x 4096 x 4096 9.9 -> 6.7 us, 32 x 8192 x 8192 16.4 -> 16.0); behind from
+  // 16384 rows on (32 x 28672 x 8192: 46.3 against 35.7 us)
+  if (packed_s4 && shorter > FEW_ROWS_AUTO) return shorter <= FEW_ROWS_MAX && longer <= 8192;
+  if (shorter > FEW_ROWS_AUTO) return false;
   if (packed_s4) return true;
   // A CTA's time grows with the length of a row (its 16 warps share it), the tile kernels
   // split K over as many CTAs as it takes: few row blocks against long rows stay on tiles.

@@ -152,7 +152,8 @@ def test_few_rows_automatic_rule():
     binding.gemm_set_kernel_family(0)
     few = lambda prec, M, N, K: binding.gemm_query_config(prec, M, N, K).startswith("few_rows")
     assert few("s4", 16, 8192, 8192) and few("s4", 1, 28672, 8192) and few("s4", 4096, 9, 1024)
-    assert not few("s4", 17, 8192, 8192) and not few("s4", 16, 500, 8192)
+    assert few("s4", 17, 8192, 8192) and few("s4", 32, 4096, 4096)       # 17-32 rows: up to 8192
+    assert not few("s4", 17, 16384, 8192) and not few("s4", 33, 8192, 8192) and not few("s4", 16, 500, 8192)
     assert few("s8", 8, 2048, 4096) and few("s8", 16, 4096, 8192) and few("s8", 16, 8192, 8192)
     assert few("s4", 16, 512, 8192)
     assert few("s8", 8, 28672, 8192)

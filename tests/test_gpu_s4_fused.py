@@ -88,7 +88,7 @@ def test_fused_pair_tiles_with_split_k(M, N, K, bn, split_k):
 
 def test_automatic_route_by_shape():
     binding.gemm_set_s4_scheme(0)
-    assert "fused_unpack" in binding.gemm_query_config("s4", 24, 8192, 8192)      # few rows
+    assert "fused_unpack" in binding.gemm_query_config("s4", 48, 8192, 8192)      # few rows
     assert binding.gemm_query_config("s4", 16, 8192, 8192).startswith("few_rows")  # up to 16: no tiles
     assert "fused_unpack" in binding.gemm_query_config("s4", 8192, 64, 4096)
     assert "fused_unpack" in binding.gemm_query_config("s4", 512, 512, 512)       # small
@@ -114,7 +114,7 @@ def test_automatic_route_by_shape():
     binding.gemm_set_s4_scheme(1)
     assert "prepass" in binding.gemm_query_config("s4", 16, 8192, 8192)
     binding.gemm_set_s4_scheme(0)
-    M, N, K = 24, 4096, 8192
+    M, N, K = 48, 4096, 8192
     A, B = synth.s4_uniform(M, N, K, seed=11)
     check_against_oracle("s4", A, B, run_gpu("s4", A, B, fill=-7), force_full=True)
     for M, N, K in [(200, 20000, 2080), (300, 5000, 1056)]:   # two waves of pair tiles; one-CTA tiles

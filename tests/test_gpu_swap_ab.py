@@ -74,7 +74,7 @@ def test_swapped_output_variants():
 
 def test_automatic_choice_for_few_rows():
     binding.gemm_set_swap_ab(0)
-    cfg = binding.gemm_query_config("s4", 24, 8192, 8192)
+    cfg = binding.gemm_query_config("s4", 48, 8192, 8192)
     assert "fused_unpack" in cfg and "swap_ab" in cfg
     assert binding.gemm_query_config("s4", 16, 8192, 8192).startswith("few_rows")
     assert "swap_ab" in binding.gemm_query_config("s4", 64, 8192, 8192)

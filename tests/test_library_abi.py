@@ -128,7 +128,8 @@ def test_selector_invariants_over_many_shapes(lib):
             c = _parse(text)
             if text.startswith("few_rows"):   # the kernel for a short side of up to 16 rows
                 short, long_ = min(M, N), max(M, N)
-                assert short <= 16 and long_ >= 512 and c["short_rows"] == short
+                assert (short <= 16 or (prec == "s4" and short <= 32 and long_ <= 8192)) and long_ >= 512
+                assert c["short_rows"] == short
                 if prec == "s8":
                     assert short <= 8 or long_ * K <= 64 << 20
                 if prec == "fp16":
@@ -141,7 +142,7 @@ def test_selector_invariants_over_many_shapes(lib):
                 w, d = c["warps"], c["depth"]
                 assert w in (1, 2, 4, 8, 16) and 2 <= d <= 8
                 assert w == 1 or -(-row_bytes // 64) >= 2 * w      # two 64-byte steps per warp
-                nt, mt = (1 if short <= 8 else 2), rows // 16
+                nt, mt = (1 if short <= 8 else 2 if short <= 16 else 4), rows // 16
                 smem = d * (2 * mt + nt) * w * 512 + w * 8 * nt * (16 * mt + 4) * 4
                 per_sm = min((227 * 1024) // (smem + 1024), 64 // w, 32)
                 assert per_sm >= 1 and 1 <= c["ctas"] <= min(c["blocks"], per_sm * 148)
@@ -235,7 +236,9 @@ def test_selector_headline_choices(lib):
     assert binding.gemm_query_config("s8", 16, 8192, 8192).startswith("few_rows")
     assert not binding.gemm_query_config("s8", 16, 28672, 8192).startswith("few_rows")
     assert binding.gemm_query_config("s8", 8, 28672, 8192).startswith("few_rows")
-    assert not binding.gemm_query_config("s4", 17, 8192, 8192).startswith("few_rows")
+    assert binding.gemm_query_config("s4", 17, 8192, 8192).startswith("few_rows")
+    assert not binding.gemm_query_config("s4", 17, 8200, 8192).startswith("few_rows")
+    assert not binding.gemm_query_config("s4", 33, 8192, 8192).startswith("few_rows")
     tail = _parse(binding.gemm_query_config("fp16", 4096, 4096, 8192))
     assert tail["split_k"] == 2 and tail["split_tiles"] == 256 % 74
     binding.gemm_set_config_override(0, 0, 0, 1)
