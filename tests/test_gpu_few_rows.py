@@ -187,3 +187,39 @@ def test_few_rows_in_a_cuda_graph():
         g.replay()
         torch.cuda.synchronize()
         assert np.array_equal(C.cpu().numpy(), ref)
+
+
+def test_few_rows_seeded_walk_of_shapes():
+    """Random short sides (1..32), long sides, K and orientations through every launch shape the
+    host picks (warps 1..16, ring depths 2..8, with and without the step through registers),
+    each checked against the oracle on sampled rows."""
+    g = np.random.Generator(np.random.PCG64(4321))
+    shapes_met = set()
+    cases = 0
+    while cases < 80:
+        M = int(g.integers(1, 33))
+        kind = int(g.integers(4))
+        N = (int(g.integers(1, 600)) if kind == 0 else int(g.integers(600, 9000)) if kind == 1
+             else int(g.integers(9000, 40000)) if kind == 2 else int(g.choice([512, 2048, 4096, 8192])))
+        K = (int(g.integers(1, 40)) * 32 if g.integers(3) == 0 else int(g.integers(1, 300)) * 32
+             if g.integers(2) == 0 else int(g.choice([4096, 8192, 16384, 32768])))
+        prec = str(g.choice(["fp16", "s8", "s4"]))
+        if (M + N) * K > 150e6:
+            continue
+        if g.integers(3) == 0:
+            M, N = N, M
+        cases += 1
+        cfg = binding.gemm_query_config(prec, M, N, K)
+        assert cfg.startswith("few_rows"), cfg
+        shapes_met.add(tuple(cfg.split(k)[1].split()[0] for k in ("warps=", "depth=", "head=")))
+        A, B = synth.make(prec, M, N, K, seed=int(g.integers(1 << 30)))
+        rows = np.unique(np.concatenate([g.choice(M, size=min(10, M), replace=False), [0, M - 1]])).astype(np.int32)
+        got = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)[rows]
+        what = "%s %d x %d x %d: %s" % (prec, M, N, K, cfg)
+        if prec == "fp16":
+            ref, S = oracle.gemm_fp16(A, B, rows=rows)
+            assert oracle.fp16_check(got, ref, S)[0], what
+        else:
+            exact = oracle.gemm_s8_i64(A, B, rows=rows) if prec == "s8" else oracle.gemm_s4_i64(A, B, K, rows=rows)
+            assert np.array_equal(got.astype(np.int64), exact), what
+    assert len(shapes_met) >= 12, shapes_met
