@@ -10,17 +10,20 @@
 // against 8 rows of the short one per instruction) from registers, and every thread fetches
 // exactly the 16-byte pieces its own fragment registers need.
 //
-// Work split: one CTA per 16 (32) rows of the long operand over the whole of K; its warps share
-// K in 64-byte steps, each warp a contiguous run of them (so that a warp streams 64 x steps
+// Work split: one CTA per 16 MT rows of the long operand (the library launches MT = 2: a warp
+// then uses every fragment of the short operand twice) over the whole of K; its warps share K
+// in 64-byte steps, each warp a contiguous run of them (so that a warp streams 64 x steps
 // consecutive bytes of each of its rows: taking the steps in turn, warp w: w, w + warps, ...,
-// measured 2-8 % slower).  Every CTA sums its warps' results in shared memory and writes its 16
-// (32) columns (or rows) of C itself: no zeroed C, no atomics, no second launch.
+// measured 2-8 % slower).  Every CTA sums its warps' results in shared memory and writes its
+// 16 MT columns (or rows) of C itself: no zeroed C, no atomics, no second launch.
 //
 // Latency: a step's pieces travel by cp.async into a ring of `depth` slots that is private to the
 // thread (nobody else reads them, so no barrier is involved: the thread waits for its own copy
 // group and loads the pieces back), which keeps that many steps -- depth KB of the long operand per
 // warp -- in flight without holding registers.  (Fetching straight into registers, two steps
-// ahead, left the warps waiting on the loads for 33 of every 39 cycles and HBM at 31 %.)
+// ahead, left the warps waiting on the loads for 33 of every 39 cycles and HBM at 31 %.)  On top
+// of the ring, HEAD steps of a CTA's first block may travel through registers, issued before
+// the ring's first copies: worth 3-9 % where the registers do not cost a resident CTA.
 //
 // K order: a dot product may take K in any order as long as both operands use the same one.
 // Lane (g, t) = (lane / 4, lane % 4) fetches the 16 bytes at offset 16 t of a step from rows g
