@@ -32,6 +32,15 @@
  * results then depend on the order the partial sums land, i.e. two runs can
  * differ in the last bits, always inside the stated bound.
  *
+ * L2.  The tile kernels fetch the operand they re-read (a band of A, or the
+ * long operand of a problem with few rows) with the L2 eviction priority "evict
+ * last".  Lines so marked are displaced by other such lines but not by ordinary
+ * traffic, so after a call part of L2 stays occupied by operand data until
+ * later calls of this library replace it or the application returns the lines
+ * to normal status (cudaCtxResetPersistingL2Cache; gemm_debug_reset_l2 in
+ * b200gemm_debug.h does that).  A timing harness that "flushes L2" by writing a
+ * large buffer does not remove them.
+ *
  * All functions return GEMM_OK (0) or a negative GEMM_ERR_* code.
  * A process may call from several host threads (the call path takes no global
  * lock); calls that share a stream are ordered by it, and two threads that
