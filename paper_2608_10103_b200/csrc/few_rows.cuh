@@ -84,7 +84,7 @@ namespace few_rows_detail {
 
 // 16 bytes global -> shared, asynchronously; bytes = 0 writes zeros and reads nothing.
 // cg: through L2 only (the long operand, read once); ca: kept in L1 too (the short operand,
-// which every CTA of the SM reads again).
+// which every CTA of the SM reads again: a third of the kernel's requests).
 __device__ __forceinline__ void cp_async_16_cg(uint32_t dst, const uint8_t* src, int bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes)
                : "memory");
@@ -93,18 +93,34 @@ __device__ __forceinline__ void cp_async_16_ca(uint32_t dst, const uint8_t* src,
   asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes)
                : "memory");
 }
+// Loads into registers.  Ordinary (coherent) loads, never ld.global.nc: the kernel may have been
+// launched while the grid in front of it was still writing its operands (programmatic dependent
+// launch), and the non-coherent path promises nothing for data written during the kernel's
+// lifetime -- with .nc here INT4 through gemm_host, whose int8 scratch is rewritten by the unpack
+// kernel right in front, came out with a few hundred wrong sums per call (stale lines of the
+// scratch from the call before).  What griddepcontrol.wait makes visible, ordinary loads see.
 __device__ __forceinline__ uint4 ld_stream_16(const uint8_t* p) {
   uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+  asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
+               : "l"(p)
+               : "memory");
   return v;
 }
 __device__ __forceinline__ uint4 ld_cached_16(const uint8_t* p) {
   uint4 v;
-  asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];"
+  asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
+               : "l"(p)
+               : "memory");
+  return v;
+}
+__device__ __forceinline__ void prefetch_l2(const uint8_t* p) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+__device__ __forceinline__ float ld_f32(const float* p) {
+  float v;
+  asm volatile("ld.global.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
   return v;
 }
 __device__ __forceinline__ void cp_async_commit() {
@@ -194,7 +210,6 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   Acc* red = reinterpret_cast<Acc*>(few_rows_smem + few_rows_ring_bytes(MT, NT, depth, warps));
 
   if (tid == 0) ptx::grid_dep_launch_dependents();
-  if (p.wait_prior_grid) ptx::grid_dep_wait();
 
   // rows past the end are read as the last row (valid memory) and dropped at the store
   const int last_l = p.rows_l - 1, last_s = p.rows_s - 1;
@@ -222,6 +237,22 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
       lrow[r] = p.L + static_cast<long long>(min(l0 + g + 8 * r, last_l)) * p.l_pitch;
   };
   rows_of(0);
+  if (p.wait_prior_grid) {
+    // Launched to start while the grid in front still runs: nothing may be read before that
+    // grid has finished (it may be writing the operands), but the lines of the first steps can
+    // be asked into L2 meanwhile -- a prefetch returns no data, and L2 is where that grid's
+    // writes land too.  The quad of a row shares its first 128-byte lines between its lanes.
+    if (my_blocks > 0) {
+      const int lines = (min(my_steps, depth + HEAD) * 64 + 127) >> 7;
+#pragma unroll
+      for (int r = 0; r < 2 * MT; ++r)
+        for (int j = t; j < lines; j += 4) {
+          const int off = first_step * 64 + j * 128;
+          if (off < p.row_bytes) prefetch_l2(lrow[r] + off);
+        }
+    }
+    ptx::grid_dep_wait();
+  }
   // The first HEAD steps of a CTA's first block travel through registers, on top of what the
   // ring holds: that much more is in flight from the start, and the ring's first round trip
   // begins one step further on.
@@ -384,7 +415,7 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
       } else if constexpr (F16) {
         static_cast<__half*>(p.C)[at] = __float2half_rn(sum);  // EPI_OUT16: rounded once
       } else {
-        const float fs = __ldg(p.scale_s + s), fl = __ldg(p.scale_l + l0 + l);
+        const float fs = ld_f32(p.scale_s + s), fl = ld_f32(p.scale_l + l0 + l);
         const float x = p.scale_s_first ? static_cast<float>(sum) * fs * fl
                                         : static_cast<float>(sum) * fl * fs;
         if constexpr (EPI == EPI_OUT16)
