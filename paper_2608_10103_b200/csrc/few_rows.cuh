@@ -429,8 +429,9 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   cp_async_wait<0>();
 }
 
-// Measurement aid: reads `bytes` (a multiple of 16) once with 16-byte loads, eight in flight per
-// thread, and keeps nothing -- what a call bound by reading one operand could at best take in a
+// Measurement aid: reads `bytes` (a multiple of 16) once with 16-byte (coherent) loads, eight in
+// flight per thread, after the wait for the grid in front like any kernel that has to assume that
+// grid wrote its input, and keeps nothing -- what a call bound by reading one operand could at best take in a
 // given harness (launch, first-byte latency and tail included).  `sink` is never written.
 __global__ void __launch_bounds__(256) read_probe_kernel(const uint8_t* data, size_t bytes,
                                                          unsigned* sink, int wait_prior_grid) {
@@ -446,9 +447,10 @@ __global__ void __launch_bounds__(256) read_probe_kernel(const uint8_t* data, si
       const size_t at = base + (static_cast<size_t>(u) * blockDim.x + threadIdx.x) * 16;
       v[u] = make_uint4(0, 0, 0, 0);
       if (at < bytes)
-        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+        asm volatile("ld.global.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
                      : "=r"(v[u].x), "=r"(v[u].y), "=r"(v[u].z), "=r"(v[u].w)
-                     : "l"(data + at));
+                     : "l"(data + at)
+                     : "memory");
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) acc += v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;

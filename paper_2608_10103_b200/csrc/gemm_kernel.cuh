@@ -969,7 +969,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             ptx::grid_dep_wait();
             prior_grid_done = true;
           }
-          if (p.row_scale && row < p.M) rs = __ldg(p.row_scale + row);
+          if (p.row_scale && row < p.M) rs = ptx::ld_global_f32(p.row_scale + row);
           if (p.col_scale && lane * 32 < BN && col0 + lane * 32 < p.N)
             ptx::prefetch_l1(p.col_scale + col0 + lane * 32);
         }
@@ -1082,7 +1082,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           // Column factors: one coalesced load per 32 columns (lane v fetches column v's),
           // handed round by shuffles -- a load per element, even from L1, made this loop
           // wait ~25 cycles per column.
-          const float cs_mine = (col + lane < p.N) ? __ldg(p.col_scale + col + lane) : 0.0f;
+          const float cs_mine = (col + lane < p.N) ? ptx::ld_global_f32(p.col_scale + col + lane) : 0.0f;
           ptx::tmem_ld_32x32b_x32(
               tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), w);
           ptx::tmem_wait_ld();
@@ -1096,7 +1096,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 #pragma unroll
           for (int h = 0; h < BLOCK_COLS / 32; ++h) {
             const int cc = col + h * 32 + lane;
-            const float cs_mine = (p.col_scale && cc < p.N) ? __ldg(p.col_scale + cc) : 0.0f;
+            const float cs_mine = (p.col_scale && cc < p.N) ? ptx::ld_global_f32(p.col_scale + cc) : 0.0f;
             uint32_t r[32];
             ptx::tmem_ld_32x32b_x32(
                 tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * BLOCK_COLS + h * 32), r);

@@ -356,7 +356,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
 #pragma unroll
           for (int a = 0; a < 2; ++a) {
             const int row = cta_row0 + a * BM + quarter * 32 + lane;
-            if (p.row_scale && row < p.M) rs[a] = __ldg(p.row_scale + row);
+            if (p.row_scale && row < p.M) rs[a] = ptx::ld_global_f32(p.row_scale + row);
           }
           if (p.col_scale && lane < 4 && col_base + lane * 32 < p.N)
             ptx::prefetch_l1(p.col_scale + col_base + lane * 32);
@@ -404,7 +404,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
 #pragma unroll
             for (int i = 0; i < 32; ++i) w[i] = v[c][i];
           } else if constexpr (EPI == EPI_F32_SCALED) {
-            const float cs_mine = (col + lane < p.N) ? __ldg(p.col_scale + col + lane) : 0.0f;
+            const float cs_mine = (col + lane < p.N) ? ptx::ld_global_f32(p.col_scale + col + lane) : 0.0f;
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const float cs = __shfl_sync(0xffffffffu, cs_mine, i);
@@ -414,7 +414,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_a,
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
               const int cc = col + h * 32 + lane;
-              const float cs_mine = (p.col_scale && cc < p.N) ? __ldg(p.col_scale + cc) : 0.0f;
+              const float cs_mine = (p.col_scale && cc < p.N) ? ptx::ld_global_f32(p.col_scale + cc) : 0.0f;
 #pragma unroll
               for (int i = 0; i < 32; i += 2) {
                 float x0 = acc_to_float<KIND>(v[2 * c + h][i]);

@@ -410,6 +410,26 @@ __device__ __forceinline__ void st_global_v4_hint(void* p, uint32_t a, uint32_t 
                : "memory");
 }
 
+// Ordinary (coherent) global loads for data that the grid in front of a kernel may have written.
+// A kernel launched with programmatic stream serialization starts before that grid has finished
+// and reads such data only after griddepcontrol.wait; loads through the non-coherent path
+// (ld.global.nc, __ldg) carry no such order -- the compiler may place them above the wait --
+// and promise nothing for data written during the kernel's lifetime, so they are not used for it.
+__device__ __forceinline__ float ld_global_f32(const float* p) {
+  float v;
+  asm volatile("ld.global.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+  return v;
+}
+// ... 16 bytes that are read once (no L1 allocation).
+__device__ __forceinline__ uint4 ld_global_stream_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p)
+               : "memory");
+  return v;
+}
+
 // Hint: bring the line at p into this SM's L1.
 __device__ __forceinline__ void prefetch_l1(const void* p) {
   asm volatile("prefetch.global.L1 [%0];" ::"l"(p));

@@ -53,7 +53,7 @@ unpack_s4_kernel(UnpackJob a, UnpackJob b, int chunks_per_row, long long out_pit
     int8_t* out = second ? b.out : a.out;
     const long long row = idx / chunks_per_row;
     const int chunk = static_cast<int>(idx - row * chunks_per_row);
-    const uint4 w = __ldg(src + idx);
+    const uint4 w = ptx::ld_global_stream_v4(src + idx);
     uint4 o0, o1;
     unpack8_s4(w.x, o0.x, o0.y);
     unpack8_s4(w.y, o0.z, o0.w);
@@ -92,7 +92,7 @@ expand_s4_slots_kernel(const uint8_t* packed, int8_t* out, long long rows, int k
     const int j = static_cast<int>(g - row * chunks_per_row);
     uint4 w = make_uint4(0, 0, 0, 0);
     if (j * 16 < k_bytes)
-      w = __ldg(reinterpret_cast<const uint4*>(packed + row * k_bytes + static_cast<long long>(j) * 16));
+      w = ptx::ld_global_stream_v4(packed + row * k_bytes + static_cast<long long>(j) * 16);
     const int ps = j >> 3, h = (j >> 2) & 1, c = j & 3;
     int8_t* dst = out + row * out_pitch + static_cast<long long>(ps) * 256 + h * 128 + c * 16;
     *reinterpret_cast<uint4*>(dst) =
