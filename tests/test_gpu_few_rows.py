@@ -223,3 +223,44 @@ def test_few_rows_seeded_walk_of_shapes():
             exact = oracle.gemm_s8_i64(A, B, rows=rows) if prec == "s8" else oracle.gemm_s4_i64(A, B, K, rows=rows)
             assert np.array_equal(got.astype(np.int64), exact), what
     assert len(shapes_met) >= 12, shapes_met
+
+
+def test_few_rows_operands_written_by_the_launch_in_front():
+    """The kernel may start while the kernel in front of it in the stream still runs and must read
+    nothing before that one has finished: operands and scale factors rewritten right in front of
+    every call (a device-to-device copy kernel, then the GEMM, no synchronisation in between), the
+    result of every call checked afterwards.  (Loads through the non-coherent path were once
+    placed above the wait for the grid in front and read the values of the call before.)"""
+    M, N, K = 8, 4096, 2048
+    rounds = 6
+    g = np.random.Generator(np.random.PCG64(11))
+    for prec in ("s8", "s4", "fp16"):
+        data = [_make(prec, M, N, K, seed=100 + r) for r in range(rounds)]
+        src = [(to_dev(A), to_dev(B)) for A, B in data]
+        dA, dB = torch.empty_like(src[0][0]), torch.empty_like(src[0][1])
+        outs = [torch.empty((M, N), dtype=torch.float32 if prec == "fp16" else torch.int32, device="cuda")
+                for _ in range(rounds)]
+        for rep in range(3):
+            for r in range(rounds):
+                dA.copy_(src[r][0])
+                dB.copy_(src[r][1])
+                binding.gemm(prec, dA, dB, outs[r])
+            torch.cuda.synchronize()
+            for r in range(rounds):
+                check_against_oracle(prec, data[r][0], data[r][1], outs[r].cpu().numpy(), force_full=(rep == 0 and r < 2))
+    # scale factors written in front of a dequantising call
+    A, B = _make("s8", M, N, K, seed=7)
+    dA, dB = to_dev(A), to_dev(B)
+    acc = oracle.gemm_s8(A, B).astype(np.int64)
+    rs_d, cs_d = torch.empty(M, device="cuda"), torch.empty(N, device="cuda")
+    C = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    for r in range(rounds):
+        rs = (g.uniform(0.5, 2.0, M) * 1e-2).astype(np.float32)
+        cs = (g.uniform(0.5, 2.0, N) * 1e-2).astype(np.float32)
+        rs_src, cs_src = to_dev(rs), to_dev(cs)
+        rs_d.copy_(rs_src)
+        cs_d.copy_(cs_src)
+        binding.gemm_s8_dequant(dA, dB, rs_d, cs_d, C, torch.float32)
+        torch.cuda.synchronize()
+        ok, worst = oracle.dequant_check(C.cpu().numpy(), oracle.dequant_ref(acc, rs, cs), False)
+        assert ok, worst

@@ -58,3 +58,24 @@ def test_host_path_argument_errors_and_release():
     hC = binding.gemm_host("s8", torch.from_numpy(A), torch.from_numpy(B))
     torch.cuda.synchronize()
     assert np.array_equal(hC.numpy(), oracle.gemm_s8(A, B))
+
+
+def test_host_path_few_rows_after_other_precisions():
+    """INT4 through the host entry point expands its operands into a scratch right in front of the
+    GEMM; with a few rows that GEMM is the kernel that starts early and must not read the scratch
+    before the expansion has finished (it once did, and returned sums of the call before)."""
+    import numpy as np
+    for rep in range(2):
+        for prec in synth.PRECISIONS:
+            for M, N, K in [(8, 4096, 2048), (3000, 12, 1056), (16, 5000, 4128)]:
+                A, B = synth.make(prec, M, N, K, seed=5 + rep)
+                hA, hB = torch.from_numpy(A).pin_memory(), torch.from_numpy(B).pin_memory()
+                C = binding.gemm_host(prec, hA, hB)
+                torch.cuda.synchronize()
+                got = C.numpy()
+                if prec == "fp16":
+                    ref, S = oracle.gemm_fp16(A, B)
+                    assert oracle.fp16_check(got, ref, S)[0], (prec, M, N, K)
+                else:
+                    ref = oracle.gemm_s8(A, B) if prec == "s8" else oracle.gemm_s4(A, B, K)
+                    assert np.array_equal(got, ref), (prec, M, N, K, int((got != ref).sum()))
