@@ -277,8 +277,7 @@ int gemm_unpack_s4(int rows, int K, const uint8_t* packed, int8_t* out, size_t o
  * kernel runs on exchanged operands (the tile is then described in the
  * kernel's orientation).  A problem that goes to the kernel for a few rows
  * instead of a tile kernel reads "few_rows rows_per_block=32 blocks=256
- * short_rows=16 warps=8 depth=3 head=1 ctas=256 kind=i8" (" s4=in_registers" for
- * INT4).
+ * short_rows=16 warps=8 depth=3 ctas=256 kind=i8" (" s4=in_registers" for INT4).
  * Describes the raw 32-bit outputs (gemm_fp16, gemm_s8, gemm_s4).  Host only,
  * no GPU work.
  */

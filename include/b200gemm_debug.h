@@ -79,7 +79,7 @@ int gemm_set_config_override(int bn, int group_m, int cta_group, int split_k);
  * wherever it exists (a short side of at most 32 rows); 1 and 2 never, nor do
  * calls with a forced tile shape, operand order or INT4 scheme, or traced ones.
  * gemm_query_config describes such a call as "few_rows rows_per_block=..
- * blocks=.. short_rows=.. warps=.. depth=.. head=.. ctas=..".
+ * blocks=.. short_rows=.. warps=.. depth=.. ctas=..".
  */
 int gemm_set_kernel_family(int family);
 

@@ -21,9 +21,9 @@
 // thread (nobody else reads them, so no barrier is involved: the thread waits for its own copy
 // group and loads the pieces back), which keeps that many steps -- depth KB of the long operand per
 // warp -- in flight without holding registers.  (Fetching straight into registers, two steps
-// ahead, left the warps waiting on the loads for 33 of every 39 cycles and HBM at 31 %.)  On top
-// of the ring, HEAD steps of a CTA's first block may travel through registers, issued before
-// the ring's first copies: worth 3-9 % where the registers do not cost a resident CTA.
+// ahead, left the warps waiting on the loads for 33 of every 39 cycles and HBM at 31 %.)  Before
+// the kernel waits for the grid in front of it (it is launched to start early) every warp asks
+// the lines of its first steps into L2: their HBM latency then overlaps that grid's tail.
 //
 // K order: a dot product may take K in any order as long as both operands use the same one.
 // Lane (g, t) = (lane / 4, lane % 4) fetches the 16 bytes at offset 16 t of a step from rows g
@@ -93,31 +93,16 @@ __device__ __forceinline__ void cp_async_16_ca(uint32_t dst, const uint8_t* src,
   asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes)
                : "memory");
 }
-// Loads into registers.  Ordinary (coherent) loads, never ld.global.nc: the kernel may have been
-// launched while the grid in front of it was still writing its operands (programmatic dependent
-// launch), and the non-coherent path promises nothing for data written during the kernel's
-// lifetime -- with .nc here INT4 through gemm_host, whose int8 scratch is rewritten by the unpack
-// kernel right in front, came out with a few hundred wrong sums per call (stale lines of the
-// scratch from the call before).  What griddepcontrol.wait makes visible, ordinary loads see.
-__device__ __forceinline__ uint4 ld_stream_16(const uint8_t* p) {
-  uint4 v;
-  asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p)
-               : "memory");
-  return v;
-}
-__device__ __forceinline__ uint4 ld_cached_16(const uint8_t* p) {
-  uint4 v;
-  asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p)
-               : "memory");
-  return v;
-}
+// (The kernel may have been launched while the grid in front of it was still writing its
+// operands -- programmatic dependent launch -- and reads nothing before griddepcontrol.wait.  The
+// non-coherent path, ld.global.nc / __ldg, carries no order against that wait and promises
+// nothing for data written during the kernel's lifetime: a version that fetched a step into
+// registers with it returned a few hundred wrong sums per call for INT4 through gemm_host, whose
+// int8 scratch is rewritten by the unpack kernel right in front.  Nothing here uses it.)
 __device__ __forceinline__ void prefetch_l2(const uint8_t* p) {
   asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
+// Scale factors: an ordinary load, for the same reason.
 __device__ __forceinline__ float ld_f32(const float* p) {
   float v;
   asm volatile("ld.global.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
@@ -185,12 +170,11 @@ __device__ __forceinline__ uint32_t high_nibbles_x16(uint32_t w) { return w & 0x
 // KIND: int8, packed 4-bit or binary16 operands.  MT: groups of 16 long rows per CTA (a warp holds the
 // fragments of all of them and uses each short fragment MT times: the short operand, fetched
 // again by every CTA, costs 8 NT / (16 MT) of the long operand's bytes in requests).  NT: groups
-// of eight short rows.  EPI: as for the tile kernels.  HEAD: steps of the first block that go
-// through registers instead of the ring (costs 4 (2 MT + NT) registers each).
+// of eight short rows.  EPI: as for the tile kernels.
 // Dynamic shared memory: few_rows_ring_bytes + few_rows_red_bytes.  Any grid size: CTA c takes
 // the row blocks c, c + grid, ...; its copies run ahead across the block boundaries, so only
 // the first block of a CTA waits for the memory latency in full.
-template <int KIND, int MT, int NT, int EPI, int HEAD = 0>
+template <int KIND, int MT, int NT, int EPI>
 __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
   using namespace few_rows_detail;
   constexpr bool S4 = KIND == FEW_ROWS_S4, F16 = KIND == FEW_ROWS_F16;
@@ -243,7 +227,7 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
     // be asked into L2 meanwhile -- a prefetch returns no data, and L2 is where that grid's
     // writes land too.  The quad of a row shares its first 128-byte lines between its lanes.
     if (my_blocks > 0) {
-      const int lines = (min(my_steps, depth + HEAD) * 64 + 127) >> 7;
+      const int lines = (min(my_steps, depth) * 64 + 127) >> 7;
 #pragma unroll
       for (int r = 0; r < 2 * MT; ++r)
         for (int j = t; j < lines; j += 4) {
@@ -252,29 +236,6 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
         }
     }
     ptx::grid_dep_wait();
-  }
-  // The first HEAD steps of a CTA's first block travel through registers, on top of what the
-  // ring holds: that much more is in flight from the start, and the ring's first round trip
-  // begins one step further on.
-  constexpr int HN = HEAD > 0 ? HEAD : 1;
-  const int head = (HEAD > 0 && my_blocks > 0) ? min(HEAD, my_steps) : 0;
-  uint4 ha[HN][2 * MT], hb[HN][NT];
-  if constexpr (HEAD > 0) {
-#pragma unroll
-    for (int h = 0; h < HEAD; ++h) {
-      const int off = (first_step + h) * 64 + t * 16;
-      const bool in = h < head && off < p.row_bytes;
-#pragma unroll
-      for (int r = 0; r < 2 * MT; ++r)
-        ha[h][r] = in ? ld_stream_16(lrow[r] + off) : make_uint4(0, 0, 0, 0);
-#pragma unroll
-      for (int j = 0; j < NT; ++j) hb[h][j] = in ? ld_cached_16(sp[j] + off) : make_uint4(0, 0, 0, 0);
-    }
-    f_step = head;
-    if (my_steps > 0 && f_step == my_steps) {
-      f_step = 0;
-      rows_of(++f_block);
-    }
   }
   auto fetch = [&]() {  // this thread's pieces of the next step into the next ring slot
     if (f_block < my_blocks && my_steps > 0) {
@@ -355,17 +316,8 @@ __global__ void __launch_bounds__(512) few_rows_kernel(const FewRowsParams p) {
       for (int j = 0; j < NT; ++j)
 #pragma unroll
         for (int v = 0; v < 4; ++v) acc[m][j][v] = 0;
-    int i0 = 0;
-    if constexpr (HEAD > 0) {
-      if (blk == 0) {
-#pragma unroll
-        for (int h = 0; h < HEAD; ++h)
-          if (h < head) mac(ha[h], hb[h], acc);
-        i0 = head;
-      }
-    }
 #pragma unroll 1
-    for (int i = i0; i < my_steps; ++i) {
+    for (int i = 0; i < my_steps; ++i) {
       cp_async_wait_all_but(depth - 1);  // all but the newest depth - 1 groups: this step has landed
       const uint32_t slot = ring + static_cast<uint32_t>(c_slot * PIECES) * piece_pitch;
       c_slot = c_slot + 1 == depth ? 0 : c_slot + 1;

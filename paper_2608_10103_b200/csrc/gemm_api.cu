@@ -169,9 +169,8 @@ int gemm_query_config(int precision, int M, int N, int K, char* buf, int len) {
     const int row_bytes = precision == GEMM_PREC_S4 ? K / 2 : precision == GEMM_PREC_FP16 ? 2 * K : K;
     const FewRowsShape f = few_rows_shape(rows_l, M < N ? M : N, row_bytes, num_sms);
     snprintf(buf, static_cast<size_t>(len),
-             "few_rows rows_per_block=%d blocks=%d short_rows=%d warps=%d depth=%d head=%d ctas=%d "
-             "kind=%s%s",
-             16 * f.mt, ceil_div(rows_l, 16 * f.mt), M < N ? M : N, f.warps, f.depth, f.head, f.grid,
+             "few_rows rows_per_block=%d blocks=%d short_rows=%d warps=%d depth=%d ctas=%d kind=%s%s",
+             16 * f.mt, ceil_div(rows_l, 16 * f.mt), M < N ? M : N, f.warps, f.depth, f.grid,
              precision == GEMM_PREC_FP16 ? "f16" : "i8",
              precision == GEMM_PREC_S4 ? " s4=in_registers" : "");
     return GEMM_OK;

@@ -790,7 +790,7 @@ bool few_rows_wanted(int M, int N, int K, bool packed_s4, const OutputSpec& out,
 }
 
 struct FewRowsShape {
-  int mt, depth, warps, grid, smem, head;
+  int mt, depth, warps, grid, smem;
 };
 
 constexpr int FEW_ROWS_SMEM_SM = 227 * 1024;  // shared memory of an SM; each CTA reserves 1 KB more
@@ -833,21 +833,15 @@ FewRowsShape few_rows_shape(int rows_l, int rows_s, int row_bytes, int num_sms) 
   f.smem = few_rows_ring_bytes(f.mt, nt, f.depth, f.warps) + red;
   const long long resident = static_cast<long long>(per_sm) * num_sms;
   f.grid = static_cast<int>(blocks < resident ? blocks : resident);
-  // One step through registers on top of the ring (up to 16 short rows: 10.1 -> 9.2 us at
-  // 16 x 8192 x 8192, 9.2 -> 8.9 us at 1 x 8192 x 8192, INT4) where its registers, up to 128 per
-  // thread, do not cost a resident CTA (three CTAs of eight warps per SM did: 13.7 -> 14.7 us at
-  // 16 x 12288 x 8192).
-  f.head = (nt <= 2 && per_sm * f.warps <= 16) ? 1 : 0;
   return f;
 }
 
-template <int FKIND, int NT, int EPI, int HEAD>
+template <int FKIND, int NT, int EPI>
 int launch_few_rows_nt(DeviceState* s, FewRowsParams& p, const FewRowsShape& f,
                        cudaStream_t stream) {
-  // attr_set bits 256..309: by operand kind, short-row groups, output mode, register head
-  constexpr int variant =
-      256 + ((FKIND * 3 + (NT == 1 ? 0 : NT == 2 ? 1 : 2)) * 3 + EPI) * 2 + HEAD;
-  auto kernel = few_rows_kernel<FKIND, FEW_ROWS_MT, NT, EPI, HEAD>;
+  // attr_set bits 256..282: by operand kind, short-row groups, output mode
+  constexpr int variant = 256 + (FKIND * 3 + (NT == 1 ? 0 : NT == 2 ? 1 : 2)) * 3 + EPI;
+  auto kernel = few_rows_kernel<FKIND, FEW_ROWS_MT, NT, EPI>;
   if (!(s->attr_set[variant >> 6].load(std::memory_order_relaxed) & (1ull << (variant & 63)))) {
     const cudaError_t e = cudaFuncSetAttribute(
         kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FEW_ROWS_SMEM_SM);
@@ -895,14 +889,10 @@ int launch_few_rows(int M, int N, int K, const void* A, size_t a_pitch, const vo
   p.wait_prior_grid = (g_l2_policy & 32) ? 0 : 1;
   const FewRowsShape f = few_rows_shape(p.rows_l, p.rows_s, p.row_bytes, s->num_sms);
   switch (ceil_div(p.rows_s, 8)) {
-    case 1:
-      return f.head ? launch_few_rows_nt<FKIND, 1, EPI, 1>(s, p, f, stream)
-                    : launch_few_rows_nt<FKIND, 1, EPI, 0>(s, p, f, stream);
-    case 2:
-      return f.head ? launch_few_rows_nt<FKIND, 2, EPI, 1>(s, p, f, stream)
-                    : launch_few_rows_nt<FKIND, 2, EPI, 0>(s, p, f, stream);
+    case 1: return launch_few_rows_nt<FKIND, 1, EPI>(s, p, f, stream);
+    case 2: return launch_few_rows_nt<FKIND, 2, EPI>(s, p, f, stream);
     case 3:
-    case 4: return launch_few_rows_nt<FKIND, 4, EPI, 0>(s, p, f, stream);
+    case 4: return launch_few_rows_nt<FKIND, 4, EPI>(s, p, f, stream);
     default: return GEMM_ERR_INVALID_ARG;
   }
 }

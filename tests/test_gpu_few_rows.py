@@ -191,7 +191,7 @@ def test_few_rows_in_a_cuda_graph():
 
 def test_few_rows_seeded_walk_of_shapes():
     """Random short sides (1..32), long sides, K and orientations through every launch shape the
-    host picks (warps 1..16, ring depths 2..8, with and without the step through registers),
+    host picks (warps 1..16, ring depths 2..8),
     each checked against the oracle on sampled rows."""
     g = np.random.Generator(np.random.PCG64(4321))
     shapes_met = set()
@@ -211,7 +211,7 @@ def test_few_rows_seeded_walk_of_shapes():
         cases += 1
         cfg = binding.gemm_query_config(prec, M, N, K)
         assert cfg.startswith("few_rows"), cfg
-        shapes_met.add(tuple(cfg.split(k)[1].split()[0] for k in ("warps=", "depth=", "head=")))
+        shapes_met.add(tuple(cfg.split(k)[1].split()[0] for k in ("warps=", "depth=")))
         A, B = synth.make(prec, M, N, K, seed=int(g.integers(1 << 30)))
         rows = np.unique(np.concatenate([g.choice(M, size=min(10, M), replace=False), [0, M - 1]])).astype(np.int32)
         got = run_gpu(prec, A, B, fill=float("nan") if prec == "fp16" else -7)[rows]
@@ -222,7 +222,7 @@ def test_few_rows_seeded_walk_of_shapes():
         else:
             exact = oracle.gemm_s8_i64(A, B, rows=rows) if prec == "s8" else oracle.gemm_s4_i64(A, B, K, rows=rows)
             assert np.array_equal(got.astype(np.int64), exact), what
-    assert len(shapes_met) >= 12, shapes_met
+    assert len(shapes_met) >= 10, shapes_met
 
 
 def test_few_rows_operands_written_by_the_launch_in_front():
